@@ -1,0 +1,232 @@
+"""Pins for the oracle's pipeline: invariants and special cases of the whole step."""
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+import oracle as O
+from oracle import OracleLGC
+from paper_2103_08870_b200 import workloads as W
+
+TOY = [4096, 64, 1500, 9000, 65, 127, 20000]     # ragged toy layer table
+
+
+def grads(numel, K, steps, seed=5):
+    src = W.GradientSource(W.LayerTable("toy", list(numel), [1] * len(numel)), K, seed=seed)
+    return [src.step(t).numpy() for t in range(steps)]
+
+
+def params(c1, c2, variant, K, seed=3):
+    return W.ae_init_params(c1, c2, variant, K, seed).numpy()
+
+
+def test_layout_counts():
+    o = OracleLGC(TOY, 2)
+    assert o.k_l == [4, 1, 2, 9, 1, 1, 20] and o.mu == 38
+    assert o.ki_l == [1, 1, 1, 1, 1, 1, 2]
+
+
+def test_identity_rar_round_trip_exact():
+    K = 4
+    gs = grads(TOY, K, 3)
+    o = OracleLGC(TOY, K, ae_kind="identity")
+    for t, g in enumerate(gs):
+        o.accumulate(g)
+        v_before = o.v.copy()
+        o.topk(leader=t % K)
+        idx = o.idx[0].copy()
+        assert all(np.array_equal(o.idx[k], idx) for k in range(K))          # shared indices
+        o.encode()
+        o.combine()
+        upd = o.decode_scatter()
+        mean = v_before[:, idx].astype(np.float64).sum(0) / K
+        assert np.array_equal(upd[idx], mean.astype(np.float32))
+        rest = np.ones(o.N, bool)
+        rest[idx] = False
+        assert not upd[rest].any()
+        assert not o.v[:, idx].any() and not o.u[:, idx].any()
+        assert np.array_equal(o.v[:, rest], v_before[:, rest])
+
+
+def test_identity_single_node_update_plus_residual_is_accumulated():
+    gs = grads(TOY, 1, 4)
+    for variant in ("rar", "ps"):
+        o = OracleLGC(TOY, 1, variant=variant, ae_kind="identity", innovation_permille=0)
+        for g in gs:
+            o.accumulate(g)
+            before = o.v[0].copy()
+            o.topk(0)
+            o.encode()
+            o.combine(0)
+            upd = o.decode_scatter()
+            if variant == "rar":
+                assert np.array_equal((upd + o.v[0]).view(np.uint32), before.view(np.uint32))
+
+
+def test_ps_identity_k1_counts_value_twice_only_where_innovation():
+    # K = 1, identity trunk, fusion (1,1,0): reconstruction = value + innovation at kept positions
+    g = grads(TOY, 1, 1)[0]
+    o = OracleLGC(TOY, 1, variant="ps", ae_kind="identity")
+    o.accumulate(g)
+    before = o.v[0].copy()
+    o.topk()
+    o.encode()
+    o.combine(0)
+    upd = o.decode_scatter()
+    idx = o.idx[0]
+    assert np.allclose(upd[idx], before[idx].astype(np.float64) + o.inn[0], rtol=1e-7)
+    assert np.count_nonzero(o.inn[0]) == sum(o.ki_l)
+
+
+def test_k_identical_nodes_mean_is_each_latent():
+    K = 4
+    g1 = grads(TOY, 1, 1)[0]
+    g = np.repeat(g1, K, axis=0)
+    o = OracleLGC(TOY, K, params=params(8, 4, "rar", K))
+    o.accumulate(g)
+    o.topk(2)
+    o.encode()
+    o.combine()
+    assert np.array_equal(o.zbar, o.z[0])          # K a power of two: exact
+
+
+def test_linear_autoencoder_commutes_with_mean():
+    # bias-free and without the ReLU clipping (all pre-activations kept positive by a large
+    # positive first-layer response) the encoder is linear: mean of latents = latent of mean.
+    K, mu = 3, 57
+    rng = np.random.default_rng(1)
+    xs = rng.random((K, mu)) + 0.5                       # positive inputs
+    w1 = np.abs(rng.standard_normal((8, 1, 3)))          # positive weights -> ReLU inactive
+    w2 = rng.standard_normal((4, 8, 3))
+    z = [O.conv1d(O.relu(O.conv1d(x[None], w1, np.zeros(8))), w2, np.zeros(4)) for x in xs]
+    zm = O.conv1d(O.relu(O.conv1d(xs.mean(0)[None], w1, np.zeros(8))), w2, np.zeros(4))
+    assert np.abs(sum(z) / K - zm).max() <= 1e-12 * np.abs(zm).max()
+
+
+def test_rar_forward_equals_torch_modules():
+    K = 3
+    gs = grads(TOY, K, 2)
+    p = params(8, 4, "rar", K)
+    o = OracleLGC(TOY, K, params=p)
+    for t, g in enumerate(gs):
+        o.accumulate(g)
+        o.topk(t)
+        val, idx = o.val.copy(), o.idx[0].copy()
+        o.encode()
+        o.combine()
+        upd = o.decode_scatter()
+    tp = {k: torch.from_numpy(v) for k, v in o.p.items()}
+    x = torch.from_numpy(val.astype(np.float64))[:, None, :]
+    z = F.conv1d(F.relu(F.conv1d(x, tp["enc.w1"], tp["enc.b1"], stride=2)), tp["enc.w2"], tp["enc.b2"], stride=2)
+    zbar = z.mean(0, keepdim=True)
+    d = F.relu(F.conv_transpose1d(zbar, tp["dec.w1"], tp["dec.b1"], stride=2, output_padding=o.op1))
+    r = F.conv_transpose1d(d, tp["dec.w2"], tp["dec.b2"], stride=2, output_padding=o.op2)[0, 0].numpy()
+    assert r.shape == (o.mu,)
+    assert np.abs(upd[idx] - r).max() <= 2e-7 * np.abs(r).max()            # fp32 rounding of the update
+
+
+def test_ps_special_weights():
+    K = 3
+    g = grads(TOY, K, 1)[0]
+    base = params(8, 4, "ps", K)
+
+    def run(w0, w1, b):
+        p = base.copy()
+        o = OracleLGC(TOY, K, variant="ps", params=p)
+        for k in range(K):
+            o.p[f"dec{k}.fuse"][:] = (w0, w1, b)
+        o.accumulate(g)
+        o.topk()
+        o.encode()
+        o.combine(common_node=1)
+        v_sel = [o.v[k, o.idx[k]].copy() for k in range(K)]
+        upd = o.decode_scatter()
+        return o, upd, v_sel
+
+    # (0,1,0): the update is the node-ordered average of the innovations alone
+    o, upd, _ = run(0.0, 1.0, 0.0)
+    ref = np.zeros(o.N)
+    for k in range(K):
+        np.add.at(ref, o.idx[k], o.inn[k].astype(np.float64) / K)
+    assert np.array_equal(upd, ref.astype(np.float32))
+    assert np.count_nonzero(o.inn) == K * sum(o.ki_l)
+    # (1,0,0): every node decodes the common code of node 1 with its own decoder
+    o, upd, _ = run(1.0, 0.0, 0.0)
+    ref = np.zeros(o.N)
+    for k in range(K):
+        d = O.relu(O.convt1d(o.z[1], o.p[f"dec{k}.w1"], o.p[f"dec{k}.b1"], o.op1))
+        y = O.convt1d(d, o.p[f"dec{k}.w2"], o.p[f"dec{k}.b2"], o.op2)[0]
+        np.add.at(ref, o.idx[k], y / K)
+    assert np.allclose(upd, ref.astype(np.float32), rtol=1e-6, atol=1e-12)
+    # per-node index sets differ but overlap (shared heavy-tailed component)
+    s0, s1 = set(o.idx[0].tolist()), set(o.idx[1].tolist())
+    assert s0 != s1 and len(s0 & s1) > 0
+    # every node cleared its own positions
+    for k in range(K):
+        assert not o.v[k, o.idx[k]].any() and not o.u[k, o.idx[k]].any()
+
+
+def test_training_gradients_by_finite_differences():
+    K = 2
+    g = grads(TOY, K, 1)[0] * 1e3                    # O(1) values: well-scaled differences
+    o = OracleLGC(TOY, K, params=params(8, 4, "rar", K, seed=12))
+    o.accumulate(g)
+    o.topk(0)
+    loss, gr = o.ae_loss_and_grads()
+    flat_g = np.concatenate([gr[n].reshape(-1) for n, _ in o.order])
+    flat_p = o.get_params()
+    rng = np.random.default_rng(0)
+    h = 1e-6
+    for j in rng.choice(flat_p.size, 40, replace=False):
+        pp, pm = flat_p.copy(), flat_p.copy()
+        pp[j] += h
+        pm[j] -= h
+        o.set_params(pp)
+        lp = o.ae_loss_and_grads()[0]
+        o.set_params(pm)
+        lm = o.ae_loss_and_grads()[0]
+        fd = (lp - lm) / (2 * h)
+        assert abs(fd - flat_g[j]) <= 1e-6 * max(1.0, abs(flat_g[j])) + 1e-7 * np.abs(flat_g).max(), j
+    o.set_params(flat_p)
+
+
+def test_training_gradients_equal_autograd_and_loss_falls():
+    K = 2
+    g = grads(TOY, K, 1)[0] * 1e3
+    o = OracleLGC(TOY, K, params=params(8, 4, "rar", K, seed=12))
+    o.accumulate(g)
+    o.topk(1)
+    loss, gr = o.ae_loss_and_grads()
+    tp = {k: torch.from_numpy(v.copy()).requires_grad_(True) for k, v in o.p.items()}
+    x = torch.from_numpy(o.val.astype(np.float64))[:, None, :]
+    z = F.conv1d(F.relu(F.conv1d(x, tp["enc.w1"], tp["enc.b1"], stride=2)), tp["enc.w2"], tp["enc.b2"], stride=2)
+    d = F.relu(F.conv_transpose1d(z.mean(0, keepdim=True), tp["dec.w1"], tp["dec.b1"], stride=2, output_padding=o.op1))
+    r = F.conv_transpose1d(d, tp["dec.w2"], tp["dec.b2"], stride=2, output_padding=o.op2)
+    tl = ((r[0, 0] - x[:, 0].mean(0)) ** 2).mean()
+    tl.backward()
+    assert abs(loss - tl.item()) <= 1e-12 * tl.item()
+    for name, _ in o.order:
+        ref = tp[name].grad.numpy()
+        assert np.abs(gr[name] - ref).max() <= 1e-10 * max(1e-3, np.abs(ref).max()), name
+    # zero training steps leave inference untouched; training lowers the loss
+    losses = [o.ae_train_step() for _ in range(50)]
+    assert losses[0] == loss
+    assert losses[-1] < 0.95 * losses[0]
+    assert all(b < a for a, b in zip(losses, losses[1:]))          # falls at every step
+    assert o.adam_t == 50
+
+
+def test_momentum_zero_is_plain_error_feedback():
+    K = 2
+    gs = grads(TOY, K, 3)
+    o = OracleLGC(TOY, K, momentum=0.0, ae_kind="identity")
+    resid = np.zeros((K, o.N), np.float32)
+    for t, g in enumerate(gs):
+        acc = resid + g                               # g_l = grad + g_acc
+        o.accumulate(g)
+        assert np.array_equal(o.v, acc)
+        o.topk(t % K)
+        o.encode(); o.combine(); o.decode_scatter()
+        resid = acc.copy()
+        resid[:, o.idx[0]] = 0                        # only the unsent part stays
+        assert np.array_equal(o.v, resid)
