@@ -1,0 +1,296 @@
+#!/usr/bin/env python
+"""Benchmark of the LGC compression step (accumulate -> top-k -> gather -> encode -> combine ->
+decode -> scatter) on synthetic ResNet-50-shaped gradients, K = 8 simulated nodes per GPU.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line.  metric = dense-gradient GB/s compressed and reconstructed per step
+(K * N * 4 bytes / step time, summed over GPUs).  With --gpus N > 1 (under torchrun) every rank
+runs an independent replica of the workload: the path has no cross-GPU exchange step.
+`--impl reference` times the CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2103_08870_b200 import workloads as W  # noqa: E402
+
+METRIC = "dense_gradient_GBps_compressed_and_reconstructed_per_step"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+GRAD_SETS = 3            # distinct gradient batches cycled through (each far larger than L2)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while a region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def visible_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+def oracle_throughput(w: W.Workload, sample_steps: int, host_grads=None):
+    """The oracle, as it stands, on `sample_steps` whole steps of the workload (host cores).
+    `host_grads`: gradient batches (numpy [K][N]) to cycle through; generated on the CPU if absent."""
+    from oracle import OracleLGC
+    params = W.ae_init_params(w.ae_c1, w.ae_c2, w.variant, w.num_nodes, w.seed).numpy()
+    if host_grads is None:
+        src = W.GradientSource(w.table, w.num_nodes, seed=w.seed)
+        host_grads = [src.step(t).numpy() for t in range(min(GRAD_SETS, sample_steps))]
+    ora = OracleLGC(w.table.numel, w.num_nodes, density_ppm=w.density_ppm, momentum=w.momentum, variant=w.variant,
+                    c1=w.ae_c1, c2=w.ae_c2, params=params, innovation_permille=w.innovation_permille)
+    times = []
+    for t in range(sample_steps):
+        g = host_grads[t % len(host_grads)]
+        t0 = time.perf_counter()
+        ora.step(g, W.choice_for_step(w.seed, t, w.num_nodes))
+        times.append(time.perf_counter() - t0)
+    bytes_per_step = w.num_nodes * w.table.total * 4
+    return bytes_per_step / 1e9 / statistics.mean(times), times
+
+
+def run_reference(args, w: W.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    total = args.steps + args.warmup
+    gbs, times = oracle_throughput(w, total)
+    timed = times[args.warmup:] or times
+    value = w.num_nodes * w.table.total * 4 / 1e9 / statistics.mean(timed)
+    base = {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{len(timed)} whole steps of {w.name} (K={w.num_nodes}, N={w.table.total}), single thread"}
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": len(timed),
+        "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(timed), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(w), "cpu_baseline": base,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(w: W.Workload):
+    return {"workload": f"{w.name}: {len(w.table.numel)} tensors, N={w.table.total}, K={w.num_nodes} nodes per GPU, "
+                        f"density {w.density_ppm} ppm, {w.variant}, AE {w.ae_c1}/{w.ae_c2}",
+            "l2": f"inputs larger than L2: {w.num_nodes * w.table.total * 20 / 1e6:.0f} MB streamed per step, "
+                  f"{GRAD_SETS} gradient batches cycled"}
+
+
+def launches_per_step(gpu) -> int:
+    """Kernels one step enqueues (ring-allreduce): accumulate, selection passes, gather, encode, mean,
+    zero-fill, decode, scatter."""
+    large = sum(1 for n in gpu_layer_numel(gpu) if n > 4096)
+    small = gpu.L - large
+    sel = (1 if small else 0) + (9 if large else 0)
+    return 1 + sel + 1 + 1 + 1 + 1 + 1 + 1
+
+
+def gpu_layer_numel(gpu):
+    return [gpu._numel[i] for i in range(gpu.L)]
+
+
+def run_ours(args, w: W.Workload):
+    from paper_2103_08870_b200 import lgc
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the LGC path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    K, N = w.num_nodes, w.table.total
+    gpu = lgc.LGC(w.table.numel, K, density_ppm=w.density_ppm, momentum=w.momentum, variant=w.variant,
+                  c1=w.ae_c1, c2=w.ae_c2, innovation_permille=w.innovation_permille, device=dev)
+    gpu.set_ae_params(W.ae_init_params(w.ae_c1, w.ae_c2, w.variant, K, w.seed))
+    src = W.GradientSource(w.table, K, seed=w.seed + rank, device=dev)
+    grads = [src.step(t) for t in range(GRAD_SETS)]
+    update = torch.empty(N, dtype=torch.float32, device=dev)
+    choices = [W.choice_for_step(w.seed, t, K) for t in range(args.steps + args.warmup)]
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for t in range(args.warmup):
+        gpu.step(grads[t % GRAD_SETS], update, choices[t])
+    gpu.check()
+    barrier()
+
+    sampler = ClockSampler(visible_gpu_index(local))
+    sampler.start()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for t in range(args.steps):
+        i = args.warmup + t
+        ev[t][0].record()
+        gpu.accumulate(grads[i % GRAD_SETS])
+        ev[t][1].record()
+        gpu.topk(choices[i])
+        gpu.encode()
+        gpu.combine(choices[i])
+        gpu.decode_scatter(update)
+    stop.record()
+    barrier()
+    clocks = sampler.stop()
+    gpu.check()
+    elapsed_ms = start.elapsed_time(stop)
+    acc_ms = [a.elapsed_time(b) for a, b in ev]
+
+    # end to end through host buffers: pinned gradients in, dense update out, every step
+    e2e_steps = max(2, min(args.steps, 5))
+    host_g = torch.empty((K, N), dtype=torch.float32).pin_memory()
+    host_g.copy_(grads[0])
+    host_u = torch.empty(N, dtype=torch.float32).pin_memory()
+    dev_g = torch.empty((K, N), dtype=torch.float32, device=dev)
+    gpu.step_host(host_g, dev_g, update, host_u, choices[0])
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(e2e_steps):
+        gpu.step_host(host_g, dev_g, update, host_u, choices[t])
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    t_all = torch.tensor([elapsed_ms, e2e_ms, statistics.mean(acc_ms)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_all, op=dist.ReduceOp.MAX)
+    elapsed_ms, e2e_ms, acc_mean_ms = t_all.tolist()
+
+    if rank == 0:
+        dense_bytes = K * N * 4 * world
+        value = dense_bytes / 1e9 / (elapsed_ms / 1e3 / args.steps)
+        e2e_value = dense_bytes / 1e9 / (e2e_ms / 1e3 / e2e_steps)
+        peak, peak_kind = measured_peak()
+        acc_bytes = 20 * K * N
+        achieved = acc_bytes / 1e9 / (acc_mean_ms / 1e3)
+        step_bytes = 20 * K * N + 4 * N
+        step_gbs = step_bytes / 1e9 / (elapsed_ms / 1e3 / args.steps)
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": workload_config(w),
+            "roofline": {"bound": "hbm", "kernel": "accumulate_kernel", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                         "traffic": None, "algorithmic_bytes_per_launch": acc_bytes,
+                         "kernel_ms": acc_mean_ms},
+            "step_hbm": {"algorithmic_bytes": step_bytes, "achieved_GBps": step_gbs,
+                         "frac_of_measured_peak": step_gbs / peak, "frac_of_nominal_8TBps": step_gbs / NOMINAL_HBM_GBS},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": K * N * 4, "d2h_bytes_per_step": N * 4,
+                    "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": launches_per_step(gpu) * args.steps,
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            gbs, times = oracle_throughput(w, args.cpu_sample_steps, [g.cpu().numpy() for g in grads])
+            out["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                   "sample": f"{len(times)} whole steps of the same workload, single thread "
+                                             f"({os.cpu_count()} host cores present)",
+                                   "s_per_step": statistics.mean(times)}
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet50", choices=list(W.WORKLOAD_NAMES))
+    ap.add_argument("--cpu-sample-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = W.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

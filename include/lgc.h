@@ -1,0 +1,182 @@
+/*
+ * lgc.h -- C ABI of the Learned Gradient Compression (LGC) per-step path for NVIDIA B200 (sm_100a).
+ *
+ * The library runs, for K data-parallel nodes held as K rows of buffers on ONE device, the
+ * per-iteration compression pipeline of "Learned Gradient Compression for Distributed Deep
+ * Learning" (arXiv 2103.08870): local accumulation with momentum correction, per-layer top-k
+ * magnitude selection, gather, the autoencoder's encoder, the across-node combination of the
+ * codes, the decoder, and the scatter back into a dense update while the sent entries leave the
+ * residual buffers; plus one training step of the autoencoder.
+ *
+ * Conventions common to every entry point
+ *  - Memory.  The caller owns every device byte: `state`, `scratch`, `params`, the gradients and
+ *    the update.  The library allocates no device memory and frees none; `lgc_ctx` is its only
+ *    host allocation (released by lgc_destroy).  Device pointers must be 16-byte aligned.
+ *  - Streams.  All work is enqueued on the stream given in lgc_config.stream (a cudaStream_t,
+ *    NULL = the legacy default stream).  Stage calls never synchronise; lgc_init, lgc_check and
+ *    the host-pointer forms of the parameter accessors do.
+ *  - Errors.  Every call returns an lgc_status; nothing aborts, throws or traps.  Argument and
+ *    call-order errors are detected on the host before anything is enqueued.  Inconsistencies a
+ *    kernel detects are recorded in a device word that lgc_check reads.
+ *  - Layout.  A node's gradient is one flat fp32 vector of N = sum_l n_l elements, layers
+ *    back to back in the order of `layer_numel`; K nodes are K such rows, row stride N.
+ *    Indices are int32 offsets inside a row (N < 2^31); offsets across rows are 64 bit.
+ *  - Call order inside one step:
+ *        lgc_accumulate -> lgc_topk -> lgc_encode -> lgc_combine -> lgc_decode_scatter
+ *    or, while the autoencoder is being trained (second phase of Section V-B):
+ *        lgc_accumulate -> lgc_topk -> [lgc_ae_train_step] -> lgc_topk_scatter
+ *    Any other order returns LGC_ERR_BAD_STATE and enqueues nothing.
+ */
+#ifndef LGC_H
+#define LGC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lgc_ctx lgc_ctx; /* opaque, host side */
+
+typedef enum {
+    LGC_OK = 0,
+    LGC_ERR_INVALID_ARG = 1,  /* null/misaligned pointer, size out of range */
+    LGC_ERR_BAD_STATE = 2,    /* stage called out of order */
+    LGC_ERR_WORKSPACE = 3,    /* a caller buffer is smaller than lgc_workspace_bytes says */
+    LGC_ERR_UNSUPPORTED = 4,  /* configuration outside what the kernels are built for */
+    LGC_ERR_CUDA = 5,         /* a CUDA runtime call failed; see lgc_last_error */
+    LGC_ERR_DEVICE_CHECK = 6, /* a kernel recorded an inconsistency; see lgc_check */
+    LGC_ERR_NO_MEMORY = 7     /* host allocation of the context failed */
+} lgc_status;
+
+typedef enum { LGC_VARIANT_RAR = 0, LGC_VARIANT_PS = 1 } lgc_variant;
+typedef enum { LGC_AE_CONV2 = 0, LGC_AE_IDENTITY = 1 } lgc_ae_kind;
+
+/*
+ * Problem description (Section V: K nodes, L layers, layer l has n_l elements).
+ */
+typedef struct {
+    int32_t num_nodes;            /* K >= 1 */
+    int32_t num_layers;           /* L >= 1 */
+    const int64_t *layer_numel;   /* host array [L], each >= 1, sum N <= 2^31 - 1; copied by lgc_init */
+    uint32_t density_ppm;         /* alpha of Section V-A in parts per million of n_l: 1000 = 0.1 %.
+                                     k_l = clamp(floor((n_l * ppm + 500000) / 10^6), 1, n_l) */
+    uint32_t innovation_permille; /* parameter-server variant: share of a layer's kept values that
+                                     form the innovation (Algorithm 1: 100 = the top tenth);
+                                     kI_l = clamp(floor((k_l * pm + 500) / 1000), 1, k_l) */
+    float momentum;               /* m of the momentum correction (Section V-A); 0 = plain residual */
+    int32_t variant;              /* lgc_variant: ring-allreduce (Algorithm 2) or parameter server (Algorithm 1) */
+    int32_t ae_kind;              /* lgc_ae_kind; IDENTITY passes the kept values through unchanged */
+    int32_t ae_c1, ae_c2;         /* channels of the two encoder convolutions: (8,4) or (16,8) */
+    float adam_lr, adam_beta1, adam_beta2, adam_eps; /* lgc_ae_train_step; 0 selects 1e-3, 0.9, 0.999, 1e-8 */
+    void *stream;                 /* cudaStream_t */
+} lgc_config;
+
+/* Sizes the caller must provide, in bytes.
+ *   state   : velocity u and residual v, 2 * K * N fp32 (Section V-A; zeroed by lgc_init)
+ *   scratch : indices, kept values, codes, selection work space, tables
+ *   params  : autoencoder parameters followed by the two Adam moment vectors (3 * P fp32)
+ * Returns LGC_ERR_INVALID_ARG / LGC_ERR_UNSUPPORTED for a configuration lgc_init would refuse. */
+lgc_status lgc_workspace_bytes(const lgc_config *cfg, size_t *state_bytes, size_t *scratch_bytes,
+                               size_t *params_bytes);
+
+/* Builds the context, uploads the layer tables, zeroes `state`, the Adam moments and the work
+ * space (Algorithm 1/2: the accumulated gradient starts at 0).  Autoencoder parameters are left
+ * as found in `params` (set them with lgc_set_ae_params).  Synchronises the stream.
+ * The three buffers are device memory of at least the sizes lgc_workspace_bytes reports and
+ * must stay valid until lgc_destroy. */
+lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void *scratch,
+                    size_t scratch_bytes, void *params, size_t params_bytes, lgc_ctx **out);
+
+/* Frees the host context.  Touches no device memory.  NULL is allowed. */
+lgc_status lgc_destroy(lgc_ctx *ctx);
+
+/* Stage 1 -- Algorithm 1/2, local accumulation, with the momentum correction of Section V-A:
+ *     u <- m * u + g (one fused rounding);  v <- v + u          for every node and element.
+ * grads: device, fp32 [K][N], read only. */
+lgc_status lgc_accumulate(lgc_ctx *ctx, const float *grads);
+
+/* Stages 2+3 -- Section V-A, Algorithm 1/2 (threshold, mask, concatenation): per layer the k_l
+ * entries of largest |v| (equal magnitudes: the lower index wins), in ascending index order,
+ * layers in order, then the gather of the kept values g~_k in R^mu for every node.
+ * Ring-allreduce: only node `leader` selects and all nodes use its indices.
+ * Parameter server: every node selects on its own; `leader` is ignored. */
+lgc_status lgc_topk(lgc_ctx *ctx, int32_t leader);
+
+/* Stage 4a -- Section IV: g~^c_k = E_c(g~_k) for every node: Conv1d(1->c1, 3 taps, stride 2),
+ * ReLU, Conv1d(c1->c2, 3 taps, stride 2), no padding. */
+lgc_status lgc_encode(lgc_ctx *ctx);
+
+/* Stage 4b -- across-node combination.
+ * Ring-allreduce (Section IV-B / V-B.2): g~^avg = (1/K) sum_k g~^c_k, summed in node order.
+ * Parameter server (Algorithm 1, Section V-B.1): the code of node `common_node` is kept as the
+ * common representation; for every node the innovation g~^I_k keeps, per layer, the kI_l kept
+ * values of largest magnitude (ties: lower position) and zero elsewhere. */
+lgc_status lgc_combine(lgc_ctx *ctx, int32_t common_node);
+
+/* Stage 5 -- Section V-B: decoding, scatter, and removal of the sent entries from u and v.
+ * Ring-allreduce: g~^rec = D_c(g~^avg) (ConvTranspose1d(c2->c1), ReLU, ConvTranspose1d(c1->1),
+ * output padding mirroring the encoder); update[idx[p]] = g~^rec[p], 0 elsewhere.
+ * Parameter server: g~^rec_k = w0_k * D_c^k(g~^c) + w1_k * g~^I_k + b_k (the innovation joins
+ * the decoder output through a 1x1 convolution); update = sum over k, in node order, of
+ * g~^rec_k / K scattered at node k's own indices, 0 elsewhere.
+ * update: device, fp32 [N], fully overwritten. */
+lgc_status lgc_decode_scatter(lgc_ctx *ctx, float *update);
+
+/* Second training phase (Section V-B, weights updated with the top-magnitude gradients): the dense
+ * mean over nodes of the kept values, no autoencoder; sent entries leave u and v.
+ * Valid after lgc_topk (and after lgc_ae_train_step).  update: device, fp32 [N]. */
+lgc_status lgc_topk_scatter(lgc_ctx *ctx, float *update);
+
+/* One training step of the autoencoder on the kept values of the last lgc_topk: ring-allreduce
+ * reconstruction loss of Section IV-B scaled by 1/mu,
+ *     loss = (1/mu) || D_c((1/K) sum_k E_c(g~_k)) - (1/K) sum_k g~_k ||^2,
+ * analytic backward pass, Adam with bias correction.  Ring-allreduce variant with LGC_AE_CONV2
+ * only.  loss_out: device fp32 scalar or NULL.  May be called several times after one lgc_topk. */
+lgc_status lgc_ae_train_step(lgc_ctx *ctx, float *loss_out);
+
+/* A whole compression step from host memory: copies `host_grads` ([K][N], ideally pinned) to
+ * `dev_grads`, runs the five stages, copies the dense update back to `host_update` ([N]).
+ * Everything is enqueued on the context's stream; the call returns without waiting.
+ * `choice` is the leader (ring-allreduce) or the common node (parameter server). */
+lgc_status lgc_step_host(lgc_ctx *ctx, const float *host_grads, float *dev_grads, float *dev_update,
+                         float *host_update, int32_t choice);
+
+/* ---- inspection --------------------------------------------------------------------------- */
+
+/* N, mu, encoder lengths L1 (after the first convolution) and L2 (code length per channel), and
+ * the parameter count P.  Any output pointer may be NULL. */
+lgc_status lgc_get_layout(const lgc_ctx *ctx, int64_t *N, int64_t *mu, int64_t *L1, int64_t *L2,
+                          int64_t *param_count);
+
+/* Host array [L] of k_l, owned by the context. */
+const int64_t *lgc_keep_counts(const lgc_ctx *ctx);
+
+/* Device pointers into the caller's buffers (any may be NULL):
+ *   u, v    [K][N]                     idx   [S][mu] int32, S = 1 (ring-allreduce) or K
+ *   val     [K][mu]                    code  [K][c2][L2] (identity: [K][mu])
+ *   combined[c2][L2] (ring-allreduce: the mean; parameter server: the common code)
+ *   inn     [K][mu] (parameter server) recon [S][mu] */
+lgc_status lgc_get_buffers(const lgc_ctx *ctx, float **u, float **v, int32_t **idx, float **val,
+                           float **code, float **combined, float **inn, float **recon);
+
+/* Autoencoder parameters, flat fp32, tensors in this order (row major):
+ *   enc.w1 [c1][1][3], enc.b1 [c1], enc.w2 [c2][c1][3], enc.b2 [c2],
+ *   then per decoder: w1 [c2][c1][3], b1 [c1], w2 [c1][1][3], b2 [1]
+ * (ring-allreduce: one decoder; parameter server: K decoders, each followed by its fusion
+ * scalars w0, w1, b).  `src`/`dst` may be host or device memory; the copy is synchronous. */
+lgc_status lgc_set_ae_params(lgc_ctx *ctx, const float *src, size_t count);
+lgc_status lgc_get_ae_params(const lgc_ctx *ctx, float *dst, size_t count);
+
+/* Waits for the stream and reports what kernels recorded: LGC_OK or LGC_ERR_DEVICE_CHECK
+ * (code readable through lgc_last_error).  Clears the record. */
+lgc_status lgc_check(lgc_ctx *ctx);
+
+const char *lgc_status_string(lgc_status s);
+const char *lgc_last_error(const lgc_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LGC_H */

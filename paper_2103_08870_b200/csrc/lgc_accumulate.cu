@@ -1,0 +1,125 @@
+// Stage 1 of the LGC step: local accumulation with momentum correction (Algorithm 1/2 of the
+// paper, Section V-A), streamed over all K*N elements of all nodes at once.
+//
+//     u <- m * u + g   (fused, one rounding)        v <- v + u
+//
+// Pure HBM streaming: 12 bytes read and 8 written per element, 128-bit accesses, every byte
+// touched once, so loads and stores carry the streaming (evict-first) hint.
+#include "lgc_internal.cuh"
+
+namespace lgc {
+
+namespace {
+
+constexpr int kAccThreads = 256;
+constexpr int kAccUnroll = 2;   // independent 128-bit triples in flight per thread
+
+__device__ __forceinline__ void acc4(float4 &u, float4 &v, const float4 &g, float m)
+{
+    u.x = __fmaf_rn(m, u.x, g.x); v.x = __fadd_rn(v.x, u.x);
+    u.y = __fmaf_rn(m, u.y, g.y); v.y = __fadd_rn(v.y, u.y);
+    u.z = __fmaf_rn(m, u.z, g.z); v.z = __fadd_rn(v.z, u.z);
+    u.w = __fmaf_rn(m, u.w, g.w); v.w = __fadd_rn(v.w, u.w);
+}
+
+__global__ void __launch_bounds__(kAccThreads)
+accumulate_kernel(const float4 *__restrict__ g4, float4 *__restrict__ u4, float4 *__restrict__ v4,
+                  uint64_t nvec, uint64_t count, float m)
+{
+    const uint64_t stride = (uint64_t)gridDim.x * kAccThreads;
+    uint64_t i = (uint64_t)blockIdx.x * kAccThreads + threadIdx.x;
+    // main loop: kAccUnroll strided vectors per trip, all loads issued before the arithmetic
+    for (; i + (kAccUnroll - 1) * stride < nvec; i += kAccUnroll * stride) {
+        float4 g[kAccUnroll], u[kAccUnroll], v[kAccUnroll];
+#pragma unroll
+        for (int r = 0; r < kAccUnroll; ++r) {
+            g[r] = __ldcs(g4 + i + r * stride);
+            u[r] = __ldcs(u4 + i + r * stride);
+            v[r] = __ldcs(v4 + i + r * stride);
+        }
+#pragma unroll
+        for (int r = 0; r < kAccUnroll; ++r) {
+            acc4(u[r], v[r], g[r], m);
+            __stcs(u4 + i + r * stride, u[r]);
+            __stcs(v4 + i + r * stride, v[r]);
+        }
+    }
+    for (; i < nvec; i += stride) {
+        float4 g = __ldcs(g4 + i), u = __ldcs(u4 + i), v = __ldcs(v4 + i);
+        acc4(u, v, g, m);
+        __stcs(u4 + i, u);
+        __stcs(v4 + i, v);
+    }
+    // up to three trailing scalars
+    if (blockIdx.x == 0 && threadIdx.x < (count & 3)) {
+        const uint64_t j = (nvec << 2) + threadIdx.x;
+        const float *gs = reinterpret_cast<const float *>(g4);
+        float *us = reinterpret_cast<float *>(u4), *vs = reinterpret_cast<float *>(v4);
+        float u = __fmaf_rn(m, us[j], gs[j]);
+        us[j] = u;
+        vs[j] = __fadd_rn(vs[j], u);
+    }
+}
+
+__global__ void __launch_bounds__(256) zero_kernel(uint4 *__restrict__ p, uint64_t nvec)
+{
+    const uint64_t stride = (uint64_t)gridDim.x * 256;
+    for (uint64_t i = (uint64_t)blockIdx.x * 256 + threadIdx.x; i < nvec; i += stride)
+        __stcs(p + i, make_uint4(0u, 0u, 0u, 0u));
+}
+
+__global__ void zero_tail_kernel(unsigned char *p, unsigned n)
+{
+    if (threadIdx.x < n) p[threadIdx.x] = 0;
+}
+
+int sm_count()
+{
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            sms = 148;
+    }
+    return sms;
+}
+
+}  // namespace
+
+cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s)
+{
+    if (count == 0) return cudaSuccess;
+    const uint64_t nvec = count >> 2;
+    uint64_t want = (nvec + kAccThreads * kAccUnroll - 1) / (kAccThreads * kAccUnroll);
+    const uint64_t resident = (uint64_t)sm_count() * 8;   // 8 CTAs of 256 threads per SM
+    if (want > resident) want = resident;
+    if (want == 0) want = 1;
+    accumulate_kernel<<<(unsigned)want, kAccThreads, 0, s>>>(
+        reinterpret_cast<const float4 *>(g), reinterpret_cast<float4 *>(u),
+        reinterpret_cast<float4 *>(v), nvec, count, m);
+    return cudaGetLastError();
+}
+
+// Zero-fill of `bytes` bytes at a 16-byte aligned address.
+cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s)
+{
+    if (bytes == 0) return cudaSuccess;
+    const uint64_t nvec = bytes >> 4;
+    if (nvec) {
+        uint64_t want = (nvec + 255) / 256;
+        const uint64_t cap = (uint64_t)sm_count() * 16;
+        if (want > cap) want = cap;
+        zero_kernel<<<(unsigned)want, 256, 0, s>>>(reinterpret_cast<uint4 *>(p), nvec);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    const unsigned tail = (unsigned)(bytes & 15);
+    if (tail) {
+        zero_tail_kernel<<<1, 16, 0, s>>>(reinterpret_cast<unsigned char *>(p) + (nvec << 4), tail);
+        return cudaGetLastError();
+    }
+    return cudaSuccess;
+}
+
+}  // namespace lgc

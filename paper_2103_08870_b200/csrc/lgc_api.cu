@@ -1,0 +1,492 @@
+// C ABI of liblgc: configuration checks, the carve-up of the caller's buffers, the per-step
+// state machine, and the stage entry points (see include/lgc.h for the contract of each).
+#include <math.h>
+#include <string.h>
+
+#include <new>
+
+#include "lgc_internal.cuh"
+
+struct lgc_ctx : lgc::Ctx {};
+
+namespace lgc {
+namespace {
+
+constexpr size_t kAlign = 256;
+
+// Bump allocator over the caller's scratch; with base == nullptr it only measures.
+struct Carver {
+    char *base;
+    size_t used = 0;
+    explicit Carver(void *b) : base(static_cast<char *>(b)) {}
+    template <typename T>
+    T *take(size_t count)
+    {
+        used = (used + kAlign - 1) / kAlign * kAlign;
+        T *p = base ? reinterpret_cast<T *>(base + used) : nullptr;
+        used += count * sizeof(T);
+        return p;
+    }
+};
+
+struct Plan {
+    int K, L, S;
+    int64_t N, mu, muI, L1, L2, P, Penc, Pdec, code_len;
+    int op1, op2;
+    std::vector<int64_t> numel, off, k_l, koff, ki_l, kioff;
+};
+
+int64_t conv_len(int64_t lin) { return lin >= 3 ? (lin - 3) / 2 + 1 : 0; }
+
+bool ae_channels_supported(int c1, int c2)
+{
+    return (c1 == 8 && c2 == 4) || (c1 == 16 && c2 == 8) || (c1 == 4 && c2 == 2) || (c1 == 3 && c2 == 2);
+}
+
+lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
+{
+    auto fail = [&](lgc_status s, const char *msg) { if (why) *why = msg; return s; };
+    if (!cfg) return fail(LGC_ERR_INVALID_ARG, "config is NULL");
+    if (cfg->num_nodes < 1 || cfg->num_nodes > 65535) return fail(LGC_ERR_INVALID_ARG, "num_nodes must be in [1, 65535]");
+    if (cfg->num_layers < 1 || !cfg->layer_numel) return fail(LGC_ERR_INVALID_ARG, "num_layers < 1 or layer_numel is NULL");
+    if (cfg->density_ppm < 1 || cfg->density_ppm > 1000000) return fail(LGC_ERR_INVALID_ARG, "density_ppm must be in [1, 10^6]");
+    if (cfg->variant != LGC_VARIANT_RAR && cfg->variant != LGC_VARIANT_PS) return fail(LGC_ERR_INVALID_ARG, "unknown variant");
+    if (cfg->ae_kind != LGC_AE_CONV2 && cfg->ae_kind != LGC_AE_IDENTITY) return fail(LGC_ERR_INVALID_ARG, "unknown ae_kind");
+    if (!(cfg->momentum >= 0.0f && cfg->momentum < 1.0f)) return fail(LGC_ERR_INVALID_ARG, "momentum must be in [0, 1)");
+    if (cfg->variant == LGC_VARIANT_PS && cfg->innovation_permille > 1000) return fail(LGC_ERR_INVALID_ARG, "innovation_permille > 1000");
+    p.K = cfg->num_nodes;
+    p.L = cfg->num_layers;
+    p.S = cfg->variant == LGC_VARIANT_PS ? p.K : 1;
+    p.numel.assign(cfg->layer_numel, cfg->layer_numel + p.L);
+    p.off.assign(p.L + 1, 0);
+    p.koff.assign(p.L + 1, 0);
+    p.kioff.assign(p.L + 1, 0);
+    p.k_l.resize(p.L);
+    p.ki_l.resize(p.L);
+    for (int l = 0; l < p.L; ++l) {
+        const int64_t n = p.numel[l];
+        if (n < 1) return fail(LGC_ERR_INVALID_ARG, "a layer has fewer than 1 element");
+        p.off[l + 1] = p.off[l] + n;
+        if (p.off[l + 1] > 2147483647LL) return fail(LGC_ERR_INVALID_ARG, "N exceeds 2^31 - 1");
+        int64_t k = (n * (int64_t)cfg->density_ppm + 500000) / 1000000;
+        k = k < 1 ? 1 : (k > n ? n : k);
+        int64_t ki = (k * (int64_t)cfg->innovation_permille + 500) / 1000;
+        ki = ki < 1 ? 1 : (ki > k ? k : ki);
+        p.k_l[l] = k;
+        p.ki_l[l] = ki;
+        p.koff[l + 1] = p.koff[l] + k;
+        p.kioff[l + 1] = p.kioff[l] + ki;
+    }
+    p.N = p.off[p.L];
+    p.mu = p.koff[p.L];
+    p.muI = p.kioff[p.L];
+    p.L1 = conv_len(p.mu);
+    p.L2 = conv_len(p.L1);
+    p.op1 = p.L1 >= 3 ? (int)((p.L1 - 3) % 2) : 0;
+    p.op2 = p.mu >= 3 ? (int)((p.mu - 3) % 2) : 0;
+    if (cfg->ae_kind == LGC_AE_CONV2) {
+        if (!ae_channels_supported(cfg->ae_c1, cfg->ae_c2))
+            return fail(LGC_ERR_UNSUPPORTED, "autoencoder channels must be (8,4), (16,8), (4,2) or (3,2)");
+        if (p.L2 < 1) return fail(LGC_ERR_UNSUPPORTED, "mu is too short for two stride-2 convolutions (needs mu >= 7)");
+        const int64_t c1 = cfg->ae_c1, c2 = cfg->ae_c2;
+        p.Penc = c1 * 3 + c1 + c2 * c1 * 3 + c2;
+        p.Pdec = c2 * c1 * 3 + c1 + c1 * 3 + 1 + (cfg->variant == LGC_VARIANT_PS ? 3 : 0);
+        p.P = p.Penc + p.Pdec * p.S;
+        p.code_len = c2 * p.L2;
+    } else {
+        p.Penc = p.Pdec = p.P = 0;
+        p.code_len = p.mu;
+    }
+    return LGC_OK;
+}
+
+void carve_select(Carver &cv, SelectTables &t, int num_segments, int num_small, int num_large, int num_chunks, int rows)
+{
+    t.num_segments = num_segments; t.num_small = num_small; t.num_large = num_large; t.num_chunks = num_chunks;
+    t.max_rows = rows;
+    t.seg_off = cv.take<int64_t>(num_segments);
+    t.seg_len = cv.take<int32_t>(num_segments);
+    t.seg_k = cv.take<int32_t>(num_segments);
+    t.seg_out = cv.take<int32_t>(num_segments);
+    t.small_ids = cv.take<int32_t>(num_small);
+    t.large_ids = cv.take<int32_t>(num_large);
+    t.large_chunk0 = cv.take<int32_t>(num_large + 1);
+    t.chunk_large = cv.take<int32_t>(num_chunks);
+    t.hist = cv.take<uint32_t>((size_t)rows * num_large * kHistBins);
+    t.prefix = cv.take<uint32_t>((size_t)rows * num_large);
+    t.k_rem = cv.take<int32_t>((size_t)rows * num_large);
+    t.chunk_cnt = cv.take<int2>((size_t)rows * num_chunks);
+}
+
+void count_segments(const std::vector<int64_t> &len, int &small, int &large, int &chunks)
+{
+    small = large = chunks = 0;
+    for (int64_t n : len) {
+        if (n <= kSelChunk) ++small;
+        else { ++large; chunks += (int)((n + kSelChunk - 1) / kSelChunk); }
+    }
+}
+
+// Lays every sub-buffer of the scratch out; identical for measuring and for real.
+void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
+{
+    const bool ps = cfg.variant == LGC_VARIANT_PS;
+    const bool conv = cfg.ae_kind == LGC_AE_CONV2;
+    c.errword = cv.take<int32_t>(4);
+    c.idx = cv.take<int32_t>((size_t)p.S * p.mu);
+    c.val = cv.take<float>((size_t)p.K * p.mu);
+    c.code = conv ? cv.take<float>((size_t)p.K * p.code_len) : nullptr;
+    c.combined = cv.take<float>((size_t)p.code_len);
+    c.recon = cv.take<float>((size_t)p.S * p.mu);
+    c.slot_layer = cv.take<int32_t>((size_t)p.mu);
+    c.koff_dev = cv.take<int32_t>((size_t)p.L + 1);
+    int sm, lg, ch;
+    count_segments(p.numel, sm, lg, ch);
+    carve_select(cv, c.sel_v, p.L, sm, lg, ch, p.S);
+    if (ps) {
+        c.inn = cv.take<float>((size_t)p.K * p.mu);
+        c.inn_pos = cv.take<int32_t>((size_t)p.K * p.muI);
+        count_segments(p.k_l, sm, lg, ch);
+        carve_select(cv, c.sel_inn, p.L, sm, lg, ch, p.K);
+    }
+    if (conv && !ps) {
+        const size_t c1 = cfg.ae_c1, c2 = cfg.ae_c2;
+        c.t_h = cv.take<float>((size_t)p.K * c1 * p.L1);
+        c.t_dh = cv.take<float>((size_t)p.K * c1 * p.L1);
+        c.t_d = cv.take<float>(c1 * p.L1);
+        c.t_dd = cv.take<float>(c1 * p.L1);
+        c.t_dr = cv.take<float>((size_t)p.mu);
+        c.t_dz = cv.take<float>(c2 * p.L2);
+        c.t_loss_blocks = (int)((p.mu + 127) / 128);
+        c.t_loss_part = cv.take<double>((size_t)c.t_loss_blocks);
+    }
+    cv.take<char>(0);
+}
+
+lgc_status fail(lgc_ctx *ctx, lgc_status s, const std::string &msg)
+{
+    if (ctx) ctx->err = msg;
+    return s;
+}
+
+lgc_status cuda_fail(lgc_ctx *ctx, cudaError_t e, const char *where)
+{
+    return fail(ctx, LGC_ERR_CUDA, std::string(where) + ": " + cudaGetErrorString(e));
+}
+
+template <typename T>
+cudaError_t upload(T *dst, const std::vector<T> &src, cudaStream_t s)
+{
+    if (src.empty()) return cudaSuccess;
+    return cudaMemcpyAsync(dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice, s);
+}
+
+// Fills and uploads the tables of one selection family; `hold` keeps the host copies alive until
+// the stream has been synchronised.
+cudaError_t upload_select(SelectTables &t, const std::vector<int64_t> &off, const std::vector<int64_t> &len,
+                          const std::vector<int64_t> &k, const std::vector<int64_t> &out_off, cudaStream_t s,
+                          std::vector<std::vector<int32_t>> &hold32, std::vector<std::vector<int64_t>> &hold64)
+{
+    const int n = (int)len.size();
+    std::vector<int64_t> h_off(off.begin(), off.begin() + n);
+    std::vector<int32_t> h_len(n), h_k(n), h_out(n), small_ids, large_ids, chunk0, chunk_large;
+    chunk0.push_back(0);
+    for (int i = 0; i < n; ++i) {
+        h_len[i] = (int32_t)len[i];
+        h_k[i] = (int32_t)k[i];
+        h_out[i] = (int32_t)out_off[i];
+        if (len[i] <= kSelChunk) small_ids.push_back(i);
+        else {
+            const int li = (int)large_ids.size();
+            large_ids.push_back(i);
+            const int nc = (int)((len[i] + kSelChunk - 1) / kSelChunk);
+            for (int q = 0; q < nc; ++q) chunk_large.push_back(li);
+            chunk0.push_back(chunk0.back() + nc);
+        }
+    }
+    hold64.push_back(std::move(h_off));
+    cudaError_t e = upload(t.seg_off, hold64.back(), s);
+    std::vector<int32_t> *arrs[] = {&h_len, &h_k, &h_out, &small_ids, &large_ids, &chunk0, &chunk_large};
+    int32_t *dsts[] = {t.seg_len, t.seg_k, t.seg_out, t.small_ids, t.large_ids, t.large_chunk0, t.chunk_large};
+    for (int i = 0; i < 7 && e == cudaSuccess; ++i) {
+        hold32.push_back(std::move(*arrs[i]));
+        e = upload(dsts[i], hold32.back(), s);
+    }
+    return e;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+}  // namespace lgc
+
+using namespace lgc;
+
+extern "C" {
+
+lgc_status lgc_workspace_bytes(const lgc_config *cfg, size_t *state_bytes, size_t *scratch_bytes, size_t *params_bytes)
+{
+    Plan p;
+    const lgc_status st = make_plan(cfg, p, nullptr);
+    if (st != LGC_OK) return st;
+    Ctx tmp;
+    Carver cv(nullptr);
+    carve(cv, tmp, p, *cfg);
+    if (state_bytes) *state_bytes = (size_t)2 * p.K * p.N * sizeof(float);
+    if (scratch_bytes) *scratch_bytes = (cv.used + kAlign - 1) / kAlign * kAlign;
+    if (params_bytes) *params_bytes = (size_t)(p.P > 0 ? 3 * p.P : 4) * sizeof(float);
+    return LGC_OK;
+}
+
+lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void *scratch, size_t scratch_bytes,
+                    void *params, size_t params_bytes, lgc_ctx **out)
+{
+    if (!out) return LGC_ERR_INVALID_ARG;
+    *out = nullptr;
+    Plan p;
+    lgc_status st = make_plan(cfg, p, nullptr);
+    if (st != LGC_OK) return st;
+    size_t need_state, need_scratch, need_params;
+    lgc_workspace_bytes(cfg, &need_state, &need_scratch, &need_params);
+    if (!state || !scratch || !params || !aligned16(state) || !aligned16(scratch) || !aligned16(params))
+        return LGC_ERR_INVALID_ARG;
+    if (state_bytes < need_state || scratch_bytes < need_scratch || params_bytes < need_params) return LGC_ERR_WORKSPACE;
+
+    lgc_ctx *c = new (std::nothrow) lgc_ctx();
+    if (!c) return LGC_ERR_NO_MEMORY;
+    c->cfg = *cfg;
+    c->cfg.layer_numel = nullptr;
+    c->stream = static_cast<cudaStream_t>(cfg->stream);
+    c->K = p.K; c->L = p.L; c->S = p.S; c->N = p.N; c->mu = p.mu; c->muI = p.muI; c->L1 = p.L1; c->L2 = p.L2;
+    c->P = p.P; c->Penc = p.Penc; c->Pdec = p.Pdec; c->op1 = p.op1; c->op2 = p.op2; c->code_len = p.code_len;
+    c->numel = p.numel; c->off = p.off; c->k_l = p.k_l; c->koff = p.koff; c->ki_l = p.ki_l; c->kioff = p.kioff;
+    c->lr = cfg->adam_lr != 0.0f ? (double)cfg->adam_lr : 1e-3;
+    c->beta1 = cfg->adam_beta1 != 0.0f ? (double)cfg->adam_beta1 : 0.9;
+    c->beta2 = cfg->adam_beta2 != 0.0f ? (double)cfg->adam_beta2 : 0.999;
+    c->eps = cfg->adam_eps != 0.0f ? (double)cfg->adam_eps : 1e-8;
+    c->u = static_cast<float *>(state);
+    c->v = c->u + (size_t)p.K * p.N;
+    c->params = static_cast<float *>(params);
+    c->adam_m = c->params + p.P;
+    c->adam_v = c->adam_m + p.P;
+    Carver cv(scratch);
+    carve(cv, *c, p, *cfg);
+    if (cfg->ae_kind == LGC_AE_IDENTITY) c->code = c->val;
+
+    cudaStream_t s = c->stream;
+    cudaError_t e = launch_zero(state, need_state, s);
+    if (e == cudaSuccess) e = launch_zero(scratch, need_scratch, s);
+    if (e == cudaSuccess && p.P > 0) e = launch_zero(c->adam_m, (size_t)2 * p.P * sizeof(float), s);
+    std::vector<std::vector<int32_t>> hold32;
+    std::vector<std::vector<int64_t>> hold64;
+    hold32.reserve(32);
+    hold64.reserve(4);
+    if (e == cudaSuccess) e = upload_select(c->sel_v, p.off, p.numel, p.k_l, p.koff, s, hold32, hold64);
+    if (e == cudaSuccess && cfg->variant == LGC_VARIANT_PS)
+        e = upload_select(c->sel_inn, p.koff, p.k_l, p.ki_l, p.kioff, s, hold32, hold64);
+    std::vector<int32_t> slot_layer((size_t)p.mu), koff32((size_t)p.L + 1);
+    for (int l = 0; l < p.L; ++l) {
+        koff32[l] = (int32_t)p.koff[l];
+        for (int64_t q = p.koff[l]; q < p.koff[l + 1]; ++q) slot_layer[(size_t)q] = l;
+    }
+    koff32[p.L] = (int32_t)p.mu;
+    if (e == cudaSuccess) e = upload(c->slot_layer, slot_layer, s);
+    if (e == cudaSuccess) e = upload(c->koff_dev, koff32, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        delete c;
+        return LGC_ERR_CUDA;
+    }
+    *out = c;
+    return LGC_OK;
+}
+
+lgc_status lgc_destroy(lgc_ctx *ctx)
+{
+    delete ctx;
+    return LGC_OK;
+}
+
+lgc_status lgc_accumulate(lgc_ctx *c, const float *grads)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (!grads || !aligned16(grads)) return fail(c, LGC_ERR_INVALID_ARG, "grads is NULL or not 16-byte aligned");
+    if (c->stage != Ctx::kIdle) return fail(c, LGC_ERR_BAD_STATE, "lgc_accumulate must open a step");
+    const cudaError_t e = launch_accumulate(grads, c->u, c->v, (uint64_t)c->K * (uint64_t)c->N, c->cfg.momentum, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_accumulate");
+    c->stage = Ctx::kAccumulated;
+    return LGC_OK;
+}
+
+lgc_status lgc_topk(lgc_ctx *c, int32_t leader)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (c->stage != Ctx::kAccumulated) return fail(c, LGC_ERR_BAD_STATE, "lgc_topk must follow lgc_accumulate");
+    const bool ps = c->cfg.variant == LGC_VARIANT_PS;
+    if (!ps && (leader < 0 || leader >= c->K)) return fail(c, LGC_ERR_INVALID_ARG, "leader out of range");
+    cudaError_t e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, c->errword, c->stream);
+    if (e == cudaSuccess) e = launch_gather(*c);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_topk");
+    c->last_leader = leader;
+    c->stage = Ctx::kSelected;
+    return LGC_OK;
+}
+
+lgc_status lgc_encode(lgc_ctx *c)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (c->stage != Ctx::kSelected) return fail(c, LGC_ERR_BAD_STATE, "lgc_encode must follow lgc_topk");
+    const cudaError_t e = launch_encode(*c);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_encode");
+    c->stage = Ctx::kEncoded;
+    return LGC_OK;
+}
+
+lgc_status lgc_combine(lgc_ctx *c, int32_t common_node)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (c->stage != Ctx::kEncoded) return fail(c, LGC_ERR_BAD_STATE, "lgc_combine must follow lgc_encode");
+    cudaError_t e;
+    if (c->cfg.variant == LGC_VARIANT_PS) {
+        if (common_node < 0 || common_node >= c->K) return fail(c, LGC_ERR_INVALID_ARG, "common_node out of range");
+        e = launch_combine_ps(*c, common_node);
+    } else {
+        e = launch_combine_mean(*c);
+    }
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_combine");
+    c->stage = Ctx::kCombined;
+    return LGC_OK;
+}
+
+lgc_status lgc_decode_scatter(lgc_ctx *c, float *update)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (!update || !aligned16(update)) return fail(c, LGC_ERR_INVALID_ARG, "update is NULL or not 16-byte aligned");
+    if (c->stage != Ctx::kCombined) return fail(c, LGC_ERR_BAD_STATE, "lgc_decode_scatter must follow lgc_combine");
+    const cudaError_t e = launch_decode_scatter(*c, update);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_decode_scatter");
+    c->stage = Ctx::kIdle;
+    return LGC_OK;
+}
+
+lgc_status lgc_topk_scatter(lgc_ctx *c, float *update)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (!update || !aligned16(update)) return fail(c, LGC_ERR_INVALID_ARG, "update is NULL or not 16-byte aligned");
+    if (c->stage != Ctx::kSelected) return fail(c, LGC_ERR_BAD_STATE, "lgc_topk_scatter must follow lgc_topk");
+    const cudaError_t e = launch_topk_scatter(*c, update);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_topk_scatter");
+    c->stage = Ctx::kIdle;
+    return LGC_OK;
+}
+
+lgc_status lgc_ae_train_step(lgc_ctx *c, float *loss_out)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (c->cfg.variant != LGC_VARIANT_RAR || c->cfg.ae_kind != LGC_AE_CONV2)
+        return fail(c, LGC_ERR_UNSUPPORTED, "training is built for the ring-allreduce convolutional autoencoder");
+    if (c->stage != Ctx::kSelected) return fail(c, LGC_ERR_BAD_STATE, "lgc_ae_train_step must follow lgc_topk");
+    const cudaError_t e = launch_train_step(*c, loss_out);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_ae_train_step");
+    return LGC_OK;
+}
+
+lgc_status lgc_step_host(lgc_ctx *c, const float *host_grads, float *dev_grads, float *dev_update, float *host_update,
+                         int32_t choice)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (!host_grads || !dev_grads || !dev_update || !host_update) return fail(c, LGC_ERR_INVALID_ARG, "NULL buffer");
+    if (c->stage != Ctx::kIdle) return fail(c, LGC_ERR_BAD_STATE, "lgc_step_host must open a step");
+    cudaError_t e = cudaMemcpyAsync(dev_grads, host_grads, (size_t)c->K * c->N * sizeof(float), cudaMemcpyHostToDevice, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (upload)");
+    lgc_status st = lgc_accumulate(c, dev_grads);
+    if (st == LGC_OK) st = lgc_topk(c, choice);
+    if (st == LGC_OK) st = lgc_encode(c);
+    if (st == LGC_OK) st = lgc_combine(c, choice);
+    if (st == LGC_OK) st = lgc_decode_scatter(c, dev_update);
+    if (st != LGC_OK) return st;
+    e = cudaMemcpyAsync(host_update, dev_update, (size_t)c->N * sizeof(float), cudaMemcpyDeviceToHost, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (download)");
+    return LGC_OK;
+}
+
+lgc_status lgc_get_layout(const lgc_ctx *c, int64_t *N, int64_t *mu, int64_t *L1, int64_t *L2, int64_t *param_count)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (N) *N = c->N;
+    if (mu) *mu = c->mu;
+    if (L1) *L1 = c->L1;
+    if (L2) *L2 = c->L2;
+    if (param_count) *param_count = c->P;
+    return LGC_OK;
+}
+
+const int64_t *lgc_keep_counts(const lgc_ctx *c) { return c ? c->k_l.data() : nullptr; }
+
+lgc_status lgc_get_buffers(const lgc_ctx *c, float **u, float **v, int32_t **idx, float **val, float **code,
+                           float **combined, float **inn, float **recon)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (u) *u = c->u;
+    if (v) *v = c->v;
+    if (idx) *idx = c->idx;
+    if (val) *val = c->val;
+    if (code) *code = c->code;
+    if (combined) *combined = c->combined;
+    if (inn) *inn = c->inn;
+    if (recon) *recon = c->recon;
+    return LGC_OK;
+}
+
+lgc_status lgc_set_ae_params(lgc_ctx *c, const float *src, size_t count)
+{
+    if (!c || !src) return LGC_ERR_INVALID_ARG;
+    if ((int64_t)count != c->P) return fail(c, LGC_ERR_INVALID_ARG, "parameter count does not match the configuration");
+    if (count == 0) return LGC_OK;
+    cudaError_t e = cudaMemcpyAsync(c->params, src, count * sizeof(float), cudaMemcpyDefault, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    return e == cudaSuccess ? LGC_OK : cuda_fail(c, e, "lgc_set_ae_params");
+}
+
+lgc_status lgc_get_ae_params(const lgc_ctx *c, float *dst, size_t count)
+{
+    if (!c || !dst) return LGC_ERR_INVALID_ARG;
+    if ((int64_t)count != c->P) return LGC_ERR_INVALID_ARG;
+    if (count == 0) return LGC_OK;
+    cudaError_t e = cudaMemcpyAsync(dst, c->params, count * sizeof(float), cudaMemcpyDefault, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    return e == cudaSuccess ? LGC_OK : LGC_ERR_CUDA;
+}
+
+lgc_status lgc_check(lgc_ctx *c)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    int32_t word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, c->errword, sizeof word, cudaMemcpyDeviceToHost, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_check");
+    if (word == 0) return LGC_OK;
+    launch_zero(c->errword, 16, c->stream);
+    char buf[96];
+    snprintf(buf, sizeof buf, "device check 0x%X: a selection kernel found inconsistent counts", (unsigned)word);
+    return fail(c, LGC_ERR_DEVICE_CHECK, buf);
+}
+
+const char *lgc_status_string(lgc_status s)
+{
+    switch (s) {
+    case LGC_OK: return "LGC_OK";
+    case LGC_ERR_INVALID_ARG: return "LGC_ERR_INVALID_ARG";
+    case LGC_ERR_BAD_STATE: return "LGC_ERR_BAD_STATE";
+    case LGC_ERR_WORKSPACE: return "LGC_ERR_WORKSPACE";
+    case LGC_ERR_UNSUPPORTED: return "LGC_ERR_UNSUPPORTED";
+    case LGC_ERR_CUDA: return "LGC_ERR_CUDA";
+    case LGC_ERR_DEVICE_CHECK: return "LGC_ERR_DEVICE_CHECK";
+    case LGC_ERR_NO_MEMORY: return "LGC_ERR_NO_MEMORY";
+    }
+    return "LGC_ERR_UNKNOWN";
+}
+
+const char *lgc_last_error(const lgc_ctx *c) { return c ? c->err.c_str() : "context is NULL"; }
+
+}  // extern "C"

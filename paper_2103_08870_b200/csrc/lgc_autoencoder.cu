@@ -1,0 +1,306 @@
+// Stages 3-5 of the LGC step: gather of the kept values, the lightweight autoencoder (Section IV
+// of the paper, two strided 1-D convolutions each way), the across-node combination of the codes
+// (ring-allreduce: mean, Section IV-B; parameter server: common code + innovation, Algorithm 1),
+// decoding, and the scatter into the dense update with the removal of sent entries from u and v.
+//
+// Everything here works on mu ~ N/1000 values: the kernels are latency bound, so each fuses what
+// it can (both convolutions of a side in one kernel, decode + scatter + clearing in one kernel)
+// and keeps the handful of weights in shared memory.  fp32 FMA arithmetic, no tensor cores: the
+// largest contraction is a 48-term dot product.
+#include "lgc_internal.cuh"
+
+namespace lgc {
+
+namespace {
+
+constexpr int kAeThreads = 128;
+
+__global__ void gather_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restrict__ idx,
+                              int S, int64_t mu, float *__restrict__ val)
+{
+    const int k = blockIdx.y;
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= mu) return;
+    const int32_t i = idx[(S == 1 ? 0 : (int64_t)k * mu) + p];
+    val[(int64_t)k * mu + p] = v[(int64_t)k * N + i];
+}
+
+// code[k][co][t] = b2[co] + sum_{ci,tau} w2[co][ci][tau] * relu(b1[ci] + sum_tau' w1[ci][tau'] x[2(2t+tau)+tau'])
+template <int C1, int C2>
+__global__ void __launch_bounds__(kAeThreads)
+encode_kernel(const float *__restrict__ val, int64_t mu, int64_t L2, const float *__restrict__ params,
+              float *__restrict__ code)
+{
+    constexpr int kEnc = C1 * 3 + C1 + C2 * C1 * 3 + C2;
+    __shared__ float w[kEnc];
+    for (int i = threadIdx.x; i < kEnc; i += kAeThreads) w[i] = params[i];
+    __syncthreads();
+    const float *w1 = w, *b1 = w + C1 * 3, *w2 = b1 + C1, *b2 = w2 + C2 * C1 * 3;
+    const int k = blockIdx.y;
+    const int64_t t = (int64_t)blockIdx.x * kAeThreads + threadIdx.x;
+    if (t >= L2) return;
+    const float *x = val + (int64_t)k * mu + 4 * t;
+    float xin[7];
+#pragma unroll
+    for (int i = 0; i < 7; ++i) xin[i] = x[i];
+    float h[3][C1];
+#pragma unroll
+    for (int ci = 0; ci < C1; ++ci)
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+            float a = b1[ci];
+#pragma unroll
+            for (int tau = 0; tau < 3; ++tau) a = __fmaf_rn(w1[ci * 3 + tau], xin[2 * j + tau], a);
+            h[j][ci] = fmaxf(a, 0.0f);
+        }
+#pragma unroll
+    for (int co = 0; co < C2; ++co) {
+        float a = b2[co];
+#pragma unroll
+        for (int ci = 0; ci < C1; ++ci)
+#pragma unroll
+            for (int tau = 0; tau < 3; ++tau) a = __fmaf_rn(w2[(co * C1 + ci) * 3 + tau], h[tau][ci], a);
+        code[((int64_t)k * C2 + co) * L2 + t] = a;
+    }
+}
+
+// out[i] = (rows[0][i] + rows[1][i] + ... + rows[K-1][i]) / K, summed in node order
+__global__ void mean_rows_kernel(const float *__restrict__ rows, int K, int64_t len, float *__restrict__ out)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= len) return;
+    float a = rows[i];
+    for (int k = 1; k < K; ++k) a = __fadd_rn(a, rows[(int64_t)k * len + i]);
+    out[i] = __fdiv_rn(a, (float)K);
+}
+
+__global__ void copy_kernel(const float *__restrict__ src, int64_t len, float *__restrict__ dst)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < len) dst[i] = src[i];
+}
+
+// inn[k][pos] = val[k][pos] at the selected positions (inn was zeroed before)
+__global__ void innovation_fill_kernel(const float *__restrict__ val, const int32_t *__restrict__ pos,
+                                       int64_t mu, int64_t muI, float *__restrict__ inn)
+{
+    const int k = blockIdx.y;
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= muI) return;
+    const int32_t p = pos[(int64_t)k * muI + q];
+    inn[(int64_t)k * mu + p] = val[(int64_t)k * mu + p];
+}
+
+// Decoder output at position p for the code z[C2][L2]:
+//   d[ci][i] = relu(b1[ci] + sum_{c2, (j,tau'): 2j+tau' = i} w1[c2][ci][tau'] z[c2][j]),   i < L1
+//   y[p]     = b2 + sum_{ci, (i,tau): 2i+tau = p} w2[ci][tau] d[ci][i]
+template <int C1, int C2>
+__device__ __forceinline__ float decode_at(int64_t p, const float *__restrict__ z, int64_t L1, int64_t L2,
+                                           const float *w1, const float *b1, const float *w2, float b2)
+{
+    float y = b2;
+    for (int tau = (int)(p & 1); tau < 3; tau += 2) {
+        const int64_t i = (p - tau) >> 1;
+        if (p < tau || i >= L1) continue;
+        float d[C1];
+#pragma unroll
+        for (int ci = 0; ci < C1; ++ci) d[ci] = b1[ci];
+        for (int tq = (int)(i & 1); tq < 3; tq += 2) {
+            const int64_t j = (i - tq) >> 1;
+            if (i < tq || j >= L2) continue;
+#pragma unroll
+            for (int c2 = 0; c2 < C2; ++c2) {
+                const float zz = z[(int64_t)c2 * L2 + j];
+#pragma unroll
+                for (int ci = 0; ci < C1; ++ci) d[ci] = __fmaf_rn(w1[(c2 * C1 + ci) * 3 + tq], zz, d[ci]);
+            }
+        }
+#pragma unroll
+        for (int ci = 0; ci < C1; ++ci) y = __fmaf_rn(w2[ci * 3 + tau], fmaxf(d[ci], 0.0f), y);
+    }
+    return y;
+}
+
+// One row of reconstructions per decoder: ring-allreduce has one decoder and no innovation;
+// the parameter server has one decoder per node and fuses the innovation with (w0, w1, b).
+template <int C1, int C2, bool PS>
+__global__ void __launch_bounds__(kAeThreads)
+decode_kernel(const float *__restrict__ z, int64_t mu, int64_t L1, int64_t L2,
+              const float *__restrict__ dec_params, int dec_stride, const float *__restrict__ inn,
+              float *__restrict__ recon)
+{
+    constexpr int kDec = C2 * C1 * 3 + C1 + C1 * 3 + 1 + (PS ? 3 : 0);
+    __shared__ float w[kDec];
+    const int s = blockIdx.y;
+    for (int i = threadIdx.x; i < kDec; i += kAeThreads) w[i] = dec_params[(int64_t)s * dec_stride + i];
+    __syncthreads();
+    const float *w1 = w, *b1 = w + C2 * C1 * 3, *w2 = b1 + C1;
+    const int64_t p = (int64_t)blockIdx.x * kAeThreads + threadIdx.x;
+    if (p >= mu) return;
+    float y = decode_at<C1, C2>(p, z, L1, L2, w1, b1, w2, w2[C1 * 3]);
+    if (PS) {
+        const float *f = w2 + C1 * 3 + 1;
+        y = __fmaf_rn(f[1], inn[(int64_t)s * mu + p], __fmaf_rn(f[0], y, f[2]));
+    }
+    recon[(int64_t)s * mu + p] = y;
+}
+
+// identity autoencoder, parameter server: recon_k = code + innovation_k
+__global__ void identity_ps_kernel(const float *__restrict__ z, const float *__restrict__ inn, int64_t mu,
+                                   float *__restrict__ recon)
+{
+    const int k = blockIdx.y;
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < mu) recon[(int64_t)k * mu + p] = __fadd_rn(z[p], inn[(int64_t)k * mu + p]);
+}
+
+// Ring-allreduce scatter: one index set for all nodes; the sent entries leave every node's u, v.
+__global__ void scatter_shared_kernel(const float *__restrict__ values, const int32_t *__restrict__ idx,
+                                      int64_t mu, int K, int64_t N, float *__restrict__ update,
+                                      float *__restrict__ u, float *__restrict__ v)
+{
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= mu) return;
+    const int32_t i = idx[p];
+    update[i] = values[p];
+    for (int k = 0; k < K; ++k) {
+        u[(int64_t)k * N + i] = 0.0f;
+        v[(int64_t)k * N + i] = 0.0f;
+    }
+}
+
+__device__ __forceinline__ int64_t find_in(const int32_t *__restrict__ a, int64_t lo, int64_t hi, int32_t x)
+{
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (a[mid] < x) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// Parameter-server scatter: update[i] = sum over nodes k (ascending) that kept i of values_k / K.
+// The lowest node holding an index sums for all of them, so the order of additions is fixed and
+// no atomics are needed.  Each node's own sent entries leave its u and v.
+__global__ void scatter_own_kernel(const float *__restrict__ values, const int32_t *__restrict__ idx,
+                                   const int32_t *__restrict__ slot_layer, const int32_t *__restrict__ koff,
+                                   int64_t mu, int K, int64_t N, float *__restrict__ update,
+                                   float *__restrict__ u, float *__restrict__ v)
+{
+    const int k = blockIdx.y;
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= mu) return;
+    const int32_t i = idx[(int64_t)k * mu + p];
+    u[(int64_t)k * N + i] = 0.0f;
+    v[(int64_t)k * N + i] = 0.0f;
+    const int l = slot_layer[p];
+    const int64_t lo = koff[l], hi = koff[l + 1];
+    for (int kk = 0; kk < k; ++kk) {
+        const int32_t *row = idx + (int64_t)kk * mu;
+        const int64_t q = find_in(row, lo, hi, i);
+        if (q < hi && row[q] == i) return;      // a lower node owns this index
+    }
+    const float fk = (float)K;
+    float acc = __fadd_rn(0.0f, __fdiv_rn(values[(int64_t)k * mu + p], fk));
+    for (int kk = k + 1; kk < K; ++kk) {
+        const int32_t *row = idx + (int64_t)kk * mu;
+        const int64_t q = find_in(row, lo, hi, i);
+        if (q < hi && row[q] == i) acc = __fadd_rn(acc, __fdiv_rn(values[(int64_t)kk * mu + q], fk));
+    }
+    update[i] = acc;
+}
+
+inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)((n + threads - 1) / threads); }
+
+#define LGC_DISPATCH_AE(c1, c2, CALL)                                   \
+    if ((c1) == 8 && (c2) == 4) { CALL(8, 4); }                         \
+    else if ((c1) == 16 && (c2) == 8) { CALL(16, 8); }                  \
+    else if ((c1) == 4 && (c2) == 2) { CALL(4, 2); }                    \
+    else if ((c1) == 3 && (c2) == 2) { CALL(3, 2); }                    \
+    else return cudaErrorInvalidValue;
+
+}  // namespace
+
+cudaError_t launch_gather(const Ctx &c)
+{
+    gather_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S, c.mu, c.val);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_encode(const Ctx &c)
+{
+    if (c.cfg.ae_kind == LGC_AE_IDENTITY) return cudaSuccess;   // the code is the kept values themselves
+    const dim3 grid(blocks_for(c.L2, kAeThreads), c.K);
+#define CALL(A, B) encode_kernel<A, B><<<grid, kAeThreads, 0, c.stream>>>(c.val, c.mu, c.L2, c.params, c.code)
+    LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
+#undef CALL
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine_mean(const Ctx &c)
+{
+    mean_rows_kernel<<<blocks_for(c.code_len, 256), 256, 0, c.stream>>>(c.code, c.K, c.code_len, c.combined);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine_ps(Ctx &c, int common_node)
+{
+    copy_kernel<<<blocks_for(c.code_len, 256), 256, 0, c.stream>>>(c.code + (int64_t)common_node * c.code_len,
+                                                                   c.code_len, c.combined);
+    cudaError_t e = launch_zero(c.inn, (size_t)c.K * c.mu * sizeof(float), c.stream);
+    if (e != cudaSuccess) return e;
+    e = launch_select(c.sel_inn, c.val, c.mu, 0, c.K, c.inn_pos, c.muI, c.errword, c.stream);
+    if (e != cudaSuccess) return e;
+    innovation_fill_kernel<<<dim3(blocks_for(c.muI, 256), c.K), 256, 0, c.stream>>>(c.val, c.inn_pos, c.mu, c.muI, c.inn);
+    return cudaGetLastError();
+}
+
+static cudaError_t launch_scatter(const Ctx &c, const float *values, float *update)
+{
+    cudaError_t e = launch_zero(update, (size_t)c.N * sizeof(float), c.stream);
+    if (e != cudaSuccess) return e;
+    if (c.S == 1)
+        scatter_shared_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(values, c.idx, c.mu, c.K, c.N, update, c.u, c.v);
+    else
+        scatter_own_kernel<<<dim3(blocks_for(c.mu, 128), c.K), 128, 0, c.stream>>>(
+            values, c.idx, c.slot_layer, c.koff_dev, c.mu, c.K, c.N, update, c.u, c.v);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_scatter(const Ctx &c, float *update)
+{
+    const bool ps = c.cfg.variant == LGC_VARIANT_PS;
+    const float *values = c.recon;
+    if (c.cfg.ae_kind == LGC_AE_IDENTITY) {
+        if (ps)
+            identity_ps_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.combined, c.inn, c.mu, c.recon);
+        else
+            values = c.combined;
+    } else {
+        const dim3 grid(blocks_for(c.mu, kAeThreads), c.S);
+        const float *dec = c.params + c.Penc;
+#define CALL(A, B)                                                                                             \
+    if (ps) decode_kernel<A, B, true><<<grid, kAeThreads, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec,    \
+                                                                        (int)c.Pdec, c.inn, c.recon);         \
+    else decode_kernel<A, B, false><<<grid, kAeThreads, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec,      \
+                                                                       (int)c.Pdec, nullptr, c.recon)
+        LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
+#undef CALL
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_scatter(c, values, update);
+}
+
+cudaError_t launch_topk_scatter(const Ctx &c, float *update)
+{
+    const float *values = c.val;
+    if (c.S == 1) {
+        mean_rows_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(c.val, c.K, c.mu, c.recon);
+        values = c.recon;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_scatter(c, values, update);
+}
+
+}  // namespace lgc

@@ -1,0 +1,97 @@
+// Internal declarations shared by the translation units of liblgc: the host context, the work
+// space carve-up, and one launcher prototype per kernel family.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "lgc.h"
+
+namespace lgc {
+
+constexpr int kSelChunk = 4096;    // elements per selection chunk: 256 threads x 16
+constexpr int kSelThreads = 256;
+constexpr int kSelPerThread = 16;
+constexpr int kHistBins = 2048;    // first radix digit: 11 bits; the next two: 10 bits each
+
+// One selection problem family: R rows of `data` (row stride in elements), each cut into the same
+// segments; per segment the k entries of largest |x| are reported, ascending, as int32 offsets.
+struct SelectTables {
+    int num_segments = 0;
+    int num_small = 0;            // segments of at most kSelChunk elements
+    int num_large = 0;
+    int num_chunks = 0;           // chunks of all large segments
+    // device tables (all in the caller's scratch)
+    int64_t *seg_off = nullptr;   // [S] first element of the segment inside a row
+    int32_t *seg_len = nullptr;   // [S]
+    int32_t *seg_k = nullptr;     // [S]
+    int32_t *seg_out = nullptr;   // [S] first output slot of the segment
+    int32_t *small_ids = nullptr; // [num_small] segment ids
+    int32_t *large_ids = nullptr; // [num_large] segment ids
+    int32_t *large_chunk0 = nullptr; // [num_large + 1] first chunk of each large segment
+    int32_t *chunk_large = nullptr;  // [num_chunks] index into large_ids
+    // per-call work space, sized for max_rows rows
+    int max_rows = 0;
+    uint32_t *hist = nullptr;     // [rows][num_large][kHistBins], all zero between passes
+    uint32_t *prefix = nullptr;   // [rows][num_large] key prefix found so far
+    int32_t *k_rem = nullptr;     // [rows][num_large] entries still to find at the prefix
+    int2 *chunk_cnt = nullptr;    // [rows][num_chunks] (#key > T, #key == T), then exclusive prefix
+};
+
+struct Ctx {
+    lgc_config cfg{};
+    cudaStream_t stream = nullptr;
+    int K = 0, L = 0, S = 0;       // S: index sets (1 ring-allreduce, K parameter server)
+    int64_t N = 0, mu = 0, muI = 0, L1 = 0, L2 = 0, P = 0, Penc = 0, Pdec = 0;
+    int op1 = 0, op2 = 0;          // output paddings of the two transposed convolutions
+    int64_t code_len = 0;          // floats per node code: c2 * L2 (identity: mu)
+    std::vector<int64_t> numel, off, k_l, koff, ki_l, kioff;
+    double lr = 0, beta1 = 0, beta2 = 0, eps = 0;
+    int64_t adam_t = 0;
+    // caller buffers
+    float *u = nullptr, *v = nullptr;
+    float *params = nullptr, *adam_m = nullptr, *adam_v = nullptr;
+    // scratch carve-up
+    int32_t *idx = nullptr;        // [S][mu]
+    float *val = nullptr;          // [K][mu]
+    float *code = nullptr;         // [K][code_len]
+    float *combined = nullptr;     // [code_len]
+    float *inn = nullptr;          // [K][mu]
+    int32_t *inn_pos = nullptr;    // [K][muI]
+    float *recon = nullptr;        // [S][mu]
+    int32_t *slot_layer = nullptr; // [mu] layer of each kept slot
+    int32_t *koff_dev = nullptr;   // [L + 1]
+    int32_t *errword = nullptr;    // device check record
+    SelectTables sel_v, sel_inn;
+    // training work space
+    float *t_h = nullptr;          // [K][c1][L1] relu(conv1)
+    float *t_d = nullptr;          // [c1][L1]    relu(convT1)
+    float *t_dr = nullptr;         // [mu]        d loss / d recon
+    float *t_dd = nullptr;         // [c1][L1]
+    float *t_dz = nullptr;         // [c2][L2]    d loss / d mean code
+    float *t_dh = nullptr;         // [K][c1][L1]
+    double *t_loss_part = nullptr; // [loss blocks]
+    int t_loss_blocks = 0;
+    // step state machine
+    enum Stage { kIdle, kAccumulated, kSelected, kEncoded, kCombined } stage = kIdle;
+    int32_t last_leader = 0;
+    std::string err;
+};
+
+// ---- launchers (each enqueues on ctx stream and returns the launch status) -------------------
+cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s);
+cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s);
+cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0,
+                          int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t s);
+cudaError_t launch_gather(const Ctx &c);
+cudaError_t launch_encode(const Ctx &c);
+cudaError_t launch_combine_mean(const Ctx &c);
+cudaError_t launch_combine_ps(Ctx &c, int common_node);
+cudaError_t launch_decode_scatter(const Ctx &c, float *update);
+cudaError_t launch_topk_scatter(const Ctx &c, float *update);
+cudaError_t launch_train_step(Ctx &c, float *loss_out);
+
+}  // namespace lgc

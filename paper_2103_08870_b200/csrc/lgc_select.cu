@@ -1,0 +1,371 @@
+// Stage 2 of the LGC step: exact per-layer top-k by magnitude (Section V-A; the threshold and
+// mask of Algorithm 1/2 made exact: exactly k_l entries, equal magnitudes go to the lower index),
+// reported in ascending index order so that the concatenated vector g~ has a fixed order.
+//
+// Keys are the fp32 bit patterns with the sign cleared (integer order == order of |x|).
+// For every (row, segment) the k-th largest key T and the number r of entries equal to T that
+// still belong to the selection are found by a most-significant-digit radix search; entries are
+// then emitted in index order by counting: an entry is selected iff key > T, or key == T and
+// fewer than r equal keys precede it.  No sorting, no order-dependent atomics: the result is a
+// pure function of the data.
+//
+//  - segments of at most kSelChunk elements: one CTA does everything (keys live in registers);
+//  - larger segments: chunked passes  histogram/scan x3 -> count -> chunk scan -> emit.
+#include "lgc_internal.cuh"
+
+namespace lgc {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kWarps = kSelThreads / 32;
+
+__device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+// Thread t of a CTA takes elements [start + 16 t, start + 16 t + 16) of a segment of `len`
+// elements; returns how many of them exist.  128-bit loads when the address allows.
+__device__ __forceinline__ int load_keys16(const float *__restrict__ seg, int start, int len,
+                                           uint32_t (&key)[kSelPerThread])
+{
+    const int j0 = start + (int)threadIdx.x * kSelPerThread;
+    int valid = len - j0;
+    valid = valid < 0 ? 0 : (valid > kSelPerThread ? kSelPerThread : valid);
+    const float *p = seg + j0;
+    if (valid == kSelPerThread && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
+        const float4 *p4 = reinterpret_cast<const float4 *>(p);
+#pragma unroll
+        for (int q = 0; q < kSelPerThread / 4; ++q) {
+            const float4 x = __ldg(p4 + q);
+            key[4 * q + 0] = mag_key(x.x);
+            key[4 * q + 1] = mag_key(x.y);
+            key[4 * q + 2] = mag_key(x.z);
+            key[4 * q + 3] = mag_key(x.w);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < kSelPerThread; ++i) key[i] = i < valid ? mag_key(__ldg(p + i)) : 0u;
+    }
+    return valid;
+}
+
+// Sum of x over threads with index >= own (inclusive suffix sum) in a CTA of kSelThreads.
+__device__ __forceinline__ int block_suffix_incl(int x, int *warp_tot)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int y = __shfl_down_sync(kFull, x, d);
+        if (lane + d < 32) x += y;
+    }
+    if (lane == 0) warp_tot[warp] = x;
+    __syncthreads();
+    int add = 0;
+    for (int w = warp + 1; w < kWarps; ++w) add += warp_tot[w];
+    __syncthreads();
+    return x + add;
+}
+
+// Sum of x over threads with index < own (exclusive prefix sum); *total gets the CTA sum.
+template <typename T>
+__device__ __forceinline__ T block_prefix_excl(T x, T *warp_tot, T *total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    T incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const T y = __shfl_up_sync(kFull, incl, d);
+        if (lane >= d) incl += y;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    T add = 0, tot = 0;
+    for (int w = 0; w < kWarps; ++w) {
+        const T t = warp_tot[w];
+        if (w < warp) add += t;
+        tot += t;
+    }
+    __syncthreads();
+    if (total) *total = tot;
+    return add + incl - x;
+}
+
+// Ordered emission of one thread's selected entries.  gt_before / eq_before: entries of the
+// segment before this thread's first element with key > T / key == T.
+__device__ __forceinline__ void emit16(const uint32_t (&key)[kSelPerThread], int valid, uint32_t T,
+                                       int r, int gt_before, int eq_before, int64_t first_index,
+                                       int32_t *__restrict__ out, int k, int32_t *errword)
+{
+    int gt = gt_before, eq = eq_before;
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i) {
+        if (i < valid) {
+            const uint32_t x = key[i];
+            int pos = -1;
+            if (x > T) {
+                pos = gt + (eq < r ? eq : r);
+                ++gt;
+            } else if (x == T) {
+                if (eq < r) pos = gt + eq;
+                ++eq;
+            }
+            if (pos >= 0) {
+                if (pos < k) out[pos] = (int32_t)(first_index + i);
+                else atomicExch(errword, 0x5E10);   // would write past the segment's slots
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// small segments: one CTA per (segment, row)
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSelThreads)
+select_small_kernel(const float *__restrict__ data, int64_t row_stride, int row0,
+                    const int64_t *__restrict__ seg_off, const int32_t *__restrict__ seg_len,
+                    const int32_t *__restrict__ seg_k, const int32_t *__restrict__ seg_out,
+                    const int32_t *__restrict__ small_ids, int32_t *__restrict__ out,
+                    int64_t out_stride, int32_t *errword)
+{
+    __shared__ int hist[256];
+    __shared__ int warp_tot[kWarps];
+    __shared__ int found[2];
+    const int s = small_ids[blockIdx.x];
+    const int row = blockIdx.y;
+    const int64_t off = seg_off[s];
+    const int len = seg_len[s], k = seg_k[s];
+    const float *seg = data + (int64_t)(row0 + row) * row_stride + off;
+    uint32_t key[kSelPerThread];
+    const int valid = load_keys16(seg, 0, len, key);
+
+    uint32_t prefix = 0, decided = 0;
+    int k_rem = k;
+#pragma unroll 1
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        hist[threadIdx.x] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kSelPerThread; ++i)
+            if (i < valid && (key[i] & decided) == prefix) atomicAdd(&hist[(key[i] >> shift) & 0xff], 1);
+        __syncthreads();
+        const int mine = hist[threadIdx.x];
+        const int incl = block_suffix_incl(mine, warp_tot);
+        if (incl >= k_rem && incl - mine < k_rem) { found[0] = threadIdx.x; found[1] = k_rem - (incl - mine); }
+        __syncthreads();
+        prefix |= (uint32_t)found[0] << shift;
+        decided |= 0xffu << shift;
+        k_rem = found[1];
+        __syncthreads();
+    }
+    const uint32_t T = prefix;
+    const int r = k_rem;
+    int gt = 0, eq = 0;
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i)
+        if (i < valid) { gt += key[i] > T; eq += key[i] == T; }
+    __shared__ unsigned scan_tot[kWarps];
+    unsigned total;
+    const unsigned before = block_prefix_excl<unsigned>((unsigned)gt | ((unsigned)eq << 16), scan_tot, &total);
+    emit16(key, valid, T, r, (int)(before & 0xffff), (int)(before >> 16),
+           off + (int64_t)threadIdx.x * kSelPerThread, out + (int64_t)row * out_stride + seg_out[s], k, errword);
+}
+
+// ------------------------------------------------------------------------------------------
+// large segments
+// ------------------------------------------------------------------------------------------
+struct LargeArgs {
+    const float *data;
+    int64_t row_stride;
+    int row0;
+    const int64_t *seg_off;
+    const int32_t *seg_len;
+    const int32_t *seg_k;
+    const int32_t *seg_out;
+    const int32_t *large_ids;
+    const int32_t *large_chunk0;
+    const int32_t *chunk_large;
+    int num_large;
+    int num_chunks;
+    uint32_t *hist;
+    uint32_t *prefix;
+    int32_t *k_rem;
+    int2 *chunk_cnt;
+    int32_t *out;
+    int64_t out_stride;
+    int32_t *errword;
+};
+
+__device__ __forceinline__ int chunk_keys(const LargeArgs &a, int chunk, int row, int &li, int &s,
+                                          int &start, uint32_t (&key)[kSelPerThread])
+{
+    li = a.chunk_large[chunk];
+    s = a.large_ids[li];
+    start = (chunk - a.large_chunk0[li]) * kSelChunk;
+    const float *seg = a.data + (int64_t)(a.row0 + row) * a.row_stride + a.seg_off[s];
+    return load_keys16(seg, start, a.seg_len[s], key);
+}
+
+// PASS 0: digit = key bits 30..20; PASS 1: bits 19..10 of keys matching the 11-bit prefix;
+// PASS 2: bits 9..0 of keys matching the 21-bit prefix.
+template <int PASS>
+__global__ void __launch_bounds__(kSelThreads) hist_kernel(LargeArgs a)
+{
+    __shared__ unsigned h[PASS == 0 ? kHistBins : 1];
+    const int row = blockIdx.y;
+    int li, s, start;
+    uint32_t key[kSelPerThread];
+    if (PASS == 0) {
+        for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0;
+        __syncthreads();
+    }
+    const int valid = chunk_keys(a, blockIdx.x, row, li, s, start, key);
+    uint32_t *gh = a.hist + ((int64_t)row * a.num_large + li) * kHistBins;
+    if (PASS == 0) {
+#pragma unroll
+        for (int i = 0; i < kSelPerThread; ++i)
+            if (i < valid) atomicAdd(&h[key[i] >> 20], 1u);
+        __syncthreads();
+        for (int b = threadIdx.x; b < kHistBins; b += kSelThreads)
+            if (h[b]) atomicAdd(gh + b, h[b]);
+    } else {
+        const uint32_t prefix = a.prefix[(int64_t)row * a.num_large + li];
+        const int pshift = PASS == 1 ? 20 : 10;
+#pragma unroll
+        for (int i = 0; i < kSelPerThread; ++i)
+            if (i < valid && (key[i] >> pshift) == prefix) atomicAdd(gh + ((key[i] >> (pshift - 10)) & 1023u), 1u);
+    }
+}
+
+// One CTA per (large segment, row): finds the digit holding the k_rem-th largest key, extends
+// the prefix, and leaves the histogram zeroed for the next pass / the next call.
+template <int PASS>
+__global__ void __launch_bounds__(kSelThreads) scan_kernel(LargeArgs a)
+{
+    constexpr int kBins = PASS == 0 ? kHistBins : 1024;
+    constexpr int kPer = kBins / kSelThreads;
+    __shared__ int warp_tot[kWarps];
+    const int li = blockIdx.x, row = blockIdx.y;
+    const int64_t slot = (int64_t)row * a.num_large + li;
+    uint32_t *gh = a.hist + slot * kHistBins;
+    const int k_rem = PASS == 0 ? a.seg_k[a.large_ids[li]] : a.k_rem[slot];
+    const uint32_t prefix = PASS == 0 ? 0u : a.prefix[slot];
+    int h[kPer], part = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) { h[i] = (int)gh[threadIdx.x * kPer + i]; part += h[i]; }
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) gh[threadIdx.x * kPer + i] = 0u;
+    const int incl = block_suffix_incl(part, warp_tot);
+    if (incl >= k_rem && incl - part < k_rem) {
+        int above = incl - part;
+#pragma unroll
+        for (int i = kPer - 1; i >= 0; --i) {
+            if (above + h[i] >= k_rem) {
+                a.prefix[slot] = (prefix << (PASS == 0 ? 0 : 10)) | (uint32_t)(threadIdx.x * kPer + i);
+                a.k_rem[slot] = k_rem - above;
+                break;
+            }
+            above += h[i];
+        }
+    }
+    if (threadIdx.x == 0 && incl < k_rem) atomicExch(a.errword, 0x5E20 + PASS);   // histogram lost entries
+}
+
+__global__ void __launch_bounds__(kSelThreads) count_kernel(LargeArgs a)
+{
+    __shared__ unsigned warp_tot[kWarps];
+    const int row = blockIdx.y;
+    int li, s, start;
+    uint32_t key[kSelPerThread];
+    const int valid = chunk_keys(a, blockIdx.x, row, li, s, start, key);
+    const uint32_t T = a.prefix[(int64_t)row * a.num_large + li];
+    unsigned gt = 0, eq = 0;
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i)
+        if (i < valid) { gt += key[i] > T; eq += key[i] == T; }
+    unsigned total;
+    block_prefix_excl<unsigned>(gt | (eq << 16), warp_tot, &total);
+    if (threadIdx.x == 0)
+        a.chunk_cnt[(int64_t)row * a.num_chunks + blockIdx.x] = make_int2((int)(total & 0xffff), (int)(total >> 16));
+}
+
+// One CTA per (large segment, row): exclusive prefix over the segment's chunk counts, in place.
+__global__ void __launch_bounds__(kSelThreads) chunk_scan_kernel(LargeArgs a)
+{
+    __shared__ unsigned long long warp_tot[kWarps];
+    const int li = blockIdx.x, row = blockIdx.y;
+    const int c0 = a.large_chunk0[li], c1 = a.large_chunk0[li + 1];
+    int2 *cnt = a.chunk_cnt + (int64_t)row * a.num_chunks;
+    unsigned long long carry = 0;
+    for (int base = c0; base < c1; base += kSelThreads) {
+        const int c = base + threadIdx.x;
+        int2 mine = make_int2(0, 0);
+        if (c < c1) mine = cnt[c];
+        unsigned long long total;
+        const unsigned long long x = (unsigned long long)(unsigned)mine.x | ((unsigned long long)(unsigned)mine.y << 32);
+        const unsigned long long before = carry + block_prefix_excl<unsigned long long>(x, warp_tot, &total);
+        if (c < c1) cnt[c] = make_int2((int)(before & 0xffffffffu), (int)(before >> 32));
+        carry += total;
+    }
+    if (threadIdx.x == 0) {
+        const int64_t slot = (int64_t)row * a.num_large + li;
+        const long long gt = (long long)(carry & 0xffffffffu), eq = (long long)(carry >> 32);
+        const int r = a.k_rem[slot], k = a.seg_k[a.large_ids[li]];
+        if (gt + r != k || eq < r) atomicExch(a.errword, 0x5E30);
+    }
+}
+
+__global__ void __launch_bounds__(kSelThreads) emit_kernel(LargeArgs a)
+{
+    __shared__ unsigned warp_tot[kWarps];
+    const int row = blockIdx.y;
+    int li, s, start;
+    uint32_t key[kSelPerThread];
+    const int valid = chunk_keys(a, blockIdx.x, row, li, s, start, key);
+    const int64_t slot = (int64_t)row * a.num_large + li;
+    const uint32_t T = a.prefix[slot];
+    const int r = a.k_rem[slot];
+    const int2 chunk_before = a.chunk_cnt[(int64_t)row * a.num_chunks + blockIdx.x];
+    unsigned gt = 0, eq = 0;
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i)
+        if (i < valid) { gt += key[i] > T; eq += key[i] == T; }
+    unsigned total;
+    const unsigned before = block_prefix_excl<unsigned>(gt | (eq << 16), warp_tot, &total);
+    if ((total & 0xffff) == 0 && chunk_before.y >= r) return;   // nothing of this chunk is selected
+    emit16(key, valid, T, r, chunk_before.x + (int)(before & 0xffff), chunk_before.y + (int)(before >> 16),
+           a.seg_off[s] + start + (int64_t)threadIdx.x * kSelPerThread,
+           a.out + (int64_t)row * a.out_stride + a.seg_out[s], a.seg_k[s], a.errword);
+}
+
+}  // namespace
+
+cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0,
+                          int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t st)
+{
+    if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
+    if (t.num_small) {
+        select_small_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(
+            data, row_stride, row0, t.seg_off, t.seg_len, t.seg_k, t.seg_out, t.small_ids, out, out_stride, errword);
+    }
+    if (t.num_large) {
+        LargeArgs a;
+        a.data = data; a.row_stride = row_stride; a.row0 = row0;
+        a.seg_off = t.seg_off; a.seg_len = t.seg_len; a.seg_k = t.seg_k; a.seg_out = t.seg_out;
+        a.large_ids = t.large_ids; a.large_chunk0 = t.large_chunk0; a.chunk_large = t.chunk_large;
+        a.num_large = t.num_large; a.num_chunks = t.num_chunks;
+        a.hist = t.hist; a.prefix = t.prefix; a.k_rem = t.k_rem; a.chunk_cnt = t.chunk_cnt;
+        a.out = out; a.out_stride = out_stride; a.errword = errword;
+        const dim3 gc(t.num_chunks, rows), gl(t.num_large, rows);
+        hist_kernel<0><<<gc, kSelThreads, 0, st>>>(a);
+        scan_kernel<0><<<gl, kSelThreads, 0, st>>>(a);
+        hist_kernel<1><<<gc, kSelThreads, 0, st>>>(a);
+        scan_kernel<1><<<gl, kSelThreads, 0, st>>>(a);
+        hist_kernel<2><<<gc, kSelThreads, 0, st>>>(a);
+        scan_kernel<2><<<gl, kSelThreads, 0, st>>>(a);
+        count_kernel<<<gc, kSelThreads, 0, st>>>(a);
+        chunk_scan_kernel<<<gl, kSelThreads, 0, st>>>(a);
+        emit_kernel<<<gc, kSelThreads, 0, st>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace lgc

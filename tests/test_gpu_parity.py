@@ -1,0 +1,198 @@
+"""CUDA path vs CPU oracle, element by element, on cases the oracle finishes in seconds."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2103_08870_b200 import lgc
+from paper_2103_08870_b200 import workloads as W
+
+from parity import assert_bitwise, assert_close, compare_step, make_pair
+
+pytestmark = pytest.mark.gpu
+
+# ragged toy table: tiny layers, sizes that are no multiple of four, chunk edges (4096, 4097,
+# 8193), several chunks with a ragged tail (20000, 70001)
+TOY = [4096, 64, 1500, 9000, 65, 127, 20000, 5001, 4097, 8193, 1, 3, 70001, 1000]
+
+
+def toy_source(numel, K, seed=5):
+    return W.GradientSource(W.LayerTable("toy", list(numel), [1 + (i % 3) for i in range(len(numel))]), K, seed=seed)
+
+
+def run_steps(numel, K, steps, **kw):
+    seed = kw.get("seed", W.DEFAULT_SEED)
+    ora, gpu = make_pair(numel, K, **kw)
+    src = toy_source(numel, K)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t in range(steps):
+        g = src.step(t)
+        compare_step(ora, gpu, g, g.cuda(), W.choice_for_step(seed, t, K), upd)
+    return ora, gpu
+
+
+def test_tiny_config_ring_allreduce():
+    # one flat tensor of 2^20 elements, K = 2, density 0.1 % (k = 1049), AE 8/4, 3 steps
+    w = W.workload("tiny")
+    ora, gpu = make_pair(w.table.numel, w.num_nodes)
+    assert gpu.mu == 1049 and (gpu.L1, gpu.L2) == (524, 261)
+    src = W.GradientSource(w.table, w.num_nodes, seed=w.seed)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t in range(w.steps):
+        g = src.step(t)
+        compare_step(ora, gpu, g, g.cuda(), W.choice_for_step(w.seed, t, w.num_nodes), upd)
+
+
+@pytest.mark.parametrize("K", [1, 3])
+def test_ragged_layers_ring_allreduce(K):
+    run_steps(TOY, K, 4)
+
+
+def test_ragged_layers_parameter_server():
+    ora, gpu = run_steps(TOY, 3, 3, variant="ps")
+    assert gpu.idx.shape == (3, gpu.mu)
+
+
+def test_parameter_server_large_innovation_segments():
+    # dense selection so that a layer keeps more than one chunk of values: the innovation
+    # selection then runs through the chunked path as well
+    run_steps([60000, 300, 5000], 2, 2, variant="ps", density_ppm=100000, innovation_permille=300)
+
+
+@pytest.mark.parametrize("variant", ["rar", "ps"])
+def test_identity_autoencoder(variant):
+    run_steps(TOY, 2, 3, variant=variant, ae_kind="identity")
+
+
+def test_wide_autoencoder_and_small_channels():
+    run_steps(TOY, 2, 2, c1=16, c2=8)
+    run_steps(TOY, 2, 1, c1=3, c2=2)
+    run_steps(TOY, 2, 1, c1=16, c2=8, variant="ps")
+
+
+def test_momentum_zero_and_other_densities():
+    run_steps(TOY, 2, 3, momentum=0.0)
+    run_steps(TOY, 2, 2, density_ppm=50000)
+    run_steps([50000, 777], 2, 2, density_ppm=1000000, ae_kind="identity")     # everything is kept
+
+
+@pytest.mark.parametrize("fill", ["zeros", "equal", "few_values", "denormal"])
+def test_degenerate_values(fill):
+    numel = [9000, 130, 4097, 33000]
+    K = 2
+    ora, gpu = make_pair(numel, K, density_ppm=20000)
+    N = gpu.N
+    rng = np.random.default_rng(3)
+    upd = torch.empty(N, dtype=torch.float32, device="cuda")
+    for t in range(3):
+        if fill == "zeros":
+            g = np.zeros((K, N), np.float32)
+        elif fill == "equal":
+            g = np.full((K, N), -0.25, np.float32)
+        elif fill == "few_values":
+            g = rng.integers(-2, 3, size=(K, N)).astype(np.float32)
+        else:
+            g = (rng.integers(-5, 6, size=(K, N)) * 1e-45).astype(np.float32)
+        gt = torch.from_numpy(g)
+        compare_step(ora, gpu, gt, gt.cuda(), t % K, upd)
+
+
+def test_same_inputs_same_bits_twice():
+    outs = []
+    for _ in range(2):
+        w = lgc.LGC(TOY, 3, variant="ps")
+        w.set_ae_params(W.ae_init_params(8, 4, "ps", 3))
+        src = toy_source(TOY, 3)
+        upd = torch.empty(w.N, dtype=torch.float32, device="cuda")
+        for t in range(3):
+            w.step(src.step(t).cuda(), upd, t % 3)
+        w.check()
+        outs.append((upd.cpu().numpy().copy(), w.v.cpu().numpy().copy(), w.idx.cpu().numpy().copy()))
+    for a, b in zip(*outs):
+        assert_bitwise(a, b, "repeat run")
+
+
+def test_call_order_and_argument_errors():
+    w = lgc.LGC(TOY, 2)
+    g = torch.zeros(2, w.N, device="cuda")
+    upd = torch.empty(w.N, device="cuda")
+    with pytest.raises(lgc.LGCError, match="BAD_STATE"):
+        w.topk(0)
+    with pytest.raises(lgc.LGCError, match="BAD_STATE"):
+        w.decode_scatter(upd)
+    w.accumulate(g)
+    with pytest.raises(lgc.LGCError, match="BAD_STATE"):
+        w.accumulate(g)
+    with pytest.raises(lgc.LGCError, match="INVALID_ARG"):
+        w.topk(5)
+    w.topk(1)
+    with pytest.raises(lgc.LGCError, match="BAD_STATE"):
+        w.combine(0)
+    with pytest.raises(ValueError):
+        w.decode_scatter(upd[:-1])
+    w.encode()
+    w.combine(0)
+    w.decode_scatter(upd)
+    w.check()
+    with pytest.raises(lgc.LGCError, match="INVALID_ARG"):
+        w.set_ae_params(torch.zeros(5))
+
+
+def test_topk_scatter_phase_two():
+    for variant in ("rar", "ps"):
+        ora, gpu = make_pair(TOY, 3, variant=variant)
+        src = toy_source(TOY, 3)
+        upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+        for t in range(2):
+            g = src.step(t)
+            ora.accumulate(g.numpy())
+            gpu.accumulate(g.cuda())
+            ora.topk(t)
+            gpu.topk(t)
+            ref = ora.topk_scatter()
+            gpu.topk_scatter(upd)
+            assert_close(upd.cpu().numpy(), ref, "sparse mean update")
+            assert_bitwise(gpu.v.cpu().numpy(), ora.v, "v")
+            assert_bitwise(gpu.u.cpu().numpy(), ora.u, "u")
+        gpu.check()
+
+
+def test_autoencoder_training_matches_oracle():
+    numel = [300000, 5000, 64, 120000]
+    K = 3
+    ora, gpu = make_pair(numel, K)
+    src = toy_source(numel, K)
+    g = src.step(0) * 1e3                       # O(1) values
+    ora.accumulate(g.numpy())
+    gpu.accumulate(g.cuda())
+    ora.topk(0)
+    gpu.topk(0)
+    loss_dev = torch.zeros(1, device="cuda")
+    losses_ref, losses = [], []
+    for _ in range(50):
+        losses_ref.append(ora.ae_train_step())
+        gpu.ae_train_step(loss_dev)
+        losses.append(loss_dev.item())
+    assert_close(np.array(losses), np.array(losses_ref), "training losses", rel=1e-5)
+    assert_close(gpu.get_ae_params().numpy(), ora.get_params(), "trained parameters")
+    assert losses[-1] < losses[0]
+    # the trained autoencoder then compresses
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    ora.encode(); ora.combine(0); ref = ora.decode_scatter()
+    gpu.encode(); gpu.combine(0); gpu.decode_scatter(upd)
+    assert_close(upd.cpu().numpy(), ref, "update with the trained autoencoder", rel=2e-5)
+    gpu.check()
+
+
+def test_step_from_host_buffers():
+    ora, gpu = make_pair(TOY, 2)
+    src = toy_source(TOY, 2)
+    g = src.step(0)
+    hg = g.clone().pin_memory()
+    hu = torch.empty(gpu.N, dtype=torch.float32).pin_memory()
+    dg = torch.empty(2, gpu.N, device="cuda")
+    du = torch.empty(gpu.N, device="cuda")
+    gpu.step_host(hg, dg, du, hu, 1)
+    torch.cuda.synchronize()
+    ref = ora.step(g.numpy(), 1)
+    assert_close(hu.numpy(), ref, "update through host buffers")
+    assert_bitwise(gpu.v.cpu().numpy(), ora.v, "v")
