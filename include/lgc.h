@@ -74,9 +74,11 @@ typedef struct {
 } lgc_config;
 
 /* Sizes the caller must provide, in bytes.
- *   state   : velocity u and residual v, 2 * K * N fp32 (Section V-A; zeroed by lgc_init)
+ *   state   : velocity u and residual v, each K * N fp32 padded to a multiple of four
+ *             (Section V-A; zeroed by lgc_init)
  *   scratch : indices, kept values, codes, selection work space, tables
- *   params  : autoencoder parameters followed by the two Adam moment vectors (3 * P fp32)
+ *   params  : autoencoder parameters followed by the two Adam moment vectors, each padded to a
+ *             multiple of four floats (3 * ceil(P/4) * 4 fp32)
  * Returns LGC_ERR_INVALID_ARG / LGC_ERR_UNSUPPORTED for a configuration lgc_init would refuse. */
 lgc_status lgc_workspace_bytes(const lgc_config *cfg, size_t *state_bytes, size_t *scratch_bytes,
                                size_t *params_bytes);
@@ -174,6 +176,8 @@ lgc_status lgc_get_ae_params(const lgc_ctx *ctx, float *dst, size_t count);
 lgc_status lgc_check(lgc_ctx *ctx);
 
 const char *lgc_status_string(lgc_status s);
+/* Text of the last failure recorded in `ctx`; with ctx == NULL, of the calling thread's last
+ * failure that had no context (lgc_init).  Owned by the library, valid until the next call. */
 const char *lgc_last_error(const lgc_ctx *ctx);
 
 #ifdef __cplusplus

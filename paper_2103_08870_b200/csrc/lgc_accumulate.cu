@@ -105,6 +105,7 @@ cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count
 cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s)
 {
     if (bytes == 0) return cudaSuccess;
+    if (reinterpret_cast<uintptr_t>(p) & 15) return cudaErrorMisalignedAddress;   // refused on the host
     const uint64_t nvec = bytes >> 4;
     if (nvec) {
         uint64_t want = (nvec + 255) / 256;

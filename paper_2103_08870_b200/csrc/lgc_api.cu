@@ -36,6 +36,8 @@ struct Plan {
     std::vector<int64_t> numel, off, k_l, koff, ki_l, kioff;
 };
 
+int64_t pad4(int64_t n) { return (n + 3) / 4 * 4; }   // keeps consecutive fp32 vectors 16-byte aligned
+
 int64_t conv_len(int64_t lin) { return lin >= 3 ? (lin - 3) / 2 + 1 : 0; }
 
 bool ae_channels_supported(int c1, int c2)
@@ -163,9 +165,13 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
     cv.take<char>(0);
 }
 
+// Message of the last failure that had no context to be stored in (lgc_init, NULL contexts).
+thread_local std::string g_last_error;
+
 lgc_status fail(lgc_ctx *ctx, lgc_status s, const std::string &msg)
 {
     if (ctx) ctx->err = msg;
+    else g_last_error = msg;
     return s;
 }
 
@@ -232,9 +238,9 @@ lgc_status lgc_workspace_bytes(const lgc_config *cfg, size_t *state_bytes, size_
     Ctx tmp;
     Carver cv(nullptr);
     carve(cv, tmp, p, *cfg);
-    if (state_bytes) *state_bytes = (size_t)2 * p.K * p.N * sizeof(float);
+    if (state_bytes) *state_bytes = (size_t)2 * pad4((int64_t)p.K * p.N) * sizeof(float);
     if (scratch_bytes) *scratch_bytes = (cv.used + kAlign - 1) / kAlign * kAlign;
-    if (params_bytes) *params_bytes = (size_t)(p.P > 0 ? 3 * p.P : 4) * sizeof(float);
+    if (params_bytes) *params_bytes = (size_t)(p.P > 0 ? 3 * pad4(p.P) : 4) * sizeof(float);
     return LGC_OK;
 }
 
@@ -265,10 +271,10 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     c->beta2 = cfg->adam_beta2 != 0.0f ? (double)cfg->adam_beta2 : 0.999;
     c->eps = cfg->adam_eps != 0.0f ? (double)cfg->adam_eps : 1e-8;
     c->u = static_cast<float *>(state);
-    c->v = c->u + (size_t)p.K * p.N;
+    c->v = c->u + pad4((int64_t)p.K * p.N);   // both halves start 16-byte aligned
     c->params = static_cast<float *>(params);
-    c->adam_m = c->params + p.P;
-    c->adam_v = c->adam_m + p.P;
+    c->adam_m = c->params + pad4(p.P);
+    c->adam_v = c->adam_m + pad4(p.P);
     Carver cv(scratch);
     carve(cv, *c, p, *cfg);
     if (cfg->ae_kind == LGC_AE_IDENTITY) c->code = c->val;
@@ -276,7 +282,7 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     cudaStream_t s = c->stream;
     cudaError_t e = launch_zero(state, need_state, s);
     if (e == cudaSuccess) e = launch_zero(scratch, need_scratch, s);
-    if (e == cudaSuccess && p.P > 0) e = launch_zero(c->adam_m, (size_t)2 * p.P * sizeof(float), s);
+    if (e == cudaSuccess && p.P > 0) e = launch_zero(c->adam_m, (size_t)2 * pad4(p.P) * sizeof(float), s);
     std::vector<std::vector<int32_t>> hold32;
     std::vector<std::vector<int64_t>> hold64;
     hold32.reserve(32);
@@ -295,7 +301,8 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
         delete c;
-        return LGC_ERR_CUDA;
+        cudaGetLastError();
+        return cuda_fail(nullptr, e, "lgc_init");
     }
     *out = c;
     return LGC_OK;
@@ -487,6 +494,6 @@ const char *lgc_status_string(lgc_status s)
     return "LGC_ERR_UNKNOWN";
 }
 
-const char *lgc_last_error(const lgc_ctx *c) { return c ? c->err.c_str() : "context is NULL"; }
+const char *lgc_last_error(const lgc_ctx *c) { return c ? c->err.c_str() : g_last_error.c_str(); }
 
 }  // extern "C"

@@ -136,7 +136,7 @@ class LGC:
     # -- plumbing -----------------------------------------------------------------------------
     def _ok(self, status: int, where: str) -> None:
         if status != LGC_OK:
-            detail = self._l.lgc_last_error(self._ctx).decode() if self._ctx else ""
+            detail = self._l.lgc_last_error(self._ctx if self._ctx else None).decode()
             raise LGCError(status, where, detail)
 
     def close(self) -> None:
