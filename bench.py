@@ -59,7 +59,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except Exception:
@@ -220,20 +220,22 @@ def run_ours(args, w: W.Workload):
     acc_ms = [a.elapsed_time(b) for a, b in ev]
 
     # end to end through host buffers: pinned gradients in, dense update out, every step
-    e2e_steps = max(2, min(args.steps, 5))
-    host_g = torch.empty((K, N), dtype=torch.float32).pin_memory()
-    host_g.copy_(grads[0])
-    host_u = torch.empty(N, dtype=torch.float32).pin_memory()
-    dev_g = torch.empty((K, N), dtype=torch.float32, device=dev)
-    gpu.step_host(host_g, dev_g, update, host_u, choices[0])
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for t in range(e2e_steps):
-        gpu.step_host(host_g, dev_g, update, host_u, choices[t])
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
+    e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 5))
+    e2e_ms = 0.0
+    if e2e_steps:
+        host_g = torch.empty((K, N), dtype=torch.float32).pin_memory()
+        host_g.copy_(grads[0])
+        host_u = torch.empty(N, dtype=torch.float32).pin_memory()
+        dev_g = torch.empty((K, N), dtype=torch.float32, device=dev)
+        gpu.step_host(host_g, dev_g, update, host_u, choices[0])
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for t in range(e2e_steps):
+            gpu.step_host(host_g, dev_g, update, host_u, choices[t])
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
 
     t_all = torch.tensor([elapsed_ms, e2e_ms, statistics.mean(acc_ms)], dtype=torch.float64, device=dev)
     if world > 1:
@@ -243,7 +245,7 @@ def run_ours(args, w: W.Workload):
     if rank == 0:
         dense_bytes = K * N * 4 * world
         value = dense_bytes / 1e9 / (elapsed_ms / 1e3 / args.steps)
-        e2e_value = dense_bytes / 1e9 / (e2e_ms / 1e3 / e2e_steps)
+        e2e_value = dense_bytes / 1e9 / (e2e_ms / 1e3 / e2e_steps) if e2e_steps else None
         peak, peak_kind = measured_peak()
         acc_bytes = 20 * K * N
         achieved = acc_bytes / 1e9 / (acc_mean_ms / 1e3)
@@ -260,7 +262,7 @@ def run_ours(args, w: W.Workload):
             "step_hbm": {"algorithmic_bytes": step_bytes, "achieved_GBps": step_gbs,
                          "frac_of_measured_peak": step_gbs / peak, "frac_of_nominal_8TBps": step_gbs / NOMINAL_HBM_GBS},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": K * N * 4, "d2h_bytes_per_step": N * 4,
-                    "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+                    "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps if e2e_steps else None},
             "gpu_launches": launches_per_step(gpu) * args.steps,
             "clocks": clocks,
         }
@@ -278,14 +280,18 @@ def run_ours(args, w: W.Workload):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=list(W.WORKLOAD_NAMES))
     ap.add_argument("--cpu-sample-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--nodes", type=int, default=0, help="override K (profiling aid: a smaller device footprint)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling aid)")
     args = ap.parse_args()
     w = W.workload(args.workload)
+    if args.nodes > 0:
+        w.num_nodes = args.nodes
     if args.impl == "reference":
         run_reference(args, w)
     else:
