@@ -1,0 +1,143 @@
+"""The five workload configurations at full size, in the launch configuration bench.py times.
+
+Configs 1-3 run the whole oracle beside the CUDA path (they fit in host memory and finish in
+tens of seconds per step); the stress config (2^30 elements per node) compares the elementwise
+stages on sampled positions, the selection against the oracle on the leader's full row, and the
+autoencoder stages in full (they work on mu values only).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from oracle import OracleLGC
+from paper_2103_08870_b200 import lgc
+from paper_2103_08870_b200 import workloads as W
+
+from parity import assert_bitwise, assert_close, compare_step, make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+def run_workload(name, steps, state_every=1):
+    w = W.workload(name)
+    ora, gpu = make_pair(w.table.numel, w.num_nodes, variant=w.variant, c1=w.ae_c1, c2=w.ae_c2,
+                         density_ppm=w.density_ppm, momentum=w.momentum,
+                         innovation_permille=w.innovation_permille, seed=w.seed)
+    src = W.GradientSource(w.table, w.num_nodes, seed=w.seed, device="cuda")
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    g = torch.empty((w.num_nodes, gpu.N), dtype=torch.float32, device="cuda")
+    for t in range(steps):
+        src.step_into(t, g)
+        check = (t % state_every == 0) or t == steps - 1
+        compare_step(ora, gpu, g.cpu(), g, W.choice_for_step(w.seed, t, w.num_nodes), upd, check_state=check)
+    return ora, gpu
+
+
+def test_resnet50_config():
+    ora, gpu = run_workload("resnet50", 10, state_every=3)
+    assert gpu.L == 161 and gpu.N == 25_557_032 and gpu.mu == sum(ora.k_l)
+
+
+def test_resnet101_parameter_server_config():
+    ora, gpu = run_workload("resnet101_ps", 4, state_every=3)
+    assert gpu.L == 314 and gpu.N == 44_549_160 and gpu.idx.shape[0] == 16
+
+
+def test_segnet_config_with_autoencoder_training():
+    w = W.workload("segnet")
+    K = w.num_nodes
+    ora, gpu = make_pair(w.table.numel, K, seed=w.seed)
+    src = W.GradientSource(w.table, K, seed=w.seed, device="cuda")
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    g = torch.empty((K, gpu.N), dtype=torch.float32, device="cuda")
+    loss_dev = torch.zeros(1, device="cuda")
+    losses, losses_ref = [], []
+    for t in range(w.ae_train_steps):                      # second phase: top-k updates while the AE trains
+        src.step_into(t, g)
+        choice = W.choice_for_step(w.seed, t, K)
+        ora.accumulate(g.cpu().numpy())
+        gpu.accumulate(g)
+        ora.topk(choice)
+        gpu.topk(choice)
+        if t % 10 == 0:
+            assert_bitwise(gpu.idx.cpu().numpy(), ora.idx[:1], f"indices at training step {t}")
+            assert_bitwise(gpu.val.cpu().numpy(), ora.val, f"values at training step {t}")
+        losses_ref.append(ora.ae_train_step())
+        gpu.ae_train_step(loss_dev)
+        losses.append(loss_dev.item())
+        ref = ora.topk_scatter()
+        gpu.topk_scatter(upd)
+        if t % 10 == 0 or t == w.ae_train_steps - 1:
+            assert_close(upd.cpu().numpy(), ref, f"sparse update at training step {t}")
+            assert_bitwise(gpu.v.cpu().numpy(), ora.v, f"v at training step {t}")
+    assert_close(np.array(losses), np.array(losses_ref), "training losses")
+    assert_close(gpu.get_ae_params().numpy(), ora.get_params(), "trained parameters")
+    gpu.check()
+    for t in range(w.ae_train_steps, w.ae_train_steps + 3):  # third phase: compressed updates
+        src.step_into(t, g)
+        compare_step(ora, gpu, g.cpu(), g, W.choice_for_step(w.seed, t, K), upd, check_state=(t == w.ae_train_steps + 2))
+
+
+def test_stress_config_sampled():
+    w = W.workload("stress")
+    K, N = w.num_nodes, w.table.total
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70 * 2**30:
+        pytest.skip("needs about 70 GiB of free device memory")
+    gpu = lgc.LGC(w.table.numel, K, density_ppm=w.density_ppm, momentum=w.momentum, c1=w.ae_c1, c2=w.ae_c2)
+    params = W.ae_init_params(w.ae_c1, w.ae_c2, "rar", K, w.seed)
+    gpu.set_ae_params(params)
+    assert gpu.mu == 107_374 and (gpu.L1, gpu.L2) == (53_686, 26_842)
+    # the oracle works on mu-sized vectors in full and on a sample of the 2^30 positions
+    ora = OracleLGC([gpu.mu * 1000], K, density_ppm=1000, c1=w.ae_c1, c2=w.ae_c2, params=params.numpy())
+    assert ora.mu == gpu.mu
+    rng = np.random.default_rng(7)
+    pos = np.unique(np.concatenate([rng.integers(0, N, 2_000_000), np.arange(0, 4096), np.arange(N - 4099, N)]))
+    pos_dev = torch.from_numpy(pos).cuda()
+    u_s = np.zeros((K, pos.size), np.float32)
+    v_s = np.zeros((K, pos.size), np.float32)
+    src = W.GradientSource(w.table, K, seed=w.seed, device="cuda", chunk=1 << 26)
+    g = torch.empty((K, N), dtype=torch.float32, device="cuda")
+    upd = torch.empty(N, dtype=torch.float32, device="cuda")
+    for t in range(w.steps):
+        src.step_into(t, g)
+        leader = W.choice_for_step(w.seed, t, K)
+        g_s = g[:, pos_dev].cpu().numpy()
+        gpu.accumulate(g)
+        for k in range(K):
+            O.accumulate(u_s[k], v_s[k], np.ascontiguousarray(g_s[k]), float(np.float32(w.momentum)))
+        assert_bitwise(gpu.u[:, pos_dev].cpu().numpy(), u_s, f"sampled u, step {t}")
+        assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_s, f"sampled v, step {t}")
+        gpu.topk(leader)
+        idx = gpu.idx.cpu().numpy()[0]
+        if t in (0, w.steps - 1):                          # the selection against the oracle, whole row
+            v_leader = gpu.v[leader].cpu().numpy()
+            ref_idx = O.topk(v_leader, gpu.mu, method="select")
+            assert_bitwise(idx, ref_idx, f"selected indices, step {t}")
+            assert_bitwise(gpu.val[leader].cpu().numpy(), O.gather(v_leader, ref_idx), "leader values")
+            del v_leader
+        assert np.all(np.diff(idx) > 0)
+        idx_dev = gpu.idx[0].long()
+        val = gpu.val.cpu().numpy()
+        assert_bitwise(val, gpu.v[:, idx_dev].cpu().numpy(), "gathered values")      # same bits as v at idx
+        ora.idx = np.broadcast_to(idx, (K, gpu.mu)).copy()
+        ora.val = val.copy()
+        ora.encode()
+        gpu.encode()
+        assert_close(gpu.code.cpu().numpy(), ora.z.reshape(K, -1), "codes")
+        ora.combine()
+        gpu.combine(leader)
+        assert_close(gpu.combined.cpu().numpy(), ora.zbar, "mean code")
+        ora.decode()
+        gpu.decode_scatter(upd)
+        assert_close(gpu.recon.cpu().numpy(), ora.r, "reconstruction")
+        assert_close(upd[idx_dev].cpu().numpy(), ora.r[0], "update at the scatter positions")
+        assert int(torch.count_nonzero(upd).item()) <= gpu.mu
+        assert float(upd.abs().sum().item()) == pytest.approx(float(np.abs(ora.r[0].astype(np.float32)).sum()), rel=1e-4)
+        sent = np.isin(pos, idx)
+        u_s[:, sent] = 0
+        v_s[:, sent] = 0
+        assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_s, f"sampled v after clearing, step {t}")
+        assert not gpu.v[:, idx_dev].any().item() and not gpu.u[:, idx_dev].any().item()
+        gpu.check()
