@@ -145,6 +145,32 @@ lgc_status lgc_ae_train_step(lgc_ctx *ctx, float *loss_out);
 lgc_status lgc_step_host(lgc_ctx *ctx, const float *host_grads, float *dev_grads, float *dev_update,
                          float *host_update, int32_t choice);
 
+/* Top-k by magnitude of ONE flat vector without any caller-provided work space.
+ * (The paper has no counterpart; this serves callers of the library, not the method.)
+ *
+ * For callers that may not allocate device memory or hand over scratch: code running under a
+ * fixed-footprint promise, plugins whose host owns the allocator and passes only inputs and
+ * outputs, jobs on a device that is already full.  The selection's tables, radix histogram and
+ * per-chunk counts live in a fixed array compiled into the library (about 60 KB, held by every
+ * GPU that loads the library until the process exits), which caps the vector length at
+ * LGC_NOALLOC_MAX_N elements.  The call itself performs no allocation of any kind.
+ *
+ *   v       : device, fp32 [n], read only          n : 1 .. LGC_NOALLOC_MAX_N
+ *   k       : 1 .. n entries to keep               stream : cudaStream_t
+ *   idx_out : device, int32 [k]; receives the offsets of the k entries of largest |v| (equal
+ *             magnitudes: the lower index wins) in ascending order -- the same result lgc_topk
+ *             gives for a single layer of n elements.
+ * Returns LGC_ERR_UNSUPPORTED when n is above the maximum and LGC_ERR_INVALID_ARG for null
+ * pointers or k outside 1..n; lgc_last_error(NULL) has the text.  Nothing is enqueued then.
+ *
+ * The first call on a device looks up the array's device address (once per device, with that
+ * device current); make that first call before any stream capture begins.
+ * All calls share the one array and it keeps the previous call's contents (the call clears what
+ * must start at zero itself): two calls whose kernels overlap on the GPU -- different streams,
+ * or different host threads -- race on it.  Serialise them. */
+#define LGC_NOALLOC_MAX_N 16777216
+lgc_status lgc_topk_noalloc(const float *v, int64_t n, int64_t k, int32_t *idx_out, void *stream);
+
 /* ---- inspection --------------------------------------------------------------------------- */
 
 /* N, mu, encoder lengths L1 (after the first convolution) and L2 (code length per channel), and

@@ -10,6 +10,10 @@
 struct lgc_ctx : lgc::Ctx {};
 
 namespace lgc {
+
+// Message of the calling thread's last failure that had no context to be stored in.
+thread_local std::string g_last_error;
+
 namespace {
 
 constexpr size_t kAlign = 256;
@@ -164,9 +168,6 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
     }
     cv.take<char>(0);
 }
-
-// Message of the last failure that had no context to be stored in (lgc_init, NULL contexts).
-thread_local std::string g_last_error;
 
 lgc_status fail(lgc_ctx *ctx, lgc_status s, const std::string &msg)
 {

@@ -81,6 +81,8 @@ struct Ctx {
     std::string err;
 };
 
+extern thread_local std::string g_last_error;   // failures without a context (see lgc_last_error)
+
 // ---- launchers (each enqueues on ctx stream and returns the launch status) -------------------
 cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s);
 cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s);

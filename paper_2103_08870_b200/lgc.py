@@ -23,8 +23,9 @@ EXPORTS = (
     "lgc_workspace_bytes", "lgc_init", "lgc_destroy", "lgc_accumulate", "lgc_topk", "lgc_encode",
     "lgc_combine", "lgc_decode_scatter", "lgc_topk_scatter", "lgc_ae_train_step", "lgc_step_host",
     "lgc_get_layout", "lgc_keep_counts", "lgc_get_buffers", "lgc_set_ae_params", "lgc_get_ae_params",
-    "lgc_check", "lgc_status_string", "lgc_last_error",
+    "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc",
 )
+NOALLOC_MAX_N = 16777216
 
 
 class lgc_config(C.Structure):
@@ -70,6 +71,7 @@ def lib() -> C.CDLL:
         l.lgc_status_string.restype = C.c_char_p
         l.lgc_last_error.argtypes = [vp]
         l.lgc_last_error.restype = C.c_char_p
+        l.lgc_topk_noalloc.argtypes = [vp, C.c_int64, C.c_int64, vp, vp]
         for name in EXPORTS:            # every declared entry point must be exported
             getattr(l, name)
         _lib = l
@@ -81,6 +83,20 @@ class LGCError(RuntimeError):
         self.status = status
         name = lib().lgc_status_string(status).decode()
         super().__init__(f"{where}: {name}" + (f" ({detail})" if detail else ""))
+
+
+def topk_noalloc(v: torch.Tensor, k: int, idx_out: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """lgc_topk_noalloc: indices of the k largest |v| of one flat fp32 CUDA vector, with the work
+    space inside the library (for callers that cannot allocate or pass scratch).  At most
+    NOALLOC_MAX_N elements; calls must not overlap on the GPU (they share the work space)."""
+    if not (v.is_cuda and v.dtype == torch.float32 and v.is_contiguous() and v.dim() == 1):
+        raise ValueError("v: need a contiguous 1-D fp32 CUDA tensor")
+    if not (idx_out.is_cuda and idx_out.dtype == torch.int32 and idx_out.is_contiguous() and idx_out.numel() == k):
+        raise ValueError("idx_out: need a contiguous int32 CUDA tensor of k elements")
+    s = stream if stream is not None else torch.cuda.current_stream(v.device)
+    st = lib().lgc_topk_noalloc(v.data_ptr(), v.numel(), k, idx_out.data_ptr(), C.c_void_p(s.cuda_stream))
+    if st != LGC_OK:
+        raise LGCError(st, "lgc_topk_noalloc", lib().lgc_last_error(None).decode())
 
 
 def status_string(status: int) -> str:
