@@ -152,11 +152,11 @@ def workload_config(w: W.Workload):
 
 
 def launches_per_step(gpu) -> int:
-    """Kernels one step enqueues (ring-allreduce): accumulate, selection passes, gather, encode, mean,
-    zero-fill, decode, scatter."""
+    """Kernels one step enqueues (ring-allreduce): accumulate, selection (small segments; histogram,
+    bucket scan, candidate collection, finish), gather, encode, mean, zero-fill, decode, scatter."""
     large = sum(1 for n in gpu_layer_numel(gpu) if n > 4096)
     small = gpu.L - large
-    sel = (1 if small else 0) + (9 if large else 0)
+    sel = (1 if small else 0) + (4 if large else 0)
     return 1 + sel + 1 + 1 + 1 + 1 + 1 + 1
 
 

@@ -106,7 +106,8 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
     return LGC_OK;
 }
 
-void carve_select(Carver &cv, SelectTables &t, int num_segments, int num_small, int num_large, int num_chunks, int rows)
+void carve_select(Carver &cv, SelectTables &t, int num_segments, int num_small, int num_large, int num_chunks,
+                  int64_t comp_total, int rows)
 {
     t.num_segments = num_segments; t.num_small = num_small; t.num_large = num_large; t.num_chunks = num_chunks;
     t.max_rows = rows;
@@ -122,14 +123,26 @@ void carve_select(Carver &cv, SelectTables &t, int num_segments, int num_small, 
     t.prefix = cv.take<uint32_t>((size_t)rows * num_large);
     t.k_rem = cv.take<int32_t>((size_t)rows * num_large);
     t.chunk_cnt = cv.take<int2>((size_t)rows * num_chunks);
+    t.cand_cnt = cv.take<int32_t>((size_t)rows * num_chunks);
+    t.cand_pos = cv.take<uint16_t>((size_t)rows * num_chunks * kSelChunk);
+    t.seg_m = cv.take<int32_t>((size_t)rows * num_large);
+    t.comp_off = cv.take<int64_t>((size_t)num_large + 1);
+    t.comp_total = comp_total;
+    t.comp_key = cv.take<uint32_t>((size_t)rows * comp_total);
+    t.comp_idx = cv.take<int32_t>((size_t)rows * comp_total);
 }
 
-void count_segments(const std::vector<int64_t> &len, int &small, int &large, int &chunks)
+void count_segments(const std::vector<int64_t> &len, int &small, int &large, int &chunks, int64_t &comp_total)
 {
     small = large = chunks = 0;
+    comp_total = 0;
     for (int64_t n : len) {
         if (n <= kSelChunk) ++small;
-        else { ++large; chunks += (int)((n + kSelChunk - 1) / kSelChunk); }
+        else {
+            ++large;
+            chunks += (int)((n + kSelChunk - 1) / kSelChunk);
+            comp_total += select_compact_capacity(n);
+        }
     }
 }
 
@@ -147,13 +160,14 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
     c.slot_layer = cv.take<int32_t>((size_t)p.mu);
     c.koff_dev = cv.take<int32_t>((size_t)p.L + 1);
     int sm, lg, ch;
-    count_segments(p.numel, sm, lg, ch);
-    carve_select(cv, c.sel_v, p.L, sm, lg, ch, p.S);
+    int64_t comp;
+    count_segments(p.numel, sm, lg, ch, comp);
+    carve_select(cv, c.sel_v, p.L, sm, lg, ch, comp, p.S);
     if (ps) {
         c.inn = cv.take<float>((size_t)p.K * p.mu);
         c.inn_pos = cv.take<int32_t>((size_t)p.K * p.muI);
-        count_segments(p.k_l, sm, lg, ch);
-        carve_select(cv, c.sel_inn, p.L, sm, lg, ch, p.K);
+        count_segments(p.k_l, sm, lg, ch, comp);
+        carve_select(cv, c.sel_inn, p.L, sm, lg, ch, comp, p.K);
     }
     if (conv && !ps) {
         const size_t c1 = cfg.ae_c1, c2 = cfg.ae_c2;
@@ -197,6 +211,7 @@ cudaError_t upload_select(SelectTables &t, const std::vector<int64_t> &off, cons
     const int n = (int)len.size();
     std::vector<int64_t> h_off(off.begin(), off.begin() + n);
     std::vector<int32_t> h_len(n), h_k(n), h_out(n), small_ids, large_ids, chunk0, chunk_large;
+    std::vector<int64_t> comp_off(1, 0);
     chunk0.push_back(0);
     for (int i = 0; i < n; ++i) {
         h_len[i] = (int32_t)len[i];
@@ -209,10 +224,13 @@ cudaError_t upload_select(SelectTables &t, const std::vector<int64_t> &off, cons
             const int nc = (int)((len[i] + kSelChunk - 1) / kSelChunk);
             for (int q = 0; q < nc; ++q) chunk_large.push_back(li);
             chunk0.push_back(chunk0.back() + nc);
+            comp_off.push_back(comp_off.back() + select_compact_capacity(len[i]));
         }
     }
     hold64.push_back(std::move(h_off));
     cudaError_t e = upload(t.seg_off, hold64.back(), s);
+    hold64.push_back(std::move(comp_off));
+    if (e == cudaSuccess) e = upload(t.comp_off, hold64.back(), s);
     std::vector<int32_t> *arrs[] = {&h_len, &h_k, &h_out, &small_ids, &large_ids, &chunk0, &chunk_large};
     int32_t *dsts[] = {t.seg_len, t.seg_k, t.seg_out, t.small_ids, t.large_ids, t.large_chunk0, t.chunk_large};
     for (int i = 0; i < 7 && e == cudaSuccess; ++i) {
@@ -287,7 +305,7 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     std::vector<std::vector<int32_t>> hold32;
     std::vector<std::vector<int64_t>> hold64;
     hold32.reserve(32);
-    hold64.reserve(4);
+    hold64.reserve(8);
     if (e == cudaSuccess) e = upload_select(c->sel_v, p.off, p.numel, p.k_l, p.koff, s, hold32, hold64);
     if (e == cudaSuccess && cfg->variant == LGC_VARIANT_PS)
         e = upload_select(c->sel_inn, p.koff, p.k_l, p.ki_l, p.kioff, s, hold32, hold64);

@@ -39,7 +39,23 @@ struct SelectTables {
     uint32_t *prefix = nullptr;   // [rows][num_large] key prefix found so far
     int32_t *k_rem = nullptr;     // [rows][num_large] entries still to find at the prefix
     int2 *chunk_cnt = nullptr;    // [rows][num_chunks] (#key > T, #key == T), then exclusive prefix
+    // two-pass path (launch_select): candidates of every chunk, and their compacted form
+    int32_t *cand_cnt = nullptr;  // [rows][num_chunks] candidates found in the chunk
+    uint16_t *cand_pos = nullptr; // [rows][num_chunks][kSelChunk] their positions inside the chunk, ascending
+    int32_t *seg_m = nullptr;     // [rows][num_large] entries at or above the bucket of the k-th key
+    int64_t *comp_off = nullptr;  // [num_large + 1] first compact slot of each large segment
+    int64_t comp_total = 0;       // compact slots per row
+    uint32_t *comp_key = nullptr; // [rows][comp_total] keys of the candidates, index order
+    int32_t *comp_idx = nullptr;  // [rows][comp_total] their offsets inside the row
 };
+
+// Compact-array capacity of a large segment of n elements: above it the segment is finished by
+// streaming over the data itself.
+inline int64_t select_compact_capacity(int64_t n)
+{
+    const int64_t c = n / 8 > 32768 ? n / 8 : 32768;
+    return c < n ? c : n;
+}
 
 struct Ctx {
     lgc_config cfg{};
@@ -88,6 +104,8 @@ cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s);
 cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s);
 cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0,
                           int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t s);
+cudaError_t launch_select_multipass(const SelectTables &t, const float *data, int64_t row_stride, int row0,
+                                    int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t s);
 cudaError_t launch_gather(const Ctx &c);
 cudaError_t launch_encode(const Ctx &c);
 cudaError_t launch_combine_mean(const Ctx &c);

@@ -119,7 +119,7 @@ extern "C" lgc_status lgc_topk_noalloc(const float *v, int64_t n, int64_t k, int
     t.prefix = reinterpret_cast<uint32_t *>(base + kOffPrefix);
     t.k_rem = reinterpret_cast<int32_t *>(base + kOffKRem);
     t.chunk_cnt = reinterpret_cast<int2 *>(base + kOffChunkCnt);
-    e = launch_select(t, v, n, 0, 1, idx_out, k, reinterpret_cast<int32_t *>(base + kOffErr), s);
+    e = launch_select_multipass(t, v, n, 0, 1, idx_out, k, reinterpret_cast<int32_t *>(base + kOffErr), s);
     if (e != cudaSuccess) return fail(LGC_ERR_CUDA, std::string("lgc_topk_noalloc: ") + cudaGetErrorString(e));
     return LGC_OK;
 }

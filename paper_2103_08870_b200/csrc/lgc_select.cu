@@ -10,7 +10,10 @@
 // pure function of the data.
 //
 //  - segments of at most kSelChunk elements: one CTA does everything (keys live in registers);
-//  - larger segments: chunked passes  histogram/scan x3 -> count -> chunk scan -> emit.
+//  - larger segments (launch_select): two reads of the data -- leading-digit histogram, then the
+//    candidates at or above the k-th key's bucket -- and one finishing CTA per segment;
+//  - launch_select_multipass: the same result from chunked passes over the data alone
+//    (histogram/scan x3 -> count -> chunk scan -> emit), for callers with minimal work space.
 #include "lgc_internal.cuh"
 
 namespace lgc {
@@ -48,7 +51,7 @@ __device__ __forceinline__ int load_keys16(const float *__restrict__ seg, int st
     return valid;
 }
 
-// Sum of x over threads with index >= own (inclusive suffix sum) in a CTA of kSelThreads.
+// Sum of x over threads with index >= own (inclusive suffix sum) in the CTA; warp_tot: one slot per warp.
 __device__ __forceinline__ int block_suffix_incl(int x, int *warp_tot)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -60,7 +63,7 @@ __device__ __forceinline__ int block_suffix_incl(int x, int *warp_tot)
     if (lane == 0) warp_tot[warp] = x;
     __syncthreads();
     int add = 0;
-    for (int w = warp + 1; w < kWarps; ++w) add += warp_tot[w];
+    for (int w = warp + 1; w < (int)(blockDim.x >> 5); ++w) add += warp_tot[w];
     __syncthreads();
     return x + add;
 }
@@ -79,7 +82,7 @@ __device__ __forceinline__ T block_prefix_excl(T x, T *warp_tot, T *total)
     if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
     T add = 0, tot = 0;
-    for (int w = 0; w < kWarps; ++w) {
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
         const T t = warp_tot[w];
         if (w < warp) add += t;
         tot += t;
@@ -336,10 +339,240 @@ __global__ void __launch_bounds__(kSelThreads) emit_kernel(LargeArgs a)
            a.out + (int64_t)row * a.out_stride + a.seg_out[s], a.seg_k[s], a.errword);
 }
 
+// ------------------------------------------------------------------------------------------
+// large segments, two reads of the data:  histogram of the leading digit -> bucket of the k-th
+// key -> every entry at or above that bucket becomes a candidate (positions kept per chunk, so
+// index order survives) -> one CTA per segment compacts the candidates, finishes the radix
+// search on them and emits.  Segments whose bucket holds too many entries (ties, e.g. a layer
+// of zeros) are finished by the same CTA streaming over the data instead.
+// ------------------------------------------------------------------------------------------
+struct FastArgs {
+    LargeArgs a;
+    int32_t *cand_cnt;
+    uint16_t *cand_pos;
+    int32_t *seg_m;
+    const int64_t *comp_off;
+    int64_t comp_total;
+    uint32_t *comp_key;
+    int32_t *comp_idx;
+};
+
+constexpr int kFinThreads = 1024;
+constexpr int kFinWarps = kFinThreads / 32;
+constexpr int kFinSmemCap = 8192;     // candidates a finishing CTA keeps in shared memory
+constexpr int kFinPerThread = 4;      // consecutive entries per thread in the ordered passes
+
+// As scan_kernel<0>, and also records how many entries lie at or above the chosen bucket.
+__global__ void __launch_bounds__(kSelThreads) scan0_fast_kernel(FastArgs f)
+{
+    const LargeArgs &a = f.a;
+    constexpr int kPer = kHistBins / kSelThreads;
+    __shared__ int warp_tot[kWarps];
+    const int li = blockIdx.x, row = blockIdx.y;
+    const int64_t slot = (int64_t)row * a.num_large + li;
+    uint32_t *gh = a.hist + slot * kHistBins;
+    const int k_rem = a.seg_k[a.large_ids[li]];
+    int h[kPer], part = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) { h[i] = (int)gh[threadIdx.x * kPer + i]; part += h[i]; }
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) gh[threadIdx.x * kPer + i] = 0u;
+    const int incl = block_suffix_incl(part, warp_tot);
+    if (incl >= k_rem && incl - part < k_rem) {
+        int above = incl - part;
+#pragma unroll
+        for (int i = kPer - 1; i >= 0; --i) {
+            if (above + h[i] >= k_rem) {
+                a.prefix[slot] = (uint32_t)(threadIdx.x * kPer + i);
+                a.k_rem[slot] = k_rem - above;
+                f.seg_m[slot] = above + h[i];
+                break;
+            }
+            above += h[i];
+        }
+    }
+    if (threadIdx.x == 0 && incl < k_rem) atomicExch(a.errword, 0x5E40);
+}
+
+// Candidates of one chunk: positions (ascending) of the entries whose leading digit is at least
+// the bucket's.  Skipped for segments that will be finished from the data.
+__global__ void __launch_bounds__(kSelThreads) collect_kernel(FastArgs f)
+{
+    const LargeArgs &a = f.a;
+    __shared__ unsigned warp_tot[kWarps];
+    const int row = blockIdx.y;
+    const int li = a.chunk_large[blockIdx.x];
+    const int64_t slot = (int64_t)row * a.num_large + li;
+    if ((int64_t)f.seg_m[slot] > f.comp_off[li + 1] - f.comp_off[li]) return;
+    int li2, s, start;
+    uint32_t key[kSelPerThread];
+    const int valid = chunk_keys(a, blockIdx.x, row, li2, s, start, key);
+    const uint32_t d0 = a.prefix[slot];
+    unsigned mine = 0;
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i)
+        if (i < valid && (key[i] >> 20) >= d0) ++mine;
+    unsigned total;
+    unsigned at = block_prefix_excl<unsigned>(mine, warp_tot, &total);
+    const int64_t c = (int64_t)row * a.num_chunks + blockIdx.x;
+    if (threadIdx.x == 0) f.cand_cnt[c] = (int)total;
+    if (mine) {
+        uint16_t *dst = f.cand_pos + c * kSelChunk;
+#pragma unroll
+        for (int i = 0; i < kSelPerThread; ++i)
+            if (i < valid && (key[i] >> 20) >= d0) dst[at++] = (uint16_t)(threadIdx.x * kSelPerThread + i);
+    }
+}
+
+// Where a finishing CTA reads its entries from: the compacted candidates or the segment itself.
+struct CompactSource {
+    const uint32_t *key;
+    const int32_t *idx;
+    int n;
+    __device__ __forceinline__ uint32_t key_at(int i) const { return key[i]; }
+    __device__ __forceinline__ int32_t idx_at(int i) const { return idx[i]; }
+};
+struct DataSource {
+    const float *seg;
+    int64_t off;
+    int n;
+    __device__ __forceinline__ uint32_t key_at(int i) const { return mag_key(__ldg(seg + i)); }
+    __device__ __forceinline__ int32_t idx_at(int i) const { return (int32_t)(off + i); }
+};
+
+struct FinishShared {
+    int hist[256];
+    int warp_i[kFinWarps];
+    unsigned warp_u[kFinWarps];
+    int found[2];
+};
+
+// Completes the radix search below the 11-bit bucket d0 (k_rem entries still to find inside it)
+// and emits the k selected offsets in order.  Entries below the bucket, if the source has any,
+// are ignored.
+template <typename Source>
+__device__ void finish_from(const Source &src, uint32_t d0, int k_rem, int k, int32_t *__restrict__ out,
+                            FinishShared &sh, int32_t *errword)
+{
+    uint32_t prefix = d0 << 20, decided = 0x7ff00000u;
+    const int shifts[3] = {12, 4, 0};
+    const uint32_t masks[3] = {0xffu, 0xffu, 0xfu};
+#pragma unroll 1
+    for (int p = 0; p < 3; ++p) {
+        if (threadIdx.x < 256) sh.hist[threadIdx.x] = 0;
+        __syncthreads();
+        for (int i = threadIdx.x; i < src.n; i += kFinThreads) {
+            const uint32_t x = src.key_at(i);
+            if ((x & decided) == prefix) atomicAdd(&sh.hist[(x >> shifts[p]) & masks[p]], 1);
+        }
+        __syncthreads();
+        const int mine = threadIdx.x < 256 ? sh.hist[threadIdx.x] : 0;
+        const int incl = block_suffix_incl(mine, sh.warp_i);
+        if (threadIdx.x < 256 && incl >= k_rem && incl - mine < k_rem) {
+            sh.found[0] = threadIdx.x;
+            sh.found[1] = k_rem - (incl - mine);
+        }
+        if (threadIdx.x == 0 && incl < k_rem) atomicExch(errword, 0x5E50 + p);
+        __syncthreads();
+        prefix |= (uint32_t)sh.found[0] << shifts[p];
+        decided |= masks[p] << shifts[p];
+        k_rem = sh.found[1];
+        __syncthreads();
+    }
+    const uint32_t T = prefix;
+    const int r = k_rem;
+    int gt_done = 0, eq_done = 0;            // entries before the current tile
+    const int tile = kFinThreads * kFinPerThread;
+    for (int base = 0; base < src.n; base += tile) {
+        uint32_t key[kFinPerThread];
+        const int first = base + (int)threadIdx.x * kFinPerThread;
+        unsigned gt = 0, eq = 0;
+#pragma unroll
+        for (int i = 0; i < kFinPerThread; ++i) {
+            key[i] = first + i < src.n ? src.key_at(first + i) : 0u;
+            if (first + i < src.n) { gt += key[i] > T; eq += key[i] == T; }
+        }
+        unsigned total;
+        const unsigned before = block_prefix_excl<unsigned>(gt | (eq << 16), sh.warp_u, &total);
+        int g = gt_done + (int)(before & 0xffff), e = eq_done + (int)(before >> 16);
+#pragma unroll
+        for (int i = 0; i < kFinPerThread; ++i) {
+            if (first + i < src.n) {
+                int pos = -1;
+                if (key[i] > T) { pos = g + (e < r ? e : r); ++g; }
+                else if (key[i] == T) { if (e < r) pos = g + e; ++e; }
+                if (pos >= 0) {
+                    if (pos < k) out[pos] = src.idx_at(first + i);
+                    else atomicExch(errword, 0x5E60);
+                }
+            }
+        }
+        gt_done += (int)(total & 0xffff);
+        eq_done += (int)(total >> 16);
+        if (gt_done + (eq_done < r ? eq_done : r) >= k) break;     // everything is emitted
+    }
+}
+
+__global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
+{
+    const LargeArgs &a = f.a;
+    __shared__ FinishShared sh;
+    extern __shared__ __align__(16) uint32_t fin_dyn[];     // kFinSmemCap keys, then kFinSmemCap offsets
+    uint32_t *s_key = fin_dyn;
+    int32_t *s_idx = reinterpret_cast<int32_t *>(fin_dyn + kFinSmemCap);
+    const int li = blockIdx.x, row = blockIdx.y;
+    const int64_t slot = (int64_t)row * a.num_large + li;
+    const int s = a.large_ids[li];
+    const int64_t off = a.seg_off[s];
+    const int len = a.seg_len[s], k = a.seg_k[s];
+    const float *seg = a.data + (int64_t)(a.row0 + row) * a.row_stride + off;
+    int32_t *out = a.out + (int64_t)row * a.out_stride + a.seg_out[s];
+    const uint32_t d0 = a.prefix[slot];
+    const int k_rem = a.k_rem[slot];
+    const int m = f.seg_m[slot];
+    const int64_t cap = f.comp_off[li + 1] - f.comp_off[li];
+    if ((int64_t)m > cap) {                   // too many entries share the bucket: work on the data
+        DataSource src{seg, off, len};
+        finish_from(src, d0, k_rem, k, out, sh, a.errword);
+        return;
+    }
+    // compact the candidates, chunk after chunk (thread t owns chunk t of a group of 1024 chunks)
+    const bool in_smem = m <= kFinSmemCap;
+    uint32_t *ckey = in_smem ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
+    int32_t *cidx = in_smem ? s_idx : f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
+    const int c0 = a.large_chunk0[li], c1 = a.large_chunk0[li + 1];
+    const int32_t *cnt = f.cand_cnt + (int64_t)row * a.num_chunks;
+    int done = 0;
+    for (int base = c0; base < c1; base += kFinThreads) {
+        const int c = base + (int)threadIdx.x;
+        const unsigned n = c < c1 ? (unsigned)cnt[c] : 0u;
+        unsigned total;
+        unsigned at = (unsigned)done + block_prefix_excl<unsigned>(n, sh.warp_u, &total);
+        if (n) {
+            const uint16_t *pos = f.cand_pos + ((int64_t)row * a.num_chunks + c) * kSelChunk;
+            const int chunk_start = (c - c0) * kSelChunk;
+            for (unsigned q = 0; q < n; ++q, ++at) {
+                const int j = chunk_start + (int)pos[q];
+                if (at < (unsigned)m) {
+                    ckey[at] = mag_key(__ldg(seg + j));
+                    cidx[at] = (int32_t)(off + j);
+                }
+            }
+        }
+        done += (int)total;
+    }
+    if (threadIdx.x == 0 && done != m) atomicExch(a.errword, 0x5E70);
+    __syncthreads();
+    CompactSource src{ckey, cidx, m};
+    finish_from(src, d0, k_rem, k, out, sh, a.errword);
+}
+
 }  // namespace
 
-cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0,
-                          int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t st)
+// Selection by full passes over the data only: small scratch (tables, one histogram per large
+// segment, per-chunk counts), five reads of every large segment.
+cudaError_t launch_select_multipass(const SelectTables &t, const float *data, int64_t row_stride, int row0,
+                                    int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t st)
 {
     if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
     if (t.num_small) {
@@ -364,6 +597,44 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
         count_kernel<<<gc, kSelThreads, 0, st>>>(a);
         chunk_scan_kernel<<<gl, kSelThreads, 0, st>>>(a);
         emit_kernel<<<gc, kSelThreads, 0, st>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+
+cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0,
+                          int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t st)
+{
+    if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
+    if (!t.cand_cnt && t.num_large)   // tables without the two-pass work space
+        return launch_select_multipass(t, data, row_stride, row0, rows, out, out_stride, errword, st);
+    if (t.num_small) {
+        select_small_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(
+            data, row_stride, row0, t.seg_off, t.seg_len, t.seg_k, t.seg_out, t.small_ids, out, out_stride, errword);
+    }
+    if (t.num_large) {
+        constexpr int kFinDyn = 2 * kFinSmemCap * (int)sizeof(uint32_t);
+        static bool configured = false;
+        if (!configured) {
+            const cudaError_t e = cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinDyn);
+            if (e != cudaSuccess) return e;
+            configured = true;
+        }
+        FastArgs f;
+        LargeArgs &a = f.a;
+        a.data = data; a.row_stride = row_stride; a.row0 = row0;
+        a.seg_off = t.seg_off; a.seg_len = t.seg_len; a.seg_k = t.seg_k; a.seg_out = t.seg_out;
+        a.large_ids = t.large_ids; a.large_chunk0 = t.large_chunk0; a.chunk_large = t.chunk_large;
+        a.num_large = t.num_large; a.num_chunks = t.num_chunks;
+        a.hist = t.hist; a.prefix = t.prefix; a.k_rem = t.k_rem; a.chunk_cnt = t.chunk_cnt;
+        a.out = out; a.out_stride = out_stride; a.errword = errword;
+        f.cand_cnt = t.cand_cnt; f.cand_pos = t.cand_pos; f.seg_m = t.seg_m; f.comp_off = t.comp_off;
+        f.comp_total = t.comp_total; f.comp_key = t.comp_key; f.comp_idx = t.comp_idx;
+        const dim3 gc(t.num_chunks, rows), gl(t.num_large, rows);
+        hist_kernel<0><<<gc, kSelThreads, 0, st>>>(a);
+        scan0_fast_kernel<<<gl, kSelThreads, 0, st>>>(f);
+        collect_kernel<<<gc, kSelThreads, 0, st>>>(f);
+        finish_kernel<<<gl, kFinThreads, kFinDyn, st>>>(f);
     }
     return cudaGetLastError();
 }

@@ -77,7 +77,7 @@ def test_momentum_zero_and_other_densities():
 
 @pytest.mark.parametrize("fill", ["zeros", "equal", "few_values", "denormal"])
 def test_degenerate_values(fill):
-    numel = [9000, 130, 4097, 33000]
+    numel = [9000, 130, 4097, 33000, 300001]      # the last two exceed the candidate capacity when all tie
     K = 2
     ora, gpu = make_pair(numel, K, density_ppm=20000)
     N = gpu.N
