@@ -183,7 +183,9 @@ const int64_t *lgc_keep_counts(const lgc_ctx *ctx);
 
 /* Device pointers into the caller's buffers (any may be NULL):
  *   u, v    [K][N]                     idx   [S][mu] int32, S = 1 (ring-allreduce) or K
- *   val     [K][mu]                    code  [K][c2][L2] (identity: [K][mu])
+ *   val     [K][mu] (filled by lgc_topk for the parameter server and the identity autoencoder,
+ *           else by lgc_encode / lgc_ae_train_step / lgc_topk_scatter)
+ *   code    [K][c2][L2] (identity: [K][mu])
  *   combined[c2][L2] (ring-allreduce: the mean; parameter server: the common code)
  *   inn     [K][mu] (parameter server) recon [S][mu] */
 lgc_status lgc_get_buffers(const lgc_ctx *ctx, float **u, float **v, int32_t **idx, float **val,

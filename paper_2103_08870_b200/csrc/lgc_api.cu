@@ -126,6 +126,7 @@ void carve_select(Carver &cv, SelectTables &t, int num_segments, int num_small, 
     t.cand_cnt = cv.take<int32_t>((size_t)rows * num_chunks);
     t.cand_pos = cv.take<uint16_t>((size_t)rows * num_chunks * kSelChunk);
     t.seg_m = cv.take<int32_t>((size_t)rows * num_large);
+    t.seg_ticket = cv.take<int32_t>((size_t)rows * num_large);
     t.comp_off = cv.take<int64_t>((size_t)num_large + 1);
     t.comp_total = comp_total;
     t.comp_key = cv.take<uint32_t>((size_t)rows * comp_total);
@@ -159,6 +160,7 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
     c.recon = cv.take<float>((size_t)p.S * p.mu);
     c.slot_layer = cv.take<int32_t>((size_t)p.mu);
     c.koff_dev = cv.take<int32_t>((size_t)p.L + 1);
+    c.tile_lo = cv.take<int32_t>((size_t)((p.N + 4095) / 4096) + 1);
     int sm, lg, ch;
     int64_t comp;
     count_segments(p.numel, sm, lg, ch, comp);
@@ -351,7 +353,11 @@ lgc_status lgc_topk(lgc_ctx *c, int32_t leader)
     const bool ps = c->cfg.variant == LGC_VARIANT_PS;
     if (!ps && (leader < 0 || leader >= c->K)) return fail(c, LGC_ERR_INVALID_ARG, "leader out of range");
     cudaError_t e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, c->errword, c->stream);
-    if (e == cudaSuccess) e = launch_gather(*c);
+    c->val_valid = false;
+    c->mean_valid = false;
+    c->tile_lo_valid = false;
+    // ring-allreduce with the convolutional autoencoder gathers inside the encoder launch
+    if (e == cudaSuccess && (ps || c->cfg.ae_kind == LGC_AE_IDENTITY)) e = launch_gather(*c);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_topk");
     c->last_leader = leader;
     c->stage = Ctx::kSelected;
@@ -412,7 +418,8 @@ lgc_status lgc_ae_train_step(lgc_ctx *c, float *loss_out)
     if (c->cfg.variant != LGC_VARIANT_RAR || c->cfg.ae_kind != LGC_AE_CONV2)
         return fail(c, LGC_ERR_UNSUPPORTED, "training is built for the ring-allreduce convolutional autoencoder");
     if (c->stage != Ctx::kSelected) return fail(c, LGC_ERR_BAD_STATE, "lgc_ae_train_step must follow lgc_topk");
-    const cudaError_t e = launch_train_step(*c, loss_out);
+    cudaError_t e = launch_gather(*c);
+    if (e == cudaSuccess) e = launch_train_step(*c, loss_out);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_ae_train_step");
     return LGC_OK;
 }

