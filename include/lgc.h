@@ -203,6 +203,10 @@ lgc_status lgc_get_ae_params(const lgc_ctx *ctx, float *dst, size_t count);
  * (code readable through lgc_last_error).  Clears the record. */
 lgc_status lgc_check(lgc_ctx *ctx);
 
+/* Number of kernels the library has enqueued from the calling thread since it was loaded
+ * (all contexts); the benchmark reports the difference over its timed region. */
+uint64_t lgc_kernel_launches(void);
+
 const char *lgc_status_string(lgc_status s);
 /* Text of the last failure recorded in `ctx`; with ctx == NULL, of the calling thread's last
  * failure that had no context (lgc_init).  Owned by the library, valid until the next call. */

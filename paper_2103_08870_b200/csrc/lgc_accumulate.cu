@@ -82,7 +82,7 @@ cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count
     if (want > 0x7fffffffull) return cudaErrorInvalidConfiguration;
     accumulate_kernel<<<(unsigned)want, kAccThreads, 0, s>>>(
         reinterpret_cast<const float4 *>(g), reinterpret_cast<float4 *>(u),
-        reinterpret_cast<float4 *>(v), nvec, count, m);
+        reinterpret_cast<float4 *>(v), nvec, count, m), ++g_kernel_launches;
     return cudaGetLastError();
 }
 
@@ -96,13 +96,13 @@ cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s)
         uint64_t want = (nvec + 255) / 256;
         const uint64_t cap = (uint64_t)sm_count() * 16;
         if (want > cap) want = cap;
-        zero_kernel<<<(unsigned)want, 256, 0, s>>>(reinterpret_cast<uint4 *>(p), nvec);
+        zero_kernel<<<(unsigned)want, 256, 0, s>>>(reinterpret_cast<uint4 *>(p), nvec), ++g_kernel_launches;
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     const unsigned tail = (unsigned)(bytes & 15);
     if (tail) {
-        zero_tail_kernel<<<1, 16, 0, s>>>(reinterpret_cast<unsigned char *>(p) + (nvec << 4), tail);
+        zero_tail_kernel<<<1, 16, 0, s>>>(reinterpret_cast<unsigned char *>(p) + (nvec << 4), tail), ++g_kernel_launches;
         return cudaGetLastError();
     }
     return cudaSuccess;

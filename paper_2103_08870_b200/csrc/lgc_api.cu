@@ -13,6 +13,7 @@ namespace lgc {
 
 // Message of the calling thread's last failure that had no context to be stored in.
 thread_local std::string g_last_error;
+thread_local uint64_t g_kernel_launches = 0;
 
 namespace {
 
@@ -504,6 +505,8 @@ lgc_status lgc_check(lgc_ctx *c)
     snprintf(buf, sizeof buf, "device check 0x%X: a selection kernel found inconsistent counts", (unsigned)word);
     return fail(c, LGC_ERR_DEVICE_CHECK, buf);
 }
+
+uint64_t lgc_kernel_launches(void) { return g_kernel_launches; }
 
 const char *lgc_status_string(lgc_status s)
 {

@@ -360,10 +360,10 @@ __global__ void scatter_own_kernel(const float *__restrict__ values, const int32
 inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)((n + threads - 1) / threads); }
 
 #define LGC_DISPATCH_AE(c1, c2, CALL)                                   \
-    if ((c1) == 8 && (c2) == 4) { CALL(8, 4); }                         \
-    else if ((c1) == 16 && (c2) == 8) { CALL(16, 8); }                  \
-    else if ((c1) == 4 && (c2) == 2) { CALL(4, 2); }                    \
-    else if ((c1) == 3 && (c2) == 2) { CALL(3, 2); }                    \
+    if ((c1) == 8 && (c2) == 4) { CALL(8, 4), ++g_kernel_launches; }                         \
+    else if ((c1) == 16 && (c2) == 8) { CALL(16, 8), ++g_kernel_launches; }                  \
+    else if ((c1) == 4 && (c2) == 2) { CALL(4, 2), ++g_kernel_launches; }                    \
+    else if ((c1) == 3 && (c2) == 2) { CALL(3, 2), ++g_kernel_launches; }                    \
     else return cudaErrorInvalidValue;
 
 }  // namespace
@@ -371,7 +371,7 @@ inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)((n + thre
 cudaError_t launch_gather(Ctx &c)
 {
     if (c.val_valid) return cudaSuccess;
-    gather_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S, c.mu, c.val);
+    gather_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S, c.mu, c.val), ++g_kernel_launches;
     c.val_valid = true;
     return cudaGetLastError();
 }
@@ -406,19 +406,19 @@ cudaError_t launch_encode(Ctx &c)
 cudaError_t launch_combine_mean(Ctx &c)
 {
     if (c.mean_valid) return cudaSuccess;   // the encoder launch already averaged the codes
-    mean_rows_kernel<<<blocks_for(c.code_len, 256), 256, 0, c.stream>>>(c.code, c.K, c.code_len, c.combined);
+    mean_rows_kernel<<<blocks_for(c.code_len, 256), 256, 0, c.stream>>>(c.code, c.K, c.code_len, c.combined), ++g_kernel_launches;
     return cudaGetLastError();
 }
 
 cudaError_t launch_combine_ps(Ctx &c, int common_node)
 {
     copy_kernel<<<blocks_for(c.code_len, 256), 256, 0, c.stream>>>(c.code + (int64_t)common_node * c.code_len,
-                                                                   c.code_len, c.combined);
+                                                                   c.code_len, c.combined), ++g_kernel_launches;
     cudaError_t e = launch_zero(c.inn, (size_t)c.K * c.mu * sizeof(float), c.stream);
     if (e != cudaSuccess) return e;
     e = launch_select(c.sel_inn, c.val, c.mu, 0, c.K, c.inn_pos, c.muI, c.errword, c.stream);
     if (e != cudaSuccess) return e;
-    innovation_fill_kernel<<<dim3(blocks_for(c.muI, 256), c.K), 256, 0, c.stream>>>(c.val, c.inn_pos, c.mu, c.muI, c.inn);
+    innovation_fill_kernel<<<dim3(blocks_for(c.muI, 256), c.K), 256, 0, c.stream>>>(c.val, c.inn_pos, c.mu, c.muI, c.inn), ++g_kernel_launches;
     return cudaGetLastError();
 }
 
@@ -427,10 +427,10 @@ static cudaError_t launch_scatter(Ctx &c, const float *values, float *update)
     cudaError_t e = launch_zero(update, (size_t)c.N * sizeof(float), c.stream);
     if (e != cudaSuccess) return e;
     if (c.S == 1)
-        scatter_shared_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(values, c.idx, c.mu, c.K, c.N, update, c.u, c.v);
+        scatter_shared_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(values, c.idx, c.mu, c.K, c.N, update, c.u, c.v), ++g_kernel_launches;
     else
         scatter_own_kernel<<<dim3(blocks_for(c.mu, 128), c.K), 128, 0, c.stream>>>(
-            values, c.idx, c.slot_layer, c.koff_dev, c.mu, c.K, c.N, update, c.u, c.v);
+            values, c.idx, c.slot_layer, c.koff_dev, c.mu, c.K, c.N, update, c.u, c.v), ++g_kernel_launches;
     return cudaGetLastError();
 }
 
@@ -438,17 +438,17 @@ static cudaError_t launch_scatter(Ctx &c, const float *values, float *update)
 static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update)
 {
     if (!c.tile_lo_valid) {
-        tile_lo_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(c.idx, c.mu, c.N, c.tile_lo);
+        tile_lo_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(c.idx, c.mu, c.N, c.tile_lo), ++g_kernel_launches;
         c.tile_lo_valid = true;
     }
     const unsigned grid = blocks_for(c.N, kDenseTile);
     const float *dec = c.params + c.Penc;
     if (mode == 1) {
         dense_scatter_kernel<3, 2, 1><<<grid, kDenseThreads, 0, c.stream>>>(
-            c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v);
+            c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
     } else if (mode == 2) {
         dense_scatter_kernel<3, 2, 2><<<grid, kDenseThreads, 0, c.stream>>>(
-            c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v);
+            c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
     } else {
 #define CALL(A, B) dense_scatter_kernel<A, B, 0><<<grid, kDenseThreads, 0, c.stream>>>(                               \
         c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v)
@@ -463,7 +463,7 @@ cudaError_t launch_decode_scatter(Ctx &c, float *update)
     const bool ps = c.cfg.variant == LGC_VARIANT_PS;
     if (!ps) return launch_dense_scatter(c, c.cfg.ae_kind == LGC_AE_IDENTITY ? 1 : 0, update);
     if (c.cfg.ae_kind == LGC_AE_IDENTITY) {
-        identity_ps_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.combined, c.inn, c.mu, c.recon);
+        identity_ps_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.combined, c.inn, c.mu, c.recon), ++g_kernel_launches;
     } else {
         const dim3 grid(blocks_for(c.mu, kAeThreads), c.S);
         const float *dec = c.params + c.Penc;

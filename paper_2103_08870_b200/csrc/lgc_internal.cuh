@@ -102,6 +102,7 @@ struct Ctx {
     std::string err;
 };
 
+extern thread_local uint64_t g_kernel_launches;   // kernels this thread has enqueued (lgc_kernel_launches)
 extern thread_local std::string g_last_error;   // failures without a context (see lgc_last_error)
 
 // ---- launchers (each enqueues on ctx stream and returns the launch status) -------------------

@@ -98,7 +98,7 @@ extern "C" lgc_status lgc_topk_noalloc(const float *v, int64_t n, int64_t k, int
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool small = n <= kSelChunk;
     const int chunks = small ? 0 : (int)((n + kSelChunk - 1) / kSelChunk);
-    noalloc_setup_kernel<<<8, 256, 0, s>>>(base, (int32_t)n, (int32_t)k, chunks);
+    noalloc_setup_kernel<<<8, 256, 0, s>>>(base, (int32_t)n, (int32_t)k, chunks), ++g_kernel_launches;
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(LGC_ERR_CUDA, std::string("lgc_topk_noalloc: ") + cudaGetErrorString(e));
     SelectTables t;

@@ -689,7 +689,7 @@ cudaError_t launch_select_multipass(const SelectTables &t, const float *data, in
     if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
     if (t.num_small) {
         select_small_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(
-            data, row_stride, row0, t.seg_off, t.seg_len, t.seg_k, t.seg_out, t.small_ids, out, out_stride, errword);
+            data, row_stride, row0, t.seg_off, t.seg_len, t.seg_k, t.seg_out, t.small_ids, out, out_stride, errword), ++g_kernel_launches;
     }
     if (t.num_large) {
         LargeArgs a;
@@ -700,15 +700,15 @@ cudaError_t launch_select_multipass(const SelectTables &t, const float *data, in
         a.hist = t.hist; a.prefix = t.prefix; a.k_rem = t.k_rem; a.chunk_cnt = t.chunk_cnt;
         a.out = out; a.out_stride = out_stride; a.errword = errword;
         const dim3 gc(t.num_chunks, rows), gl(t.num_large, rows);
-        hist_kernel<0><<<gc, kSelThreads, 0, st>>>(a);
-        scan_kernel<0><<<gl, kSelThreads, 0, st>>>(a);
-        hist_kernel<1><<<gc, kSelThreads, 0, st>>>(a);
-        scan_kernel<1><<<gl, kSelThreads, 0, st>>>(a);
-        hist_kernel<2><<<gc, kSelThreads, 0, st>>>(a);
-        scan_kernel<2><<<gl, kSelThreads, 0, st>>>(a);
-        count_kernel<<<gc, kSelThreads, 0, st>>>(a);
-        chunk_scan_kernel<<<gl, kSelThreads, 0, st>>>(a);
-        emit_kernel<<<gc, kSelThreads, 0, st>>>(a);
+        hist_kernel<0><<<gc, kSelThreads, 0, st>>>(a), ++g_kernel_launches;
+        scan_kernel<0><<<gl, kSelThreads, 0, st>>>(a), ++g_kernel_launches;
+        hist_kernel<1><<<gc, kSelThreads, 0, st>>>(a), ++g_kernel_launches;
+        scan_kernel<1><<<gl, kSelThreads, 0, st>>>(a), ++g_kernel_launches;
+        hist_kernel<2><<<gc, kSelThreads, 0, st>>>(a), ++g_kernel_launches;
+        scan_kernel<2><<<gl, kSelThreads, 0, st>>>(a), ++g_kernel_launches;
+        count_kernel<<<gc, kSelThreads, 0, st>>>(a), ++g_kernel_launches;
+        chunk_scan_kernel<<<gl, kSelThreads, 0, st>>>(a), ++g_kernel_launches;
+        emit_kernel<<<gc, kSelThreads, 0, st>>>(a), ++g_kernel_launches;
     }
     return cudaGetLastError();
 }
@@ -722,7 +722,7 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
         return launch_select_multipass(t, data, row_stride, row0, rows, out, out_stride, errword, st);
     if (!t.num_large) {
         select_small_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(
-            data, row_stride, row0, t.seg_off, t.seg_len, t.seg_k, t.seg_out, t.small_ids, out, out_stride, errword);
+            data, row_stride, row0, t.seg_off, t.seg_len, t.seg_k, t.seg_out, t.small_ids, out, out_stride, errword), ++g_kernel_launches;
     } else {
         constexpr int kFinDyn = 2 * kFinSmemCap * (int)sizeof(uint32_t);
         static bool configured = false;
@@ -743,9 +743,9 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
         f.comp_off = t.comp_off;
         f.comp_total = t.comp_total; f.comp_key = t.comp_key; f.comp_idx = t.comp_idx;
         const dim3 gc(t.num_chunks, rows), gl(t.num_large, rows);
-        hist0_fast_kernel<<<gc, kSelThreads, 0, st>>>(f);
-        collect_small_kernel<<<dim3(t.num_chunks + t.num_small, rows), kSelThreads, 0, st>>>(f, t.small_ids, t.num_small);
-        finish_kernel<<<gl, kFinThreads, kFinDyn, st>>>(f);
+        hist0_fast_kernel<<<gc, kSelThreads, 0, st>>>(f), ++g_kernel_launches;
+        collect_small_kernel<<<dim3(t.num_chunks + t.num_small, rows), kSelThreads, 0, st>>>(f, t.small_ids, t.num_small), ++g_kernel_launches;
+        finish_kernel<<<gl, kFinThreads, kFinDyn, st>>>(f), ++g_kernel_launches;
     }
     return cudaGetLastError();
 }

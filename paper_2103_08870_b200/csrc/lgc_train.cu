@@ -307,17 +307,17 @@ cudaError_t train_step(Ctx &c, float *loss_out, const AdamArgs &ad)
     cudaStream_t s = c.stream;
     const float *enc = c.params, *dec = c.params + c.Penc;
     const float *dec_w2 = dec + C2 * C1 * 3 + C1;
-    fwd_enc1_kernel<C1><<<dim3(blocks_for(c.L1, kTrThreads), c.K), kTrThreads, 0, s>>>(c.val, c.mu, c.L1, enc, c.t_h);
-    fwd_enc2_mean_kernel<C1, C2><<<blocks_for(c.L2, kTrThreads), kTrThreads, 0, s>>>(c.t_h, c.K, c.L1, c.L2, enc, c.combined);
-    fwd_dec1_kernel<C1, C2><<<blocks_for(c.L1, kTrThreads), kTrThreads, 0, s>>>(c.combined, c.L1, c.L2, dec, c.t_d);
+    fwd_enc1_kernel<C1><<<dim3(blocks_for(c.L1, kTrThreads), c.K), kTrThreads, 0, s>>>(c.val, c.mu, c.L1, enc, c.t_h), ++g_kernel_launches;
+    fwd_enc2_mean_kernel<C1, C2><<<blocks_for(c.L2, kTrThreads), kTrThreads, 0, s>>>(c.t_h, c.K, c.L1, c.L2, enc, c.combined), ++g_kernel_launches;
+    fwd_dec1_kernel<C1, C2><<<blocks_for(c.L1, kTrThreads), kTrThreads, 0, s>>>(c.combined, c.L1, c.L2, dec, c.t_d), ++g_kernel_launches;
     fwd_dec2_loss_kernel<C1><<<c.t_loss_blocks, kTrThreads, 0, s>>>(c.t_d, c.val, c.K, c.mu, c.L1, dec_w2, c.recon,
-                                                                     c.t_dr, c.t_loss_part);
-    bwd_dec2_kernel<C1><<<blocks_for(c.L1, kTrThreads), kTrThreads, 0, s>>>(c.t_dr, c.t_d, c.L1, dec_w2, c.t_dd);
-    bwd_dec1_kernel<C1, C2><<<blocks_for(c.L2, kTrThreads), kTrThreads, 0, s>>>(c.t_dd, c.K, c.L1, c.L2, dec, c.t_dz);
-    bwd_enc2_kernel<C1, C2><<<dim3(blocks_for(c.L1, kTrThreads), c.K), kTrThreads, 0, s>>>(c.t_dz, c.t_h, c.L1, c.L2, enc, c.t_dh);
+                                                                     c.t_dr, c.t_loss_part), ++g_kernel_launches;
+    bwd_dec2_kernel<C1><<<blocks_for(c.L1, kTrThreads), kTrThreads, 0, s>>>(c.t_dr, c.t_d, c.L1, dec_w2, c.t_dd), ++g_kernel_launches;
+    bwd_dec1_kernel<C1, C2><<<blocks_for(c.L2, kTrThreads), kTrThreads, 0, s>>>(c.t_dd, c.K, c.L1, c.L2, dec, c.t_dz), ++g_kernel_launches;
+    bwd_enc2_kernel<C1, C2><<<dim3(blocks_for(c.L1, kTrThreads), c.K), kTrThreads, 0, s>>>(c.t_dz, c.t_h, c.L1, c.L2, enc, c.t_dh), ++g_kernel_launches;
     param_grad_adam_kernel<C1, C2><<<(unsigned)c.P, kRedThreads, 0, s>>>(c.val, c.t_h, c.combined, c.t_d, c.t_dr, c.t_dd,
-                                                                        c.t_dz, c.t_dh, c.K, c.mu, c.L1, c.L2, ad);
-    if (loss_out) loss_finalize_kernel<<<1, kRedThreads, 0, s>>>(c.t_loss_part, c.t_loss_blocks, c.mu, loss_out);
+                                                                        c.t_dz, c.t_dh, c.K, c.mu, c.L1, c.L2, ad), ++g_kernel_launches;
+    if (loss_out) loss_finalize_kernel<<<1, kRedThreads, 0, s>>>(c.t_loss_part, c.t_loss_blocks, c.mu, loss_out), ++g_kernel_launches;
     return cudaGetLastError();
 }
 

@@ -23,7 +23,7 @@ EXPORTS = (
     "lgc_workspace_bytes", "lgc_init", "lgc_destroy", "lgc_accumulate", "lgc_topk", "lgc_encode",
     "lgc_combine", "lgc_decode_scatter", "lgc_topk_scatter", "lgc_ae_train_step", "lgc_step_host",
     "lgc_get_layout", "lgc_keep_counts", "lgc_get_buffers", "lgc_set_ae_params", "lgc_get_ae_params",
-    "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc",
+    "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc", "lgc_kernel_launches",
 )
 NOALLOC_MAX_N = 16777216
 
@@ -72,6 +72,8 @@ def lib() -> C.CDLL:
         l.lgc_last_error.argtypes = [vp]
         l.lgc_last_error.restype = C.c_char_p
         l.lgc_topk_noalloc.argtypes = [vp, C.c_int64, C.c_int64, vp, vp]
+        l.lgc_kernel_launches.argtypes = []
+        l.lgc_kernel_launches.restype = C.c_uint64
         for name in EXPORTS:            # every declared entry point must be exported
             getattr(l, name)
         _lib = l
@@ -97,6 +99,11 @@ def topk_noalloc(v: torch.Tensor, k: int, idx_out: torch.Tensor, stream: Optiona
     st = lib().lgc_topk_noalloc(v.data_ptr(), v.numel(), k, idx_out.data_ptr(), C.c_void_p(s.cuda_stream))
     if st != LGC_OK:
         raise LGCError(st, "lgc_topk_noalloc", lib().lgc_last_error(None).decode())
+
+
+def kernel_launches() -> int:
+    """Kernels the library has enqueued from this thread so far."""
+    return int(lib().lgc_kernel_launches())
 
 
 def status_string(status: int) -> str:
