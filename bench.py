@@ -208,7 +208,7 @@ def run_ours(args, w: W.Workload):
     for t in range(args.steps):
         i = args.warmup + t
         ev[t][0].record()
-        gpu.accumulate(grads[i % GRAD_SETS])
+        gpu.accumulate(grads[i % GRAD_SETS], choices[i])
         ev[t][1].record()
         gpu.topk(choices[i])
         gpu.encode()

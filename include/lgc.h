@@ -96,8 +96,13 @@ lgc_status lgc_destroy(lgc_ctx *ctx);
 
 /* Stage 1 -- Algorithm 1/2, local accumulation, with the momentum correction of Section V-A:
  *     u <- m * u + g (one fused rounding);  v <- v + u          for every node and element.
- * grads: device, fp32 [K][N], read only. */
-lgc_status lgc_accumulate(lgc_ctx *ctx, const float *grads);
+ * grads: device, fp32 [K][N], read only.
+ * leader_hint (ring-allreduce only; ignored for the parameter server): the node that lgc_topk
+ * will be given as leader in this step, or -1 if not known yet.  With a hint the kernel also
+ * collects that node's selection candidates while it streams (against a threshold predicted from
+ * the previous step and verified afterwards), which saves lgc_topk its reads of v.  The hint
+ * never changes a result: a wrong or missing hint only makes lgc_topk do the reads itself. */
+lgc_status lgc_accumulate(lgc_ctx *ctx, const float *grads, int32_t leader_hint);
 
 /* Stages 2+3 -- Section V-A, Algorithm 1/2 (threshold, mask, concatenation): per layer the k_l
  * entries of largest |v| (equal magnitudes: the lower index wins), in ascending index order,

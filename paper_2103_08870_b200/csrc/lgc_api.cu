@@ -107,45 +107,83 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
     return LGC_OK;
 }
 
-void carve_select(Carver &cv, SelectTables &t, int num_segments, int num_small, int num_large, int num_chunks,
-                  int64_t comp_total, int rows)
-{
-    t.num_segments = num_segments; t.num_small = num_small; t.num_large = num_large; t.num_chunks = num_chunks;
-    t.max_rows = rows;
-    t.seg_off = cv.take<int64_t>(num_segments);
-    t.seg_len = cv.take<int32_t>(num_segments);
-    t.seg_k = cv.take<int32_t>(num_segments);
-    t.seg_out = cv.take<int32_t>(num_segments);
-    t.small_ids = cv.take<int32_t>(num_small);
-    t.large_ids = cv.take<int32_t>(num_large);
-    t.large_chunk0 = cv.take<int32_t>(num_large + 1);
-    t.chunk_large = cv.take<int32_t>(num_chunks);
-    t.hist = cv.take<uint32_t>((size_t)rows * num_large * kHistBins);
-    t.prefix = cv.take<uint32_t>((size_t)rows * num_large);
-    t.k_rem = cv.take<int32_t>((size_t)rows * num_large);
-    t.chunk_cnt = cv.take<int2>((size_t)rows * num_chunks);
-    t.cand_cnt = cv.take<int32_t>((size_t)rows * num_chunks);
-    t.cand_pos = cv.take<uint16_t>((size_t)rows * num_chunks * kSelChunk);
-    t.seg_m = cv.take<int32_t>((size_t)rows * num_large);
-    t.seg_ticket = cv.take<int32_t>((size_t)rows * num_large);
-    t.comp_off = cv.take<int64_t>((size_t)num_large + 1);
-    t.comp_total = comp_total;
-    t.comp_key = cv.take<uint32_t>((size_t)rows * comp_total);
-    t.comp_idx = cv.take<int32_t>((size_t)rows * comp_total);
-}
+// Host-side description of one selection family: which segments are small or large, and how the
+// large ones are cut by the row's tiles of kSelChunk elements.
+struct SelectPlan {
+    std::vector<int64_t> seg_off, comp_off;
+    std::vector<int32_t> seg_len, seg_k, seg_out, small_ids, large_ids, seg_large, large_q0, tchunk0, tchunk_large,
+        tile_seg0;
+    int tiles_per_row = 0;
+    int64_t comp_total = 0;
+};
 
-void count_segments(const std::vector<int64_t> &len, int &small, int &large, int &chunks, int64_t &comp_total)
+SelectPlan plan_select(const std::vector<int64_t> &off, const std::vector<int64_t> &len, const std::vector<int64_t> &k,
+                       const std::vector<int64_t> &out_off)
 {
-    small = large = chunks = 0;
-    comp_total = 0;
-    for (int64_t n : len) {
-        if (n <= kSelChunk) ++small;
-        else {
-            ++large;
-            chunks += (int)((n + kSelChunk - 1) / kSelChunk);
-            comp_total += select_compact_capacity(n);
+    SelectPlan sp;
+    const int n = (int)len.size();
+    sp.comp_off.push_back(0);
+    sp.tchunk0.push_back(0);
+    for (int i = 0; i < n; ++i) {
+        sp.seg_off.push_back(off[i]);
+        sp.seg_len.push_back((int32_t)len[i]);
+        sp.seg_k.push_back((int32_t)k[i]);
+        sp.seg_out.push_back((int32_t)out_off[i]);
+        if (len[i] <= kSelChunk) {
+            sp.small_ids.push_back(i);
+            sp.seg_large.push_back(-1);
+        } else {
+            const int li = (int)sp.large_ids.size();
+            sp.large_ids.push_back(i);
+            sp.seg_large.push_back(li);
+            const int64_t q0 = off[i] / kSelChunk, q1 = (off[i] + len[i] - 1) / kSelChunk;
+            sp.large_q0.push_back((int32_t)q0);
+            for (int64_t q = q0; q <= q1; ++q) sp.tchunk_large.push_back(li);
+            sp.tchunk0.push_back((int32_t)sp.tchunk_large.size());
+            sp.comp_off.push_back(sp.comp_off.back() + select_compact_capacity(len[i]));
         }
     }
+    sp.comp_total = sp.comp_off.back();
+    const int64_t row_len = off[n - 1] + len[n - 1];
+    sp.tiles_per_row = (int)((row_len + kSelChunk - 1) / kSelChunk);
+    int s = 0;
+    for (int q = 0; q < sp.tiles_per_row; ++q) {
+        while (off[s] + len[s] <= (int64_t)q * kSelChunk) ++s;     // first segment that reaches into tile q
+        sp.tile_seg0.push_back(s);
+    }
+    return sp;
+}
+
+void carve_select(Carver &cv, SelectTables &t, const SelectPlan &sp, int rows)
+{
+    const int S = (int)sp.seg_len.size(), ns = (int)sp.small_ids.size(), nl = (int)sp.large_ids.size();
+    const int nc = (int)sp.tchunk_large.size();
+    t.num_segments = S; t.num_small = ns; t.num_large = nl; t.num_tchunks = nc; t.tiles_per_row = sp.tiles_per_row;
+    t.max_rows = rows;
+    t.seg_off = cv.take<int64_t>(S);
+    t.seg_len = cv.take<int32_t>(S);
+    t.seg_k = cv.take<int32_t>(S);
+    t.seg_out = cv.take<int32_t>(S);
+    t.seg_large = cv.take<int32_t>(S);
+    t.small_ids = cv.take<int32_t>(ns);
+    t.large_ids = cv.take<int32_t>(nl);
+    t.large_q0 = cv.take<int32_t>(nl);
+    t.tchunk0 = cv.take<int32_t>(nl + 1);
+    t.tchunk_large = cv.take<int32_t>(nc);
+    t.tile_seg0 = cv.take<int32_t>(sp.tiles_per_row);
+    t.hist = cv.take<uint32_t>((size_t)rows * nl * kHistBins);
+    t.prefix = cv.take<uint32_t>((size_t)rows * nl);
+    t.k_rem = cv.take<int32_t>((size_t)rows * nl);
+    t.seg_m = cv.take<int32_t>((size_t)rows * nl);
+    t.seg_ticket = cv.take<int32_t>((size_t)rows * nl);
+    t.seg_epoch = cv.take<int32_t>((size_t)rows * nl);
+    t.lb = cv.take<int32_t>((size_t)rows * nl);
+    t.cand_cnt = cv.take<int32_t>((size_t)rows * nc);
+    t.cand_pos = cv.take<uint16_t>((size_t)rows * nc * kSelChunk);
+    t.comp_off = cv.take<int64_t>((size_t)nl + 1);
+    t.comp_total = sp.comp_total;
+    t.comp_key = cv.take<uint32_t>((size_t)rows * sp.comp_total);
+    t.comp_idx = cv.take<int32_t>((size_t)rows * sp.comp_total);
 }
 
 // Lays every sub-buffer of the scratch out; identical for measuring and for real.
@@ -162,15 +200,11 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
     c.slot_layer = cv.take<int32_t>((size_t)p.mu);
     c.koff_dev = cv.take<int32_t>((size_t)p.L + 1);
     c.tile_lo = cv.take<int32_t>((size_t)((p.N + 4095) / 4096) + 1);
-    int sm, lg, ch;
-    int64_t comp;
-    count_segments(p.numel, sm, lg, ch, comp);
-    carve_select(cv, c.sel_v, p.L, sm, lg, ch, comp, p.S);
+    carve_select(cv, c.sel_v, plan_select(p.off, p.numel, p.k_l, p.koff), p.S);
     if (ps) {
         c.inn = cv.take<float>((size_t)p.K * p.mu);
         c.inn_pos = cv.take<int32_t>((size_t)p.K * p.muI);
-        count_segments(p.k_l, sm, lg, ch, comp);
-        carve_select(cv, c.sel_inn, p.L, sm, lg, ch, comp, p.K);
+        carve_select(cv, c.sel_inn, plan_select(p.koff, p.k_l, p.ki_l, p.kioff), p.K);
     }
     if (conv && !ps) {
         const size_t c1 = cfg.ae_c1, c2 = cfg.ae_c2;
@@ -205,41 +239,19 @@ cudaError_t upload(T *dst, const std::vector<T> &src, cudaStream_t s)
     return cudaMemcpyAsync(dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice, s);
 }
 
-// Fills and uploads the tables of one selection family; `hold` keeps the host copies alive until
-// the stream has been synchronised.
-cudaError_t upload_select(SelectTables &t, const std::vector<int64_t> &off, const std::vector<int64_t> &len,
-                          const std::vector<int64_t> &k, const std::vector<int64_t> &out_off, cudaStream_t s,
-                          std::vector<std::vector<int32_t>> &hold32, std::vector<std::vector<int64_t>> &hold64)
+// Uploads the tables of one selection family; `hold` keeps the host copies alive until the
+// stream has been synchronised.
+cudaError_t upload_select(SelectTables &t, SelectPlan sp, cudaStream_t s, std::vector<SelectPlan> &hold)
 {
-    const int n = (int)len.size();
-    std::vector<int64_t> h_off(off.begin(), off.begin() + n);
-    std::vector<int32_t> h_len(n), h_k(n), h_out(n), small_ids, large_ids, chunk0, chunk_large;
-    std::vector<int64_t> comp_off(1, 0);
-    chunk0.push_back(0);
-    for (int i = 0; i < n; ++i) {
-        h_len[i] = (int32_t)len[i];
-        h_k[i] = (int32_t)k[i];
-        h_out[i] = (int32_t)out_off[i];
-        if (len[i] <= kSelChunk) small_ids.push_back(i);
-        else {
-            const int li = (int)large_ids.size();
-            large_ids.push_back(i);
-            const int nc = (int)((len[i] + kSelChunk - 1) / kSelChunk);
-            for (int q = 0; q < nc; ++q) chunk_large.push_back(li);
-            chunk0.push_back(chunk0.back() + nc);
-            comp_off.push_back(comp_off.back() + select_compact_capacity(len[i]));
-        }
-    }
-    hold64.push_back(std::move(h_off));
-    cudaError_t e = upload(t.seg_off, hold64.back(), s);
-    hold64.push_back(std::move(comp_off));
-    if (e == cudaSuccess) e = upload(t.comp_off, hold64.back(), s);
-    std::vector<int32_t> *arrs[] = {&h_len, &h_k, &h_out, &small_ids, &large_ids, &chunk0, &chunk_large};
-    int32_t *dsts[] = {t.seg_len, t.seg_k, t.seg_out, t.small_ids, t.large_ids, t.large_chunk0, t.chunk_large};
-    for (int i = 0; i < 7 && e == cudaSuccess; ++i) {
-        hold32.push_back(std::move(*arrs[i]));
-        e = upload(dsts[i], hold32.back(), s);
-    }
+    hold.push_back(std::move(sp));
+    const SelectPlan &h = hold.back();
+    cudaError_t e = upload(t.seg_off, h.seg_off, s);
+    if (e == cudaSuccess) e = upload(t.comp_off, h.comp_off, s);
+    const std::vector<int32_t> *arrs[] = {&h.seg_len, &h.seg_k, &h.seg_out, &h.seg_large, &h.small_ids, &h.large_ids,
+                                          &h.large_q0, &h.tchunk0, &h.tchunk_large, &h.tile_seg0};
+    int32_t *dsts[] = {t.seg_len, t.seg_k, t.seg_out, t.seg_large, t.small_ids, t.large_ids,
+                       t.large_q0, t.tchunk0, t.tchunk_large, t.tile_seg0};
+    for (int i = 0; i < 10 && e == cudaSuccess; ++i) e = upload(dsts[i], *arrs[i], s);
     return e;
 }
 
@@ -305,13 +317,11 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     cudaError_t e = launch_zero(state, need_state, s);
     if (e == cudaSuccess) e = launch_zero(scratch, need_scratch, s);
     if (e == cudaSuccess && p.P > 0) e = launch_zero(c->adam_m, (size_t)2 * pad4(p.P) * sizeof(float), s);
-    std::vector<std::vector<int32_t>> hold32;
-    std::vector<std::vector<int64_t>> hold64;
-    hold32.reserve(32);
-    hold64.reserve(8);
-    if (e == cudaSuccess) e = upload_select(c->sel_v, p.off, p.numel, p.k_l, p.koff, s, hold32, hold64);
+    std::vector<SelectPlan> hold;
+    hold.reserve(2);
+    if (e == cudaSuccess) e = upload_select(c->sel_v, plan_select(p.off, p.numel, p.k_l, p.koff), s, hold);
     if (e == cudaSuccess && cfg->variant == LGC_VARIANT_PS)
-        e = upload_select(c->sel_inn, p.koff, p.k_l, p.ki_l, p.kioff, s, hold32, hold64);
+        e = upload_select(c->sel_inn, plan_select(p.koff, p.k_l, p.ki_l, p.kioff), s, hold);
     std::vector<int32_t> slot_layer((size_t)p.mu), koff32((size_t)p.L + 1);
     for (int l = 0; l < p.L; ++l) {
         koff32[l] = (int32_t)p.koff[l];
@@ -336,12 +346,24 @@ lgc_status lgc_destroy(lgc_ctx *ctx)
     return LGC_OK;
 }
 
-lgc_status lgc_accumulate(lgc_ctx *c, const float *grads)
+lgc_status lgc_accumulate(lgc_ctx *c, const float *grads, int32_t leader_hint)
 {
     if (!c) return LGC_ERR_INVALID_ARG;
     if (!grads || !aligned16(grads)) return fail(c, LGC_ERR_INVALID_ARG, "grads is NULL or not 16-byte aligned");
     if (c->stage != Ctx::kIdle) return fail(c, LGC_ERR_BAD_STATE, "lgc_accumulate must open a step");
-    const cudaError_t e = launch_accumulate(grads, c->u, c->v, (uint64_t)c->K * (uint64_t)c->N, c->cfg.momentum, c->stream);
+    const bool ps = c->cfg.variant == LGC_VARIANT_PS;
+    if (!ps && leader_hint >= c->K) return fail(c, LGC_ERR_INVALID_ARG, "leader_hint out of range");
+    c->epoch = c->epoch == 0x7fffffff ? 1 : c->epoch + 1;
+    cudaError_t e;
+    // the fused form needs rows that start 16-byte aligned and someone to select for
+    if (c->N % 4 == 0 && c->sel_v.num_large > 0 && (ps || leader_hint >= 0)) {
+        e = launch_accumulate_select(c->sel_v, grads, c->u, c->v, c->K, c->N, c->cfg.momentum, ps ? 0 : leader_hint,
+                                     ps ? c->K : 1, c->epoch, c->errword, c->stream);
+        c->fused_leader = ps ? -1 : leader_hint;
+    } else {
+        e = launch_accumulate(grads, c->u, c->v, (uint64_t)c->K * (uint64_t)c->N, c->cfg.momentum, c->stream);
+        c->fused_leader = -2;
+    }
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_accumulate");
     c->stage = Ctx::kAccumulated;
     return LGC_OK;
@@ -353,7 +375,10 @@ lgc_status lgc_topk(lgc_ctx *c, int32_t leader)
     if (c->stage != Ctx::kAccumulated) return fail(c, LGC_ERR_BAD_STATE, "lgc_topk must follow lgc_accumulate");
     const bool ps = c->cfg.variant == LGC_VARIANT_PS;
     if (!ps && (leader < 0 || leader >= c->K)) return fail(c, LGC_ERR_INVALID_ARG, "leader out of range");
-    cudaError_t e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, c->errword, c->stream);
+    // candidates collected during the accumulation count only if they are this leader's
+    const bool fused = ps ? c->fused_leader == -1 : c->fused_leader == leader;
+    cudaError_t e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, fused ? c->epoch : -1,
+                                  c->errword, c->stream);
     c->val_valid = false;
     c->mean_valid = false;
     c->tile_lo_valid = false;
@@ -433,7 +458,7 @@ lgc_status lgc_step_host(lgc_ctx *c, const float *host_grads, float *dev_grads, 
     if (c->stage != Ctx::kIdle) return fail(c, LGC_ERR_BAD_STATE, "lgc_step_host must open a step");
     cudaError_t e = cudaMemcpyAsync(dev_grads, host_grads, (size_t)c->K * c->N * sizeof(float), cudaMemcpyHostToDevice, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (upload)");
-    lgc_status st = lgc_accumulate(c, dev_grads);
+    lgc_status st = lgc_accumulate(c, dev_grads, choice);
     if (st == LGC_OK) st = lgc_topk(c, choice);
     if (st == LGC_OK) st = lgc_encode(c);
     if (st == LGC_OK) st = lgc_combine(c, choice);

@@ -19,35 +19,46 @@ constexpr int kHistBins = 2048;    // first radix digit: 11 bits; the next two: 
 
 // One selection problem family: R rows of `data` (row stride in elements), each cut into the same
 // segments; per segment the k entries of largest |x| are reported, ascending, as int32 offsets.
+// All pointers are device memory.
 struct SelectTables {
     int num_segments = 0;
     int num_small = 0;            // segments of at most kSelChunk elements
     int num_large = 0;
-    int num_chunks = 0;           // chunks of all large segments
-    // device tables (all in the caller's scratch)
+    int max_rows = 0;
     int64_t *seg_off = nullptr;   // [S] first element of the segment inside a row
     int32_t *seg_len = nullptr;   // [S]
     int32_t *seg_k = nullptr;     // [S]
     int32_t *seg_out = nullptr;   // [S] first output slot of the segment
     int32_t *small_ids = nullptr; // [num_small] segment ids
     int32_t *large_ids = nullptr; // [num_large] segment ids
-    int32_t *large_chunk0 = nullptr; // [num_large + 1] first chunk of each large segment
-    int32_t *chunk_large = nullptr;  // [num_chunks] index into large_ids
-    // per-call work space, sized for max_rows rows
-    int max_rows = 0;
     uint32_t *hist = nullptr;     // [rows][num_large][kHistBins], all zero between passes
     uint32_t *prefix = nullptr;   // [rows][num_large] key prefix found so far
     int32_t *k_rem = nullptr;     // [rows][num_large] entries still to find at the prefix
-    int2 *chunk_cnt = nullptr;    // [rows][num_chunks] (#key > T, #key == T), then exclusive prefix
-    // two-pass path (launch_select): candidates of every chunk, and their compacted form
-    int32_t *cand_cnt = nullptr;  // [rows][num_chunks] candidates found in the chunk
-    uint16_t *cand_pos = nullptr; // [rows][num_chunks][kSelChunk] their positions inside the chunk, ascending
-    int32_t *seg_m = nullptr;     // [rows][num_large] entries at or above the bucket of the k-th key
-    int32_t *seg_ticket = nullptr; // [rows][num_large] chunks that have added their histogram; zero between calls
-    int64_t *comp_off = nullptr;  // [num_large + 1] first compact slot of each large segment
-    int64_t comp_total = 0;       // compact slots per row
-    uint32_t *comp_key = nullptr; // [rows][comp_total] keys of the candidates, index order
-    int32_t *comp_idx = nullptr;  // [rows][comp_total] their offsets inside the row
+
+    // -- launch_select_multipass: chunks of kSelChunk elements counted from each segment's start
+    int num_chunks = 0;
+    int32_t *large_chunk0 = nullptr; // [num_large + 1] first chunk of each large segment
+    int32_t *chunk_large = nullptr;  // [num_chunks] index into large_ids
+    int2 *chunk_cnt = nullptr;       // [rows][num_chunks] (#key > T, #key == T), then exclusive prefix
+
+    // -- launch_select: chunks are the intersections of a segment with the row's 4096-element tiles
+    int num_tchunks = 0;
+    int tiles_per_row = 0;
+    int32_t *seg_large = nullptr;    // [S] index into large_ids, -1 for small segments
+    int32_t *large_q0 = nullptr;     // [num_large] first tile the segment overlaps
+    int32_t *tchunk0 = nullptr;      // [num_large + 1] first tile-chunk of each large segment
+    int32_t *tchunk_large = nullptr; // [num_tchunks] index into large_ids
+    int32_t *tile_seg0 = nullptr;    // [tiles_per_row] first segment a tile overlaps
+    int32_t *cand_cnt = nullptr;     // [rows][num_tchunks] candidates found in the chunk
+    uint16_t *cand_pos = nullptr;    // [rows][num_tchunks][kSelChunk] their positions inside the tile, ascending
+    int32_t *seg_m = nullptr;        // [rows][num_large] candidates of the segment
+    int32_t *seg_ticket = nullptr;   // [rows][num_large] chunks that have reported; zero between passes
+    int32_t *seg_epoch = nullptr;    // [rows][num_large] step whose accumulation already produced the candidates
+    int32_t *lb = nullptr;           // [rows][num_large] predicted lower bucket for the next step (0: none)
+    int64_t *comp_off = nullptr;     // [num_large + 1] first compact slot of each large segment
+    int64_t comp_total = 0;          // compact slots per row
+    uint32_t *comp_key = nullptr;    // [rows][comp_total] keys of the candidates, index order
+    int32_t *comp_idx = nullptr;     // [rows][comp_total] their offsets inside the row
 };
 
 // Compact-array capacity of a large segment of n elements: above it the segment is finished by
@@ -96,6 +107,8 @@ struct Ctx {
     // step state machine
     enum Stage { kIdle, kAccumulated, kSelected, kEncoded, kCombined } stage = kIdle;
     int32_t last_leader = 0;
+    int32_t epoch = 0;             // step counter (accumulations so far)
+    int32_t fused_leader = -2;     // row whose candidates the last accumulation collected (-1: all rows, -2: none)
     bool val_valid = false;        // val holds the kept values of the current selection
     bool tile_lo_valid = false;    // tile_lo matches the current selection
     bool mean_valid = false;       // combined holds the mean code of the current selection
@@ -108,8 +121,15 @@ extern thread_local std::string g_last_error;   // failures without a context (s
 // ---- launchers (each enqueues on ctx stream and returns the launch status) -------------------
 cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s);
 cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s);
+// epoch: the step whose fused accumulation may already hold candidates (-1: none).
 cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0,
-                          int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t s);
+                          int rows, int32_t *out, int64_t out_stride, int32_t epoch, int32_t *errword,
+                          cudaStream_t s);
+// Accumulation that also collects the selection candidates of the selecting rows (sel_row0 .. +sel_rows
+// of the K rows) against the predicted buckets; needs N % 4 == 0.
+cudaError_t launch_accumulate_select(const SelectTables &t, const float *g, float *u, float *v, int K, int64_t N,
+                                     float m, int sel_row0, int sel_rows, int32_t epoch, int32_t *errword,
+                                     cudaStream_t s);
 cudaError_t launch_select_multipass(const SelectTables &t, const float *data, int64_t row_stride, int row0,
                                     int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t s);
 cudaError_t launch_gather(Ctx &c);

@@ -1,0 +1,539 @@
+// The selection path the LGC step uses (Section V-A of the paper: per layer, the alpha% entries
+// of largest magnitude), built to touch the residual v as little as possible.
+//
+// A large segment (layer) of a row is cut where the row's 4096-element tiles cut it.  For every
+// such chunk the positions of its CANDIDATES are kept, ascending: the entries whose leading key
+// digit (11 bits: exponent + 3 mantissa bits) is at least a lower bucket.  One CTA per segment
+// then compacts the candidates in index order, finishes the radix search on them and emits the
+// k selected offsets by counting -- exact, ties to the lower index, no sorting.
+//
+// Where the candidates come from:
+//  (a) fused: the accumulation kernel (accumulate_select_kernel, below) tests the freshly written
+//      v of the selecting rows against a bucket PREDICTED from the previous step, histograms the
+//      entries that pass, and the CTA that completes a segment (a ticket counter tells; nobody
+//      waits) checks that at least k entries passed.  Then no further read of v is needed.
+//  (b) otherwise (first step, prediction too high, leader not announced, N not a multiple of 4):
+//      hist0_fast_kernel histograms the segment, the completing CTA finds the bucket of the k-th
+//      key, and collect_small_kernel gathers the candidates: two reads of v.
+// A segment whose candidates exceed its compact capacity (ties, e.g. a layer of zeros) is
+// finished by its CTA streaming over the data instead.  Either way the result is exact.
+#include "lgc_select_common.cuh"
+
+namespace lgc {
+
+namespace {
+
+using namespace sel;
+
+struct FastArgs {
+    const float *data;
+    int64_t row_stride;
+    int row0;
+    int num_large, num_small, num_tchunks;
+    int32_t epoch;                 // step whose fused accumulation may have filled the lists (-1: none)
+    const int64_t *seg_off;
+    const int32_t *seg_len, *seg_k, *seg_out, *small_ids, *large_ids, *seg_large, *large_q0, *tchunk0, *tchunk_large,
+        *tile_seg0;
+    uint32_t *hist, *prefix;
+    int32_t *k_rem, *cand_cnt, *seg_m, *seg_ticket, *seg_epoch, *lb;
+    uint16_t *cand_pos;
+    const int64_t *comp_off;
+    int64_t comp_total;
+    uint32_t *comp_key;
+    int32_t *comp_idx;
+    int32_t *out;
+    int64_t out_stride;
+    int32_t *errword;
+};
+
+constexpr int kFinThreads = 1024;
+constexpr int kFinWarps = kFinThreads / 32;
+constexpr int kFinSmemCap = 8192;     // candidates a finishing CTA keeps in shared memory
+constexpr int kFinPerThread = 4;      // consecutive entries per thread in the ordered passes
+constexpr int kAccThreads = 1024;     // accumulation: one 128-bit g/u/v triple per thread, 4096 elements per CTA
+
+// How far below the bucket of this step's k-th key the next step's candidates start.  The k-th
+// largest of few entries moves more from step to step, so small k gets a wider margin.
+__device__ __forceinline__ int lb_margin(int k) { return k >= 512 ? 1 : (k >= 64 ? 2 : 4); }
+
+// Geometry of tile-chunk c: the part [lo, hi) of tile q (positions inside the tile) that belongs
+// to large segment li.
+struct ChunkGeom {
+    int li, s, q, lo, hi;
+};
+__device__ __forceinline__ ChunkGeom chunk_geom(const FastArgs &f, int c)
+{
+    ChunkGeom g;
+    g.li = f.tchunk_large[c];
+    g.s = f.large_ids[g.li];
+    g.q = f.large_q0[g.li] + (c - f.tchunk0[g.li]);
+    const int64_t tile_base = (int64_t)g.q * kSelChunk, off = f.seg_off[g.s], end = off + f.seg_len[g.s];
+    g.lo = off > tile_base ? (int)(off - tile_base) : 0;
+    g.hi = end - tile_base < kSelChunk ? (int)(end - tile_base) : kSelChunk;
+    return g;
+}
+
+// Keys of the tile at `tile` in striped order: key[4 r + j] is position 1024 r + 4 t + j (thread
+// t of 256), so a warp reads 512 consecutive bytes per request.  Only positions in [lo, hi) are
+// loaded; returns their 16-bit validity mask.
+__device__ __forceinline__ unsigned load_keys_tile(const float *__restrict__ tile, int lo, int hi,
+                                                   uint32_t (&key)[kSelPerThread])
+{
+    const bool vec = (reinterpret_cast<uintptr_t>(tile) & 15) == 0;
+    unsigned valid = 0;
+#pragma unroll
+    for (int r = 0; r < kSelPerThread / 4; ++r) {
+        const int e = r * (kSelThreads * 4) + (int)threadIdx.x * 4;
+        if (vec && e >= lo && e + 4 <= hi) {
+            const float4 x = __ldg(reinterpret_cast<const float4 *>(tile + e));
+            key[4 * r + 0] = mag_key(x.x);
+            key[4 * r + 1] = mag_key(x.y);
+            key[4 * r + 2] = mag_key(x.z);
+            key[4 * r + 3] = mag_key(x.w);
+            valid |= 0xfu << (4 * r);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool in = e + j >= lo && e + j < hi;
+                key[4 * r + j] = in ? mag_key(__ldg(tile + e + j)) : 0u;
+                valid |= (in ? 1u : 0u) << (4 * r + j);
+            }
+        }
+    }
+    return valid;
+}
+
+// Run by every thread of the CTA that completed a segment's histogram.  Finds the bucket d0 of
+// the k-th largest key.  FUSED: bins below the predicted bucket were not counted, the candidates
+// are all counted entries, and the result stands only if at least k were counted.  Otherwise the
+// histogram is complete and the candidates are the entries from bucket d0 upwards.  On success
+// stores d0, the rank still to find inside it, the candidate count and the prediction for the
+// next step, and returns true.  Always leaves histogram and ticket zeroed.
+template <int THREADS, bool FUSED>
+__device__ __forceinline__ bool bucket_scan(const FastArgs &f, int64_t slot, int k, int *warp_tot, int *flag)
+{
+    constexpr int kPer = kHistBins / THREADS;
+    uint32_t *gh = f.hist + slot * kHistBins;
+    int hh[kPer], part = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        hh[i] = (int)__ldcg(gh + threadIdx.x * kPer + i);
+        part += hh[i];
+    }
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) gh[threadIdx.x * kPer + i] = 0u;
+    if (threadIdx.x == 0) {
+        f.seg_ticket[slot] = 0;
+        *flag = 0;
+    }
+    const int incl = block_suffix_incl(part, warp_tot);      // two barriers inside: *flag = 0 is visible
+    if (incl >= k && incl - part < k) {
+        int above = incl - part;
+#pragma unroll
+        for (int i = kPer - 1; i >= 0; --i) {
+            if (above + hh[i] >= k) {
+                const int d0 = threadIdx.x * kPer + i;
+                f.prefix[slot] = (uint32_t)d0;
+                f.k_rem[slot] = k - above;
+                if (!FUSED) f.seg_m[slot] = above + hh[i];
+                const int lbn = d0 - lb_margin(k);
+                f.lb[slot] = lbn > 1 ? lbn : 1;
+                *flag = 1;
+                break;
+            }
+            above += hh[i];
+        }
+    }
+    if (FUSED && threadIdx.x == 0) f.seg_m[slot] = incl;      // thread 0's suffix sum is the total
+    __syncthreads();
+    const bool ok = *flag != 0;
+    if (!ok && threadIdx.x == 0) f.lb[slot] = 0;              // no usable prediction
+    return ok;
+}
+
+// (b) Leading-digit histogram of one tile-chunk.  Segments whose candidates the accumulation of
+// this step already produced are skipped.
+__global__ void __launch_bounds__(kSelThreads) hist0_fast_kernel(FastArgs f)
+{
+    __shared__ unsigned h[kHistBins];
+    __shared__ int warp_tot[kWarps];
+    __shared__ int is_last, scan_flag;
+    const int row = blockIdx.y;
+    const ChunkGeom g = chunk_geom(f, blockIdx.x);
+    const int64_t slot = (int64_t)row * f.num_large + g.li;
+    if (f.seg_epoch[slot] == f.epoch) return;
+    for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0;
+    __syncthreads();
+    const float *tile = f.data + (int64_t)(f.row0 + row) * f.row_stride + (int64_t)g.q * kSelChunk;
+    uint32_t key[kSelPerThread];
+    const unsigned valid = load_keys_tile(tile, g.lo, g.hi, key);
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i)
+        if (valid >> i & 1u) atomicAdd(&h[key[i] >> 20], 1u);
+    __syncthreads();
+    uint32_t *gh = f.hist + slot * kHistBins;
+    for (int b = threadIdx.x; b < kHistBins; b += kSelThreads)
+        if (h[b]) atomicAdd(gh + b, h[b]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int chunks = f.tchunk0[g.li + 1] - f.tchunk0[g.li];
+        is_last = atomicAdd(&f.seg_ticket[slot], 1) == chunks - 1;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    if (!bucket_scan<kSelThreads, false>(f, slot, f.seg_k[g.s], warp_tot, &scan_flag) && threadIdx.x == 0)
+        atomicExch(f.errword, 0x5E40);                         // a complete histogram always holds k entries
+}
+
+// (b) Candidates of one tile-chunk: positions (ascending) of the entries at or above the bucket
+// of the k-th key; skipped for segments already served by the accumulation and for segments that
+// will be finished from the data.  The first num_small CTAs each select one small segment.
+__global__ void __launch_bounds__(kSelThreads) collect_small_kernel(FastArgs f)
+{
+    __shared__ SmallShared small_sh;
+    const int row = blockIdx.y;
+    if ((int)blockIdx.x < f.num_small) {          // the longer-running CTAs go first
+        select_small_body(f.data, f.row_stride, f.row0, f.seg_off, f.seg_len, f.seg_k, f.seg_out,
+                          f.small_ids[blockIdx.x], row, f.out, f.out_stride, f.errword, small_sh);
+        return;
+    }
+    const int chunk = (int)blockIdx.x - f.num_small;
+    unsigned long long *warp_tot = reinterpret_cast<unsigned long long *>(small_sh.hist);
+    const ChunkGeom g = chunk_geom(f, chunk);
+    const int64_t slot = (int64_t)row * f.num_large + g.li;
+    if (f.seg_epoch[slot] == f.epoch) return;
+    if ((int64_t)f.seg_m[slot] > f.comp_off[g.li + 1] - f.comp_off[g.li]) return;
+    const float *tile = f.data + (int64_t)(f.row0 + row) * f.row_stride + (int64_t)g.q * kSelChunk;
+    uint32_t key[kSelPerThread];
+    const unsigned valid = load_keys_tile(tile, g.lo, g.hi, key);
+    const uint32_t d0 = f.prefix[slot];
+    unsigned flags = 0;
+#pragma unroll
+    for (int i = 0; i < kSelPerThread; ++i)
+        if ((valid >> i & 1u) && (key[i] >> 20) >= d0) flags |= 1u << i;
+    // per-stripe counts packed into four 16-bit fields, one CTA-wide scan for all four
+    unsigned long long mine = 0;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) mine |= (unsigned long long)__popc(flags >> (4 * r) & 0xfu) << (16 * r);
+    unsigned long long total;
+    const unsigned long long before = block_prefix_excl<unsigned long long>(mine, warp_tot, &total);
+    const int64_t c = (int64_t)row * f.num_tchunks + chunk;
+    if (threadIdx.x == 0)
+        f.cand_cnt[c] = (int)((total & 0xffff) + (total >> 16 & 0xffff) + (total >> 32 & 0xffff) + (total >> 48));
+    if (flags) {
+        uint16_t *dst = f.cand_pos + c * kSelChunk;
+        unsigned stripe_base = 0;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            unsigned at = stripe_base + (unsigned)(before >> (16 * r) & 0xffff);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (flags >> (4 * r + j) & 1u) dst[at++] = (uint16_t)(r * (kSelThreads * 4) + threadIdx.x * 4 + j);
+            stripe_base += (unsigned)(total >> (16 * r) & 0xffff);
+        }
+    }
+}
+
+// Where a finishing CTA reads its entries from: the compacted candidates or the segment itself.
+struct CompactSource {
+    const uint32_t *key;
+    const int32_t *idx;
+    int n;
+    __device__ __forceinline__ uint32_t key_at(int i) const { return key[i]; }
+    __device__ __forceinline__ int32_t idx_at(int i) const { return idx[i]; }
+};
+struct DataSource {
+    const float *seg;
+    int64_t off;
+    int n;
+    __device__ __forceinline__ uint32_t key_at(int i) const { return mag_key(__ldg(seg + i)); }
+    __device__ __forceinline__ int32_t idx_at(int i) const { return (int32_t)(off + i); }
+};
+
+struct FinishShared {
+    int hist[256];
+    int warp_i[kFinWarps];
+    unsigned warp_u[kFinWarps];
+    int found[2];
+};
+
+// Completes the radix search below the 11-bit bucket d0 (k_rem entries still to find inside it)
+// and emits the k selected offsets in order.  Entries below the bucket, if the source has any,
+// are ignored.
+template <typename Source>
+__device__ void finish_from(const Source &src, uint32_t d0, int k_rem, int k, int32_t *__restrict__ out,
+                            FinishShared &sh, int32_t *errword)
+{
+    uint32_t prefix = d0 << 20, decided = 0x7ff00000u;
+    const int shifts[3] = {12, 4, 0};
+    const uint32_t masks[3] = {0xffu, 0xffu, 0xfu};
+#pragma unroll 1
+    for (int p = 0; p < 3; ++p) {
+        if (threadIdx.x < 256) sh.hist[threadIdx.x] = 0;
+        __syncthreads();
+        for (int i = threadIdx.x; i < src.n; i += kFinThreads) {
+            const uint32_t x = src.key_at(i);
+            if ((x & decided) == prefix) atomicAdd(&sh.hist[(x >> shifts[p]) & masks[p]], 1);
+        }
+        __syncthreads();
+        const int mine = threadIdx.x < 256 ? sh.hist[threadIdx.x] : 0;
+        const int incl = block_suffix_incl(mine, sh.warp_i);
+        if (threadIdx.x < 256 && incl >= k_rem && incl - mine < k_rem) {
+            sh.found[0] = threadIdx.x;
+            sh.found[1] = k_rem - (incl - mine);
+        }
+        if (threadIdx.x == 0 && incl < k_rem) atomicExch(errword, 0x5E50 + p);
+        __syncthreads();
+        prefix |= (uint32_t)sh.found[0] << shifts[p];
+        decided |= masks[p] << shifts[p];
+        k_rem = sh.found[1];
+        __syncthreads();
+    }
+    const uint32_t T = prefix;
+    const int r = k_rem;
+    int gt_done = 0, eq_done = 0;            // entries before the current tile
+    const int tile = kFinThreads * kFinPerThread;
+    for (int base = 0; base < src.n; base += tile) {
+        uint32_t key[kFinPerThread];
+        const int first = base + (int)threadIdx.x * kFinPerThread;
+        unsigned gt = 0, eq = 0;
+#pragma unroll
+        for (int i = 0; i < kFinPerThread; ++i) {
+            key[i] = first + i < src.n ? src.key_at(first + i) : 0u;
+            if (first + i < src.n) { gt += key[i] > T; eq += key[i] == T; }
+        }
+        unsigned total;
+        const unsigned before = block_prefix_excl<unsigned>(gt | (eq << 16), sh.warp_u, &total);
+        int g = gt_done + (int)(before & 0xffff), e = eq_done + (int)(before >> 16);
+#pragma unroll
+        for (int i = 0; i < kFinPerThread; ++i) {
+            if (first + i < src.n) {
+                int pos = -1;
+                if (key[i] > T) { pos = g + (e < r ? e : r); ++g; }
+                else if (key[i] == T) { if (e < r) pos = g + e; ++e; }
+                if (pos >= 0) {
+                    if (pos < k) out[pos] = src.idx_at(first + i);
+                    else atomicExch(errword, 0x5E60);
+                }
+            }
+        }
+        gt_done += (int)(total & 0xffff);
+        eq_done += (int)(total >> 16);
+        if (gt_done + (eq_done < r ? eq_done : r) >= k) break;     // everything is emitted
+    }
+}
+
+// One CTA per (large segment, row): compacts the segment's candidates in index order (thread t
+// owns chunk t of a group of 1024 chunks), then finishes on them; or on the data when the
+// candidates exceed the compact capacity.
+__global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
+{
+    __shared__ FinishShared sh;
+    extern __shared__ __align__(16) uint32_t fin_dyn[];     // kFinSmemCap keys, then kFinSmemCap offsets
+    uint32_t *s_key = fin_dyn;
+    int32_t *s_idx = reinterpret_cast<int32_t *>(fin_dyn + kFinSmemCap);
+    const int li = blockIdx.x, row = blockIdx.y;
+    const int64_t slot = (int64_t)row * f.num_large + li;
+    const int s = f.large_ids[li];
+    const int64_t off = f.seg_off[s];
+    const int len = f.seg_len[s], k = f.seg_k[s];
+    const float *rowp = f.data + (int64_t)(f.row0 + row) * f.row_stride;
+    int32_t *out = f.out + (int64_t)row * f.out_stride + f.seg_out[s];
+    const uint32_t d0 = f.prefix[slot];
+    const int k_rem = f.k_rem[slot];
+    const int m = f.seg_m[slot];
+    const int64_t cap = f.comp_off[li + 1] - f.comp_off[li];
+    if ((int64_t)m > cap) {                   // too many entries share the bucket: work on the data
+        DataSource src{rowp + off, off, len};
+        finish_from(src, d0, k_rem, k, out, sh, f.errword);
+        return;
+    }
+    const bool in_smem = m <= kFinSmemCap;
+    uint32_t *ckey = in_smem ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
+    int32_t *cidx = in_smem ? s_idx : f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
+    const int c0 = f.tchunk0[li], c1 = f.tchunk0[li + 1];
+    const int q0 = f.large_q0[li];
+    const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
+    int done = 0;
+    for (int base = c0; base < c1; base += kFinThreads) {
+        const int c = base + (int)threadIdx.x;
+        const unsigned n = c < c1 ? (unsigned)cnt[c] : 0u;
+        unsigned total;
+        unsigned at = (unsigned)done + block_prefix_excl<unsigned>(n, sh.warp_u, &total);
+        if (n) {
+            // eight positions per 128-bit load, then eight independent gathers
+            const uint4 *pos8 = reinterpret_cast<const uint4 *>(f.cand_pos + ((int64_t)row * f.num_tchunks + c) * kSelChunk);
+            const int tile_base = (q0 + (c - c0)) * kSelChunk;          // N < 2^31
+            for (unsigned b0 = 0; b0 < n; b0 += 8) {
+                const uint4 pv = pos8[b0 >> 3];
+                const unsigned w[4] = {pv.x, pv.y, pv.z, pv.w};
+                uint32_t kk[8];
+#pragma unroll
+                for (int b = 0; b < 8; ++b) {
+                    const int j = tile_base + (int)(w[b >> 1] >> (16 * (b & 1)) & 0xffffu);
+                    kk[b] = b0 + b < n ? mag_key(__ldg(rowp + j)) : 0u;
+                }
+#pragma unroll
+                for (int b = 0; b < 8; ++b) {
+                    if (b0 + b < n && at + b < (unsigned)m) {
+                        ckey[at + b] = kk[b];
+                        cidx[at + b] = tile_base + (int)(w[b >> 1] >> (16 * (b & 1)) & 0xffffu);
+                    }
+                }
+                at += 8;
+            }
+        }
+        done += (int)total;
+    }
+    if (threadIdx.x == 0 && done != m) atomicExch(f.errword, 0x5E70);
+    __syncthreads();
+    CompactSource src{ckey, cidx, m};
+    finish_from(src, d0, k_rem, k, out, sh, f.errword);
+}
+
+// ------------------------------------------------------------------------------------------
+// (a) Stage 1 fused with candidate collection.  Grid (tiles per row, K); a CTA streams one tile
+// of one row exactly as accumulate_kernel does (u <- m u + g fused, v <- v + u; Algorithm 1/2 and
+// Section V-A).  A CTA of a selecting row then looks at its fresh v: for every large segment the
+// tile overlaps and that has a predicted bucket, the entries at or above the bucket are
+// histogrammed and listed, and the CTA that completes the segment settles the bucket of its k-th
+// key.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void acc4(float4 &u, float4 &v, const float4 &g, float m)
+{
+    u.x = __fmaf_rn(m, u.x, g.x); v.x = __fadd_rn(v.x, u.x);
+    u.y = __fmaf_rn(m, u.y, g.y); v.y = __fadd_rn(v.y, u.y);
+    u.z = __fmaf_rn(m, u.z, g.z); v.z = __fadd_rn(v.z, u.z);
+    u.w = __fmaf_rn(m, u.w, g.w); v.w = __fadd_rn(v.w, u.w);
+}
+
+__global__ void __launch_bounds__(kAccThreads, 2)
+accumulate_select_kernel(FastArgs f, const float *__restrict__ g, float *__restrict__ u, float *__restrict__ v,
+                         int64_t N, float m, int sel_row0, int sel_rows)
+{
+    __shared__ unsigned warp_u[kAccThreads / 32];
+    __shared__ int warp_i[kAccThreads / 32];
+    __shared__ int is_last, scan_flag;
+    const int row = blockIdx.y, q = blockIdx.x;
+    const int64_t tile_base = (int64_t)q * kSelChunk;
+    const int in_tile = N - tile_base < kSelChunk ? (int)(N - tile_base) : kSelChunk;    // a multiple of 4
+    const int p0 = (int)threadIdx.x * 4;
+    const bool live = p0 < in_tile;
+    float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (live) {
+        const int64_t e = ((int64_t)row * N + tile_base + p0) >> 2;
+        const float4 gg = __ldcs(reinterpret_cast<const float4 *>(g) + e);
+        float4 uu = __ldcs(reinterpret_cast<float4 *>(u) + e);
+        vv = __ldcs(reinterpret_cast<float4 *>(v) + e);
+        acc4(uu, vv, gg, m);
+        __stcs(reinterpret_cast<float4 *>(u) + e, uu);
+        __stcs(reinterpret_cast<float4 *>(v) + e, vv);
+    }
+    const int sel = row - sel_row0;
+    if (sel < 0 || sel >= sel_rows) return;
+    const uint32_t key[4] = {mag_key(vv.x), mag_key(vv.y), mag_key(vv.z), mag_key(vv.w)};
+    const int64_t tile_end = tile_base + in_tile;
+    for (int s = f.tile_seg0[q]; s < f.num_large + f.num_small && f.seg_off[s] < tile_end; ++s) {
+        const int li = f.seg_large[s];
+        if (li < 0) continue;
+        const int64_t slot = (int64_t)sel * f.num_large + li;
+        const uint32_t lb = (uint32_t)f.lb[slot];
+        if (lb == 0) continue;                                  // no prediction: path (b) will serve it
+        const int64_t off = f.seg_off[s], end = off + f.seg_len[s];
+        const int lo = off > tile_base ? (int)(off - tile_base) : 0;
+        const int hi = end < tile_end ? (int)(end - tile_base) : in_tile;
+        unsigned flags = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (live && p0 + i >= lo && p0 + i < hi && (key[i] >> 20) >= lb) flags |= 1u << i;
+        uint32_t *gh = f.hist + slot * kHistBins;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (flags >> i & 1u) atomicAdd(gh + (key[i] >> 20), 1u);
+        unsigned total;
+        unsigned at = block_prefix_excl<unsigned>((unsigned)__popc(flags), warp_u, &total);
+        const int64_t c = (int64_t)sel * f.num_tchunks + f.tchunk0[li] + (q - f.large_q0[li]);
+        if (threadIdx.x == 0) f.cand_cnt[c] = (int)total;
+        if (flags) {
+            uint16_t *dst = f.cand_pos + c * kSelChunk;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (flags >> i & 1u) dst[at++] = (uint16_t)(p0 + i);
+        }
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int chunks = f.tchunk0[li + 1] - f.tchunk0[li];
+            is_last = atomicAdd(&f.seg_ticket[slot], 1) == chunks - 1;
+        }
+        __syncthreads();
+        const bool last = is_last != 0;                         // uniform over the CTA
+        __syncthreads();                                        // everyone has read it before it is reused
+        if (last) {
+            __threadfence();
+            const bool ok = bucket_scan<kAccThreads, true>(f, slot, f.seg_k[s], warp_i, &scan_flag);
+            if (ok && threadIdx.x == 0) f.seg_epoch[slot] = f.epoch;
+        }
+    }
+}
+
+void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t row_stride, int row0, int32_t *out,
+               int64_t out_stride, int32_t epoch, int32_t *errword)
+{
+    f.data = data; f.row_stride = row_stride; f.row0 = row0;
+    f.num_large = t.num_large; f.num_small = t.num_small; f.num_tchunks = t.num_tchunks; f.epoch = epoch;
+    f.seg_off = t.seg_off; f.seg_len = t.seg_len; f.seg_k = t.seg_k; f.seg_out = t.seg_out;
+    f.small_ids = t.small_ids; f.large_ids = t.large_ids; f.seg_large = t.seg_large; f.large_q0 = t.large_q0;
+    f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_seg0 = t.tile_seg0;
+    f.hist = t.hist; f.prefix = t.prefix; f.k_rem = t.k_rem; f.cand_cnt = t.cand_cnt; f.seg_m = t.seg_m;
+    f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.lb = t.lb; f.cand_pos = t.cand_pos;
+    f.comp_off = t.comp_off; f.comp_total = t.comp_total; f.comp_key = t.comp_key; f.comp_idx = t.comp_idx;
+    f.out = out; f.out_stride = out_stride; f.errword = errword;
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_small_only_kernel(FastArgs f)
+{
+    __shared__ SmallShared sh;
+    select_small_body(f.data, f.row_stride, f.row0, f.seg_off, f.seg_len, f.seg_k, f.seg_out, f.small_ids[blockIdx.x],
+                      blockIdx.y, f.out, f.out_stride, f.errword, sh);
+}
+
+}  // namespace
+
+cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0, int rows,
+                          int32_t *out, int64_t out_stride, int32_t epoch, int32_t *errword, cudaStream_t st)
+{
+    if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
+    FastArgs f;
+    fill_args(f, t, data, row_stride, row0, out, out_stride, epoch, errword);
+    if (!t.num_large) {
+        select_small_only_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
+        return cudaGetLastError();
+    }
+    constexpr int kFinDyn = 2 * kFinSmemCap * (int)sizeof(uint32_t);
+    static bool configured = false;
+    if (!configured) {
+        const cudaError_t e = cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinDyn);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    hist0_fast_kernel<<<dim3(t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
+    collect_small_kernel<<<dim3(t.num_small + t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
+    finish_kernel<<<dim3(t.num_large, rows), kFinThreads, kFinDyn, st>>>(f), ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_accumulate_select(const SelectTables &t, const float *g, float *u, float *v, int K, int64_t N,
+                                     float m, int sel_row0, int sel_rows, int32_t epoch, int32_t *errword,
+                                     cudaStream_t st)
+{
+    FastArgs f;
+    fill_args(f, t, v, N, 0, nullptr, 0, epoch, errword);
+    accumulate_select_kernel<<<dim3(t.tiles_per_row, K), kAccThreads, 0, st>>>(f, g, u, v, N, m, sel_row0, sel_rows),
+        ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+}  // namespace lgc

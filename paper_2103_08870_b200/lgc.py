@@ -52,7 +52,7 @@ def lib() -> C.CDLL:
         l.lgc_workspace_bytes.argtypes = [C.POINTER(lgc_config), C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
         l.lgc_init.argtypes = [C.POINTER(lgc_config), vp, sz, vp, sz, vp, sz, C.POINTER(vp)]
         l.lgc_destroy.argtypes = [vp]
-        l.lgc_accumulate.argtypes = [vp, vp]
+        l.lgc_accumulate.argtypes = [vp, vp, C.c_int32]
         l.lgc_topk.argtypes = [vp, C.c_int32]
         l.lgc_encode.argtypes = [vp]
         l.lgc_combine.argtypes = [vp, C.c_int32]
@@ -180,8 +180,9 @@ class LGC:
         return t.data_ptr()
 
     # -- the stages ---------------------------------------------------------------------------
-    def accumulate(self, grads: torch.Tensor) -> None:
-        self._ok(self._l.lgc_accumulate(self._ctx, self._dev_f32(grads, self.K * self.N, "grads")), "lgc_accumulate")
+    def accumulate(self, grads: torch.Tensor, leader_hint: int = -1) -> None:
+        self._ok(self._l.lgc_accumulate(self._ctx, self._dev_f32(grads, self.K * self.N, "grads"), leader_hint),
+                 "lgc_accumulate")
 
     def topk(self, leader: int = 0) -> None:
         self._ok(self._l.lgc_topk(self._ctx, leader), "lgc_topk")
@@ -204,7 +205,7 @@ class LGC:
 
     def step(self, grads: torch.Tensor, update: torch.Tensor, choice: int = 0) -> None:
         """The five stages of one compression step, in order."""
-        self.accumulate(grads)
+        self.accumulate(grads, choice)
         self.topk(choice)
         self.encode()
         self.combine(choice)

@@ -51,11 +51,12 @@ def make_pair(numel, K, variant="rar", ae_kind="conv2", c1=8, c2=4, density_ppm=
 
 
 def compare_step(ora, gpu, g_cpu: torch.Tensor, g_dev: torch.Tensor, choice: int, update_dev: torch.Tensor,
-                 check_state=True):
-    """One full compression step on both sides, compared after every stage."""
+                 check_state=True, hint="leader"):
+    """One full compression step on both sides, compared after every stage.  `hint`: what
+    lgc_accumulate is told about the coming leader ("leader", "none", or "wrong")."""
     K = ora.K
     ora.accumulate(g_cpu.numpy())
-    gpu.accumulate(g_dev)
+    gpu.accumulate(g_dev, {"leader": choice, "none": -1, "wrong": (choice + 1) % K}[hint])
     if check_state:
         assert_bitwise(gpu.u.cpu().numpy(), ora.u, "u after accumulate")
         assert_bitwise(gpu.v.cpu().numpy(), ora.v, "v after accumulate")

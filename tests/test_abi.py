@@ -82,7 +82,7 @@ def test_status_strings_and_null_context(lib):
     assert lib.lgc_status_string(0) == b"LGC_OK"
     assert lib.lgc_status_string(2) == b"LGC_ERR_BAD_STATE"
     assert lib.lgc_status_string(99) == b"LGC_ERR_UNKNOWN"
-    assert lib.lgc_accumulate(None, None) == 1
+    assert lib.lgc_accumulate(None, None, 0) == 1
     assert lib.lgc_destroy(None) == 0
     assert isinstance(lib.lgc_last_error(None), bytes)
 

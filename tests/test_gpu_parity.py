@@ -19,14 +19,14 @@ def toy_source(numel, K, seed=5):
     return W.GradientSource(W.LayerTable("toy", list(numel), [1 + (i % 3) for i in range(len(numel))]), K, seed=seed)
 
 
-def run_steps(numel, K, steps, **kw):
+def run_steps(numel, K, steps, hints=("leader",), **kw):
     seed = kw.get("seed", W.DEFAULT_SEED)
     ora, gpu = make_pair(numel, K, **kw)
     src = toy_source(numel, K)
     upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
     for t in range(steps):
         g = src.step(t)
-        compare_step(ora, gpu, g, g.cuda(), W.choice_for_step(seed, t, K), upd)
+        compare_step(ora, gpu, g, g.cuda(), W.choice_for_step(seed, t, K), upd, hint=hints[t % len(hints)])
     return ora, gpu
 
 
@@ -44,7 +44,36 @@ def test_tiny_config_ring_allreduce():
 
 @pytest.mark.parametrize("K", [1, 3])
 def test_ragged_layers_ring_allreduce(K):
-    run_steps(TOY, K, 4)
+    assert sum(TOY) % 4 == 0                      # rows start 16-byte aligned: the fused accumulation runs
+    run_steps(TOY, K, 6)
+
+
+def test_leader_hint_never_changes_a_result():
+    # candidates collected while accumulating are used only when the hint was right; a missing or
+    # wrong hint, and hints that come and go, give the same bits
+    run_steps(TOY, 3, 8, hints=("none", "leader", "leader", "wrong", "leader", "none", "leader", "leader"))
+
+
+def test_rows_that_do_not_start_aligned():
+    numel = TOY + [2]                             # N % 4 == 2: the plain accumulation kernel is used
+    assert sum(numel) % 4 != 0
+    run_steps(numel, 3, 4)
+    run_steps(numel, 2, 3, variant="ps")
+
+
+def test_prediction_survives_a_collapse_of_the_gradient_scale():
+    # the predicted bucket comes from the previous step; when the residual's large entries vanish
+    # (scale drops by 1e4) the prediction is too high and the selection must fall back
+    numel = [200000, 3000, 50000]
+    K = 2
+    ora, gpu = make_pair(numel, K, momentum=0.0, density_ppm=5000)
+    src = toy_source(numel, K)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t, scale in enumerate([1.0, 1.0, 1e-4, 1e-4, 1.0, 10.0, 1e-6]):
+        g = src.step(t) * scale
+        if t in (2, 6):                           # wipe the residual: only the tiny gradient remains
+            gpu.v.zero_(); gpu.u.zero_(); ora.v[:] = 0; ora.u[:] = 0
+        compare_step(ora, gpu, g, g.cuda(), t % K, upd)
 
 
 def test_ragged_layers_parameter_server():
@@ -145,7 +174,7 @@ def test_topk_scatter_phase_two():
         for t in range(2):
             g = src.step(t)
             ora.accumulate(g.numpy())
-            gpu.accumulate(g.cuda())
+            gpu.accumulate(g.cuda(), t)
             ora.topk(t)
             gpu.topk(t)
             ref = ora.topk_scatter()

@@ -57,7 +57,7 @@ def test_segnet_config_with_autoencoder_training():
         src.step_into(t, g)
         choice = W.choice_for_step(w.seed, t, K)
         ora.accumulate(g.cpu().numpy())
-        gpu.accumulate(g)
+        gpu.accumulate(g, choice)
         ora.topk(choice)
         gpu.topk(choice)
         losses_ref.append(ora.ae_train_step())
@@ -104,7 +104,7 @@ def test_stress_config_sampled():
         src.step_into(t, g)
         leader = W.choice_for_step(w.seed, t, K)
         g_s = g[:, pos_dev].cpu().numpy()
-        gpu.accumulate(g)
+        gpu.accumulate(g, leader)
         for k in range(K):
             O.accumulate(u_s[k], v_s[k], np.ascontiguousarray(g_s[k]), float(np.float32(w.momentum)))
         assert_bitwise(gpu.u[:, pos_dev].cpu().numpy(), u_s, f"sampled u, step {t}")
