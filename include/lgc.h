@@ -208,6 +208,14 @@ lgc_status lgc_get_ae_params(const lgc_ctx *ctx, float *dst, size_t count);
  * (code readable through lgc_last_error).  Clears the record. */
 lgc_status lgc_check(lgc_ctx *ctx);
 
+/* How the last lgc_topk got its entries: the number of (selecting row, layer) pairs with more
+ * than 4096 elements; how many of them were finished from candidates collected during
+ * lgc_accumulate (no further pass over v); and the total and the largest number of candidates
+ * per pair (the k_l selected entries are found among them).  Any pointer may be NULL.  Waits
+ * for the stream. */
+lgc_status lgc_selection_stats(lgc_ctx *ctx, int64_t *large_segments, int64_t *served_by_accumulation,
+                               int64_t *candidates_total, int64_t *candidates_max);
+
 /* Number of kernels the library has enqueued from the calling thread since it was loaded
  * (all contexts); the benchmark reports the difference over its timed region. */
 uint64_t lgc_kernel_launches(void);

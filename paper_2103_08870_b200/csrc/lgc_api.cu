@@ -111,8 +111,8 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
 // large ones are cut by the row's tiles of kSelChunk elements.
 struct SelectPlan {
     std::vector<int64_t> seg_off, comp_off;
-    std::vector<int32_t> seg_len, seg_k, seg_out, small_ids, large_ids, seg_large, large_q0, tchunk0, tchunk_large,
-        tile_seg0;
+    std::vector<int32_t> seg_len, seg_k, seg_out, small_ids, large_ids, seg_large, large_q0, tchunk0, tchunk_large;
+    std::vector<int4> tile_desc;
     int tiles_per_row = 0;
     int64_t comp_total = 0;
 };
@@ -148,8 +148,17 @@ SelectPlan plan_select(const std::vector<int64_t> &off, const std::vector<int64_
     sp.tiles_per_row = (int)((row_len + kSelChunk - 1) / kSelChunk);
     int s = 0;
     for (int q = 0; q < sp.tiles_per_row; ++q) {
-        while (off[s] + len[s] <= (int64_t)q * kSelChunk) ++s;     // first segment that reaches into tile q
-        sp.tile_seg0.push_back(s);
+        const int64_t t0 = (int64_t)q * kSelChunk, t1 = t0 + kSelChunk < row_len ? t0 + kSelChunk : row_len;
+        while (off[s] + len[s] <= t0) ++s;                          // first segment that reaches into tile q
+        int4 d = make_int4(s, -2, 0, 0);
+        if (off[s] <= t0 && off[s] + len[s] >= t1 && sp.seg_large[s] >= 0) {
+            d.y = sp.seg_large[s];                                  // one large segment covers the tile
+            d.z = sp.tchunk0[d.y] + (q - sp.large_q0[d.y]);
+        } else {
+            for (int r = s; r < n && off[r] < t1; ++r)
+                if (sp.seg_large[r] >= 0) d.y = -1;                 // several segments, at least one large
+        }
+        sp.tile_desc.push_back(d);
     }
     return sp;
 }
@@ -170,14 +179,15 @@ void carve_select(Carver &cv, SelectTables &t, const SelectPlan &sp, int rows)
     t.large_q0 = cv.take<int32_t>(nl);
     t.tchunk0 = cv.take<int32_t>(nl + 1);
     t.tchunk_large = cv.take<int32_t>(nc);
-    t.tile_seg0 = cv.take<int32_t>(sp.tiles_per_row);
+    t.tile_desc = cv.take<int4>(sp.tiles_per_row);
     t.hist = cv.take<uint32_t>((size_t)rows * nl * kHistBins);
     t.prefix = cv.take<uint32_t>((size_t)rows * nl);
     t.k_rem = cv.take<int32_t>((size_t)rows * nl);
     t.seg_m = cv.take<int32_t>((size_t)rows * nl);
     t.seg_ticket = cv.take<int32_t>((size_t)rows * nl);
     t.seg_epoch = cv.take<int32_t>((size_t)rows * nl);
-    t.lb = cv.take<int32_t>((size_t)rows * nl);
+    t.lbkey = cv.take<uint32_t>((size_t)rows * nl);
+    t.seg_path = cv.take<int32_t>((size_t)rows * nl);
     t.cand_cnt = cv.take<int32_t>((size_t)rows * nc);
     t.cand_pos = cv.take<uint16_t>((size_t)rows * nc * kSelChunk);
     t.comp_off = cv.take<int64_t>((size_t)nl + 1);
@@ -247,11 +257,12 @@ cudaError_t upload_select(SelectTables &t, SelectPlan sp, cudaStream_t s, std::v
     const SelectPlan &h = hold.back();
     cudaError_t e = upload(t.seg_off, h.seg_off, s);
     if (e == cudaSuccess) e = upload(t.comp_off, h.comp_off, s);
+    if (e == cudaSuccess) e = upload(t.tile_desc, h.tile_desc, s);
     const std::vector<int32_t> *arrs[] = {&h.seg_len, &h.seg_k, &h.seg_out, &h.seg_large, &h.small_ids, &h.large_ids,
-                                          &h.large_q0, &h.tchunk0, &h.tchunk_large, &h.tile_seg0};
+                                          &h.large_q0, &h.tchunk0, &h.tchunk_large};
     int32_t *dsts[] = {t.seg_len, t.seg_k, t.seg_out, t.seg_large, t.small_ids, t.large_ids,
-                       t.large_q0, t.tchunk0, t.tchunk_large, t.tile_seg0};
-    for (int i = 0; i < 10 && e == cudaSuccess; ++i) e = upload(dsts[i], *arrs[i], s);
+                       t.large_q0, t.tchunk0, t.tchunk_large};
+    for (int i = 0; i < 9 && e == cudaSuccess; ++i) e = upload(dsts[i], *arrs[i], s);
     return e;
 }
 
@@ -355,8 +366,9 @@ lgc_status lgc_accumulate(lgc_ctx *c, const float *grads, int32_t leader_hint)
     if (!ps && leader_hint >= c->K) return fail(c, LGC_ERR_INVALID_ARG, "leader_hint out of range");
     c->epoch = c->epoch == 0x7fffffff ? 1 : c->epoch + 1;
     cudaError_t e;
-    // the fused form needs rows that start 16-byte aligned and someone to select for
-    if (c->N % 4 == 0 && c->sel_v.num_large > 0 && (ps || leader_hint >= 0)) {
+    // the fused form needs rows that start 16-byte aligned, someone to select for, and the keys a
+    // previous selection left to collect against
+    if (c->N % 4 == 0 && c->sel_v.num_large > 0 && c->have_prediction && (ps || leader_hint >= 0)) {
         e = launch_accumulate_select(c->sel_v, grads, c->u, c->v, c->K, c->N, c->cfg.momentum, ps ? 0 : leader_hint,
                                      ps ? c->K : 1, c->epoch, c->errword, c->stream);
         c->fused_leader = ps ? -1 : leader_hint;
@@ -376,9 +388,10 @@ lgc_status lgc_topk(lgc_ctx *c, int32_t leader)
     const bool ps = c->cfg.variant == LGC_VARIANT_PS;
     if (!ps && (leader < 0 || leader >= c->K)) return fail(c, LGC_ERR_INVALID_ARG, "leader out of range");
     // candidates collected during the accumulation count only if they are this leader's
-    const bool fused = ps ? c->fused_leader == -1 : c->fused_leader == leader;
-    cudaError_t e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, fused ? c->epoch : -1,
+    const bool served = ps ? c->fused_leader == -1 : c->fused_leader == leader;
+    cudaError_t e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, served, c->epoch,
                                   c->errword, c->stream);
+    c->have_prediction = true;
     c->val_valid = false;
     c->mean_valid = false;
     c->tile_lo_valid = false;
@@ -532,6 +545,32 @@ lgc_status lgc_check(lgc_ctx *c)
 }
 
 uint64_t lgc_kernel_launches(void) { return g_kernel_launches; }
+
+lgc_status lgc_selection_stats(lgc_ctx *c, int64_t *large_segments, int64_t *served_by_accumulation,
+                               int64_t *candidates_total, int64_t *candidates_max)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    const size_t n = (size_t)c->S * c->sel_v.num_large;
+    std::vector<int32_t> ep(n), m(n);
+    if (n) {
+        cudaError_t e = cudaMemcpyAsync(ep.data(), c->sel_v.seg_path, n * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(m.data(), c->sel_v.seg_m, n * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+        if (e != cudaSuccess) return cuda_fail(c, e, "lgc_selection_stats");
+    }
+    int64_t served = 0, total = 0, most = 0;
+    for (size_t i = 0; i < n; ++i) {
+        served += ep[i] == 0;
+        total += m[i];
+        if (m[i] > most) most = m[i];
+    }
+    if (large_segments) *large_segments = (int64_t)n;
+    if (served_by_accumulation) *served_by_accumulation = served;
+    if (candidates_total) *candidates_total = total;
+    if (candidates_max) *candidates_max = most;
+    return LGC_OK;
+}
 
 const char *lgc_status_string(lgc_status s)
 {

@@ -416,7 +416,7 @@ cudaError_t launch_combine_ps(Ctx &c, int common_node)
                                                                    c.code_len, c.combined), ++g_kernel_launches;
     cudaError_t e = launch_zero(c.inn, (size_t)c.K * c.mu * sizeof(float), c.stream);
     if (e != cudaSuccess) return e;
-    e = launch_select(c.sel_inn, c.val, c.mu, 0, c.K, c.inn_pos, c.muI, -1, c.errword, c.stream);
+    e = launch_select(c.sel_inn, c.val, c.mu, 0, c.K, c.inn_pos, c.muI, false, ++c.inn_epoch, c.errword, c.stream);
     if (e != cudaSuccess) return e;
     innovation_fill_kernel<<<dim3(blocks_for(c.muI, 256), c.K), 256, 0, c.stream>>>(c.val, c.inn_pos, c.mu, c.muI, c.inn), ++g_kernel_launches;
     return cudaGetLastError();

@@ -48,13 +48,15 @@ struct SelectTables {
     int32_t *large_q0 = nullptr;     // [num_large] first tile the segment overlaps
     int32_t *tchunk0 = nullptr;      // [num_large + 1] first tile-chunk of each large segment
     int32_t *tchunk_large = nullptr; // [num_tchunks] index into large_ids
-    int32_t *tile_seg0 = nullptr;    // [tiles_per_row] first segment a tile overlaps
+    int4 *tile_desc = nullptr;       // [tiles_per_row] x: first segment the tile overlaps; y: the large segment that
+                                     // covers the whole tile (-1: several segments, -2: no large one); z: its chunk
     int32_t *cand_cnt = nullptr;     // [rows][num_tchunks] candidates found in the chunk
     uint16_t *cand_pos = nullptr;    // [rows][num_tchunks][kSelChunk] their positions inside the tile, ascending
     int32_t *seg_m = nullptr;        // [rows][num_large] candidates of the segment
     int32_t *seg_ticket = nullptr;   // [rows][num_large] chunks that have reported; zero between passes
-    int32_t *seg_epoch = nullptr;    // [rows][num_large] step whose accumulation already produced the candidates
-    int32_t *lb = nullptr;           // [rows][num_large] predicted lower bucket for the next step (0: none)
+    int32_t *seg_epoch = nullptr;    // [rows][num_large] step in which the two-pass path settled the segment
+    int32_t *seg_path = nullptr;     // [rows][num_large] how the last selection got its entries (see lgc_selection_stats)
+    uint32_t *lbkey = nullptr;       // [rows][num_large] key from which the next accumulation collects candidates (0: none)
     int64_t *comp_off = nullptr;     // [num_large + 1] first compact slot of each large segment
     int64_t comp_total = 0;          // compact slots per row
     uint32_t *comp_key = nullptr;    // [rows][comp_total] keys of the candidates, index order
@@ -108,6 +110,8 @@ struct Ctx {
     enum Stage { kIdle, kAccumulated, kSelected, kEncoded, kCombined } stage = kIdle;
     int32_t last_leader = 0;
     int32_t epoch = 0;             // step counter (accumulations so far)
+    int32_t inn_epoch = 0;         // the same counter for the innovation selection's tables
+    bool have_prediction = false;  // a selection has run, so the next accumulation has keys to collect against
     int32_t fused_leader = -2;     // row whose candidates the last accumulation collected (-1: all rows, -2: none)
     bool val_valid = false;        // val holds the kept values of the current selection
     bool tile_lo_valid = false;    // tile_lo matches the current selection
@@ -121,9 +125,9 @@ extern thread_local std::string g_last_error;   // failures without a context (s
 // ---- launchers (each enqueues on ctx stream and returns the launch status) -------------------
 cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s);
 cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s);
-// epoch: the step whose fused accumulation may already hold candidates (-1: none).
+// served: the accumulation of step `epoch` collected the candidates of exactly these rows.
 cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0,
-                          int rows, int32_t *out, int64_t out_stride, int32_t epoch, int32_t *errword,
+                          int rows, int32_t *out, int64_t out_stride, bool served, int32_t epoch, int32_t *errword,
                           cudaStream_t s);
 // Accumulation that also collects the selection candidates of the selecting rows (sel_row0 .. +sel_rows
 // of the K rows) against the predicted buckets; needs N % 4 == 0.

@@ -111,12 +111,13 @@ __device__ __forceinline__ void emit16(const uint32_t (&key)[kSelPerThread], int
 // ------------------------------------------------------------------------------------------
 struct alignas(16) SmallShared {
     int hist[256];
-    int warp_tot[kWarps];
-    unsigned scan_tot[kWarps];
+    int warp_tot[32];
+    unsigned scan_tot[32];
     int found[2];
 };
 
-// Whole selection of segment `s` of row `row` by one CTA of kSelThreads threads.
+// Whole selection of segment `s` of row `row` by one CTA of at least kSelThreads threads (the
+// first kSelThreads hold the keys; any further threads only take part in the barriers).
 __device__ __forceinline__ void
 select_small_body(const float *__restrict__ data, int64_t row_stride, int row0,
                   const int64_t *__restrict__ seg_off, const int32_t *__restrict__ seg_len,
@@ -124,7 +125,7 @@ select_small_body(const float *__restrict__ data, int64_t row_stride, int row0,
                   int32_t *__restrict__ out, int64_t out_stride, int32_t *errword, SmallShared &sh)
 {
     int (&hist)[256] = sh.hist;
-    int (&warp_tot)[kWarps] = sh.warp_tot;
+    int (&warp_tot)[32] = sh.warp_tot;
     int (&found)[2] = sh.found;
     const int64_t off = seg_off[s];
     const int len = seg_len[s], k = seg_k[s];
@@ -136,15 +137,18 @@ select_small_body(const float *__restrict__ data, int64_t row_stride, int row0,
     int k_rem = k;
 #pragma unroll 1
     for (int shift = 24; shift >= 0; shift -= 8) {
-        hist[threadIdx.x] = 0;
+        if (threadIdx.x < 256) hist[threadIdx.x] = 0;
         __syncthreads();
 #pragma unroll
         for (int i = 0; i < kSelPerThread; ++i)
             if (i < valid && (key[i] & decided) == prefix) atomicAdd(&hist[(key[i] >> shift) & 0xff], 1);
         __syncthreads();
-        const int mine = hist[threadIdx.x];
+        const int mine = threadIdx.x < 256 ? hist[threadIdx.x] : 0;
         const int incl = block_suffix_incl(mine, warp_tot);
-        if (incl >= k_rem && incl - mine < k_rem) { found[0] = threadIdx.x; found[1] = k_rem - (incl - mine); }
+        if (threadIdx.x < 256 && incl >= k_rem && incl - mine < k_rem) {
+            found[0] = threadIdx.x;
+            found[1] = k_rem - (incl - mine);
+        }
         __syncthreads();
         prefix |= (uint32_t)found[0] << shift;
         decided |= 0xffu << shift;

@@ -9,14 +9,16 @@
 //
 // Where the candidates come from:
 //  (a) fused: the accumulation kernel (accumulate_select_kernel, below) tests the freshly written
-//      v of the selecting rows against a bucket PREDICTED from the previous step, histograms the
-//      entries that pass, and the CTA that completes a segment (a ticket counter tells; nobody
-//      waits) checks that at least k entries passed.  Then no further read of v is needed.
-//  (b) otherwise (first step, prediction too high, leader not announced, N not a multiple of 4):
-//      hist0_fast_kernel histograms the segment, the completing CTA finds the bucket of the k-th
-//      key, and collect_small_kernel gathers the candidates: two reads of v.
-// A segment whose candidates exceed its compact capacity (ties, e.g. a layer of zeros) is
-// finished by its CTA streaming over the data instead.  Either way the result is exact.
+//      v of the selecting rows against a key PREDICTED from the previous step (a few per cent
+//      below that step's k-th key) and histograms and lists the entries that pass.  The finishing
+//      CTA checks that at least k entries passed; then v is not read again except at the candidates.
+//  (b) without a usable prediction (first step, leader not announced, rows not 16-byte aligned):
+//      hist0_fast_kernel histograms the segment, the CTA that completes it (a ticket counter
+//      tells; nobody waits) finds the bucket of the k-th key, and collect_kernel lists the
+//      entries from that bucket upwards: two reads of v.
+// If a prediction turns out too high, or a segment's candidates exceed its compact capacity
+// (ties, e.g. a layer of zeros), the finishing CTA works on the data itself.  The result is
+// exact in every case.
 #include "lgc_select_common.cuh"
 
 namespace lgc {
@@ -32,10 +34,10 @@ struct FastArgs {
     int num_large, num_small, num_tchunks;
     int32_t epoch;                 // step whose fused accumulation may have filled the lists (-1: none)
     const int64_t *seg_off;
-    const int32_t *seg_len, *seg_k, *seg_out, *small_ids, *large_ids, *seg_large, *large_q0, *tchunk0, *tchunk_large,
-        *tile_seg0;
-    uint32_t *hist, *prefix;
-    int32_t *k_rem, *cand_cnt, *seg_m, *seg_ticket, *seg_epoch, *lb;
+    const int32_t *seg_len, *seg_k, *seg_out, *small_ids, *large_ids, *seg_large, *large_q0, *tchunk0, *tchunk_large;
+    const int4 *tile_desc;
+    uint32_t *hist, *prefix, *lbkey;
+    int32_t *k_rem, *cand_cnt, *seg_m, *seg_ticket, *seg_epoch, *seg_path;
     uint16_t *cand_pos;
     const int64_t *comp_off;
     int64_t comp_total;
@@ -52,9 +54,15 @@ constexpr int kFinSmemCap = 8192;     // candidates a finishing CTA keeps in sha
 constexpr int kFinPerThread = 4;      // consecutive entries per thread in the ordered passes
 constexpr int kAccThreads = 1024;     // accumulation: one 128-bit g/u/v triple per thread, 4096 elements per CTA
 
-// How far below the bucket of this step's k-th key the next step's candidates start.  The k-th
-// largest of few entries moves more from step to step, so small k gets a wider margin.
-__device__ __forceinline__ int lb_margin(int k) { return k >= 512 ? 1 : (k >= 64 ? 2 : 4); }
+// The key from which the next step collects candidates, given this step's k-th key T.  Error
+// feedback piles entries up just below the threshold (each 3 % below T holds about k more), and
+// from step to step T moves by a per cent or two, more for small k: 3 % (6 % for k < 64) below T
+// keeps the candidates at 2-4 k.  A prediction that turns out too high only costs the fallback.
+__device__ __forceinline__ uint32_t predict_lbkey(uint32_t T, int k)
+{
+    const float t = __uint_as_float(T) * (k >= 64 ? 0.97f : 0.94f);
+    return __float_as_uint(t) & 0x7fffffffu;     // 0 (no prediction) when T is 0 or the product underflows
+}
 
 // Geometry of tile-chunk c: the part [lo, hi) of tile q (positions inside the tile) that belongs
 // to large segment li.
@@ -103,12 +111,12 @@ __device__ __forceinline__ unsigned load_keys_tile(const float *__restrict__ til
     return valid;
 }
 
-// Run by every thread of the CTA that completed a segment's histogram.  Finds the bucket d0 of
-// the k-th largest key.  FUSED: bins below the predicted bucket were not counted, the candidates
-// are all counted entries, and the result stands only if at least k were counted.  Otherwise the
-// histogram is complete and the candidates are the entries from bucket d0 upwards.  On success
-// stores d0, the rank still to find inside it, the candidate count and the prediction for the
-// next step, and returns true.  Always leaves histogram and ticket zeroed.
+// Run by every thread of a CTA on a segment's finished histogram: finds the bucket d0 of the
+// k-th largest key.  FUSED: the histogram holds only the entries at or above the predicted key,
+// all of them are the candidates, and the result stands only if there are at least k.
+// Otherwise the histogram is complete and the candidates are the entries from bucket d0 upwards.
+// On success stores d0, the rank still to find inside d0 and the candidate count, and returns
+// true.  The global histogram and the ticket are left zeroed either way.
 template <int THREADS, bool FUSED>
 __device__ __forceinline__ bool bucket_scan(const FastArgs &f, int64_t slot, int k, int *warp_tot, int *flag)
 {
@@ -132,12 +140,9 @@ __device__ __forceinline__ bool bucket_scan(const FastArgs &f, int64_t slot, int
 #pragma unroll
         for (int i = kPer - 1; i >= 0; --i) {
             if (above + hh[i] >= k) {
-                const int d0 = threadIdx.x * kPer + i;
-                f.prefix[slot] = (uint32_t)d0;
+                f.prefix[slot] = (uint32_t)(threadIdx.x * kPer + i);
                 f.k_rem[slot] = k - above;
                 if (!FUSED) f.seg_m[slot] = above + hh[i];
-                const int lbn = d0 - lb_margin(k);
-                f.lb[slot] = lbn > 1 ? lbn : 1;
                 *flag = 1;
                 break;
             }
@@ -146,13 +151,10 @@ __device__ __forceinline__ bool bucket_scan(const FastArgs &f, int64_t slot, int
     }
     if (FUSED && threadIdx.x == 0) f.seg_m[slot] = incl;      // thread 0's suffix sum is the total
     __syncthreads();
-    const bool ok = *flag != 0;
-    if (!ok && threadIdx.x == 0) f.lb[slot] = 0;              // no usable prediction
-    return ok;
+    return *flag != 0;
 }
 
-// (b) Leading-digit histogram of one tile-chunk.  Segments whose candidates the accumulation of
-// this step already produced are skipped.
+// (b) Leading-digit histogram of one tile-chunk; the CTA that completes a segment settles it.
 __global__ void __launch_bounds__(kSelThreads) hist0_fast_kernel(FastArgs f)
 {
     __shared__ unsigned h[kHistBins];
@@ -161,7 +163,6 @@ __global__ void __launch_bounds__(kSelThreads) hist0_fast_kernel(FastArgs f)
     const int row = blockIdx.y;
     const ChunkGeom g = chunk_geom(f, blockIdx.x);
     const int64_t slot = (int64_t)row * f.num_large + g.li;
-    if (f.seg_epoch[slot] == f.epoch) return;
     for (int b = threadIdx.x; b < kHistBins; b += kSelThreads) h[b] = 0;
     __syncthreads();
     const float *tile = f.data + (int64_t)(f.row0 + row) * f.row_stride + (int64_t)g.q * kSelChunk;
@@ -183,27 +184,21 @@ __global__ void __launch_bounds__(kSelThreads) hist0_fast_kernel(FastArgs f)
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    if (!bucket_scan<kSelThreads, false>(f, slot, f.seg_k[g.s], warp_tot, &scan_flag) && threadIdx.x == 0)
-        atomicExch(f.errword, 0x5E40);                         // a complete histogram always holds k entries
+    const bool ok = bucket_scan<kSelThreads, false>(f, slot, f.seg_k[g.s], warp_tot, &scan_flag);
+    if (threadIdx.x == 0) {
+        if (ok) f.seg_epoch[slot] = f.epoch;                   // settled for this step
+        else atomicExch(f.errword, 0x5E40);                    // a complete histogram always holds k entries
+    }
 }
 
 // (b) Candidates of one tile-chunk: positions (ascending) of the entries at or above the bucket
-// of the k-th key; skipped for segments already served by the accumulation and for segments that
-// will be finished from the data.  The first num_small CTAs each select one small segment.
-__global__ void __launch_bounds__(kSelThreads) collect_small_kernel(FastArgs f)
+// of the k-th key; skipped for segments that will be finished from the data.
+__global__ void __launch_bounds__(kSelThreads) collect_kernel(FastArgs f)
 {
-    __shared__ SmallShared small_sh;
-    const int row = blockIdx.y;
-    if ((int)blockIdx.x < f.num_small) {          // the longer-running CTAs go first
-        select_small_body(f.data, f.row_stride, f.row0, f.seg_off, f.seg_len, f.seg_k, f.seg_out,
-                          f.small_ids[blockIdx.x], row, f.out, f.out_stride, f.errword, small_sh);
-        return;
-    }
-    const int chunk = (int)blockIdx.x - f.num_small;
-    unsigned long long *warp_tot = reinterpret_cast<unsigned long long *>(small_sh.hist);
+    __shared__ unsigned long long warp_tot[kWarps];
+    const int row = blockIdx.y, chunk = blockIdx.x;
     const ChunkGeom g = chunk_geom(f, chunk);
     const int64_t slot = (int64_t)row * f.num_large + g.li;
-    if (f.seg_epoch[slot] == f.epoch) return;
     if ((int64_t)f.seg_m[slot] > f.comp_off[g.li + 1] - f.comp_off[g.li]) return;
     const float *tile = f.data + (int64_t)(f.row0 + row) * f.row_stride + (int64_t)g.q * kSelChunk;
     uint32_t key[kSelPerThread];
@@ -260,11 +255,11 @@ struct FinishShared {
 };
 
 // Completes the radix search below the 11-bit bucket d0 (k_rem entries still to find inside it)
-// and emits the k selected offsets in order.  Entries below the bucket, if the source has any,
-// are ignored.
+// and emits the k selected offsets in order; returns the k-th key.  Entries below the bucket, if
+// the source has any, are ignored.
 template <typename Source>
-__device__ void finish_from(const Source &src, uint32_t d0, int k_rem, int k, int32_t *__restrict__ out,
-                            FinishShared &sh, int32_t *errword)
+__device__ uint32_t finish_from(const Source &src, uint32_t d0, int k_rem, int k, int32_t *__restrict__ out,
+                                FinishShared &sh, int32_t *errword)
 {
     uint32_t prefix = d0 << 20, decided = 0x7ff00000u;
     const int shifts[3] = {12, 4, 0};
@@ -323,74 +318,119 @@ __device__ void finish_from(const Source &src, uint32_t d0, int k_rem, int k, in
         eq_done += (int)(total >> 16);
         if (gt_done + (eq_done < r ? eq_done : r) >= k) break;     // everything is emitted
     }
+    return T;
 }
 
-// One CTA per (large segment, row): compacts the segment's candidates in index order (thread t
-// owns chunk t of a group of 1024 chunks), then finishes on them; or on the data when the
-// candidates exceed the compact capacity.
+// The selection of one (segment, row) is completed by one CTA.  The first num_small CTAs of a
+// row each do one small segment outright.  For a large segment the CTA
+//  1. settles the bucket of the k-th key from the histogram the accumulation left, unless path
+//     (b) already did; if fewer than k entries had passed the predicted key it counts the
+//     leading digits of the whole segment itself;
+//  2. compacts the candidates in index order (thread t owns chunk t of a group of 1024 chunks)
+//     and finishes on them -- or on the data when there are no valid lists or too many entries;
+//  3. stores the key from which the next step should collect candidates.
 __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
 {
     __shared__ FinishShared sh;
+    __shared__ SmallShared small_sh;
+    __shared__ unsigned full_hist[kHistBins];
+    __shared__ int scan_flag;
     extern __shared__ __align__(16) uint32_t fin_dyn[];     // kFinSmemCap keys, then kFinSmemCap offsets
+    const int row = blockIdx.y;
+    if ((int)blockIdx.x < f.num_small) {
+        select_small_body(f.data, f.row_stride, f.row0, f.seg_off, f.seg_len, f.seg_k, f.seg_out,
+                          f.small_ids[blockIdx.x], row, f.out, f.out_stride, f.errword, small_sh);
+        return;
+    }
     uint32_t *s_key = fin_dyn;
     int32_t *s_idx = reinterpret_cast<int32_t *>(fin_dyn + kFinSmemCap);
-    const int li = blockIdx.x, row = blockIdx.y;
+    const int li = (int)blockIdx.x - f.num_small;
     const int64_t slot = (int64_t)row * f.num_large + li;
     const int s = f.large_ids[li];
     const int64_t off = f.seg_off[s];
     const int len = f.seg_len[s], k = f.seg_k[s];
     const float *rowp = f.data + (int64_t)(f.row0 + row) * f.row_stride;
     int32_t *out = f.out + (int64_t)row * f.out_stride + f.seg_out[s];
+    const int64_t cap = f.comp_off[li + 1] - f.comp_off[li];
+    bool lists = true;                        // the chunk lists hold this step's candidates
+    int path = 1;                             // 0: lists from the accumulation, 1: from the two passes, 2/3: data
+    if (f.seg_epoch[slot] != f.epoch) {
+        path = 0;       // not settled by path (b): use what the accumulation counted
+        lists = bucket_scan<kFinThreads, true>(f, slot, k, sh.warp_i, &scan_flag);
+        if (!lists) {
+            // no prediction, or too high: leading-digit histogram of the whole segment, in this CTA
+            for (int b = threadIdx.x; b < kHistBins; b += kFinThreads) full_hist[b] = 0;
+            __syncthreads();
+            for (int i = threadIdx.x; i < len; i += kFinThreads)
+                atomicAdd(&full_hist[mag_key(__ldg(rowp + off + i)) >> 20], 1u);
+            __syncthreads();
+            int part = (int)(full_hist[2 * threadIdx.x] + full_hist[2 * threadIdx.x + 1]);
+            const int incl = block_suffix_incl(part, sh.warp_i);
+            if (incl >= k && incl - part < k) {
+                const int hi = (int)full_hist[2 * threadIdx.x + 1];
+                const bool upper = incl - part + hi >= k;
+                f.prefix[slot] = (uint32_t)(2 * threadIdx.x + (upper ? 1 : 0));
+                f.k_rem[slot] = k - (incl - part) - (upper ? 0 : hi);
+            }
+            __syncthreads();
+        }
+    }
     const uint32_t d0 = f.prefix[slot];
     const int k_rem = f.k_rem[slot];
     const int m = f.seg_m[slot];
-    const int64_t cap = f.comp_off[li + 1] - f.comp_off[li];
-    if ((int64_t)m > cap) {                   // too many entries share the bucket: work on the data
+    uint32_t T;
+    if (!lists || (int64_t)m > cap) {
+        path = lists ? 3 : 2;
         DataSource src{rowp + off, off, len};
-        finish_from(src, d0, k_rem, k, out, sh, f.errword);
-        return;
-    }
-    const bool in_smem = m <= kFinSmemCap;
-    uint32_t *ckey = in_smem ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
-    int32_t *cidx = in_smem ? s_idx : f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
-    const int c0 = f.tchunk0[li], c1 = f.tchunk0[li + 1];
-    const int q0 = f.large_q0[li];
-    const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
-    int done = 0;
-    for (int base = c0; base < c1; base += kFinThreads) {
-        const int c = base + (int)threadIdx.x;
-        const unsigned n = c < c1 ? (unsigned)cnt[c] : 0u;
-        unsigned total;
-        unsigned at = (unsigned)done + block_prefix_excl<unsigned>(n, sh.warp_u, &total);
-        if (n) {
-            // eight positions per 128-bit load, then eight independent gathers
-            const uint4 *pos8 = reinterpret_cast<const uint4 *>(f.cand_pos + ((int64_t)row * f.num_tchunks + c) * kSelChunk);
-            const int tile_base = (q0 + (c - c0)) * kSelChunk;          // N < 2^31
-            for (unsigned b0 = 0; b0 < n; b0 += 8) {
-                const uint4 pv = pos8[b0 >> 3];
-                const unsigned w[4] = {pv.x, pv.y, pv.z, pv.w};
-                uint32_t kk[8];
+        T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
+    } else {
+        const bool in_smem = m <= kFinSmemCap;
+        uint32_t *ckey = in_smem ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
+        int32_t *cidx = in_smem ? s_idx : f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
+        const int c0 = f.tchunk0[li], c1 = f.tchunk0[li + 1];
+        const int q0 = f.large_q0[li];
+        const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
+        int done = 0;
+        for (int base = c0; base < c1; base += kFinThreads) {
+            const int c = base + (int)threadIdx.x;
+            const unsigned n = c < c1 ? (unsigned)cnt[c] : 0u;
+            unsigned total;
+            unsigned at = (unsigned)done + block_prefix_excl<unsigned>(n, sh.warp_u, &total);
+            if (n) {
+                // eight positions per 128-bit load, then eight independent gathers
+                const uint4 *pos8 =
+                    reinterpret_cast<const uint4 *>(f.cand_pos + ((int64_t)row * f.num_tchunks + c) * kSelChunk);
+                const int tile_base = (q0 + (c - c0)) * kSelChunk;          // N < 2^31
+                for (unsigned b0 = 0; b0 < n; b0 += 8) {
+                    const uint4 pv = pos8[b0 >> 3];
+                    const unsigned w[4] = {pv.x, pv.y, pv.z, pv.w};
+                    uint32_t kk[8];
 #pragma unroll
-                for (int b = 0; b < 8; ++b) {
-                    const int j = tile_base + (int)(w[b >> 1] >> (16 * (b & 1)) & 0xffffu);
-                    kk[b] = b0 + b < n ? mag_key(__ldg(rowp + j)) : 0u;
-                }
-#pragma unroll
-                for (int b = 0; b < 8; ++b) {
-                    if (b0 + b < n && at + b < (unsigned)m) {
-                        ckey[at + b] = kk[b];
-                        cidx[at + b] = tile_base + (int)(w[b >> 1] >> (16 * (b & 1)) & 0xffffu);
+                    for (int b = 0; b < 8; ++b) {
+                        const int j = tile_base + (int)(w[b >> 1] >> (16 * (b & 1)) & 0xffffu);
+                        kk[b] = b0 + b < n ? mag_key(__ldg(rowp + j)) : 0u;
                     }
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) {
+                        if (b0 + b < n && at + b < (unsigned)m) {
+                            ckey[at + b] = kk[b];
+                            cidx[at + b] = tile_base + (int)(w[b >> 1] >> (16 * (b & 1)) & 0xffffu);
+                        }
+                    }
+                    at += 8;
                 }
-                at += 8;
             }
+            done += (int)total;
         }
-        done += (int)total;
+        if (threadIdx.x == 0 && done != m) atomicExch(f.errword, 0x5E70);
+        __syncthreads();
+        CompactSource src{ckey, cidx, m};
+        T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
     }
-    if (threadIdx.x == 0 && done != m) atomicExch(f.errword, 0x5E70);
-    __syncthreads();
-    CompactSource src{ckey, cidx, m};
-    finish_from(src, d0, k_rem, k, out, sh, f.errword);
+    if (threadIdx.x == 0) {
+        f.lbkey[slot] = predict_lbkey(T, k);
+        f.seg_path[slot] = path;
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -401,6 +441,31 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
 // histogrammed and listed, and the CTA that completes the segment settles the bucket of its k-th
 // key.
 // ------------------------------------------------------------------------------------------
+// The part [lo, hi) of a tile, held four consecutive entries per thread (positions p0 .. p0+3):
+// entries whose key reaches lbkey are added to the segment's leading-digit histogram and their
+// positions written, ascending, to the chunk's list.
+__device__ __forceinline__ void collect_tile(const FastArgs &f, int64_t slot, int64_t chunk, const uint32_t (&key)[4],
+                                             uint32_t lbkey, bool live, int p0, int lo, int hi, unsigned *warp_u)
+{
+    unsigned flags = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        if (live && p0 + i >= lo && p0 + i < hi && key[i] >= lbkey) flags |= 1u << i;
+    uint32_t *gh = f.hist + slot * kHistBins;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        if (flags >> i & 1u) atomicAdd(gh + (key[i] >> 20), 1u);
+    unsigned total;
+    unsigned at = block_prefix_excl<unsigned>((unsigned)__popc(flags), warp_u, &total);
+    if (threadIdx.x == 0) f.cand_cnt[chunk] = (int)total;
+    if (flags) {
+        uint16_t *dst = f.cand_pos + chunk * kSelChunk;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (flags >> i & 1u) dst[at++] = (uint16_t)(p0 + i);
+    }
+}
+
 __device__ __forceinline__ void acc4(float4 &u, float4 &v, const float4 &g, float m)
 {
     u.x = __fmaf_rn(m, u.x, g.x); v.x = __fadd_rn(v.x, u.x);
@@ -414,8 +479,6 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, float *__restr
                          int64_t N, float m, int sel_row0, int sel_rows)
 {
     __shared__ unsigned warp_u[kAccThreads / 32];
-    __shared__ int warp_i[kAccThreads / 32];
-    __shared__ int is_last, scan_flag;
     const int row = blockIdx.y, q = blockIdx.x;
     const int64_t tile_base = (int64_t)q * kSelChunk;
     const int in_tile = N - tile_base < kSelChunk ? (int)(N - tile_base) : kSelChunk;    // a multiple of 4
@@ -433,49 +496,30 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, float *__restr
     }
     const int sel = row - sel_row0;
     if (sel < 0 || sel >= sel_rows) return;
+    const int4 desc = f.tile_desc[q];           // x: first segment, y: the one large segment covering the tile
+                                                // (-1: several segments, -2: no large segment), z: its chunk
+    if (desc.y == -2) return;
     const uint32_t key[4] = {mag_key(vv.x), mag_key(vv.y), mag_key(vv.z), mag_key(vv.w)};
+    if (desc.y >= 0) {
+        const int64_t slot = (int64_t)sel * f.num_large + desc.y;
+        const uint32_t lbkey = f.lbkey[slot];
+        if (lbkey == 0) return;                                  // no prediction: the finishing CTA counts itself
+        collect_tile(f, slot, (int64_t)sel * f.num_tchunks + desc.z, key, lbkey, live, p0, 0, in_tile, warp_u);
+        return;
+    }
     const int64_t tile_end = tile_base + in_tile;
-    for (int s = f.tile_seg0[q]; s < f.num_large + f.num_small && f.seg_off[s] < tile_end; ++s) {
+    for (int s = desc.x; s < f.num_large + f.num_small && f.seg_off[s] < tile_end; ++s) {
         const int li = f.seg_large[s];
         if (li < 0) continue;
         const int64_t slot = (int64_t)sel * f.num_large + li;
-        const uint32_t lb = (uint32_t)f.lb[slot];
-        if (lb == 0) continue;                                  // no prediction: path (b) will serve it
+        const uint32_t lbkey = f.lbkey[slot];
+        if (lbkey == 0) continue;
         const int64_t off = f.seg_off[s], end = off + f.seg_len[s];
         const int lo = off > tile_base ? (int)(off - tile_base) : 0;
         const int hi = end < tile_end ? (int)(end - tile_base) : in_tile;
-        unsigned flags = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (live && p0 + i >= lo && p0 + i < hi && (key[i] >> 20) >= lb) flags |= 1u << i;
-        uint32_t *gh = f.hist + slot * kHistBins;
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-            if (flags >> i & 1u) atomicAdd(gh + (key[i] >> 20), 1u);
-        unsigned total;
-        unsigned at = block_prefix_excl<unsigned>((unsigned)__popc(flags), warp_u, &total);
-        const int64_t c = (int64_t)sel * f.num_tchunks + f.tchunk0[li] + (q - f.large_q0[li]);
-        if (threadIdx.x == 0) f.cand_cnt[c] = (int)total;
-        if (flags) {
-            uint16_t *dst = f.cand_pos + c * kSelChunk;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (flags >> i & 1u) dst[at++] = (uint16_t)(p0 + i);
-        }
-        __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            const int chunks = f.tchunk0[li + 1] - f.tchunk0[li];
-            is_last = atomicAdd(&f.seg_ticket[slot], 1) == chunks - 1;
-        }
-        __syncthreads();
-        const bool last = is_last != 0;                         // uniform over the CTA
-        __syncthreads();                                        // everyone has read it before it is reused
-        if (last) {
-            __threadfence();
-            const bool ok = bucket_scan<kAccThreads, true>(f, slot, f.seg_k[s], warp_i, &scan_flag);
-            if (ok && threadIdx.x == 0) f.seg_epoch[slot] = f.epoch;
-        }
+        collect_tile(f, slot, (int64_t)sel * f.num_tchunks + f.tchunk0[li] + (q - f.large_q0[li]), key, lbkey, live,
+                     p0, lo, hi, warp_u);
+        __syncthreads();                                         // warp_u is reused by the next segment
     }
 }
 
@@ -486,32 +530,24 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
     f.num_large = t.num_large; f.num_small = t.num_small; f.num_tchunks = t.num_tchunks; f.epoch = epoch;
     f.seg_off = t.seg_off; f.seg_len = t.seg_len; f.seg_k = t.seg_k; f.seg_out = t.seg_out;
     f.small_ids = t.small_ids; f.large_ids = t.large_ids; f.seg_large = t.seg_large; f.large_q0 = t.large_q0;
-    f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_seg0 = t.tile_seg0;
+    f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_desc = t.tile_desc;
     f.hist = t.hist; f.prefix = t.prefix; f.k_rem = t.k_rem; f.cand_cnt = t.cand_cnt; f.seg_m = t.seg_m;
-    f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.lb = t.lb; f.cand_pos = t.cand_pos;
+    f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.seg_path = t.seg_path; f.lbkey = t.lbkey; f.cand_pos = t.cand_pos;
     f.comp_off = t.comp_off; f.comp_total = t.comp_total; f.comp_key = t.comp_key; f.comp_idx = t.comp_idx;
     f.out = out; f.out_stride = out_stride; f.errword = errword;
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_small_only_kernel(FastArgs f)
-{
-    __shared__ SmallShared sh;
-    select_small_body(f.data, f.row_stride, f.row0, f.seg_off, f.seg_len, f.seg_k, f.seg_out, f.small_ids[blockIdx.x],
-                      blockIdx.y, f.out, f.out_stride, f.errword, sh);
-}
-
 }  // namespace
 
+// `served`: the accumulation of this step collected the candidates of exactly these rows (path a);
+// otherwise the two passes of path (b) run first.
 cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0, int rows,
-                          int32_t *out, int64_t out_stride, int32_t epoch, int32_t *errword, cudaStream_t st)
+                          int32_t *out, int64_t out_stride, bool served, int32_t epoch, int32_t *errword,
+                          cudaStream_t st)
 {
     if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
     FastArgs f;
     fill_args(f, t, data, row_stride, row0, out, out_stride, epoch, errword);
-    if (!t.num_large) {
-        select_small_only_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
-        return cudaGetLastError();
-    }
     constexpr int kFinDyn = 2 * kFinSmemCap * (int)sizeof(uint32_t);
     static bool configured = false;
     if (!configured) {
@@ -519,9 +555,14 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    hist0_fast_kernel<<<dim3(t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
-    collect_small_kernel<<<dim3(t.num_small + t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
-    finish_kernel<<<dim3(t.num_large, rows), kFinThreads, kFinDyn, st>>>(f), ++g_kernel_launches;
+    if (t.num_large && !served) {
+        // whatever an accumulation may have counted for other rows must not mix in
+        const cudaError_t e = launch_zero(t.hist, (size_t)rows * t.num_large * kHistBins * sizeof(uint32_t), st);
+        if (e != cudaSuccess) return e;
+        hist0_fast_kernel<<<dim3(t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
+        collect_kernel<<<dim3(t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
+    }
+    finish_kernel<<<dim3(t.num_small + t.num_large, rows), kFinThreads, kFinDyn, st>>>(f), ++g_kernel_launches;
     return cudaGetLastError();
 }
 

@@ -23,7 +23,7 @@ EXPORTS = (
     "lgc_workspace_bytes", "lgc_init", "lgc_destroy", "lgc_accumulate", "lgc_topk", "lgc_encode",
     "lgc_combine", "lgc_decode_scatter", "lgc_topk_scatter", "lgc_ae_train_step", "lgc_step_host",
     "lgc_get_layout", "lgc_keep_counts", "lgc_get_buffers", "lgc_set_ae_params", "lgc_get_ae_params",
-    "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc", "lgc_kernel_launches",
+    "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc", "lgc_kernel_launches", "lgc_selection_stats",
 )
 NOALLOC_MAX_N = 16777216
 
@@ -72,6 +72,7 @@ def lib() -> C.CDLL:
         l.lgc_last_error.argtypes = [vp]
         l.lgc_last_error.restype = C.c_char_p
         l.lgc_topk_noalloc.argtypes = [vp, C.c_int64, C.c_int64, vp, vp]
+        l.lgc_selection_stats.argtypes = [vp] + [C.POINTER(C.c_int64)] * 4
         l.lgc_kernel_launches.argtypes = []
         l.lgc_kernel_launches.restype = C.c_uint64
         for name in EXPORTS:            # every declared entry point must be exported
@@ -220,6 +221,12 @@ class LGC:
                                        self._dev_f32(dev_grads, self.K * self.N, "dev_grads"),
                                        self._dev_f32(dev_update, self.N, "dev_update"),
                                        host_update.data_ptr(), choice), "lgc_step_host")
+
+    def selection_stats(self):
+        """(large (row, layer) pairs, pairs served by the last accumulate, candidates in total, largest count)."""
+        v = [C.c_int64() for _ in range(4)]
+        self._ok(self._l.lgc_selection_stats(self._ctx, *[C.byref(x) for x in v]), "lgc_selection_stats")
+        return tuple(x.value for x in v)
 
     def check(self) -> None:
         self._ok(self._l.lgc_check(self._ctx), "lgc_check")
