@@ -210,7 +210,7 @@ def run_ours(args, w: W.Workload):
         ev[t][0].record()
         gpu.accumulate(grads[i % GRAD_SETS], choices[i])
         ev[t][1].record()
-        gpu.topk(choices[i])
+        gpu.topk(choices[i], update)
         gpu.encode()
         gpu.combine(choices[i])
         gpu.decode_scatter(update)

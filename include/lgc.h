@@ -108,8 +108,13 @@ lgc_status lgc_accumulate(lgc_ctx *ctx, const float *grads, int32_t leader_hint)
  * entries of largest |v| (equal magnitudes: the lower index wins), in ascending index order,
  * layers in order, then the gather of the kept values g~_k in R^mu for every node.
  * Ring-allreduce: only node `leader` selects and all nodes use its indices.
- * Parameter server: every node selects on its own; `leader` is ignored. */
-lgc_status lgc_topk(lgc_ctx *ctx, int32_t leader);
+ * Parameter server: every node selects on its own; `leader` is ignored.
+ * update_hint: NULL, or the device buffer (fp32 [N], 16-byte aligned) that this step's
+ * lgc_decode_scatter / lgc_topk_scatter will be given.  With a hint the library clears that buffer
+ * while the selection runs (spare thread blocks of the same launch), so that the scatter call
+ * only writes the kept entries; the caller must leave the buffer alone from this call until the
+ * scatter call has run.  A different buffer may still be passed later (it is then cleared there). */
+lgc_status lgc_topk(lgc_ctx *ctx, int32_t leader, float *update_hint);
 
 /* Stage 4a -- Section IV: g~^c_k = E_c(g~_k) for every node: Conv1d(1->c1, 3 taps, stride 2),
  * ReLU, Conv1d(c1->c2, 3 taps, stride 2), no padding. */

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 
 #include "lgc_internal.cuh"
@@ -111,7 +112,8 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
 // large ones are cut by the row's tiles of kSelChunk elements.
 struct SelectPlan {
     std::vector<int64_t> seg_off, comp_off;
-    std::vector<int32_t> seg_len, seg_k, seg_out, small_ids, large_ids, seg_large, large_q0, tchunk0, tchunk_large;
+    std::vector<int32_t> seg_len, seg_k, seg_out, small_ids, large_ids, seg_large, large_q0, large_order, tchunk0,
+        tchunk_large;
     std::vector<int4> tile_desc;
     int tiles_per_row = 0;
     int64_t comp_total = 0;
@@ -144,6 +146,11 @@ SelectPlan plan_select(const std::vector<int64_t> &off, const std::vector<int64_
         }
     }
     sp.comp_total = sp.comp_off.back();
+    sp.large_order.resize(sp.large_ids.size());
+    for (size_t i = 0; i < sp.large_order.size(); ++i) sp.large_order[i] = (int32_t)i;
+    std::stable_sort(sp.large_order.begin(), sp.large_order.end(), [&](int32_t a, int32_t b) {
+        return len[sp.large_ids[a]] > len[sp.large_ids[b]];
+    });
     const int64_t row_len = off[n - 1] + len[n - 1];
     sp.tiles_per_row = (int)((row_len + kSelChunk - 1) / kSelChunk);
     int s = 0;
@@ -177,6 +184,7 @@ void carve_select(Carver &cv, SelectTables &t, const SelectPlan &sp, int rows)
     t.small_ids = cv.take<int32_t>(ns);
     t.large_ids = cv.take<int32_t>(nl);
     t.large_q0 = cv.take<int32_t>(nl);
+    t.large_order = cv.take<int32_t>(nl);
     t.tchunk0 = cv.take<int32_t>(nl + 1);
     t.tchunk_large = cv.take<int32_t>(nc);
     t.tile_desc = cv.take<int4>(sp.tiles_per_row);
@@ -259,10 +267,10 @@ cudaError_t upload_select(SelectTables &t, SelectPlan sp, cudaStream_t s, std::v
     if (e == cudaSuccess) e = upload(t.comp_off, h.comp_off, s);
     if (e == cudaSuccess) e = upload(t.tile_desc, h.tile_desc, s);
     const std::vector<int32_t> *arrs[] = {&h.seg_len, &h.seg_k, &h.seg_out, &h.seg_large, &h.small_ids, &h.large_ids,
-                                          &h.large_q0, &h.tchunk0, &h.tchunk_large};
+                                          &h.large_q0, &h.large_order, &h.tchunk0, &h.tchunk_large};
     int32_t *dsts[] = {t.seg_len, t.seg_k, t.seg_out, t.seg_large, t.small_ids, t.large_ids,
-                       t.large_q0, t.tchunk0, t.tchunk_large};
-    for (int i = 0; i < 9 && e == cudaSuccess; ++i) e = upload(dsts[i], *arrs[i], s);
+                       t.large_q0, t.large_order, t.tchunk0, t.tchunk_large};
+    for (int i = 0; i < 10 && e == cudaSuccess; ++i) e = upload(dsts[i], *arrs[i], s);
     return e;
 }
 
@@ -365,6 +373,7 @@ lgc_status lgc_accumulate(lgc_ctx *c, const float *grads, int32_t leader_hint)
     const bool ps = c->cfg.variant == LGC_VARIANT_PS;
     if (!ps && leader_hint >= c->K) return fail(c, LGC_ERR_INVALID_ARG, "leader_hint out of range");
     c->epoch = c->epoch == 0x7fffffff ? 1 : c->epoch + 1;
+    c->cleared_update = nullptr;
     cudaError_t e;
     // the fused form needs rows that start 16-byte aligned, someone to select for, and the keys a
     // previous selection left to collect against
@@ -381,16 +390,18 @@ lgc_status lgc_accumulate(lgc_ctx *c, const float *grads, int32_t leader_hint)
     return LGC_OK;
 }
 
-lgc_status lgc_topk(lgc_ctx *c, int32_t leader)
+lgc_status lgc_topk(lgc_ctx *c, int32_t leader, float *update_hint)
 {
     if (!c) return LGC_ERR_INVALID_ARG;
     if (c->stage != Ctx::kAccumulated) return fail(c, LGC_ERR_BAD_STATE, "lgc_topk must follow lgc_accumulate");
+    if (update_hint && !aligned16(update_hint)) return fail(c, LGC_ERR_INVALID_ARG, "update_hint is not 16-byte aligned");
     const bool ps = c->cfg.variant == LGC_VARIANT_PS;
     if (!ps && (leader < 0 || leader >= c->K)) return fail(c, LGC_ERR_INVALID_ARG, "leader out of range");
     // candidates collected during the accumulation count only if they are this leader's
     const bool served = ps ? c->fused_leader == -1 : c->fused_leader == leader;
     cudaError_t e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, served, c->epoch,
-                                  c->errword, c->stream);
+                                  update_hint, c->N, c->errword, c->stream);
+    c->cleared_update = c->sel_v.num_large ? update_hint : nullptr;
     c->have_prediction = true;
     c->val_valid = false;
     c->mean_valid = false;
@@ -472,7 +483,7 @@ lgc_status lgc_step_host(lgc_ctx *c, const float *host_grads, float *dev_grads, 
     cudaError_t e = cudaMemcpyAsync(dev_grads, host_grads, (size_t)c->K * c->N * sizeof(float), cudaMemcpyHostToDevice, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (upload)");
     lgc_status st = lgc_accumulate(c, dev_grads, choice);
-    if (st == LGC_OK) st = lgc_topk(c, choice);
+    if (st == LGC_OK) st = lgc_topk(c, choice, dev_update);
     if (st == LGC_OK) st = lgc_encode(c);
     if (st == LGC_OK) st = lgc_combine(c, choice);
     if (st == LGC_OK) st = lgc_decode_scatter(c, dev_update);

@@ -269,8 +269,8 @@ constexpr int kDenseThreads = 256;
 // whose index falls into its range (the range of kept slots of a tile comes from tile_lo),
 // places them in the tile, removes those entries from every node's u and v, and streams the
 // tile out: every entry of the update is written exactly once and no store waits for another.
-// MODE 0: two-layer decoder on the mean code; 1: identity (the mean code is the value);
-// 2: mean over nodes of the kept values.
+// MODE 0: the values are the decoder's output already in recon; 1: identity (the mean code is
+// the value); 2: mean over nodes of the kept values.
 template <int C1, int C2, int MODE>
 __global__ void __launch_bounds__(kDenseThreads)
 dense_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val, const int32_t *__restrict__ idx,
@@ -289,8 +289,7 @@ dense_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val,
     for (int64_t p = lo + threadIdx.x; p < hi; p += kDenseThreads) {
         float y;
         if (MODE == 0) {
-            const float *w1 = dec, *b1 = dec + C2 * C1 * 3, *w2 = b1 + C1;
-            y = decode_at<C1, C2>(p, z, L1, L2, w1, b1, w2, __ldg(w2 + C1 * 3));
+            y = recon[p];                 // decoded by decode_kernel just before
         } else if (MODE == 1) {
             y = z[p];
         } else {
@@ -298,13 +297,8 @@ dense_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val,
             for (int k = 1; k < K; ++k) y = __fadd_rn(y, val[(int64_t)k * mu + p]);
             y = __fdiv_rn(y, (float)K);
         }
-        const int32_t i = idx[p];
-        tile[i - base] = y;
-        recon[p] = y;
-        for (int k = 0; k < K; ++k) {
-            u[(int64_t)k * N + i] = 0.0f;
-            v[(int64_t)k * N + i] = 0.0f;
-        }
+        tile[idx[p] - base] = y;
+        if (MODE != 0) recon[p] = y;
     }
     __syncthreads();
     float *dst = update + base;
@@ -314,6 +308,53 @@ dense_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val,
             __stcs(reinterpret_cast<float4 *>(dst) + i, reinterpret_cast<const float4 *>(tile)[i]);
     } else {
         for (int i = threadIdx.x; i < (int)(end - base); i += kDenseThreads) dst[i] = tile[i];
+    }
+    // the sent entries leave every node's u and v; these scattered stores come last so that no
+    // thread reaches the barrier late because of them
+    for (int64_t p = lo + threadIdx.x; p < hi; p += kDenseThreads) {
+        const int32_t i = idx[p];
+        for (int k = 0; k < K; ++k) {
+            u[(int64_t)k * N + i] = 0.0f;
+            v[(int64_t)k * N + i] = 0.0f;
+        }
+    }
+}
+
+// Ring-allreduce stage 5 when the update buffer has been cleared already: decode (MODE 0), take the
+// mean code (1) or average the kept values (2) for slot p, write it at its index, and remove the
+// entry from every node's u and v.  One thread per kept slot.
+template <int C1, int C2, int MODE>
+__global__ void __launch_bounds__(kAeThreads)
+sparse_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val, const int32_t *__restrict__ idx,
+                      int64_t mu, int64_t L1, int64_t L2, const float *__restrict__ dec, int K, int64_t N,
+                      float *__restrict__ recon, float *__restrict__ update, float *__restrict__ u,
+                      float *__restrict__ v)
+{
+    constexpr int kDec = C2 * C1 * 3 + C1 + C1 * 3 + 1;
+    __shared__ float w[kDec];
+    if (MODE == 0) {
+        for (int i = threadIdx.x; i < kDec; i += kAeThreads) w[i] = dec[i];
+        __syncthreads();
+    }
+    const int64_t p = (int64_t)blockIdx.x * kAeThreads + threadIdx.x;
+    if (p >= mu) return;
+    const int32_t i = idx[p];
+    float y;
+    if (MODE == 0) {
+        const float *w1 = w, *b1 = w + C2 * C1 * 3, *w2 = b1 + C1;
+        y = decode_at<C1, C2>(p, z, L1, L2, w1, b1, w2, w2[C1 * 3]);
+    } else if (MODE == 1) {
+        y = z[p];
+    } else {
+        y = val[p];
+        for (int k = 1; k < K; ++k) y = __fadd_rn(y, val[(int64_t)k * mu + p]);
+        y = __fdiv_rn(y, (float)K);
+    }
+    update[i] = y;
+    recon[p] = y;
+    for (int k = 0; k < K; ++k) {
+        u[(int64_t)k * N + i] = 0.0f;
+        v[(int64_t)k * N + i] = 0.0f;
     }
 }
 
@@ -416,7 +457,8 @@ cudaError_t launch_combine_ps(Ctx &c, int common_node)
                                                                    c.code_len, c.combined), ++g_kernel_launches;
     cudaError_t e = launch_zero(c.inn, (size_t)c.K * c.mu * sizeof(float), c.stream);
     if (e != cudaSuccess) return e;
-    e = launch_select(c.sel_inn, c.val, c.mu, 0, c.K, c.inn_pos, c.muI, false, ++c.inn_epoch, c.errword, c.stream);
+    e = launch_select(c.sel_inn, c.val, c.mu, 0, c.K, c.inn_pos, c.muI, false, ++c.inn_epoch, nullptr, 0, c.errword,
+                      c.stream);
     if (e != cudaSuccess) return e;
     innovation_fill_kernel<<<dim3(blocks_for(c.muI, 256), c.K), 256, 0, c.stream>>>(c.val, c.inn_pos, c.mu, c.muI, c.inn), ++g_kernel_launches;
     return cudaGetLastError();
@@ -424,8 +466,10 @@ cudaError_t launch_combine_ps(Ctx &c, int common_node)
 
 static cudaError_t launch_scatter(Ctx &c, const float *values, float *update)
 {
-    cudaError_t e = launch_zero(update, (size_t)c.N * sizeof(float), c.stream);
-    if (e != cudaSuccess) return e;
+    if (update != c.cleared_update) {       // otherwise lgc_topk's finishing launch has cleared it already
+        const cudaError_t e = launch_zero(update, (size_t)c.N * sizeof(float), c.stream);
+        if (e != cudaSuccess) return e;
+    }
     if (c.S == 1)
         scatter_shared_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(values, c.idx, c.mu, c.K, c.N, update, c.u, c.v), ++g_kernel_launches;
     else
@@ -437,12 +481,29 @@ static cudaError_t launch_scatter(Ctx &c, const float *values, float *update)
 // Ring-allreduce: the whole of stage 5 (or the phase-two sparse mean) in one pass over the update.
 static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update)
 {
+    const float *dec = c.params + c.Penc;
+    if (update == c.cleared_update) {
+        // lgc_topk's finishing launch has cleared the buffer: only the kept entries are written
+        const unsigned sgrid = blocks_for(c.mu, kAeThreads);
+        if (mode == 1) {
+            sparse_scatter_kernel<3, 2, 1><<<sgrid, kAeThreads, 0, c.stream>>>(
+                c.combined, c.val, c.idx, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
+        } else if (mode == 2) {
+            sparse_scatter_kernel<3, 2, 2><<<sgrid, kAeThreads, 0, c.stream>>>(
+                c.combined, c.val, c.idx, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
+        } else {
+#define CALL(A, B) sparse_scatter_kernel<A, B, 0><<<sgrid, kAeThreads, 0, c.stream>>>(                                \
+        c.combined, c.val, c.idx, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v)
+            LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
+#undef CALL
+        }
+        return cudaGetLastError();
+    }
     if (!c.tile_lo_valid) {
         tile_lo_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(c.idx, c.mu, c.N, c.tile_lo), ++g_kernel_launches;
         c.tile_lo_valid = true;
     }
     const unsigned grid = blocks_for(c.N, kDenseTile);
-    const float *dec = c.params + c.Penc;
     if (mode == 1) {
         dense_scatter_kernel<3, 2, 1><<<grid, kDenseThreads, 0, c.stream>>>(
             c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
@@ -450,10 +511,15 @@ static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update)
         dense_scatter_kernel<3, 2, 2><<<grid, kDenseThreads, 0, c.stream>>>(
             c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
     } else {
-#define CALL(A, B) dense_scatter_kernel<A, B, 0><<<grid, kDenseThreads, 0, c.stream>>>(                               \
-        c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v)
+        // the decoder runs as its own short, fully parallel launch: inside the dense pass its serial
+        // chain would hold every CTA's barrier for several microseconds
+        const dim3 dgrid(blocks_for(c.mu, kAeThreads), 1);
+#define CALL(A, B) decode_kernel<A, B, false><<<dgrid, kAeThreads, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec,    \
+                                                                                 (int)c.Pdec, nullptr, c.recon)
         LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
 #undef CALL
+        dense_scatter_kernel<3, 2, 0><<<grid, kDenseThreads, 0, c.stream>>>(
+            c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
     }
     return cudaGetLastError();
 }

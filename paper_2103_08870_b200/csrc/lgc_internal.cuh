@@ -46,6 +46,7 @@ struct SelectTables {
     int tiles_per_row = 0;
     int32_t *seg_large = nullptr;    // [S] index into large_ids, -1 for small segments
     int32_t *large_q0 = nullptr;     // [num_large] first tile the segment overlaps
+    int32_t *large_order = nullptr;  // [num_large] indices into large_ids, longest segment first
     int32_t *tchunk0 = nullptr;      // [num_large + 1] first tile-chunk of each large segment
     int32_t *tchunk_large = nullptr; // [num_tchunks] index into large_ids
     int4 *tile_desc = nullptr;       // [tiles_per_row] x: first segment the tile overlaps; y: the large segment that
@@ -111,6 +112,7 @@ struct Ctx {
     int32_t last_leader = 0;
     int32_t epoch = 0;             // step counter (accumulations so far)
     int32_t inn_epoch = 0;         // the same counter for the innovation selection's tables
+    float *cleared_update = nullptr; // buffer the last lgc_topk already cleared (its first N & ~3 floats)
     bool have_prediction = false;  // a selection has run, so the next accumulation has keys to collect against
     int32_t fused_leader = -2;     // row whose candidates the last accumulation collected (-1: all rows, -2: none)
     bool val_valid = false;        // val holds the kept values of the current selection
@@ -126,9 +128,11 @@ extern thread_local std::string g_last_error;   // failures without a context (s
 cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s);
 cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s);
 // served: the accumulation of step `epoch` collected the candidates of exactly these rows.
+// clear/clear_floats: optional 16-byte aligned buffer that spare CTAs of the finishing launch set to zero
+// (only when the tables have large segments).
 cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0,
-                          int rows, int32_t *out, int64_t out_stride, bool served, int32_t epoch, int32_t *errword,
-                          cudaStream_t s);
+                          int rows, int32_t *out, int64_t out_stride, bool served, int32_t epoch, float *clear,
+                          int64_t clear_floats, int32_t *errword, cudaStream_t s);
 // Accumulation that also collects the selection candidates of the selecting rows (sel_row0 .. +sel_rows
 // of the K rows) against the predicted buckets; needs N % 4 == 0.
 cudaError_t launch_accumulate_select(const SelectTables &t, const float *g, float *u, float *v, int K, int64_t N,

@@ -32,6 +32,11 @@ struct FastArgs {
     int64_t row_stride;
     int row0;
     int num_large, num_small, num_tchunks;
+    int fin_small;                 // small segments served by CTAs of finish_kernel (0 or num_small)
+    const int32_t *large_order;    // large segments, longest first: the order the finishing CTAs take them in
+    uint4 *zero_ptr;               // buffer the spare CTAs of the finishing launch clear (row 0 only), or nullptr
+    uint64_t zero_vecs;            // its length in whole 16-byte units
+    int zero_tail;                 // floats beyond them (0..3)
     int32_t epoch;                 // step whose fused accumulation may have filled the lists (-1: none)
     const int64_t *seg_off;
     const int32_t *seg_len, *seg_k, *seg_out, *small_ids, *large_ids, *seg_large, *large_q0, *tchunk0, *tchunk_large;
@@ -48,10 +53,11 @@ struct FastArgs {
     int32_t *errword;
 };
 
-constexpr int kFinThreads = 1024;
+constexpr int kFinThreads = 512;      // two finishing CTAs fit on an SM, so every segment of a ResNet starts at once
 constexpr int kFinWarps = kFinThreads / 32;
 constexpr int kFinSmemCap = 8192;     // candidates a finishing CTA keeps in shared memory
 constexpr int kFinPerThread = 4;      // consecutive entries per thread in the ordered passes
+constexpr int kZeroPerThread = 8;     // 16-byte stores per thread of a CTA that clears a slice of the update
 constexpr int kAccThreads = 1024;     // accumulation: one 128-bit g/u/v triple per thread, 4096 elements per CTA
 
 // The key from which the next step collects candidates, given this step's k-th key T.  Error
@@ -326,9 +332,11 @@ __device__ uint32_t finish_from(const Source &src, uint32_t d0, int k_rem, int k
 //  1. settles the bucket of the k-th key from the histogram the accumulation left, unless path
 //     (b) already did; if fewer than k entries had passed the predicted key it counts the
 //     leading digits of the whole segment itself;
-//  2. compacts the candidates in index order (thread t owns chunk t of a group of 1024 chunks)
+//  2. compacts the candidates in index order (thread t owns chunk t of a group of chunks)
 //     and finishes on them -- or on the data when there are no valid lists or too many entries;
 //  3. stores the key from which the next step should collect candidates.
+// CTA order: large segments longest first, then the small ones, then spare CTAs that clear the
+// dense update buffer (if the caller announced it) while the rest of the launch is busy.
 __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
 {
     __shared__ FinishShared sh;
@@ -337,14 +345,26 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
     __shared__ int scan_flag;
     extern __shared__ __align__(16) uint32_t fin_dyn[];     // kFinSmemCap keys, then kFinSmemCap offsets
     const int row = blockIdx.y;
-    if ((int)blockIdx.x < f.num_small) {
+    if ((int)blockIdx.x >= f.num_large + f.fin_small) {      // spare CTAs: clear the dense update meanwhile
+        if (row != 0) return;
+        const uint64_t first = (uint64_t)(blockIdx.x - f.num_large - f.fin_small) * (kFinThreads * kZeroPerThread);
+#pragma unroll
+        for (int i = 0; i < kZeroPerThread; ++i) {
+            const uint64_t e = first + (uint64_t)i * kFinThreads + threadIdx.x;
+            if (e < f.zero_vecs) __stcs(f.zero_ptr + e, make_uint4(0u, 0u, 0u, 0u));
+            else if (e == f.zero_vecs)
+                for (int j = 0; j < f.zero_tail; ++j) reinterpret_cast<float *>(f.zero_ptr + e)[j] = 0.0f;
+        }
+        return;
+    }
+    if ((int)blockIdx.x >= f.num_large) {
         select_small_body(f.data, f.row_stride, f.row0, f.seg_off, f.seg_len, f.seg_k, f.seg_out,
-                          f.small_ids[blockIdx.x], row, f.out, f.out_stride, f.errword, small_sh);
+                          f.small_ids[blockIdx.x - f.num_large], row, f.out, f.out_stride, f.errword, small_sh);
         return;
     }
     uint32_t *s_key = fin_dyn;
     int32_t *s_idx = reinterpret_cast<int32_t *>(fin_dyn + kFinSmemCap);
-    const int li = (int)blockIdx.x - f.num_small;
+    const int li = f.large_order[blockIdx.x];
     const int64_t slot = (int64_t)row * f.num_large + li;
     const int s = f.large_ids[li];
     const int64_t off = f.seg_off[s];
@@ -364,13 +384,22 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
             for (int i = threadIdx.x; i < len; i += kFinThreads)
                 atomicAdd(&full_hist[mag_key(__ldg(rowp + off + i)) >> 20], 1u);
             __syncthreads();
-            int part = (int)(full_hist[2 * threadIdx.x] + full_hist[2 * threadIdx.x + 1]);
+            constexpr int kPer = kHistBins / kFinThreads;
+            int part = 0;
+#pragma unroll
+            for (int i = 0; i < kPer; ++i) part += (int)full_hist[threadIdx.x * kPer + i];
             const int incl = block_suffix_incl(part, sh.warp_i);
             if (incl >= k && incl - part < k) {
-                const int hi = (int)full_hist[2 * threadIdx.x + 1];
-                const bool upper = incl - part + hi >= k;
-                f.prefix[slot] = (uint32_t)(2 * threadIdx.x + (upper ? 1 : 0));
-                f.k_rem[slot] = k - (incl - part) - (upper ? 0 : hi);
+                int above = incl - part;
+                for (int i = kPer - 1; i >= 0; --i) {
+                    const int h = (int)full_hist[threadIdx.x * kPer + i];
+                    if (above + h >= k) {
+                        f.prefix[slot] = (uint32_t)(threadIdx.x * kPer + i);
+                        f.k_rem[slot] = k - above;
+                        break;
+                    }
+                    above += h;
+                }
             }
             __syncthreads();
         }
@@ -484,6 +513,17 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, float *__restr
     const int in_tile = N - tile_base < kSelChunk ? (int)(N - tile_base) : kSelChunk;    // a multiple of 4
     const int p0 = (int)threadIdx.x * 4;
     const bool live = p0 < in_tile;
+    // a selecting row fetches its tile's description and predicted key before the stream, so that
+    // they are at hand when the stores have been issued
+    const int sel = row - sel_row0;
+    const bool selecting = sel >= 0 && sel < sel_rows;
+    int4 desc = make_int4(0, -2, 0, 0);         // x: first segment, y: the one large segment covering the tile
+                                                // (-1: several segments, -2: no large segment), z: its chunk
+    uint32_t lbkey1 = 0;
+    if (selecting) {
+        desc = __ldg(f.tile_desc + q);
+        if (desc.y >= 0) lbkey1 = f.lbkey[(int64_t)sel * f.num_large + desc.y];
+    }
     float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
     if (live) {
         const int64_t e = ((int64_t)row * N + tile_base + p0) >> 2;
@@ -494,17 +534,12 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, float *__restr
         __stcs(reinterpret_cast<float4 *>(u) + e, uu);
         __stcs(reinterpret_cast<float4 *>(v) + e, vv);
     }
-    const int sel = row - sel_row0;
-    if (sel < 0 || sel >= sel_rows) return;
-    const int4 desc = f.tile_desc[q];           // x: first segment, y: the one large segment covering the tile
-                                                // (-1: several segments, -2: no large segment), z: its chunk
-    if (desc.y == -2) return;
+    if (!selecting || desc.y == -2) return;
     const uint32_t key[4] = {mag_key(vv.x), mag_key(vv.y), mag_key(vv.z), mag_key(vv.w)};
     if (desc.y >= 0) {
-        const int64_t slot = (int64_t)sel * f.num_large + desc.y;
-        const uint32_t lbkey = f.lbkey[slot];
-        if (lbkey == 0) return;                                  // no prediction: the finishing CTA counts itself
-        collect_tile(f, slot, (int64_t)sel * f.num_tchunks + desc.z, key, lbkey, live, p0, 0, in_tile, warp_u);
+        if (lbkey1 == 0) return;                                 // no prediction: the finishing CTA counts itself
+        collect_tile(f, (int64_t)sel * f.num_large + desc.y, (int64_t)sel * f.num_tchunks + desc.z, key, lbkey1, live,
+                     p0, 0, in_tile, warp_u);
         return;
     }
     const int64_t tile_end = tile_base + in_tile;
@@ -528,6 +563,8 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
 {
     f.data = data; f.row_stride = row_stride; f.row0 = row0;
     f.num_large = t.num_large; f.num_small = t.num_small; f.num_tchunks = t.num_tchunks; f.epoch = epoch;
+    f.fin_small = 0;
+    f.large_order = t.large_order; f.zero_ptr = nullptr; f.zero_vecs = 0; f.zero_tail = 0;
     f.seg_off = t.seg_off; f.seg_len = t.seg_len; f.seg_k = t.seg_k; f.seg_out = t.seg_out;
     f.small_ids = t.small_ids; f.large_ids = t.large_ids; f.seg_large = t.seg_large; f.large_q0 = t.large_q0;
     f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_desc = t.tile_desc;
@@ -537,13 +574,21 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
     f.out = out; f.out_stride = out_stride; f.errword = errword;
 }
 
+__global__ void __launch_bounds__(kSelThreads) select_small_only_kernel(FastArgs f)
+{
+    __shared__ SmallShared sh;
+    select_small_body(f.data, f.row_stride, f.row0, f.seg_off, f.seg_len, f.seg_k, f.seg_out, f.small_ids[blockIdx.x],
+                      blockIdx.y, f.out, f.out_stride, f.errword, sh);
+}
+
 }  // namespace
 
 // `served`: the accumulation of this step collected the candidates of exactly these rows (path a);
-// otherwise the two passes of path (b) run first.
+// otherwise the two passes of path (b) run first.  `clear` (may be null): a buffer of `clear_floats`
+// floats that spare CTAs of the finishing launch set to zero; used only when there are large segments.
 cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0, int rows,
-                          int32_t *out, int64_t out_stride, bool served, int32_t epoch, int32_t *errword,
-                          cudaStream_t st)
+                          int32_t *out, int64_t out_stride, bool served, int32_t epoch, float *clear, int64_t clear_floats,
+                          int32_t *errword, cudaStream_t st)
 {
     if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
     FastArgs f;
@@ -562,7 +607,19 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
         hist0_fast_kernel<<<dim3(t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
         collect_kernel<<<dim3(t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
     }
-    finish_kernel<<<dim3(t.num_small + t.num_large, rows), kFinThreads, kFinDyn, st>>>(f), ++g_kernel_launches;
+    // a few small segments ride along in the finishing launch; many get CTAs of their own size
+    f.fin_small = (int64_t)rows * t.num_small <= 512 && t.num_large ? t.num_small : 0;
+    if (t.num_small && !f.fin_small)
+        select_small_only_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
+    unsigned spare = 0;
+    if (clear && clear_floats > 0 && t.num_large) {
+        f.zero_ptr = reinterpret_cast<uint4 *>(clear);
+        f.zero_vecs = (uint64_t)clear_floats >> 2;
+        f.zero_tail = (int)(clear_floats & 3);
+        spare = (unsigned)((f.zero_vecs + 1 + kFinThreads * kZeroPerThread - 1) / (kFinThreads * kZeroPerThread));
+    }
+    if (t.num_large + f.fin_small)
+        finish_kernel<<<dim3(t.num_large + f.fin_small + spare, rows), kFinThreads, kFinDyn, st>>>(f), ++g_kernel_launches;
     return cudaGetLastError();
 }
 

@@ -53,7 +53,7 @@ def lib() -> C.CDLL:
         l.lgc_init.argtypes = [C.POINTER(lgc_config), vp, sz, vp, sz, vp, sz, C.POINTER(vp)]
         l.lgc_destroy.argtypes = [vp]
         l.lgc_accumulate.argtypes = [vp, vp, C.c_int32]
-        l.lgc_topk.argtypes = [vp, C.c_int32]
+        l.lgc_topk.argtypes = [vp, C.c_int32, vp]
         l.lgc_encode.argtypes = [vp]
         l.lgc_combine.argtypes = [vp, C.c_int32]
         l.lgc_decode_scatter.argtypes = [vp, vp]
@@ -185,8 +185,9 @@ class LGC:
         self._ok(self._l.lgc_accumulate(self._ctx, self._dev_f32(grads, self.K * self.N, "grads"), leader_hint),
                  "lgc_accumulate")
 
-    def topk(self, leader: int = 0) -> None:
-        self._ok(self._l.lgc_topk(self._ctx, leader), "lgc_topk")
+    def topk(self, leader: int = 0, update_hint: Optional[torch.Tensor] = None) -> None:
+        ptr = self._dev_f32(update_hint, self.N, "update_hint") if update_hint is not None else None
+        self._ok(self._l.lgc_topk(self._ctx, leader, ptr), "lgc_topk")
 
     def encode(self) -> None:
         self._ok(self._l.lgc_encode(self._ctx), "lgc_encode")
@@ -207,7 +208,7 @@ class LGC:
     def step(self, grads: torch.Tensor, update: torch.Tensor, choice: int = 0) -> None:
         """The five stages of one compression step, in order."""
         self.accumulate(grads, choice)
-        self.topk(choice)
+        self.topk(choice, update)
         self.encode()
         self.combine(choice)
         self.decode_scatter(update)

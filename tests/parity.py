@@ -51,9 +51,10 @@ def make_pair(numel, K, variant="rar", ae_kind="conv2", c1=8, c2=4, density_ppm=
 
 
 def compare_step(ora, gpu, g_cpu: torch.Tensor, g_dev: torch.Tensor, choice: int, update_dev: torch.Tensor,
-                 check_state=True, hint="leader"):
+                 check_state=True, hint="leader", announce_update=True):
     """One full compression step on both sides, compared after every stage.  `hint`: what
-    lgc_accumulate is told about the coming leader ("leader", "none", or "wrong")."""
+    lgc_accumulate is told about the coming leader ("leader", "none", or "wrong");
+    `announce_update`: whether lgc_topk is told the update buffer (and clears it early)."""
     K = ora.K
     ora.accumulate(g_cpu.numpy())
     gpu.accumulate(g_dev, {"leader": choice, "none": -1, "wrong": (choice + 1) % K}[hint])
@@ -61,7 +62,9 @@ def compare_step(ora, gpu, g_cpu: torch.Tensor, g_dev: torch.Tensor, choice: int
         assert_bitwise(gpu.u.cpu().numpy(), ora.u, "u after accumulate")
         assert_bitwise(gpu.v.cpu().numpy(), ora.v, "v after accumulate")
     ora.topk(choice)
-    gpu.topk(choice)
+    if announce_update:
+        update_dev.fill_(float("nan"))           # whatever is there must be overwritten
+    gpu.topk(choice, update_dev if announce_update else None)
     idx_ref = ora.idx if ora.variant == "ps" else ora.idx[:1]
     assert_bitwise(gpu.idx.cpu().numpy(), idx_ref, "selected indices")
     ora.encode()

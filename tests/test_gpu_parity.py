@@ -26,7 +26,8 @@ def run_steps(numel, K, steps, hints=("leader",), **kw):
     upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
     for t in range(steps):
         g = src.step(t)
-        compare_step(ora, gpu, g, g.cuda(), W.choice_for_step(seed, t, K), upd, hint=hints[t % len(hints)])
+        compare_step(ora, gpu, g, g.cuda(), W.choice_for_step(seed, t, K), upd, hint=hints[t % len(hints)],
+                     announce_update=(t % 3 != 1))
     return ora, gpu
 
 

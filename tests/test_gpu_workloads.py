@@ -109,7 +109,7 @@ def test_stress_config_sampled():
             O.accumulate(u_s[k], v_s[k], np.ascontiguousarray(g_s[k]), float(np.float32(w.momentum)))
         assert_bitwise(gpu.u[:, pos_dev].cpu().numpy(), u_s, f"sampled u, step {t}")
         assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_s, f"sampled v, step {t}")
-        gpu.topk(leader)
+        gpu.topk(leader, upd)
         idx = gpu.idx.cpu().numpy()[0]
         if t in (0, w.steps - 1):                          # the selection against the oracle, whole row
             v_leader = gpu.v[leader].cpu().numpy()
