@@ -53,6 +53,7 @@ struct SelectTables {
                                      // covers the whole tile (-1: several segments, -2: no large one); z: its chunk
     int32_t *cand_cnt = nullptr;     // [rows][num_tchunks] candidates found in the chunk
     uint16_t *cand_pos = nullptr;    // [rows][num_tchunks][kSelChunk] their positions inside the tile, ascending
+    uint32_t *cand_key = nullptr;    // [rows][num_tchunks][kSelChunk] their keys, same order
     int32_t *seg_m = nullptr;        // [rows][num_large] candidates of the segment
     int32_t *seg_ticket = nullptr;   // [rows][num_large] chunks that have reported; zero between passes
     int32_t *seg_epoch = nullptr;    // [rows][num_large] step in which the two-pass path settled the segment

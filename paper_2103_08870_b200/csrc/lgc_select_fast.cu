@@ -44,6 +44,7 @@ struct FastArgs {
     uint32_t *hist, *prefix, *lbkey;
     int32_t *k_rem, *cand_cnt, *seg_m, *seg_ticket, *seg_epoch, *seg_path;
     uint16_t *cand_pos;
+    uint32_t *cand_key;
     const int64_t *comp_off;
     int64_t comp_total;
     uint32_t *comp_key;
@@ -55,8 +56,9 @@ struct FastArgs {
 
 constexpr int kFinThreads = 512;      // two finishing CTAs fit on an SM, so every segment of a ResNet starts at once
 constexpr int kFinWarps = kFinThreads / 32;
-constexpr int kFinSmemCap = 8192;     // candidates a finishing CTA keeps in shared memory
-constexpr int kFinPerThread = 4;      // consecutive entries per thread in the ordered passes
+constexpr int kFinSmemCap = 20480;    // candidate keys a finishing CTA keeps in shared memory (80 KB; two CTAs per SM)
+constexpr int kFinGroup = 2048;       // chunks whose candidate counts are scanned together during the compaction
+constexpr int kFinPerThread = 16;     // consecutive entries per thread in the ordered passes
 constexpr int kZeroPerThread = 8;     // 16-byte stores per thread of a CTA that clears a slice of the update
 constexpr int kAccThreads = 1024;     // accumulation: one 128-bit g/u/v triple per thread, 4096 elements per CTA
 
@@ -225,13 +227,17 @@ __global__ void __launch_bounds__(kSelThreads) collect_kernel(FastArgs f)
         f.cand_cnt[c] = (int)((total & 0xffff) + (total >> 16 & 0xffff) + (total >> 32 & 0xffff) + (total >> 48));
     if (flags) {
         uint16_t *dst = f.cand_pos + c * kSelChunk;
+        uint32_t *dkey = f.cand_key + c * kSelChunk;
         unsigned stripe_base = 0;
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
             unsigned at = stripe_base + (unsigned)(before >> (16 * r) & 0xffff);
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                if (flags >> (4 * r + j) & 1u) dst[at++] = (uint16_t)(r * (kSelThreads * 4) + threadIdx.x * 4 + j);
+                if (flags >> (4 * r + j) & 1u) {
+                    dst[at] = (uint16_t)(r * (kSelThreads * 4) + threadIdx.x * 4 + j);
+                    dkey[at++] = key[4 * r + j];
+                }
             stripe_base += (unsigned)(total >> (16 * r) & 0xffff);
         }
     }
@@ -254,7 +260,7 @@ struct DataSource {
 };
 
 struct FinishShared {
-    int hist[256];
+    int hist[1024];
     int warp_i[kFinWarps];
     unsigned warp_u[kFinWarps];
     int found[2];
@@ -267,28 +273,45 @@ template <typename Source>
 __device__ uint32_t finish_from(const Source &src, uint32_t d0, int k_rem, int k, int32_t *__restrict__ out,
                                 FinishShared &sh, int32_t *errword)
 {
+    // the 20 bits below the bucket, ten at a time
     uint32_t prefix = d0 << 20, decided = 0x7ff00000u;
-    const int shifts[3] = {12, 4, 0};
-    const uint32_t masks[3] = {0xffu, 0xffu, 0xfu};
+    constexpr int kBinsPer = 1024 / kFinThreads;
 #pragma unroll 1
-    for (int p = 0; p < 3; ++p) {
-        if (threadIdx.x < 256) sh.hist[threadIdx.x] = 0;
+    for (int shift = 10; shift >= 0; shift -= 10) {
+        for (int b = threadIdx.x; b < 1024; b += kFinThreads) sh.hist[b] = 0;
         __syncthreads();
-        for (int i = threadIdx.x; i < src.n; i += kFinThreads) {
-            const uint32_t x = src.key_at(i);
-            if ((x & decided) == prefix) atomicAdd(&sh.hist[(x >> shifts[p]) & masks[p]], 1);
+        for (int base = 0; base < src.n; base += kFinThreads * 8) {      // eight independent loads per thread
+            uint32_t x[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = base + j * kFinThreads + (int)threadIdx.x;
+                x[j] = i < src.n ? src.key_at(i) : 0xffffffffu;          // never matches the prefix
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if ((x[j] & decided) == prefix) atomicAdd(&sh.hist[(x[j] >> shift) & 1023u], 1);
         }
         __syncthreads();
-        const int mine = threadIdx.x < 256 ? sh.hist[threadIdx.x] : 0;
+        int mine = 0;
+#pragma unroll
+        for (int j = 0; j < kBinsPer; ++j) mine += sh.hist[threadIdx.x * kBinsPer + j];
         const int incl = block_suffix_incl(mine, sh.warp_i);
-        if (threadIdx.x < 256 && incl >= k_rem && incl - mine < k_rem) {
-            sh.found[0] = threadIdx.x;
-            sh.found[1] = k_rem - (incl - mine);
+        if (incl >= k_rem && incl - mine < k_rem) {
+            int above = incl - mine;
+            for (int j = kBinsPer - 1; j >= 0; --j) {
+                const int h = sh.hist[threadIdx.x * kBinsPer + j];
+                if (above + h >= k_rem) {
+                    sh.found[0] = threadIdx.x * kBinsPer + j;
+                    sh.found[1] = k_rem - above;
+                    break;
+                }
+                above += h;
+            }
         }
-        if (threadIdx.x == 0 && incl < k_rem) atomicExch(errword, 0x5E50 + p);
+        if (threadIdx.x == 0 && incl < k_rem) atomicExch(errword, 0x5E50 + shift);
         __syncthreads();
-        prefix |= (uint32_t)sh.found[0] << shifts[p];
-        decided |= masks[p] << shifts[p];
+        prefix |= (uint32_t)sh.found[0] << shift;
+        decided |= 1023u << shift;
         k_rem = sh.found[1];
         __syncthreads();
     }
@@ -342,8 +365,9 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
     __shared__ FinishShared sh;
     __shared__ SmallShared small_sh;
     __shared__ unsigned full_hist[kHistBins];
+    __shared__ int group_off[kFinGroup];
     __shared__ int scan_flag;
-    extern __shared__ __align__(16) uint32_t fin_dyn[];     // kFinSmemCap keys, then kFinSmemCap offsets
+    extern __shared__ __align__(16) uint32_t fin_dyn[];     // kFinSmemCap candidate keys
     const int row = blockIdx.y;
     if ((int)blockIdx.x >= f.num_large + f.fin_small) {      // spare CTAs: clear the dense update meanwhile
         if (row != 0) return;
@@ -363,7 +387,6 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
         return;
     }
     uint32_t *s_key = fin_dyn;
-    int32_t *s_idx = reinterpret_cast<int32_t *>(fin_dyn + kFinSmemCap);
     const int li = f.large_order[blockIdx.x];
     const int64_t slot = (int64_t)row * f.num_large + li;
     const int s = f.large_ids[li];
@@ -413,43 +436,72 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
         DataSource src{rowp + off, off, len};
         T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
     } else {
-        const bool in_smem = m <= kFinSmemCap;
-        uint32_t *ckey = in_smem ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
-        int32_t *cidx = in_smem ? s_idx : f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
+        // keys stay in shared memory when they fit; the offsets are needed only for the k winners
+        uint32_t *ckey = m <= kFinSmemCap ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
+        int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
         const int c0 = f.tchunk0[li], c1 = f.tchunk0[li + 1];
         const int q0 = f.large_q0[li];
         const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
+        constexpr int kPerT = kFinGroup / kFinThreads;
         int done = 0;
-        for (int base = c0; base < c1; base += kFinThreads) {
-            const int c = base + (int)threadIdx.x;
-            const unsigned n = c < c1 ? (unsigned)cnt[c] : 0u;
+        for (int gb = c0; gb < c1; gb += kFinGroup) {
+            // exclusive prefix of the chunk counts of this group, in shared memory
+            const int gn = c1 - gb < kFinGroup ? c1 - gb : kFinGroup;
+            int mine[kPerT];
+            unsigned sum = 0;
+#pragma unroll
+            for (int j = 0; j < kPerT; ++j) {
+                const int e = (int)threadIdx.x * kPerT + j;
+                mine[j] = e < gn ? cnt[gb + e] : 0;
+                sum += (unsigned)mine[j];
+            }
             unsigned total;
-            unsigned at = (unsigned)done + block_prefix_excl<unsigned>(n, sh.warp_u, &total);
-            if (n) {
-                // eight positions per 128-bit load, then eight independent gathers
-                const uint4 *pos8 =
-                    reinterpret_cast<const uint4 *>(f.cand_pos + ((int64_t)row * f.num_tchunks + c) * kSelChunk);
-                const int tile_base = (q0 + (c - c0)) * kSelChunk;          // N < 2^31
-                for (unsigned b0 = 0; b0 < n; b0 += 8) {
-                    const uint4 pv = pos8[b0 >> 3];
-                    const unsigned w[4] = {pv.x, pv.y, pv.z, pv.w};
-                    uint32_t kk[8];
+            unsigned at = block_prefix_excl<unsigned>(sum, sh.warp_u, &total);
 #pragma unroll
-                    for (int b = 0; b < 8; ++b) {
-                        const int j = tile_base + (int)(w[b >> 1] >> (16 * (b & 1)) & 0xffffu);
-                        kk[b] = b0 + b < n ? mag_key(__ldg(rowp + j)) : 0u;
-                    }
+            for (int j = 0; j < kPerT; ++j) {
+                group_off[threadIdx.x * kPerT + j] = (int)at;
+                at += (unsigned)mine[j];
+            }
+            __syncthreads();
+            // one candidate per thread and trip, eight trips in flight: its chunk by binary search in
+            // shared memory, then its key and position from the chunk's lists (neighbouring ranks
+            // read neighbouring entries)
+            for (int base = 0; base < (int)total; base += kFinThreads * 8) {
+                int64_t at_list[8];
+                int tile0[8];
 #pragma unroll
-                    for (int b = 0; b < 8; ++b) {
-                        if (b0 + b < n && at + b < (unsigned)m) {
-                            ckey[at + b] = kk[b];
-                            cidx[at + b] = tile_base + (int)(w[b >> 1] >> (16 * (b & 1)) & 0xffffu);
+                for (int t = 0; t < 8; ++t) {
+                    const int r = base + t * kFinThreads + (int)threadIdx.x;
+                    at_list[t] = -1;
+                    tile0[t] = 0;
+                    if (r < (int)total) {
+                        int lo = 0, hi = gn;                       // last chunk whose offset is <= rank
+                        while (hi - lo > 1) {
+                            const int mid = (lo + hi) >> 1;
+                            if (group_off[mid] <= r) lo = mid; else hi = mid;
                         }
+                        at_list[t] = ((int64_t)row * f.num_tchunks + gb + lo) * kSelChunk + (r - group_off[lo]);
+                        tile0[t] = (q0 + (gb + lo - c0)) * kSelChunk;                 // N < 2^31
                     }
-                    at += 8;
+                }
+                uint32_t kk[8];
+                int pp[8];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    kk[t] = at_list[t] >= 0 ? __ldg(f.cand_key + at_list[t]) : 0u;
+                    pp[t] = at_list[t] >= 0 ? (int)__ldg(f.cand_pos + at_list[t]) : 0;
+                }
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    const int r = base + t * kFinThreads + (int)threadIdx.x;
+                    if (at_list[t] >= 0 && done + r < m) {
+                        ckey[done + r] = kk[t];
+                        cidx[done + r] = tile0[t] + pp[t];
+                    }
                 }
             }
             done += (int)total;
+            __syncthreads();                                       // group_off is rewritten by the next group
         }
         if (threadIdx.x == 0 && done != m) atomicExch(f.errword, 0x5E70);
         __syncthreads();
@@ -489,9 +541,13 @@ __device__ __forceinline__ void collect_tile(const FastArgs &f, int64_t slot, in
     if (threadIdx.x == 0) f.cand_cnt[chunk] = (int)total;
     if (flags) {
         uint16_t *dst = f.cand_pos + chunk * kSelChunk;
+        uint32_t *dkey = f.cand_key + chunk * kSelChunk;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            if (flags >> i & 1u) dst[at++] = (uint16_t)(p0 + i);
+            if (flags >> i & 1u) {
+                dst[at] = (uint16_t)(p0 + i);
+                dkey[at++] = key[i];
+            }
     }
 }
 
@@ -569,7 +625,7 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
     f.small_ids = t.small_ids; f.large_ids = t.large_ids; f.seg_large = t.seg_large; f.large_q0 = t.large_q0;
     f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_desc = t.tile_desc;
     f.hist = t.hist; f.prefix = t.prefix; f.k_rem = t.k_rem; f.cand_cnt = t.cand_cnt; f.seg_m = t.seg_m;
-    f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.seg_path = t.seg_path; f.lbkey = t.lbkey; f.cand_pos = t.cand_pos;
+    f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.seg_path = t.seg_path; f.lbkey = t.lbkey; f.cand_pos = t.cand_pos; f.cand_key = t.cand_key;
     f.comp_off = t.comp_off; f.comp_total = t.comp_total; f.comp_key = t.comp_key; f.comp_idx = t.comp_idx;
     f.out = out; f.out_stride = out_stride; f.errword = errword;
 }
@@ -593,7 +649,7 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
     if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
     FastArgs f;
     fill_args(f, t, data, row_stride, row0, out, out_stride, epoch, errword);
-    constexpr int kFinDyn = 2 * kFinSmemCap * (int)sizeof(uint32_t);
+    constexpr int kFinDyn = kFinSmemCap * (int)sizeof(uint32_t);
     static bool configured = false;
     if (!configured) {
         const cudaError_t e = cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinDyn);
