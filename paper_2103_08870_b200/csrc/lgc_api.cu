@@ -197,8 +197,7 @@ void carve_select(Carver &cv, SelectTables &t, const SelectPlan &sp, int rows)
     t.lbkey = cv.take<uint32_t>((size_t)rows * nl);
     t.seg_path = cv.take<int32_t>((size_t)rows * nl);
     t.cand_cnt = cv.take<int32_t>((size_t)rows * nc);
-    t.cand_pos = cv.take<uint16_t>((size_t)rows * nc * kSelChunk);
-    t.cand_key = cv.take<uint32_t>((size_t)rows * nc * kSelChunk);
+    t.cand = cv.take<uint2>((size_t)rows * nc * kSelCandCap);
     t.comp_off = cv.take<int64_t>((size_t)nl + 1);
     t.comp_total = sp.comp_total;
     t.comp_key = cv.take<uint32_t>((size_t)rows * sp.comp_total);

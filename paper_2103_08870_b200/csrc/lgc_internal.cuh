@@ -15,6 +15,7 @@ namespace lgc {
 constexpr int kSelChunk = 4096;    // elements per selection chunk: 256 threads x 16
 constexpr int kSelThreads = 256;
 constexpr int kSelPerThread = 16;
+constexpr int kSelCandCap = 1024;  // candidates a chunk's list holds; more than that and the segment is finished from the data
 constexpr int kHistBins = 2048;    // first radix digit: 11 bits; the next two: 10 bits each
 
 // One selection problem family: R rows of `data` (row stride in elements), each cut into the same
@@ -52,8 +53,7 @@ struct SelectTables {
     int4 *tile_desc = nullptr;       // [tiles_per_row] x: first segment the tile overlaps; y: the large segment that
                                      // covers the whole tile (-1: several segments, -2: no large one); z: its chunk
     int32_t *cand_cnt = nullptr;     // [rows][num_tchunks] candidates found in the chunk
-    uint16_t *cand_pos = nullptr;    // [rows][num_tchunks][kSelChunk] their positions inside the tile, ascending
-    uint32_t *cand_key = nullptr;    // [rows][num_tchunks][kSelChunk] their keys, same order
+    uint2 *cand = nullptr;           // [rows][num_tchunks][kSelCandCap] (key, position inside the tile), ascending position
     int32_t *seg_m = nullptr;        // [rows][num_large] candidates of the segment
     int32_t *seg_ticket = nullptr;   // [rows][num_large] chunks that have reported; zero between passes
     int32_t *seg_epoch = nullptr;    // [rows][num_large] step in which the two-pass path settled the segment

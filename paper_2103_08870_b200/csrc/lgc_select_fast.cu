@@ -43,8 +43,7 @@ struct FastArgs {
     const int4 *tile_desc;
     uint32_t *hist, *prefix, *lbkey;
     int32_t *k_rem, *cand_cnt, *seg_m, *seg_ticket, *seg_epoch, *seg_path;
-    uint16_t *cand_pos;
-    uint32_t *cand_key;
+    uint2 *cand;                   // [rows][num_tchunks][kCandCap] candidates of a chunk: (key, position in tile), ascending position
     const int64_t *comp_off;
     int64_t comp_total;
     uint32_t *comp_key;
@@ -59,6 +58,7 @@ constexpr int kFinWarps = kFinThreads / 32;
 constexpr int kFinSmemCap = 20480;    // candidate keys a finishing CTA keeps in shared memory (80 KB; two CTAs per SM)
 constexpr int kFinGroup = 2048;       // chunks whose candidate counts are scanned together during the compaction
 constexpr int kFinPerThread = 16;     // consecutive entries per thread in the ordered passes
+constexpr int kCandCap = kSelCandCap;  // entries a chunk's list can hold; a chunk with more sends its segment to the data
 constexpr int kZeroPerThread = 8;     // 16-byte stores per thread of a CTA that clears a slice of the update
 constexpr int kAccThreads = 1024;     // accumulation: one 128-bit g/u/v triple per thread, 4096 elements per CTA
 
@@ -119,13 +119,11 @@ __device__ __forceinline__ unsigned load_keys_tile(const float *__restrict__ til
     return valid;
 }
 
-// Run by every thread of a CTA on a segment's finished histogram: finds the bucket d0 of the
-// k-th largest key.  FUSED: the histogram holds only the entries at or above the predicted key,
-// all of them are the candidates, and the result stands only if there are at least k.
-// Otherwise the histogram is complete and the candidates are the entries from bucket d0 upwards.
-// On success stores d0, the rank still to find inside d0 and the candidate count, and returns
-// true.  The global histogram and the ticket are left zeroed either way.
-template <int THREADS, bool FUSED>
+// Run by every thread of the CTA that completed a segment's leading-digit histogram: finds the
+// bucket d0 of the k-th largest key, stores d0, the rank still to find inside d0 and the number
+// of entries from d0 upwards (the candidates), and leaves histogram and ticket zeroed.  Returns
+// false if the histogram holds fewer than k entries.
+template <int THREADS>
 __device__ __forceinline__ bool bucket_scan(const FastArgs &f, int64_t slot, int k, int *warp_tot, int *flag)
 {
     constexpr int kPer = kHistBins / THREADS;
@@ -150,14 +148,13 @@ __device__ __forceinline__ bool bucket_scan(const FastArgs &f, int64_t slot, int
             if (above + hh[i] >= k) {
                 f.prefix[slot] = (uint32_t)(threadIdx.x * kPer + i);
                 f.k_rem[slot] = k - above;
-                if (!FUSED) f.seg_m[slot] = above + hh[i];
+                f.seg_m[slot] = above + hh[i];
                 *flag = 1;
                 break;
             }
             above += hh[i];
         }
     }
-    if (FUSED && threadIdx.x == 0) f.seg_m[slot] = incl;      // thread 0's suffix sum is the total
     __syncthreads();
     return *flag != 0;
 }
@@ -192,7 +189,7 @@ __global__ void __launch_bounds__(kSelThreads) hist0_fast_kernel(FastArgs f)
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    const bool ok = bucket_scan<kSelThreads, false>(f, slot, f.seg_k[g.s], warp_tot, &scan_flag);
+    const bool ok = bucket_scan<kSelThreads>(f, slot, f.seg_k[g.s], warp_tot, &scan_flag);
     if (threadIdx.x == 0) {
         if (ok) f.seg_epoch[slot] = f.epoch;                   // settled for this step
         else atomicExch(f.errword, 0x5E40);                    // a complete histogram always holds k entries
@@ -226,8 +223,7 @@ __global__ void __launch_bounds__(kSelThreads) collect_kernel(FastArgs f)
     if (threadIdx.x == 0)
         f.cand_cnt[c] = (int)((total & 0xffff) + (total >> 16 & 0xffff) + (total >> 32 & 0xffff) + (total >> 48));
     if (flags) {
-        uint16_t *dst = f.cand_pos + c * kSelChunk;
-        uint32_t *dkey = f.cand_key + c * kSelChunk;
+        uint2 *dst = f.cand + c * kCandCap;
         unsigned stripe_base = 0;
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
@@ -235,8 +231,9 @@ __global__ void __launch_bounds__(kSelThreads) collect_kernel(FastArgs f)
 #pragma unroll
             for (int j = 0; j < 4; ++j)
                 if (flags >> (4 * r + j) & 1u) {
-                    dst[at] = (uint16_t)(r * (kSelThreads * 4) + threadIdx.x * 4 + j);
-                    dkey[at++] = key[4 * r + j];
+                    if (at < (unsigned)kCandCap)
+                        dst[at] = make_uint2(key[4 * r + j], (unsigned)(r * (kSelThreads * 4) + threadIdx.x * 4 + j));
+                    ++at;
                 }
             stripe_base += (unsigned)(total >> (16 * r) & 0xffff);
         }
@@ -350,6 +347,31 @@ __device__ uint32_t finish_from(const Source &src, uint32_t d0, int k_rem, int k
     return T;
 }
 
+// Bucket of the k-th largest key from a complete leading-digit histogram in shared memory (which
+// holds at least k entries): leaves the bucket in sh.found[0] and the rank still to find inside
+// it in sh.found[1].  Run by every thread of the CTA; ends with a barrier.
+__device__ __forceinline__ void digit_scan(const unsigned *hist, int k, FinishShared &sh)
+{
+    constexpr int kPer = kHistBins / kFinThreads;
+    int part = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) part += (int)hist[threadIdx.x * kPer + i];
+    const int incl = block_suffix_incl(part, sh.warp_i);
+    if (incl >= k && incl - part < k) {
+        int above = incl - part;
+        for (int i = kPer - 1; i >= 0; --i) {
+            const int h = (int)hist[threadIdx.x * kPer + i];
+            if (above + h >= k) {
+                sh.found[0] = threadIdx.x * kPer + i;
+                sh.found[1] = k - above;
+                break;
+            }
+            above += h;
+        }
+    }
+    __syncthreads();
+}
+
 // The selection of one (segment, row) is completed by one CTA.  The first num_small CTAs of a
 // row each do one small segment outright.  For a large segment the CTA
 //  1. settles the bucket of the k-th key from the histogram the accumulation left, unless path
@@ -366,7 +388,6 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
     __shared__ SmallShared small_sh;
     __shared__ unsigned full_hist[kHistBins];
     __shared__ int group_off[kFinGroup];
-    __shared__ int scan_flag;
     extern __shared__ __align__(16) uint32_t fin_dyn[];     // kFinSmemCap candidate keys
     const int row = blockIdx.y;
     if ((int)blockIdx.x >= f.num_large + f.fin_small) {      // spare CTAs: clear the dense update meanwhile
@@ -395,54 +416,35 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
     const float *rowp = f.data + (int64_t)(f.row0 + row) * f.row_stride;
     int32_t *out = f.out + (int64_t)row * f.out_stride + f.seg_out[s];
     const int64_t cap = f.comp_off[li + 1] - f.comp_off[li];
-    bool lists = true;                        // the chunk lists hold this step's candidates
-    int path = 1;                             // 0: lists from the accumulation, 1: from the two passes, 2/3: data
-    if (f.seg_epoch[slot] != f.epoch) {
-        path = 0;       // not settled by path (b): use what the accumulation counted
-        lists = bucket_scan<kFinThreads, true>(f, slot, k, sh.warp_i, &scan_flag);
-        if (!lists) {
-            // no prediction, or too high: leading-digit histogram of the whole segment, in this CTA
-            for (int b = threadIdx.x; b < kHistBins; b += kFinThreads) full_hist[b] = 0;
-            __syncthreads();
-            for (int i = threadIdx.x; i < len; i += kFinThreads)
-                atomicAdd(&full_hist[mag_key(__ldg(rowp + off + i)) >> 20], 1u);
-            __syncthreads();
-            constexpr int kPer = kHistBins / kFinThreads;
-            int part = 0;
-#pragma unroll
-            for (int i = 0; i < kPer; ++i) part += (int)full_hist[threadIdx.x * kPer + i];
-            const int incl = block_suffix_incl(part, sh.warp_i);
-            if (incl >= k && incl - part < k) {
-                int above = incl - part;
-                for (int i = kPer - 1; i >= 0; --i) {
-                    const int h = (int)full_hist[threadIdx.x * kPer + i];
-                    if (above + h >= k) {
-                        f.prefix[slot] = (uint32_t)(threadIdx.x * kPer + i);
-                        f.k_rem[slot] = k - above;
-                        break;
-                    }
-                    above += h;
-                }
-            }
-            __syncthreads();
+    const int c0 = f.tchunk0[li], c1 = f.tchunk0[li + 1];
+    const int q0 = f.large_q0[li];
+    const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
+    constexpr int kPerT = kFinGroup / kFinThreads;
+    // 1. are there lists for this step, and how many candidates do they hold?
+    const bool settled = f.seg_epoch[slot] == f.epoch;        // path (b) ran and found the bucket
+    bool lists = settled ? (int64_t)f.seg_m[slot] <= cap : f.lbkey[slot] != 0;
+    int64_t m64 = 0;
+    if (lists) {
+        unsigned sum = 0, over = 0;
+        for (int c = c0 + (int)threadIdx.x; c < c1; c += kFinThreads) {
+            const unsigned n = (unsigned)cnt[c];
+            sum += n;
+            over |= n > (unsigned)kCandCap;
         }
+        unsigned total;
+        block_prefix_excl<unsigned>(sum, sh.warp_u, &total);   // per-segment totals stay below 2^31
+        m64 = total;
+        if (__syncthreads_or((int)over) || m64 > cap || (!settled && m64 < k)) lists = false;
     }
-    const uint32_t d0 = f.prefix[slot];
-    const int k_rem = f.k_rem[slot];
-    const int m = f.seg_m[slot];
-    uint32_t T;
-    if (!lists || (int64_t)m > cap) {
-        path = lists ? 3 : 2;
-        DataSource src{rowp + off, off, len};
-        T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
-    } else {
-        // keys stay in shared memory when they fit; the offsets are needed only for the k winners
+    const int m = (int)m64;
+    int path;
+    uint32_t d0 = 0, T;
+    int k_rem = 0;
+    if (lists) {
+        path = settled ? 1 : 0;
+        // 2. compaction.  Keys stay in shared memory when they fit; offsets are needed only for the winners.
         uint32_t *ckey = m <= kFinSmemCap ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
         int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
-        const int c0 = f.tchunk0[li], c1 = f.tchunk0[li + 1];
-        const int q0 = f.large_q0[li];
-        const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
-        constexpr int kPerT = kFinGroup / kFinThreads;
         int done = 0;
         for (int gb = c0; gb < c1; gb += kFinGroup) {
             // exclusive prefix of the chunk counts of this group, in shared memory
@@ -464,15 +466,15 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
             }
             __syncthreads();
             // one candidate per thread and trip, eight trips in flight: its chunk by binary search in
-            // shared memory, then its key and position from the chunk's lists (neighbouring ranks
-            // read neighbouring entries)
+            // shared memory, then its record from the chunk's list (neighbouring ranks read
+            // neighbouring records)
             for (int base = 0; base < (int)total; base += kFinThreads * 8) {
-                int64_t at_list[8];
+                const uint2 *rec[8];
                 int tile0[8];
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     const int r = base + t * kFinThreads + (int)threadIdx.x;
-                    at_list[t] = -1;
+                    rec[t] = nullptr;
                     tile0[t] = 0;
                     if (r < (int)total) {
                         int lo = 0, hi = gn;                       // last chunk whose offset is <= rank
@@ -480,23 +482,19 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
                             const int mid = (lo + hi) >> 1;
                             if (group_off[mid] <= r) lo = mid; else hi = mid;
                         }
-                        at_list[t] = ((int64_t)row * f.num_tchunks + gb + lo) * kSelChunk + (r - group_off[lo]);
+                        rec[t] = f.cand + ((int64_t)row * f.num_tchunks + gb + lo) * kCandCap + (r - group_off[lo]);
                         tile0[t] = (q0 + (gb + lo - c0)) * kSelChunk;                 // N < 2^31
                     }
                 }
-                uint32_t kk[8];
-                int pp[8];
+                uint2 kp[8];
 #pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    kk[t] = at_list[t] >= 0 ? __ldg(f.cand_key + at_list[t]) : 0u;
-                    pp[t] = at_list[t] >= 0 ? (int)__ldg(f.cand_pos + at_list[t]) : 0;
-                }
+                for (int t = 0; t < 8; ++t) kp[t] = rec[t] ? __ldg(rec[t]) : make_uint2(0u, 0u);
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     const int r = base + t * kFinThreads + (int)threadIdx.x;
-                    if (at_list[t] >= 0 && done + r < m) {
-                        ckey[done + r] = kk[t];
-                        cidx[done + r] = tile0[t] + pp[t];
+                    if (rec[t]) {
+                        ckey[done + r] = kp[t].x;
+                        cidx[done + r] = tile0[t] + (int)kp[t].y;
                     }
                 }
             }
@@ -504,10 +502,46 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
             __syncthreads();                                       // group_off is rewritten by the next group
         }
         if (threadIdx.x == 0 && done != m) atomicExch(f.errword, 0x5E70);
+        // 3. the bucket of the k-th key: from path (b), or from the candidates' own leading digits
+        // (every entry at or above the predicted key is a candidate, and there are at least k)
+        if (settled) {
+            d0 = f.prefix[slot];
+            k_rem = f.k_rem[slot];
+        } else {
+            for (int b = threadIdx.x; b < kHistBins; b += kFinThreads) full_hist[b] = 0;
+            __syncthreads();
+            for (int i = threadIdx.x; i < m; i += kFinThreads) atomicAdd(&full_hist[ckey[i] >> 20], 1u);
+            __syncthreads();
+            digit_scan(full_hist, k, sh);
+            d0 = (uint32_t)sh.found[0];
+            k_rem = sh.found[1];
+        }
         __syncthreads();
         CompactSource src{ckey, cidx, m};
         T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
+    } else {
+        // no lists for this step, a chunk list overflowed, too many candidates, or a prediction
+        // that turned out too high: work on the data
+        if (settled) {
+            path = 3;
+            d0 = f.prefix[slot];
+            k_rem = f.k_rem[slot];
+        } else {
+            path = 2;
+            for (int b = threadIdx.x; b < kHistBins; b += kFinThreads) full_hist[b] = 0;
+            __syncthreads();
+            for (int i = threadIdx.x; i < len; i += kFinThreads)
+                atomicAdd(&full_hist[mag_key(__ldg(rowp + off + i)) >> 20], 1u);
+            __syncthreads();
+            digit_scan(full_hist, k, sh);
+            d0 = (uint32_t)sh.found[0];
+            k_rem = sh.found[1];
+            __syncthreads();
+        }
+        DataSource src{rowp + off, off, len};
+        T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
     }
+    if (threadIdx.x == 0) f.seg_m[slot] = lists ? m : len;
     if (threadIdx.x == 0) {
         f.lbkey[slot] = predict_lbkey(T, k);
         f.seg_path[slot] = path;
@@ -523,30 +557,24 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
 // key.
 // ------------------------------------------------------------------------------------------
 // The part [lo, hi) of a tile, held four consecutive entries per thread (positions p0 .. p0+3):
-// entries whose key reaches lbkey are added to the segment's leading-digit histogram and their
-// positions written, ascending, to the chunk's list.
-__device__ __forceinline__ void collect_tile(const FastArgs &f, int64_t slot, int64_t chunk, const uint32_t (&key)[4],
-                                             uint32_t lbkey, bool live, int p0, int lo, int hi, unsigned *warp_u)
+// the entries whose key reaches lbkey are written, ascending, to the chunk's candidate list.
+__device__ __forceinline__ void collect_tile(const FastArgs &f, int64_t chunk, const uint32_t (&key)[4], uint32_t lbkey,
+                                             bool live, int p0, int lo, int hi, unsigned *warp_u)
 {
     unsigned flags = 0;
 #pragma unroll
     for (int i = 0; i < 4; ++i)
         if (live && p0 + i >= lo && p0 + i < hi && key[i] >= lbkey) flags |= 1u << i;
-    uint32_t *gh = f.hist + slot * kHistBins;
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-        if (flags >> i & 1u) atomicAdd(gh + (key[i] >> 20), 1u);
     unsigned total;
     unsigned at = block_prefix_excl<unsigned>((unsigned)__popc(flags), warp_u, &total);
     if (threadIdx.x == 0) f.cand_cnt[chunk] = (int)total;
     if (flags) {
-        uint16_t *dst = f.cand_pos + chunk * kSelChunk;
-        uint32_t *dkey = f.cand_key + chunk * kSelChunk;
+        uint2 *dst = f.cand + chunk * kCandCap;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
             if (flags >> i & 1u) {
-                dst[at] = (uint16_t)(p0 + i);
-                dkey[at++] = key[i];
+                if (at < (unsigned)kCandCap) dst[at] = make_uint2(key[i], (unsigned)(p0 + i));
+                ++at;
             }
     }
 }
@@ -594,8 +622,7 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, float *__restr
     const uint32_t key[4] = {mag_key(vv.x), mag_key(vv.y), mag_key(vv.z), mag_key(vv.w)};
     if (desc.y >= 0) {
         if (lbkey1 == 0) return;                                 // no prediction: the finishing CTA counts itself
-        collect_tile(f, (int64_t)sel * f.num_large + desc.y, (int64_t)sel * f.num_tchunks + desc.z, key, lbkey1, live,
-                     p0, 0, in_tile, warp_u);
+        collect_tile(f, (int64_t)sel * f.num_tchunks + desc.z, key, lbkey1, live, p0, 0, in_tile, warp_u);
         return;
     }
     const int64_t tile_end = tile_base + in_tile;
@@ -608,8 +635,8 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, float *__restr
         const int64_t off = f.seg_off[s], end = off + f.seg_len[s];
         const int lo = off > tile_base ? (int)(off - tile_base) : 0;
         const int hi = end < tile_end ? (int)(end - tile_base) : in_tile;
-        collect_tile(f, slot, (int64_t)sel * f.num_tchunks + f.tchunk0[li] + (q - f.large_q0[li]), key, lbkey, live,
-                     p0, lo, hi, warp_u);
+        collect_tile(f, (int64_t)sel * f.num_tchunks + f.tchunk0[li] + (q - f.large_q0[li]), key, lbkey, live, p0, lo,
+                     hi, warp_u);
         __syncthreads();                                         // warp_u is reused by the next segment
     }
 }
@@ -625,7 +652,7 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
     f.small_ids = t.small_ids; f.large_ids = t.large_ids; f.seg_large = t.seg_large; f.large_q0 = t.large_q0;
     f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_desc = t.tile_desc;
     f.hist = t.hist; f.prefix = t.prefix; f.k_rem = t.k_rem; f.cand_cnt = t.cand_cnt; f.seg_m = t.seg_m;
-    f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.seg_path = t.seg_path; f.lbkey = t.lbkey; f.cand_pos = t.cand_pos; f.cand_key = t.cand_key;
+    f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.seg_path = t.seg_path; f.lbkey = t.lbkey; f.cand = t.cand;
     f.comp_off = t.comp_off; f.comp_total = t.comp_total; f.comp_key = t.comp_key; f.comp_idx = t.comp_idx;
     f.out = out; f.out_stride = out_stride; f.errword = errword;
 }
@@ -657,9 +684,6 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
         configured = true;
     }
     if (t.num_large && !served) {
-        // whatever an accumulation may have counted for other rows must not mix in
-        const cudaError_t e = launch_zero(t.hist, (size_t)rows * t.num_large * kHistBins * sizeof(uint32_t), st);
-        if (e != cudaSuccess) return e;
         hist0_fast_kernel<<<dim3(t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
         collect_kernel<<<dim3(t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
     }
