@@ -254,7 +254,7 @@ def run_ours(args, w: W.Workload):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic", "config": workload_config(w),
-            "roofline": {"bound": "hbm", "kernel": "accumulate_kernel", "achieved": achieved, "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": "accumulate_select_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                          "traffic": None, "algorithmic_bytes_per_launch": acc_bytes,
                          "kernel_ms": acc_mean_ms},

@@ -63,12 +63,14 @@ constexpr int kZeroPerThread = 8;     // 16-byte stores per thread of a CTA that
 constexpr int kAccThreads = 1024;     // accumulation: one 128-bit g/u/v triple per thread, 4096 elements per CTA
 
 // The key from which the next step collects candidates, given this step's k-th key T.  Error
-// feedback piles entries up just below the threshold (each 3 % below T holds about k more), and
-// from step to step T moves by a per cent or two, more for small k: 3 % (6 % for k < 64) below T
-// keeps the candidates at 2-4 k.  A prediction that turns out too high only costs the fallback.
+// feedback piles entries up just below the threshold (each 3 % below T holds about k more).  In
+// steady state T itself moves by a per cent or two per step, but the rows differ: a row that led
+// recently has had its own largest entries removed and sits a few per cent lower than one that
+// has not.  6 % (10 % for k < 64, whose k-th key is noisier) below T keeps the candidates at
+// 4-6 k and makes a prediction that is too high rare; when it happens only the fallback is paid.
 __device__ __forceinline__ uint32_t predict_lbkey(uint32_t T, int k)
 {
-    const float t = __uint_as_float(T) * (k >= 64 ? 0.97f : 0.94f);
+    const float t = __uint_as_float(T) * (k >= 64 ? 0.94f : 0.90f);
     return __float_as_uint(t) & 0x7fffffffu;     // 0 (no prediction) when T is 0 or the product underflows
 }
 
@@ -528,19 +530,62 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
             k_rem = f.k_rem[slot];
         } else {
             path = 2;
+            // first read of the segment: its complete leading-digit histogram
             for (int b = threadIdx.x; b < kHistBins; b += kFinThreads) full_hist[b] = 0;
             __syncthreads();
-            for (int i = threadIdx.x; i < len; i += kFinThreads)
-                atomicAdd(&full_hist[mag_key(__ldg(rowp + off + i)) >> 20], 1u);
+            constexpr int kTile = kFinThreads * kSelPerThread;
+            for (int base = 0; base < len; base += kTile) {
+                uint32_t key[kSelPerThread];
+                const int valid = load_keys16(rowp + off, base, len, key);
+#pragma unroll
+                for (int i = 0; i < kSelPerThread; ++i)
+                    if (i < valid) atomicAdd(&full_hist[key[i] >> 20], 1u);
+            }
             __syncthreads();
             digit_scan(full_hist, k, sh);
             d0 = (uint32_t)sh.found[0];
             k_rem = sh.found[1];
+            const int64_t at_or_above = (int64_t)(k - k_rem) + (int64_t)full_hist[d0];
             __syncthreads();
+            if (at_or_above <= cap) {
+                // second read: the entries from the bucket upwards, compacted in index order
+                const int mm = (int)at_or_above;
+                uint32_t *ckey = mm <= kFinSmemCap ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
+                int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
+                int done = 0;
+                for (int base = 0; base < len; base += kTile) {
+                    uint32_t key[kSelPerThread];
+                    const int valid = load_keys16(rowp + off, base, len, key);
+                    unsigned flags = 0;
+#pragma unroll
+                    for (int i = 0; i < kSelPerThread; ++i)
+                        if (i < valid && (key[i] >> 20) >= d0) flags |= 1u << i;
+                    unsigned total;
+                    unsigned at = (unsigned)done + block_prefix_excl<unsigned>((unsigned)__popc(flags), sh.warp_u, &total);
+                    if (flags) {
+                        const int first = base + (int)threadIdx.x * kSelPerThread;
+#pragma unroll
+                        for (int i = 0; i < kSelPerThread; ++i)
+                            if (flags >> i & 1u) {
+                                ckey[at] = key[i];
+                                cidx[at++] = (int32_t)(off + first + i);
+                            }
+                    }
+                    done += (int)total;
+                }
+                if (threadIdx.x == 0 && done != mm) atomicExch(f.errword, 0x5E80);
+                __syncthreads();
+                CompactSource src{ckey, cidx, mm};
+                T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
+                goto finished;
+            }
         }
-        DataSource src{rowp + off, off, len};
-        T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
+        {
+            DataSource src{rowp + off, off, len};
+            T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
+        }
     }
+finished:
     if (threadIdx.x == 0) f.seg_m[slot] = lists ? m : len;
     if (threadIdx.x == 0) {
         f.lbkey[slot] = predict_lbkey(T, k);
