@@ -33,6 +33,10 @@ UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 GRAD_SETS = 3            # distinct gradient batches cycled through (each far larger than L2)
+# DRAM bytes (read + write) per element that ncu measured for accumulate_select_kernel on the small
+# capture case (profiles/accumulate_select_kernel_resnet50_k2.md); traffic grows in proportion to K * N.
+# Set to None whenever that kernel changes until the counters are taken again.
+NCU_DRAM_BYTES_PER_ELEMENT = 18.99
 
 
 def measured_peak():
@@ -256,7 +260,8 @@ def run_ours(args, w: W.Workload):
             "dtype": "f32", "data": "synthetic", "config": workload_config(w),
             "roofline": {"bound": "hbm", "kernel": "accumulate_select_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                         "traffic": None, "algorithmic_bytes_per_launch": acc_bytes,
+                         "traffic": None if NCU_DRAM_BYTES_PER_ELEMENT is None else NCU_DRAM_BYTES_PER_ELEMENT * K * N,
+                         "algorithmic_bytes_per_launch": acc_bytes,
                          "kernel_ms": acc_mean_ms},
             "step_hbm": {"algorithmic_bytes": step_bytes, "achieved_GBps": step_gbs,
                          "frac_of_measured_peak": step_gbs / peak, "frac_of_nominal_8TBps": step_gbs / NOMINAL_HBM_GBS},
