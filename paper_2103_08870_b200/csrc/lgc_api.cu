@@ -195,6 +195,7 @@ void carve_select(Carver &cv, SelectTables &t, const SelectPlan &sp, int rows)
     t.seg_ticket = cv.take<int32_t>((size_t)rows * nl);
     t.seg_epoch = cv.take<int32_t>((size_t)rows * nl);
     t.lbkey = cv.take<uint32_t>((size_t)rows * nl);
+    t.last_key = cv.take<uint32_t>((size_t)rows * nl);
     t.seg_path = cv.take<int32_t>((size_t)rows * nl);
     t.cand_cnt = cv.take<int32_t>((size_t)rows * nc);
     t.cand = cv.take<uint2>((size_t)rows * nc * kSelCandCap);
@@ -375,9 +376,10 @@ lgc_status lgc_accumulate(lgc_ctx *c, const float *grads, int32_t leader_hint)
     c->epoch = c->epoch == 0x7fffffff ? 1 : c->epoch + 1;
     c->cleared_update = nullptr;
     cudaError_t e;
-    // the fused form needs rows that start 16-byte aligned, someone to select for, and the keys a
-    // previous selection left to collect against
-    if (c->N % 4 == 0 && c->sel_v.num_large > 0 && c->have_prediction && (ps || leader_hint >= 0)) {
+    // the fused form needs rows that start 16-byte aligned, someone to select for, and the keys two
+    // previous selections left to collect against (one key says where the threshold was, two how
+    // fast it moves)
+    if (c->N % 4 == 0 && c->sel_v.num_large > 0 && c->selections >= 2 && (ps || leader_hint >= 0)) {
         e = launch_accumulate_select(c->sel_v, grads, c->u, c->v, c->K, c->N, c->cfg.momentum, ps ? 0 : leader_hint,
                                      ps ? c->K : 1, c->epoch, c->errword, c->stream);
         c->fused_leader = ps ? -1 : leader_hint;
@@ -402,7 +404,7 @@ lgc_status lgc_topk(lgc_ctx *c, int32_t leader, float *update_hint)
     cudaError_t e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, served, c->epoch,
                                   update_hint, c->N, c->errword, c->stream);
     c->cleared_update = c->sel_v.num_large ? update_hint : nullptr;
-    c->have_prediction = true;
+    if (c->selections < 2) ++c->selections;
     c->val_valid = false;
     c->mean_valid = false;
     c->tile_lo_valid = false;

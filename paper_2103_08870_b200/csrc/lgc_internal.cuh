@@ -58,6 +58,7 @@ struct SelectTables {
     int32_t *seg_ticket = nullptr;   // [rows][num_large] chunks that have reported; zero between passes
     int32_t *seg_epoch = nullptr;    // [rows][num_large] step in which the two-pass path settled the segment
     int32_t *seg_path = nullptr;     // [rows][num_large] how the last selection got its entries (see lgc_selection_stats)
+    uint32_t *last_key = nullptr;    // [rows][num_large] k-th key of the previous selection (0: none)
     uint32_t *lbkey = nullptr;       // [rows][num_large] key from which the next accumulation collects candidates (0: none)
     int64_t *comp_off = nullptr;     // [num_large + 1] first compact slot of each large segment
     int64_t comp_total = 0;          // compact slots per row
@@ -114,7 +115,8 @@ struct Ctx {
     int32_t epoch = 0;             // step counter (accumulations so far)
     int32_t inn_epoch = 0;         // the same counter for the innovation selection's tables
     float *cleared_update = nullptr; // buffer the last lgc_topk already cleared (its first N & ~3 floats)
-    bool have_prediction = false;  // a selection has run, so the next accumulation has keys to collect against
+    int selections = 0;            // selections run so far (saturating); the accumulation collects candidates from the
+                                   // third step on, when the prediction knows how fast the threshold is growing
     int32_t fused_leader = -2;     // row whose candidates the last accumulation collected (-1: all rows, -2: none)
     bool val_valid = false;        // val holds the kept values of the current selection
     bool tile_lo_valid = false;    // tile_lo matches the current selection

@@ -41,7 +41,7 @@ struct FastArgs {
     const int64_t *seg_off;
     const int32_t *seg_len, *seg_k, *seg_out, *small_ids, *large_ids, *seg_large, *large_q0, *tchunk0, *tchunk_large;
     const int4 *tile_desc;
-    uint32_t *hist, *prefix, *lbkey;
+    uint32_t *hist, *prefix, *lbkey, *last_key;
     int32_t *k_rem, *cand_cnt, *seg_m, *seg_ticket, *seg_epoch, *seg_path;
     uint2 *cand;                   // [rows][num_tchunks][kCandCap] candidates of a chunk: (key, position in tile), ascending position
     const int64_t *comp_off;
@@ -68,9 +68,19 @@ constexpr int kAccThreads = 1024;     // accumulation: one 128-bit g/u/v triple 
 // recently has had its own largest entries removed and sits a few per cent lower than one that
 // has not.  6 % (10 % for k < 64, whose k-th key is noisier) below T keeps the candidates at
 // 4-6 k and makes a prediction that is too high rare; when it happens only the fallback is paid.
-__device__ __forceinline__ uint32_t predict_lbkey(uint32_t T, int k)
+// While the residual is still filling up (the first tens of steps of a run) T grows from step to
+// step, by a factor r that itself shrinks towards 1 (about 1.8, 1.45, 1.35, ... 1.1 after a
+// dozen steps on the synthetic gradients); the prediction follows with 60 % of the last excess
+// growth, which stays below the growth actually seen next.  Tprev = 0: no earlier key known.
+__device__ __forceinline__ uint32_t predict_lbkey(uint32_t T, uint32_t Tprev, int k)
 {
-    const float t = __uint_as_float(T) * (k >= 64 ? 0.94f : 0.90f);
+    float t = __uint_as_float(T);
+    if (Tprev != 0 && T > Tprev) {
+        float r = t / __uint_as_float(Tprev);
+        r = r < 2.0f ? r : 2.0f;
+        t *= 1.0f + 0.6f * (r - 1.0f);
+    }
+    t *= k >= 64 ? 0.94f : 0.90f;
     return __float_as_uint(t) & 0x7fffffffu;     // 0 (no prediction) when T is 0 or the product underflows
 }
 
@@ -588,7 +598,8 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
 finished:
     if (threadIdx.x == 0) f.seg_m[slot] = lists ? m : len;
     if (threadIdx.x == 0) {
-        f.lbkey[slot] = predict_lbkey(T, k);
+        f.lbkey[slot] = predict_lbkey(T, f.last_key[slot], k);
+        f.last_key[slot] = T;
         f.seg_path[slot] = path;
     }
 }
@@ -697,7 +708,7 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
     f.small_ids = t.small_ids; f.large_ids = t.large_ids; f.seg_large = t.seg_large; f.large_q0 = t.large_q0;
     f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_desc = t.tile_desc;
     f.hist = t.hist; f.prefix = t.prefix; f.k_rem = t.k_rem; f.cand_cnt = t.cand_cnt; f.seg_m = t.seg_m;
-    f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.seg_path = t.seg_path; f.lbkey = t.lbkey; f.cand = t.cand;
+    f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.seg_path = t.seg_path; f.lbkey = t.lbkey; f.last_key = t.last_key; f.cand = t.cand;
     f.comp_off = t.comp_off; f.comp_total = t.comp_total; f.comp_key = t.comp_key; f.comp_idx = t.comp_idx;
     f.out = out; f.out_stride = out_stride; f.errword = errword;
 }
