@@ -215,11 +215,13 @@ lgc_status lgc_check(lgc_ctx *ctx);
 
 /* How the last lgc_topk got its entries: the number of (selecting row, layer) pairs with more
  * than 4096 elements; how many of them were finished from candidates collected during
- * lgc_accumulate (no further pass over v); and the total and the largest number of candidates
- * per pair (the k_l selected entries are found among them).  Any pointer may be NULL.  Waits
- * for the stream. */
+ * lgc_accumulate (no further pass over v); the total and the largest number of candidates per
+ * pair (the k_l selected entries are found among them; a pair finished from the data counts
+ * with its length); and how many pairs were finished from the data itself (no usable lists, a
+ * list overflow, too many candidates, or a prediction that was too high).  Any pointer may be
+ * NULL.  Waits for the stream. */
 lgc_status lgc_selection_stats(lgc_ctx *ctx, int64_t *large_segments, int64_t *served_by_accumulation,
-                               int64_t *candidates_total, int64_t *candidates_max);
+                               int64_t *candidates_total, int64_t *candidates_max, int64_t *finished_from_data);
 
 /* Number of kernels the library has enqueued from the calling thread since it was loaded
  * (all contexts); the benchmark reports the difference over its timed region. */

@@ -560,7 +560,7 @@ lgc_status lgc_check(lgc_ctx *c)
 uint64_t lgc_kernel_launches(void) { return g_kernel_launches; }
 
 lgc_status lgc_selection_stats(lgc_ctx *c, int64_t *large_segments, int64_t *served_by_accumulation,
-                               int64_t *candidates_total, int64_t *candidates_max)
+                               int64_t *candidates_total, int64_t *candidates_max, int64_t *finished_from_data)
 {
     if (!c) return LGC_ERR_INVALID_ARG;
     const size_t n = (size_t)c->S * c->sel_v.num_large;
@@ -572,9 +572,10 @@ lgc_status lgc_selection_stats(lgc_ctx *c, int64_t *large_segments, int64_t *ser
         if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
         if (e != cudaSuccess) return cuda_fail(c, e, "lgc_selection_stats");
     }
-    int64_t served = 0, total = 0, most = 0;
+    int64_t served = 0, total = 0, most = 0, from_data = 0;
     for (size_t i = 0; i < n; ++i) {
         served += ep[i] == 0;
+        from_data += ep[i] >= 2;
         total += m[i];
         if (m[i] > most) most = m[i];
     }
@@ -582,6 +583,7 @@ lgc_status lgc_selection_stats(lgc_ctx *c, int64_t *large_segments, int64_t *ser
     if (served_by_accumulation) *served_by_accumulation = served;
     if (candidates_total) *candidates_total = total;
     if (candidates_max) *candidates_max = most;
+    if (finished_from_data) *finished_from_data = from_data;
     return LGC_OK;
 }
 

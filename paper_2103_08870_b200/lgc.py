@@ -72,7 +72,7 @@ def lib() -> C.CDLL:
         l.lgc_last_error.argtypes = [vp]
         l.lgc_last_error.restype = C.c_char_p
         l.lgc_topk_noalloc.argtypes = [vp, C.c_int64, C.c_int64, vp, vp]
-        l.lgc_selection_stats.argtypes = [vp] + [C.POINTER(C.c_int64)] * 4
+        l.lgc_selection_stats.argtypes = [vp] + [C.POINTER(C.c_int64)] * 5
         l.lgc_kernel_launches.argtypes = []
         l.lgc_kernel_launches.restype = C.c_uint64
         for name in EXPORTS:            # every declared entry point must be exported
@@ -224,8 +224,9 @@ class LGC:
                                        host_update.data_ptr(), choice), "lgc_step_host")
 
     def selection_stats(self):
-        """(large (row, layer) pairs, pairs served by the last accumulate, candidates in total, largest count)."""
-        v = [C.c_int64() for _ in range(4)]
+        """(large (row, layer) pairs, pairs served by the last accumulate, candidates in total, largest
+        count, pairs finished from the data)."""
+        v = [C.c_int64() for _ in range(5)]
         self._ok(self._l.lgc_selection_stats(self._ctx, *[C.byref(x) for x in v]), "lgc_selection_stats")
         return tuple(x.value for x in v)
 

@@ -105,6 +105,47 @@ def test_momentum_zero_and_other_densities():
     run_steps([50000, 777], 2, 2, density_ppm=1000000, ae_kind="identity")     # everything is kept
 
 
+def test_layer_spanning_several_compaction_groups():
+    # more than 2048 chunks in one layer: the finishing CTA compacts group after group
+    numel = [9_000_000, 5000]
+    ora, gpu = make_pair(numel, 2, topk_method="select")
+    src = W.GradientSource(W.LayerTable("big", numel, [1, 1]), 2, seed=11, device="cuda")
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t in range(5):
+        g = src.step(t)
+        compare_step(ora, gpu, g.cpu(), g, t % 2, upd)
+    assert gpu.selection_stats()[1] == 2          # both layers served from the accumulation by now
+
+
+def test_dense_selection_uses_the_global_compact_arrays():
+    # k = 40,000 of 2,000,000: more candidates than the finishing CTA keeps in shared memory
+    numel = [2_000_000]
+    ora, gpu = make_pair(numel, 2, density_ppm=20000, topk_method="select")
+    src = W.GradientSource(W.LayerTable("dense", numel, [1]), 2, seed=12, device="cuda")
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t in range(5):
+        g = src.step(t)
+        compare_step(ora, gpu, g.cpu(), g, t % 2, upd)
+    assert gpu.selection_stats()[3] > 20480
+
+
+def test_a_chunk_with_more_candidates_than_its_list_holds():
+    # 3000 large entries side by side land in one or two 4096-element tiles: their lists (1024
+    # records) overflow and the layer is finished from the data; the layer next to it is not affected
+    numel = [400_000, 100_000]
+    K = 2
+    ora, gpu = make_pair(numel, K, density_ppm=20000, momentum=0.0)
+    rng = np.random.default_rng(5)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t in range(6):
+        g = (rng.standard_normal((K, gpu.N)) * 1e-3).astype(np.float32)
+        g[:, 10_000:13_000] += np.float32(1.0) * rng.choice([-1, 1], size=(K, 3000)).astype(np.float32)
+        gt = torch.from_numpy(g)
+        compare_step(ora, gpu, gt, gt.cuda(), t % K, upd)
+    large, served, _, _, from_data = gpu.selection_stats()
+    assert (large, served, from_data) == (2, 1, 1)
+
+
 @pytest.mark.parametrize("fill", ["zeros", "equal", "few_values", "denormal"])
 def test_degenerate_values(fill):
     numel = [9000, 130, 4097, 33000, 300001]      # the last two exceed the candidate capacity when all tie
