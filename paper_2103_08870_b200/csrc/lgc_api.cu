@@ -115,6 +115,7 @@ struct SelectPlan {
     std::vector<int32_t> seg_len, seg_k, seg_out, small_ids, large_ids, seg_large, large_q0, large_order, tchunk0,
         tchunk_large;
     std::vector<int4> tile_desc;
+    std::vector<int2> group_job;
     int tiles_per_row = 0;
     int64_t comp_total = 0;
 };
@@ -141,7 +142,10 @@ SelectPlan plan_select(const std::vector<int64_t> &off, const std::vector<int64_
             const int64_t q0 = off[i] / kSelChunk, q1 = (off[i] + len[i] - 1) / kSelChunk;
             sp.large_q0.push_back((int32_t)q0);
             for (int64_t q = q0; q <= q1; ++q) sp.tchunk_large.push_back(li);
-            sp.tchunk0.push_back((int32_t)sp.tchunk_large.size());
+            const int32_t c0 = sp.tchunk0.back(), c1 = (int32_t)sp.tchunk_large.size();
+            if (c1 - c0 > kSelGroup)
+                for (int32_t gb = c0; gb < c1; gb += kSelGroup) sp.group_job.push_back(make_int2(li, gb));
+            sp.tchunk0.push_back(c1);
             sp.comp_off.push_back(sp.comp_off.back() + select_compact_capacity(len[i]));
         }
     }
@@ -188,6 +192,11 @@ void carve_select(Carver &cv, SelectTables &t, const SelectPlan &sp, int rows)
     t.tchunk0 = cv.take<int32_t>(nl + 1);
     t.tchunk_large = cv.take<int32_t>(nc);
     t.tile_desc = cv.take<int4>(sp.tiles_per_row);
+    t.num_group_jobs = (int)sp.group_job.size();
+    t.group_job = cv.take<int2>(sp.group_job.size());
+    t.job_range = cv.take<int2>((size_t)rows * sp.group_job.size());
+    t.job_cnt = cv.take<int2>((size_t)rows * sp.group_job.size());
+    t.seg_wide = cv.take<int32_t>((size_t)rows * nl);
     t.hist = cv.take<uint32_t>((size_t)rows * nl * kHistBins);
     t.prefix = cv.take<uint32_t>((size_t)rows * nl);
     t.k_rem = cv.take<int32_t>((size_t)rows * nl);
@@ -267,6 +276,7 @@ cudaError_t upload_select(SelectTables &t, SelectPlan sp, cudaStream_t s, std::v
     cudaError_t e = upload(t.seg_off, h.seg_off, s);
     if (e == cudaSuccess) e = upload(t.comp_off, h.comp_off, s);
     if (e == cudaSuccess) e = upload(t.tile_desc, h.tile_desc, s);
+    if (e == cudaSuccess) e = upload(t.group_job, h.group_job, s);
     const std::vector<int32_t> *arrs[] = {&h.seg_len, &h.seg_k, &h.seg_out, &h.seg_large, &h.small_ids, &h.large_ids,
                                           &h.large_q0, &h.large_order, &h.tchunk0, &h.tchunk_large};
     int32_t *dsts[] = {t.seg_len, t.seg_k, t.seg_out, t.seg_large, t.small_ids, t.large_ids,

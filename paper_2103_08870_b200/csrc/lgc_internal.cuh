@@ -17,6 +17,8 @@ constexpr int kSelThreads = 256;
 constexpr int kSelPerThread = 16;
 constexpr int kSelCandCap = 1024;  // candidates a chunk's list holds; more than that and the segment is finished from the data
 constexpr int kHistBins = 2048;    // first radix digit: 11 bits; the next two: 10 bits each
+constexpr int kSelGroup = 2048;    // chunks whose candidate lists one CTA compacts at a time; a segment of more chunks
+                                   // than this has its groups compacted by CTAs of their own before it is finished
 
 // One selection problem family: R rows of `data` (row stride in elements), each cut into the same
 // segments; per segment the k entries of largest |x| are reported, ascending, as int32 offsets.
@@ -48,6 +50,12 @@ struct SelectTables {
     int32_t *seg_large = nullptr;    // [S] index into large_ids, -1 for small segments
     int32_t *large_q0 = nullptr;     // [num_large] first tile the segment overlaps
     int32_t *large_order = nullptr;  // [num_large] indices into large_ids, longest segment first
+    int num_group_jobs = 0;
+    int2 *group_job = nullptr;       // [num_group_jobs] (index into large_ids, first chunk of the group), for the
+                                     // segments of more than kSelGroup chunks
+    int2 *job_range = nullptr;       // [rows][num_group_jobs] candidates before the group, candidates of the group
+    int2 *job_cnt = nullptr;         // [rows][num_group_jobs] entries of the group above / at the k-th key
+    int32_t *seg_wide = nullptr;     // [rows][num_large] the segment's selection was completed group by group
     int32_t *tchunk0 = nullptr;      // [num_large + 1] first tile-chunk of each large segment
     int32_t *tchunk_large = nullptr; // [num_tchunks] index into large_ids
     int4 *tile_desc = nullptr;       // [tiles_per_row] x: first segment the tile overlaps; y: the large segment that

@@ -34,6 +34,11 @@ struct FastArgs {
     int num_large, num_small, num_tchunks;
     int fin_small;                 // small segments served by CTAs of finish_kernel (0 or num_small)
     const int32_t *large_order;    // large segments, longest first: the order the finishing CTAs take them in
+    const int2 *group_job;         // (large segment, first chunk) of every group that the wide kernels serve
+    int num_group_jobs;
+    int2 *job_range;               // [rows][groups] (candidates of the segment before the group, candidates of the group)
+    int2 *job_cnt;                 // [rows][groups] (entries above the k-th key, entries equal to it)
+    int32_t *seg_wide;             // [rows][num_large] 1: the wide kernels serve the segment in this step
     uint4 *zero_ptr;               // buffer the spare CTAs of the finishing launch clear (row 0 only), or nullptr
     uint64_t zero_vecs;            // its length in whole 16-byte units
     int zero_tail;                 // floats beyond them (0..3)
@@ -56,7 +61,7 @@ struct FastArgs {
 constexpr int kFinThreads = 512;      // two finishing CTAs fit on an SM, so every segment of a ResNet starts at once
 constexpr int kFinWarps = kFinThreads / 32;
 constexpr int kFinSmemCap = 20480;    // candidate keys a finishing CTA keeps in shared memory (80 KB; two CTAs per SM)
-constexpr int kFinGroup = 2048;       // chunks whose candidate counts are scanned together during the compaction
+constexpr int kFinGroup = kSelGroup;  // chunks whose candidate counts are scanned together during the compaction
 constexpr int kFinPerThread = 16;     // consecutive entries per thread in the ordered passes
 constexpr int kCandCap = kSelCandCap;  // entries a chunk's list can hold; a chunk with more sends its segment to the data
 constexpr int kZeroPerThread = 8;     // 16-byte stores per thread of a CTA that clears a slice of the update
@@ -275,6 +280,44 @@ struct FinishShared {
     int found[2];
 };
 
+// Ordered emission by counting: an entry of `src` is selected iff its key is above T, or equals T
+// and fewer than r equal keys precede it in the whole segment; its output slot is the number of
+// selected entries before it.  gt_done / eq_done: entries with key > T / == T that precede src.
+template <typename Source>
+__device__ void emit_ordered(const Source &src, uint32_t T, int r, int gt_done, int eq_done, int k,
+                             int32_t *__restrict__ out, FinishShared &sh, int32_t *errword)
+{
+    const int tile = kFinThreads * kFinPerThread;
+    for (int base = 0; base < src.n; base += tile) {
+        uint32_t key[kFinPerThread];
+        const int first = base + (int)threadIdx.x * kFinPerThread;
+        unsigned gt = 0, eq = 0;
+#pragma unroll
+        for (int i = 0; i < kFinPerThread; ++i) {
+            key[i] = first + i < src.n ? src.key_at(first + i) : 0u;
+            if (first + i < src.n) { gt += key[i] > T; eq += key[i] == T; }
+        }
+        unsigned total;
+        const unsigned before = block_prefix_excl<unsigned>(gt | (eq << 16), sh.warp_u, &total);
+        int g = gt_done + (int)(before & 0xffff), e = eq_done + (int)(before >> 16);
+#pragma unroll
+        for (int i = 0; i < kFinPerThread; ++i) {
+            if (first + i < src.n) {
+                int pos = -1;
+                if (key[i] > T) { pos = g + (e < r ? e : r); ++g; }
+                else if (key[i] == T) { if (e < r) pos = g + e; ++e; }
+                if (pos >= 0) {
+                    if (pos < k) out[pos] = src.idx_at(first + i);
+                    else atomicExch(errword, 0x5E60);
+                }
+            }
+        }
+        gt_done += (int)(total & 0xffff);
+        eq_done += (int)(total >> 16);
+        if (gt_done + (eq_done < r ? eq_done : r) >= k) break;     // everything is emitted
+    }
+}
+
 // Completes the radix search below the 11-bit bucket d0 (k_rem entries still to find inside it)
 // and emits the k selected offsets in order; returns the k-th key.  Entries below the bucket, if
 // the source has any, are ignored.
@@ -324,38 +367,8 @@ __device__ uint32_t finish_from(const Source &src, uint32_t d0, int k_rem, int k
         k_rem = sh.found[1];
         __syncthreads();
     }
+    emit_ordered(src, prefix, k_rem, 0, 0, k, out, sh, errword);
     const uint32_t T = prefix;
-    const int r = k_rem;
-    int gt_done = 0, eq_done = 0;            // entries before the current tile
-    const int tile = kFinThreads * kFinPerThread;
-    for (int base = 0; base < src.n; base += tile) {
-        uint32_t key[kFinPerThread];
-        const int first = base + (int)threadIdx.x * kFinPerThread;
-        unsigned gt = 0, eq = 0;
-#pragma unroll
-        for (int i = 0; i < kFinPerThread; ++i) {
-            key[i] = first + i < src.n ? src.key_at(first + i) : 0u;
-            if (first + i < src.n) { gt += key[i] > T; eq += key[i] == T; }
-        }
-        unsigned total;
-        const unsigned before = block_prefix_excl<unsigned>(gt | (eq << 16), sh.warp_u, &total);
-        int g = gt_done + (int)(before & 0xffff), e = eq_done + (int)(before >> 16);
-#pragma unroll
-        for (int i = 0; i < kFinPerThread; ++i) {
-            if (first + i < src.n) {
-                int pos = -1;
-                if (key[i] > T) { pos = g + (e < r ? e : r); ++g; }
-                else if (key[i] == T) { if (e < r) pos = g + e; ++e; }
-                if (pos >= 0) {
-                    if (pos < k) out[pos] = src.idx_at(first + i);
-                    else atomicExch(errword, 0x5E60);
-                }
-            }
-        }
-        gt_done += (int)(total & 0xffff);
-        eq_done += (int)(total >> 16);
-        if (gt_done + (eq_done < r ? eq_done : r) >= k) break;     // everything is emitted
-    }
     return T;
 }
 
@@ -384,13 +397,322 @@ __device__ __forceinline__ void digit_scan(const unsigned *hist, int k, FinishSh
     __syncthreads();
 }
 
+// Whether the candidate lists of large segment li of `row` can serve this step's selection, and
+// how many candidates they hold.  They cannot if they are not from this step, a chunk's list
+// overflowed, the candidates exceed the segment's compact capacity, or fewer than k entries
+// passed a predicted key.  `upto`: a chunk of the segment; *before gets the candidates of the
+// chunks in front of it.  Every thread of the CTA calls this and gets the same answer; it is a
+// pure function of what earlier launches left, so separate launches agree on it.
+struct ListVerdict {
+    bool settled;    // the two-pass path found the bucket of the k-th key in this step
+    bool lists;
+    int m;           // candidates of the segment (valid when lists)
+};
+__device__ __forceinline__ ListVerdict list_verdict(const FastArgs &f, int row, int li, int upto, unsigned *before,
+                                                    unsigned *warp_u)
+{
+    const int64_t slot = (int64_t)row * f.num_large + li;
+    const int k = f.seg_k[f.large_ids[li]];
+    const int64_t cap = f.comp_off[li + 1] - f.comp_off[li];
+    const int c0 = f.tchunk0[li], c1 = f.tchunk0[li + 1];
+    const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
+    ListVerdict v;
+    v.settled = f.seg_epoch[slot] == f.epoch;
+    v.lists = v.settled ? (int64_t)f.seg_m[slot] <= cap : f.lbkey[slot] != 0;
+    v.m = 0;
+    if (before) *before = 0;
+    if (!v.lists) return v;
+    unsigned sum = 0, front = 0, over = 0;
+    for (int c = c0 + (int)threadIdx.x; c < c1; c += (int)blockDim.x) {
+        const unsigned n = (unsigned)cnt[c];
+        sum += n;
+        if (c < upto) front += n;
+        over |= n > (unsigned)kCandCap;
+    }
+    unsigned total, total_front;
+    block_prefix_excl<unsigned>(sum, warp_u, &total);            // per-segment totals stay below 2^31
+    if (before) {
+        block_prefix_excl<unsigned>(front, warp_u, &total_front);
+        *before = total_front;
+    }
+    const int64_t m64 = total;
+    if (__syncthreads_or((int)over) || m64 > cap || (!v.settled && m64 < k)) v.lists = false;
+    v.m = (int)m64;
+    return v;
+}
+
+// Compacts the candidates of the gn chunks from chunk gb on (large segment li of `row`) in index
+// order into ckey/cidx, which already hold `done` entries; returns how many it added.
+// group_off: kFinGroup ints of shared memory.  All kFinThreads threads take part.
+__device__ __forceinline__ int compact_group(const FastArgs &f, int row, int li, int gb, int gn, int done,
+                                             uint32_t *ckey, int32_t *cidx, int *group_off, unsigned *warp_u)
+{
+    constexpr int kPerT = kFinGroup / kFinThreads;
+    const int c0 = f.tchunk0[li], q0 = f.large_q0[li];
+    const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
+    // exclusive prefix of the chunk counts of this group, in shared memory
+    int mine[kPerT];
+    unsigned sum = 0;
+#pragma unroll
+    for (int j = 0; j < kPerT; ++j) {
+        const int e = (int)threadIdx.x * kPerT + j;
+        mine[j] = e < gn ? cnt[gb + e] : 0;
+        sum += (unsigned)mine[j];
+    }
+    unsigned total;
+    unsigned at = block_prefix_excl<unsigned>(sum, warp_u, &total);
+#pragma unroll
+    for (int j = 0; j < kPerT; ++j) {
+        group_off[threadIdx.x * kPerT + j] = (int)at;
+        at += (unsigned)mine[j];
+    }
+    __syncthreads();
+    // one candidate per thread and trip, eight trips in flight: its chunk by binary search in
+    // shared memory, then its record from the chunk's list (neighbouring ranks read
+    // neighbouring records)
+    for (int base = 0; base < (int)total; base += kFinThreads * 8) {
+        const uint2 *rec[8];
+        int tile0[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const int r = base + t * kFinThreads + (int)threadIdx.x;
+            rec[t] = nullptr;
+            tile0[t] = 0;
+            if (r < (int)total) {
+                int lo = 0, hi = gn;                       // last chunk whose offset is <= rank
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (group_off[mid] <= r) lo = mid; else hi = mid;
+                }
+                rec[t] = f.cand + ((int64_t)row * f.num_tchunks + gb + lo) * kCandCap + (r - group_off[lo]);
+                tile0[t] = (q0 + (gb + lo - c0)) * kSelChunk;                 // N < 2^31
+            }
+        }
+        uint2 kp[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) kp[t] = rec[t] ? __ldg(rec[t]) : make_uint2(0u, 0u);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            const int r = base + t * kFinThreads + (int)threadIdx.x;
+            if (rec[t]) {
+                ckey[done + r] = kp[t].x;
+                cidx[done + r] = tile0[t] + (int)kp[t].y;
+            }
+        }
+    }
+    __syncthreads();                                       // group_off may be rewritten by the caller's next group
+    return (int)total;
+}
+
+// ------------------------------------------------------------------------------------------
+// Segments of more than kFinGroup chunks (tens of millions of entries) are not left to one CTA:
+// every step of the finishing is spread over the groups of chunks, one CTA per group and launch,
+// grid (groups, rows).  compact_groups_kernel compacts each group's candidates into the
+// segment's global compact arrays and finds the bucket of the k-th key; wide_digit_kernel<10>
+// and <0> settle the remaining 20 bits of the key; wide_count_kernel counts, per group, the
+// entries above and at the key; wide_emit_kernel writes each group's selected offsets behind
+// those of the groups before it.  Where CTAs of a launch contribute to one result, the CTA that
+// arrives last (a ticket counter tells; nobody waits) completes it.  If the lists cannot serve
+// the step, all five return at once and the finishing CTA of finish_kernel works on the data.
+// ------------------------------------------------------------------------------------------
+struct JobGeom {
+    int li, gb, job, njobs;      // large segment, first chunk of the group, its number inside the segment, groups of the segment
+    int64_t slot, rec;           // (row, segment) and (row, group) record
+};
+__device__ __forceinline__ JobGeom job_geom(const FastArgs &f, int row)
+{
+    JobGeom g;
+    const int2 j = f.group_job[blockIdx.x];
+    g.li = j.x;
+    g.gb = j.y;
+    const int c0 = f.tchunk0[g.li], c1 = f.tchunk0[g.li + 1];
+    g.job = (g.gb - c0) / kFinGroup;
+    g.njobs = (c1 - c0 + kFinGroup - 1) / kFinGroup;
+    g.slot = (int64_t)row * f.num_large + g.li;
+    g.rec = (int64_t)row * f.num_group_jobs + blockIdx.x;
+    return g;
+}
+
+// True in the CTA that is the last of n to arrive at the ticket; its later reads see what the
+// others wrote before they arrived.  Every thread of the CTA calls this.
+__device__ __forceinline__ bool arrives_last(int32_t *ticket, int n, int *flag)
+{
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) *flag = atomicAdd(ticket, 1) == n - 1;
+    __syncthreads();
+    const bool last = *flag != 0;
+    if (last) __threadfence();
+    return last;
+}
+
+__global__ void __launch_bounds__(kFinThreads) compact_groups_kernel(FastArgs f)
+{
+    __shared__ unsigned h[kHistBins];
+    __shared__ int group_off[kFinGroup];
+    __shared__ unsigned warp_u[kFinWarps];
+    __shared__ int warp_i[kFinWarps];
+    __shared__ int is_last, scan_flag;
+    const int row = blockIdx.y;
+    const JobGeom g = job_geom(f, row);
+    unsigned before;
+    const ListVerdict v = list_verdict(f, row, g.li, g.gb, &before, warp_u);
+    if (g.job == 0 && threadIdx.x == 0) f.seg_wide[g.slot] = v.lists ? 1 : 0;
+    if (!v.lists) return;
+    const int c1 = f.tchunk0[g.li + 1];
+    const int gn = c1 - g.gb < kFinGroup ? c1 - g.gb : kFinGroup;
+    uint32_t *ckey = f.comp_key + (int64_t)row * f.comp_total + f.comp_off[g.li];
+    int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[g.li];
+    const int added = compact_group(f, row, g.li, g.gb, gn, (int)before, ckey, cidx, group_off, warp_u);
+    if (threadIdx.x == 0) {
+        f.job_range[g.rec] = make_int2((int)before, added);
+        if ((int64_t)before + added > (int64_t)v.m) atomicExch(f.errword, 0x5E71);
+    }
+    if (v.settled) return;                                   // the two-pass path found the bucket already
+    // leading digits of this group's candidates (every entry at or above the predicted key is a
+    // candidate and there are at least k, so the bucket of the k-th key is among them)
+    for (int b = threadIdx.x; b < kHistBins; b += kFinThreads) h[b] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < added; i += kFinThreads) atomicAdd(&h[ckey[before + i] >> 20], 1u);
+    __syncthreads();
+    uint32_t *gh = f.hist + g.slot * kHistBins;
+    for (int b = threadIdx.x; b < kHistBins; b += kFinThreads)
+        if (h[b]) atomicAdd(gh + b, h[b]);
+    if (!arrives_last(&f.seg_ticket[g.slot], g.njobs, &is_last)) return;
+    const bool ok = bucket_scan<kFinThreads>(f, g.slot, f.seg_k[f.large_ids[g.li]], warp_i, &scan_flag);
+    if (threadIdx.x == 0 && !ok) atomicExch(f.errword, 0x5E41);
+}
+
+// Ten more bits of the k-th key: histogram of that digit over the candidates that match the bits
+// found so far; SHIFT 10 follows the bucket (prefix holds the 11-bit bucket), SHIFT 0 follows
+// that (prefix holds the key so far).  Leaves the key so far in prefix and the rank inside it in k_rem.
+template <int SHIFT>
+__global__ void __launch_bounds__(kFinThreads) wide_digit_kernel(FastArgs f)
+{
+    __shared__ int h[1024];
+    __shared__ int warp_i[kFinWarps];
+    __shared__ int is_last;
+    const int row = blockIdx.y;
+    const JobGeom g = job_geom(f, row);
+    if (!f.seg_wide[g.slot]) return;
+    const int2 range = f.job_range[g.rec];
+    const uint32_t prefix = SHIFT == 10 ? f.prefix[g.slot] << 20 : f.prefix[g.slot];
+    const uint32_t decided = SHIFT == 10 ? 0x7ff00000u : 0x7ffffc00u;
+    for (int b = threadIdx.x; b < 1024; b += kFinThreads) h[b] = 0;
+    __syncthreads();
+    const uint32_t *key = f.comp_key + (int64_t)row * f.comp_total + f.comp_off[g.li] + range.x;
+    for (int base = 0; base < range.y; base += kFinThreads * 8) {        // eight independent loads per thread
+        uint32_t x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = base + j * kFinThreads + (int)threadIdx.x;
+            x[j] = i < range.y ? key[i] : 0xffffffffu;                   // never matches the prefix
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if ((x[j] & decided) == prefix) atomicAdd(&h[(x[j] >> SHIFT) & 1023u], 1);
+    }
+    __syncthreads();
+    uint32_t *gh = f.hist + g.slot * kHistBins;
+    for (int b = threadIdx.x; b < 1024; b += kFinThreads)
+        if (h[b]) atomicAdd(gh + b, (unsigned)h[b]);
+    if (!arrives_last(&f.seg_ticket[g.slot], g.njobs, &is_last)) return;
+    constexpr int kPer = 1024 / kFinThreads;
+    const int k_rem = f.k_rem[g.slot];
+    int hh[kPer], part = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        hh[i] = (int)__ldcg(gh + threadIdx.x * kPer + i);
+        part += hh[i];
+        gh[threadIdx.x * kPer + i] = 0u;
+    }
+    if (threadIdx.x == 0) f.seg_ticket[g.slot] = 0;
+    const int incl = block_suffix_incl(part, warp_i);
+    if (incl >= k_rem && incl - part < k_rem) {
+        int above = incl - part;
+#pragma unroll
+        for (int i = kPer - 1; i >= 0; --i) {
+            if (above + hh[i] >= k_rem) {
+                f.prefix[g.slot] = prefix | (uint32_t)(threadIdx.x * kPer + i) << SHIFT;
+                f.k_rem[g.slot] = k_rem - above;
+                break;
+            }
+            above += hh[i];
+        }
+    }
+    if (threadIdx.x == 0 && incl < k_rem) atomicExch(f.errword, 0x5E51 + SHIFT);
+}
+
+// Entries of each group above and at the k-th key.
+__global__ void __launch_bounds__(kFinThreads) wide_count_kernel(FastArgs f)
+{
+    __shared__ unsigned long long warp_l[kFinWarps];
+    const int row = blockIdx.y;
+    const JobGeom g = job_geom(f, row);
+    if (!f.seg_wide[g.slot]) return;
+    const int2 range = f.job_range[g.rec];
+    const uint32_t T = f.prefix[g.slot];
+    const uint32_t *key = f.comp_key + (int64_t)row * f.comp_total + f.comp_off[g.li] + range.x;
+    unsigned long long mine = 0;
+    for (int i = threadIdx.x; i < range.y; i += kFinThreads) {
+        const uint32_t x = key[i];
+        mine += (unsigned long long)(x > T) | (unsigned long long)(x == T) << 32;
+    }
+    unsigned long long total;
+    block_prefix_excl<unsigned long long>(mine, warp_l, &total);
+    if (threadIdx.x == 0) f.job_cnt[g.rec] = make_int2((int)(total & 0xffffffffu), (int)(total >> 32));
+}
+
+// Selected offsets of each group, behind those of the groups before it; the first group's CTA
+// also stores the key from which the next step collects candidates.
+__global__ void __launch_bounds__(kFinThreads) wide_emit_kernel(FastArgs f)
+{
+    __shared__ FinishShared sh;
+    __shared__ unsigned long long warp_l[kFinWarps];
+    const int row = blockIdx.y;
+    const JobGeom g = job_geom(f, row);
+    if (!f.seg_wide[g.slot]) return;
+    const int2 range = f.job_range[g.rec];
+    const uint32_t T = f.prefix[g.slot];
+    const int r = f.k_rem[g.slot];
+    const int s = f.large_ids[g.li];
+    const int k = f.seg_k[s];
+    unsigned long long mine = 0;
+    unsigned cands = 0;
+    for (int j = threadIdx.x; j < g.njobs; j += kFinThreads) {
+        const int64_t rec = g.rec - g.job + j;
+        cands += (unsigned)f.job_range[rec].y;
+        if (j < g.job) {
+            const int2 c = f.job_cnt[rec];
+            mine += (unsigned long long)(unsigned)c.x | (unsigned long long)(unsigned)c.y << 32;
+        }
+    }
+    unsigned long long total;
+    block_prefix_excl<unsigned long long>(mine, warp_l, &total);
+    unsigned m;
+    block_prefix_excl<unsigned>(cands, sh.warp_u, &m);
+    const int gt0 = (int)(total & 0xffffffffu), eq0 = (int)(total >> 32);
+    if (gt0 + (eq0 < r ? eq0 : r) < k) {
+        const int64_t base = (int64_t)row * f.comp_total + f.comp_off[g.li] + range.x;
+        CompactSource src{f.comp_key + base, f.comp_idx + base, range.y};
+        emit_ordered(src, T, r, gt0, eq0, k, f.out + (int64_t)row * f.out_stride + f.seg_out[s], sh, f.errword);
+    }
+    if (g.job == 0 && threadIdx.x == 0) {
+        f.seg_m[g.slot] = (int)m;
+        f.lbkey[g.slot] = predict_lbkey(T, f.last_key[g.slot], k);
+        f.last_key[g.slot] = T;
+        f.seg_path[g.slot] = f.seg_epoch[g.slot] == f.epoch ? 1 : 0;
+    }
+}
+
 // The selection of one (segment, row) is completed by one CTA.  The first num_small CTAs of a
 // row each do one small segment outright.  For a large segment the CTA
 //  1. settles the bucket of the k-th key from the histogram the accumulation left, unless path
 //     (b) already did; if fewer than k entries had passed the predicted key it counts the
 //     leading digits of the whole segment itself;
-//  2. compacts the candidates in index order (thread t owns chunk t of a group of chunks)
-//     and finishes on them -- or on the data when there are no valid lists or too many entries;
+//  2. compacts the candidates in index order (each thread takes candidate ranks and finds their
+//     chunk by binary search; a segment of more than kFinGroup chunks arrives compacted) and
+//     finishes on them -- or on the data when there are no valid lists or too many entries;
 //  3. stores the key from which the next step should collect candidates.
 // CTA order: large segments longest first, then the small ones, then spare CTAs that clear the
 // dense update buffer (if the caller announced it) while the rest of the launch is busy.
@@ -429,26 +751,20 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
     int32_t *out = f.out + (int64_t)row * f.out_stride + f.seg_out[s];
     const int64_t cap = f.comp_off[li + 1] - f.comp_off[li];
     const int c0 = f.tchunk0[li], c1 = f.tchunk0[li + 1];
-    const int q0 = f.large_q0[li];
-    const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
-    constexpr int kPerT = kFinGroup / kFinThreads;
-    // 1. are there lists for this step, and how many candidates do they hold?
-    const bool settled = f.seg_epoch[slot] == f.epoch;        // path (b) ran and found the bucket
-    bool lists = settled ? (int64_t)f.seg_m[slot] <= cap : f.lbkey[slot] != 0;
-    int64_t m64 = 0;
-    if (lists) {
-        unsigned sum = 0, over = 0;
-        for (int c = c0 + (int)threadIdx.x; c < c1; c += kFinThreads) {
-            const unsigned n = (unsigned)cnt[c];
-            sum += n;
-            over |= n > (unsigned)kCandCap;
-        }
-        unsigned total;
-        block_prefix_excl<unsigned>(sum, sh.warp_u, &total);   // per-segment totals stay below 2^31
-        m64 = total;
-        if (__syncthreads_or((int)over) || m64 > cap || (!settled && m64 < k)) lists = false;
+    // 1. are there lists for this step, and how many candidates do they hold?  A segment of more than
+    // one group of chunks has been served by the wide kernels, or is left to the data.
+    const bool grouped = c1 - c0 > kFinGroup;
+    if (grouped && f.seg_wide[slot]) return;
+    ListVerdict verdict;
+    if (grouped) {
+        verdict.settled = f.seg_epoch[slot] == f.epoch;
+        verdict.lists = false;
+        verdict.m = 0;
+    } else {
+        verdict = list_verdict(f, row, li, c0, nullptr, sh.warp_u);
     }
-    const int m = (int)m64;
+    const bool settled = verdict.settled, lists = verdict.lists;
+    const int m = verdict.m;
     int path;
     uint32_t d0 = 0, T;
     int k_rem = 0;
@@ -457,62 +773,7 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
         // 2. compaction.  Keys stay in shared memory when they fit; offsets are needed only for the winners.
         uint32_t *ckey = m <= kFinSmemCap ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
         int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
-        int done = 0;
-        for (int gb = c0; gb < c1; gb += kFinGroup) {
-            // exclusive prefix of the chunk counts of this group, in shared memory
-            const int gn = c1 - gb < kFinGroup ? c1 - gb : kFinGroup;
-            int mine[kPerT];
-            unsigned sum = 0;
-#pragma unroll
-            for (int j = 0; j < kPerT; ++j) {
-                const int e = (int)threadIdx.x * kPerT + j;
-                mine[j] = e < gn ? cnt[gb + e] : 0;
-                sum += (unsigned)mine[j];
-            }
-            unsigned total;
-            unsigned at = block_prefix_excl<unsigned>(sum, sh.warp_u, &total);
-#pragma unroll
-            for (int j = 0; j < kPerT; ++j) {
-                group_off[threadIdx.x * kPerT + j] = (int)at;
-                at += (unsigned)mine[j];
-            }
-            __syncthreads();
-            // one candidate per thread and trip, eight trips in flight: its chunk by binary search in
-            // shared memory, then its record from the chunk's list (neighbouring ranks read
-            // neighbouring records)
-            for (int base = 0; base < (int)total; base += kFinThreads * 8) {
-                const uint2 *rec[8];
-                int tile0[8];
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    const int r = base + t * kFinThreads + (int)threadIdx.x;
-                    rec[t] = nullptr;
-                    tile0[t] = 0;
-                    if (r < (int)total) {
-                        int lo = 0, hi = gn;                       // last chunk whose offset is <= rank
-                        while (hi - lo > 1) {
-                            const int mid = (lo + hi) >> 1;
-                            if (group_off[mid] <= r) lo = mid; else hi = mid;
-                        }
-                        rec[t] = f.cand + ((int64_t)row * f.num_tchunks + gb + lo) * kCandCap + (r - group_off[lo]);
-                        tile0[t] = (q0 + (gb + lo - c0)) * kSelChunk;                 // N < 2^31
-                    }
-                }
-                uint2 kp[8];
-#pragma unroll
-                for (int t = 0; t < 8; ++t) kp[t] = rec[t] ? __ldg(rec[t]) : make_uint2(0u, 0u);
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    const int r = base + t * kFinThreads + (int)threadIdx.x;
-                    if (rec[t]) {
-                        ckey[done + r] = kp[t].x;
-                        cidx[done + r] = tile0[t] + (int)kp[t].y;
-                    }
-                }
-            }
-            done += (int)total;
-            __syncthreads();                                       // group_off is rewritten by the next group
-        }
+        const int done = compact_group(f, row, li, c0, c1 - c0, 0, ckey, cidx, group_off, sh.warp_u);
         if (threadIdx.x == 0 && done != m) atomicExch(f.errword, 0x5E70);
         // 3. the bucket of the k-th key: from path (b), or from the candidates' own leading digits
         // (every entry at or above the predicted key is a candidate, and there are at least k)
@@ -703,7 +964,8 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
     f.data = data; f.row_stride = row_stride; f.row0 = row0;
     f.num_large = t.num_large; f.num_small = t.num_small; f.num_tchunks = t.num_tchunks; f.epoch = epoch;
     f.fin_small = 0;
-    f.large_order = t.large_order; f.zero_ptr = nullptr; f.zero_vecs = 0; f.zero_tail = 0;
+    f.large_order = t.large_order; f.group_job = t.group_job; f.num_group_jobs = t.num_group_jobs;
+    f.job_range = t.job_range; f.job_cnt = t.job_cnt; f.seg_wide = t.seg_wide; f.zero_ptr = nullptr; f.zero_vecs = 0; f.zero_tail = 0;
     f.seg_off = t.seg_off; f.seg_len = t.seg_len; f.seg_k = t.seg_k; f.seg_out = t.seg_out;
     f.small_ids = t.small_ids; f.large_ids = t.large_ids; f.seg_large = t.seg_large; f.large_q0 = t.large_q0;
     f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_desc = t.tile_desc;
@@ -747,6 +1009,14 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
     f.fin_small = (int64_t)rows * t.num_small <= 512 && t.num_large ? t.num_small : 0;
     if (t.num_small && !f.fin_small)
         select_small_only_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
+    if (t.num_group_jobs) {
+        const dim3 grid(t.num_group_jobs, rows);
+        compact_groups_kernel<<<grid, kFinThreads, 0, st>>>(f), ++g_kernel_launches;
+        wide_digit_kernel<10><<<grid, kFinThreads, 0, st>>>(f), ++g_kernel_launches;
+        wide_digit_kernel<0><<<grid, kFinThreads, 0, st>>>(f), ++g_kernel_launches;
+        wide_count_kernel<<<grid, kFinThreads, 0, st>>>(f), ++g_kernel_launches;
+        wide_emit_kernel<<<grid, kFinThreads, 0, st>>>(f), ++g_kernel_launches;
+    }
     unsigned spare = 0;
     if (clear && clear_floats > 0 && t.num_large) {
         f.zero_ptr = reinterpret_cast<uint4 *>(clear);

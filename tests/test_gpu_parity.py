@@ -106,7 +106,7 @@ def test_momentum_zero_and_other_densities():
 
 
 def test_layer_spanning_several_compaction_groups():
-    # more than 2048 chunks in one layer: the finishing CTA compacts group after group
+    # more than 2048 chunks in one layer: its selection is completed group by group, one CTA per group
     numel = [9_000_000, 5000]
     ora, gpu = make_pair(numel, 2, topk_method="select")
     src = W.GradientSource(W.LayerTable("big", numel, [1, 1]), 2, seed=11, device="cuda")
@@ -115,6 +115,25 @@ def test_layer_spanning_several_compaction_groups():
         g = src.step(t)
         compare_step(ora, gpu, g.cpu(), g, t % 2, upd)
     assert gpu.selection_stats()[1] == 2          # both layers served from the accumulation by now
+
+
+@pytest.mark.parametrize("levels, first_from_data", [(50, 0), (3, 1)])
+def test_layer_of_several_groups_with_ties(levels, first_from_data):
+    # integer-valued gradients: the k-th magnitude is shared by many entries of the 9 M layer, which
+    # is finished group by group (51 levels: ~178 k entries tie for 9000 places in the first step)
+    # or, when the tied entries exceed the layer's compact capacity (4 levels: 2.6 M), from the data
+    numel = [9_000_000, 5000]
+    K = 2
+    ora, gpu = make_pair(numel, K, momentum=0.0, topk_method="select")
+    rng = np.random.default_rng(levels)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    from_data = []
+    for t in range(4):
+        g = rng.integers(-levels, levels + 1, size=(K, gpu.N)).astype(np.float32)
+        gt = torch.from_numpy(g)
+        compare_step(ora, gpu, gt, gt.cuda(), t % K, upd)
+        from_data.append(gpu.selection_stats()[4])
+    assert from_data[0] == first_from_data
 
 
 def test_dense_selection_uses_the_global_compact_arrays():
