@@ -75,15 +75,18 @@ constexpr int kAccThreads = 1024;     // accumulation: one 128-bit g/u/v triple 
 // 4-6 k and makes a prediction that is too high rare; when it happens only the fallback is paid.
 // While the residual is still filling up (the first tens of steps of a run) T grows from step to
 // step, by a factor r that itself shrinks towards 1 (about 1.8, 1.45, 1.35, ... 1.1 after a
-// dozen steps on the synthetic gradients); the prediction follows with 60 % of the last excess
-// growth, which stays below the growth actually seen next.  Tprev = 0: no earlier key known.
+// dozen steps on the synthetic gradients); the prediction follows with 60 % of the last growth
+// beyond 10 %, which stays below the growth actually seen next.  Growth of less than 10 % is
+// not followed: in steady state that is the difference between rows (leaders alternate), and
+// chasing it put the prediction above the next key for most layers of a step every ~15 steps.
+// Tprev = 0: no earlier key known.
 __device__ __forceinline__ uint32_t predict_lbkey(uint32_t T, uint32_t Tprev, int k)
 {
     float t = __uint_as_float(T);
     if (Tprev != 0 && T > Tprev) {
         float r = t / __uint_as_float(Tprev);
         r = r < 2.0f ? r : 2.0f;
-        t *= 1.0f + 0.6f * (r - 1.0f);
+        if (r > 1.1f) t *= 1.0f + 0.6f * (r - 1.1f);
     }
     t *= k >= 64 ? 0.94f : 0.90f;
     return __float_as_uint(t) & 0x7fffffffu;     // 0 (no prediction) when T is 0 or the product underflows
@@ -869,9 +872,8 @@ finished:
 // (a) Stage 1 fused with candidate collection.  Grid (tiles per row, K); a CTA streams one tile
 // of one row exactly as accumulate_kernel does (u <- m u + g fused, v <- v + u; Algorithm 1/2 and
 // Section V-A).  A CTA of a selecting row then looks at its fresh v: for every large segment the
-// tile overlaps and that has a predicted bucket, the entries at or above the bucket are
-// histogrammed and listed, and the CTA that completes the segment settles the bucket of its k-th
-// key.
+// tile overlaps and that has a predicted key, the entries at or above that key are listed, in
+// position order, with their keys.
 // ------------------------------------------------------------------------------------------
 // The part [lo, hi) of a tile, held four consecutive entries per thread (positions p0 .. p0+3):
 // the entries whose key reaches lbkey are written, ascending, to the chunk's candidate list.
@@ -882,10 +884,27 @@ __device__ __forceinline__ void collect_tile(const FastArgs &f, int64_t chunk, c
 #pragma unroll
     for (int i = 0; i < 4; ++i)
         if (live && p0 + i >= lo && p0 + i < hi && key[i] >= lbkey) flags |= 1u << i;
-    unsigned total;
-    unsigned at = block_prefix_excl<unsigned>((unsigned)__popc(flags), warp_u, &total);
-    if (threadIdx.x == 0) f.cand_cnt[chunk] = (int)total;
+    // Candidates are rare (a handful per tile): most warps have none and skip the scan; one barrier,
+    // and only the threads that hold a candidate add up the warps before theirs.
+    const unsigned lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const unsigned cnt = (unsigned)__popc(flags);
+    unsigned incl = cnt;
+    if (__ballot_sync(kFull, cnt != 0)) {
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned y = __shfl_up_sync(kFull, incl, d);
+            if (lane >= (unsigned)d) incl += y;
+        }
+    }
+    if (lane == 31) warp_u[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const unsigned total = __reduce_add_sync(kFull, warp_u[lane]);
+        if (lane == 0) f.cand_cnt[chunk] = (int)total;
+    }
     if (flags) {
+        unsigned at = incl - cnt;
+        for (unsigned w = 0; w < warp; ++w) at += warp_u[w];
         uint2 *dst = f.cand + chunk * kCandCap;
 #pragma unroll
         for (int i = 0; i < 4; ++i)
