@@ -36,7 +36,7 @@ GRAD_SETS = 3            # distinct gradient batches cycled through (each far la
 # DRAM bytes (read + write) per element that ncu measured for accumulate_select_kernel on the small
 # capture case (profiles/accumulate_select_kernel_resnet50_k2.md); traffic grows in proportion to K * N.
 # Set to None whenever that kernel changes until the counters are taken again.
-NCU_DRAM_BYTES_PER_ELEMENT = 18.99
+NCU_DRAM_BYTES_PER_ELEMENT = 19.00
 
 
 def measured_peak():
