@@ -358,18 +358,12 @@ sparse_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val
     }
 }
 
-__device__ __forceinline__ int64_t find_in(const int32_t *__restrict__ a, int64_t lo, int64_t hi, int32_t x)
-{
-    while (lo < hi) {
-        const int64_t mid = (lo + hi) >> 1;
-        if (a[mid] < x) lo = mid + 1; else hi = mid;
-    }
-    return lo;
-}
-
 // Parameter-server scatter: update[i] = sum over nodes k (ascending) that kept i of values_k / K.
 // The lowest node holding an index sums for all of them, so the order of additions is fixed and
 // no atomics are needed.  Each node's own sent entries leave its u and v.
+// The index is looked up in the other nodes' lists of the same layer eight nodes at a time: the
+// searches halve the same range in lock step, so their loads are in flight together.
+constexpr int kOwnBatch = 8;
 __global__ void scatter_own_kernel(const float *__restrict__ values, const int32_t *__restrict__ idx,
                                    const int32_t *__restrict__ slot_layer, const int32_t *__restrict__ koff,
                                    int64_t mu, int K, int64_t N, float *__restrict__ update,
@@ -382,18 +376,46 @@ __global__ void scatter_own_kernel(const float *__restrict__ values, const int32
     u[(int64_t)k * N + i] = 0.0f;
     v[(int64_t)k * N + i] = 0.0f;
     const int l = slot_layer[p];
-    const int64_t lo = koff[l], hi = koff[l + 1];
-    for (int kk = 0; kk < k; ++kk) {
-        const int32_t *row = idx + (int64_t)kk * mu;
-        const int64_t q = find_in(row, lo, hi, i);
-        if (q < hi && row[q] == i) return;      // a lower node owns this index
-    }
+    const int lo = koff[l], len = koff[l + 1] - lo;            // at least one kept entry per layer
     const float fk = (float)K;
-    float acc = __fadd_rn(0.0f, __fdiv_rn(values[(int64_t)k * mu + p], fk));
-    for (int kk = k + 1; kk < K; ++kk) {
-        const int32_t *row = idx + (int64_t)kk * mu;
-        const int64_t q = find_in(row, lo, hi, i);
-        if (q < hi && row[q] == i) acc = __fadd_rn(acc, __fdiv_rn(values[(int64_t)kk * mu + q], fk));
+    float acc = 0.0f;
+    bool own_added = false;
+    for (int k0 = 0; k0 < K; k0 += kOwnBatch) {
+        // lower bound of i in the layer's slice of nodes k0 .. k0 + 7 (the own node and nodes >= K idle)
+        const int32_t *base[kOwnBatch];
+#pragma unroll
+        for (int j = 0; j < kOwnBatch; ++j) base[j] = idx + (int64_t)(k0 + j < K ? k0 + j : k) * mu + lo;
+        for (int n = len; n > 1;) {
+            const int half = n >> 1;
+            int32_t probe[kOwnBatch];
+#pragma unroll
+            for (int j = 0; j < kOwnBatch; ++j) probe[j] = __ldg(base[j] + half - 1);
+#pragma unroll
+            for (int j = 0; j < kOwnBatch; ++j)
+                if (probe[j] < i) base[j] += half;
+            n -= half;
+        }
+        // the lower bound is base[j], or the slot after it when that entry is still below i
+        int32_t at[kOwnBatch];
+#pragma unroll
+        for (int j = 0; j < kOwnBatch; ++j) at[j] = __ldg(base[j]);
+#pragma unroll
+        for (int j = 0; j < kOwnBatch; ++j) {
+            const int kk = k0 + j;
+            if (kk >= K) break;
+            if (kk == k) {
+                acc = __fadd_rn(acc, __fdiv_rn(values[(int64_t)k * mu + p], fk));
+                own_added = true;
+                continue;
+            }
+            const int32_t *row = idx + (int64_t)kk * mu;
+            const int32_t *hit = nullptr;
+            if (at[j] == i) hit = base[j];
+            else if (at[j] < i && base[j] + 1 < row + lo + len && __ldg(base[j] + 1) == i) hit = base[j] + 1;
+            if (!hit) continue;
+            if (!own_added) return;                               // a lower node owns this index
+            acc = __fadd_rn(acc, __fdiv_rn(values[(int64_t)kk * mu + (hit - row)], fk));
+        }
     }
     update[i] = acc;
 }
