@@ -21,6 +21,7 @@ from typing import Dict, List, Optional, Sequence
 import numpy as np
 
 import oracle as O
+from oracle import full_ae as A5
 
 
 def _param_order(c1: int, c2: int, variant: str, K: int):
@@ -43,7 +44,8 @@ class OracleLGC:
                  c1: int = 8, c2: int = 4, params: Optional[np.ndarray] = None,
                  innovation_permille: int = 100, lr: float = 1e-3, beta1: float = 0.9,
                  beta2: float = 0.999, eps: float = 1e-8, topk_method: str = "auto"):
-        assert variant in ("rar", "ps") and ae_kind in ("conv2", "identity")
+        assert variant in ("rar", "ps") and ae_kind in ("conv2", "identity", "conv5")
+        assert ae_kind != "conv5" or variant == "rar"
         self.numel = [int(n) for n in layer_numel]
         self.L = len(self.numel)
         self.K = int(num_nodes)
@@ -64,7 +66,7 @@ class OracleLGC:
         self.op1 = (self.L1 - 3) % 2 if self.L1 >= 3 else 0   # decoder layer 1: L2 -> L1
         self.op2 = (self.mu - 3) % 2 if self.mu >= 3 else 0   # decoder layer 2: L1 -> mu
         self.p: Dict[str, np.ndarray] = {}
-        self.order = _param_order(c1, c2, variant, self.K)
+        self.order = A5.param_shapes() if ae_kind == "conv5" else _param_order(c1, c2, variant, self.K)
         if params is not None:
             self.set_params(params)
         self.adam_m = self.adam_v = None
@@ -117,6 +119,9 @@ class OracleLGC:
         if self.ae_kind == "identity":
             self.z = self.val.astype(np.float64).reshape(self.K, 1, self.mu)
             return
+        if self.ae_kind == "conv5":          # the paper's full-size encoder (Section IV-C)
+            self.z = np.stack([A5.encode(self.val[k], self.p) for k in range(self.K)])
+            return
         self.z = np.stack([self._enc(self.val[k].astype(np.float64))[1] for k in range(self.K)])
 
     def combine(self, common_node: int = 0) -> None:
@@ -142,6 +147,8 @@ class OracleLGC:
         if self.variant == "rar":
             if self.ae_kind == "identity":
                 self.r = self.zbar.reshape(1, self.mu).copy()
+            elif self.ae_kind == "conv5":
+                self.r = A5.decode(self.zbar, self.p, self.mu).reshape(1, self.mu)
             else:
                 self.r = self._dec(self.zbar, "dec")[1].reshape(1, self.mu)
             return

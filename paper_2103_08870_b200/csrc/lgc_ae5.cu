@@ -1,0 +1,652 @@
+// The paper's full-size autoencoder (Section IV-C: encoder of five 1-D convolutions with 64, 128,
+// 256, 64 and 4 filters, decoder of five transposed convolutions with 4, 32, 64, 128, 32 filters
+// and a final 1x1 convolution, leaky ReLU between layers) for the ring-allreduce form of
+// Section IV-B: every node's kept values are encoded, the codes averaged, one decoder
+// reconstructs.
+//
+// Activations are kept channels-last, [node][position][channel], so that row t of the im2col
+// matrix of a kernel-3 stride-2 convolution is the contiguous slice [2t C_in, (2t+3) C_in) of the
+// activation: the convolutions with 64, 128 and 256 input channels are GEMMs
+//     out[t][co] = sum_j A[t][j] W[co][j],   j = tau C_in + ci,
+// run on the tensor cores (tcgen05.mma kind::tf32, operands staged by TMA into 128-byte-swizzled
+// shared memory, accumulator in tensor memory).  fp32 accuracy is kept by splitting every
+// operand into two tf32 numbers, x = hi + lo, and accumulating hi*hi + hi*lo + lo*hi.
+// The first convolution (one input channel), the 1x1 convolutions and the decoder (which runs
+// once, not once per node) use the ordinary fp32 pipes.
+#include "lgc_internal.cuh"
+
+namespace lgc {
+
+namespace {
+
+constexpr float kSlope = 0.01f;       // leaky-ReLU slope (the paper names the activation, not the slope)
+constexpr int kTileM = 128;           // output positions per CTA of the GEMM: the M of one tcgen05.mma
+constexpr int kBlockK = 32;           // fp32 per 128-byte swizzled row
+constexpr int kSpinLimit = 4000000;   // mbarrier polls before a wait gives up
+
+__device__ __forceinline__ float leaky(float x) { return x > 0.0f ? x : kSlope * x; }
+
+// x = hi + lo with both parts representable in tf32 (10 explicit mantissa bits)
+__device__ __forceinline__ void split_tf32(float x, float &hi, float &lo)
+{
+    uint32_t h;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(x));
+    hi = __uint_as_float(h);
+    const float r = __fsub_rn(x, hi);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(r));
+    lo = __uint_as_float(h);
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Waits for the phase of the given parity to complete; false if it did not within the limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (int i = 0; i < kSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile of 128-byte rows, 128-byte swizzle: rows of
+// one 8-row group are 128 bytes apart, groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);         // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                               // leading byte offset (unused with this swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                               // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                               // 128-byte swizzle
+    return d;
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, one 128 x N x 8 tf32 step
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate)
+{
+    const uint32_t acc = accumulate ? 1u : 0u;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// Makes the mbarrier complete once every tcgen05.mma issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&x)[32])
+{
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) x[i] = __uint_as_float(r[i]);
+}
+
+// ------------------------------------------------------------------------------------------
+// conv1: gather of the kept values + Conv1d(1 -> 64, k3, s2) + leaky ReLU, written channels-last
+// as (hi, lo).  Grid (ceil(L1 / 64), K), 256 threads: thread = (position, group of 16 channels).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+ae5_conv1_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restrict__ idx, int64_t mu, int64_t L1,
+                 int64_t Lpad1, const float *__restrict__ w1, const float *__restrict__ b1, float *__restrict__ val,
+                 float *__restrict__ a_hi, float *__restrict__ a_lo)
+{
+    __shared__ float x[2 * 64 + 2];
+    __shared__ float w[64 * 3], b[64];
+    const int k = blockIdx.y;
+    const int64_t t0 = (int64_t)blockIdx.x * 64;
+    for (int i = threadIdx.x; i < 64 * 3; i += 256) w[i] = w1[i];
+    if (threadIdx.x < 64) b[threadIdx.x] = b1[threadIdx.x];
+    for (int i = threadIdx.x; i < 2 * 64 + 2; i += 256) {
+        const int64_t p = 2 * t0 + i;
+        float xv = 0.0f;
+        if (p < mu) {
+            xv = v[(int64_t)k * N + idx[p]];
+            val[(int64_t)k * mu + p] = xv;           // the two slots shared with the next CTA are written by
+        }                                            // both, with the same value
+        x[i] = xv;
+    }
+    __syncthreads();
+    const int tl = threadIdx.x >> 2, cg = threadIdx.x & 3;
+    const int64_t t = t0 + tl;
+    if (t >= L1) return;
+    const float x0 = x[2 * tl], x1 = x[2 * tl + 1], x2 = x[2 * tl + 2];
+    float *oh = a_hi + ((int64_t)k * Lpad1 + t) * 64 + cg * 16;
+    float *ol = a_lo + ((int64_t)k * Lpad1 + t) * 64 + cg * 16;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        float hi[4], lo[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int co = cg * 16 + q * 4 + j;
+            float acc = b[co];
+            acc = __fmaf_rn(w[co * 3 + 0], x0, acc);
+            acc = __fmaf_rn(w[co * 3 + 1], x1, acc);
+            acc = __fmaf_rn(w[co * 3 + 2], x2, acc);
+            split_tf32(leaky(acc), hi[j], lo[j]);
+        }
+        reinterpret_cast<float4 *>(oh)[q] = make_float4(hi[0], hi[1], hi[2], hi[3]);
+        reinterpret_cast<float4 *>(ol)[q] = make_float4(lo[0], lo[1], lo[2], lo[3]);
+    }
+}
+
+// Weights of a kernel-3 convolution w[co][ci][tau] -> GEMM operand W[co][tau C_in + ci] as (hi, lo).
+__global__ void ae5_prep_weights_kernel(const float *__restrict__ w, int cin, int cout, float *__restrict__ w_hi,
+                                        float *__restrict__ w_lo)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= cout * cin * 3) return;
+    const int co = i / (cin * 3), rem = i % (cin * 3), tau = rem / cin, ci = rem % cin;
+    float hi, lo;
+    split_tf32(w[(co * cin + ci) * 3 + tau], hi, lo);
+    w_hi[i] = hi;
+    w_lo[i] = lo;
+}
+
+// ------------------------------------------------------------------------------------------
+// Conv1d(CIN -> COUT, k3, s2) + leaky ReLU as a GEMM on the tensor cores.  Grid (ceil(L_out /
+// 128), K), 128 threads.  Thread 0 issues the TMA loads, thread 32 the MMAs, and all four warps
+// read the accumulator back (warp w owns TMEM lanes 32 w .. 32 w + 31 = rows of the tile).
+// The activation is addressed as rows of 2 CIN floats (a pair of positions): im2col row t is row
+// t followed by the first half of row t + 1.
+// FUSE_CODE: the layer is conv4; its output goes straight through conv5 (1x1, 64 -> 4, no
+// activation) and only the code is written.
+// Every wait has a limit; a CTA whose wait runs out records it and leaves without touching the
+// output (tensor memory is released on every path).
+// ------------------------------------------------------------------------------------------
+template <int CIN, int COUT>
+struct GemmShape {
+    static constexpr int kBlocks = 3 * CIN / kBlockK;
+    static constexpr int kABytes = kTileM * kBlockK * 4;       // one (hi or lo) activation tile of a k-block
+    static constexpr int kBBytes = COUT * kBlockK * 4;
+    static constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;
+    static constexpr int kStages = (200 * 1024) / kStageBytes < kBlocks ? (200 * 1024) / kStageBytes : kBlocks;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024;   // + slack to align the tiles to 1024 bytes
+};
+
+template <int CIN, int COUT, bool FUSE_CODE>
+__global__ void __launch_bounds__(128)
+ae5_conv_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
+                     const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
+                     const float *__restrict__ bias, int64_t L_out, int64_t Lpad_out, float *__restrict__ out_hi,
+                     float *__restrict__ out_lo, const float *__restrict__ w5, const float *__restrict__ b5,
+                     float *__restrict__ code, int32_t *errword)
+{
+    using S = GemmShape<CIN, COUT>;
+    extern __shared__ uint8_t dyn_smem[];
+    __shared__ __align__(8) uint64_t full_bar[S::kStages], empty_bar[S::kStages], accum_bar;
+    __shared__ uint32_t tmem_base_smem;
+    __shared__ int failed;
+    __shared__ float s_bias[COUT];
+    __shared__ float s_w5[FUSE_CODE ? 4 * 64 : 1], s_b5[4];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int node = blockIdx.y;
+    const int t0 = blockIdx.x * kTileM;
+    const uint32_t tiles = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+
+    for (int i = threadIdx.x; i < COUT; i += 128) s_bias[i] = bias[i];
+    if (FUSE_CODE) {
+        for (int i = threadIdx.x; i < 4 * 64; i += 128) s_w5[i] = w5[i];
+        if (threadIdx.x < 4) s_b5[threadIdx.x] = b5[threadIdx.x];
+    }
+    if (threadIdx.x == 0) {
+        failed = 0;
+        for (int s = 0; s < S::kStages; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), 1);
+            mbar_init(smem_u32(&empty_bar[s]), 1);
+        }
+        mbar_init(smem_u32(&accum_bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {                      // one warp allocates COUT columns of tensor memory (a power of two >= 32)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)),
+                     "r"((uint32_t)COUT)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_base_smem;
+
+    if (threadIdx.x == 0) {
+        // producer: one k-block (32 floats of the im2col row) of both operands, hi and lo, per stage
+        for (int kb = 0; kb < S::kBlocks; ++kb) {
+            const int s = kb % S::kStages;
+            if (kb >= S::kStages && !mbar_wait(smem_u32(&empty_bar[s]), ((kb / S::kStages) & 1) ^ 1)) {
+                atomicExch(&failed, 1);
+                break;
+            }
+            const uint32_t bar = smem_u32(&full_bar[s]);
+            const uint32_t st = tiles + (uint32_t)s * S::kStageBytes;
+            mbar_expect_tx(bar, S::kStageBytes);
+            const int c = kb * kBlockK;                       // column inside the 3 CIN wide im2col row
+            const int col = c < 2 * CIN ? c : c - 2 * CIN;
+            const int row = c < 2 * CIN ? t0 : t0 + 1;
+            tma_load_3d(st, &map_a_hi, bar, col, row, node);
+            tma_load_3d(st + S::kABytes, &map_a_lo, bar, col, row, node);
+            tma_load_2d(st + 2 * S::kABytes, &map_b_hi, bar, c, 0);
+            tma_load_2d(st + 2 * S::kABytes + S::kBBytes, &map_b_lo, bar, c, 0);
+        }
+    } else if (threadIdx.x == 32) {
+        // instruction descriptor: fp32 accumulator, tf32 x tf32, both operands K-major, N = COUT, M = 128
+        constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(COUT >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+        bool ok = true;
+        for (int kb = 0; kb < S::kBlocks && ok; ++kb) {
+            const int s = kb % S::kStages;
+            if (!mbar_wait(smem_u32(&full_bar[s]), (kb / S::kStages) & 1)) {
+                atomicExch(&failed, 1);
+                ok = false;
+                break;
+            }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t st = tiles + (uint32_t)s * S::kStageBytes;
+            const uint64_t a_hi = umma_desc(st), a_lo = umma_desc(st + S::kABytes);
+            const uint64_t b_hi = umma_desc(st + 2 * S::kABytes), b_lo = umma_desc(st + 2 * S::kABytes + S::kBBytes);
+#pragma unroll
+            for (int ks = 0; ks < kBlockK / 8; ++ks) {        // 8 tf32 = 32 bytes per step along K
+                const uint64_t adv = (uint64_t)(ks * 32 >> 4);
+                umma_tf32(tmem, a_hi + adv, b_hi + adv, idesc, kb > 0 || ks > 0);
+                umma_tf32(tmem, a_hi + adv, b_lo + adv, idesc, true);
+                umma_tf32(tmem, a_lo + adv, b_hi + adv, idesc, true);
+            }
+            umma_commit(smem_u32(&empty_bar[s]));             // the stage may be refilled once these have run
+        }
+        if (ok) umma_commit(smem_u32(&accum_bar));
+    }
+    __syncwarp();
+    // everyone: wait for the accumulator (or for the verdict that it will not come)
+    bool have = false;
+    if (lane == 0) {
+        for (int i = 0; i < kSpinLimit && !have; ++i) {
+            uint32_t done;
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(done)
+                : "r"(smem_u32(&accum_bar))
+                : "memory");
+            have = done != 0;
+            if (!have && *(volatile int *)&failed) break;
+        }
+    }
+    have = __shfl_sync(0xffffffffu, have ? 1 : 0, 0) != 0;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (have) {
+        const int64_t t = (int64_t)t0 + warp * 32 + lane;       // this thread's output position
+        const uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
+        float c4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+        for (int c0 = 0; c0 < COUT; c0 += 32) {
+            float x[32];
+            tmem_load32(trow + (uint32_t)c0, x);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) x[j] = leaky(__fadd_rn(x[j], s_bias[c0 + j]));
+            if (FUSE_CODE) {
+#pragma unroll
+                for (int o = 0; o < 4; ++o)
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) c4[o] = __fmaf_rn(s_w5[o * 64 + c0 + j], x[j], c4[o]);
+            } else if (t < L_out) {
+                float *oh = out_hi + ((int64_t)node * Lpad_out + t) * COUT + c0;
+                float *ol = out_lo + ((int64_t)node * Lpad_out + t) * COUT + c0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    float hi[4], lo[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) split_tf32(x[4 * q + j], hi[j], lo[j]);
+                    reinterpret_cast<float4 *>(oh)[q] = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                    reinterpret_cast<float4 *>(ol)[q] = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                }
+            }
+        }
+        if (FUSE_CODE && t < L_out)
+            reinterpret_cast<float4 *>(code)[(int64_t)node * L_out + t] =
+                make_float4(__fadd_rn(c4[0], s_b5[0]), __fadd_rn(c4[1], s_b5[1]), __fadd_rn(c4[2], s_b5[2]),
+                            __fadd_rn(c4[3], s_b5[3]));
+    } else if (threadIdx.x == 0) {
+        atomicExch(errword, 0x5EA5);                              // a wait ran out
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)COUT) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------
+// Decoder (one pass, fp32 pipes), channels-last.
+// ------------------------------------------------------------------------------------------
+// deconv1: ConvTranspose1d(4 -> 4, k3, stride 1, padding 1) + leaky ReLU on the mean code.
+__global__ void ae5_deconv1_kernel(const float *__restrict__ z, int64_t L4, const float *__restrict__ w,
+                                   const float *__restrict__ b, float *__restrict__ out)
+{
+    const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= L4) return;
+    float acc[4] = {b[0], b[1], b[2], b[3]};
+#pragma unroll
+    for (int tau = 0; tau < 3; ++tau) {
+        const int64_t j = s + 1 - tau;                            // y[s] += w[ci][co][tau] x[ci][j], s = j + tau - 1
+        if (j < 0 || j >= L4) continue;
+        const float4 x = reinterpret_cast<const float4 *>(z)[j];
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int ci = 0; ci < 4; ++ci)
+#pragma unroll
+            for (int co = 0; co < 4; ++co) acc[co] = __fmaf_rn(w[(ci * 4 + co) * 3 + tau], xs[ci], acc[co]);
+    }
+    reinterpret_cast<float4 *>(out)[s] = make_float4(leaky(acc[0]), leaky(acc[1]), leaky(acc[2]), leaky(acc[3]));
+}
+
+// ConvTranspose1d(CIN -> COUT, k3, s2, output padding) + leaky ReLU:
+//   y[2j]     = b + sum_ci w[ci][co][0] x[j][ci] + w[ci][co][2] x[j-1][ci]
+//   y[2j + 1] = b + sum_ci w[ci][co][1] x[j][ci]
+// CTA: TP input positions j0 .. j0 + TP - 1 -> outputs 2 j0 .. 2 j0 + 2 TP - 1; thread = (output
+// channel, slice of positions); weights and the input rows sit in shared memory.
+template <int CIN, int COUT, int TP>
+__global__ void __launch_bounds__(256)
+ae5_deconv_kernel(const float *__restrict__ x, int64_t L_in, int64_t L_out, const float *__restrict__ w,
+                  const float *__restrict__ b, float *__restrict__ y)
+{
+    extern __shared__ float dsm[];
+    float *sw = dsm;                          // [tau][ci][co]
+    float *sx = dsm + 3 * CIN * COUT;         // [TP + 1][CIN]: rows j0 - 1 .. j0 + TP - 1
+    const int64_t j0 = (int64_t)blockIdx.x * TP;
+    for (int i = threadIdx.x; i < 3 * CIN * COUT; i += 256) {
+        const int tau = i / (CIN * COUT), rem = i % (CIN * COUT), ci = rem / COUT, co = rem % COUT;
+        sw[i] = w[(ci * COUT + co) * 3 + tau];
+    }
+    for (int i = threadIdx.x; i < (TP + 1) * CIN; i += 256) {
+        const int64_t j = j0 - 1 + i / CIN;
+        sx[i] = j >= 0 && j < L_in ? x[j * CIN + i % CIN] : 0.0f;
+    }
+    __syncthreads();
+    constexpr int kSlices = 256 / COUT;       // threads along positions
+    const int co = threadIdx.x % COUT, sl = threadIdx.x / COUT;
+    const float bias = b[co];
+    for (int jl = sl; jl < TP; jl += kSlices) {
+        const int64_t j = j0 + jl;
+        if (2 * j >= L_out) break;
+        float even = bias, odd = bias;
+        const float *xj = sx + (jl + 1) * CIN, *xp = sx + jl * CIN;
+#pragma unroll 8
+        for (int ci = 0; ci < CIN; ++ci) {
+            const float a = xj[ci], p = xp[ci];
+            even = __fmaf_rn(sw[(0 * CIN + ci) * COUT + co], a, even);
+            even = __fmaf_rn(sw[(2 * CIN + ci) * COUT + co], p, even);
+            odd = __fmaf_rn(sw[(1 * CIN + ci) * COUT + co], a, odd);
+        }
+        y[(2 * j) * COUT + co] = leaky(even);
+        if (2 * j + 1 < L_out) y[(2 * j + 1) * COUT + co] = leaky(odd);
+    }
+}
+
+// Final Conv1d(32 -> 1, k1): the reconstruction of every kept slot.
+__global__ void ae5_final_kernel(const float *__restrict__ d5, int64_t mu, const float *__restrict__ w6,
+                                 const float *__restrict__ b6, float *__restrict__ recon)
+{
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= mu) return;
+    float acc = b6[0];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const float4 x = reinterpret_cast<const float4 *>(d5)[p * 8 + q];
+        acc = __fmaf_rn(w6[4 * q + 0], x.x, acc);
+        acc = __fmaf_rn(w6[4 * q + 1], x.y, acc);
+        acc = __fmaf_rn(w6[4 * q + 2], x.z, acc);
+        acc = __fmaf_rn(w6[4 * q + 3], x.w, acc);
+    }
+    recon[p] = acc;
+}
+
+inline unsigned blocks(int64_t n, int per) { return (unsigned)((n + per - 1) / per); }
+
+// cuTensorMapEncodeTiled, fetched through the runtime so that the library does not link the driver
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+cudaError_t encode_fn(EncodeTiledFn *out)
+{
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    const cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess) return e;
+    if (q != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    *out = reinterpret_cast<EncodeTiledFn>(fn);
+    return cudaSuccess;
+}
+
+// Activation [K][Lpad][C] (Lpad even) seen as [K][Lpad / 2][2 C]; box: 32 floats x 128 rows.
+bool make_act_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int C, int64_t Lpad, int K)
+{
+    const cuuint64_t dims[3] = {(cuuint64_t)(2 * C), (cuuint64_t)(Lpad / 2), (cuuint64_t)K};
+    const cuuint64_t strides[2] = {(cuuint64_t)(2 * C) * 4, (cuuint64_t)Lpad * C * 4};
+    const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileM, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// Weights [COUT][3 CIN]; box: 32 floats x COUT rows.
+bool make_weight_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int cin, int cout)
+{
+    const cuuint64_t dims[2] = {(cuuint64_t)(3 * cin), (cuuint64_t)cout};
+    const cuuint64_t strides[1] = {(cuuint64_t)(3 * cin) * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)cout};
+    const cuuint32_t es[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// g = 0, 1, 2: conv2, conv3, conv4 (input: the output of conv1 + g)
+template <int CIN, int COUT, bool FUSE>
+cudaError_t launch_gemm(Ctx &c, int g, int64_t L_out, int64_t Lpad_out, float *out_hi, float *out_lo)
+{
+    using S = GemmShape<CIN, COUT>;
+    Ae5 &a = *c.ae5;
+    auto kern = ae5_conv_gemm_kernel<CIN, COUT, FUSE>;
+    static bool configured = false;
+    if (!configured) {
+        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    kern<<<dim3(blocks(L_out, kTileM), c.K), 128, S::kSmemBytes, c.stream>>>(
+        a.map_act_hi[g], a.map_act_lo[g], a.map_w_hi[g], a.map_w_lo[g], c.params + a.off_b[g + 1], L_out, Lpad_out, out_hi,
+        out_lo, c.params + a.off_w[4], c.params + a.off_b[4], c.code, c.errword),
+        ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+template <int CIN, int COUT, int TP>
+cudaError_t launch_deconv(Ctx &c, const float *x, int64_t L_in, int64_t L_out, const float *w, const float *b, float *y)
+{
+    constexpr int smem = (3 * CIN * COUT + (TP + 1) * CIN) * 4;
+    auto kern = ae5_deconv_kernel<CIN, COUT, TP>;
+    static bool configured = false;
+    if (!configured) {
+        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    // one more input position than L_in covers the output-padding slot at the end
+    kern<<<blocks(L_in + 1, TP), 256, smem, c.stream>>>(x, L_in, L_out, w, b, y), ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+const int kAe5EncCh[5] = {1, 64, 128, 256, 64};
+const int kAe5DecCh[6] = {4, 4, 32, 64, 128, 32};
+
+int64_t ae5_param_count()
+{
+    int64_t n = 0;
+    for (int i = 0; i < 4; ++i) n += (int64_t)kAe5EncCh[i + 1] * kAe5EncCh[i] * 3 + kAe5EncCh[i + 1];
+    n += 4 * 64 + 4;
+    for (int i = 0; i < 5; ++i) n += (int64_t)kAe5DecCh[i] * kAe5DecCh[i + 1] * 3 + kAe5DecCh[i + 1];
+    return n + 32 + 1;
+}
+
+// Lengths after conv1..conv4; false when the input is too short.
+bool ae5_lengths(int64_t mu, int64_t (&len)[5])
+{
+    len[0] = mu;
+    for (int i = 0; i < 4; ++i) {
+        if (len[i] < 3) return false;
+        len[i + 1] = (len[i] - 3) / 2 + 1;
+    }
+    return true;
+}
+
+void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used)
+{
+    ae5_lengths(mu, a.len);
+    size_t at = *used;
+    auto take = [&](size_t floats) {
+        at = (at + 1023) / 1024 * 1024;                     // TMA sources: generously aligned
+        float *p = base ? reinterpret_cast<float *>(base + at) : nullptr;
+        at += floats * sizeof(float);
+        return p;
+    };
+    for (int l = 0; l < 3; ++l) {                           // outputs of conv1..conv3
+        a.lpad[l] = (a.len[l + 1] + 1) / 2 * 2;
+        const size_t n = (size_t)K * a.lpad[l] * kAe5EncCh[l + 1];
+        a.act_hi[l] = take(n);
+        a.act_lo[l] = take(n);
+    }
+    for (int l = 0; l < 3; ++l) {                           // GEMM weights of conv2..conv4
+        const size_t n = (size_t)kAe5EncCh[l + 2] * kAe5EncCh[l + 1] * 3;
+        a.w_hi[l] = take(n);
+        a.w_lo[l] = take(n);
+    }
+    a.d[0] = take((size_t)a.len[4] * 4);
+    a.d[1] = take((size_t)a.len[3] * 32);
+    a.d[2] = take((size_t)a.len[2] * 64);
+    a.d[3] = take((size_t)a.len[1] * 128);
+    a.d[4] = take((size_t)a.len[0] * 32);
+    *used = at;
+    // offsets of the layers' parameters inside the flat vector (encoder, then decoder)
+    int64_t pos = 0;
+    for (int i = 0; i < 4; ++i) {
+        a.off_w[i] = pos; pos += (int64_t)kAe5EncCh[i + 1] * kAe5EncCh[i] * 3;
+        a.off_b[i] = pos; pos += kAe5EncCh[i + 1];
+    }
+    a.off_w[4] = pos; pos += 4 * 64;
+    a.off_b[4] = pos; pos += 4;
+    for (int i = 0; i < 5; ++i) {
+        a.off_dw[i] = pos; pos += (int64_t)kAe5DecCh[i] * kAe5DecCh[i + 1] * 3;
+        a.off_db[i] = pos; pos += kAe5DecCh[i + 1];
+    }
+    a.off_dw[5] = pos; pos += 32;
+    a.off_db[5] = pos;
+}
+
+cudaError_t ae5_make_maps(Ctx &c)
+{
+    Ae5 &a = *c.ae5;
+    EncodeTiledFn enc = nullptr;
+    const cudaError_t e = encode_fn(&enc);
+    if (e != cudaSuccess) return e;
+    bool ok = true;
+    for (int l = 0; l < 3; ++l) {
+        ok = ok && make_act_map(enc, &a.map_act_hi[l], a.act_hi[l], kAe5EncCh[l + 1], a.lpad[l], c.K);
+        ok = ok && make_act_map(enc, &a.map_act_lo[l], a.act_lo[l], kAe5EncCh[l + 1], a.lpad[l], c.K);
+        ok = ok && make_weight_map(enc, &a.map_w_hi[l], a.w_hi[l], kAe5EncCh[l + 1], kAe5EncCh[l + 2]);
+        ok = ok && make_weight_map(enc, &a.map_w_lo[l], a.w_lo[l], kAe5EncCh[l + 1], kAe5EncCh[l + 2]);
+    }
+    return ok ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+// Stage 4 for the full-size autoencoder: gather, conv1..conv5 for every node; the codes are
+// [K][L4][4] (position-major).
+cudaError_t launch_ae5_encode(Ctx &c)
+{
+    Ae5 &a = *c.ae5;
+    const float *P = c.params;
+    if (!a.weights_ready) {
+        for (int l = 0; l < 3; ++l) {
+            const int cin = kAe5EncCh[l + 1], cout = kAe5EncCh[l + 2];
+            ae5_prep_weights_kernel<<<blocks((int64_t)cin * cout * 3, 256), 256, 0, c.stream>>>(P + a.off_w[l + 1], cin, cout,
+                                                                                               a.w_hi[l], a.w_lo[l]),
+                ++g_kernel_launches;
+        }
+        a.weights_ready = true;
+    }
+    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.mu, a.len[1], a.lpad[0],
+                                                                            P + a.off_w[0], P + a.off_b[0], c.val, a.act_hi[0],
+                                                                            a.act_lo[0]),
+        ++g_kernel_launches;
+    c.val_valid = true;
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = launch_gemm<64, 128, false>(c, 0, a.len[2], a.lpad[1], a.act_hi[1], a.act_lo[1]);
+    if (e == cudaSuccess) e = launch_gemm<128, 256, false>(c, 1, a.len[3], a.lpad[2], a.act_hi[2], a.act_lo[2]);
+    if (e == cudaSuccess) e = launch_gemm<256, 64, true>(c, 2, a.len[4], 0, nullptr, nullptr);
+    return e;
+}
+
+// Stage 5 up to the reconstruction: the decoder on the mean code; c.recon gets the mu values.
+cudaError_t launch_ae5_decode(Ctx &c)
+{
+    Ae5 &a = *c.ae5;
+    const float *P = c.params;
+    ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d[0]),
+        ++g_kernel_launches;
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = launch_deconv<4, 32, 64>(c, a.d[0], a.len[4], a.len[3], P + a.off_dw[1], P + a.off_db[1], a.d[1]);
+    if (e == cudaSuccess) e = launch_deconv<32, 64, 32>(c, a.d[1], a.len[3], a.len[2], P + a.off_dw[2], P + a.off_db[2], a.d[2]);
+    if (e == cudaSuccess) e = launch_deconv<64, 128, 64>(c, a.d[2], a.len[2], a.len[1], P + a.off_dw[3], P + a.off_db[3], a.d[3]);
+    if (e == cudaSuccess) e = launch_deconv<128, 32, 64>(c, a.d[3], a.len[1], a.len[0], P + a.off_dw[4], P + a.off_db[4], a.d[4]);
+    if (e != cudaSuccess) return e;
+    ae5_final_kernel<<<blocks(c.mu, 256), 256, 0, c.stream>>>(a.d[4], c.mu, P + a.off_dw[5], P + a.off_db[5], c.recon),
+        ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+}  // namespace lgc

@@ -59,7 +59,8 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
     if (cfg->num_layers < 1 || !cfg->layer_numel) return fail(LGC_ERR_INVALID_ARG, "num_layers < 1 or layer_numel is NULL");
     if (cfg->density_ppm < 1 || cfg->density_ppm > 1000000) return fail(LGC_ERR_INVALID_ARG, "density_ppm must be in [1, 10^6]");
     if (cfg->variant != LGC_VARIANT_RAR && cfg->variant != LGC_VARIANT_PS) return fail(LGC_ERR_INVALID_ARG, "unknown variant");
-    if (cfg->ae_kind != LGC_AE_CONV2 && cfg->ae_kind != LGC_AE_IDENTITY) return fail(LGC_ERR_INVALID_ARG, "unknown ae_kind");
+    if (cfg->ae_kind != LGC_AE_CONV2 && cfg->ae_kind != LGC_AE_IDENTITY && cfg->ae_kind != LGC_AE_CONV5)
+        return fail(LGC_ERR_INVALID_ARG, "unknown ae_kind");
     if (!(cfg->momentum >= 0.0f && cfg->momentum < 1.0f)) return fail(LGC_ERR_INVALID_ARG, "momentum must be in [0, 1)");
     if (cfg->variant == LGC_VARIANT_PS && cfg->innovation_permille > 1000) return fail(LGC_ERR_INVALID_ARG, "innovation_permille > 1000");
     p.K = cfg->num_nodes;
@@ -101,6 +102,13 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
         p.Pdec = c2 * c1 * 3 + c1 + c1 * 3 + 1 + (cfg->variant == LGC_VARIANT_PS ? 3 : 0);
         p.P = p.Penc + p.Pdec * p.S;
         p.code_len = c2 * p.L2;
+    } else if (cfg->ae_kind == LGC_AE_CONV5) {
+        if (cfg->variant != LGC_VARIANT_RAR) return fail(LGC_ERR_UNSUPPORTED, "the full-size autoencoder is built for ring-allreduce only");
+        int64_t len[5];
+        if (!ae5_lengths(p.mu, len) || len[4] < 1) return fail(LGC_ERR_UNSUPPORTED, "mu is too short for four stride-2 convolutions (needs mu >= 31)");
+        p.P = ae5_param_count();
+        p.Penc = p.Pdec = 0;
+        p.code_len = 4 * len[4];
     } else {
         p.Penc = p.Pdec = p.P = 0;
         p.code_len = p.mu;
@@ -219,10 +227,11 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
 {
     const bool ps = cfg.variant == LGC_VARIANT_PS;
     const bool conv = cfg.ae_kind == LGC_AE_CONV2;
+    const bool conv5 = cfg.ae_kind == LGC_AE_CONV5;
     c.errword = cv.take<int32_t>(4);
     c.idx = cv.take<int32_t>((size_t)p.S * p.mu);
     c.val = cv.take<float>((size_t)p.K * p.mu);
-    c.code = conv ? cv.take<float>((size_t)p.K * p.code_len) : nullptr;
+    c.code = conv || conv5 ? cv.take<float>((size_t)p.K * p.code_len) : nullptr;
     c.combined = cv.take<float>((size_t)p.code_len);
     c.recon = cv.take<float>((size_t)p.S * p.mu);
     c.slot_layer = cv.take<int32_t>((size_t)p.mu);
@@ -244,6 +253,10 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
         c.t_dz = cv.take<float>(c2 * p.L2);
         c.t_loss_blocks = (int)((p.mu + 127) / 128);
         c.t_loss_part = cv.take<double>((size_t)c.t_loss_blocks);
+    }
+    if (conv5) {
+        if (!c.ae5) c.ae5.reset(new Ae5());
+        ae5_carve(*c.ae5, p.K, p.mu, cv.base, &cv.used);
     }
     cv.take<char>(0);
 }
@@ -360,6 +373,7 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     koff32[p.L] = (int32_t)p.mu;
     if (e == cudaSuccess) e = upload(c->slot_layer, slot_layer, s);
     if (e == cudaSuccess) e = upload(c->koff_dev, koff32, s);
+    if (e == cudaSuccess && cfg->ae_kind == LGC_AE_CONV5) e = ae5_make_maps(*c);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
         delete c;
@@ -539,6 +553,7 @@ lgc_status lgc_set_ae_params(lgc_ctx *c, const float *src, size_t count)
     if ((int64_t)count != c->P) return fail(c, LGC_ERR_INVALID_ARG, "parameter count does not match the configuration");
     if (count == 0) return LGC_OK;
     cudaError_t e = cudaMemcpyAsync(c->params, src, count * sizeof(float), cudaMemcpyDefault, c->stream);
+    if (c->ae5) c->ae5->weights_ready = false;
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
     return e == cudaSuccess ? LGC_OK : cuda_fail(c, e, "lgc_set_ae_params");
 }

@@ -442,6 +442,7 @@ cudaError_t launch_gather(Ctx &c)
 cudaError_t launch_encode(Ctx &c)
 {
     if (c.cfg.ae_kind == LGC_AE_IDENTITY) return cudaSuccess;   // the code is the kept values themselves
+    if (c.cfg.ae_kind == LGC_AE_CONV5) return launch_ae5_encode(c);
     if (c.S == 1 && c.K <= 256) {   // ring-allreduce: gather + encode + mean in one launch
         int tt = 256 / c.K;
         if (tt > 64) tt = 64;
@@ -501,15 +502,18 @@ static cudaError_t launch_scatter(Ctx &c, const float *values, float *update)
 }
 
 // Ring-allreduce: the whole of stage 5 (or the phase-two sparse mean) in one pass over the update.
-static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update)
+// mode 0: decode the mean code; 1: the values are in `src` (default: the mean code of the identity
+// autoencoder); 2: mean over nodes of the kept values.
+static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update, const float *src = nullptr)
 {
     const float *dec = c.params + c.Penc;
+    const float *z1 = src ? src : c.combined;
     if (update == c.cleared_update) {
         // lgc_topk's finishing launch has cleared the buffer: only the kept entries are written
         const unsigned sgrid = blocks_for(c.mu, kAeThreads);
         if (mode == 1) {
             sparse_scatter_kernel<3, 2, 1><<<sgrid, kAeThreads, 0, c.stream>>>(
-                c.combined, c.val, c.idx, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
+                z1, c.val, c.idx, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
         } else if (mode == 2) {
             sparse_scatter_kernel<3, 2, 2><<<sgrid, kAeThreads, 0, c.stream>>>(
                 c.combined, c.val, c.idx, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
@@ -528,7 +532,7 @@ static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update)
     const unsigned grid = blocks_for(c.N, kDenseTile);
     if (mode == 1) {
         dense_scatter_kernel<3, 2, 1><<<grid, kDenseThreads, 0, c.stream>>>(
-            c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
+            z1, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
     } else if (mode == 2) {
         dense_scatter_kernel<3, 2, 2><<<grid, kDenseThreads, 0, c.stream>>>(
             c.combined, c.val, c.idx, c.tile_lo, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
@@ -549,6 +553,10 @@ static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update)
 cudaError_t launch_decode_scatter(Ctx &c, float *update)
 {
     const bool ps = c.cfg.variant == LGC_VARIANT_PS;
+    if (!ps && c.cfg.ae_kind == LGC_AE_CONV5) {
+        const cudaError_t e = launch_ae5_decode(c);
+        return e != cudaSuccess ? e : launch_dense_scatter(c, 1, update, c.recon);
+    }
     if (!ps) return launch_dense_scatter(c, c.cfg.ae_kind == LGC_AE_IDENTITY ? 1 : 0, update);
     if (c.cfg.ae_kind == LGC_AE_IDENTITY) {
         identity_ps_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.combined, c.inn, c.mu, c.recon), ++g_kernel_launches;

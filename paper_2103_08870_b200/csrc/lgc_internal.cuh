@@ -2,9 +2,11 @@
 // space carve-up, and one launcher prototype per kernel family.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <memory>
 #include <string>
 #include <vector>
 
@@ -82,6 +84,19 @@ inline int64_t select_compact_capacity(int64_t n)
     return c < n ? c : n;
 }
 
+// Work space and tables of the full-size autoencoder (LGC_AE_CONV5; Section IV-C).
+struct Ae5 {
+    int64_t len[5] = {0, 0, 0, 0, 0};   // mu and the lengths after conv1..conv4
+    int64_t lpad[3] = {0, 0, 0};        // positions allocated per node for the outputs of conv1..conv3 (even)
+    float *act_hi[3] = {}, *act_lo[3] = {};   // [K][lpad][C] outputs of conv1..conv3, channels-last, split into two tf32 parts
+    float *w_hi[3] = {}, *w_lo[3] = {};       // [C_out][3 C_in] GEMM weights of conv2..conv4, split likewise
+    float *d[5] = {};                   // decoder activations: [L4][4], [L3][32], [L2][64], [L1][128], [mu][32]
+    int64_t off_w[5] = {}, off_b[5] = {};     // offsets of the encoder layers' weights / biases in the parameter vector
+    int64_t off_dw[6] = {}, off_db[6] = {};   // the same for the decoder's six layers
+    CUtensorMap map_act_hi[3], map_act_lo[3], map_w_hi[3], map_w_lo[3];
+    bool weights_ready = false;         // w_hi / w_lo match the parameter vector
+};
+
 struct Ctx {
     lgc_config cfg{};
     cudaStream_t stream = nullptr;
@@ -108,6 +123,7 @@ struct Ctx {
     int32_t *tile_lo = nullptr;    // [ceil(N / 4096) + 1] first kept slot at or after each 4096-entry tile (ring-allreduce)
     int32_t *errword = nullptr;    // device check record
     SelectTables sel_v, sel_inn;
+    std::unique_ptr<Ae5> ae5;      // full-size autoencoder only
     // training work space
     float *t_h = nullptr;          // [K][c1][L1] relu(conv1)
     float *t_d = nullptr;          // [c1][L1]    relu(convT1)
@@ -158,5 +174,12 @@ cudaError_t launch_combine_ps(Ctx &c, int common_node);
 cudaError_t launch_decode_scatter(Ctx &c, float *update);
 cudaError_t launch_topk_scatter(Ctx &c, float *update);
 cudaError_t launch_train_step(Ctx &c, float *loss_out);
+// full-size autoencoder (lgc_ae5.cu)
+int64_t ae5_param_count();
+bool ae5_lengths(int64_t mu, int64_t (&len)[5]);
+void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used);   // base may be null (sizes only)
+cudaError_t ae5_make_maps(Ctx &c);
+cudaError_t launch_ae5_encode(Ctx &c);
+cudaError_t launch_ae5_decode(Ctx &c);
 
 }  // namespace lgc

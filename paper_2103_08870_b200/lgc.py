@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "liblgc.so")
 
 LGC_OK = 0
 VARIANT_RAR, VARIANT_PS = 0, 1
-AE_CONV2, AE_IDENTITY = 0, 1
+AE_CONV2, AE_IDENTITY, AE_CONV5 = 0, 1, 2
 
 EXPORTS = (
     "lgc_workspace_bytes", "lgc_init", "lgc_destroy", "lgc_accumulate", "lgc_topk", "lgc_encode",
@@ -134,7 +134,7 @@ class LGC:
             num_nodes=num_nodes, num_layers=len(layer_numel), layer_numel=self._numel,
             density_ppm=density_ppm, innovation_permille=innovation_permille, momentum=momentum,
             variant={"rar": VARIANT_RAR, "ps": VARIANT_PS}[variant],
-            ae_kind={"conv2": AE_CONV2, "identity": AE_IDENTITY}[ae_kind], ae_c1=c1, ae_c2=c2,
+            ae_kind={"conv2": AE_CONV2, "identity": AE_IDENTITY, "conv5": AE_CONV5}[ae_kind], ae_c1=c1, ae_c2=c2,
             adam_lr=lr, adam_beta1=beta1, adam_beta2=beta2, adam_eps=eps,
             stream=C.c_void_p(self.stream.cuda_stream))
         self.variant, self.ae_kind, self.K, self.c1, self.c2 = variant, ae_kind, num_nodes, c1, c2
@@ -156,6 +156,11 @@ class LGC:
         self.k_l = [kc[i] for i in range(self.L)]
         self.S = self.K if variant == "ps" else 1
         self.code_len = self.mu if ae_kind == "identity" else c2 * self.L2
+        if ae_kind == "conv5":          # four stride-2 convolutions, four code channels, stored [L4][4]
+            n = self.mu
+            for _ in range(4):
+                n = (n - 3) // 2 + 1
+            self.L4, self.code_len = n, 4 * n
 
     # -- plumbing -----------------------------------------------------------------------------
     def _ok(self, status: int, where: str) -> None:

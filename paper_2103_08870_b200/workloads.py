@@ -333,6 +333,39 @@ def ae_init_params(c1: int, c2: int, variant: str, num_nodes: int, seed: int = D
     return torch.cat(parts)
 
 
+def ae5_param_shapes() -> List[Tuple[str, Tuple[int, ...], int]]:
+    """(name, shape, fan_in) of the full-size autoencoder's tensors (Section IV-C: encoder filters
+    64/128/256/64 of 3 taps and 4 of 1 tap; decoder filters 4/32/64/128/32 of 3 taps and one 1-tap
+    filter), in the order of the flat parameter vector.  Convolutions: w[co][ci][tap]; transposed
+    convolutions: w[ci][co][tap]."""
+    enc_ch, dec_ch = [1, 64, 128, 256, 64], [4, 4, 32, 64, 128, 32]
+    out = []
+    for i in range(4):
+        fan = 3 * enc_ch[i]
+        out += [(f"enc.w{i + 1}", (enc_ch[i + 1], enc_ch[i], 3), fan), (f"enc.b{i + 1}", (enc_ch[i + 1],), fan)]
+    out += [("enc.w5", (4, 64, 1), 64), ("enc.b5", (4,), 64)]
+    for i in range(5):
+        fan = 3 * dec_ch[i]
+        out += [(f"dec.w{i + 1}", (dec_ch[i], dec_ch[i + 1], 3), fan), (f"dec.b{i + 1}", (dec_ch[i + 1],), fan)]
+    out += [("dec.w6", (1, 32, 1), 32), ("dec.b6", (1,), 32)]
+    return out
+
+
+def ae5_init_params(seed: int = DEFAULT_SEED) -> torch.Tensor:
+    """U(-1/sqrt(fan_in), +1/sqrt(fan_in)) for every tensor of the full-size autoencoder; flat
+    fp32 CPU tensor."""
+    key = stream_key(seed, 1, STREAM_AE)
+    parts = []
+    ctr = 0
+    for _, shape, fan in ae5_param_shapes():
+        n = math.prod(shape)
+        c = torch.arange(ctr, ctr + n, dtype=torch.int64)
+        u = _uniform23(_lsr(hash_counters(key, c), 41))
+        parts.append(((2.0 * u - 1.0) * (1.0 / math.sqrt(fan))).to(torch.float32))
+        ctr += n
+    return torch.cat(parts)
+
+
 # --------------------------------------------------------------------------------------
 # the five workload configurations
 # --------------------------------------------------------------------------------------

@@ -136,6 +136,18 @@ def test_layer_of_several_groups_with_ties(levels, first_from_data):
     assert from_data[0] == first_from_data
 
 
+@pytest.mark.parametrize("numel, K", [([300_000, 5000, 120_000], 2), ([2_000_000, 700_000, 300_001], 3)])
+def test_full_size_autoencoder(numel, K):
+    # the autoencoder of Section IV-C (filters 64/128/256/64/4 and 4/32/64/128/32 + 1x1): mu = 425
+    # (every GEMM tile ragged) and mu = 3000 (several tiles per layer and node, ragged tails)
+    ora, gpu = make_pair(numel, K, ae_kind="conv5")
+    src = W.GradientSource(W.LayerTable("ae5", numel, [1 + i for i in range(len(numel))]), K, seed=21)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t in range(3):
+        g = src.step(t)
+        compare_step(ora, gpu, g, g.cuda(), t % K, upd)
+
+
 def test_dense_selection_uses_the_global_compact_arrays():
     # k = 40,000 of 2,000,000: more candidates than the finishing CTA keeps in shared memory
     numel = [2_000_000]
