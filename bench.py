@@ -113,12 +113,13 @@ def oracle_throughput(w: W.Workload, sample_steps: int, host_grads=None):
     """The oracle, as it stands, on `sample_steps` whole steps of the workload (host cores).
     `host_grads`: gradient batches (numpy [K][N]) to cycle through; generated on the CPU if absent."""
     from oracle import OracleLGC
-    params = W.ae_init_params(w.ae_c1, w.ae_c2, w.variant, w.num_nodes, w.seed).numpy()
+    params = w.init_params().numpy()
     if host_grads is None:
         src = W.GradientSource(w.table, w.num_nodes, seed=w.seed)
         host_grads = [src.step(t).numpy() for t in range(min(GRAD_SETS, sample_steps))]
     ora = OracleLGC(w.table.numel, w.num_nodes, density_ppm=w.density_ppm, momentum=w.momentum, variant=w.variant,
-                    c1=w.ae_c1, c2=w.ae_c2, params=params, innovation_permille=w.innovation_permille)
+                    ae_kind=w.ae_kind, c1=w.ae_c1, c2=w.ae_c2, params=params,
+                    innovation_permille=w.innovation_permille)
     times = []
     for t in range(sample_steps):
         g = host_grads[t % len(host_grads)]
@@ -150,7 +151,8 @@ def run_reference(args, w: W.Workload):
 
 def workload_config(w: W.Workload):
     return {"workload": f"{w.name}: {len(w.table.numel)} tensors, N={w.table.total}, K={w.num_nodes} nodes per GPU, "
-                        f"density {w.density_ppm} ppm, {w.variant}, AE {w.ae_c1}/{w.ae_c2}",
+                        f"density {w.density_ppm} ppm, {w.variant}, AE "
+                        + ("64/128/256/64/4 (full size)" if w.ae_kind == "conv5" else f"{w.ae_c1}/{w.ae_c2}"),
             "l2": f"inputs larger than L2: {w.num_nodes * w.table.total * 20 / 1e6:.0f} MB streamed per step, "
                   f"{GRAD_SETS} gradient batches cycled"}
 
@@ -185,8 +187,8 @@ def run_ours(args, w: W.Workload):
 
     K, N = w.num_nodes, w.table.total
     gpu = lgc.LGC(w.table.numel, K, density_ppm=w.density_ppm, momentum=w.momentum, variant=w.variant,
-                  c1=w.ae_c1, c2=w.ae_c2, innovation_permille=w.innovation_permille, device=dev)
-    gpu.set_ae_params(W.ae_init_params(w.ae_c1, w.ae_c2, w.variant, K, w.seed))
+                  ae_kind=w.ae_kind, c1=w.ae_c1, c2=w.ae_c2, innovation_permille=w.innovation_permille, device=dev)
+    gpu.set_ae_params(w.init_params())
     src = W.GradientSource(w.table, K, seed=w.seed + rank, device=dev)
     grads = [src.step(t) for t in range(GRAD_SETS)]
     update = torch.empty(N, dtype=torch.float32, device=dev)

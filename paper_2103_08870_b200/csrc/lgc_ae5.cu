@@ -188,42 +188,79 @@ __global__ void ae5_prep_weights_kernel(const float *__restrict__ w, int cin, in
     w_lo[i] = lo;
 }
 
+// Weights of a kernel-3 stride-2 transposed convolution w[ci][co][tau] -> GEMM operand
+// W[n][k], n in [0, 2 C_out), k in [0, 2 C_in), as (hi, lo): the first C_out rows make the even
+// output position (tap 2 on the previous input position, tap 0 on the current one), the others
+// the odd position (tap 1 on the current one).
+__global__ void ae5_prep_deconv_weights_kernel(const float *__restrict__ w, int cin, int cout, float *__restrict__ w_hi,
+                                               float *__restrict__ w_lo)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 4 * cin * cout) return;
+    const int n = i / (2 * cin), k = i % (2 * cin);
+    const int ci = k < cin ? k : k - cin;
+    float x = 0.0f;
+    if (n < cout) x = w[(ci * cout + n) * 3 + (k < cin ? 2 : 0)];
+    else if (k >= cin) x = w[(ci * cout + (n - cout)) * 3 + 1];
+    float hi, lo;
+    split_tf32(x, hi, lo);
+    w_hi[i] = hi;
+    w_lo[i] = lo;
+}
+
 // ------------------------------------------------------------------------------------------
-// Conv1d(CIN -> COUT, k3, s2) + leaky ReLU as a GEMM on the tensor cores.  Grid (ceil(L_out /
-// 128), K), 128 threads.  Thread 0 issues the TMA loads, thread 32 the MMAs, and all four warps
-// read the accumulator back (warp w owns TMEM lanes 32 w .. 32 w + 31 = rows of the tile).
-// The activation is addressed as rows of 2 CIN floats (a pair of positions): im2col row t is row
-// t followed by the first half of row t + 1.
-// FUSE_CODE: the layer is conv4; its output goes straight through conv5 (1x1, 64 -> 4, no
-// activation) and only the code is written.
+// The wide layers as GEMMs on the tensor cores.  Grid (ceil(rows / 128), nodes), 128 threads.
+// Thread 0 issues the TMA loads, thread 32 the MMAs, and all four warps read the accumulator
+// back (warp w owns TMEM lanes 32 w .. 32 w + 31 = rows of the tile).
+//
+// kConv / kConvCode: Conv1d(CIN -> COUT, k3, s2) + leaky ReLU.  Row t of the GEMM is output
+//   position t; its K = 3 CIN operands are the activation floats [2t CIN, (2t + 3) CIN).  The
+//   activation is addressed as rows of 2 CIN floats (a pair of positions): row t followed by the
+//   first half of row t + 1.  kConvCode is conv4: its output goes straight through conv5 (1x1,
+//   64 -> 4, no activation) and only the code is written.
+// kDeconv / kDeconvFinal: ConvTranspose1d(CIN -> COUT, k3, s2) + leaky ReLU.  Row j of the GEMM
+//   makes output positions 2j and 2j + 1 (N = 2 COUT columns: even position, then odd) from the
+//   K = 2 CIN floats of input positions j - 1 and j:
+//       y[2j]     = b + sum_ci w[ci][co][2] x[j-1][ci] + w[ci][co][0] x[j][ci]
+//       y[2j + 1] = b + sum_ci w[ci][co][1] x[j][ci]
+//   (input rows -1 and L_in read as zeros).  kDeconvFinal is deconv5: its output goes through
+//   the final 1x1 convolution (32 -> 1) and only the reconstruction is written.
+// Outputs that feed another GEMM are written channels-last as two tf32 parts.
 // Every wait has a limit; a CTA whose wait runs out records it and leaves without touching the
 // output (tensor memory is released on every path).
 // ------------------------------------------------------------------------------------------
-template <int CIN, int COUT>
+enum GemmMode { kConv = 0, kConvCode = 1, kDeconv = 2, kDeconvFinal = 3 };
+
+template <int MODE, int CIN, int COUT>
 struct GemmShape {
-    static constexpr int kBlocks = 3 * CIN / kBlockK;
-    static constexpr int kABytes = kTileM * kBlockK * 4;       // one (hi or lo) activation tile of a k-block
-    static constexpr int kBBytes = COUT * kBlockK * 4;
+    static constexpr bool kIsConv = MODE == kConv || MODE == kConvCode;
+    static constexpr int kK = kIsConv ? 3 * CIN : 2 * CIN;      // operands per row
+    static constexpr int kN = kIsConv ? COUT : 2 * COUT;        // accumulator columns
+    static constexpr int kBlocks = kK / kBlockK;
+    static constexpr int kABytes = kTileM * kBlockK * 4;        // one (hi or lo) activation tile of a k-block
+    static constexpr int kBBytes = kN * kBlockK * 4;
     static constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;
     static constexpr int kStages = (200 * 1024) / kStageBytes < kBlocks ? (200 * 1024) / kStageBytes : kBlocks;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024;   // + slack to align the tiles to 1024 bytes
+    static_assert(kN >= 32 && kN <= 256 && (kN & (kN - 1)) == 0, "accumulator columns: a power of two in [32, 256]");
 };
 
-template <int CIN, int COUT, bool FUSE_CODE>
+template <int MODE, int CIN, int COUT>
 __global__ void __launch_bounds__(128)
-ae5_conv_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
-                     const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
-                     const float *__restrict__ bias, int64_t L_out, int64_t Lpad_out, float *__restrict__ out_hi,
-                     float *__restrict__ out_lo, const float *__restrict__ w5, const float *__restrict__ b5,
-                     float *__restrict__ code, int32_t *errword)
+ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
+                const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
+                const float *__restrict__ bias, int64_t L_out, int64_t Lpad_out, float *__restrict__ out_hi,
+                float *__restrict__ out_lo, const float *__restrict__ w_last, const float *__restrict__ b_last,
+                float *__restrict__ out_last, int32_t *errword)
 {
-    using S = GemmShape<CIN, COUT>;
+    using S = GemmShape<MODE, CIN, COUT>;
+    constexpr int N = S::kN;
     extern __shared__ uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t full_bar[S::kStages], empty_bar[S::kStages], accum_bar;
     __shared__ uint32_t tmem_base_smem;
     __shared__ int failed;
     __shared__ float s_bias[COUT];
-    __shared__ float s_w5[FUSE_CODE ? 4 * 64 : 1], s_b5[4];
+    __shared__ float s_wl[MODE == kConvCode ? 4 * 64 : 32], s_bl[4];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int node = blockIdx.y;
@@ -231,9 +268,13 @@ ae5_conv_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_
     const uint32_t tiles = (smem_u32(dyn_smem) + 1023u) & ~1023u;
 
     for (int i = threadIdx.x; i < COUT; i += 128) s_bias[i] = bias[i];
-    if (FUSE_CODE) {
-        for (int i = threadIdx.x; i < 4 * 64; i += 128) s_w5[i] = w5[i];
-        if (threadIdx.x < 4) s_b5[threadIdx.x] = b5[threadIdx.x];
+    if (MODE == kConvCode) {
+        for (int i = threadIdx.x; i < 4 * 64; i += 128) s_wl[i] = w_last[i];
+        if (threadIdx.x < 4) s_bl[threadIdx.x] = b_last[threadIdx.x];
+    }
+    if (MODE == kDeconvFinal) {
+        if (threadIdx.x < 32) s_wl[threadIdx.x] = w_last[threadIdx.x];
+        if (threadIdx.x == 0) s_bl[0] = b_last[0];
     }
     if (threadIdx.x == 0) {
         failed = 0;
@@ -244,9 +285,9 @@ ae5_conv_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_
         mbar_init(smem_u32(&accum_bar), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {                      // one warp allocates COUT columns of tensor memory (a power of two >= 32)
+    if (warp == 1) {                      // one warp allocates N columns of tensor memory
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)),
-                     "r"((uint32_t)COUT)
+                     "r"((uint32_t)N)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -256,7 +297,7 @@ ae5_conv_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_
     const uint32_t tmem = tmem_base_smem;
 
     if (threadIdx.x == 0) {
-        // producer: one k-block (32 floats of the im2col row) of both operands, hi and lo, per stage
+        // producer: one k-block (32 floats of the operand row) of both operands, hi and lo, per stage
         for (int kb = 0; kb < S::kBlocks; ++kb) {
             const int s = kb % S::kStages;
             if (kb >= S::kStages && !mbar_wait(smem_u32(&empty_bar[s]), ((kb / S::kStages) & 1) ^ 1)) {
@@ -266,17 +307,23 @@ ae5_conv_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_
             const uint32_t bar = smem_u32(&full_bar[s]);
             const uint32_t st = tiles + (uint32_t)s * S::kStageBytes;
             mbar_expect_tx(bar, S::kStageBytes);
-            const int c = kb * kBlockK;                       // column inside the 3 CIN wide im2col row
-            const int col = c < 2 * CIN ? c : c - 2 * CIN;
-            const int row = c < 2 * CIN ? t0 : t0 + 1;
+            const int c = kb * kBlockK;                       // column inside the operand row
+            int col, row;
+            if (S::kIsConv) {                                 // activation rows hold a pair of positions
+                col = c < 2 * CIN ? c : c - 2 * CIN;
+                row = c < 2 * CIN ? t0 : t0 + 1;
+            } else {                                          // activation rows hold one position: j - 1, then j
+                col = c < CIN ? c : c - CIN;
+                row = c < CIN ? t0 - 1 : t0;
+            }
             tma_load_3d(st, &map_a_hi, bar, col, row, node);
             tma_load_3d(st + S::kABytes, &map_a_lo, bar, col, row, node);
             tma_load_2d(st + 2 * S::kABytes, &map_b_hi, bar, c, 0);
             tma_load_2d(st + 2 * S::kABytes + S::kBBytes, &map_b_lo, bar, c, 0);
         }
     } else if (threadIdx.x == 32) {
-        // instruction descriptor: fp32 accumulator, tf32 x tf32, both operands K-major, N = COUT, M = 128
-        constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(COUT >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+        // instruction descriptor: fp32 accumulator, tf32 x tf32, both operands K-major, N columns, M = 128
+        constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
         bool ok = true;
         for (int kb = 0; kb < S::kBlocks && ok; ++kb) {
             const int s = kb % S::kStages;
@@ -320,44 +367,58 @@ ae5_conv_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_
     have = __shfl_sync(0xffffffffu, have ? 1 : 0, 0) != 0;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     if (have) {
-        const int64_t t = (int64_t)t0 + warp * 32 + lane;       // this thread's output position
+        const int64_t t = (int64_t)t0 + warp * 32 + lane;       // this thread's row
         const uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
-        float c4[4] = {0.f, 0.f, 0.f, 0.f};
+        float last[4] = {0.f, 0.f, 0.f, 0.f};                   // kConvCode: the 4 code channels; kDeconvFinal: 2 positions
 #pragma unroll 1
-        for (int c0 = 0; c0 < COUT; c0 += 32) {
+        for (int c0 = 0; c0 < N; c0 += 32) {
             float x[32];
             tmem_load32(trow + (uint32_t)c0, x);
+            const int cb = S::kIsConv ? c0 : c0 % COUT;         // channel of column c0
 #pragma unroll
-            for (int j = 0; j < 32; ++j) x[j] = leaky(__fadd_rn(x[j], s_bias[c0 + j]));
-            if (FUSE_CODE) {
+            for (int j = 0; j < 32; ++j) x[j] = leaky(__fadd_rn(x[j], s_bias[cb + j]));
+            if (MODE == kConvCode) {
 #pragma unroll
                 for (int o = 0; o < 4; ++o)
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) c4[o] = __fmaf_rn(s_w5[o * 64 + c0 + j], x[j], c4[o]);
-            } else if (t < L_out) {
-                float *oh = out_hi + ((int64_t)node * Lpad_out + t) * COUT + c0;
-                float *ol = out_lo + ((int64_t)node * Lpad_out + t) * COUT + c0;
+                    for (int j = 0; j < 32; ++j) last[o] = __fmaf_rn(s_wl[o * 64 + c0 + j], x[j], last[o]);
+            } else if (MODE == kDeconvFinal) {                   // COUT = 32: columns 0..31 position 2t, 32..63 position 2t + 1
+                float acc = 0.f;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    float hi[4], lo[4];
+                for (int j = 0; j < 32; ++j) acc = __fmaf_rn(s_wl[j], x[j], acc);
+                last[c0 / 32] = acc;
+            } else {
+                // conv: row t is position t; deconv: columns below COUT are position 2t, the others 2t + 1
+                const int64_t pos = S::kIsConv ? t : 2 * t + (c0 >= COUT ? 1 : 0);
+                if (pos < L_out) {
+                    const int64_t at = S::kIsConv ? ((int64_t)node * Lpad_out + t) * COUT + c0 : 2 * t * COUT + c0;
+                    float *oh = out_hi + at, *ol = out_lo + at;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) split_tf32(x[4 * q + j], hi[j], lo[j]);
-                    reinterpret_cast<float4 *>(oh)[q] = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                    reinterpret_cast<float4 *>(ol)[q] = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                    for (int q = 0; q < 8; ++q) {
+                        float hi[4], lo[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) split_tf32(x[4 * q + j], hi[j], lo[j]);
+                        reinterpret_cast<float4 *>(oh)[q] = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                        reinterpret_cast<float4 *>(ol)[q] = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                    }
                 }
             }
         }
-        if (FUSE_CODE && t < L_out)
-            reinterpret_cast<float4 *>(code)[(int64_t)node * L_out + t] =
-                make_float4(__fadd_rn(c4[0], s_b5[0]), __fadd_rn(c4[1], s_b5[1]), __fadd_rn(c4[2], s_b5[2]),
-                            __fadd_rn(c4[3], s_b5[3]));
+        if (MODE == kConvCode && t < L_out)
+            reinterpret_cast<float4 *>(out_last)[(int64_t)node * L_out + t] =
+                make_float4(__fadd_rn(last[0], s_bl[0]), __fadd_rn(last[1], s_bl[1]), __fadd_rn(last[2], s_bl[2]),
+                            __fadd_rn(last[3], s_bl[3]));
+        if (MODE == kDeconvFinal) {
+            if (2 * t < L_out) out_last[2 * t] = __fadd_rn(last[0], s_bl[0]);
+            if (2 * t + 1 < L_out) out_last[2 * t + 1] = __fadd_rn(last[1], s_bl[0]);
+        }
     } else if (threadIdx.x == 0) {
         atomicExch(errword, 0x5EA5);                              // a wait ran out
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)COUT) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)N) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------
@@ -384,7 +445,7 @@ __global__ void ae5_deconv1_kernel(const float *__restrict__ z, int64_t L4, cons
     reinterpret_cast<float4 *>(out)[s] = make_float4(leaky(acc[0]), leaky(acc[1]), leaky(acc[2]), leaky(acc[3]));
 }
 
-// ConvTranspose1d(CIN -> COUT, k3, s2, output padding) + leaky ReLU:
+// ConvTranspose1d(CIN -> COUT, k3, s2, output padding) + leaky ReLU on the fp32 pipes (deconv2, 4 -> 32):
 //   y[2j]     = b + sum_ci w[ci][co][0] x[j][ci] + w[ci][co][2] x[j-1][ci]
 //   y[2j + 1] = b + sum_ci w[ci][co][1] x[j][ci]
 // CTA: TP input positions j0 .. j0 + TP - 1 -> outputs 2 j0 .. 2 j0 + 2 TP - 1; thread = (output
@@ -392,7 +453,7 @@ __global__ void ae5_deconv1_kernel(const float *__restrict__ z, int64_t L4, cons
 template <int CIN, int COUT, int TP>
 __global__ void __launch_bounds__(256)
 ae5_deconv_kernel(const float *__restrict__ x, int64_t L_in, int64_t L_out, const float *__restrict__ w,
-                  const float *__restrict__ b, float *__restrict__ y)
+                  const float *__restrict__ b, float *__restrict__ y, float *__restrict__ y_lo)
 {
     extern __shared__ float dsm[];
     float *sw = dsm;                          // [tau][ci][co]
@@ -422,27 +483,16 @@ ae5_deconv_kernel(const float *__restrict__ x, int64_t L_in, int64_t L_out, cons
             even = __fmaf_rn(sw[(2 * CIN + ci) * COUT + co], p, even);
             odd = __fmaf_rn(sw[(1 * CIN + ci) * COUT + co], a, odd);
         }
-        y[(2 * j) * COUT + co] = leaky(even);
-        if (2 * j + 1 < L_out) y[(2 * j + 1) * COUT + co] = leaky(odd);
+        float hi, lo;                                          // the output feeds a GEMM: two tf32 parts
+        split_tf32(leaky(even), hi, lo);
+        y[(2 * j) * COUT + co] = hi;
+        y_lo[(2 * j) * COUT + co] = lo;
+        if (2 * j + 1 < L_out) {
+            split_tf32(leaky(odd), hi, lo);
+            y[(2 * j + 1) * COUT + co] = hi;
+            y_lo[(2 * j + 1) * COUT + co] = lo;
+        }
     }
-}
-
-// Final Conv1d(32 -> 1, k1): the reconstruction of every kept slot.
-__global__ void ae5_final_kernel(const float *__restrict__ d5, int64_t mu, const float *__restrict__ w6,
-                                 const float *__restrict__ b6, float *__restrict__ recon)
-{
-    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= mu) return;
-    float acc = b6[0];
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-        const float4 x = reinterpret_cast<const float4 *>(d5)[p * 8 + q];
-        acc = __fmaf_rn(w6[4 * q + 0], x.x, acc);
-        acc = __fmaf_rn(w6[4 * q + 1], x.y, acc);
-        acc = __fmaf_rn(w6[4 * q + 2], x.z, acc);
-        acc = __fmaf_rn(w6[4 * q + 3], x.w, acc);
-    }
-    recon[p] = acc;
 }
 
 inline unsigned blocks(int64_t n, int per) { return (unsigned)((n + per - 1) / per); }
@@ -473,50 +523,43 @@ bool make_act_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int C, int64_t
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-// Weights [COUT][3 CIN]; box: 32 floats x COUT rows.
-bool make_weight_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int cin, int cout)
+// Decoder activation [L][C] seen as [1][L][C]; box: 32 floats x 128 rows.
+bool make_dact_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int C, int64_t L)
 {
-    const cuuint64_t dims[2] = {(cuuint64_t)(3 * cin), (cuuint64_t)cout};
-    const cuuint64_t strides[1] = {(cuuint64_t)(3 * cin) * 4};
-    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)cout};
+    const cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)L, 1};
+    const cuuint64_t strides[2] = {(cuuint64_t)C * 4, (cuuint64_t)L * C * 4};
+    const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileM, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// GEMM weights [rows][k]; box: 32 floats x all rows.
+bool make_matrix_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int k, int rows)
+{
+    const cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)k * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)rows};
     const cuuint32_t es[2] = {1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// g = 0, 1, 2: conv2, conv3, conv4 (input: the output of conv1 + g)
-template <int CIN, int COUT, bool FUSE>
-cudaError_t launch_gemm(Ctx &c, int g, int64_t L_out, int64_t Lpad_out, float *out_hi, float *out_lo)
+template <int MODE, int CIN, int COUT>
+cudaError_t launch_gemm(Ctx &c, const CUtensorMap &a_hi, const CUtensorMap &a_lo, const CUtensorMap &b_hi,
+                        const CUtensorMap &b_lo, const float *bias, int64_t rows, int nodes, int64_t L_out, int64_t Lpad_out,
+                        float *out_hi, float *out_lo, const float *w_last, const float *b_last, float *out_last)
 {
-    using S = GemmShape<CIN, COUT>;
-    Ae5 &a = *c.ae5;
-    auto kern = ae5_conv_gemm_kernel<CIN, COUT, FUSE>;
+    using S = GemmShape<MODE, CIN, COUT>;
+    auto kern = ae5_gemm_kernel<MODE, CIN, COUT>;
     static bool configured = false;
     if (!configured) {
         const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    kern<<<dim3(blocks(L_out, kTileM), c.K), 128, S::kSmemBytes, c.stream>>>(
-        a.map_act_hi[g], a.map_act_lo[g], a.map_w_hi[g], a.map_w_lo[g], c.params + a.off_b[g + 1], L_out, Lpad_out, out_hi,
-        out_lo, c.params + a.off_w[4], c.params + a.off_b[4], c.code, c.errword),
+    kern<<<dim3(blocks(rows, kTileM), nodes), 128, S::kSmemBytes, c.stream>>>(a_hi, a_lo, b_hi, b_lo, bias, L_out, Lpad_out, out_hi,
+                                                                              out_lo, w_last, b_last, out_last, c.errword),
         ++g_kernel_launches;
-    return cudaGetLastError();
-}
-
-template <int CIN, int COUT, int TP>
-cudaError_t launch_deconv(Ctx &c, const float *x, int64_t L_in, int64_t L_out, const float *w, const float *b, float *y)
-{
-    constexpr int smem = (3 * CIN * COUT + (TP + 1) * CIN) * 4;
-    auto kern = ae5_deconv_kernel<CIN, COUT, TP>;
-    static bool configured = false;
-    if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    // one more input position than L_in covers the output-padding slot at the end
-    kern<<<blocks(L_in + 1, TP), 256, smem, c.stream>>>(x, L_in, L_out, w, b, y), ++g_kernel_launches;
     return cudaGetLastError();
 }
 
@@ -566,11 +609,17 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used)
         a.w_hi[l] = take(n);
         a.w_lo[l] = take(n);
     }
-    a.d[0] = take((size_t)a.len[4] * 4);
-    a.d[1] = take((size_t)a.len[3] * 32);
-    a.d[2] = take((size_t)a.len[2] * 64);
-    a.d[3] = take((size_t)a.len[1] * 128);
-    a.d[4] = take((size_t)a.len[0] * 32);
+    a.d0 = take((size_t)a.len[4] * 4);
+    for (int l = 0; l < 3; ++l) {                           // outputs of deconv2..deconv4: lengths L3, L2, L1
+        const size_t n = (size_t)a.len[3 - l] * kAe5DecCh[l + 2];
+        a.dact_hi[l] = take(n);
+        a.dact_lo[l] = take(n);
+    }
+    for (int l = 0; l < 3; ++l) {                           // GEMM weights of deconv3..deconv5
+        const size_t n = (size_t)4 * kAe5DecCh[l + 2] * kAe5DecCh[l + 3];
+        a.dw_hi[l] = take(n);
+        a.dw_lo[l] = take(n);
+    }
     *used = at;
     // offsets of the layers' parameters inside the flat vector (encoder, then decoder)
     int64_t pos = 0;
@@ -596,12 +645,37 @@ cudaError_t ae5_make_maps(Ctx &c)
     if (e != cudaSuccess) return e;
     bool ok = true;
     for (int l = 0; l < 3; ++l) {
-        ok = ok && make_act_map(enc, &a.map_act_hi[l], a.act_hi[l], kAe5EncCh[l + 1], a.lpad[l], c.K);
-        ok = ok && make_act_map(enc, &a.map_act_lo[l], a.act_lo[l], kAe5EncCh[l + 1], a.lpad[l], c.K);
-        ok = ok && make_weight_map(enc, &a.map_w_hi[l], a.w_hi[l], kAe5EncCh[l + 1], kAe5EncCh[l + 2]);
-        ok = ok && make_weight_map(enc, &a.map_w_lo[l], a.w_lo[l], kAe5EncCh[l + 1], kAe5EncCh[l + 2]);
+        const int cin = kAe5EncCh[l + 1], cout = kAe5EncCh[l + 2];
+        ok = ok && make_act_map(enc, &a.map_act_hi[l], a.act_hi[l], cin, a.lpad[l], c.K);
+        ok = ok && make_act_map(enc, &a.map_act_lo[l], a.act_lo[l], cin, a.lpad[l], c.K);
+        ok = ok && make_matrix_map(enc, &a.map_w_hi[l], a.w_hi[l], 3 * cin, cout);
+        ok = ok && make_matrix_map(enc, &a.map_w_lo[l], a.w_lo[l], 3 * cin, cout);
+        const int dcin = kAe5DecCh[l + 2], dcout = kAe5DecCh[l + 3];
+        ok = ok && make_dact_map(enc, &a.map_dact_hi[l], a.dact_hi[l], dcin, a.len[3 - l]);
+        ok = ok && make_dact_map(enc, &a.map_dact_lo[l], a.dact_lo[l], dcin, a.len[3 - l]);
+        ok = ok && make_matrix_map(enc, &a.map_dw_hi[l], a.dw_hi[l], 2 * dcin, 2 * dcout);
+        ok = ok && make_matrix_map(enc, &a.map_dw_lo[l], a.dw_lo[l], 2 * dcin, 2 * dcout);
     }
     return ok ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+// The GEMM forms of the weights follow the parameter vector; redone after lgc_set_ae_params.
+static void prepare_weights(Ctx &c)
+{
+    Ae5 &a = *c.ae5;
+    if (a.weights_ready) return;
+    const float *P = c.params;
+    for (int l = 0; l < 3; ++l) {
+        const int cin = kAe5EncCh[l + 1], cout = kAe5EncCh[l + 2];
+        ae5_prep_weights_kernel<<<blocks((int64_t)cin * cout * 3, 256), 256, 0, c.stream>>>(P + a.off_w[l + 1], cin, cout, a.w_hi[l],
+                                                                                           a.w_lo[l]),
+            ++g_kernel_launches;
+        const int dcin = kAe5DecCh[l + 2], dcout = kAe5DecCh[l + 3];
+        ae5_prep_deconv_weights_kernel<<<blocks((int64_t)4 * dcin * dcout, 256), 256, 0, c.stream>>>(P + a.off_dw[l + 2], dcin, dcout,
+                                                                                                    a.dw_hi[l], a.dw_lo[l]),
+            ++g_kernel_launches;
+    }
+    a.weights_ready = true;
 }
 
 // Stage 4 for the full-size autoencoder: gather, conv1..conv5 for every node; the codes are
@@ -610,24 +684,22 @@ cudaError_t launch_ae5_encode(Ctx &c)
 {
     Ae5 &a = *c.ae5;
     const float *P = c.params;
-    if (!a.weights_ready) {
-        for (int l = 0; l < 3; ++l) {
-            const int cin = kAe5EncCh[l + 1], cout = kAe5EncCh[l + 2];
-            ae5_prep_weights_kernel<<<blocks((int64_t)cin * cout * 3, 256), 256, 0, c.stream>>>(P + a.off_w[l + 1], cin, cout,
-                                                                                               a.w_hi[l], a.w_lo[l]),
-                ++g_kernel_launches;
-        }
-        a.weights_ready = true;
-    }
+    prepare_weights(c);
     ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.mu, a.len[1], a.lpad[0],
                                                                             P + a.off_w[0], P + a.off_b[0], c.val, a.act_hi[0],
                                                                             a.act_lo[0]),
         ++g_kernel_launches;
     c.val_valid = true;
     cudaError_t e = cudaGetLastError();
-    if (e == cudaSuccess) e = launch_gemm<64, 128, false>(c, 0, a.len[2], a.lpad[1], a.act_hi[1], a.act_lo[1]);
-    if (e == cudaSuccess) e = launch_gemm<128, 256, false>(c, 1, a.len[3], a.lpad[2], a.act_hi[2], a.act_lo[2]);
-    if (e == cudaSuccess) e = launch_gemm<256, 64, true>(c, 2, a.len[4], 0, nullptr, nullptr);
+    if (e == cudaSuccess)
+        e = launch_gemm<kConv, 64, 128>(c, a.map_act_hi[0], a.map_act_lo[0], a.map_w_hi[0], a.map_w_lo[0], P + a.off_b[1],
+                                        a.len[2], c.K, a.len[2], a.lpad[1], a.act_hi[1], a.act_lo[1], nullptr, nullptr, nullptr);
+    if (e == cudaSuccess)
+        e = launch_gemm<kConv, 128, 256>(c, a.map_act_hi[1], a.map_act_lo[1], a.map_w_hi[1], a.map_w_lo[1], P + a.off_b[2],
+                                         a.len[3], c.K, a.len[3], a.lpad[2], a.act_hi[2], a.act_lo[2], nullptr, nullptr, nullptr);
+    if (e == cudaSuccess)
+        e = launch_gemm<kConvCode, 256, 64>(c, a.map_act_hi[2], a.map_act_lo[2], a.map_w_hi[2], a.map_w_lo[2], P + a.off_b[3],
+                                            a.len[4], c.K, a.len[4], 0, nullptr, nullptr, P + a.off_w[4], P + a.off_b[4], c.code);
     return e;
 }
 
@@ -636,17 +708,27 @@ cudaError_t launch_ae5_decode(Ctx &c)
 {
     Ae5 &a = *c.ae5;
     const float *P = c.params;
-    ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d[0]),
+    prepare_weights(c);
+    ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0),
+        ++g_kernel_launches;
+    // deconv2 (4 -> 32): too narrow for the tensor cores
+    constexpr int kTp = 64, kSmem2 = (3 * 4 * 32 + (kTp + 1) * 4) * 4;
+    ae5_deconv_kernel<4, 32, kTp><<<blocks(a.len[4] + 1, kTp), 256, kSmem2, c.stream>>>(a.d0, a.len[4], a.len[3], P + a.off_dw[1],
+                                                                                        P + a.off_db[1], a.dact_hi[0], a.dact_lo[0]),
         ++g_kernel_launches;
     cudaError_t e = cudaGetLastError();
-    if (e == cudaSuccess) e = launch_deconv<4, 32, 64>(c, a.d[0], a.len[4], a.len[3], P + a.off_dw[1], P + a.off_db[1], a.d[1]);
-    if (e == cudaSuccess) e = launch_deconv<32, 64, 32>(c, a.d[1], a.len[3], a.len[2], P + a.off_dw[2], P + a.off_db[2], a.d[2]);
-    if (e == cudaSuccess) e = launch_deconv<64, 128, 64>(c, a.d[2], a.len[2], a.len[1], P + a.off_dw[3], P + a.off_db[3], a.d[3]);
-    if (e == cudaSuccess) e = launch_deconv<128, 32, 64>(c, a.d[3], a.len[1], a.len[0], P + a.off_dw[4], P + a.off_db[4], a.d[4]);
-    if (e != cudaSuccess) return e;
-    ae5_final_kernel<<<blocks(c.mu, 256), 256, 0, c.stream>>>(a.d[4], c.mu, P + a.off_dw[5], P + a.off_db[5], c.recon),
-        ++g_kernel_launches;
-    return cudaGetLastError();
+    // deconv3..5: rows j = 0 .. L_in (one more than the input positions: the last makes the tail)
+    if (e == cudaSuccess)
+        e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], a.map_dw_hi[0], a.map_dw_lo[0], P + a.off_db[2],
+                                         a.len[3] + 1, 1, a.len[2], 0, a.dact_hi[1], a.dact_lo[1], nullptr, nullptr, nullptr);
+    if (e == cudaSuccess)
+        e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], a.map_dw_hi[1], a.map_dw_lo[1], P + a.off_db[3],
+                                          a.len[2] + 1, 1, a.len[1], 0, a.dact_hi[2], a.dact_lo[2], nullptr, nullptr, nullptr);
+    if (e == cudaSuccess)
+        e = launch_gemm<kDeconvFinal, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], a.map_dw_hi[2], a.map_dw_lo[2],
+                                               P + a.off_db[4], a.len[1] + 1, 1, a.len[0], 0, nullptr, nullptr, P + a.off_dw[5],
+                                               P + a.off_db[5], c.recon);
+    return e;
 }
 
 }  // namespace lgc

@@ -90,10 +90,13 @@ struct Ae5 {
     int64_t lpad[3] = {0, 0, 0};        // positions allocated per node for the outputs of conv1..conv3 (even)
     float *act_hi[3] = {}, *act_lo[3] = {};   // [K][lpad][C] outputs of conv1..conv3, channels-last, split into two tf32 parts
     float *w_hi[3] = {}, *w_lo[3] = {};       // [C_out][3 C_in] GEMM weights of conv2..conv4, split likewise
-    float *d[5] = {};                   // decoder activations: [L4][4], [L3][32], [L2][64], [L1][128], [mu][32]
+    float *d0 = nullptr;                // [L4][4] output of deconv1
+    float *dact_hi[3] = {}, *dact_lo[3] = {}; // [L3][32], [L2][64], [L1][128]: outputs of deconv2..deconv4, split likewise
+    float *dw_hi[3] = {}, *dw_lo[3] = {};     // [2 C_out][2 C_in] GEMM weights of deconv3..deconv5, split likewise
     int64_t off_w[5] = {}, off_b[5] = {};     // offsets of the encoder layers' weights / biases in the parameter vector
     int64_t off_dw[6] = {}, off_db[6] = {};   // the same for the decoder's six layers
     CUtensorMap map_act_hi[3], map_act_lo[3], map_w_hi[3], map_w_lo[3];
+    CUtensorMap map_dact_hi[3], map_dact_lo[3], map_dw_hi[3], map_dw_lo[3];
     bool weights_ready = false;         // w_hi / w_lo match the parameter vector
 };
 

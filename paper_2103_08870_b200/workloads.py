@@ -383,6 +383,13 @@ class Workload:
     momentum: float = 0.9
     innovation_permille: int = 100
     seed: int = DEFAULT_SEED
+    ae_kind: str = "conv2"    # "conv2": two layers each way with (ae_c1, ae_c2) channels; "conv5": the full-size one
+
+    def init_params(self) -> torch.Tensor:
+        """The autoencoder's seeded initial parameters, flat fp32 on the CPU."""
+        if self.ae_kind == "conv5":
+            return ae5_init_params(self.seed)
+        return ae_init_params(self.ae_c1, self.ae_c2, self.variant, self.num_nodes, self.seed)
 
 
 def workload(name: str) -> Workload:
@@ -396,7 +403,9 @@ def workload(name: str) -> Workload:
         return Workload("segnet", segnet_table(), 4, 1000, "rar", 8, 4, 10, ae_train_steps=50)
     if name == "stress":
         return Workload("stress", flat_table(1 << 30), 4, 100, "rar", 16, 8, 5)
+    if name == "resnet50_ae5":      # the ResNet-50-shaped case with the paper's full-size autoencoder
+        return Workload("resnet50_ae5", resnet50_table(), 8, 1000, "rar", 64, 4, 10, ae_kind="conv5")
     raise KeyError(name)
 
 
-WORKLOAD_NAMES = ("tiny", "resnet50", "resnet101_ps", "segnet", "stress")
+WORKLOAD_NAMES = ("tiny", "resnet50", "resnet101_ps", "segnet", "stress", "resnet50_ae5")
