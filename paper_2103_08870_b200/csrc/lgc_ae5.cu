@@ -240,6 +240,7 @@ struct GemmShape {
     static constexpr int kABytes = kTileM * kBlockK * 4;        // one (hi or lo) activation tile of a k-block
     static constexpr int kBBytes = kN * kBlockK * 4;
     static constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;
+    // as many stages as fit (one CTA per SM; two CTAs of half the stages each measured slower)
     static constexpr int kStages = (200 * 1024) / kStageBytes < kBlocks ? (200 * 1024) / kStageBytes : kBlocks;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024;   // + slack to align the tiles to 1024 bytes
     static_assert(kN >= 32 && kN <= 256 && (kN & (kN - 1)) == 0, "accumulator columns: a power of two in [32, 256]");

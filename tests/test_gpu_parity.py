@@ -136,15 +136,17 @@ def test_layer_of_several_groups_with_ties(levels, first_from_data):
     assert from_data[0] == first_from_data
 
 
-@pytest.mark.parametrize("numel, K", [([300_000, 5000, 120_000], 2), ([2_000_000, 700_000, 300_001], 3)])
-def test_full_size_autoencoder(numel, K):
+@pytest.mark.parametrize("numel, K, scale", [([300_000, 5000, 120_000], 2, 1.0), ([300_000, 5000, 120_000], 2, 500.0),
+                                             ([2_000_000, 700_000, 300_001], 3, 1.0)])
+def test_full_size_autoencoder(numel, K, scale):
     # the autoencoder of Section IV-C (filters 64/128/256/64/4 and 4/32/64/128/32 + 1x1): mu = 425
-    # (every GEMM tile ragged) and mu = 3000 (several tiles per layer and node, ragged tails)
+    # (every GEMM tile ragged) and mu = 3000 (several tiles per layer and node, ragged tails).
+    # scale 500 makes the kept values O(1), so that the data, not the biases, dominate every layer.
     ora, gpu = make_pair(numel, K, ae_kind="conv5")
     src = W.GradientSource(W.LayerTable("ae5", numel, [1 + i for i in range(len(numel))]), K, seed=21)
     upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
     for t in range(3):
-        g = src.step(t)
+        g = src.step(t) * scale
         compare_step(ora, gpu, g, g.cuda(), t % K, upd)
 
 

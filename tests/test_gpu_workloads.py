@@ -21,7 +21,7 @@ pytestmark = pytest.mark.gpu
 
 def run_workload(name, steps, state_every=1):
     w = W.workload(name)
-    ora, gpu = make_pair(w.table.numel, w.num_nodes, variant=w.variant, c1=w.ae_c1, c2=w.ae_c2,
+    ora, gpu = make_pair(w.table.numel, w.num_nodes, variant=w.variant, ae_kind=w.ae_kind, c1=w.ae_c1, c2=w.ae_c2,
                          density_ppm=w.density_ppm, momentum=w.momentum,
                          innovation_permille=w.innovation_permille, seed=w.seed)
     src = W.GradientSource(w.table, w.num_nodes, seed=w.seed, device="cuda")
@@ -37,6 +37,12 @@ def run_workload(name, steps, state_every=1):
 def test_resnet50_config():
     ora, gpu = run_workload("resnet50", 10, state_every=3)
     assert gpu.L == 161 and gpu.N == 25_557_032 and gpu.mu == sum(ora.k_l)
+
+
+def test_resnet50_config_with_the_full_size_autoencoder():
+    # the ResNet-50-shaped case, K = 8, with the autoencoder of Section IV-C: mu = 25,617, code 4 x 1600
+    ora, gpu = run_workload("resnet50_ae5", 3, state_every=2)
+    assert gpu.mu == 25_617 and gpu.code_len == 4 * 1600 and gpu.P == 216_729
 
 
 def test_resnet101_parameter_server_config():
