@@ -13,6 +13,7 @@ Stages (Algorithm 1 = parameter server "ps", Algorithm 2 = ring-allreduce "rar")
   decode_scatter  rar: g~^rec = D_c(g~^avg); ps: g~^rec_k = D_c^k(g~^c, g~^I_k), averaged over k
                   (Sec. V-B.1); written back to dense positions; sent entries leave u and v
   ae_train_step   ring-allreduce reconstruction loss (Sec. IV-B), mean over mu, one Adam step
+  ae_train_step_ps  parameter-server loss lam_rec L_rec + lam_sim L_sim (Sec. IV-A), one Adam step
 """
 from __future__ import annotations
 
@@ -219,6 +220,75 @@ class OracleLGC:
             dh = O.relu_bwd(hs[k], dh)
             O.conv1d_bwd(xs[k], self.p["enc.w1"], dh, g["enc.w1"], g["enc.b1"], want_dx=False)
         return loss, g
+
+    # -- autoencoder training (parameter-server loss, Sec. IV-A) ----------------------------
+    def ae_loss_and_grads_ps(self, common_node: int, lam_rec: float = 1.0, lam_sim: float = 1.0):
+        """L = lam_rec L_rec + lam_sim L_sim (Sec. IV-A): every node's kept values go through the
+        encoder; L_sim sums ||E_c(g~_k) - E_c(g~_m)||^2 over all ordered pairs k != m; the code of
+        `common_node` is decoded by every node's decoder together with that node's innovation and
+        L_rec sums ||g~_k - g~^rec_k||^2 over the nodes.  Reading: L_rec is divided by mu and L_sim
+        by the number of code entries (c2 L2), so that lam_rec = lam_sim = 1 weighs an average
+        entry of either kind alike.  Returns (loss, L_rec / mu, L_sim / (c2 L2), gradients)."""
+        assert self.variant == "ps" and self.ae_kind == "conv2"
+        K, mu = self.K, self.mu
+        xs = [self.val[k].astype(np.float64).reshape(1, -1) for k in range(K)]
+        hs, zs = [], []
+        for k in range(K):
+            h, z = self._enc(xs[k][0])
+            hs.append(h)
+            zs.append(z)
+        nz = zs[0].size
+        sim = 0.0
+        for k in range(K):
+            for m in range(K):
+                if m != k:
+                    sim += float(np.sum((zs[k] - zs[m]) ** 2))
+        sim /= nz
+        zc = zs[common_node]
+        g = {name: np.zeros(shape, dtype=np.float64) for name, shape in self.order}
+        dzs = [np.zeros_like(zc) for _ in range(K)]
+        rec = 0.0
+        for k in range(K):
+            inn = np.zeros(mu, dtype=np.float64)
+            for l in range(self.L):
+                a, b = int(self.koff[l]), int(self.koff[l + 1])
+                inn[a:b] = O.innovation(self.val[k, a:b], self.ki_l[l])
+            d, y = self._dec(zc, f"dec{k}")
+            w0, w1, b = (float(t) for t in self.p[f"dec{k}.fuse"])
+            r = w0 * y + w1 * inn.reshape(1, -1) + b
+            diff = r - xs[k]
+            rec += float(np.sum(diff * diff)) / mu
+            dr = lam_rec * 2.0 * diff / mu
+            g[f"dec{k}.fuse"] += np.array([np.sum(dr * y), np.sum(dr * inn), np.sum(dr)])
+            dy = w0 * dr
+            dd = O.convt1d_bwd(d, self.p[f"dec{k}.w2"], self.op2, dy, g[f"dec{k}.w2"], g[f"dec{k}.b2"])
+            dd = O.relu_bwd(d, dd)
+            dzs[common_node] = dzs[common_node] + O.convt1d_bwd(zc, self.p[f"dec{k}.w1"], self.op1, dd,
+                                                                 g[f"dec{k}.w1"], g[f"dec{k}.b1"])
+        zsum = sum(zs[1:], zs[0].copy())
+        for k in range(K):
+            # d/dz_k of sum over ordered pairs: every unordered pair appears twice
+            dz = dzs[k] + lam_sim * 4.0 * (K * zs[k] - zsum) / nz
+            dh = O.conv1d_bwd(hs[k], self.p["enc.w2"], dz, g["enc.w2"], g["enc.b2"])
+            dh = O.relu_bwd(hs[k], dh)
+            O.conv1d_bwd(xs[k], self.p["enc.w1"], dh, g["enc.w1"], g["enc.b1"], want_dx=False)
+        return lam_rec * rec + lam_sim * sim, rec, sim, g
+
+    def _adam_step(self, g) -> None:
+        flat_p = self.get_params()
+        flat_g = np.concatenate([g[name].reshape(-1) for name, _ in self.order])
+        if self.adam_m is None:
+            self.adam_m = np.zeros_like(flat_p)
+            self.adam_v = np.zeros_like(flat_p)
+        self.adam_t += 1
+        O.adam(flat_p, self.adam_m, self.adam_v, flat_g, self.adam_t, self.lr, self.beta1,
+               self.beta2, self.eps)
+        self.set_params(flat_p)
+
+    def ae_train_step_ps(self, common_node: int, lam_rec: float = 1.0, lam_sim: float = 1.0) -> float:
+        loss, _, _, g = self.ae_loss_and_grads_ps(common_node, lam_rec, lam_sim)
+        self._adam_step(g)
+        return loss
 
     def ae_train_step(self) -> float:
         loss, g = self.ae_loss_and_grads()

@@ -216,6 +216,87 @@ def test_training_gradients_equal_autograd_and_loss_falls():
     assert o.adam_t == 50
 
 
+def ps_training_oracle(K=3, seed=12):
+    g = grads(TOY, K, 1)[0] * 1e3
+    o = OracleLGC(TOY, K, variant="ps", params=params(8, 4, "ps", K, seed=seed))
+    for k in range(K):                                # fusion scalars away from their (1, 1, 0) start
+        o.p[f"dec{k}.fuse"][:] = (0.8 + 0.1 * k, 0.6 - 0.1 * k, 0.05 * k)
+    o.accumulate(g)
+    o.topk()
+    return o
+
+
+def test_ps_training_gradients_by_finite_differences():
+    o = ps_training_oracle()
+    loss, rec, sim, gr = o.ae_loss_and_grads_ps(1, 0.7, 0.3)
+    assert abs(loss - (0.7 * rec + 0.3 * sim)) <= 1e-12 * loss
+    flat_g = np.concatenate([gr[n].reshape(-1) for n, _ in o.order])
+    flat_p = o.get_params()
+    rng = np.random.default_rng(1)
+    h = 1e-6
+    fuse = [i for i in range(flat_p.size - 3, flat_p.size)]          # the last node's fusion scalars
+    for j in list(rng.choice(flat_p.size, 60, replace=False)) + fuse:
+        pp, pm = flat_p.copy(), flat_p.copy()
+        pp[j] += h
+        pm[j] -= h
+        o.set_params(pp)
+        lp = o.ae_loss_and_grads_ps(1, 0.7, 0.3)[0]
+        o.set_params(pm)
+        lm = o.ae_loss_and_grads_ps(1, 0.7, 0.3)[0]
+        fd = (lp - lm) / (2 * h)
+        assert abs(fd - flat_g[j]) <= 1e-6 * max(1.0, abs(flat_g[j])) + 1e-7 * np.abs(flat_g).max(), j
+    o.set_params(flat_p)
+
+
+def test_ps_training_loss_and_gradients_equal_autograd():
+    K = 3
+    o = ps_training_oracle(K)
+    c = 2
+    loss, rec, sim, gr = o.ae_loss_and_grads_ps(c, 1.0, 1.0)
+    tp = {k: torch.from_numpy(v.copy()).requires_grad_(True) for k, v in o.p.items()}
+    x = torch.from_numpy(o.val.astype(np.float64))[:, None, :]
+    z = F.conv1d(F.relu(F.conv1d(x, tp["enc.w1"], tp["enc.b1"], stride=2)), tp["enc.w2"], tp["enc.b2"], stride=2)
+    t_sim = sum(((z[k] - z[m]) ** 2).sum() for k in range(K) for m in range(K) if m != k) / z[0].numel()
+    t_rec = 0.0
+    for k in range(K):
+        inn = np.zeros(o.mu)
+        for l in range(o.L):
+            a, b = int(o.koff[l]), int(o.koff[l + 1])
+            inn[a:b] = O.innovation(o.val[k, a:b], o.ki_l[l])
+        d = F.relu(F.conv_transpose1d(z[c:c + 1], tp[f"dec{k}.w1"], tp[f"dec{k}.b1"], stride=2, output_padding=o.op1))
+        y = F.conv_transpose1d(d, tp[f"dec{k}.w2"], tp[f"dec{k}.b2"], stride=2, output_padding=o.op2)[0, 0]
+        f = tp[f"dec{k}.fuse"]
+        r = f[0] * y + f[1] * torch.from_numpy(inn) + f[2]
+        t_rec = t_rec + ((r - x[k, 0]) ** 2).sum() / o.mu
+    tl = t_rec + t_sim
+    tl.backward()
+    assert abs(rec - t_rec.item()) <= 1e-12 * t_rec.item() and abs(sim - t_sim.item()) <= 1e-12 * t_sim.item()
+    for name, _ in o.order:
+        ref = tp[name].grad.numpy()
+        assert np.abs(gr[name] - ref).max() <= 1e-10 * max(1e-3, np.abs(ref).max()), name
+
+
+def test_ps_training_special_cases():
+    # one node: no pairs, L_sim = 0 and the loss is the reconstruction term alone
+    g = grads(TOY, 1, 1)[0] * 1e3
+    o = OracleLGC(TOY, 1, variant="ps", params=params(8, 4, "ps", 1, seed=3))
+    o.accumulate(g)
+    o.topk()
+    loss, rec, sim, _ = o.ae_loss_and_grads_ps(0, 1.0, 5.0)
+    assert sim == 0.0 and loss == rec
+    # identical nodes: all codes coincide, L_sim = 0 and its gradient vanishes: with lam_rec = 0 nothing moves
+    K = 3
+    o = OracleLGC(TOY, K, variant="ps", params=params(8, 4, "ps", K, seed=3))
+    o.accumulate(np.repeat(g, K, axis=0))
+    o.topk()
+    loss, rec, sim, gr = o.ae_loss_and_grads_ps(1, 0.0, 1.0)
+    assert sim == 0.0 and loss == 0.0 and all(not v.any() for v in gr.values())
+    # training lowers the loss
+    o = ps_training_oracle()
+    losses = [o.ae_train_step_ps(t % 3) for t in range(40)]
+    assert losses[-1] < 0.95 * losses[0] and o.adam_t == 40
+
+
 def test_momentum_zero_is_plain_error_feedback():
     K = 2
     gs = grads(TOY, K, 3)
