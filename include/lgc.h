@@ -146,7 +146,7 @@ lgc_status lgc_decode_scatter(lgc_ctx *ctx, float *update);
 
 /* Second training phase (Section V-B, weights updated with the top-magnitude gradients): the dense
  * mean over nodes of the kept values, no autoencoder; sent entries leave u and v.
- * Valid after lgc_topk (and after lgc_ae_train_step).  update: device, fp32 [N]. */
+ * Valid after lgc_topk (and after lgc_ae_train_step / lgc_ae_train_step_ps).  update: device, fp32 [N]. */
 lgc_status lgc_topk_scatter(lgc_ctx *ctx, float *update);
 
 /* One training step of the autoencoder on the kept values of the last lgc_topk: ring-allreduce
@@ -155,6 +155,17 @@ lgc_status lgc_topk_scatter(lgc_ctx *ctx, float *update);
  * analytic backward pass, Adam with bias correction.  Ring-allreduce variant with LGC_AE_CONV2
  * only.  loss_out: device fp32 scalar or NULL.  May be called several times after one lgc_topk. */
 lgc_status lgc_ae_train_step(lgc_ctx *ctx, float *loss_out);
+
+/* The same for the parameter-server autoencoder (Section IV-A): every node's kept values are
+ * encoded; the code of `common_node` goes through all K decoders, each with its node's innovation;
+ *     loss = lambda_rec * (1/mu) sum_k || g~_k - g~^rec_k ||^2
+ *          + lambda_sim * (1/(c2 L2)) sum_k sum_{m != k} || E_c(g~_k) - E_c(g~_m) ||^2
+ * (the paper's L_rec and L_sim, each divided by the number of entries it sums over per node),
+ * analytic backward pass through the K decoders, their fusion scalars and the encoder, Adam.
+ * Parameter-server variant with LGC_AE_CONV2 only; valid after lgc_topk.  Overwrites the codes,
+ * the common code and the innovations of the context.  loss_out: device fp32 scalar or NULL. */
+lgc_status lgc_ae_train_step_ps(lgc_ctx *ctx, int32_t common_node, float lambda_rec, float lambda_sim,
+                                float *loss_out);
 
 /* A whole compression step from host memory: copies `host_grads` ([K][N], ideally pinned) to
  * `dev_grads`, runs the five stages, copies the dense update back to `host_update` ([N]).

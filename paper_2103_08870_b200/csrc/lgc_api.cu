@@ -243,6 +243,22 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
         c.inn_pos = cv.take<int32_t>((size_t)p.K * p.muI);
         carve_select(cv, c.sel_inn, plan_select(p.koff, p.k_l, p.ki_l, p.kioff), p.K);
     }
+    if (conv && ps) {                       // training work space, one slice per node
+        const size_t c1 = cfg.ae_c1, c2 = cfg.ae_c2, K = p.K;
+        c.t_h = cv.take<float>(K * c1 * p.L1);
+        c.t_dh = cv.take<float>(K * c1 * p.L1);
+        c.t_d = cv.take<float>(K * c1 * p.L1);
+        c.t_dd = cv.take<float>(K * c1 * p.L1);
+        c.t_dr = cv.take<float>(K * p.mu);
+        c.t_y = cv.take<float>(K * p.mu);
+        c.t_dy = cv.take<float>(K * p.mu);
+        c.t_dz = cv.take<float>(K * c2 * p.L2);
+        c.t_dzc = cv.take<float>(K * c2 * p.L2);
+        c.t_zsum = cv.take<float>(c2 * p.L2);
+        c.t_loss_blocks = (int)((p.mu + 127) / 128);
+        c.t_loss_part = cv.take<double>(K * (size_t)c.t_loss_blocks);
+        c.t_sim_part = cv.take<double>((size_t)((p.L2 + 127) / 128));
+    }
     if (conv && !ps) {
         const size_t c1 = cfg.ae_c1, c2 = cfg.ae_c2;
         c.t_h = cv.take<float>((size_t)p.K * c1 * p.L1);
@@ -497,6 +513,20 @@ lgc_status lgc_ae_train_step(lgc_ctx *c, float *loss_out)
     cudaError_t e = launch_gather(*c);
     if (e == cudaSuccess) e = launch_train_step(*c, loss_out);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_ae_train_step");
+    return LGC_OK;
+}
+
+lgc_status lgc_ae_train_step_ps(lgc_ctx *c, int32_t common_node, float lambda_rec, float lambda_sim, float *loss_out)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (c->cfg.variant != LGC_VARIANT_PS || c->cfg.ae_kind != LGC_AE_CONV2)
+        return fail(c, LGC_ERR_UNSUPPORTED, "lgc_ae_train_step_ps needs the parameter-server variant with the two-layer autoencoder");
+    if (common_node < 0 || common_node >= c->K) return fail(c, LGC_ERR_INVALID_ARG, "common_node out of range");
+    if (!(lambda_rec >= 0.0f) || !(lambda_sim >= 0.0f)) return fail(c, LGC_ERR_INVALID_ARG, "the loss weights must not be negative");
+    if (c->stage != Ctx::kSelected) return fail(c, LGC_ERR_BAD_STATE, "lgc_ae_train_step_ps must follow lgc_topk");
+    cudaError_t e = launch_gather(*c);
+    if (e == cudaSuccess) e = launch_train_step_ps(*c, common_node, lambda_rec, lambda_sim, loss_out);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_ae_train_step_ps");
     return LGC_OK;
 }
 

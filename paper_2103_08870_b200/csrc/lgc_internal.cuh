@@ -136,6 +136,12 @@ struct Ctx {
     float *t_dh = nullptr;         // [K][c1][L1]
     double *t_loss_part = nullptr; // [loss blocks]
     int t_loss_blocks = 0;
+    // parameter-server training: the buffers above hold one slice per node ([K] in front), plus
+    float *t_y = nullptr;          // [K][mu]     decoder output before the fusion with the innovation
+    float *t_dy = nullptr;         // [K][mu]     d loss / d that output
+    float *t_dzc = nullptr;        // [K][c2][L2] every decoder's gradient at the common code
+    float *t_zsum = nullptr;       // [c2][L2]    sum over nodes of the codes
+    double *t_sim_part = nullptr;  // [blocks over L2] partial sums of the similarity loss
     // step state machine
     enum Stage { kIdle, kAccumulated, kSelected, kEncoded, kCombined } stage = kIdle;
     int32_t last_leader = 0;
@@ -177,6 +183,7 @@ cudaError_t launch_combine_ps(Ctx &c, int common_node);
 cudaError_t launch_decode_scatter(Ctx &c, float *update);
 cudaError_t launch_topk_scatter(Ctx &c, float *update);
 cudaError_t launch_train_step(Ctx &c, float *loss_out);
+cudaError_t launch_train_step_ps(Ctx &c, int common, float lam_rec, float lam_sim, float *loss_out);
 // full-size autoencoder (lgc_ae5.cu)
 int64_t ae5_param_count();
 bool ae5_lengths(int64_t mu, int64_t (&len)[5]);

@@ -21,7 +21,8 @@ AE_CONV2, AE_IDENTITY, AE_CONV5 = 0, 1, 2
 
 EXPORTS = (
     "lgc_workspace_bytes", "lgc_init", "lgc_destroy", "lgc_accumulate", "lgc_topk", "lgc_encode",
-    "lgc_combine", "lgc_decode_scatter", "lgc_topk_scatter", "lgc_ae_train_step", "lgc_step_host",
+    "lgc_combine", "lgc_decode_scatter", "lgc_topk_scatter", "lgc_ae_train_step", "lgc_ae_train_step_ps",
+    "lgc_step_host",
     "lgc_get_layout", "lgc_keep_counts", "lgc_get_buffers", "lgc_set_ae_params", "lgc_get_ae_params",
     "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc", "lgc_kernel_launches", "lgc_selection_stats",
 )
@@ -59,6 +60,7 @@ def lib() -> C.CDLL:
         l.lgc_decode_scatter.argtypes = [vp, vp]
         l.lgc_topk_scatter.argtypes = [vp, vp]
         l.lgc_ae_train_step.argtypes = [vp, vp]
+        l.lgc_ae_train_step_ps.argtypes = [vp, C.c_int32, C.c_float, C.c_float, vp]
         l.lgc_step_host.argtypes = [vp, vp, vp, vp, vp, C.c_int32]
         l.lgc_get_layout.argtypes = [vp] + [C.POINTER(C.c_int64)] * 5
         l.lgc_keep_counts.argtypes = [vp]
@@ -209,6 +211,11 @@ class LGC:
     def ae_train_step(self, loss_out: Optional[torch.Tensor] = None) -> None:
         ptr = self._dev_f32(loss_out, 1, "loss_out") if loss_out is not None else None
         self._ok(self._l.lgc_ae_train_step(self._ctx, ptr), "lgc_ae_train_step")
+
+    def ae_train_step_ps(self, common_node: int, lambda_rec: float = 1.0, lambda_sim: float = 1.0,
+                         loss_out: Optional[torch.Tensor] = None) -> None:
+        ptr = self._dev_f32(loss_out, 1, "loss_out") if loss_out is not None else None
+        self._ok(self._l.lgc_ae_train_step_ps(self._ctx, common_node, lambda_rec, lambda_sim, ptr), "lgc_ae_train_step_ps")
 
     def step(self, grads: torch.Tensor, update: torch.Tensor, choice: int = 0) -> None:
         """The five stages of one compression step, in order."""

@@ -150,6 +150,36 @@ def test_full_size_autoencoder(numel, K, scale):
         compare_step(ora, gpu, g, g.cuda(), t % K, upd)
 
 
+@pytest.mark.parametrize("c1, c2, K", [(8, 4, 3), (16, 8, 4)])
+def test_parameter_server_autoencoder_training(c1, c2, K):
+    # Section IV-A: reconstruction loss through the K decoders (innovation fused in) + similarity loss
+    # between the nodes' codes; 12 Adam steps with a changing common node, then a compression step
+    numel = [70001, 9000, 20000, 4097, 127]
+    ora, gpu = make_pair(numel, K, variant="ps", c1=c1, c2=c2)
+    src = toy_source(numel, K, seed=31)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    loss_dev = torch.zeros(1, device="cuda")
+    losses, losses_ref = [], []
+    for t in range(12):
+        g = src.step(t) * 300.0                       # kept values of O(1): well-conditioned gradients
+        ora.accumulate(g.numpy())
+        gpu.accumulate(g.cuda())
+        ora.topk()
+        gpu.topk(0)
+        common = (5 * t + 1) % K
+        losses_ref.append(ora.ae_train_step_ps(common, 0.7, 0.3))
+        gpu.ae_train_step_ps(common, 0.7, 0.3, loss_dev)
+        losses.append(loss_dev.item())
+        ref = ora.topk_scatter()
+        gpu.topk_scatter(upd)
+        assert_close(upd.cpu().numpy(), ref, f"sparse update at training step {t}")
+    assert_close(np.array(losses), np.array(losses_ref), "training losses")
+    assert_close(gpu.get_ae_params().numpy(), ora.get_params(), "trained parameters")
+    gpu.check()
+    g = src.step(12) * 300.0
+    compare_step(ora, gpu, g, g.cuda(), 1, upd)
+
+
 def test_dense_selection_uses_the_global_compact_arrays():
     # k = 40,000 of 2,000,000: more candidates than the finishing CTA keeps in shared memory
     numel = [2_000_000]

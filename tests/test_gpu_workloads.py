@@ -48,6 +48,30 @@ def test_resnet50_config_with_the_full_size_autoencoder():
 def test_resnet101_parameter_server_config():
     ora, gpu = run_workload("resnet101_ps", 4, state_every=3)
     assert gpu.L == 314 and gpu.N == 44_549_160 and gpu.idx.shape[0] == 16
+    # two training steps of the parameter-server autoencoder (Section IV-A) at this size
+    w = W.workload("resnet101_ps")
+    src = W.GradientSource(w.table, w.num_nodes, seed=w.seed, device="cuda")
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    g = torch.empty((w.num_nodes, gpu.N), dtype=torch.float32, device="cuda")
+    loss_dev = torch.zeros(1, device="cuda")
+    for t in range(4, 6):
+        src.step_into(t, g)
+        ora.accumulate(g.cpu().numpy())
+        gpu.accumulate(g)
+        ora.topk()
+        gpu.topk(0)
+        common = W.choice_for_step(w.seed, t, w.num_nodes)
+        ref_loss = ora.ae_train_step_ps(common)
+        gpu.ae_train_step_ps(common, 1.0, 1.0, loss_dev)
+        assert_close(np.array([loss_dev.item()]), np.array([ref_loss]), f"training loss at step {t}")
+        assert_close(upd_after(gpu, upd), ora.topk_scatter(), f"sparse update at step {t}")
+    assert_close(gpu.get_ae_params().numpy(), ora.get_params(), "trained parameters")
+    gpu.check()
+
+
+def upd_after(gpu, upd):
+    gpu.topk_scatter(upd)
+    return upd.cpu().numpy()
 
 
 def test_segnet_config_with_autoencoder_training():
