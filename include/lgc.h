@@ -167,6 +167,18 @@ lgc_status lgc_ae_train_step(lgc_ctx *ctx, float *loss_out);
 lgc_status lgc_ae_train_step_ps(lgc_ctx *ctx, int32_t common_node, float lambda_rec, float lambda_sim,
                                 float *loss_out);
 
+/* Entropy coding of an index list (Section V-A: the transferred indices are DEFLATE-coded and
+ * their rate counts in the compression ratio).  The ascending offsets of every layer become gaps
+ * (the first counted from the layer's start, the others from the previous offset + 1), each gap
+ * a little-endian base-128 varint; the bytes are written as one raw DEFLATE block (RFC 1951,
+ * dynamic Huffman codes, literals only), which any inflate implementation decodes.
+ * node: whose list (ring-allreduce: all nodes share the leader's; parameter server: 0 .. K-1).
+ * stream_out: device, `capacity` bytes, 4-byte aligned, capacity a multiple of 4; zero-filled
+ * beyond the stream.  sizes_out: device, two uint64: bytes of the DEFLATE stream and bytes of the
+ * varint form.  If the stream is larger than the capacity only the sizes are valid.
+ * Valid from lgc_topk until the next lgc_accumulate. */
+lgc_status lgc_encode_indices(lgc_ctx *ctx, int32_t node, void *stream_out, size_t capacity, uint64_t *sizes_out);
+
 /* A whole compression step from host memory: copies `host_grads` ([K][N], ideally pinned) to
  * `dev_grads`, runs the five stages, copies the dense update back to `host_update` ([N]).
  * Everything is enqueued on the context's stream; the call returns without waiting.

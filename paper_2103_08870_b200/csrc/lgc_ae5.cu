@@ -23,6 +23,7 @@ constexpr float kSlope = 0.01f;       // leaky-ReLU slope (the paper names the a
 constexpr int kTileM = 128;           // output positions per CTA of the GEMM: the M of one tcgen05.mma
 constexpr int kBlockK = 32;           // fp32 per 128-byte swizzled row
 constexpr int kSpinLimit = 4000000;   // mbarrier polls before a wait gives up
+constexpr int kStagePitch = 36;       // floats per row of the epilogue's staging blocks (16-byte aligned, spreads the banks)
 
 __device__ __forceinline__ float leaky(float x) { return x > 0.0f ? x : kSlope * x; }
 
@@ -243,6 +244,7 @@ struct GemmShape {
     // as many stages as fit (one CTA per SM; two CTAs of half the stages each measured slower)
     static constexpr int kStages = (200 * 1024) / kStageBytes < kBlocks ? (200 * 1024) / kStageBytes : kBlocks;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024;   // + slack to align the tiles to 1024 bytes
+    static_assert(kStages * kStageBytes >= 4 * 2 * 32 * kStagePitch * 4, "the epilogue stages its blocks in the operand area");
     static_assert(kN >= 32 && kN <= 256 && (kN & (kN - 1)) == 0, "accumulator columns: a power of two in [32, 256]");
 };
 
@@ -370,6 +372,7 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
     if (have) {
         const int64_t t = (int64_t)t0 + warp * 32 + lane;       // this thread's row
         const uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
+        float *stage = reinterpret_cast<float *>(dyn_smem + (tiles - smem_u32(dyn_smem)));
         float last[4] = {0.f, 0.f, 0.f, 0.f};                   // kConvCode: the 4 code channels; kDeconvFinal: 2 positions
 #pragma unroll 1
         for (int c0 = 0; c0 < N; c0 += 32) {
@@ -389,18 +392,29 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
                 for (int j = 0; j < 32; ++j) acc = __fmaf_rn(s_wl[j], x[j], acc);
                 last[c0 / 32] = acc;
             } else {
-                // conv: row t is position t; deconv: columns below COUT are position 2t, the others 2t + 1
-                const int64_t pos = S::kIsConv ? t : 2 * t + (c0 >= COUT ? 1 : 0);
-                if (pos < L_out) {
-                    const int64_t at = S::kIsConv ? ((int64_t)node * Lpad_out + t) * COUT + c0 : 2 * t * COUT + c0;
-                    float *oh = out_hi + at, *ol = out_lo + at;
+                // The 32 x 32 block of this warp (row = lane) goes through shared memory so that the global
+                // stores are whole 128-byte rows: the operand stages are free once the accumulator is complete.
+                float *sh_hi = stage + warp * (2 * 32 * kStagePitch), *sh_lo = sh_hi + 32 * kStagePitch;
+                __syncwarp();                                    // the previous block has been read out
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        float hi[4], lo[4];
+                for (int q = 0; q < 8; ++q) {
+                    float hi[4], lo[4];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) split_tf32(x[4 * q + j], hi[j], lo[j]);
-                        reinterpret_cast<float4 *>(oh)[q] = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                        reinterpret_cast<float4 *>(ol)[q] = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                    for (int j = 0; j < 4; ++j) split_tf32(x[4 * q + j], hi[j], lo[j]);
+                    *reinterpret_cast<float4 *>(sh_hi + lane * kStagePitch + 4 * q) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+                    *reinterpret_cast<float4 *>(sh_lo + lane * kStagePitch + 4 * q) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                }
+                __syncwarp();
+#pragma unroll
+                for (int it = 0; it < 8; ++it) {
+                    const int rr = it * 4 + (lane >> 3), cq = lane & 7;      // four rows per pass, eight lanes per row
+                    const int64_t tr = (int64_t)t0 + warp * 32 + rr;
+                    // conv: row tr is position tr; deconv: columns below COUT are position 2 tr, the others 2 tr + 1
+                    const int64_t pos = S::kIsConv ? tr : 2 * tr + (c0 >= COUT ? 1 : 0);
+                    if (pos < L_out) {
+                        const int64_t at = (S::kIsConv ? ((int64_t)node * Lpad_out + tr) * COUT : 2 * tr * COUT) + c0 + 4 * cq;
+                        *reinterpret_cast<float4 *>(out_hi + at) = *reinterpret_cast<const float4 *>(sh_hi + rr * kStagePitch + 4 * cq);
+                        *reinterpret_cast<float4 *>(out_lo + at) = *reinterpret_cast<const float4 *>(sh_lo + rr * kStagePitch + 4 * cq);
                     }
                 }
             }

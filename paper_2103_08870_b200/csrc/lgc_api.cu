@@ -236,6 +236,8 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
     c.recon = cv.take<float>((size_t)p.S * p.mu);
     c.slot_layer = cv.take<int32_t>((size_t)p.mu);
     c.koff_dev = cv.take<int32_t>((size_t)p.L + 1);
+    c.layer_off_dev = cv.take<int64_t>((size_t)p.L);
+    c.ic_bytes = cv.take<unsigned char>((size_t)5 * p.mu);
     c.tile_lo = cv.take<int32_t>((size_t)((p.N + 4095) / 4096) + 1);
     carve_select(cv, c.sel_v, plan_select(p.off, p.numel, p.k_l, p.koff), p.S);
     if (ps) {
@@ -389,6 +391,8 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     koff32[p.L] = (int32_t)p.mu;
     if (e == cudaSuccess) e = upload(c->slot_layer, slot_layer, s);
     if (e == cudaSuccess) e = upload(c->koff_dev, koff32, s);
+    std::vector<int64_t> layer_off(p.off.begin(), p.off.begin() + p.L);
+    if (e == cudaSuccess) e = upload(c->layer_off_dev, layer_off, s);
     if (e == cudaSuccess && cfg->ae_kind == LGC_AE_CONV5) e = ae5_make_maps(*c);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
@@ -527,6 +531,22 @@ lgc_status lgc_ae_train_step_ps(lgc_ctx *c, int32_t common_node, float lambda_re
     cudaError_t e = launch_gather(*c);
     if (e == cudaSuccess) e = launch_train_step_ps(*c, common_node, lambda_rec, lambda_sim, loss_out);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_ae_train_step_ps");
+    return LGC_OK;
+}
+
+lgc_status lgc_encode_indices(lgc_ctx *c, int32_t node, void *stream_out, size_t capacity, uint64_t *sizes_out)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (!stream_out || !sizes_out || capacity < 4 || capacity % 4 != 0 || (reinterpret_cast<uintptr_t>(stream_out) & 3) != 0 ||
+        (reinterpret_cast<uintptr_t>(sizes_out) & 7) != 0)
+        return fail(c, LGC_ERR_INVALID_ARG, "lgc_encode_indices: buffers must be non-NULL, the stream 4-byte aligned with a capacity that is a multiple of 4");
+    if (c->stage == Ctx::kIdle || c->stage == Ctx::kAccumulated)
+        return fail(c, LGC_ERR_BAD_STATE, "lgc_encode_indices needs the index sets of this step's lgc_topk");
+    if (c->cfg.variant == LGC_VARIANT_PS ? (node < 0 || node >= c->K) : node != 0 && (node < 0 || node >= c->K))
+        return fail(c, LGC_ERR_INVALID_ARG, "node out of range");
+    const cudaError_t e = launch_encode_indices(*c, node, static_cast<unsigned char *>(stream_out), (int64_t)capacity,
+                                                reinterpret_cast<unsigned long long *>(sizes_out));
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_encode_indices");
     return LGC_OK;
 }
 

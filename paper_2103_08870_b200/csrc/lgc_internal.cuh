@@ -123,6 +123,8 @@ struct Ctx {
     float *recon = nullptr;        // [S][mu]
     int32_t *slot_layer = nullptr; // [mu] layer of each kept slot
     int32_t *koff_dev = nullptr;   // [L + 1]
+    int64_t *layer_off_dev = nullptr; // [L] first element of each layer inside a row
+    unsigned char *ic_bytes = nullptr; // [5 mu] varint form of an index list (index coding)
     int32_t *tile_lo = nullptr;    // [ceil(N / 4096) + 1] first kept slot at or after each 4096-entry tile (ring-allreduce)
     int32_t *errword = nullptr;    // device check record
     SelectTables sel_v, sel_inn;
@@ -183,6 +185,7 @@ cudaError_t launch_combine_ps(Ctx &c, int common_node);
 cudaError_t launch_decode_scatter(Ctx &c, float *update);
 cudaError_t launch_topk_scatter(Ctx &c, float *update);
 cudaError_t launch_train_step(Ctx &c, float *loss_out);
+cudaError_t launch_encode_indices(Ctx &c, int node, unsigned char *out, int64_t capacity, unsigned long long *result);
 cudaError_t launch_train_step_ps(Ctx &c, int common, float lam_rec, float lam_sim, float *loss_out);
 // full-size autoencoder (lgc_ae5.cu)
 int64_t ae5_param_count();
