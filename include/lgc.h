@@ -79,6 +79,11 @@ typedef struct {
     int32_t ae_c1, ae_c2;         /* channels of the two encoder convolutions: (8,4) or (16,8) */
     float adam_lr, adam_beta1, adam_beta2, adam_eps; /* lgc_ae_train_step; 0 selects 1e-3, 0.9, 0.999, 1e-8 */
     void *stream;                 /* cudaStream_t */
+    int64_t grad_row_stride;      /* elements between consecutive nodes' rows of the `grads` argument of
+                                     lgc_accumulate; 0 = N (rows back to back).  A larger stride lets a context
+                                     work on a run of layers inside a longer flat gradient (Section VI-A: the first
+                                     layer is sent dense and the last one without the autoencoder, so a model is
+                                     served by one context per run of layers that are treated alike) */
 } lgc_config;
 
 /* Sizes the caller must provide, in bytes.
@@ -166,6 +171,13 @@ lgc_status lgc_ae_train_step(lgc_ctx *ctx, float *loss_out);
  * the common code and the innovations of the context.  loss_out: device fp32 scalar or NULL. */
 lgc_status lgc_ae_train_step_ps(lgc_ctx *ctx, int32_t common_node, float lambda_rec, float lambda_sim,
                                 float *loss_out);
+
+/* Dense average of K rows (first training phase of Section V-B, and the layers Section VI-A leaves
+ * uncompressed): update[j] = (((g_0[j] + g_1[j]) + ...) + g_{K-1}[j]) / K in fp32, for j < n.
+ * grads: device, row k starts at grads + k * row_stride; update: device, n floats.  Needs no context;
+ * enqueued on `stream` (a cudaStream_t). */
+lgc_status lgc_dense_mean(const float *grads, int64_t row_stride, int32_t num_nodes, int64_t n, float *update,
+                          void *stream);
 
 /* Entropy coding of an index list (Section V-A: the transferred indices are DEFLATE-coded and
  * their rate counts in the compression ratio).  The ascending offsets of every layer become gaps

@@ -47,6 +47,56 @@ accumulate_kernel(const float4 *__restrict__ g4, float4 *__restrict__ u4, float4
     }
 }
 
+// The same for gradient rows that are not back to back (row k of g starts at g + k * g_stride):
+// grid (tiles of 4096 elements, K); 128-bit accesses where the addresses allow, scalars otherwise.
+__global__ void __launch_bounds__(kAccThreads)
+accumulate_rows_kernel(const float *__restrict__ g, int64_t g_stride, float *__restrict__ u, float *__restrict__ v,
+                       int64_t N, float m)
+{
+    const int row = blockIdx.y;
+    const int64_t p0 = ((int64_t)blockIdx.x * kAccThreads + threadIdx.x) * 4;
+    if (p0 >= N) return;
+    const float *gp = g + (int64_t)row * g_stride + p0;
+    float *up = u + (int64_t)row * N + p0, *vp = v + (int64_t)row * N + p0;
+    if (p0 + 4 <= N && ((reinterpret_cast<uintptr_t>(gp) | reinterpret_cast<uintptr_t>(up) | reinterpret_cast<uintptr_t>(vp)) & 15) == 0) {
+        const float4 gg = __ldcs(reinterpret_cast<const float4 *>(gp));
+        float4 uu = __ldcs(reinterpret_cast<float4 *>(up)), vv = __ldcs(reinterpret_cast<float4 *>(vp));
+        acc4(uu, vv, gg, m);
+        __stcs(reinterpret_cast<float4 *>(up), uu);
+        __stcs(reinterpret_cast<float4 *>(vp), vv);
+    } else {
+        for (int i = 0; i < 4 && p0 + i < N; ++i) {
+            const float x = __fmaf_rn(m, up[i], gp[i]);
+            up[i] = x;
+            vp[i] = __fadd_rn(vp[i], x);
+        }
+    }
+}
+
+// update[j] = node-ordered sum of the K rows, divided by K.
+__global__ void __launch_bounds__(256)
+dense_mean_kernel(const float *__restrict__ g, int64_t g_stride, int K, int64_t n, float *__restrict__ update)
+{
+    const int64_t p0 = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
+    if (p0 >= n) return;
+    const float fk = (float)K;
+    if (p0 + 4 <= n && (g_stride & 3) == 0 && ((reinterpret_cast<uintptr_t>(g + p0) | reinterpret_cast<uintptr_t>(update + p0)) & 15) == 0) {
+        float4 a = __ldcs(reinterpret_cast<const float4 *>(g + p0));
+        for (int k = 1; k < K; ++k) {
+            const float4 b = __ldcs(reinterpret_cast<const float4 *>(g + (int64_t)k * g_stride + p0));
+            a.x = __fadd_rn(a.x, b.x); a.y = __fadd_rn(a.y, b.y); a.z = __fadd_rn(a.z, b.z); a.w = __fadd_rn(a.w, b.w);
+        }
+        __stcs(reinterpret_cast<float4 *>(update + p0),
+               make_float4(__fdiv_rn(a.x, fk), __fdiv_rn(a.y, fk), __fdiv_rn(a.z, fk), __fdiv_rn(a.w, fk)));
+    } else {
+        for (int i = 0; i < 4 && p0 + i < n; ++i) {
+            float a = g[p0 + i];
+            for (int k = 1; k < K; ++k) a = __fadd_rn(a, g[(int64_t)k * g_stride + p0 + i]);
+            update[p0 + i] = __fdiv_rn(a, fk);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(256) zero_kernel(uint4 *__restrict__ p, uint64_t nvec)
 {
     const uint64_t stride = (uint64_t)gridDim.x * 256;
@@ -72,6 +122,22 @@ int sm_count()
 }
 
 }  // namespace
+
+cudaError_t launch_accumulate_rows(const float *g, int64_t g_stride, float *u, float *v, int K, int64_t N, float m,
+                                   cudaStream_t s)
+{
+    if (K <= 0 || N <= 0) return cudaSuccess;
+    const unsigned tiles = (unsigned)((N + 4 * kAccThreads - 1) / (4 * kAccThreads));
+    accumulate_rows_kernel<<<dim3(tiles, K), kAccThreads, 0, s>>>(g, g_stride, u, v, N, m), ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dense_mean(const float *g, int64_t g_stride, int K, int64_t n, float *update, cudaStream_t s)
+{
+    if (n <= 0) return cudaSuccess;
+    dense_mean_kernel<<<(unsigned)((n + 1023) / 1024), 256, 0, s>>>(g, g_stride, K, n, update), ++g_kernel_launches;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s)
 {

@@ -63,6 +63,7 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
         return fail(LGC_ERR_INVALID_ARG, "unknown ae_kind");
     if (!(cfg->momentum >= 0.0f && cfg->momentum < 1.0f)) return fail(LGC_ERR_INVALID_ARG, "momentum must be in [0, 1)");
     if (cfg->variant == LGC_VARIANT_PS && cfg->innovation_permille > 1000) return fail(LGC_ERR_INVALID_ARG, "innovation_permille > 1000");
+    if (cfg->grad_row_stride < 0) return fail(LGC_ERR_INVALID_ARG, "grad_row_stride must not be negative");
     p.K = cfg->num_nodes;
     p.L = cfg->num_layers;
     p.S = cfg->variant == LGC_VARIANT_PS ? p.K : 1;
@@ -87,6 +88,7 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
         p.kioff[l + 1] = p.kioff[l] + ki;
     }
     p.N = p.off[p.L];
+    if (cfg->grad_row_stride != 0 && cfg->grad_row_stride < p.N) return fail(LGC_ERR_INVALID_ARG, "grad_row_stride is smaller than N");
     p.mu = p.koff[p.L];
     p.muI = p.kioff[p.L];
     p.L1 = conv_len(p.mu);
@@ -423,12 +425,14 @@ lgc_status lgc_accumulate(lgc_ctx *c, const float *grads, int32_t leader_hint)
     // the fused form needs rows that start 16-byte aligned, someone to select for, and the keys two
     // previous selections left to collect against (one key says where the threshold was, two how
     // fast it moves)
-    if (c->N % 4 == 0 && c->sel_v.num_large > 0 && c->selections >= 2 && (ps || leader_hint >= 0)) {
-        e = launch_accumulate_select(c->sel_v, grads, c->u, c->v, c->K, c->N, c->cfg.momentum, ps ? 0 : leader_hint,
+    const int64_t gs = c->cfg.grad_row_stride ? c->cfg.grad_row_stride : c->N;
+    if (c->N % 4 == 0 && gs % 4 == 0 && c->sel_v.num_large > 0 && c->selections >= 2 && (ps || leader_hint >= 0)) {
+        e = launch_accumulate_select(c->sel_v, grads, gs, c->u, c->v, c->K, c->N, c->cfg.momentum, ps ? 0 : leader_hint,
                                      ps ? c->K : 1, c->epoch, c->errword, c->stream);
         c->fused_leader = ps ? -1 : leader_hint;
     } else {
-        e = launch_accumulate(grads, c->u, c->v, (uint64_t)c->K * (uint64_t)c->N, c->cfg.momentum, c->stream);
+        e = gs == c->N ? launch_accumulate(grads, c->u, c->v, (uint64_t)c->K * (uint64_t)c->N, c->cfg.momentum, c->stream)
+                       : launch_accumulate_rows(grads, gs, c->u, c->v, c->K, c->N, c->cfg.momentum, c->stream);
         c->fused_leader = -2;
     }
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_accumulate");
@@ -534,6 +538,17 @@ lgc_status lgc_ae_train_step_ps(lgc_ctx *c, int32_t common_node, float lambda_re
     return LGC_OK;
 }
 
+lgc_status lgc_dense_mean(const float *grads, int64_t row_stride, int32_t num_nodes, int64_t n, float *update, void *stream)
+{
+    if (!grads || !update || num_nodes < 1 || n < 0 || (num_nodes > 1 && row_stride < n)) {
+        g_last_error = "lgc_dense_mean: NULL buffer, no nodes, or rows that overlap";
+        return LGC_ERR_INVALID_ARG;
+    }
+    const cudaError_t e = launch_dense_mean(grads, row_stride, num_nodes, n, update, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "lgc_dense_mean");
+    return LGC_OK;
+}
+
 lgc_status lgc_encode_indices(lgc_ctx *c, int32_t node, void *stream_out, size_t capacity, uint64_t *sizes_out)
 {
     if (!c) return LGC_ERR_INVALID_ARG;
@@ -556,6 +571,8 @@ lgc_status lgc_step_host(lgc_ctx *c, const float *host_grads, float *dev_grads, 
     if (!c) return LGC_ERR_INVALID_ARG;
     if (!host_grads || !dev_grads || !dev_update || !host_update) return fail(c, LGC_ERR_INVALID_ARG, "NULL buffer");
     if (c->stage != Ctx::kIdle) return fail(c, LGC_ERR_BAD_STATE, "lgc_step_host must open a step");
+    if (c->cfg.grad_row_stride != 0 && c->cfg.grad_row_stride != c->N)
+        return fail(c, LGC_ERR_UNSUPPORTED, "lgc_step_host copies rows that are back to back: grad_row_stride must be 0 or N");
     cudaError_t e = cudaMemcpyAsync(dev_grads, host_grads, (size_t)c->K * c->N * sizeof(float), cudaMemcpyHostToDevice, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (upload)");
     lgc_status st = lgc_accumulate(c, dev_grads, choice);

@@ -165,6 +165,10 @@ extern thread_local std::string g_last_error;   // failures without a context (s
 // ---- launchers (each enqueues on ctx stream and returns the launch status) -------------------
 cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s);
 cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s);
+// rows of g are g_stride elements apart (u and v stay back to back)
+cudaError_t launch_accumulate_rows(const float *g, int64_t g_stride, float *u, float *v, int K, int64_t N, float m,
+                                   cudaStream_t s);
+cudaError_t launch_dense_mean(const float *g, int64_t g_stride, int K, int64_t n, float *update, cudaStream_t s);
 // served: the accumulation of step `epoch` collected the candidates of exactly these rows.
 // clear/clear_floats: optional 16-byte aligned buffer that spare CTAs of the finishing launch set to zero
 // (only when the tables have large segments).
@@ -172,9 +176,10 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
                           int rows, int32_t *out, int64_t out_stride, bool served, int32_t epoch, float *clear,
                           int64_t clear_floats, int32_t *errword, cudaStream_t s);
 // Accumulation that also collects the selection candidates of the selecting rows (sel_row0 .. +sel_rows
-// of the K rows) against the predicted buckets; needs N % 4 == 0.
-cudaError_t launch_accumulate_select(const SelectTables &t, const float *g, float *u, float *v, int K, int64_t N,
-                                     float m, int sel_row0, int sel_rows, int32_t epoch, int32_t *errword,
+// of the K rows) against the predicted buckets; needs N % 4 == 0 and g_stride % 4 == 0 (rows of g are
+// g_stride elements apart).
+cudaError_t launch_accumulate_select(const SelectTables &t, const float *g, int64_t g_stride, float *u, float *v, int K,
+                                     int64_t N, float m, int sel_row0, int sel_rows, int32_t epoch, int32_t *errword,
                                      cudaStream_t s);
 cudaError_t launch_select_multipass(const SelectTables &t, const float *data, int64_t row_stride, int row0,
                                     int rows, int32_t *out, int64_t out_stride, int32_t *errword, cudaStream_t s);

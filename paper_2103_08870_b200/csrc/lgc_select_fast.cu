@@ -924,8 +924,8 @@ __device__ __forceinline__ void acc4(float4 &u, float4 &v, const float4 &g, floa
 }
 
 __global__ void __launch_bounds__(kAccThreads, 2)
-accumulate_select_kernel(FastArgs f, const float *__restrict__ g, float *__restrict__ u, float *__restrict__ v,
-                         int64_t N, float m, int sel_row0, int sel_rows)
+accumulate_select_kernel(FastArgs f, const float *__restrict__ g, int64_t g_stride, float *__restrict__ u,
+                         float *__restrict__ v, int64_t N, float m, int sel_row0, int sel_rows)
 {
     __shared__ unsigned warp_u[kAccThreads / 32];
     const int row = blockIdx.y, q = blockIdx.x;
@@ -947,7 +947,7 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, float *__restr
     float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
     if (live) {
         const int64_t e = ((int64_t)row * N + tile_base + p0) >> 2;
-        const float4 gg = __ldcs(reinterpret_cast<const float4 *>(g) + e);
+        const float4 gg = __ldcs(reinterpret_cast<const float4 *>(g) + (((int64_t)row * g_stride + tile_base + p0) >> 2));
         float4 uu = __ldcs(reinterpret_cast<float4 *>(u) + e);
         vv = __ldcs(reinterpret_cast<float4 *>(v) + e);
         acc4(uu, vv, gg, m);
@@ -1048,13 +1048,13 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
     return cudaGetLastError();
 }
 
-cudaError_t launch_accumulate_select(const SelectTables &t, const float *g, float *u, float *v, int K, int64_t N,
-                                     float m, int sel_row0, int sel_rows, int32_t epoch, int32_t *errword,
+cudaError_t launch_accumulate_select(const SelectTables &t, const float *g, int64_t g_stride, float *u, float *v, int K,
+                                     int64_t N, float m, int sel_row0, int sel_rows, int32_t epoch, int32_t *errword,
                                      cudaStream_t st)
 {
     FastArgs f;
     fill_args(f, t, v, N, 0, nullptr, 0, epoch, errword);
-    accumulate_select_kernel<<<dim3(t.tiles_per_row, K), kAccThreads, 0, st>>>(f, g, u, v, N, m, sel_row0, sel_rows),
+    accumulate_select_kernel<<<dim3(t.tiles_per_row, K), kAccThreads, 0, st>>>(f, g, g_stride, u, v, N, m, sel_row0, sel_rows),
         ++g_kernel_launches;
     return cudaGetLastError();
 }

@@ -22,7 +22,7 @@ AE_CONV2, AE_IDENTITY, AE_CONV5 = 0, 1, 2
 EXPORTS = (
     "lgc_workspace_bytes", "lgc_init", "lgc_destroy", "lgc_accumulate", "lgc_topk", "lgc_encode",
     "lgc_combine", "lgc_decode_scatter", "lgc_topk_scatter", "lgc_ae_train_step", "lgc_ae_train_step_ps",
-    "lgc_encode_indices", "lgc_step_host",
+    "lgc_encode_indices", "lgc_dense_mean", "lgc_step_host",
     "lgc_get_layout", "lgc_keep_counts", "lgc_get_buffers", "lgc_set_ae_params", "lgc_get_ae_params",
     "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc", "lgc_kernel_launches", "lgc_selection_stats",
 )
@@ -35,7 +35,7 @@ class lgc_config(C.Structure):
         ("density_ppm", C.c_uint32), ("innovation_permille", C.c_uint32), ("momentum", C.c_float),
         ("variant", C.c_int32), ("ae_kind", C.c_int32), ("ae_c1", C.c_int32), ("ae_c2", C.c_int32),
         ("adam_lr", C.c_float), ("adam_beta1", C.c_float), ("adam_beta2", C.c_float), ("adam_eps", C.c_float),
-        ("stream", C.c_void_p),
+        ("stream", C.c_void_p), ("grad_row_stride", C.c_int64),
     ]
 
 
@@ -62,6 +62,7 @@ def lib() -> C.CDLL:
         l.lgc_ae_train_step.argtypes = [vp, vp]
         l.lgc_ae_train_step_ps.argtypes = [vp, C.c_int32, C.c_float, C.c_float, vp]
         l.lgc_encode_indices.argtypes = [vp, C.c_int32, vp, C.c_size_t, vp]
+        l.lgc_dense_mean.argtypes = [vp, C.c_int64, C.c_int32, C.c_int64, vp, vp]
         l.lgc_step_host.argtypes = [vp, vp, vp, vp, vp, C.c_int32]
         l.lgc_get_layout.argtypes = [vp] + [C.POINTER(C.c_int64)] * 5
         l.lgc_keep_counts.argtypes = [vp]
@@ -89,6 +90,20 @@ class LGCError(RuntimeError):
         self.status = status
         name = lib().lgc_status_string(status).decode()
         super().__init__(f"{where}: {name}" + (f" ({detail})" if detail else ""))
+
+
+def dense_mean(grads: torch.Tensor, update: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """update[j] = node-ordered mean over the K rows of `grads` ([K][n] fp32 CUDA view, unit column stride)."""
+    if not (grads.is_cuda and grads.dtype == torch.float32 and grads.dim() == 2 and grads.stride(1) == 1):
+        raise ValueError("grads: need a 2-D fp32 CUDA view with unit column stride")
+    K, n = grads.shape
+    if not (update.is_cuda and update.dtype == torch.float32 and update.is_contiguous() and update.numel() == n):
+        raise ValueError(f"update: need a contiguous fp32 CUDA tensor of {n} elements")
+    st = stream if stream is not None else torch.cuda.current_stream(grads.device)
+    status = lib().lgc_dense_mean(grads.data_ptr(), grads.stride(0) if K > 1 else n, K, n, update.data_ptr(),
+                                  C.c_void_p(st.cuda_stream))
+    if status != LGC_OK:
+        raise LGCError(status, "lgc_dense_mean", lib().lgc_last_error(None).decode())
 
 
 def topk_noalloc(v: torch.Tensor, k: int, idx_out: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
@@ -125,7 +140,7 @@ class LGC:
                  momentum: float = 0.9, variant: str = "rar", ae_kind: str = "conv2", c1: int = 8,
                  c2: int = 4, innovation_permille: int = 100, lr: float = 0.0, beta1: float = 0.0,
                  beta2: float = 0.0, eps: float = 0.0, device: Optional[torch.device] = None,
-                 stream: Optional[torch.cuda.Stream] = None):
+                 stream: Optional[torch.cuda.Stream] = None, grad_row_stride: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2103_08870_b200.lgc needs a CUDA device; there is no CPU path")
         self._l = lib()
@@ -139,7 +154,8 @@ class LGC:
             variant={"rar": VARIANT_RAR, "ps": VARIANT_PS}[variant],
             ae_kind={"conv2": AE_CONV2, "identity": AE_IDENTITY, "conv5": AE_CONV5}[ae_kind], ae_c1=c1, ae_c2=c2,
             adam_lr=lr, adam_beta1=beta1, adam_beta2=beta2, adam_eps=eps,
-            stream=C.c_void_p(self.stream.cuda_stream))
+            stream=C.c_void_p(self.stream.cuda_stream), grad_row_stride=grad_row_stride)
+        self.grad_row_stride = grad_row_stride
         self.variant, self.ae_kind, self.K, self.c1, self.c2 = variant, ae_kind, num_nodes, c1, c2
         sb, wb, pb = C.c_size_t(), C.c_size_t(), C.c_size_t()
         self._ctx = C.c_void_p()
@@ -190,8 +206,15 @@ class LGC:
 
     # -- the stages ---------------------------------------------------------------------------
     def accumulate(self, grads: torch.Tensor, leader_hint: int = -1) -> None:
-        self._ok(self._l.lgc_accumulate(self._ctx, self._dev_f32(grads, self.K * self.N, "grads"), leader_hint),
-                 "lgc_accumulate")
+        """grads: fp32 CUDA, K x N; with a grad_row_stride a [K][N] view whose rows are that far apart."""
+        if self.grad_row_stride:
+            if not (grads.is_cuda and grads.dtype == torch.float32 and tuple(grads.shape) == (self.K, self.N)
+                    and grads.stride(1) == 1 and (self.K == 1 or grads.stride(0) == self.grad_row_stride)):
+                raise ValueError("grads: need a [K][N] fp32 CUDA view with unit column stride and the configured row stride")
+            ptr = grads.data_ptr()
+        else:
+            ptr = self._dev_f32(grads, self.K * self.N, "grads")
+        self._ok(self._l.lgc_accumulate(self._ctx, ptr, leader_hint), "lgc_accumulate")
 
     def topk(self, leader: int = 0, update_hint: Optional[torch.Tensor] = None) -> None:
         ptr = self._dev_f32(update_hint, self.N, "update_hint") if update_hint is not None else None

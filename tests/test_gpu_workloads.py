@@ -173,3 +173,30 @@ def test_stress_config_sampled():
         assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_s, f"sampled v after clearing, step {t}")
         assert not gpu.v[:, idx_dev].any().item() and not gpu.u[:, idx_dev].any().item()
         gpu.check()
+
+
+def test_resnet50_config_with_the_layer_treatment_of_the_paper():
+    # Section VI-A on the ResNet-50-shaped table: first tensor dense, the classifier's two tensors top-k only,
+    # everything in between through the autoencoder; one step of each phase of Section V-B and two more compressed
+    from oracle.phases import OraclePhased
+    from paper_2103_08870_b200.phases import PhasedLGC
+    w = W.workload("resnet50")
+    K, numel = w.num_nodes, w.table.numel
+    modes = ["dense"] + ["ae"] * (len(numel) - 3) + ["topk", "topk"]
+    params = W.ae_init_params(w.ae_c1, w.ae_c2, "rar", K, w.seed)
+    gpu = PhasedLGC(numel, modes, K, density_ppm=w.density_ppm, momentum=w.momentum)
+    gpu.ae_runs()[0].ctx.set_ae_params(params)
+    ora = OraclePhased(numel, modes, K, {1: params.numpy()}, density_ppm=w.density_ppm, momentum=w.momentum)
+    src = W.GradientSource(w.table, K, seed=w.seed, device="cuda")
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    g = torch.empty((K, gpu.N), dtype=torch.float32, device="cuda")
+    for t, phase in enumerate(["raw", "topk_train", "compressed", "compressed", "compressed"]):
+        src.step_into(t, g)
+        choice = W.choice_for_step(w.seed, t, K)
+        gpu.step(g, upd, phase, choice)
+        ref, _ = ora.step(g.cpu().numpy(), phase, choice)
+        assert_close(upd.cpu().numpy(), ref, f"step {t} ({phase}): update")
+    for r, gr in zip(gpu.runs, ora.groups):
+        if r.ctx is not None:
+            assert_bitwise(r.ctx.v.cpu().numpy(), gr["o"].v, f"residual of the {r.mode} run")
+    gpu.check()
