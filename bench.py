@@ -229,7 +229,7 @@ def run_ours(args, w: W.Workload):
     acc_ms = [a.elapsed_time(b) for a, b in ev]
 
     # end to end through host buffers: pinned gradients in, dense update out, every step
-    e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 5))
+    e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 20))
     e2e_ms = 0.0
     if e2e_steps:
         host_g = torch.empty((K, N), dtype=torch.float32).pin_memory()

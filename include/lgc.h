@@ -191,10 +191,19 @@ lgc_status lgc_dense_mean(const float *grads, int64_t row_stride, int32_t num_no
  * Valid from lgc_topk until the next lgc_accumulate. */
 lgc_status lgc_encode_indices(lgc_ctx *ctx, int32_t node, void *stream_out, size_t capacity, uint64_t *sizes_out);
 
-/* A whole compression step from host memory: copies `host_grads` ([K][N], ideally pinned) to
- * `dev_grads`, runs the five stages, copies the dense update back to `host_update` ([N]).
- * Everything is enqueued on the context's stream; the call returns without waiting.
- * `choice` is the leader (ring-allreduce) or the common node (parameter server). */
+/* A whole compression step from host memory: uploads `host_grads` ([K][N], ideally pinned) to
+ * `dev_grads`, runs the five stages, downloads the dense update to `host_update` ([N]).
+ * The call returns without waiting; when the context's stream has drained, `host_update` is
+ * complete.  `choice` is the leader (ring-allreduce) or the common node (parameter server).
+ * The upload goes node by node over a stream of the library's own (created at the first call,
+ * released by lgc_destroy), and each node's row is accumulated as soon as it has arrived, so
+ * stage 1 hides under the transfer; the download stays on the context's stream.  The upload of
+ * one call waits for the scatter of the previous lgc_step_host, not for that call's download:
+ * back-to-back calls keep both directions of the bus busy.  From the moment of the call
+ * `host_grads` and `dev_grads` belong to it: the upload does not wait for work the caller
+ * queued on the context's stream after the previous lgc_step_host, so such work must not touch
+ * `dev_grads`, and `host_grads` must already hold the gradients.  Results are bit for bit those
+ * of the five stage calls. */
 lgc_status lgc_step_host(lgc_ctx *ctx, const float *host_grads, float *dev_grads, float *dev_update,
                          float *host_update, int32_t choice);
 

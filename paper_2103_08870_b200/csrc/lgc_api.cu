@@ -408,34 +408,62 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
 
 lgc_status lgc_destroy(lgc_ctx *ctx)
 {
+    if (ctx) {
+        for (cudaEvent_t e : ctx->row_uploaded) cudaEventDestroy(e);
+        if (ctx->tail_done) cudaEventDestroy(ctx->tail_done);
+        if (ctx->upload_stream) cudaStreamDestroy(ctx->upload_stream);
+    }
     delete ctx;
     return LGC_OK;
 }
 
-lgc_status lgc_accumulate(lgc_ctx *c, const float *grads, int32_t leader_hint)
+namespace {
+
+// Opens a step: checks, advances the step counter and decides whether the accumulation also collects
+// selection candidates.  The fused form needs rows that start 16-byte aligned, someone to select for,
+// and the keys two previous selections left to collect against (one key says where the threshold was,
+// two how fast it moves).
+lgc_status open_step(lgc_ctx *c, const float *grads, int32_t leader_hint, bool *fused)
 {
-    if (!c) return LGC_ERR_INVALID_ARG;
     if (!grads || !aligned16(grads)) return fail(c, LGC_ERR_INVALID_ARG, "grads is NULL or not 16-byte aligned");
     if (c->stage != Ctx::kIdle) return fail(c, LGC_ERR_BAD_STATE, "lgc_accumulate must open a step");
     const bool ps = c->cfg.variant == LGC_VARIANT_PS;
     if (!ps && leader_hint >= c->K) return fail(c, LGC_ERR_INVALID_ARG, "leader_hint out of range");
     c->epoch = c->epoch == 0x7fffffff ? 1 : c->epoch + 1;
     c->cleared_update = nullptr;
-    cudaError_t e;
-    // the fused form needs rows that start 16-byte aligned, someone to select for, and the keys two
-    // previous selections left to collect against (one key says where the threshold was, two how
-    // fast it moves)
     const int64_t gs = c->cfg.grad_row_stride ? c->cfg.grad_row_stride : c->N;
-    if (c->N % 4 == 0 && gs % 4 == 0 && c->sel_v.num_large > 0 && c->selections >= 2 && (ps || leader_hint >= 0)) {
-        e = launch_accumulate_select(c->sel_v, grads, gs, c->u, c->v, c->K, c->N, c->cfg.momentum, ps ? 0 : leader_hint,
-                                     ps ? c->K : 1, c->epoch, c->errword, c->stream);
-        c->fused_leader = ps ? -1 : leader_hint;
-    } else {
-        e = gs == c->N ? launch_accumulate(grads, c->u, c->v, (uint64_t)c->K * (uint64_t)c->N, c->cfg.momentum, c->stream)
-                       : launch_accumulate_rows(grads, gs, c->u, c->v, c->K, c->N, c->cfg.momentum, c->stream);
-        c->fused_leader = -2;
-    }
+    *fused = c->N % 4 == 0 && gs % 4 == 0 && c->sel_v.num_large > 0 && c->selections >= 2 && (ps || leader_hint >= 0);
+    c->fused_leader = *fused ? (ps ? -1 : leader_hint) : -2;
+    return LGC_OK;
+}
+
+// Stage 1 for the nodes r0 .. r1 - 1 of an opened step.  Every element is updated by the same two
+// operations whichever kernel and however many launches serve it.
+cudaError_t accumulate_nodes(lgc_ctx *c, const float *grads, int32_t leader_hint, bool fused, int r0, int r1)
+{
+    const bool ps = c->cfg.variant == LGC_VARIANT_PS;
+    const int64_t gs = c->cfg.grad_row_stride ? c->cfg.grad_row_stride : c->N;
+    const float *g = grads + (int64_t)r0 * gs;
+    float *u = c->u + (int64_t)r0 * c->N, *v = c->v + (int64_t)r0 * c->N;
+    if (fused)   // the kernel's row y is node r0 + y; node n selects into table row n (parameter server) or 0 (the leader)
+        return launch_accumulate_select(c->sel_v, g, gs, u, v, r1 - r0, c->N, c->cfg.momentum, (ps ? 0 : leader_hint) - r0,
+                                        ps ? c->K : 1, c->epoch, c->errword, c->stream);
+    if (gs == c->N && r0 == 0 && r1 == c->K)
+        return launch_accumulate(g, u, v, (uint64_t)c->K * (uint64_t)c->N, c->cfg.momentum, c->stream);
+    return launch_accumulate_rows(g, gs, u, v, r1 - r0, c->N, c->cfg.momentum, c->stream);
+}
+
+}  // namespace
+
+lgc_status lgc_accumulate(lgc_ctx *c, const float *grads, int32_t leader_hint)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    bool fused;
+    const lgc_status st = open_step(c, grads, leader_hint, &fused);
+    if (st != LGC_OK) return st;
+    const cudaError_t e = accumulate_nodes(c, grads, leader_hint, fused, 0, c->K);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_accumulate");
+    c->tail_recorded = false;      // a later lgc_step_host orders its upload behind this step
     c->stage = Ctx::kAccumulated;
     return LGC_OK;
 }
@@ -573,15 +601,49 @@ lgc_status lgc_step_host(lgc_ctx *c, const float *host_grads, float *dev_grads, 
     if (c->stage != Ctx::kIdle) return fail(c, LGC_ERR_BAD_STATE, "lgc_step_host must open a step");
     if (c->cfg.grad_row_stride != 0 && c->cfg.grad_row_stride != c->N)
         return fail(c, LGC_ERR_UNSUPPORTED, "lgc_step_host copies rows that are back to back: grad_row_stride must be 0 or N");
-    cudaError_t e = cudaMemcpyAsync(dev_grads, host_grads, (size_t)c->K * c->N * sizeof(float), cudaMemcpyHostToDevice, c->stream);
-    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (upload)");
-    lgc_status st = lgc_accumulate(c, dev_grads, choice);
-    if (st == LGC_OK) st = lgc_topk(c, choice, dev_update);
+    cudaError_t e = cudaSuccess;
+    if (!c->upload_stream) {
+        e = cudaStreamCreateWithFlags(&c->upload_stream, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->tail_done, cudaEventDisableTiming);
+        for (int k = 0; e == cudaSuccess && k < c->K; ++k) {
+            cudaEvent_t ev = nullptr;
+            e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+            if (e == cudaSuccess) c->row_uploaded.push_back(ev);
+        }
+        if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (streams)");
+    }
+    // The upload may begin once everything queued on the context's stream up to the previous call's
+    // scatter has run (that call's download may still be on the bus: the two directions overlap).
+    if (!c->tail_recorded) e = cudaEventRecord(c->tail_done, c->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(c->upload_stream, c->tail_done, 0);
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (order)");
+    bool fused;
+    lgc_status st = open_step(c, dev_grads, choice, &fused);
+    if (st != LGC_OK) return st;
+    // node by node: row k is accumulated while rows k+1.. are still being uploaded
+    const size_t row_bytes = (size_t)c->N * sizeof(float);
+    const bool by_rows = c->N % 4 == 0;           // rows of dev_grads, u and v then start 16-byte aligned
+    for (int k = 0; k < c->K; ++k) {
+        e = cudaMemcpyAsync(dev_grads + (int64_t)k * c->N, host_grads + (int64_t)k * c->N, row_bytes, cudaMemcpyHostToDevice,
+                            c->upload_stream);
+        if (e == cudaSuccess && (by_rows || k == c->K - 1)) {
+            e = cudaEventRecord(c->row_uploaded[k], c->upload_stream);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(c->stream, c->row_uploaded[k], 0);
+            if (e == cudaSuccess) e = by_rows ? accumulate_nodes(c, dev_grads, choice, fused, k, k + 1)
+                                              : accumulate_nodes(c, dev_grads, choice, fused, 0, c->K);
+        }
+        if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (upload)");
+    }
+    c->stage = Ctx::kAccumulated;
+    st = lgc_topk(c, choice, dev_update);
     if (st == LGC_OK) st = lgc_encode(c);
     if (st == LGC_OK) st = lgc_combine(c, choice);
     if (st == LGC_OK) st = lgc_decode_scatter(c, dev_update);
     if (st != LGC_OK) return st;
-    e = cudaMemcpyAsync(host_update, dev_update, (size_t)c->N * sizeof(float), cudaMemcpyDeviceToHost, c->stream);
+    e = cudaEventRecord(c->tail_done, c->stream);
+    c->tail_recorded = e == cudaSuccess;
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(host_update, dev_update, (size_t)c->N * sizeof(float), cudaMemcpyDeviceToHost, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (download)");
     return LGC_OK;
 }

@@ -156,6 +156,12 @@ struct Ctx {
     bool val_valid = false;        // val holds the kept values of the current selection
     bool tile_lo_valid = false;    // tile_lo matches the current selection
     bool mean_valid = false;       // combined holds the mean code of the current selection
+    // lgc_step_host: the upload runs row by row on a stream of the library's own, so that rows are
+    // accumulated while later rows are still on the bus (created at the first call, released by lgc_destroy)
+    cudaStream_t upload_stream = nullptr;
+    std::vector<cudaEvent_t> row_uploaded;   // [K]
+    cudaEvent_t tail_done = nullptr;         // the previous lgc_step_host has finished with dev_grads (before its download)
+    bool tail_recorded = false;
     std::string err;
 };
 

@@ -330,3 +330,35 @@ def test_step_from_host_buffers():
     ref = ora.step(g.numpy(), 1)
     assert_close(hu.numpy(), ref, "update through host buffers")
     assert_bitwise(gpu.v.cpu().numpy(), ora.v, "v")
+
+
+@pytest.mark.parametrize("variant,K,extra", [("rar", 3, []), ("ps", 2, []), ("rar", 2, [2])])
+def test_steps_from_host_buffers_back_to_back(variant, K, extra):
+    # Six calls queued without waiting in between: each node's row is accumulated as it arrives
+    # (from the third step on by the kernel that also collects the selection candidates), the
+    # upload of one call overlaps the download of the one before.  extra = [2]: N % 4 != 0, rows
+    # do not start 16-byte aligned and the step falls back to one accumulation of all rows.
+    numel = TOY + extra
+    steps = 6
+    ora, gpu = make_pair(numel, K, variant=variant)
+    src = toy_source(numel, K)
+    gs = [src.step(t) for t in range(steps)]
+    hg = [g.clone().pin_memory() for g in gs]
+    hu = [torch.full((gpu.N,), float("nan"), dtype=torch.float32).pin_memory() for _ in range(steps)]
+    dg = torch.empty(K, gpu.N, device="cuda")
+    du = torch.empty(gpu.N, device="cuda")
+    choices = [W.choice_for_step(7, t, K) for t in range(steps)]
+    for t in range(steps):
+        gpu.step_host(hg[t], dg, du, hu[t], choices[t])
+    torch.cuda.synchronize()
+    for t in range(steps):
+        ref = ora.step(gs[t].numpy(), choices[t])
+        assert_close(hu[t].numpy(), ref, f"update of step {t} through host buffers")
+    assert_bitwise(gpu.u.cpu().numpy(), ora.u, "u")
+    assert_bitwise(gpu.v.cpu().numpy(), ora.v, "v")
+    idx_ref = ora.idx if variant == "ps" else ora.idx[:1]
+    assert_bitwise(gpu.idx.cpu().numpy(), idx_ref, "selected indices of the last step")
+    if (gpu.N % 4) == 0:
+        large, served, _, _, _ = gpu.selection_stats()
+        assert large > 0 and served > 0, "the row-by-row accumulation did not collect any candidates"
+    gpu.check()
