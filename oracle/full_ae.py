@@ -24,7 +24,9 @@ Readings where the paper is silent or at odds with itself:
 
 Every function is the layer's defining sum written out with numpy slices; no blocking, no
 reordering.  Pinned in tests/test_oracle_full_ae.py against torch's CPU convolutions, the
-parameter counts the tables imply, and the length chain.
+parameter counts the tables imply, and the length chain.  The training step (loss of Section
+IV-B, derivative of every layer, written the same way) is pinned there against torch's autograd
+on the same graph, central differences of the loss, and the cases where loss and gradients vanish.
 """
 from __future__ import annotations
 
@@ -142,3 +144,112 @@ def rar_forward(val: np.ndarray, p: Dict[str, np.ndarray]):
         acc = acc + z[k]
     zbar = acc / float(K)
     return z, zbar, decode(zbar, p, mu)
+
+
+# ---- training step of the ring-allreduce form (Section IV-B: the reconstruction of the averaged
+# code is compared with the average of the nodes' vectors; Section V-B trains on the kept values) ----
+#
+# Each *_bwd function is the derivative of the layer's defining sum above, written the same way:
+# given dL/dy it adds dL/dw and dL/db into gw / gb and returns dL/dx.
+
+def leaky_bwd(pre: np.ndarray, dy: np.ndarray) -> np.ndarray:
+    return np.where(pre > 0, dy, SLOPE * dy)
+
+
+def conv_k3s2_bwd(x, w, dy, gw, gb, want_dx=True):
+    lout = dy.shape[1]
+    gb += dy.sum(axis=1)
+    dx = np.zeros_like(x) if want_dx else None
+    for tau in range(3):
+        xs = x[:, tau:tau + 2 * (lout - 1) + 1:2]
+        gw[:, :, tau] += dy @ xs.T
+        if want_dx:
+            dx[:, tau:tau + 2 * (lout - 1) + 1:2] += w[:, :, tau].T @ dy
+    return dx
+
+
+def conv_k1_bwd(x, w, dy, gw, gb):
+    gb += dy.sum(axis=1)
+    gw[:, :, 0] += dy @ x.T
+    return w[:, :, 0].T @ dy
+
+
+def convt_k3s2_bwd(x, w, dy, gw, gb):
+    lin = x.shape[1]
+    gb += dy.sum(axis=1)
+    dx = np.zeros_like(x)
+    for tau in range(3):
+        dys = dy[:, tau:tau + 2 * (lin - 1) + 1:2]
+        gw[:, :, tau] += x @ dys.T
+        dx += w[:, :, tau] @ dys
+    return dx
+
+
+def convt_k3s1p1_bwd(x, w, dy, gw, gb):
+    lin = x.shape[1]
+    gb += dy.sum(axis=1)
+    dx = np.zeros_like(x)
+    for tau in range(3):
+        lo, hi = max(0, 1 - tau), min(lin, lin + 1 - tau)      # inputs j whose target j + tau - 1 exists
+        dys = dy[:, lo + tau - 1:hi + tau - 1]
+        gw[:, :, tau] += x[:, lo:hi] @ dys.T
+        dx[:, lo:hi] += w[:, :, tau] @ dys
+    return dx
+
+
+def rar_loss_and_grads(val: np.ndarray, p: Dict[str, np.ndarray]):
+    """loss = (1/mu) || D_c((1/K) sum_k E_c(val_k)) - (1/K) sum_k val_k ||^2 and dloss/dparameter
+    for every tensor of param_shapes()."""
+    val = np.asarray(val, dtype=np.float64)
+    K, mu = val.shape
+    ln = lengths(mu)
+    g = {name: np.zeros(shape, dtype=np.float64) for name, shape in param_shapes()}
+    # forward, keeping every layer's input and pre-activation
+    enc_in, enc_pre, codes = [], [], []
+    for k in range(K):
+        h = val[k].reshape(1, -1)
+        ins, pres = [], []
+        for i in range(1, 5):
+            ins.append(h)
+            pre = conv_k3s2(h, p[f"enc.w{i}"], p[f"enc.b{i}"])
+            pres.append(pre)
+            h = leaky(pre)
+        ins.append(h)
+        codes.append(conv_k1(h, p["enc.w5"], p["enc.b5"]))
+        enc_in.append(ins)
+        enc_pre.append(pres)
+    acc = np.zeros_like(codes[0])
+    for k in range(K):
+        acc = acc + codes[k]
+    zbar = acc / float(K)
+    dec_in, dec_pre = [zbar], []
+    pre = convt_k3s1p1(zbar, p["dec.w1"], p["dec.b1"])
+    dec_pre.append(pre)
+    d = leaky(pre)
+    for i in range(2, 6):
+        dec_in.append(d)
+        pre = convt_k3s2(d, p[f"dec.w{i}"], p[f"dec.b{i}"], (ln[5 - i] - 3) % 2)
+        dec_pre.append(pre)
+        d = leaky(pre)
+    dec_in.append(d)
+    r = conv_k1(d, p["dec.w6"], p["dec.b6"]).reshape(-1)
+    target = np.zeros(mu)
+    for k in range(K):
+        target = target + val[k]
+    target = target / float(K)
+    diff = r - target
+    loss = float(np.sum(diff * diff) / mu)
+    # backward
+    dy = (2.0 * diff / mu).reshape(1, -1)
+    dd = conv_k1_bwd(dec_in[5], p["dec.w6"], dy, g["dec.w6"], g["dec.b6"])
+    for i in range(5, 1, -1):
+        dd = leaky_bwd(dec_pre[i - 1], dd)
+        dd = convt_k3s2_bwd(dec_in[i - 1], p[f"dec.w{i}"], dd, g[f"dec.w{i}"], g[f"dec.b{i}"])
+    dd = leaky_bwd(dec_pre[0], dd)
+    dzbar = convt_k3s1p1_bwd(dec_in[0], p["dec.w1"], dd, g["dec.w1"], g["dec.b1"])
+    for k in range(K):
+        dh = conv_k1_bwd(enc_in[k][4], p["enc.w5"], dzbar / float(K), g["enc.w5"], g["enc.b5"])
+        for i in range(4, 0, -1):
+            dh = leaky_bwd(enc_pre[k][i - 1], dh)
+            dh = conv_k3s2_bwd(enc_in[k][i - 1], p[f"enc.w{i}"], dh, g[f"enc.w{i}"], g[f"enc.b{i}"], want_dx=i > 1)
+    return loss, g

@@ -196,7 +196,9 @@ class OracleLGC:
     # -- autoencoder training (ring-allreduce loss, Sec. IV-B) ----------------------------
     def ae_loss_and_grads(self):
         """loss = (1/mu) || D_c(mean_k E_c(g~_k)) - mean_k g~_k ||^2 and its parameter gradients."""
-        assert self.variant == "rar" and self.ae_kind == "conv2"
+        assert self.variant == "rar" and self.ae_kind in ("conv2", "conv5")
+        if self.ae_kind == "conv5":          # the paper's full-size autoencoder (Section IV-C)
+            return A5.rar_loss_and_grads(self.val, self.p)
         K, mu = self.K, self.mu
         xs = [self.val[k].astype(np.float64).reshape(1, -1) for k in range(K)]
         hs, zs = [], []

@@ -111,3 +111,98 @@ def test_identical_nodes_average_to_their_own_code():
     z, zbar, r = A.rar_forward(np.stack([x] * 4), p)
     assert np.array_equal(zbar, z[0])                       # K a power of two: exact
     assert np.array_equal(r, A.decode(A.encode(x, p), p, 200))
+
+
+# ---- training step (ring-allreduce reconstruction loss of Section IV-B on the full-size autoencoder) ----
+
+def flat_grads(g):
+    return np.concatenate([g[name].reshape(-1) for name, _ in A.param_shapes()])
+
+
+@pytest.mark.parametrize("mu, K", [(61, 1), (100, 3), (130, 2)])
+def test_training_gradients_against_torch_autograd(mu, K):
+    # the same graph built from torch's CPU convolutions, differentiated by autograd
+    rng = np.random.default_rng(mu + K)
+    val = rng.standard_normal((K, mu)).astype(np.float32)
+    flat = rand_params(mu)
+    loss, g = A.rar_loss_and_grads(val, A.unpack(flat))
+    tp = {k: torch.from_numpy(np.ascontiguousarray(v)).requires_grad_(True) for k, v in A.unpack(flat).items()}
+    ln = A.lengths(mu)
+    zs = []
+    for k in range(K):
+        h = torch.from_numpy(val[k].astype(np.float64)).reshape(1, 1, -1)
+        for i in range(1, 5):
+            h = F.leaky_relu(F.conv1d(h, tp[f"enc.w{i}"], tp[f"enc.b{i}"], stride=2), 0.01)
+        zs.append(F.conv1d(h, tp["enc.w5"], tp["enc.b5"]))
+    zbar = sum(zs[1:], zs[0]) / K
+    d = F.leaky_relu(F.conv_transpose1d(zbar, tp["dec.w1"], tp["dec.b1"], stride=1, padding=1), 0.01)
+    for i in range(2, 6):
+        d = F.leaky_relu(F.conv_transpose1d(d, tp[f"dec.w{i}"], tp[f"dec.b{i}"], stride=2,
+                                            output_padding=(ln[5 - i] - 3) % 2), 0.01)
+    r = F.conv1d(d, tp["dec.w6"], tp["dec.b6"]).reshape(-1)
+    target = torch.from_numpy(val.astype(np.float64)).sum(0) / K
+    tl = ((r - target) ** 2).sum() / mu
+    tl.backward()
+    assert abs(loss - tl.item()) <= 1e-12 * max(1.0, abs(tl.item()))
+    for name, _ in A.param_shapes():
+        ref = tp[name].grad.numpy()
+        assert np.abs(g[name] - ref).max() <= 1e-10 * max(1e-3, np.abs(ref).max()), name
+
+
+def test_training_gradients_against_finite_differences():
+    # central differences of the loss itself, on parameters drawn from every tensor
+    rng = np.random.default_rng(17)
+    mu, K = 75, 2
+    val = rng.standard_normal((K, mu)).astype(np.float32)
+    flat = rand_params(17)
+    _, g = A.rar_loss_and_grads(val, A.unpack(flat))
+    gf = flat_grads(g)
+    pos, picks = 0, []
+    for _, shape in A.param_shapes():
+        n = int(np.prod(shape))
+        picks += list(pos + rng.choice(n, size=min(3, n), replace=False))
+        pos += n
+    eps = 1e-6
+    for i in picks:
+        hi, lo = flat.copy(), flat.copy()
+        hi[i] += eps
+        lo[i] -= eps
+        fd = (A.rar_loss_and_grads(val, A.unpack(hi))[0] - A.rar_loss_and_grads(val, A.unpack(lo))[0]) / (2 * eps)
+        assert abs(fd - gf[i]) <= 1e-5 * max(1e-3, abs(gf[i])) + 1e-8, (i, fd, gf[i])
+
+
+def test_training_loss_is_the_forward_pass_error_and_vanishes_for_a_perfect_decoder():
+    rng = np.random.default_rng(4)
+    val = rng.standard_normal((3, 90)).astype(np.float32)
+    p = A.unpack(rand_params(4))
+    loss, _ = A.rar_loss_and_grads(val, p)
+    _, _, r = A.rar_forward(val, p)
+    target = (val[0].astype(np.float64) + val[1] + val[2]) / 3.0
+    assert abs(loss - np.sum((r - target) ** 2) / 90) <= 1e-15 * max(1.0, loss)
+    # zero weights in the last layer and a target that equals its bias: loss 0, and only the
+    # last layer's weights can have a gradient (which is zero too, the error being zero)
+    flat = rand_params(5)
+    q = A.unpack(flat)
+    q["dec.w6"][...] = 0.0
+    q["dec.b6"][...] = 0.25
+    same = np.full((2, 90), 0.25, dtype=np.float32)
+    loss, g = A.rar_loss_and_grads(same, q)
+    assert loss == 0.0 and all(not g[name].any() for name, _ in A.param_shapes())
+
+
+def test_training_step_moves_every_parameter_against_its_gradient():
+    from oracle import OracleLGC
+    numel = [60_000, 30_000]
+    ora = OracleLGC(numel, 2, ae_kind="conv5", params=rand_params(8) * 0.5)
+    rng = np.random.default_rng(8)
+    ora.accumulate(rng.standard_normal((2, ora.N)).astype(np.float32))
+    ora.topk(0)
+    before = ora.get_params()
+    _, g = ora.ae_loss_and_grads()
+    loss = ora.ae_train_step()
+    after = ora.get_params()
+    gf = flat_grads(g)
+    big = np.abs(gf) > 1e-5                    # |g| >> eps: the first Adam step is lr * sign(g)
+    assert big.sum() > 1000
+    assert np.allclose(after[big] - before[big], -1e-3 * np.sign(gf[big]), rtol=2e-3, atol=0)
+    assert ora.ae_train_step() < loss          # and the loss goes down
