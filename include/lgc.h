@@ -53,7 +53,7 @@ typedef enum {
 typedef enum { LGC_VARIANT_RAR = 0, LGC_VARIANT_PS = 1 } lgc_variant;
 /* CONV2: two stride-2 convolutions each way with (ae_c1, ae_c2) channels.  IDENTITY: no autoencoder.
  * CONV5: the autoencoder of the paper's Section IV-C (encoder filters 64/128/256/64/4, decoder filters
- * 4/32/64/128/32 and a 1x1 convolution, leaky ReLU); ring-allreduce only, inference only, mu >= 31;
+ * 4/32/64/128/32 and a 1x1 convolution, leaky ReLU); ring-allreduce only, mu >= 31;
  * ae_c1 / ae_c2 are ignored.  Parameter vector: per layer the weights then the bias, encoder
  * conv1..conv5 (w[co][ci][tap]) then decoder deconv1..deconv5 (w[ci][co][tap]) and the final
  * convolution; 216,729 floats.  deconv1 has stride 1 and padding 1, the others stride 2 with the
@@ -157,8 +157,10 @@ lgc_status lgc_topk_scatter(lgc_ctx *ctx, float *update);
 /* One training step of the autoencoder on the kept values of the last lgc_topk: ring-allreduce
  * reconstruction loss of Section IV-B scaled by 1/mu,
  *     loss = (1/mu) || D_c((1/K) sum_k E_c(g~_k)) - (1/K) sum_k g~_k ||^2,
- * analytic backward pass, Adam with bias correction.  Ring-allreduce variant with LGC_AE_CONV2
- * only.  loss_out: device fp32 scalar or NULL.  May be called several times after one lgc_topk. */
+ * analytic backward pass, Adam with bias correction.  Ring-allreduce variant, LGC_AE_CONV2 or
+ * LGC_AE_CONV5 (whose forward pass runs on the tensor cores as in lgc_encode, the backward pass
+ * on the fp32 pipes; gradient sums in fp64 over per-chunk fp32 partial sums).
+ * loss_out: device fp32 scalar or NULL.  May be called several times after one lgc_topk. */
 lgc_status lgc_ae_train_step(lgc_ctx *ctx, float *loss_out);
 
 /* The same for the parameter-server autoencoder (Section IV-A): every node's kept values are

@@ -13,6 +13,8 @@
 // operand into two tf32 numbers, x = hi + lo, and accumulating hi*hi + hi*lo + lo*hi.
 // The first convolution (one input channel), the 1x1 convolutions and the decoder (which runs
 // once, not once per node) use the ordinary fp32 pipes.
+#include <algorithm>
+
 #include "lgc_internal.cuh"
 
 namespace lgc {
@@ -635,6 +637,26 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used)
         a.dw_hi[l] = take(n);
         a.dw_lo[l] = take(n);
     }
+    // training: the two outputs inference never stores, the gradients at every layer's pre-activation,
+    // the products of the backward GEMMs and the per-chunk partial sums of the parameter gradients
+    a.act4_hi = take((size_t)K * a.len[4] * 64);
+    a.act4_lo = take((size_t)K * a.len[4] * 64);
+    a.dact5_hi = take((size_t)mu * 32);
+    a.dact5_lo = take((size_t)mu * 32);
+    size_t pmax = 0;
+    for (int l = 0; l < 4; ++l) {
+        a.g_enc[l] = take((size_t)K * a.len[l + 1] * kAe5EncCh[l + 1]);
+        if (l > 0) pmax = std::max(pmax, (size_t)K * a.len[l + 1] * 3 * kAe5EncCh[l]);
+    }
+    a.g_dec[0] = take((size_t)a.len[4] * 4);
+    for (int l = 1; l < 5; ++l) a.g_dec[l] = take((size_t)a.len[4 - l] * kAe5DecCh[l + 1]);
+    a.dzk = take((size_t)K * a.len[4] * 4);
+    a.dzbar = take((size_t)a.len[4] * 4);
+    a.dr = take((size_t)mu);
+    a.pbuf = take(pmax);
+    a.wt = take((size_t)256 * 384);
+    a.loss_blocks = (int)((mu + 255) / 256);
+    a.loss_part = reinterpret_cast<double *>(take((size_t)a.loss_blocks * 2));
     *used = at;
     // offsets of the layers' parameters inside the flat vector (encoder, then decoder)
     int64_t pos = 0;
@@ -650,6 +672,32 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used)
     }
     a.off_dw[5] = pos; pos += 32;
     a.off_db[5] = pos;
+    // parameter tensors in order, with the rows their gradient sums run over and the chunks these are cut into
+    int64_t part = 0;
+    auto tensor = [&](int i, int64_t off, int64_t count, int64_t rows, int kind, int cin, int cout) {
+        Ae5::Tensor &t = a.tensors[i];
+        t.param_off = off; t.count = count; t.rows = rows; t.kind = kind; t.cin = cin; t.cout = cout;
+        t.chunk = std::max<int64_t>(256, (rows + 47) / 48);
+        t.chunks = kind == 3 ? 1 : (int)((rows + t.chunk - 1) / t.chunk);
+        t.partial_off = part;
+        part += t.chunks * ((count + 3) / 4 * 4);
+    };
+    for (int i = 0; i < 4; ++i) {            // conv1..conv4: sums over K L_out rows
+        tensor(2 * i, a.off_w[i], (int64_t)kAe5EncCh[i + 1] * kAe5EncCh[i] * 3, (int64_t)K * a.len[i + 1], 1, kAe5EncCh[i], kAe5EncCh[i + 1]);
+        tensor(2 * i + 1, a.off_b[i], kAe5EncCh[i + 1], (int64_t)K * a.len[i + 1], 0, 0, 0);
+    }
+    tensor(8, a.off_w[4], 4 * 64, (int64_t)K * a.len[4], 0, 0, 0);
+    tensor(9, a.off_b[4], 4, (int64_t)K * a.len[4], 0, 0, 0);
+    tensor(10, a.off_dw[0], 48, a.len[4], 3, 0, 0);       // deconv1: reduced by a kernel of its own
+    tensor(11, a.off_db[0], 4, a.len[4], 3, 0, 0);
+    for (int i = 1; i < 5; ++i) {            // deconv2..deconv5: weights sum over L_in rows, biases over L_out rows
+        tensor(10 + 2 * i, a.off_dw[i], (int64_t)kAe5DecCh[i] * kAe5DecCh[i + 1] * 3, a.len[5 - i], 2, kAe5DecCh[i], kAe5DecCh[i + 1]);
+        tensor(11 + 2 * i, a.off_db[i], kAe5DecCh[i + 1], a.len[4 - i], 0, 0, 0);
+    }
+    tensor(20, a.off_dw[5], 32, mu, 0, 0, 0);
+    tensor(21, a.off_db[5], 1, mu, 0, 0, 0);
+    if (base) a.partial = reinterpret_cast<float *>(base + (*used + 1023) / 1024 * 1024);
+    *used = (*used + 1023) / 1024 * 1024 + (size_t)part * sizeof(float);
 }
 
 cudaError_t ae5_make_maps(Ctx &c)
@@ -715,6 +763,78 @@ cudaError_t launch_ae5_encode(Ctx &c)
     if (e == cudaSuccess)
         e = launch_gemm<kConvCode, 256, 64>(c, a.map_act_hi[2], a.map_act_lo[2], a.map_w_hi[2], a.map_w_lo[2], P + a.off_b[3],
                                             a.len[4], c.K, a.len[4], 0, nullptr, nullptr, P + a.off_w[4], P + a.off_b[4], c.code);
+    return e;
+}
+
+// conv5 (1x1, 64 -> 4, no activation) on the stored output of conv4: thread per (node, position).
+__global__ void ae5_conv5_kernel(const float *__restrict__ a_hi, const float *__restrict__ a_lo, int64_t rows,
+                                 const float *__restrict__ w5, const float *__restrict__ b5, float *__restrict__ code)
+{
+    __shared__ float w[4 * 64], b[4];
+    for (int i = threadIdx.x; i < 4 * 64; i += blockDim.x) w[i] = w5[i];
+    if (threadIdx.x < 4) b[threadIdx.x] = b5[threadIdx.x];
+    __syncthreads();
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int q = 0; q < 16; ++q) {
+        const float4 h = reinterpret_cast<const float4 *>(a_hi + r * 64)[q], l = reinterpret_cast<const float4 *>(a_lo + r * 64)[q];
+        const float x[4] = {__fadd_rn(h.x, l.x), __fadd_rn(h.y, l.y), __fadd_rn(h.z, l.z), __fadd_rn(h.w, l.w)};
+#pragma unroll
+        for (int o = 0; o < 4; ++o)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[o] = __fmaf_rn(w[o * 64 + 4 * q + j], x[j], acc[o]);
+    }
+    reinterpret_cast<float4 *>(code)[r] = make_float4(__fadd_rn(acc[0], b[0]), __fadd_rn(acc[1], b[1]), __fadd_rn(acc[2], b[2]),
+                                                      __fadd_rn(acc[3], b[3]));
+}
+
+// Forward pass of a training step: the same kernels as inference, but conv4 and deconv5 store
+// their outputs (the backward pass needs them) and conv5 and the mean run as launches of their own.
+// Leaves the codes in c.code, their mean in c.combined and deconv5's output in dact5.
+cudaError_t launch_ae5_train_forward(Ctx &c)
+{
+    Ae5 &a = *c.ae5;
+    const float *P = c.params;
+    prepare_weights(c);
+    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.mu, a.len[1], a.lpad[0],
+                                                                            P + a.off_w[0], P + a.off_b[0], c.val, a.act_hi[0],
+                                                                            a.act_lo[0]),
+        ++g_kernel_launches;
+    c.val_valid = true;
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess)
+        e = launch_gemm<kConv, 64, 128>(c, a.map_act_hi[0], a.map_act_lo[0], a.map_w_hi[0], a.map_w_lo[0], P + a.off_b[1],
+                                        a.len[2], c.K, a.len[2], a.lpad[1], a.act_hi[1], a.act_lo[1], nullptr, nullptr, nullptr);
+    if (e == cudaSuccess)
+        e = launch_gemm<kConv, 128, 256>(c, a.map_act_hi[1], a.map_act_lo[1], a.map_w_hi[1], a.map_w_lo[1], P + a.off_b[2],
+                                         a.len[3], c.K, a.len[3], a.lpad[2], a.act_hi[2], a.act_lo[2], nullptr, nullptr, nullptr);
+    if (e == cudaSuccess)
+        e = launch_gemm<kConv, 256, 64>(c, a.map_act_hi[2], a.map_act_lo[2], a.map_w_hi[2], a.map_w_lo[2], P + a.off_b[3],
+                                        a.len[4], c.K, a.len[4], a.len[4], a.act4_hi, a.act4_lo, nullptr, nullptr, nullptr);
+    if (e != cudaSuccess) return e;
+    const int64_t rows = (int64_t)c.K * a.len[4];
+    ae5_conv5_kernel<<<blocks(rows, 128), 128, 0, c.stream>>>(a.act4_hi, a.act4_lo, rows, P + a.off_w[4], P + a.off_b[4], c.code),
+        ++g_kernel_launches;
+    c.mean_valid = false;
+    e = launch_combine_mean(c);
+    if (e != cudaSuccess) return e;
+    ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0),
+        ++g_kernel_launches;
+    constexpr int kTp = 64, kSmem2 = (3 * 4 * 32 + (kTp + 1) * 4) * 4;
+    ae5_deconv_kernel<4, 32, kTp><<<blocks(a.len[4] + 1, kTp), 256, kSmem2, c.stream>>>(a.d0, a.len[4], a.len[3], P + a.off_dw[1],
+                                                                                        P + a.off_db[1], a.dact_hi[0], a.dact_lo[0]),
+        ++g_kernel_launches;
+    e = cudaGetLastError();
+    if (e == cudaSuccess)
+        e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], a.map_dw_hi[0], a.map_dw_lo[0], P + a.off_db[2],
+                                         a.len[3] + 1, 1, a.len[2], 0, a.dact_hi[1], a.dact_lo[1], nullptr, nullptr, nullptr);
+    if (e == cudaSuccess)
+        e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], a.map_dw_hi[1], a.map_dw_lo[1], P + a.off_db[3],
+                                          a.len[2] + 1, 1, a.len[1], 0, a.dact_hi[2], a.dact_lo[2], nullptr, nullptr, nullptr);
+    if (e == cudaSuccess)
+        e = launch_gemm<kDeconv, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], a.map_dw_hi[2], a.map_dw_lo[2], P + a.off_db[4],
+                                          a.len[1] + 1, 1, a.len[0], 0, a.dact5_hi, a.dact5_lo, nullptr, nullptr, nullptr);
     return e;
 }
 

@@ -1,0 +1,524 @@
+// Training step of the paper's full-size autoencoder (Section IV-C) for the ring-allreduce form:
+// loss of Section IV-B on the kept values of the last selection (Section V-B, second phase),
+//     loss = (1/mu) || D_c((1/K) sum_k E_c(g~_k)) - (1/K) sum_k g~_k ||^2,
+// backward pass through every layer, Adam.
+//
+// The forward pass is the inference path's (tensor cores; lgc_ae5.cu) with every layer's output
+// kept.  The backward pass works on channels-last fp32 buffers.  With G the gradient at a
+// layer's pre-activation output and X its (post-activation) input:
+//   convolution  y[t][co] = b + sum w[co][ci][tau] x[2t+tau][ci]
+//     dW[co][tau C_in + ci] = sum_t G[t][co] X[2t+tau][ci]      (rows of X seen as slices of 3 C_in floats)
+//     dX                    = fold(G W), W[co][tau C_in + ci]    (products first, then summed onto 2t+tau)
+//   transposed convolution  y[2j+tau][co] += w[ci][co][tau] x[j][ci]
+//     dW[ci][tau C_out + co] = sum_j X[j][ci] G[2j+tau][co]      (rows of G seen as slices of 3 C_out floats)
+//     dX[j][ci]              = sum G[2j+tau][co] w[ci][co][tau]
+// so every layer is one GEMM over rows (dX) and one GEMM that sums over rows (dW), here on the fp32
+// pipes; the sums over rows are cut into chunks whose partial results are added up in fp64, in
+// chunk order, by the kernel that applies Adam.  Leaky-ReLU derivatives are taken from the sign of
+// the stored outputs (the slope is positive, so output and pre-activation have the same sign).
+#include <algorithm>
+
+#include "lgc_internal.cuh"
+
+namespace lgc {
+
+namespace {
+
+constexpr float kSlope = 0.01f;       // leaky-ReLU slope of the full-size autoencoder
+constexpr int kTile = 64;             // GEMM tile: 64 x 64 outputs per CTA of 256 threads (4 x 4 per thread)
+constexpr int kStep = 16;             // rows (TN) or inner entries (NN) staged per trip
+constexpr int kPitch = kTile + 4;
+
+// M rows of `len` floats, row m = (node, t): value hi[...] (+ lo[...] when the buffer is kept as two tf32 parts).
+struct Rows {
+    const float *hi, *lo;
+    int64_t node_stride, row_stride, rows_per_node;
+    int len;
+    int vec;                          // rows start 16-byte aligned and len % 4 == 0
+    __device__ __forceinline__ int64_t at(int64_t m) const
+    {
+        const int64_t k = m / rows_per_node, t = m - k * rows_per_node;
+        return k * node_stride + t * row_stride;
+    }
+};
+
+Rows rows_of(const float *hi, const float *lo, int64_t node_stride, int64_t row_stride, int64_t rows_per_node, int len)
+{
+    Rows r;
+    r.hi = hi; r.lo = lo; r.node_stride = node_stride; r.row_stride = row_stride; r.rows_per_node = rows_per_node; r.len = len;
+    r.vec = len % 4 == 0 && node_stride % 4 == 0 && row_stride % 4 == 0 && (reinterpret_cast<uintptr_t>(hi) & 15) == 0 &&
+            (lo == nullptr || (reinterpret_cast<uintptr_t>(lo) & 15) == 0);
+    return r;
+}
+
+// four consecutive entries of a row from column c on (zeros beyond the row's length)
+__device__ __forceinline__ float4 load4(const Rows &r, int64_t base, int c)
+{
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (r.vec) {
+        if (c < r.len) {
+            x = *reinterpret_cast<const float4 *>(r.hi + base + c);
+            if (r.lo) {
+                const float4 l = *reinterpret_cast<const float4 *>(r.lo + base + c);
+                x.x = __fadd_rn(x.x, l.x); x.y = __fadd_rn(x.y, l.y); x.z = __fadd_rn(x.z, l.z); x.w = __fadd_rn(x.w, l.w);
+            }
+        }
+        return x;
+    }
+    float *e = &x.x;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if (c + j < r.len) e[j] = r.lo ? __fadd_rn(r.hi[base + c + j], r.lo[base + c + j]) : r.hi[base + c + j];
+    return x;
+}
+
+// C[m][n] = sum_kd A(m, kd) B[kd][n] for m < M, n < N; B dense [Kd][N], Kd a multiple of 16, N of 4.
+// MASK: the result is the gradient at the output of a leaky ReLU whose stored output is X(m, n):
+// it is multiplied by 1 or by the slope.  Grid (ceil(N / 64), ceil(M / 64)), 256 threads.
+template <bool MASK>
+__global__ void __launch_bounds__(256)
+nn_gemm_kernel(Rows A, int64_t M, const float *__restrict__ B, int N, float *__restrict__ C, int64_t ldc, Rows X)
+{
+    __shared__ __align__(16) float As[kStep][kPitch], Bs[kStep][kPitch];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int64_t m0 = (int64_t)blockIdx.y * kTile;
+    const int n0 = blockIdx.x * kTile;
+    float acc[4][4] = {};
+    const int ar = threadIdx.x >> 2, akq = threadIdx.x & 3;          // A tile: 64 rows x 16 entries, a float4 per thread
+    const int64_t am = m0 + ar;
+    const int64_t abase = am < M ? A.at(am) : 0;
+    const int bk = threadIdx.x >> 4, bnq = threadIdx.x & 15;         // B tile: 16 rows x 64 columns
+    for (int k0 = 0; k0 < A.len; k0 += kStep) {
+        const float4 a = am < M ? load4(A, abase, k0 + 4 * akq) : make_float4(0.f, 0.f, 0.f, 0.f);
+        As[4 * akq + 0][ar] = a.x; As[4 * akq + 1][ar] = a.y; As[4 * akq + 2][ar] = a.z; As[4 * akq + 3][ar] = a.w;
+        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (n0 + 4 * bnq < N) b = *reinterpret_cast<const float4 *>(B + (int64_t)(k0 + bk) * N + n0 + 4 * bnq);
+        *reinterpret_cast<float4 *>(&Bs[bk][4 * bnq]) = b;
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kStep; ++k) {
+            const float4 av = *reinterpret_cast<const float4 *>(&As[k][4 * ty]);
+            const float4 bv = *reinterpret_cast<const float4 *>(&Bs[k][4 * tx]);
+            const float aa[4] = {av.x, av.y, av.z, av.w}, bb[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = __fmaf_rn(aa[i], bb[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    const int n = n0 + 4 * tx;
+    if (n >= N) return;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t m = m0 + 4 * ty + i;
+        if (m >= M) break;
+        float4 out = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        if (MASK) {
+            const int64_t xb = X.at(m);
+            const float4 x = *reinterpret_cast<const float4 *>(X.hi + xb + n);   // the sign of the leading part is the value's
+            out.x = x.x > 0.f ? out.x : __fmul_rn(kSlope, out.x);
+            out.y = x.y > 0.f ? out.y : __fmul_rn(kSlope, out.y);
+            out.z = x.z > 0.f ? out.z : __fmul_rn(kSlope, out.z);
+            out.w = x.w > 0.f ? out.w : __fmul_rn(kSlope, out.w);
+        }
+        *reinterpret_cast<float4 *>(C + m * ldc + n) = out;
+    }
+}
+
+// partial[s][p][q] = sum over the rows m of chunk s of A(m, p) B(m, q).  Grid (ceil(Q / 64), ceil(P / 64), chunks).
+__global__ void __launch_bounds__(256)
+tn_gemm_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ partial, int64_t pstride)
+{
+    __shared__ __align__(16) float As[kStep][kPitch], Bs[kStep][kPitch];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int p0 = blockIdx.y * kTile, q0 = blockIdx.x * kTile;
+    const int64_t first = (int64_t)blockIdx.z * chunk;
+    const int64_t last = first + chunk < M ? first + chunk : M;
+    float acc[4][4] = {};
+    const int lr = threadIdx.x >> 4, lc = threadIdx.x & 15;          // 16 rows x 64 columns of each operand per trip
+    for (int64_t r0 = first; r0 < last; r0 += kStep) {
+        const int64_t m = r0 + lr;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+        if (m < last) {
+            a = load4(A, A.at(m), p0 + 4 * lc);
+            b = load4(B, B.at(m), q0 + 4 * lc);
+        }
+        *reinterpret_cast<float4 *>(&As[lr][4 * lc]) = a;
+        *reinterpret_cast<float4 *>(&Bs[lr][4 * lc]) = b;
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kStep; ++k) {
+            const float4 av = *reinterpret_cast<const float4 *>(&As[k][4 * ty]);
+            const float4 bv = *reinterpret_cast<const float4 *>(&Bs[k][4 * tx]);
+            const float aa[4] = {av.x, av.y, av.z, av.w}, bb[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = __fmaf_rn(aa[i], bb[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+    float *out = partial + (int64_t)blockIdx.z * pstride;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int p = p0 + 4 * ty + i;
+        if (p >= A.len) break;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int q = q0 + 4 * tx + j;
+            if (q < B.len) out[(int64_t)p * B.len + q] = acc[i][j];
+        }
+    }
+}
+
+// partial[s][p] = sum over the rows of chunk s of A(m, p) (bias gradients).  Grid (chunks), 256 threads.
+__global__ void __launch_bounds__(256)
+colsum_kernel(Rows A, int64_t M, int64_t chunk, float *__restrict__ partial, int64_t pstride)
+{
+    const int64_t first = (int64_t)blockIdx.x * chunk;
+    const int64_t last = first + chunk < M ? first + chunk : M;
+    for (int p = threadIdx.x; p < A.len; p += 256) {
+        float acc = 0.f;
+        for (int64_t m = first; m < last; ++m) acc = __fadd_rn(acc, A.hi[A.at(m) + p]);
+        partial[(int64_t)blockIdx.x * pstride + p] = acc;
+    }
+}
+
+// Gradient at a convolution's input from the products prod[k][t][tau C_in + ci] = (G W)[t]:
+//   g_in[k][pos][ci] = leaky'(x[k][pos][ci]) * sum over (t, tau) with 2t + tau = pos of prod[k][t][tau C_in + ci].
+// Thread per (node, position, four channels).
+__global__ void fold_kernel(const float *__restrict__ prod, int K, int64_t L_out, int64_t L_in, int cin,
+                            const float *__restrict__ x_hi, int64_t x_node_stride, float *__restrict__ g_in)
+{
+    const int quads = cin >> 2;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (int64_t)K * L_in * quads) return;
+    const int cq = (int)(i % quads);
+    const int64_t pos = (i / quads) % L_in, k = i / quads / L_in;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int tau = 0; tau < 3; ++tau) {
+        const int64_t d = pos - tau;
+        if (d < 0 || (d & 1) || (d >> 1) >= L_out) continue;
+        const float4 p = *reinterpret_cast<const float4 *>(prod + ((k * L_out + (d >> 1)) * 3 + tau) * cin + 4 * cq);
+        acc.x = __fadd_rn(acc.x, p.x); acc.y = __fadd_rn(acc.y, p.y); acc.z = __fadd_rn(acc.z, p.z); acc.w = __fadd_rn(acc.w, p.w);
+    }
+    const float4 x = *reinterpret_cast<const float4 *>(x_hi + k * x_node_stride + pos * cin + 4 * cq);
+    acc.x = x.x > 0.f ? acc.x : __fmul_rn(kSlope, acc.x);
+    acc.y = x.y > 0.f ? acc.y : __fmul_rn(kSlope, acc.y);
+    acc.z = x.z > 0.f ? acc.z : __fmul_rn(kSlope, acc.z);
+    acc.w = x.w > 0.f ? acc.w : __fmul_rn(kSlope, acc.w);
+    *reinterpret_cast<float4 *>(g_in + (k * L_in + pos) * cin + 4 * cq) = acc;
+}
+
+// One layer's weights arranged as the dense [Kd][N] operand of nn_gemm_kernel.
+//   mode 0, convolution w[co][ci][tau]            -> W[co][tau C_in + ci]   (Kd = C_out, N = 3 C_in)
+//   mode 1, transposed convolution w[ci][co][tau] -> W[tau C_out + co][ci]  (Kd = 3 C_out, N = C_in)
+__global__ void arrange_weights_kernel(const float *__restrict__ w, int cin, int cout, int mode, float *__restrict__ out)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 3 * cin * cout) return;
+    if (mode == 0) {
+        const int co = i / (3 * cin), tau = i % (3 * cin) / cin, ci = i % cin;
+        out[i] = w[(co * cin + ci) * 3 + tau];
+    } else {
+        const int tau = i / (cout * cin), co = i / cin % cout, ci = i % cin;
+        out[i] = w[(ci * cout + co) * 3 + tau];
+    }
+}
+
+__device__ __forceinline__ double block_sum256(double x, double *warp_part)
+{
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) x += __shfl_down_sync(0xffffffffu, x, d);
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = x;
+    __syncthreads();
+    double tot = 0.0;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < 8; ++w) tot += warp_part[w];
+    return tot;                                                   // valid in thread 0
+}
+
+// The last convolution (1x1, 32 -> 1) on deconv5's stored output, the loss, and the way back through
+// it: recon[p], dr[p] = 2 (recon[p] - target[p]) / mu with target = (1/K) sum_k val_k (node order),
+// this CTA's part of sum (recon - target)^2, and g5[p][c] = dr[p] w6[c] leaky'(d5[p][c]).
+__global__ void __launch_bounds__(256)
+final_loss_kernel(const float *__restrict__ d5_hi, const float *__restrict__ d5_lo, const float *__restrict__ val, int K,
+                  int64_t mu, const float *__restrict__ w6, const float *__restrict__ b6, float *__restrict__ recon,
+                  float *__restrict__ dr, float *__restrict__ g5, double *__restrict__ loss_part)
+{
+    __shared__ float w[32];
+    __shared__ double warp_part[8];
+    if (threadIdx.x < 32) w[threadIdx.x] = w6[threadIdx.x];
+    __syncthreads();
+    const int64_t p = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    double sq = 0.0;
+    if (p < mu) {
+        float hi[32];
+        float r = b6[0];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float4 h = reinterpret_cast<const float4 *>(d5_hi + p * 32)[q], l = reinterpret_cast<const float4 *>(d5_lo + p * 32)[q];
+            hi[4 * q] = h.x; hi[4 * q + 1] = h.y; hi[4 * q + 2] = h.z; hi[4 * q + 3] = h.w;
+            r = __fmaf_rn(w[4 * q], __fadd_rn(h.x, l.x), r);
+            r = __fmaf_rn(w[4 * q + 1], __fadd_rn(h.y, l.y), r);
+            r = __fmaf_rn(w[4 * q + 2], __fadd_rn(h.z, l.z), r);
+            r = __fmaf_rn(w[4 * q + 3], __fadd_rn(h.w, l.w), r);
+        }
+        float target = 0.f;
+        for (int k = 0; k < K; ++k) target = __fadd_rn(target, val[(int64_t)k * mu + p]);
+        target = __fdiv_rn(target, (float)K);
+        const double diff = (double)r - (double)target;
+        sq = diff * diff;
+        const float g = (float)(2.0 * diff / (double)mu);
+        recon[p] = r;
+        dr[p] = g;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            float4 o;
+            o.x = __fmul_rn(g, w[4 * q]);     o.x = hi[4 * q] > 0.f ? o.x : __fmul_rn(kSlope, o.x);
+            o.y = __fmul_rn(g, w[4 * q + 1]); o.y = hi[4 * q + 1] > 0.f ? o.y : __fmul_rn(kSlope, o.y);
+            o.z = __fmul_rn(g, w[4 * q + 2]); o.z = hi[4 * q + 2] > 0.f ? o.z : __fmul_rn(kSlope, o.z);
+            o.w = __fmul_rn(g, w[4 * q + 3]); o.w = hi[4 * q + 3] > 0.f ? o.w : __fmul_rn(kSlope, o.w);
+            reinterpret_cast<float4 *>(g5 + p * 32)[q] = o;
+        }
+    }
+    const double tot = block_sum256(sq, warp_part);
+    if (threadIdx.x == 0) loss_part[blockIdx.x] = tot;
+}
+
+__global__ void __launch_bounds__(256)
+loss_sum_kernel(const double *__restrict__ part, int n, int64_t mu, float *__restrict__ out)
+{
+    __shared__ double warp_part[8];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n; i += 256) acc += part[i];
+    const double tot = block_sum256(acc, warp_part);
+    if (threadIdx.x == 0) *out = (float)(tot / (double)mu);
+}
+
+// deconv1 (4 -> 4, stride 1, padding 1), y[s][co] = b + sum w[ci][co][tau] zbar[s + 1 - tau][ci]:
+// gradient at the mean code, dzbar[j][ci] = sum over (tau, co) of w[ci][co][tau] g1[j + tau - 1][co].
+__global__ void dec1_bwd_kernel(const float *__restrict__ g1, int64_t L4, const float *__restrict__ w, float *__restrict__ dzbar)
+{
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= L4) return;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int tau = 0; tau < 3; ++tau) {
+        const int64_t s = j + tau - 1;
+        if (s < 0 || s >= L4) continue;
+        const float4 g = reinterpret_cast<const float4 *>(g1)[s];
+        const float gs[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+        for (int ci = 0; ci < 4; ++ci)
+#pragma unroll
+            for (int co = 0; co < 4; ++co) acc[ci] = __fmaf_rn(w[(ci * 4 + co) * 3 + tau], gs[co], acc[ci]);
+    }
+    reinterpret_cast<float4 *>(dzbar)[j] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+}
+
+// deconv1's 48 weight and 4 bias gradients: one CTA each, summed in fp64.
+__global__ void __launch_bounds__(256)
+dec1_grad_kernel(const float *__restrict__ zbar, const float *__restrict__ g1, int64_t L4, float *__restrict__ gw,
+                 float *__restrict__ gb)
+{
+    __shared__ double warp_part[8];
+    const int id = blockIdx.x;
+    double acc = 0.0;
+    if (id < 48) {
+        const int ci = id / 12, co = id / 3 % 4, tau = id % 3;
+        for (int64_t j = threadIdx.x; j < L4; j += 256) {
+            const int64_t s = j + tau - 1;
+            if (s >= 0 && s < L4) acc += (double)zbar[j * 4 + ci] * (double)g1[s * 4 + co];
+        }
+    } else {
+        for (int64_t s = threadIdx.x; s < L4; s += 256) acc += (double)g1[s * 4 + (id - 48)];
+    }
+    const double tot = block_sum256(acc, warp_part);
+    if (threadIdx.x == 0) (id < 48 ? gw[id] : gb[id - 48]) = (float)tot;
+}
+
+// Way back through the mean and conv5 (1x1, 64 -> 4): every node's code gets dzbar / K, and
+//   g4[k][t][c] = leaky'(a4[k][t][c]) * sum_o w5[o][c] dzk[k][t][o].   Thread per (node, position).
+__global__ void code_bwd_kernel(const float *__restrict__ dzbar, int K, int64_t L4, const float *__restrict__ w5,
+                                const float *__restrict__ a4_hi, float *__restrict__ dzk, float *__restrict__ g4)
+{
+    __shared__ float w[4 * 64];
+    for (int i = threadIdx.x; i < 4 * 64; i += blockDim.x) w[i] = w5[i];
+    __syncthreads();
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= (int64_t)K * L4) return;
+    const float4 z = reinterpret_cast<const float4 *>(dzbar)[r % L4];
+    const float fk = (float)K;
+    const float dz[4] = {__fdiv_rn(z.x, fk), __fdiv_rn(z.y, fk), __fdiv_rn(z.z, fk), __fdiv_rn(z.w, fk)};
+    reinterpret_cast<float4 *>(dzk)[r] = make_float4(dz[0], dz[1], dz[2], dz[3]);
+    for (int q = 0; q < 16; ++q) {
+        const float4 a = reinterpret_cast<const float4 *>(a4_hi + r * 64)[q];
+        const float as[4] = {a.x, a.y, a.z, a.w};
+        float o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float acc = 0.f;
+#pragma unroll
+            for (int oo = 0; oo < 4; ++oo) acc = __fmaf_rn(w[oo * 64 + 4 * q + j], dz[oo], acc);
+            o[j] = as[j] > 0.f ? acc : __fmul_rn(kSlope, acc);
+        }
+        reinterpret_cast<float4 *>(g4 + r * 64)[q] = make_float4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// Gradient of one parameter tensor from its chunks' partial sums (fp64, chunk order), then Adam.
+//   kind 0 / 3: entry e is parameter e;  kind 1: e = (co, tau, ci) -> w[co][ci][tau];
+//   kind 2: e = (ci, tau, co) -> w[ci][co][tau].
+__global__ void reduce_adam_kernel(const float *__restrict__ partial, int chunks, int64_t pstride, int64_t count, int kind,
+                                   int cin, int cout, int64_t param_off, AdamArgs ad)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= count) return;
+    double g = 0.0;
+    for (int s = 0; s < chunks; ++s) g += (double)partial[(int64_t)s * pstride + e];
+    int64_t i = e;
+    if (kind == 1) {
+        const int64_t co = e / (3 * cin), tau = e % (3 * cin) / cin, ci = e % cin;
+        i = (co * cin + ci) * 3 + tau;
+    } else if (kind == 2) {
+        const int64_t ci = e / (3 * cout), tau = e % (3 * cout) / cout, co = e % cout;
+        i = (ci * cout + co) * 3 + tau;
+    }
+    i += param_off;
+    const double m = ad.beta1 * (double)ad.m[i] + (1.0 - ad.beta1) * g;
+    const double v = ad.beta2 * (double)ad.v[i] + (1.0 - ad.beta2) * g * g;
+    ad.m[i] = (float)m;
+    ad.v[i] = (float)v;
+    ad.params[i] = (float)((double)ad.params[i] - ad.lr * (m / ad.corr1) / (sqrt(v / ad.corr2) + ad.eps));
+}
+
+inline unsigned blocks(int64_t n, int per) { return (unsigned)((n + per - 1) / per); }
+
+struct Launcher {
+    Ctx &c;
+    Ae5 &a;
+    cudaError_t err = cudaSuccess;
+    bool ok() { if (err == cudaSuccess) err = cudaGetLastError(); return err == cudaSuccess; }
+
+    float *partial_of(int t) { return a.partial + a.tensors[t].partial_off; }
+    int64_t pstride_of(int t) { return (a.tensors[t].count + 3) / 4 * 4; }
+
+    void nn(const Rows &A, int64_t M, const float *B, int N, float *C, const Rows *mask)
+    {
+        if (!ok()) return;
+        const dim3 grid(blocks(N, kTile), blocks(M, kTile));
+        if (mask) nn_gemm_kernel<true><<<grid, 256, 0, c.stream>>>(A, M, B, N, C, N, *mask);
+        else nn_gemm_kernel<false><<<grid, 256, 0, c.stream>>>(A, M, B, N, C, N, A);
+        ++g_kernel_launches;
+    }
+    // weight gradient of tensor t: sum over rows of A(m, .)^T B(m, .)
+    void tn(int t, const Rows &A, const Rows &B)
+    {
+        if (!ok()) return;
+        const Ae5::Tensor &T = a.tensors[t];
+        const dim3 grid(blocks(B.len, kTile), blocks(A.len, kTile), T.chunks);
+        tn_gemm_kernel<<<grid, 256, 0, c.stream>>>(A, B, T.rows, T.chunk, partial_of(t), pstride_of(t));
+        ++g_kernel_launches;
+    }
+    void colsum(int t, const Rows &A)
+    {
+        if (!ok()) return;
+        const Ae5::Tensor &T = a.tensors[t];
+        colsum_kernel<<<T.chunks, 256, 0, c.stream>>>(A, T.rows, T.chunk, partial_of(t), pstride_of(t));
+        ++g_kernel_launches;
+    }
+    void arrange(const float *w, int cin, int cout, int mode)
+    {
+        if (!ok()) return;
+        arrange_weights_kernel<<<blocks(3 * cin * cout, 256), 256, 0, c.stream>>>(w, cin, cout, mode, a.wt);
+        ++g_kernel_launches;
+    }
+};
+
+}  // namespace
+
+cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out)
+{
+    Ae5 &a = *c.ae5;
+    const float *P = c.params;
+    const int K = c.K;
+    const int64_t mu = c.mu;
+    const int64_t *len = a.len;                   // mu, L1, L2, L3, L4
+    cudaError_t e = launch_ae5_train_forward(c);
+    if (e != cudaSuccess) return e;
+    Launcher L{c, a};
+    cudaStream_t s = c.stream;
+
+    // ---- the last convolution and the loss ----
+    final_loss_kernel<<<a.loss_blocks, 256, 0, s>>>(a.dact5_hi, a.dact5_lo, c.val, K, mu, P + a.off_dw[5], P + a.off_db[5], c.recon,
+                                                    a.dr, a.g_dec[4], a.loss_part),
+        ++g_kernel_launches;
+    if (loss_out) loss_sum_kernel<<<1, 256, 0, s>>>(a.loss_part, a.loss_blocks, mu, loss_out), ++g_kernel_launches;
+    const Rows dr_rows = rows_of(a.dr, nullptr, 0, 1, mu, 1);
+    L.tn(20, dr_rows, rows_of(a.dact5_hi, a.dact5_lo, 0, 32, mu, 32));
+    L.colsum(21, dr_rows);
+
+    // ---- deconv5 .. deconv2: input of deconv i+1 is the output of deconv i ----
+    // inputs: deconv5 <- dact[2] [L1][128], deconv4 <- dact[1] [L2][64], deconv3 <- dact[0] [L3][32], deconv2 <- d0 [L4][4]
+    for (int i = 4; i >= 1; --i) {
+        const int cin = kAe5DecCh[i], cout = kAe5DecCh[i + 1];
+        const int64_t lin = len[5 - i], lout = len[4 - i];
+        const float *g_out = a.g_dec[i];                                    // [lout][cout]
+        const float *x_hi = i == 1 ? a.d0 : a.dact_hi[i - 2], *x_lo = i == 1 ? nullptr : a.dact_lo[i - 2];
+        const Rows x = rows_of(x_hi, x_lo, 0, cin, lin, cin);
+        const Rows g_slices = rows_of(g_out, nullptr, 0, 2 * cout, lin, 3 * cout);   // row j: positions 2j .. 2j + 2
+        L.colsum(11 + 2 * i, rows_of(g_out, nullptr, 0, cout, lout, cout));
+        L.tn(10 + 2 * i, x, g_slices);
+        L.arrange(P + a.off_dw[i], cin, cout, 1);
+        L.nn(g_slices, lin, a.wt, cin, a.g_dec[i - 1], &x);
+    }
+    // ---- deconv1, the mean, conv5 ----
+    if (L.ok()) {
+        dec1_grad_kernel<<<52, 256, 0, s>>>(c.combined, a.g_dec[0], len[4], L.partial_of(10), L.partial_of(11)), ++g_kernel_launches;
+        dec1_bwd_kernel<<<blocks(len[4], 128), 128, 0, s>>>(a.g_dec[0], len[4], P + a.off_dw[0], a.dzbar), ++g_kernel_launches;
+        code_bwd_kernel<<<blocks((int64_t)K * len[4], 128), 128, 0, s>>>(a.dzbar, K, len[4], P + a.off_w[4], a.act4_hi, a.dzk,
+                                                                       a.g_enc[3]),
+            ++g_kernel_launches;
+    }
+    const Rows dzk_rows = rows_of(a.dzk, nullptr, len[4] * 4, 4, len[4], 4);
+    L.tn(8, dzk_rows, rows_of(a.act4_hi, a.act4_lo, len[4] * 64, 64, len[4], 64));
+    L.colsum(9, dzk_rows);
+
+    // ---- conv4 .. conv1 ----
+    for (int i = 3; i >= 0; --i) {
+        const int cin = kAe5EncCh[i], cout = kAe5EncCh[i + 1];
+        const int64_t lin = len[i], lout = len[i + 1];
+        const Rows g = rows_of(a.g_enc[i], nullptr, lout * cout, cout, lout, cout);  // [K][lout][cout]
+        L.colsum(2 * i + 1, g);
+        if (i == 0) {        // conv1 reads the kept values themselves: rows of three floats, two apart
+            L.tn(0, g, rows_of(c.val, nullptr, mu, 2, lout, 3));
+            break;
+        }
+        const int64_t x_node = a.lpad[i - 1] * cin;
+        L.tn(2 * i, g, rows_of(a.act_hi[i - 1], a.act_lo[i - 1], x_node, 2 * cin, lout, 3 * cin));
+        L.arrange(P + a.off_w[i], cin, cout, 0);
+        L.nn(g, (int64_t)K * lout, a.wt, 3 * cin, a.pbuf, nullptr);
+        if (L.ok()) {
+            fold_kernel<<<blocks((int64_t)K * lin * (cin / 4), 256), 256, 0, s>>>(a.pbuf, K, lout, lin, cin, a.act_hi[i - 1], x_node,
+                                                                                 a.g_enc[i - 1]),
+                ++g_kernel_launches;
+        }
+    }
+    if (!L.ok()) return L.err;
+
+    // ---- Adam on every tensor ----
+    const AdamArgs ad = next_adam(c);
+    for (int t = 0; t < 22; ++t) {
+        const Ae5::Tensor &T = a.tensors[t];
+        reduce_adam_kernel<<<blocks(T.count, 256), 256, 0, s>>>(L.partial_of(t), T.chunks, L.pstride_of(t), T.count, T.kind, T.cin,
+                                                                T.cout, T.param_off, ad),
+            ++g_kernel_launches;
+    }
+    a.weights_ready = false;                       // the GEMM forms of the weights follow the new parameters
+    return cudaGetLastError();
+}
+
+}  // namespace lgc

@@ -543,11 +543,16 @@ lgc_status lgc_topk_scatter(lgc_ctx *c, float *update)
 lgc_status lgc_ae_train_step(lgc_ctx *c, float *loss_out)
 {
     if (!c) return LGC_ERR_INVALID_ARG;
-    if (c->cfg.variant != LGC_VARIANT_RAR || c->cfg.ae_kind != LGC_AE_CONV2)
-        return fail(c, LGC_ERR_UNSUPPORTED, "training is built for the ring-allreduce convolutional autoencoder");
+    if (c->cfg.variant != LGC_VARIANT_RAR || c->cfg.ae_kind == LGC_AE_IDENTITY)
+        return fail(c, LGC_ERR_UNSUPPORTED, "training is built for the ring-allreduce convolutional autoencoders");
     if (c->stage != Ctx::kSelected) return fail(c, LGC_ERR_BAD_STATE, "lgc_ae_train_step must follow lgc_topk");
-    cudaError_t e = launch_gather(*c);
-    if (e == cudaSuccess) e = launch_train_step(*c, loss_out);
+    cudaError_t e;
+    if (c->cfg.ae_kind == LGC_AE_CONV5) {
+        e = launch_ae5_train_step(*c, loss_out);       // its first convolution gathers the kept values itself
+    } else {
+        e = launch_gather(*c);
+        if (e == cudaSuccess) e = launch_train_step(*c, loss_out);
+    }
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_ae_train_step");
     return LGC_OK;
 }

@@ -98,6 +98,24 @@ struct Ae5 {
     CUtensorMap map_act_hi[3], map_act_lo[3], map_w_hi[3], map_w_lo[3];
     CUtensorMap map_dact_hi[3], map_dact_lo[3], map_dw_hi[3], map_dw_lo[3];
     bool weights_ready = false;         // w_hi / w_lo match the parameter vector
+    // ---- training step (lgc_ae_train_step) ----
+    float *act4_hi = nullptr, *act4_lo = nullptr;    // [K][L4][64] output of conv4 (inference folds it into conv5)
+    float *dact5_hi = nullptr, *dact5_lo = nullptr;  // [mu][32] output of deconv5 (inference folds it into the last conv)
+    float *g_enc[4] = {};               // dLoss/d(pre-activation) of conv1..conv4: [K][L_i][C_i]
+    float *g_dec[5] = {};               // the same for deconv1..deconv5: [L][C], g_dec[4] is [mu][32]
+    float *dzk = nullptr;               // [K][L4][4] gradient at every node's code
+    float *dzbar = nullptr;             // [L4][4]    gradient at the mean code
+    float *dr = nullptr;                // [mu]       gradient at the reconstruction
+    float *pbuf = nullptr;              // products dY W of a convolution, before they are folded onto the input positions
+    float *wt = nullptr;                // one layer's weights arranged for the backward GEMM
+    float *partial = nullptr;           // per-chunk partial sums of every parameter tensor's gradient
+    double *loss_part = nullptr;        // [loss_blocks]
+    int loss_blocks = 0;
+    struct Tensor {                     // one parameter tensor: where its partial sums live and how many chunks made them
+        int64_t param_off = 0, count = 0, partial_off = 0, rows = 0, chunk = 0;
+        int chunks = 0, kind = 0, cin = 0, cout = 0;
+    };
+    Tensor tensors[22];                 // encoder w,b x 5, decoder w,b x 6, in parameter order
 };
 
 struct Ctx {
@@ -199,11 +217,21 @@ cudaError_t launch_train_step(Ctx &c, float *loss_out);
 cudaError_t launch_encode_indices(Ctx &c, int node, unsigned char *out, int64_t capacity, unsigned long long *result);
 cudaError_t launch_train_step_ps(Ctx &c, int common, float lam_rec, float lam_sim, float *loss_out);
 // full-size autoencoder (lgc_ae5.cu)
+extern const int kAe5EncCh[5];        // channels through conv1..conv4 (conv5 maps the last to 4)
+extern const int kAe5DecCh[6];        // channels through deconv1..deconv5 (the last convolution maps them to 1)
 int64_t ae5_param_count();
 bool ae5_lengths(int64_t mu, int64_t (&len)[5]);
 void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used);   // base may be null (sizes only)
 cudaError_t ae5_make_maps(Ctx &c);
 cudaError_t launch_ae5_encode(Ctx &c);
 cudaError_t launch_ae5_decode(Ctx &c);
+// training: the forward pass that keeps every layer's output (lgc_ae5.cu), then the backward pass and Adam
+cudaError_t launch_ae5_train_forward(Ctx &c);
+cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out);
+struct AdamArgs {
+    float *params, *m, *v;
+    double lr, beta1, beta2, eps, corr1, corr2;
+};
+AdamArgs next_adam(Ctx &c);           // advances the step counter
 
 }  // namespace lgc

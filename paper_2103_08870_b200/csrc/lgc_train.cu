@@ -242,11 +242,6 @@ bwd_enc2_kernel(const float *__restrict__ dz, int64_t dz_stride, const float *__
     }
 }
 
-struct AdamArgs {
-    float *params, *m, *v;
-    double lr, beta1, beta2, eps, corr1, corr2;
-};
-
 // One CTA per parameter: reduce its gradient in fp64, then apply Adam to it.
 template <int C1, int C2>
 __global__ void __launch_bounds__(kRedThreads)
@@ -577,7 +572,7 @@ cudaError_t train_step_ps(Ctx &c, int common, float lam_rec, float lam_sim, floa
 
 }  // namespace
 
-static AdamArgs next_adam(Ctx &c)
+AdamArgs next_adam(Ctx &c)
 {
     c.adam_t += 1;
     AdamArgs ad;

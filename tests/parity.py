@@ -33,7 +33,8 @@ def assert_close(got, ref, what, rel=REL_TOL):
 
 
 def make_pair(numel, K, variant="rar", ae_kind="conv2", c1=8, c2=4, density_ppm=1000, momentum=0.9,
-              innovation_permille=100, seed=W.DEFAULT_SEED, topk_method="auto"):
+              innovation_permille=100, seed=W.DEFAULT_SEED, topk_method="auto", **adam):
+    """`adam`: lr, beta1, beta2, eps for both sides (defaults 1e-3, 0.9, 0.999, 1e-8)."""
     params = None
     if ae_kind == "conv2":
         params = W.ae_init_params(c1, c2, variant, K, seed)
@@ -41,9 +42,9 @@ def make_pair(numel, K, variant="rar", ae_kind="conv2", c1=8, c2=4, density_ppm=
         params = W.ae5_init_params(seed)
     ora = OracleLGC(numel, K, density_ppm=density_ppm, momentum=momentum, variant=variant, ae_kind=ae_kind,
                     c1=c1, c2=c2, params=None if params is None else params.numpy(),
-                    innovation_permille=innovation_permille, topk_method=topk_method)
+                    innovation_permille=innovation_permille, topk_method=topk_method, **adam)
     gpu = lgc.LGC(numel, K, density_ppm=density_ppm, momentum=momentum, variant=variant, ae_kind=ae_kind,
-                  c1=c1, c2=c2, innovation_permille=innovation_permille)
+                  c1=c1, c2=c2, innovation_permille=innovation_permille, **adam)
     if params is not None:
         gpu.set_ae_params(params)
     assert (gpu.N, gpu.mu) == (ora.N, ora.mu) and gpu.k_l == ora.k_l

@@ -362,3 +362,105 @@ def test_steps_from_host_buffers_back_to_back(variant, K, extra):
         large, served, _, _, _ = gpu.selection_stats()
         assert large > 0 and served > 0, "the row-by-row accumulation did not collect any candidates"
     gpu.check()
+
+
+def per_tensor(flat, shapes):
+    pos = 0
+    for name, shape in shapes:
+        n = int(np.prod(shape))
+        yield name, np.asarray(flat[pos:pos + n], dtype=np.float64)
+        pos += n
+
+
+def adam_moments(gpu):
+    """Adam's two moment vectors as the library keeps them behind the parameters (caller-owned buffer)."""
+    pad = (gpu.P + 3) // 4 * 4
+    return gpu.params_buf[pad:pad + gpu.P], gpu.params_buf[2 * pad:2 * pad + gpu.P]
+
+
+@pytest.mark.parametrize("numel, K", [([300_000, 5000, 120_000], 2), ([2_000_000, 700_000, 300_001], 3)])
+def test_full_size_autoencoder_gradients_and_first_steps(numel, K):
+    # Section IV-C's autoencoder, loss of Section IV-B.  mu = 425 (every GEMM tile ragged, a single chunk
+    # per gradient sum) and mu = 3000.  After the first step Adam's first moment is (1 - beta1) times the
+    # gradient, so every tensor's gradient is compared with the oracle's directly, at its own scale;
+    # then the parameters after that step, and the losses of two more steps on the same kept values.
+    from oracle import full_ae as A5
+    ora, gpu = make_pair(numel, K, ae_kind="conv5")
+    src = toy_source(numel, K, seed=41)
+    g = src.step(0) * 300.0                           # kept values of O(1)
+    ora.accumulate(g.numpy())
+    gpu.accumulate(g.cuda(), 0)
+    ora.topk(0)
+    gpu.topk(0)
+    loss_dev = torch.zeros(1, device="cuda")
+    _, grads_ref = ora.ae_loss_and_grads()
+    losses_ref, losses = [ora.ae_train_step()], []
+    gpu.ae_train_step(loss_dev)
+    losses.append(loss_dev.item())
+    m = adam_moments(gpu)[0].cpu().numpy().astype(np.float64)
+    for name, got in per_tensor(m / 0.1, A5.param_shapes()):
+        assert_close(got, grads_ref[name], f"gradient of {name}")
+    assert_close(gpu.get_ae_params().numpy(), ora.get_params(), "parameters after the first step")
+    for _ in range(2):
+        losses_ref.append(ora.ae_train_step())
+        gpu.ae_train_step(loss_dev)
+        losses.append(loss_dev.item())
+    assert_close(np.array(losses), np.array(losses_ref), "training losses")
+    assert losses[2] < losses[0]
+    assert_bitwise(gpu.val.cpu().numpy(), ora.val, "kept values")
+    gpu.check()
+
+
+def test_full_size_autoencoder_training_phase():
+    # Section V-B's second phase: fresh gradients every step, selection, one training step on the kept
+    # values, the sparse mean as the update; then a compression step with the trained autoencoder.
+    # Adam's step lr m^ / (sqrt(v^) + eps) amplifies a gradient's rounding error by up to lr / eps, so
+    # two correct runs in different precisions drift apart over the steps.  Each step is therefore
+    # compared from the same state: the oracle's parameters and moments, rounded to fp32, are given to
+    # both sides before every step (nothing of the library's flows into the oracle), and eps = 1e-2
+    # (above most gradients: close to the plain SGD the paper trains with) keeps the step itself well
+    # conditioned.  Per step: loss, every tensor's gradient (from the change of the first moment),
+    # the parameters after the step, the sparse update.
+    from oracle import full_ae as A5
+    numel, K = [2_000_000, 700_000, 300_001], 3
+    ora, gpu = make_pair(numel, K, ae_kind="conv5", lr=1e-3, eps=1e-2)
+    src = toy_source(numel, K, seed=41)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    loss_dev = torch.zeros(1, device="cuda")
+    m_dev, v_dev = adam_moments(gpu)
+    ora.adam_m = np.zeros(ora.get_params().size)
+    ora.adam_v = np.zeros(ora.get_params().size)
+    for t in range(4):
+        p32, m32, v32 = (x.astype(np.float32) for x in (ora.get_params(), ora.adam_m, ora.adam_v))
+        ora.set_params(p32.astype(np.float64))
+        ora.adam_m, ora.adam_v = m32.astype(np.float64), v32.astype(np.float64)
+        gpu.set_ae_params(torch.from_numpy(p32))
+        m_dev.copy_(torch.from_numpy(m32))
+        v_dev.copy_(torch.from_numpy(v32))
+        g = src.step(t) * 300.0
+        ora.accumulate(g.numpy())
+        gpu.accumulate(g.cuda(), t % K)
+        ora.topk(t % K)
+        gpu.topk(t % K, upd)
+        _, grads_ref = ora.ae_loss_and_grads()
+        loss_ref = ora.ae_train_step()
+        gpu.ae_train_step(loss_dev)
+        assert abs(loss_dev.item() - loss_ref) <= 1e-5 * loss_ref, f"loss at step {t}"
+        got = (m_dev.cpu().numpy().astype(np.float64) - 0.9 * m32) / 0.1
+        for name, gg in per_tensor(got, A5.param_shapes()):
+            # The leaky ReLU's derivative jumps at zero: a unit whose pre-activation lies within rounding of
+            # zero (about one in a million, so about one per step here) takes the other slope in fp32 than in
+            # fp64, which moves the gradient entries that pass through it by up to about 1e-2 of their
+            # tensor's scale (one row of a few hundred in a sum).  The test above holds the gradients to
+            # 1e-5 on two selections where no unit does.
+            assert_close(gg, grads_ref[name], f"gradient of {name} at step {t}", rel=3e-2)
+        assert_close(gpu.get_ae_params().numpy(), ora.get_params(), f"parameters after step {t}")
+        ref = ora.topk_scatter()
+        gpu.topk_scatter(upd)
+        assert_close(upd.cpu().numpy(), ref, f"sparse update at training step {t}")
+    gpu.check()
+    p32 = ora.get_params().astype(np.float32)
+    ora.set_params(p32.astype(np.float64))
+    gpu.set_ae_params(torch.from_numpy(p32))
+    g = src.step(4) * 300.0
+    compare_step(ora, gpu, g, g.cuda(), 1, upd)
