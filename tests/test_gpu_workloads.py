@@ -43,6 +43,36 @@ def test_resnet50_config_with_the_full_size_autoencoder():
     # the ResNet-50-shaped case, K = 8, with the autoencoder of Section IV-C: mu = 25,617, code 4 x 1600
     ora, gpu = run_workload("resnet50_ae5", 3, state_every=2)
     assert gpu.mu == 25_617 and gpu.code_len == 4 * 1600 and gpu.P == 216_729
+    # one training step of that autoencoder at this size (every gradient sum cut into 48 chunks): the
+    # loss, every tensor's gradient (Adam's first moment after a first step is a tenth of it) and the
+    # sparse update.  About eight of the 7 million leaky-ReLU units lie within rounding of zero here and
+    # take the other slope in fp32 than in fp64, hence the tolerance on the gradients (see
+    # test_full_size_autoencoder_training_phase in test_gpu_parity.py).
+    from oracle import full_ae as A5
+    w = W.workload("resnet50_ae5")
+    src = W.GradientSource(w.table, w.num_nodes, seed=w.seed, device="cuda")
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    g = torch.empty((w.num_nodes, gpu.N), dtype=torch.float32, device="cuda")
+    loss_dev = torch.zeros(1, device="cuda")
+    src.step_into(3, g)
+    leader = W.choice_for_step(w.seed, 3, w.num_nodes)
+    ora.accumulate(g.cpu().numpy())
+    gpu.accumulate(g, leader)
+    ora.topk(leader)
+    gpu.topk(leader, None)
+    _, grads_ref = ora.ae_loss_and_grads()
+    ref_loss = ora.ae_train_step()
+    gpu.ae_train_step(loss_dev)
+    assert_close(np.array([loss_dev.item()]), np.array([ref_loss]), "training loss")
+    pad = (gpu.P + 3) // 4 * 4
+    m = gpu.params_buf[pad:pad + gpu.P].cpu().numpy().astype(np.float64) / 0.1
+    pos = 0
+    for name, shape in A5.param_shapes():
+        n = int(np.prod(shape))
+        assert_close(m[pos:pos + n], grads_ref[name], f"gradient of {name}", rel=3e-2)
+        pos += n
+    assert_close(upd_after(gpu, upd), ora.topk_scatter(), "sparse update after the training step")
+    gpu.check()
 
 
 def test_resnet101_parameter_server_config():
