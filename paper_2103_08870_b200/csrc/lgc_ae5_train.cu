@@ -172,16 +172,46 @@ tn_gemm_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ par
     }
 }
 
-// partial[s][p] = sum over the rows of chunk s of A(m, p) (bias gradients).  Grid (chunks), 256 threads.
+// The same for a narrow right-hand side (at most four columns; B.hi == nullptr: one column of ones,
+// which makes the column sums of A, i.e. a bias gradient): partial[s][p][q] = sum_m A(m, p) B(m, q).
+// Grid (chunks), 256 threads: lane = column p (32 at a time), the eight warps stride over the rows
+// and are added up in warp order.
 __global__ void __launch_bounds__(256)
-colsum_kernel(Rows A, int64_t M, int64_t chunk, float *__restrict__ partial, int64_t pstride)
+tn_narrow_kernel(Rows A, Rows B, int Q, int64_t M, int64_t chunk, float *__restrict__ partial, int64_t pstride)
 {
+    __shared__ float part[8][32][4];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t first = (int64_t)blockIdx.x * chunk;
     const int64_t last = first + chunk < M ? first + chunk : M;
-    for (int p = threadIdx.x; p < A.len; p += 256) {
-        float acc = 0.f;
-        for (int64_t m = first; m < last; ++m) acc = __fadd_rn(acc, A.hi[A.at(m) + p]);
-        partial[(int64_t)blockIdx.x * pstride + p] = acc;
+    for (int p0 = 0; p0 < A.len; p0 += 32) {
+        const int p = p0 + lane;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int64_t m = first + warp; m < last; m += 8) {
+            float b[4] = {1.f, 0.f, 0.f, 0.f};
+            if (B.hi) {
+                const int64_t bb = B.at(m);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (q < Q) b[q] = B.lo ? __fadd_rn(B.hi[bb + q], B.lo[bb + q]) : B.hi[bb + q];
+            }
+            if (p < A.len) {
+                const int64_t ab = A.at(m) + p;
+                const float a = A.lo ? __fadd_rn(A.hi[ab], A.lo[ab]) : A.hi[ab];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[q] = __fmaf_rn(a, b[q], acc[q]);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) part[warp][lane][q] = acc[q];
+        __syncthreads();
+        if (warp == 0 && p < A.len) {
+            for (int q = 0; q < Q; ++q) {
+                float tot = 0.f;
+                for (int w = 0; w < 8; ++w) tot = __fadd_rn(tot, part[w][lane][q]);
+                partial[(int64_t)blockIdx.x * pstride + (int64_t)p * Q + q] = tot;
+            }
+        }
+        __syncthreads();
     }
 }
 
@@ -369,25 +399,33 @@ __global__ void code_bwd_kernel(const float *__restrict__ dzbar, int K, int64_t 
     }
 }
 
-// Gradient of one parameter tensor from its chunks' partial sums (fp64, chunk order), then Adam.
-//   kind 0 / 3: entry e is parameter e;  kind 1: e = (co, tau, ci) -> w[co][ci][tau];
-//   kind 2: e = (ci, tau, co) -> w[ci][co][tau].
-__global__ void reduce_adam_kernel(const float *__restrict__ partial, int chunks, int64_t pstride, int64_t count, int kind,
-                                   int cin, int cout, int64_t param_off, AdamArgs ad)
+// Gradient of every parameter from its tensor's per-chunk partial sums (fp64, chunk order), then Adam.
+//   kind 0 / 3: entry e of the tensor is parameter e;  kind 1: e = (co, tau, ci) -> w[co][ci][tau];
+//   kind 2: e = (ci, tau, co) -> w[ci][co][tau].   Thread per parameter; `first` lists the tensors' first threads.
+struct TensorTable {
+    int64_t first[23], param_off[22], partial_off[22], pstride[22];
+    int chunks[22], kind[22], cin[22], cout[22];
+};
+__global__ void reduce_adam_kernel(const float *__restrict__ partial, TensorTable tt, AdamArgs ad)
 {
-    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= count) return;
+    const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (id >= tt.first[22]) return;
+    int t = 0;
+    while (id >= tt.first[t + 1]) ++t;
+    const int64_t e = id - tt.first[t];
+    const float *part = partial + tt.partial_off[t];
     double g = 0.0;
-    for (int s = 0; s < chunks; ++s) g += (double)partial[(int64_t)s * pstride + e];
+    for (int s = 0; s < tt.chunks[t]; ++s) g += (double)part[(int64_t)s * tt.pstride[t] + e];
     int64_t i = e;
-    if (kind == 1) {
+    const int cin = tt.cin[t], cout = tt.cout[t];
+    if (tt.kind[t] == 1) {
         const int64_t co = e / (3 * cin), tau = e % (3 * cin) / cin, ci = e % cin;
         i = (co * cin + ci) * 3 + tau;
-    } else if (kind == 2) {
+    } else if (tt.kind[t] == 2) {
         const int64_t ci = e / (3 * cout), tau = e % (3 * cout) / cout, co = e % cout;
         i = (ci * cout + co) * 3 + tau;
     }
-    i += param_off;
+    i += tt.param_off[t];
     const double m = ad.beta1 * (double)ad.m[i] + (1.0 - ad.beta1) * g;
     const double v = ad.beta2 * (double)ad.v[i] + (1.0 - ad.beta2) * g * g;
     ad.m[i] = (float)m;
@@ -423,13 +461,15 @@ struct Launcher {
         tn_gemm_kernel<<<grid, 256, 0, c.stream>>>(A, B, T.rows, T.chunk, partial_of(t), pstride_of(t));
         ++g_kernel_launches;
     }
-    void colsum(int t, const Rows &A)
+    // the same with at most four columns on the right (B.hi == nullptr: column sums of A, a bias gradient)
+    void tn_narrow(int t, const Rows &A, const Rows &B, int Q)
     {
         if (!ok()) return;
         const Ae5::Tensor &T = a.tensors[t];
-        colsum_kernel<<<T.chunks, 256, 0, c.stream>>>(A, T.rows, T.chunk, partial_of(t), pstride_of(t));
+        tn_narrow_kernel<<<T.chunks, 256, 0, c.stream>>>(A, B, Q, T.rows, T.chunk, partial_of(t), pstride_of(t));
         ++g_kernel_launches;
     }
+    void colsum(int t, const Rows &A) { tn_narrow(t, A, rows_of(nullptr, nullptr, 0, 0, 1, 1), 1); }
     void arrange(const float *w, int cin, int cout, int mode)
     {
         if (!ok()) return;
@@ -458,7 +498,7 @@ cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out)
         ++g_kernel_launches;
     if (loss_out) loss_sum_kernel<<<1, 256, 0, s>>>(a.loss_part, a.loss_blocks, mu, loss_out), ++g_kernel_launches;
     const Rows dr_rows = rows_of(a.dr, nullptr, 0, 1, mu, 1);
-    L.tn(20, dr_rows, rows_of(a.dact5_hi, a.dact5_lo, 0, 32, mu, 32));
+    L.tn_narrow(20, rows_of(a.dact5_hi, a.dact5_lo, 0, 32, mu, 32), dr_rows, 1);     // dW6[c] = sum_p d5[p][c] dr[p]
     L.colsum(21, dr_rows);
 
     // ---- deconv5 .. deconv2: input of deconv i+1 is the output of deconv i ----
@@ -494,7 +534,7 @@ cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out)
         const Rows g = rows_of(a.g_enc[i], nullptr, lout * cout, cout, lout, cout);  // [K][lout][cout]
         L.colsum(2 * i + 1, g);
         if (i == 0) {        // conv1 reads the kept values themselves: rows of three floats, two apart
-            L.tn(0, g, rows_of(c.val, nullptr, mu, 2, lout, 3));
+            L.tn_narrow(0, g, rows_of(c.val, nullptr, mu, 2, lout, 3), 3);
             break;
         }
         const int64_t x_node = a.lpad[i - 1] * cin;
@@ -511,12 +551,15 @@ cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out)
 
     // ---- Adam on every tensor ----
     const AdamArgs ad = next_adam(c);
+    TensorTable tt;
+    tt.first[0] = 0;
     for (int t = 0; t < 22; ++t) {
         const Ae5::Tensor &T = a.tensors[t];
-        reduce_adam_kernel<<<blocks(T.count, 256), 256, 0, s>>>(L.partial_of(t), T.chunks, L.pstride_of(t), T.count, T.kind, T.cin,
-                                                                T.cout, T.param_off, ad),
-            ++g_kernel_launches;
+        tt.first[t + 1] = tt.first[t] + T.count;
+        tt.param_off[t] = T.param_off; tt.partial_off[t] = T.partial_off; tt.pstride[t] = L.pstride_of(t);
+        tt.chunks[t] = T.chunks; tt.kind[t] = T.kind; tt.cin[t] = T.cin; tt.cout[t] = T.cout;
     }
+    reduce_adam_kernel<<<blocks(tt.first[22], 256), 256, 0, s>>>(a.partial, tt, ad), ++g_kernel_launches;
     a.weights_ready = false;                       // the GEMM forms of the weights follow the new parameters
     return cudaGetLastError();
 }
