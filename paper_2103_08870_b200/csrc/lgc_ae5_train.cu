@@ -42,6 +42,21 @@ struct Rows {
     }
 };
 
+// Walks the rows m, m + step, m + 2 step, ... of a Rows without a division per row.
+struct RowCursor {
+    int64_t k, t;
+    __device__ __forceinline__ RowCursor(const Rows &r, int64_t m) : k(m / r.rows_per_node), t(m - (m / r.rows_per_node) * r.rows_per_node) {}
+    __device__ __forceinline__ int64_t at(const Rows &r) const { return k * r.node_stride + t * r.row_stride; }
+    __device__ __forceinline__ void advance(const Rows &r, int step)
+    {
+        t += step;
+        while (t >= r.rows_per_node) {
+            t -= r.rows_per_node;
+            ++k;
+        }
+    }
+};
+
 Rows rows_of(const float *hi, const float *lo, int64_t node_stride, int64_t row_stride, int64_t rows_per_node, int len)
 {
     Rows r;
@@ -137,12 +152,13 @@ tn_gemm_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ par
     const int64_t last = first + chunk < M ? first + chunk : M;
     float acc[4][4] = {};
     const int lr = threadIdx.x >> 4, lc = threadIdx.x & 15;          // 16 rows x 64 columns of each operand per trip
-    for (int64_t r0 = first; r0 < last; r0 += kStep) {
+    RowCursor ca(A, first + lr), cb(B, first + lr);
+    for (int64_t r0 = first; r0 < last; r0 += kStep, ca.advance(A, kStep), cb.advance(B, kStep)) {
         const int64_t m = r0 + lr;
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
         if (m < last) {
-            a = load4(A, A.at(m), p0 + 4 * lc);
-            b = load4(B, B.at(m), q0 + 4 * lc);
+            a = load4(A, ca.at(A), p0 + 4 * lc);
+            b = load4(B, cb.at(B), q0 + 4 * lc);
         }
         *reinterpret_cast<float4 *>(&As[lr][4 * lc]) = a;
         *reinterpret_cast<float4 *>(&Bs[lr][4 * lc]) = b;
@@ -174,8 +190,8 @@ tn_gemm_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ par
 
 // The same for a narrow right-hand side (at most four columns; B.hi == nullptr: one column of ones,
 // which makes the column sums of A, i.e. a bias gradient): partial[s][p][q] = sum_m A(m, p) B(m, q).
-// Grid (chunks), 256 threads: lane = column p (32 at a time), the eight warps stride over the rows
-// and are added up in warp order.
+// Grid (chunks, ceil(P / 32)), 256 threads: lane = column p, the eight warps stride over the rows and are
+// added up in warp order.
 __global__ void __launch_bounds__(256)
 tn_narrow_kernel(Rows A, Rows B, int Q, int64_t M, int64_t chunk, float *__restrict__ partial, int64_t pstride)
 {
@@ -183,35 +199,33 @@ tn_narrow_kernel(Rows A, Rows B, int Q, int64_t M, int64_t chunk, float *__restr
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t first = (int64_t)blockIdx.x * chunk;
     const int64_t last = first + chunk < M ? first + chunk : M;
-    for (int p0 = 0; p0 < A.len; p0 += 32) {
-        const int p = p0 + lane;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int64_t m = first + warp; m < last; m += 8) {
-            float b[4] = {1.f, 0.f, 0.f, 0.f};
-            if (B.hi) {
-                const int64_t bb = B.at(m);
+    const int p = blockIdx.y * 32 + lane;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    RowCursor ca(A, first + warp), cb(B, first + warp);
+    for (int64_t m = first + warp; m < last; m += 8, ca.advance(A, 8), cb.advance(B, 8)) {
+        float b[4] = {1.f, 0.f, 0.f, 0.f};
+        if (B.hi) {
+            const int64_t bb = cb.at(B);
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    if (q < Q) b[q] = B.lo ? __fadd_rn(B.hi[bb + q], B.lo[bb + q]) : B.hi[bb + q];
-            }
-            if (p < A.len) {
-                const int64_t ab = A.at(m) + p;
-                const float a = A.lo ? __fadd_rn(A.hi[ab], A.lo[ab]) : A.hi[ab];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) acc[q] = __fmaf_rn(a, b[q], acc[q]);
-            }
+            for (int q = 0; q < 4; ++q)
+                if (q < Q) b[q] = B.lo ? __fadd_rn(B.hi[bb + q], B.lo[bb + q]) : B.hi[bb + q];
         }
+        if (p < A.len) {
+            const int64_t ab = ca.at(A) + p;
+            const float a = A.lo ? __fadd_rn(A.hi[ab], A.lo[ab]) : A.hi[ab];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) part[warp][lane][q] = acc[q];
-        __syncthreads();
-        if (warp == 0 && p < A.len) {
-            for (int q = 0; q < Q; ++q) {
-                float tot = 0.f;
-                for (int w = 0; w < 8; ++w) tot = __fadd_rn(tot, part[w][lane][q]);
-                partial[(int64_t)blockIdx.x * pstride + (int64_t)p * Q + q] = tot;
-            }
+            for (int q = 0; q < 4; ++q) acc[q] = __fmaf_rn(a, b[q], acc[q]);
         }
-        __syncthreads();
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) part[warp][lane][q] = acc[q];
+    __syncthreads();
+    if (warp == 0 && p < A.len) {
+        for (int q = 0; q < Q; ++q) {
+            float tot = 0.f;
+            for (int w = 0; w < 8; ++w) tot = __fadd_rn(tot, part[w][lane][q]);
+            partial[(int64_t)blockIdx.x * pstride + (int64_t)p * Q + q] = tot;
+        }
     }
 }
 
@@ -466,7 +480,8 @@ struct Launcher {
     {
         if (!ok()) return;
         const Ae5::Tensor &T = a.tensors[t];
-        tn_narrow_kernel<<<T.chunks, 256, 0, c.stream>>>(A, B, Q, T.rows, T.chunk, partial_of(t), pstride_of(t));
+        tn_narrow_kernel<<<dim3(T.chunks, blocks(A.len, 32)), 256, 0, c.stream>>>(A, B, Q, T.rows, T.chunk, partial_of(t),
+                                                                                  pstride_of(t));
         ++g_kernel_launches;
     }
     void colsum(int t, const Rows &A) { tn_narrow(t, A, rows_of(nullptr, nullptr, 0, 0, 1, 1), 1); }
