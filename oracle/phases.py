@@ -57,7 +57,7 @@ class OraclePhased:
             o.accumulate(gs)
             o.topk(choice)
             if gr["mode"] == "topk" or phase == "topk_train":
-                if gr["mode"] == "ae" and o.ae_kind == "conv2":
+                if gr["mode"] == "ae" and o.ae_kind != "identity":
                     losses.append(o.ae_train_step() if o.variant == "rar" else o.ae_train_step_ps(choice, 1.0, 1.0))
                 upd[a:b] = o.topk_scatter()
             else:

@@ -50,7 +50,8 @@ def layer_runs(layer_numel: Sequence[int], layer_mode: Sequence[str]) -> List[Ru
 class PhasedLGC:
     def __init__(self, layer_numel: Sequence[int], layer_mode: Sequence[str], num_nodes: int, density_ppm: int = 1000,
                  momentum: float = 0.9, variant: str = "rar", ae_kind: str = "conv2", c1: int = 8, c2: int = 4,
-                 innovation_permille: int = 100, device: Optional[torch.device] = None):
+                 innovation_permille: int = 100, device: Optional[torch.device] = None, **adam):
+        """`adam`: lr, beta1, beta2, eps of the autoencoder's training steps (defaults 1e-3, 0.9, 0.999, 1e-8)."""
         self.numel = [int(n) for n in layer_numel]
         self.N, self.K, self.variant = sum(self.numel), int(num_nodes), variant
         self.runs = layer_runs(self.numel, layer_mode)
@@ -61,7 +62,7 @@ class PhasedLGC:
                 continue
             r.ctx = lgc.LGC(self.numel[r.first:r.last], num_nodes, density_ppm=density_ppm, momentum=momentum,
                             variant=variant, ae_kind=ae_kind if r.mode == "ae" else "identity", c1=c1, c2=c2,
-                            innovation_permille=innovation_permille, device=device, grad_row_stride=self.N)
+                            innovation_permille=innovation_permille, device=device, grad_row_stride=self.N, **adam)
 
     def ae_runs(self) -> List[Run]:
         return [r for r in self.runs if r.mode == "ae"]
@@ -86,7 +87,7 @@ class PhasedLGC:
             c.accumulate(g, choice)
             c.topk(choice, u)
             if r.mode == "topk" or phase == "topk_train":
-                if r.mode == "ae" and c.ae_kind == "conv2":
+                if r.mode == "ae" and c.ae_kind != "identity":
                     if self.variant == "rar":
                         c.ae_train_step(loss_out)
                     else:

@@ -56,6 +56,31 @@ def test_three_phases_against_the_oracle(variant, K):
     gpu.check()
 
 
+def test_three_phases_with_the_full_size_autoencoder():
+    # the same schedule with Section IV-C's autoencoder on the middle layers (mu = 96 kept values there).
+    # eps = 1e-2 keeps Adam's step well conditioned, so that the two sides' parameters stay together
+    # through the training phase (see test_full_size_autoencoder_training_phase in test_gpu_parity.py).
+    K = 2
+    params = W.ae5_init_params(5)
+    gpu = PhasedLGC(NUMEL, MODES, K, ae_kind="conv5", eps=1e-2)
+    gpu.ae_runs()[0].ctx.set_ae_params(params)
+    ora = OraclePhased(NUMEL, MODES, K, {1: params.numpy()}, ae_kind="conv5", eps=1e-2)
+    src = W.GradientSource(W.LayerTable("ph", NUMEL, [1, 2, 3, 1, 2, 3, 1]), K, seed=29)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    loss = torch.zeros(1, device="cuda")
+    for t, phase in enumerate(["raw"] + ["topk_train"] * 3 + ["compressed"] * 2):
+        g = src.step(t) * 300.0
+        choice = W.choice_for_step(5, t, K)
+        upd.fill_(float("nan"))
+        gpu.step(g.cuda(), upd, phase, choice, loss)
+        ref, losses = ora.step(g.numpy(), phase, choice)
+        assert_close(upd.cpu().numpy(), ref, f"step {t} ({phase}): update")
+        if losses:
+            assert_close(np.array([loss.item()]), np.array(losses), f"step {t}: training loss")
+    assert_close(gpu.ae_runs()[0].ctx.get_ae_params().numpy(), ora.groups[1]["o"].get_params(), "trained parameters")
+    gpu.check()
+
+
 def test_dense_mean_on_ragged_and_strided_rows():
     rng = np.random.default_rng(2)
     g = torch.from_numpy(rng.standard_normal((5, 10007)).astype(np.float32)).cuda()
