@@ -98,7 +98,7 @@ nn_gemm_kernel(Rows A, int64_t M, const float *__restrict__ B, int N, float *__r
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
     const int64_t m0 = (int64_t)blockIdx.y * kTile;
     const int n0 = blockIdx.x * kTile;
-    float acc[4][4] = {};
+    float2 acc[4][2] = {};
     const int ar = threadIdx.x >> 2, akq = threadIdx.x & 3;          // A tile: 64 rows x 16 entries, a float4 per thread
     const int64_t am = m0 + ar;
     const int64_t abase = am < M ? A.at(am) : 0;
@@ -114,11 +114,15 @@ nn_gemm_kernel(Rows A, int64_t M, const float *__restrict__ B, int N, float *__r
         for (int k = 0; k < kStep; ++k) {
             const float4 av = *reinterpret_cast<const float4 *>(&As[k][4 * ty]);
             const float4 bv = *reinterpret_cast<const float4 *>(&Bs[k][4 * tx]);
-            const float aa[4] = {av.x, av.y, av.z, av.w}, bb[4] = {bv.x, bv.y, bv.z, bv.w};
+            // packed fp32 FMAs (two per instruction on this architecture), each lane rounded like __fmaf_rn
+            const float aa[4] = {av.x, av.y, av.z, av.w};
+            const float2 b01 = make_float2(bv.x, bv.y), b23 = make_float2(bv.z, bv.w);
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = __fmaf_rn(aa[i], bb[j], acc[i][j]);
+            for (int i = 0; i < 4; ++i) {
+                const float2 a2 = make_float2(aa[i], aa[i]);
+                acc[i][0] = __ffma2_rn(a2, b01, acc[i][0]);
+                acc[i][1] = __ffma2_rn(a2, b23, acc[i][1]);
+            }
         }
         __syncthreads();
     }
@@ -128,7 +132,7 @@ nn_gemm_kernel(Rows A, int64_t M, const float *__restrict__ B, int N, float *__r
     for (int i = 0; i < 4; ++i) {
         const int64_t m = m0 + 4 * ty + i;
         if (m >= M) break;
-        float4 out = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+        float4 out = make_float4(acc[i][0].x, acc[i][0].y, acc[i][1].x, acc[i][1].y);
         if (MASK) {
             const int64_t xb = X.at(m);
             const float4 x = *reinterpret_cast<const float4 *>(X.hi + xb + n);   // the sign of the leading part is the value's
@@ -150,7 +154,7 @@ tn_gemm_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ par
     const int p0 = blockIdx.y * kTile, q0 = blockIdx.x * kTile;
     const int64_t first = (int64_t)blockIdx.z * chunk;
     const int64_t last = first + chunk < M ? first + chunk : M;
-    float acc[4][4] = {};
+    float2 acc[4][2] = {};
     const int lr = threadIdx.x >> 4, lc = threadIdx.x & 15;          // 16 rows x 64 columns of each operand per trip
     RowCursor ca(A, first + lr), cb(B, first + lr);
     for (int64_t r0 = first; r0 < last; r0 += kStep, ca.advance(A, kStep), cb.advance(B, kStep)) {
@@ -167,11 +171,15 @@ tn_gemm_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ par
         for (int k = 0; k < kStep; ++k) {
             const float4 av = *reinterpret_cast<const float4 *>(&As[k][4 * ty]);
             const float4 bv = *reinterpret_cast<const float4 *>(&Bs[k][4 * tx]);
-            const float aa[4] = {av.x, av.y, av.z, av.w}, bb[4] = {bv.x, bv.y, bv.z, bv.w};
+            // packed fp32 FMAs (two per instruction on this architecture), each lane rounded like __fmaf_rn
+            const float aa[4] = {av.x, av.y, av.z, av.w};
+            const float2 b01 = make_float2(bv.x, bv.y), b23 = make_float2(bv.z, bv.w);
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = __fmaf_rn(aa[i], bb[j], acc[i][j]);
+            for (int i = 0; i < 4; ++i) {
+                const float2 a2 = make_float2(aa[i], aa[i]);
+                acc[i][0] = __ffma2_rn(a2, b01, acc[i][0]);
+                acc[i][1] = __ffma2_rn(a2, b23, acc[i][1]);
+            }
         }
         __syncthreads();
     }
@@ -183,7 +191,7 @@ tn_gemm_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ par
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int q = q0 + 4 * tx + j;
-            if (q < B.len) out[(int64_t)p * B.len + q] = acc[i][j];
+            if (q < B.len) out[(int64_t)p * B.len + q] = j & 1 ? acc[i][j >> 1].y : acc[i][j >> 1].x;
         }
     }
 }
