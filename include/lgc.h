@@ -193,6 +193,14 @@ lgc_status lgc_dense_mean(const float *grads, int64_t row_stride, int32_t num_no
  * Valid from lgc_topk until the next lgc_accumulate. */
 lgc_status lgc_encode_indices(lgc_ctx *ctx, int32_t node, void *stream_out, size_t capacity, uint64_t *sizes_out);
 
+/* The same coding for the positions of node `node`'s innovation (parameter server, Algorithm 1: the
+ * node sends the top tenth of each layer's kept values, so the receiver must learn which of the
+ * kept slots they are): per layer the ascending slots inside the layer's run of kept values, the
+ * first gap counted from the run's first slot.  Same buffers, sizes and stream format as
+ * lgc_encode_indices.  Valid between lgc_combine and lgc_decode_scatter. */
+lgc_status lgc_encode_innovation_positions(lgc_ctx *ctx, int32_t node, void *stream_out, size_t capacity,
+                                           uint64_t *sizes_out);
+
 /* A whole compression step from host memory: uploads `host_grads` ([K][N], ideally pinned) to
  * `dev_grads`, runs the five stages, downloads the dense update to `host_update` ([N]).
  * The call returns without waiting; when the context's stream has drained, `host_update` is

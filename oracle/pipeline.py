@@ -134,10 +134,14 @@ class OracleLGC:
             return
         self.zc = self.z[common_node].copy()
         self.inn = np.zeros((self.K, self.mu), dtype=np.float32)
+        self.inn_pos = np.zeros((self.K, int(sum(self.ki_l))), dtype=np.int32)    # the kept slots the innovation holds
         for k in range(self.K):
+            at = 0
             for l in range(self.L):
                 a, b = int(self.koff[l]), int(self.koff[l + 1])
                 self.inn[k, a:b] = O.innovation(self.val[k, a:b], self.ki_l[l])
+                self.inn_pos[k, at:at + self.ki_l[l]] = O.topk(self.val[k, a:b], self.ki_l[l], base=a, method="sort")
+                at += self.ki_l[l]
 
     # -- stage 5 ------------------------------------------------------------------------
     def _dec(self, z: np.ndarray, prefix: str):

@@ -245,6 +245,9 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
     if (ps) {
         c.inn = cv.take<float>((size_t)p.K * p.mu);
         c.inn_pos = cv.take<int32_t>((size_t)p.K * p.muI);
+        c.inn_slot_layer = cv.take<int32_t>((size_t)p.muI);
+        c.kioff_dev = cv.take<int32_t>((size_t)p.L + 1);
+        c.koff64_dev = cv.take<int64_t>((size_t)p.L);
         carve_select(cv, c.sel_inn, plan_select(p.koff, p.k_l, p.ki_l, p.kioff), p.K);
     }
     if (conv && ps) {                       // training work space, one slice per node
@@ -395,6 +398,21 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     if (e == cudaSuccess) e = upload(c->koff_dev, koff32, s);
     std::vector<int64_t> layer_off(p.off.begin(), p.off.begin() + p.L);
     if (e == cudaSuccess) e = upload(c->layer_off_dev, layer_off, s);
+    std::vector<int32_t> inn_slot_layer, kioff32;
+    std::vector<int64_t> koff64;
+    if (cfg->variant == LGC_VARIANT_PS) {
+        inn_slot_layer.resize((size_t)p.muI);
+        kioff32.resize((size_t)p.L + 1);
+        koff64.assign(p.koff.begin(), p.koff.begin() + p.L);
+        for (int l = 0; l < p.L; ++l) {
+            kioff32[l] = (int32_t)p.kioff[l];
+            for (int64_t q = p.kioff[l]; q < p.kioff[l + 1]; ++q) inn_slot_layer[(size_t)q] = l;
+        }
+        kioff32[p.L] = (int32_t)p.muI;
+        if (e == cudaSuccess) e = upload(c->inn_slot_layer, inn_slot_layer, s);
+        if (e == cudaSuccess) e = upload(c->kioff_dev, kioff32, s);
+        if (e == cudaSuccess) e = upload(c->koff64_dev, koff64, s);
+    }
     if (e == cudaSuccess && cfg->ae_kind == LGC_AE_CONV5) e = ae5_make_maps(*c);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) {
@@ -595,6 +613,22 @@ lgc_status lgc_encode_indices(lgc_ctx *c, int32_t node, void *stream_out, size_t
     const cudaError_t e = launch_encode_indices(*c, node, static_cast<unsigned char *>(stream_out), (int64_t)capacity,
                                                 reinterpret_cast<unsigned long long *>(sizes_out));
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_encode_indices");
+    return LGC_OK;
+}
+
+lgc_status lgc_encode_innovation_positions(lgc_ctx *c, int32_t node, void *stream_out, size_t capacity, uint64_t *sizes_out)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (c->cfg.variant != LGC_VARIANT_PS) return fail(c, LGC_ERR_UNSUPPORTED, "only the parameter-server variant has innovations");
+    if (!stream_out || !sizes_out || capacity < 4 || capacity % 4 != 0 || (reinterpret_cast<uintptr_t>(stream_out) & 3) != 0 ||
+        (reinterpret_cast<uintptr_t>(sizes_out) & 7) != 0)
+        return fail(c, LGC_ERR_INVALID_ARG, "lgc_encode_innovation_positions: buffers must be non-NULL, the stream 4-byte aligned with a capacity that is a multiple of 4");
+    if (c->stage != Ctx::kCombined)
+        return fail(c, LGC_ERR_BAD_STATE, "lgc_encode_innovation_positions needs the innovations of this step's lgc_combine");
+    if (node < 0 || node >= c->K) return fail(c, LGC_ERR_INVALID_ARG, "node out of range");
+    const cudaError_t e = launch_encode_innovation_positions(*c, node, static_cast<unsigned char *>(stream_out), (int64_t)capacity,
+                                                             reinterpret_cast<unsigned long long *>(sizes_out));
+    if (e != cudaSuccess) return cuda_fail(c, e, "lgc_encode_innovation_positions");
     return LGC_OK;
 }
 

@@ -269,4 +269,16 @@ cudaError_t launch_encode_indices(Ctx &c, int node, unsigned char *out, int64_t 
     return cudaGetLastError();
 }
 
+// The same coding for a node's innovation positions (parameter server): ascending slots inside each
+// layer's run of kept values, gaps counted from the run's first slot.
+cudaError_t launch_encode_innovation_positions(Ctx &c, int node, unsigned char *out, int64_t capacity,
+                                               unsigned long long *result)
+{
+    deflate_indices_kernel<<<1, kIcThreads, 0, c.stream>>>(c.inn_pos + (int64_t)node * c.muI, c.inn_slot_layer, c.kioff_dev,
+                                                          c.koff64_dev, c.muI, c.ic_bytes, reinterpret_cast<uint32_t *>(out),
+                                                          capacity, result),
+        ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
 }  // namespace lgc

@@ -138,6 +138,9 @@ struct Ctx {
     float *combined = nullptr;     // [code_len]
     float *inn = nullptr;          // [K][mu]
     int32_t *inn_pos = nullptr;    // [K][muI]
+    int32_t *inn_slot_layer = nullptr; // [muI] layer of each innovation slot (parameter server)
+    int32_t *kioff_dev = nullptr;  // [L + 1] first innovation slot of each layer
+    int64_t *koff64_dev = nullptr; // [L] first kept slot of each layer: where a layer's innovation positions count from
     float *recon = nullptr;        // [S][mu]
     int32_t *slot_layer = nullptr; // [mu] layer of each kept slot
     int32_t *koff_dev = nullptr;   // [L + 1]
@@ -215,6 +218,8 @@ cudaError_t launch_decode_scatter(Ctx &c, float *update);
 cudaError_t launch_topk_scatter(Ctx &c, float *update);
 cudaError_t launch_train_step(Ctx &c, float *loss_out);
 cudaError_t launch_encode_indices(Ctx &c, int node, unsigned char *out, int64_t capacity, unsigned long long *result);
+cudaError_t launch_encode_innovation_positions(Ctx &c, int node, unsigned char *out, int64_t capacity,
+                                               unsigned long long *result);
 cudaError_t launch_train_step_ps(Ctx &c, int common, float lam_rec, float lam_sim, float *loss_out);
 // full-size autoencoder (lgc_ae5.cu)
 extern const int kAe5EncCh[5];        // channels through conv1..conv4 (conv5 maps the last to 4)

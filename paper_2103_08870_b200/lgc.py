@@ -22,7 +22,7 @@ AE_CONV2, AE_IDENTITY, AE_CONV5 = 0, 1, 2
 EXPORTS = (
     "lgc_workspace_bytes", "lgc_init", "lgc_destroy", "lgc_accumulate", "lgc_topk", "lgc_encode",
     "lgc_combine", "lgc_decode_scatter", "lgc_topk_scatter", "lgc_ae_train_step", "lgc_ae_train_step_ps",
-    "lgc_encode_indices", "lgc_dense_mean", "lgc_step_host",
+    "lgc_encode_indices", "lgc_encode_innovation_positions", "lgc_dense_mean", "lgc_step_host",
     "lgc_get_layout", "lgc_keep_counts", "lgc_get_buffers", "lgc_set_ae_params", "lgc_get_ae_params",
     "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc", "lgc_kernel_launches", "lgc_selection_stats",
 )
@@ -62,6 +62,7 @@ def lib() -> C.CDLL:
         l.lgc_ae_train_step.argtypes = [vp, vp]
         l.lgc_ae_train_step_ps.argtypes = [vp, C.c_int32, C.c_float, C.c_float, vp]
         l.lgc_encode_indices.argtypes = [vp, C.c_int32, vp, C.c_size_t, vp]
+        l.lgc_encode_innovation_positions.argtypes = [vp, C.c_int32, vp, C.c_size_t, vp]
         l.lgc_dense_mean.argtypes = [vp, C.c_int64, C.c_int32, C.c_int64, vp, vp]
         l.lgc_step_host.argtypes = [vp, vp, vp, vp, vp, C.c_int32]
         l.lgc_get_layout.argtypes = [vp] + [C.POINTER(C.c_int64)] * 5
@@ -250,6 +251,15 @@ class LGC:
             raise ValueError("sizes_out: need an int64 CUDA tensor of 2 elements")
         self._ok(self._l.lgc_encode_indices(self._ctx, node, stream_out.data_ptr(), stream_out.numel(), sizes_out.data_ptr()),
                  "lgc_encode_indices")
+
+    def encode_innovation_positions(self, node: int, stream_out: torch.Tensor, sizes_out: torch.Tensor) -> None:
+        """The same for the positions of `node`'s innovation (parameter server; between combine and decode_scatter)."""
+        if not (stream_out.is_cuda and stream_out.dtype == torch.uint8 and stream_out.is_contiguous()):
+            raise ValueError("stream_out: need a contiguous uint8 CUDA tensor")
+        if not (sizes_out.is_cuda and sizes_out.dtype == torch.int64 and sizes_out.numel() == 2):
+            raise ValueError("sizes_out: need an int64 CUDA tensor of 2 elements")
+        self._ok(self._l.lgc_encode_innovation_positions(self._ctx, node, stream_out.data_ptr(), stream_out.numel(),
+                                                         sizes_out.data_ptr()), "lgc_encode_innovation_positions")
 
     def step(self, grads: torch.Tensor, update: torch.Tensor, choice: int = 0) -> None:
         """The five stages of one compression step, in order."""

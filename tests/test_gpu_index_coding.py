@@ -79,3 +79,44 @@ def test_resnet50_shaped_list_and_compression_ratio():
     leader = IC.compression_ratio(gpu.N, code_floats, n_stream)
     others = IC.compression_ratio(gpu.N, code_floats, 0)
     assert 300 < leader < others == 4.0 * gpu.N / (4.0 * code_floats)
+
+
+def test_parameter_server_innovation_positions_and_ratio():
+    # Algorithm 1: besides its code (one node) every node sends the top tenth of each layer's kept
+    # values; the receiver needs their slots.  The stream of those slots (counted inside each layer's
+    # run of kept values) must inflate to the oracle's varint bytes and decode to the oracle's slots.
+    numel = [400_000, 9000, 50_000, 64]
+    K = 3
+    ora, gpu = make_pair(numel, K, variant="ps", density_ppm=5000)
+    g = W.GradientSource(W.LayerTable("ic", numel, [1, 2, 3, 1]), K, seed=8).step(0)
+    ora.accumulate(g.numpy())
+    gpu.accumulate(g.cuda())
+    ora.topk()
+    gpu.topk(0)
+    ora.encode()
+    gpu.encode()
+    ora.combine(1)
+    gpu.combine(1)
+    kioff = np.concatenate([[0], np.cumsum(ora.ki_l)])
+    for k in range(K):
+        ref_bytes = IC.varint_bytes(ora.inn_pos[k], ora.koff[:-1], kioff)
+        out = torch.full((8 * gpu.mu + 1024,), 0xEE, dtype=torch.uint8, device="cuda")
+        sizes = torch.zeros(2, dtype=torch.int64, device="cuda")
+        gpu.encode_innovation_positions(k, out, sizes)
+        n_stream, n_bytes = (int(x) for x in sizes.cpu())
+        gpu.check()
+        assert n_bytes == len(ref_bytes)
+        stream = out[:n_stream].cpu().numpy().tobytes()
+        assert IC.inflate(stream) == ref_bytes
+        assert np.array_equal(IC.indices_from_varint(IC.inflate(stream), ora.koff[:-1], kioff), ora.inn_pos[k])
+        assert IC.entropy_bytes(ref_bytes) <= n_stream <= 1.05 * len(IC.deflate(ref_bytes)) + 160
+    # Section VI-A's ratio for a node that is not the common one: innovation values + both streams
+    idx_sizes = torch.zeros(2, dtype=torch.int64, device="cuda")
+    gpu.encode_indices(0, out, idx_sizes)
+    ratio = IC.compression_ratio(gpu.N, 0, int(idx_sizes[0]) + n_stream, extra_floats=int(kioff[-1]))
+    assert ratio > 100
+    upd = torch.empty(gpu.N, device="cuda")
+    gpu.decode_scatter(upd)
+    ora.decode_scatter()
+    with pytest.raises(Exception):                       # the innovations belong to the step that made them
+        gpu.encode_innovation_positions(0, out, sizes)

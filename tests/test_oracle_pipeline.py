@@ -311,3 +311,26 @@ def test_momentum_zero_is_plain_error_feedback():
         resid = acc.copy()
         resid[:, o.idx[0]] = 0                        # only the unsent part stays
         assert np.array_equal(o.v, resid)
+
+
+def test_ps_innovation_positions_are_the_slots_of_the_nonzero_innovation_entries():
+    # the innovation keeps, per layer, the kI_l kept values of largest magnitude: its positions list
+    # is ascending inside each layer, has kI_l entries per layer, and names exactly the slots where
+    # the innovation vector is non-zero (random values: no kept value is zero)
+    from oracle import OracleLGC
+    numel = [3000, 800, 64, 5000]
+    rng = np.random.default_rng(12)
+    ora = OracleLGC(numel, 2, density_ppm=20000, variant="ps", ae_kind="identity")
+    ora.accumulate(rng.standard_normal((2, ora.N)).astype(np.float32))
+    ora.topk()
+    ora.encode()
+    ora.combine(0)
+    kioff = np.concatenate([[0], np.cumsum(ora.ki_l)])
+    for k in range(2):
+        assert np.array_equal(np.flatnonzero(ora.inn[k]), np.sort(ora.inn_pos[k]))
+        for l in range(len(numel)):
+            seg = ora.inn_pos[k, kioff[l]:kioff[l + 1]]
+            assert len(seg) == ora.ki_l[l] and np.all(np.diff(seg) > 0)
+            assert ora.koff[l] <= seg[0] and seg[-1] < ora.koff[l + 1]
+            kept = np.abs(ora.val[k, ora.koff[l]:ora.koff[l + 1]])
+            assert np.sort(kept)[::-1][:ora.ki_l[l]].min() == np.abs(ora.val[k, seg]).min()
