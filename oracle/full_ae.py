@@ -27,6 +27,10 @@ reordering.  Pinned in tests/test_oracle_full_ae.py against torch's CPU convolut
 parameter counts the tables imply, and the length chain.  The training step (loss of Section
 IV-B, derivative of every layer, written the same way) is pinned there against torch's autograd
 on the same graph, central differences of the loss, and the cases where loss and gradients vanish.
+The parameter-server form (Section IV-A: one decoder per node, the node's innovation concatenated
+with the decoder's 32 feature channels in front of the last convolution) is pinned against the
+same construction with torch.cat and torch's convolutions and by the last filters that reduce it
+to the innovation alone and to the ring-allreduce decoder.
 """
 from __future__ import annotations
 
@@ -48,6 +52,17 @@ def param_shapes() -> List[Tuple[str, Tuple[int, ...]]]:
     for i in range(5):
         out += [(f"dec.w{i + 1}", (DEC_CH[i], DEC_CH[i + 1], 3)), (f"dec.b{i + 1}", (DEC_CH[i + 1],))]
     out += [("dec.w6", (1, DEC_CH[5], 1)), ("dec.b6", (1,))]
+    return out
+
+
+def param_shapes_ps(K: int) -> List[Tuple[str, Tuple[int, ...]]]:
+    """Parameter-server form (Section IV-A): one encoder, one decoder per node; the node's innovation
+    joins its decoder as a 33rd channel in front of the last convolution."""
+    out = [t for t in param_shapes() if t[0].startswith("enc.")]
+    for k in range(K):
+        for i in range(5):
+            out += [(f"dec{k}.w{i + 1}", (DEC_CH[i], DEC_CH[i + 1], 3)), (f"dec{k}.b{i + 1}", (DEC_CH[i + 1],))]
+        out += [(f"dec{k}.w6", (1, DEC_CH[5] + 1, 1)), (f"dec{k}.b6", (1,))]
     return out
 
 
@@ -122,16 +137,20 @@ def encode(x: np.ndarray, p: Dict[str, np.ndarray]) -> np.ndarray:
     return conv_k1(h, p["enc.w5"], p["enc.b5"])
 
 
-def decode(z: np.ndarray, p: Dict[str, np.ndarray], mu: int) -> np.ndarray:
-    """code[4][L4] -> reconstruction[mu]."""
+def decode(z: np.ndarray, p: Dict[str, np.ndarray], mu: int, prefix: str = "dec", inn: np.ndarray = None) -> np.ndarray:
+    """code[4][L4] -> reconstruction[mu].  With `inn` (parameter server, Section IV-A: the innovation is
+    concatenated with the decoder's features before the last convolution) the last convolution sees
+    33 channels, the 33rd being the innovation vector."""
     ln = lengths(mu)
-    d = leaky(convt_k3s1p1(z, p["dec.w1"], p["dec.b1"]))
+    d = leaky(convt_k3s1p1(z, p[f"{prefix}.w1"], p[f"{prefix}.b1"]))
     for i in range(2, 6):                     # deconv2..5 undo conv4..conv1
         enc_in = ln[5 - i]                    # length the mirrored encoder layer saw
-        d = convt_k3s2(d, p[f"dec.w{i}"], p[f"dec.b{i}"], (enc_in - 3) % 2)
+        d = convt_k3s2(d, p[f"{prefix}.w{i}"], p[f"{prefix}.b{i}"], (enc_in - 3) % 2)
         assert d.shape[1] == enc_in
         d = leaky(d)
-    return conv_k1(d, p["dec.w6"], p["dec.b6"]).reshape(-1)
+    if inn is not None:
+        d = np.concatenate([d, np.asarray(inn, dtype=np.float64).reshape(1, -1)], axis=0)
+    return conv_k1(d, p[f"{prefix}.w6"], p[f"{prefix}.b6"]).reshape(-1)
 
 
 def rar_forward(val: np.ndarray, p: Dict[str, np.ndarray]):

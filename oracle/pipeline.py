@@ -46,7 +46,6 @@ class OracleLGC:
                  innovation_permille: int = 100, lr: float = 1e-3, beta1: float = 0.9,
                  beta2: float = 0.999, eps: float = 1e-8, topk_method: str = "auto"):
         assert variant in ("rar", "ps") and ae_kind in ("conv2", "identity", "conv5")
-        assert ae_kind != "conv5" or variant == "rar"
         self.numel = [int(n) for n in layer_numel]
         self.L = len(self.numel)
         self.K = int(num_nodes)
@@ -67,7 +66,10 @@ class OracleLGC:
         self.op1 = (self.L1 - 3) % 2 if self.L1 >= 3 else 0   # decoder layer 1: L2 -> L1
         self.op2 = (self.mu - 3) % 2 if self.mu >= 3 else 0   # decoder layer 2: L1 -> mu
         self.p: Dict[str, np.ndarray] = {}
-        self.order = A5.param_shapes() if ae_kind == "conv5" else _param_order(c1, c2, variant, self.K)
+        if ae_kind == "conv5":
+            self.order = A5.param_shapes() if variant == "rar" else A5.param_shapes_ps(self.K)
+        else:
+            self.order = _param_order(c1, c2, variant, self.K)
         if params is not None:
             self.set_params(params)
         self.adam_m = self.adam_v = None
@@ -159,6 +161,9 @@ class OracleLGC:
             return
         self.r = np.empty((self.K, self.mu), dtype=np.float64)
         for k in range(self.K):
+            if self.ae_kind == "conv5":      # full-size decoder of node k, its innovation as the 33rd channel
+                self.r[k] = A5.decode(self.zc, self.p, self.mu, prefix=f"dec{k}", inn=self.inn[k])
+                continue
             if self.ae_kind == "identity":
                 y = self.zc.reshape(-1)
                 w0, w1, b = 1.0, 1.0, 0.0

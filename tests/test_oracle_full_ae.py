@@ -206,3 +206,89 @@ def test_training_step_moves_every_parameter_against_its_gradient():
     assert big.sum() > 1000
     assert np.allclose(after[big] - before[big], -1e-3 * np.sign(gf[big]), rtol=2e-3, atol=0)
     assert ora.ae_train_step() < loss          # and the loss goes down
+
+
+# ---- parameter-server form (Section IV-A): one decoder per node, the innovation as a 33rd channel ----
+
+def rand_params_ps(K, seed=0):
+    rng = np.random.default_rng(seed)
+    n = sum(int(np.prod(s)) for _, s in A.param_shapes_ps(K))
+    return rng.uniform(-0.3, 0.3, size=n)
+
+
+def unpack_ps(flat, K):
+    out, pos = {}, 0
+    for name, shape in A.param_shapes_ps(K):
+        n = int(np.prod(shape))
+        out[name] = flat[pos:pos + n].reshape(shape)
+        pos += n
+    assert pos == flat.size
+    return out
+
+
+def test_ps_parameter_count_one_encoder_and_one_decoder_per_node():
+    shapes = A.param_shapes_ps(3)
+    assert sum(int(np.prod(s)) for _, s in shapes) == 172_996 + 3 * (43_733 + 1)    # the last filter has one more tap
+    assert [n for n, _ in shapes if n.endswith(".w6")] == ["dec0.w6", "dec1.w6", "dec2.w6"]
+
+
+def test_ps_decoder_against_torch_concatenation():
+    # the definition itself with torch's CPU ops: transposed convolutions, then torch.cat of the 32
+    # feature channels with the innovation, then a 1-tap convolution over 33 channels
+    rng = np.random.default_rng(21)
+    mu, K = 130, 2
+    p = unpack_ps(rand_params_ps(K, 21), K)
+    z = rng.standard_normal((4, A.lengths(mu)[4]))
+    inn = np.where(rng.random((K, mu)) < 0.1, rng.standard_normal((K, mu)), 0.0).astype(np.float32)
+    ln = A.lengths(mu)
+    for k in range(K):
+        tp = {n[len(f"dec{k}."):]: torch.from_numpy(np.ascontiguousarray(v)) for n, v in p.items() if n.startswith(f"dec{k}.")}
+        d = F.leaky_relu(F.conv_transpose1d(torch.from_numpy(z)[None], tp["w1"], tp["b1"], stride=1, padding=1), 0.01)
+        for i in range(2, 6):
+            d = F.leaky_relu(F.conv_transpose1d(d, tp[f"w{i}"], tp[f"b{i}"], stride=2, output_padding=(ln[5 - i] - 3) % 2), 0.01)
+        cat = torch.cat([d, torch.from_numpy(inn[k].astype(np.float64))[None, None]], dim=1)
+        ref = F.conv1d(cat, tp["w6"], tp["b6"]).reshape(-1).numpy()
+        got = A.decode(z, p, mu, prefix=f"dec{k}", inn=inn[k])
+        assert np.abs(got - ref).max() <= 1e-12 * max(1.0, np.abs(ref).max())
+
+
+def test_ps_special_last_filters():
+    from oracle import OracleLGC
+    numel = [60_000, 30_000]
+    K = 3
+    flat = rand_params_ps(K, 3)
+    p = unpack_ps(flat, K)
+    rng = np.random.default_rng(3)
+    g = rng.standard_normal((K, sum(numel))).astype(np.float32)
+
+    def run(params):
+        ora = OracleLGC(numel, K, variant="ps", ae_kind="conv5", params=params)
+        ora.accumulate(g)
+        ora.topk()
+        ora.encode()
+        ora.combine(1)
+        ora.decode()
+        return ora
+
+    # (a) last filter = the innovation channel alone: every node reconstructs exactly its innovation
+    for k in range(K):
+        p[f"dec{k}.w6"][...] = 0.0
+        p[f"dec{k}.w6"][0, 32, 0] = 1.0
+        p[f"dec{k}.b6"][...] = 0.0
+    ora = run(flat)
+    assert np.array_equal(ora.r, ora.inn.astype(np.float64))
+    # (b) the innovation channel switched off and all decoders alike: every node gets the ring-allreduce
+    # decoder's output for the common node's code
+    flat2 = rand_params_ps(K, 4)
+    q = unpack_ps(flat2, K)
+    for k in range(K):
+        for name in ("w1", "b1", "w2", "b2", "w3", "b3", "w4", "b4", "w5", "b5", "w6", "b6"):
+            q[f"dec{k}.{name}"][...] = q[f"dec0.{name}"]
+        q[f"dec{k}.w6"][0, 32, 0] = 0.0
+    ora = run(flat2)
+    rar = {n.replace("dec0.", "dec."): v for n, v in q.items() if n.startswith("dec0.") or n.startswith("enc.")}
+    rar["dec.w6"] = rar["dec.w6"][:, :32, :]
+    ref = A.decode(ora.z[1], rar, ora.mu)
+    for k in range(K):
+        assert np.array_equal(ora.r[k], ref)
+    assert np.array_equal(ora.zc, ora.z[1])
