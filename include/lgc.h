@@ -53,12 +53,15 @@ typedef enum {
 typedef enum { LGC_VARIANT_RAR = 0, LGC_VARIANT_PS = 1 } lgc_variant;
 /* CONV2: two stride-2 convolutions each way with (ae_c1, ae_c2) channels.  IDENTITY: no autoencoder.
  * CONV5: the autoencoder of the paper's Section IV-C (encoder filters 64/128/256/64/4, decoder filters
- * 4/32/64/128/32 and a 1x1 convolution, leaky ReLU); ring-allreduce only, mu >= 31;
- * ae_c1 / ae_c2 are ignored.  Parameter vector: per layer the weights then the bias, encoder
- * conv1..conv5 (w[co][ci][tap]) then decoder deconv1..deconv5 (w[ci][co][tap]) and the final
- * convolution; 216,729 floats.  deconv1 has stride 1 and padding 1, the others stride 2 with the
- * output padding that returns each length to the one the mirrored encoder layer saw.  Codes are
- * stored position-major: code[K][L4][4]. */
+ * 4/32/64/128/32 and a 1x1 convolution, leaky ReLU); mu >= 31; ae_c1 / ae_c2 are ignored.
+ * Parameter vector: per layer the weights then the bias, encoder conv1..conv5 (w[co][ci][tap])
+ * then decoder deconv1..deconv5 (w[ci][co][tap]) and the final convolution; 216,729 floats for
+ * the ring-allreduce variant.  Parameter server (Section IV-A): the encoder (172,996 floats), then
+ * one decoder per node, whose final convolution has a 33rd weight, on the node's innovation, which
+ * joins the decoder's 32 feature channels in front of that convolution (43,734 floats per decoder).
+ * deconv1 has stride 1 and padding 1, the others stride 2 with the output padding that returns each
+ * length to the one the mirrored encoder layer saw.  Codes are stored position-major:
+ * code[K][L4][4].  Training (lgc_ae_train_step) is built for the ring-allreduce variant. */
 typedef enum { LGC_AE_CONV2 = 0, LGC_AE_IDENTITY = 1, LGC_AE_CONV5 = 2 } lgc_ae_kind;
 
 /*

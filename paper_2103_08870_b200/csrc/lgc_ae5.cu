@@ -135,8 +135,8 @@ __device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&x)[32])
 // as (hi, lo).  Grid (ceil(L1 / 64), K), 256 threads: thread = (position, group of 16 channels).
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-ae5_conv1_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restrict__ idx, int64_t mu, int64_t L1,
-                 int64_t Lpad1, const float *__restrict__ w1, const float *__restrict__ b1, float *__restrict__ val,
+ae5_conv1_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restrict__ idx, int64_t idx_node_stride, int64_t mu,
+                 int64_t L1, int64_t Lpad1, const float *__restrict__ w1, const float *__restrict__ b1, float *__restrict__ val,
                  float *__restrict__ a_hi, float *__restrict__ a_lo)
 {
     __shared__ float x[2 * 64 + 2];
@@ -149,7 +149,7 @@ ae5_conv1_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restri
         const int64_t p = 2 * t0 + i;
         float xv = 0.0f;
         if (p < mu) {
-            xv = v[(int64_t)k * N + idx[p]];
+            xv = v[(int64_t)k * N + idx[(int64_t)k * idx_node_stride + p]];   // ring-allreduce: one list (stride 0)
             val[(int64_t)k * mu + p] = xv;           // the two slots shared with the next CTA are written by
         }                                            // both, with the same value
         x[i] = xv;
@@ -256,7 +256,7 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
                 const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
                 const float *__restrict__ bias, int64_t L_out, int64_t Lpad_out, float *__restrict__ out_hi,
                 float *__restrict__ out_lo, const float *__restrict__ w_last, const float *__restrict__ b_last,
-                float *__restrict__ out_last, int32_t *errword)
+                float *__restrict__ out_last, const float *__restrict__ extra, int32_t *errword)
 {
     using S = GemmShape<MODE, CIN, COUT>;
     constexpr int N = S::kN;
@@ -279,7 +279,10 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
     }
     if (MODE == kDeconvFinal) {
         if (threadIdx.x < 32) s_wl[threadIdx.x] = w_last[threadIdx.x];
-        if (threadIdx.x == 0) s_bl[0] = b_last[0];
+        if (threadIdx.x == 0) {
+            s_bl[0] = b_last[0];
+            s_bl[1] = extra ? w_last[32] : 0.0f;          // parameter server: the filter's tap on the innovation channel
+        }
     }
     if (threadIdx.x == 0) {
         failed = 0;
@@ -426,8 +429,14 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
                 make_float4(__fadd_rn(last[0], s_bl[0]), __fadd_rn(last[1], s_bl[1]), __fadd_rn(last[2], s_bl[2]),
                             __fadd_rn(last[3], s_bl[3]));
         if (MODE == kDeconvFinal) {
-            if (2 * t < L_out) out_last[2 * t] = __fadd_rn(last[0], s_bl[0]);
-            if (2 * t + 1 < L_out) out_last[2 * t + 1] = __fadd_rn(last[1], s_bl[0]);
+            if (2 * t < L_out) {
+                const float y = __fadd_rn(last[0], s_bl[0]);
+                out_last[2 * t] = extra ? __fmaf_rn(s_bl[1], extra[2 * t], y) : y;
+            }
+            if (2 * t + 1 < L_out) {
+                const float y = __fadd_rn(last[1], s_bl[0]);
+                out_last[2 * t + 1] = extra ? __fmaf_rn(s_bl[1], extra[2 * t + 1], y) : y;
+            }
         }
     } else if (threadIdx.x == 0) {
         atomicExch(errword, 0x5EA5);                              // a wait ran out
@@ -564,7 +573,8 @@ bool make_matrix_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int k, int 
 template <int MODE, int CIN, int COUT>
 cudaError_t launch_gemm(Ctx &c, const CUtensorMap &a_hi, const CUtensorMap &a_lo, const CUtensorMap &b_hi,
                         const CUtensorMap &b_lo, const float *bias, int64_t rows, int nodes, int64_t L_out, int64_t Lpad_out,
-                        float *out_hi, float *out_lo, const float *w_last, const float *b_last, float *out_last)
+                        float *out_hi, float *out_lo, const float *w_last, const float *b_last, float *out_last,
+                        const float *extra = nullptr)
 {
     using S = GemmShape<MODE, CIN, COUT>;
     auto kern = ae5_gemm_kernel<MODE, CIN, COUT>;
@@ -575,7 +585,7 @@ cudaError_t launch_gemm(Ctx &c, const CUtensorMap &a_hi, const CUtensorMap &a_lo
         configured = true;
     }
     kern<<<dim3(blocks(rows, kTileM), nodes), 128, S::kSmemBytes, c.stream>>>(a_hi, a_lo, b_hi, b_lo, bias, L_out, Lpad_out, out_hi,
-                                                                              out_lo, w_last, b_last, out_last, c.errword),
+                                                                              out_lo, w_last, b_last, out_last, extra, c.errword),
         ++g_kernel_launches;
     return cudaGetLastError();
 }
@@ -585,13 +595,19 @@ cudaError_t launch_gemm(Ctx &c, const CUtensorMap &a_hi, const CUtensorMap &a_lo
 const int kAe5EncCh[5] = {1, 64, 128, 256, 64};
 const int kAe5DecCh[6] = {4, 4, 32, 64, 128, 32};
 
-int64_t ae5_param_count()
+static int64_t ae5_decoder_params(bool innovation_channel)
+{
+    int64_t n = 0;
+    for (int i = 0; i < 5; ++i) n += (int64_t)kAe5DecCh[i] * kAe5DecCh[i + 1] * 3 + kAe5DecCh[i + 1];
+    return n + 32 + 1 + (innovation_channel ? 1 : 0);
+}
+
+int64_t ae5_param_count(int decoders, bool innovation_channel)
 {
     int64_t n = 0;
     for (int i = 0; i < 4; ++i) n += (int64_t)kAe5EncCh[i + 1] * kAe5EncCh[i] * 3 + kAe5EncCh[i + 1];
     n += 4 * 64 + 4;
-    for (int i = 0; i < 5; ++i) n += (int64_t)kAe5DecCh[i] * kAe5DecCh[i + 1] * 3 + kAe5DecCh[i + 1];
-    return n + 32 + 1;
+    return n + decoders * ae5_decoder_params(innovation_channel);
 }
 
 // Lengths after conv1..conv4; false when the input is too short.
@@ -605,9 +621,11 @@ bool ae5_lengths(int64_t mu, int64_t (&len)[5])
     return true;
 }
 
-void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used)
+void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
 {
     ae5_lengths(mu, a.len);
+    a.decoders = ps ? K : 1;
+    a.dec_stride = ae5_decoder_params(ps);
     size_t at = *used;
     auto take = [&](size_t floats) {
         at = (at + 1023) / 1024 * 1024;                     // TMA sources: generously aligned
@@ -632,31 +650,33 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used)
         a.dact_hi[l] = take(n);
         a.dact_lo[l] = take(n);
     }
-    for (int l = 0; l < 3; ++l) {                           // GEMM weights of deconv3..deconv5
-        const size_t n = (size_t)4 * kAe5DecCh[l + 2] * kAe5DecCh[l + 3];
+    for (int l = 0; l < 3; ++l) {                           // GEMM weights of deconv3..deconv5, every decoder's
+        const size_t n = (size_t)a.decoders * 4 * kAe5DecCh[l + 2] * kAe5DecCh[l + 3];
         a.dw_hi[l] = take(n);
         a.dw_lo[l] = take(n);
     }
-    // training: the two outputs inference never stores, the gradients at every layer's pre-activation,
-    // the products of the backward GEMMs and the per-chunk partial sums of the parameter gradients
-    a.act4_hi = take((size_t)K * a.len[4] * 64);
-    a.act4_lo = take((size_t)K * a.len[4] * 64);
-    a.dact5_hi = take((size_t)mu * 32);
-    a.dact5_lo = take((size_t)mu * 32);
-    size_t pmax = 0;
-    for (int l = 0; l < 4; ++l) {
-        a.g_enc[l] = take((size_t)K * a.len[l + 1] * kAe5EncCh[l + 1]);
-        if (l > 0) pmax = std::max(pmax, (size_t)K * a.len[l + 1] * 3 * kAe5EncCh[l]);
+    if (!ps) {      // training is built for the ring-allreduce form
+        // training: the two outputs inference never stores, the gradients at every layer's pre-activation,
+        // the products of the backward GEMMs and the per-chunk partial sums of the parameter gradients
+        a.act4_hi = take((size_t)K * a.len[4] * 64);
+        a.act4_lo = take((size_t)K * a.len[4] * 64);
+        a.dact5_hi = take((size_t)mu * 32);
+        a.dact5_lo = take((size_t)mu * 32);
+        size_t pmax = 0;
+        for (int l = 0; l < 4; ++l) {
+            a.g_enc[l] = take((size_t)K * a.len[l + 1] * kAe5EncCh[l + 1]);
+            if (l > 0) pmax = std::max(pmax, (size_t)K * a.len[l + 1] * 3 * kAe5EncCh[l]);
+        }
+        a.g_dec[0] = take((size_t)a.len[4] * 4);
+        for (int l = 1; l < 5; ++l) a.g_dec[l] = take((size_t)a.len[4 - l] * kAe5DecCh[l + 1]);
+        a.dzk = take((size_t)K * a.len[4] * 4);
+        a.dzbar = take((size_t)a.len[4] * 4);
+        a.dr = take((size_t)mu);
+        a.pbuf = take(pmax);
+        a.wt = take((size_t)256 * 384);
+        a.loss_blocks = (int)((mu + 255) / 256);
+        a.loss_part = reinterpret_cast<double *>(take((size_t)a.loss_blocks * 2));
     }
-    a.g_dec[0] = take((size_t)a.len[4] * 4);
-    for (int l = 1; l < 5; ++l) a.g_dec[l] = take((size_t)a.len[4 - l] * kAe5DecCh[l + 1]);
-    a.dzk = take((size_t)K * a.len[4] * 4);
-    a.dzbar = take((size_t)a.len[4] * 4);
-    a.dr = take((size_t)mu);
-    a.pbuf = take(pmax);
-    a.wt = take((size_t)256 * 384);
-    a.loss_blocks = (int)((mu + 255) / 256);
-    a.loss_part = reinterpret_cast<double *>(take((size_t)a.loss_blocks * 2));
     *used = at;
     // offsets of the layers' parameters inside the flat vector (encoder, then decoder)
     int64_t pos = 0;
@@ -698,6 +718,7 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used)
     }
     tensor(20, a.off_dw[5], 32, mu, 0, 0, 0);
     tensor(21, a.off_db[5], 1, mu, 0, 0, 0);
+    if (ps) return;
     if (base) a.partial = reinterpret_cast<float *>(base + (*used + 1023) / 1024 * 1024);
     *used = (*used + 1023) / 1024 * 1024 + (size_t)part * sizeof(float);
 }
@@ -715,12 +736,19 @@ cudaError_t ae5_make_maps(Ctx &c)
         ok = ok && make_act_map(enc, &a.map_act_lo[l], a.act_lo[l], cin, a.lpad[l], c.K);
         ok = ok && make_matrix_map(enc, &a.map_w_hi[l], a.w_hi[l], 3 * cin, cout);
         ok = ok && make_matrix_map(enc, &a.map_w_lo[l], a.w_lo[l], 3 * cin, cout);
-        const int dcin = kAe5DecCh[l + 2], dcout = kAe5DecCh[l + 3];
+        const int dcin = kAe5DecCh[l + 2];
         ok = ok && make_dact_map(enc, &a.map_dact_hi[l], a.dact_hi[l], dcin, a.len[3 - l]);
         ok = ok && make_dact_map(enc, &a.map_dact_lo[l], a.dact_lo[l], dcin, a.len[3 - l]);
-        ok = ok && make_matrix_map(enc, &a.map_dw_hi[l], a.dw_hi[l], 2 * dcin, 2 * dcout);
-        ok = ok && make_matrix_map(enc, &a.map_dw_lo[l], a.dw_lo[l], 2 * dcin, 2 * dcout);
     }
+    a.map_dw_hi.resize((size_t)a.decoders * 3);
+    a.map_dw_lo.resize((size_t)a.decoders * 3);
+    for (int d = 0; d < a.decoders; ++d)
+        for (int l = 0; l < 3; ++l) {
+            const int dcin = kAe5DecCh[l + 2], dcout = kAe5DecCh[l + 3];
+            const size_t at = (size_t)d * 4 * dcin * dcout;
+            ok = ok && make_matrix_map(enc, &a.map_dw_hi[d * 3 + l], a.dw_hi[l] + at, 2 * dcin, 2 * dcout);
+            ok = ok && make_matrix_map(enc, &a.map_dw_lo[d * 3 + l], a.dw_lo[l] + at, 2 * dcin, 2 * dcout);
+        }
     return ok ? cudaSuccess : cudaErrorInvalidValue;
 }
 
@@ -736,9 +764,12 @@ static void prepare_weights(Ctx &c)
                                                                                            a.w_lo[l]),
             ++g_kernel_launches;
         const int dcin = kAe5DecCh[l + 2], dcout = kAe5DecCh[l + 3];
-        ae5_prep_deconv_weights_kernel<<<blocks((int64_t)4 * dcin * dcout, 256), 256, 0, c.stream>>>(P + a.off_dw[l + 2], dcin, dcout,
-                                                                                                    a.dw_hi[l], a.dw_lo[l]),
-            ++g_kernel_launches;
+        for (int d = 0; d < a.decoders; ++d) {
+            const size_t at = (size_t)d * 4 * dcin * dcout;
+            ae5_prep_deconv_weights_kernel<<<blocks((int64_t)4 * dcin * dcout, 256), 256, 0, c.stream>>>(
+                P + a.off_dw[l + 2] + d * a.dec_stride, dcin, dcout, a.dw_hi[l] + at, a.dw_lo[l] + at),
+                ++g_kernel_launches;
+        }
     }
     a.weights_ready = true;
 }
@@ -750,7 +781,7 @@ cudaError_t launch_ae5_encode(Ctx &c)
     Ae5 &a = *c.ae5;
     const float *P = c.params;
     prepare_weights(c);
-    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.mu, a.len[1], a.lpad[0],
+    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu, c.mu, a.len[1], a.lpad[0],
                                                                             P + a.off_w[0], P + a.off_b[0], c.val, a.act_hi[0],
                                                                             a.act_lo[0]),
         ++g_kernel_launches;
@@ -799,7 +830,7 @@ cudaError_t launch_ae5_train_forward(Ctx &c)
     Ae5 &a = *c.ae5;
     const float *P = c.params;
     prepare_weights(c);
-    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.mu, a.len[1], a.lpad[0],
+    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu, c.mu, a.len[1], a.lpad[0],
                                                                             P + a.off_w[0], P + a.off_b[0], c.val, a.act_hi[0],
                                                                             a.act_lo[0]),
         ++g_kernel_launches;
@@ -840,31 +871,40 @@ cudaError_t launch_ae5_train_forward(Ctx &c)
     return e;
 }
 
-// Stage 5 up to the reconstruction: the decoder on the mean code; c.recon gets the mu values.
+// Stage 5 up to the reconstruction.  Ring-allreduce: the decoder on the mean code; c.recon gets the mu
+// values.  Parameter server (Section IV-A): node k's decoder on the common code, its innovation as the 33rd
+// input of the last convolution; c.recon gets [K][mu].  The decoders run one after the other through the
+// same activation buffers (each pass fills the device at the benchmark sizes).
 cudaError_t launch_ae5_decode(Ctx &c)
 {
     Ae5 &a = *c.ae5;
-    const float *P = c.params;
     prepare_weights(c);
-    ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0),
-        ++g_kernel_launches;
-    // deconv2 (4 -> 32): too narrow for the tensor cores
-    constexpr int kTp = 64, kSmem2 = (3 * 4 * 32 + (kTp + 1) * 4) * 4;
-    ae5_deconv_kernel<4, 32, kTp><<<blocks(a.len[4] + 1, kTp), 256, kSmem2, c.stream>>>(a.d0, a.len[4], a.len[3], P + a.off_dw[1],
-                                                                                        P + a.off_db[1], a.dact_hi[0], a.dact_lo[0]),
-        ++g_kernel_launches;
-    cudaError_t e = cudaGetLastError();
-    // deconv3..5: rows j = 0 .. L_in (one more than the input positions: the last makes the tail)
-    if (e == cudaSuccess)
-        e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], a.map_dw_hi[0], a.map_dw_lo[0], P + a.off_db[2],
-                                         a.len[3] + 1, 1, a.len[2], 0, a.dact_hi[1], a.dact_lo[1], nullptr, nullptr, nullptr);
-    if (e == cudaSuccess)
-        e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], a.map_dw_hi[1], a.map_dw_lo[1], P + a.off_db[3],
-                                          a.len[2] + 1, 1, a.len[1], 0, a.dact_hi[2], a.dact_lo[2], nullptr, nullptr, nullptr);
-    if (e == cudaSuccess)
-        e = launch_gemm<kDeconvFinal, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], a.map_dw_hi[2], a.map_dw_lo[2],
-                                               P + a.off_db[4], a.len[1] + 1, 1, a.len[0], 0, nullptr, nullptr, P + a.off_dw[5],
-                                               P + a.off_db[5], c.recon);
+    const bool ps = c.cfg.variant == LGC_VARIANT_PS;
+    cudaError_t e = cudaSuccess;
+    for (int d = 0; d < a.decoders && e == cudaSuccess; ++d) {
+        const float *P = c.params + d * a.dec_stride;          // decoder d's tensors sit at the offsets of decoder 0 from here
+        ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0),
+            ++g_kernel_launches;
+        // deconv2 (4 -> 32): too narrow for the tensor cores
+        constexpr int kTp = 64, kSmem2 = (3 * 4 * 32 + (kTp + 1) * 4) * 4;
+        ae5_deconv_kernel<4, 32, kTp><<<blocks(a.len[4] + 1, kTp), 256, kSmem2, c.stream>>>(a.d0, a.len[4], a.len[3], P + a.off_dw[1],
+                                                                                            P + a.off_db[1], a.dact_hi[0], a.dact_lo[0]),
+            ++g_kernel_launches;
+        e = cudaGetLastError();
+        const CUtensorMap *whi = &a.map_dw_hi[d * 3], *wlo = &a.map_dw_lo[d * 3];
+        // deconv3..5: rows j = 0 .. L_in (one more than the input positions: the last makes the tail)
+        if (e == cudaSuccess)
+            e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], whi[0], wlo[0], P + a.off_db[2],
+                                             a.len[3] + 1, 1, a.len[2], 0, a.dact_hi[1], a.dact_lo[1], nullptr, nullptr, nullptr);
+        if (e == cudaSuccess)
+            e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], whi[1], wlo[1], P + a.off_db[3],
+                                              a.len[2] + 1, 1, a.len[1], 0, a.dact_hi[2], a.dact_lo[2], nullptr, nullptr, nullptr);
+        if (e == cudaSuccess)
+            e = launch_gemm<kDeconvFinal, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], whi[2], wlo[2], P + a.off_db[4],
+                                                   a.len[1] + 1, 1, a.len[0], 0, nullptr, nullptr, P + a.off_dw[5],
+                                                   P + a.off_db[5] + (ps ? 1 : 0), c.recon + (int64_t)d * c.mu,
+                                                   ps ? c.inn + (int64_t)d * c.mu : nullptr);
+    }
     return e;
 }
 

@@ -105,10 +105,9 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
         p.P = p.Penc + p.Pdec * p.S;
         p.code_len = c2 * p.L2;
     } else if (cfg->ae_kind == LGC_AE_CONV5) {
-        if (cfg->variant != LGC_VARIANT_RAR) return fail(LGC_ERR_UNSUPPORTED, "the full-size autoencoder is built for ring-allreduce only");
         int64_t len[5];
         if (!ae5_lengths(p.mu, len) || len[4] < 1) return fail(LGC_ERR_UNSUPPORTED, "mu is too short for four stride-2 convolutions (needs mu >= 31)");
-        p.P = ae5_param_count();
+        p.P = ae5_param_count(p.S, cfg->variant == LGC_VARIANT_PS);
         p.Penc = p.Pdec = 0;
         p.code_len = 4 * len[4];
     } else {
@@ -279,7 +278,7 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
     }
     if (conv5) {
         if (!c.ae5) c.ae5.reset(new Ae5());
-        ae5_carve(*c.ae5, p.K, p.mu, cv.base, &cv.used);
+        ae5_carve(*c.ae5, p.K, p.mu, ps, cv.base, &cv.used);
     }
     cv.take<char>(0);
 }

@@ -558,6 +558,10 @@ cudaError_t launch_decode_scatter(Ctx &c, float *update)
         return e != cudaSuccess ? e : launch_dense_scatter(c, 1, update, c.recon);
     }
     if (!ps) return launch_dense_scatter(c, c.cfg.ae_kind == LGC_AE_IDENTITY ? 1 : 0, update);
+    if (c.cfg.ae_kind == LGC_AE_CONV5) {                 // K full-size decoders, each with its node's innovation
+        const cudaError_t e = launch_ae5_decode(c);
+        return e != cudaSuccess ? e : launch_scatter(c, c.recon, update);
+    }
     if (c.cfg.ae_kind == LGC_AE_IDENTITY) {
         identity_ps_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.combined, c.inn, c.mu, c.recon), ++g_kernel_launches;
     } else {

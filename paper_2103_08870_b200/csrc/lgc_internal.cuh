@@ -96,7 +96,13 @@ struct Ae5 {
     int64_t off_w[5] = {}, off_b[5] = {};     // offsets of the encoder layers' weights / biases in the parameter vector
     int64_t off_dw[6] = {}, off_db[6] = {};   // the same for the decoder's six layers
     CUtensorMap map_act_hi[3], map_act_lo[3], map_w_hi[3], map_w_lo[3];
-    CUtensorMap map_dact_hi[3], map_dact_lo[3], map_dw_hi[3], map_dw_lo[3];
+    CUtensorMap map_dact_hi[3], map_dact_lo[3];
+    // Decoders: one (ring-allreduce) or one per node (parameter server: Section IV-A), `dec_stride` parameters
+    // apart; off_dw / off_db below are decoder 0's.  The parameter server's last convolution has a 33rd input,
+    // the node's innovation.  dw_hi / dw_lo hold the decoders' GEMM weights back to back.
+    int decoders = 1;
+    int64_t dec_stride = 0;
+    std::vector<CUtensorMap> map_dw_hi, map_dw_lo;   // [decoders][3]
     bool weights_ready = false;         // w_hi / w_lo match the parameter vector
     // ---- training step (lgc_ae_train_step) ----
     float *act4_hi = nullptr, *act4_lo = nullptr;    // [K][L4][64] output of conv4 (inference folds it into conv5)
@@ -224,9 +230,9 @@ cudaError_t launch_train_step_ps(Ctx &c, int common, float lam_rec, float lam_si
 // full-size autoencoder (lgc_ae5.cu)
 extern const int kAe5EncCh[5];        // channels through conv1..conv4 (conv5 maps the last to 4)
 extern const int kAe5DecCh[6];        // channels through deconv1..deconv5 (the last convolution maps them to 1)
-int64_t ae5_param_count();
+int64_t ae5_param_count(int decoders, bool innovation_channel);
 bool ae5_lengths(int64_t mu, int64_t (&len)[5]);
-void ae5_carve(Ae5 &a, int K, int64_t mu, char *base, size_t *used);   // base may be null (sizes only)
+void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used);   // base may be null (sizes only)
 cudaError_t ae5_make_maps(Ctx &c);
 cudaError_t launch_ae5_encode(Ctx &c);
 cudaError_t launch_ae5_decode(Ctx &c);

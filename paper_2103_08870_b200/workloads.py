@@ -333,31 +333,36 @@ def ae_init_params(c1: int, c2: int, variant: str, num_nodes: int, seed: int = D
     return torch.cat(parts)
 
 
-def ae5_param_shapes() -> List[Tuple[str, Tuple[int, ...], int]]:
+def ae5_param_shapes(variant: str = "rar", num_nodes: int = 1) -> List[Tuple[str, Tuple[int, ...], int]]:
     """(name, shape, fan_in) of the full-size autoencoder's tensors (Section IV-C: encoder filters
     64/128/256/64 of 3 taps and 4 of 1 tap; decoder filters 4/32/64/128/32 of 3 taps and one 1-tap
     filter), in the order of the flat parameter vector.  Convolutions: w[co][ci][tap]; transposed
-    convolutions: w[ci][co][tap]."""
+    convolutions: w[ci][co][tap].  Parameter server: one decoder per node, whose last filter has a
+    33rd tap on the node's innovation (Section IV-A)."""
     enc_ch, dec_ch = [1, 64, 128, 256, 64], [4, 4, 32, 64, 128, 32]
     out = []
     for i in range(4):
         fan = 3 * enc_ch[i]
         out += [(f"enc.w{i + 1}", (enc_ch[i + 1], enc_ch[i], 3), fan), (f"enc.b{i + 1}", (enc_ch[i + 1],), fan)]
     out += [("enc.w5", (4, 64, 1), 64), ("enc.b5", (4,), 64)]
-    for i in range(5):
-        fan = 3 * dec_ch[i]
-        out += [(f"dec.w{i + 1}", (dec_ch[i], dec_ch[i + 1], 3), fan), (f"dec.b{i + 1}", (dec_ch[i + 1],), fan)]
-    out += [("dec.w6", (1, 32, 1), 32), ("dec.b6", (1,), 32)]
+    ps = variant == "ps"
+    for k in range(num_nodes if ps else 1):
+        pre = f"dec{k}" if ps else "dec"
+        for i in range(5):
+            fan = 3 * dec_ch[i]
+            out += [(f"{pre}.w{i + 1}", (dec_ch[i], dec_ch[i + 1], 3), fan), (f"{pre}.b{i + 1}", (dec_ch[i + 1],), fan)]
+        taps = 33 if ps else 32
+        out += [(f"{pre}.w6", (1, taps, 1), taps), (f"{pre}.b6", (1,), taps)]
     return out
 
 
-def ae5_init_params(seed: int = DEFAULT_SEED) -> torch.Tensor:
+def ae5_init_params(seed: int = DEFAULT_SEED, variant: str = "rar", num_nodes: int = 1) -> torch.Tensor:
     """U(-1/sqrt(fan_in), +1/sqrt(fan_in)) for every tensor of the full-size autoencoder; flat
     fp32 CPU tensor."""
     key = stream_key(seed, 1, STREAM_AE)
     parts = []
     ctr = 0
-    for _, shape, fan in ae5_param_shapes():
+    for _, shape, fan in ae5_param_shapes(variant, num_nodes):
         n = math.prod(shape)
         c = torch.arange(ctr, ctr + n, dtype=torch.int64)
         u = _uniform23(_lsr(hash_counters(key, c), 41))
@@ -388,7 +393,7 @@ class Workload:
     def init_params(self) -> torch.Tensor:
         """The autoencoder's seeded initial parameters, flat fp32 on the CPU."""
         if self.ae_kind == "conv5":
-            return ae5_init_params(self.seed)
+            return ae5_init_params(self.seed, self.variant, self.num_nodes)
         return ae_init_params(self.ae_c1, self.ae_c2, self.variant, self.num_nodes, self.seed)
 
 
@@ -405,7 +410,9 @@ def workload(name: str) -> Workload:
         return Workload("stress", flat_table(1 << 30), 4, 100, "rar", 16, 8, 5)
     if name == "resnet50_ae5":      # the ResNet-50-shaped case with the paper's full-size autoencoder
         return Workload("resnet50_ae5", resnet50_table(), 8, 1000, "rar", 64, 4, 10, ae_kind="conv5")
+    if name == "resnet101_ps_ae5":  # the ResNet-101-shaped parameter-server case with the full-size autoencoder
+        return Workload("resnet101_ps_ae5", resnet101_table(), 16, 1000, "ps", 64, 4, 10, ae_kind="conv5")
     raise KeyError(name)
 
 
-WORKLOAD_NAMES = ("tiny", "resnet50", "resnet101_ps", "segnet", "stress", "resnet50_ae5")
+WORKLOAD_NAMES = ("tiny", "resnet50", "resnet101_ps", "segnet", "stress", "resnet50_ae5", "resnet101_ps_ae5")

@@ -39,7 +39,7 @@ def make_pair(numel, K, variant="rar", ae_kind="conv2", c1=8, c2=4, density_ppm=
     if ae_kind == "conv2":
         params = W.ae_init_params(c1, c2, variant, K, seed)
     elif ae_kind == "conv5":
-        params = W.ae5_init_params(seed)
+        params = W.ae5_init_params(seed, variant, K)
     ora = OracleLGC(numel, K, density_ppm=density_ppm, momentum=momentum, variant=variant, ae_kind=ae_kind,
                     c1=c1, c2=c2, params=None if params is None else params.numpy(),
                     innovation_permille=innovation_permille, topk_method=topk_method, **adam)
@@ -83,7 +83,7 @@ def compare_step(ora, gpu, g_cpu: torch.Tensor, g_dev: torch.Tensor, choice: int
         zbar = ora.zbar.T if ora.ae_kind == "conv5" else ora.zbar
         assert_close(gpu.combined.cpu().numpy(), zbar, "mean code", rel=rel)
     else:
-        assert_close(gpu.combined.cpu().numpy(), ora.zc, "common code")
+        assert_close(gpu.combined.cpu().numpy(), ora.zc.T if ora.ae_kind == "conv5" else ora.zc, "common code", rel=rel)
         assert_bitwise(gpu.inn.cpu().numpy(), ora.inn, "innovation")
     upd_ref = ora.decode_scatter()
     gpu.decode_scatter(update_dev)

@@ -464,3 +464,31 @@ def test_full_size_autoencoder_training_phase():
     gpu.set_ae_params(torch.from_numpy(p32))
     g = src.step(4) * 300.0
     compare_step(ora, gpu, g, g.cuda(), 1, upd)
+
+
+@pytest.mark.parametrize("numel, K", [([300_000, 5000, 120_000], 2), ([2_000_000, 700_000, 300_001], 3)])
+def test_full_size_autoencoder_parameter_server(numel, K):
+    # Section IV-A with Section IV-C's layers: every node encodes, the common node's code goes through
+    # every node's own decoder, whose last convolution also sees the node's innovation (33rd channel);
+    # node-ordered average at each node's own indices.  Every stage compared, three steps.
+    ora, gpu = make_pair(numel, K, variant="ps", ae_kind="conv5")
+    assert gpu.P == 172_996 + K * 43_734
+    src = toy_source(numel, K, seed=43)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t in range(3):
+        g = src.step(t) * 300.0
+        compare_step(ora, gpu, g, g.cuda(), (2 * t + 1) % K, upd)
+    # training of this form is not built: the call says so and leaves the step usable
+    ora.accumulate(g.numpy())
+    gpu.accumulate(g.cuda())
+    ora.topk()
+    gpu.topk(0)
+    with pytest.raises(lgc.LGCError):
+        gpu.ae_train_step_ps(0)
+    assert_close(upd_of(gpu, upd), ora.topk_scatter(), "sparse update")
+    gpu.check()
+
+
+def upd_of(gpu, upd):
+    gpu.topk_scatter(upd)
+    return upd.cpu().numpy()

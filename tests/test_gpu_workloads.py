@@ -99,6 +99,12 @@ def test_resnet101_parameter_server_config():
     gpu.check()
 
 
+def test_resnet101_parameter_server_config_with_the_full_size_autoencoder():
+    # K = 16 decoders of Section IV-C's size, each with its node's innovation: mu = 44,657, code 4 x 2789
+    ora, gpu = run_workload("resnet101_ps_ae5", 2, state_every=1)
+    assert gpu.mu == 44_657 and gpu.P == 172_996 + 16 * 43_734
+
+
 def upd_after(gpu, upd):
     gpu.topk_scatter(upd)
     return upd.cpu().numpy()
