@@ -492,3 +492,34 @@ def test_full_size_autoencoder_parameter_server(numel, K):
 def upd_of(gpu, upd):
     gpu.topk_scatter(upd)
     return upd.cpu().numpy()
+
+
+@pytest.mark.parametrize("variant", ["rar", "ps"])
+@pytest.mark.parametrize("numel", [[31_000], [16_000, 17_000], [34_000, 64]])
+def test_full_size_autoencoder_at_its_shortest_inputs(variant, numel):
+    # mu = 31 (the code is one position of four channels), 33 and 35: every layer of the autoencoder is a
+    # single ragged tile, the transposed convolutions' output paddings take both values
+    K = 2
+    ora, gpu = make_pair(numel, K, variant=variant, ae_kind="conv5")
+    assert gpu.mu in (31, 33, 35)
+    src = toy_source(numel, K, seed=47)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t in range(2):
+        g = src.step(t) * 300.0
+        compare_step(ora, gpu, g, g.cuda(), t % K, upd)
+    if variant == "rar":                               # and one training step: loss and every tensor's gradient
+        from oracle import full_ae as A5
+        g = src.step(2) * 300.0
+        ora.accumulate(g.numpy())
+        gpu.accumulate(g.cuda(), 0)
+        ora.topk(0)
+        gpu.topk(0)
+        loss_dev = torch.zeros(1, device="cuda")
+        _, grads_ref = ora.ae_loss_and_grads()
+        loss_ref = ora.ae_train_step()
+        gpu.ae_train_step(loss_dev)
+        assert abs(loss_dev.item() - loss_ref) <= 1e-5 * loss_ref
+        m = adam_moments(gpu)[0].cpu().numpy().astype(np.float64)
+        for name, got in per_tensor(m / 0.1, A5.param_shapes()):
+            assert_close(got, grads_ref[name], f"gradient of {name}", rel=2e-5)
+    gpu.check()
