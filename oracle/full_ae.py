@@ -30,7 +30,9 @@ on the same graph, central differences of the loss, and the cases where loss and
 The parameter-server form (Section IV-A: one decoder per node, the node's innovation concatenated
 with the decoder's 32 feature channels in front of the last convolution) is pinned against the
 same construction with torch.cat and torch's convolutions and by the last filters that reduce it
-to the innovation alone and to the ring-allreduce decoder.
+to the innovation alone and to the ring-allreduce decoder; its training loss (reconstruction through
+the K decoders + similarity of the codes) against torch's autograd, central differences and the
+cases where the similarity term vanishes.
 """
 from __future__ import annotations
 
@@ -272,3 +274,74 @@ def rar_loss_and_grads(val: np.ndarray, p: Dict[str, np.ndarray]):
             dh = leaky_bwd(enc_pre[k][i - 1], dh)
             dh = conv_k3s2_bwd(enc_in[k][i - 1], p[f"enc.w{i}"], dh, g[f"enc.w{i}"], g[f"enc.b{i}"], want_dx=i > 1)
     return loss, g
+
+
+def ps_loss_and_grads(val: np.ndarray, inn: np.ndarray, p: Dict[str, np.ndarray], common: int,
+                      lam_rec: float = 1.0, lam_sim: float = 1.0):
+    """Parameter-server training loss of Section IV-A on the full-size autoencoder and its gradients:
+        loss = lam_rec (1/mu) sum_k || val_k - D_k(E(val_common), inn_k) ||^2
+             + lam_sim (1/(4 L4)) sum_k sum_{m != k} || E(val_k) - E(val_m) ||^2
+    (each term divided by the entries it sums per node, as for the two-layer autoencoders).
+    Returns (loss, rec term, sim term, gradients by tensor name of param_shapes_ps(K))."""
+    val = np.asarray(val, dtype=np.float64)
+    inn = np.asarray(inn, dtype=np.float64)
+    K, mu = val.shape
+    ln = lengths(mu)
+    g = {name: np.zeros(shape, dtype=np.float64) for name, shape in param_shapes_ps(K)}
+    enc_in, enc_pre, codes = [], [], []
+    for k in range(K):
+        h = val[k].reshape(1, -1)
+        ins, pres = [], []
+        for i in range(1, 5):
+            ins.append(h)
+            pre = conv_k3s2(h, p[f"enc.w{i}"], p[f"enc.b{i}"])
+            pres.append(pre)
+            h = leaky(pre)
+        ins.append(h)
+        codes.append(conv_k1(h, p["enc.w5"], p["enc.b5"]))
+        enc_in.append(ins)
+        enc_pre.append(pres)
+    nz = codes[0].size
+    sim = 0.0
+    for k in range(K):
+        for m in range(K):
+            if m != k:
+                sim += float(np.sum((codes[k] - codes[m]) ** 2))
+    sim /= nz
+    zc = codes[common]
+    dzs = [np.zeros_like(zc) for _ in range(K)]
+    rec = 0.0
+    for k in range(K):
+        pre_name = f"dec{k}"
+        dec_in, dec_pre = [zc], []
+        pre = convt_k3s1p1(zc, p[f"{pre_name}.w1"], p[f"{pre_name}.b1"])
+        dec_pre.append(pre)
+        d = leaky(pre)
+        for i in range(2, 6):
+            dec_in.append(d)
+            pre = convt_k3s2(d, p[f"{pre_name}.w{i}"], p[f"{pre_name}.b{i}"], (ln[5 - i] - 3) % 2)
+            dec_pre.append(pre)
+            d = leaky(pre)
+        cat = np.concatenate([d, inn[k].reshape(1, -1)], axis=0)          # 32 features + the innovation
+        r = conv_k1(cat, p[f"{pre_name}.w6"], p[f"{pre_name}.b6"]).reshape(-1)
+        diff = r - val[k]
+        rec += float(np.sum(diff * diff)) / mu
+        dy = (lam_rec * 2.0 * diff / mu).reshape(1, -1)
+        dcat = conv_k1_bwd(cat, p[f"{pre_name}.w6"], dy, g[f"{pre_name}.w6"], g[f"{pre_name}.b6"])
+        dd = dcat[:32]                                                     # the innovation is data: no gradient kept
+        for i in range(5, 1, -1):
+            dd = leaky_bwd(dec_pre[i - 1], dd)
+            dd = convt_k3s2_bwd(dec_in[i - 1], p[f"{pre_name}.w{i}"], dd, g[f"{pre_name}.w{i}"], g[f"{pre_name}.b{i}"])
+        dd = leaky_bwd(dec_pre[0], dd)
+        dzs[common] = dzs[common] + convt_k3s1p1_bwd(zc, p[f"{pre_name}.w1"], dd, g[f"{pre_name}.w1"], g[f"{pre_name}.b1"])
+    zsum = np.zeros_like(zc)
+    for k in range(K):
+        zsum = zsum + codes[k]
+    for k in range(K):
+        # d/dz_k of the sum over ordered pairs: every unordered pair appears twice
+        dz = dzs[k] + lam_sim * 4.0 * (K * codes[k] - zsum) / nz
+        dh = conv_k1_bwd(enc_in[k][4], p["enc.w5"], dz, g["enc.w5"], g["enc.b5"])
+        for i in range(4, 0, -1):
+            dh = leaky_bwd(enc_pre[k][i - 1], dh)
+            dh = conv_k3s2_bwd(enc_in[k][i - 1], p[f"enc.w{i}"], dh, g[f"enc.w{i}"], g[f"enc.b{i}"], want_dx=i > 1)
+    return lam_rec * rec + lam_sim * sim, rec, sim, g

@@ -240,8 +240,15 @@ class OracleLGC:
         L_rec sums ||g~_k - g~^rec_k||^2 over the nodes.  Reading: L_rec is divided by mu and L_sim
         by the number of code entries (c2 L2), so that lam_rec = lam_sim = 1 weighs an average
         entry of either kind alike.  Returns (loss, L_rec / mu, L_sim / (c2 L2), gradients)."""
-        assert self.variant == "ps" and self.ae_kind == "conv2"
+        assert self.variant == "ps" and self.ae_kind in ("conv2", "conv5")
         K, mu = self.K, self.mu
+        if self.ae_kind == "conv5":          # the full-size autoencoder: innovation as the 33rd channel
+            inn = np.zeros((K, mu), dtype=np.float64)
+            for k in range(K):
+                for l in range(self.L):
+                    a, b = int(self.koff[l]), int(self.koff[l + 1])
+                    inn[k, a:b] = O.innovation(self.val[k, a:b], self.ki_l[l])
+            return A5.ps_loss_and_grads(self.val, inn, self.p, common_node, lam_rec, lam_sim)
         xs = [self.val[k].astype(np.float64).reshape(1, -1) for k in range(K)]
         hs, zs = [], []
         for k in range(K):

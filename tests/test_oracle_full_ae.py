@@ -292,3 +292,75 @@ def test_ps_special_last_filters():
     for k in range(K):
         assert np.array_equal(ora.r[k], ref)
     assert np.array_equal(ora.zc, ora.z[1])
+
+
+def ps_flat_grads(g, K):
+    return np.concatenate([g[name].reshape(-1) for name, _ in A.param_shapes_ps(K)])
+
+
+def test_ps_training_gradients_against_torch_autograd():
+    rng = np.random.default_rng(31)
+    mu, K, common = 100, 3, 1
+    val = rng.standard_normal((K, mu)).astype(np.float32)
+    inn = np.where(rng.random((K, mu)) < 0.1, val, 0.0).astype(np.float32)
+    flat = rand_params_ps(K, 31)
+    loss, rec, sim, g = A.ps_loss_and_grads(val, inn, unpack_ps(flat, K), common, 0.7, 0.3)
+    tp = {k: torch.from_numpy(np.ascontiguousarray(v)).requires_grad_(True) for k, v in unpack_ps(flat, K).items()}
+    ln = A.lengths(mu)
+    zs = []
+    for k in range(K):
+        h = torch.from_numpy(val[k].astype(np.float64)).reshape(1, 1, -1)
+        for i in range(1, 5):
+            h = F.leaky_relu(F.conv1d(h, tp[f"enc.w{i}"], tp[f"enc.b{i}"], stride=2), 0.01)
+        zs.append(F.conv1d(h, tp["enc.w5"], tp["enc.b5"]))
+    tsim = sum(((zs[k] - zs[m]) ** 2).sum() for k in range(K) for m in range(K) if m != k) / zs[0].numel()
+    trec = 0.0
+    for k in range(K):
+        d = F.leaky_relu(F.conv_transpose1d(zs[common], tp[f"dec{k}.w1"], tp[f"dec{k}.b1"], stride=1, padding=1), 0.01)
+        for i in range(2, 6):
+            d = F.leaky_relu(F.conv_transpose1d(d, tp[f"dec{k}.w{i}"], tp[f"dec{k}.b{i}"], stride=2,
+                                                output_padding=(ln[5 - i] - 3) % 2), 0.01)
+        cat = torch.cat([d, torch.from_numpy(inn[k].astype(np.float64))[None, None]], dim=1)
+        r = F.conv1d(cat, tp[f"dec{k}.w6"], tp[f"dec{k}.b6"]).reshape(-1)
+        trec = trec + ((r - torch.from_numpy(val[k].astype(np.float64))) ** 2).sum() / mu
+    tl = 0.7 * trec + 0.3 * tsim
+    tl.backward()
+    assert abs(loss - tl.item()) <= 1e-12 * abs(tl.item()) and abs(rec - trec.item()) <= 1e-12 * rec
+    assert abs(sim - tsim.item()) <= 1e-12 * sim
+    for name, _ in A.param_shapes_ps(K):
+        ref = tp[name].grad.numpy()
+        assert np.abs(g[name] - ref).max() <= 1e-10 * max(1e-3, np.abs(ref).max()), name
+
+
+def test_ps_training_similarity_term_vanishes_for_one_node_and_for_identical_nodes():
+    rng = np.random.default_rng(33)
+    mu = 80
+    x = rng.standard_normal(mu).astype(np.float32)
+    inn = np.where(rng.random(mu) < 0.1, x, 0.0).astype(np.float32)
+    _, _, sim, _ = A.ps_loss_and_grads(x[None], inn[None], unpack_ps(rand_params_ps(1, 1), 1), 0)
+    assert sim == 0.0
+    _, _, sim, g = A.ps_loss_and_grads(np.stack([x] * 3), np.stack([inn] * 3), unpack_ps(rand_params_ps(3, 2), 3), 2, 0.0, 1.0)
+    assert sim == 0.0 and not any(v.any() for v in g.values())        # lam_rec = 0: nothing else contributes
+
+
+def test_ps_training_gradients_against_finite_differences():
+    rng = np.random.default_rng(35)
+    mu, K = 70, 2
+    val = rng.standard_normal((K, mu)).astype(np.float32)
+    inn = np.where(rng.random((K, mu)) < 0.1, val, 0.0).astype(np.float32)
+    flat = rand_params_ps(K, 35)
+    _, _, _, g = A.ps_loss_and_grads(val, inn, unpack_ps(flat, K), 0, 1.0, 0.5)
+    gf = ps_flat_grads(g, K)
+    pos, picks = 0, []
+    for _, shape in A.param_shapes_ps(K):
+        n = int(np.prod(shape))
+        picks += list(pos + rng.choice(n, size=min(2, n), replace=False))
+        pos += n
+    eps = 1e-6
+    for i in picks:
+        hi, lo = flat.copy(), flat.copy()
+        hi[i] += eps
+        lo[i] -= eps
+        fd = (A.ps_loss_and_grads(val, inn, unpack_ps(hi, K), 0, 1.0, 0.5)[0]
+              - A.ps_loss_and_grads(val, inn, unpack_ps(lo, K), 0, 1.0, 0.5)[0]) / (2 * eps)
+        assert abs(fd - gf[i]) <= 1e-5 * max(1e-3, abs(gf[i])) + 1e-8, (i, fd, gf[i])
