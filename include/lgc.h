@@ -61,7 +61,7 @@ typedef enum { LGC_VARIANT_RAR = 0, LGC_VARIANT_PS = 1 } lgc_variant;
  * joins the decoder's 32 feature channels in front of that convolution (43,734 floats per decoder).
  * deconv1 has stride 1 and padding 1, the others stride 2 with the output padding that returns each
  * length to the one the mirrored encoder layer saw.  Codes are stored position-major:
- * code[K][L4][4].  Training (lgc_ae_train_step) is built for the ring-allreduce variant. */
+ * code[K][L4][4].  Training: lgc_ae_train_step (ring-allreduce), lgc_ae_train_step_ps (parameter server). */
 typedef enum { LGC_AE_CONV2 = 0, LGC_AE_IDENTITY = 1, LGC_AE_CONV5 = 2 } lgc_ae_kind;
 
 /*
@@ -172,8 +172,10 @@ lgc_status lgc_ae_train_step(lgc_ctx *ctx, float *loss_out);
  *          + lambda_sim * (1/(c2 L2)) sum_k sum_{m != k} || E_c(g~_k) - E_c(g~_m) ||^2
  * (the paper's L_rec and L_sim, each divided by the number of entries it sums over per node),
  * analytic backward pass through the K decoders, their fusion scalars and the encoder, Adam.
- * Parameter-server variant with LGC_AE_CONV2 only; valid after lgc_topk.  Overwrites the codes,
- * the common code and the innovations of the context.  loss_out: device fp32 scalar or NULL. */
+ * Parameter-server variant, LGC_AE_CONV2 or LGC_AE_CONV5 (there the code has 4 L4 entries and the
+ * innovation is the 33rd input of each decoder's last convolution; the K decoders are run, differentiated
+ * and updated one after the other); valid after lgc_topk.  Overwrites the codes, the common code and
+ * the innovations of the context.  loss_out: device fp32 scalar or NULL. */
 lgc_status lgc_ae_train_step_ps(lgc_ctx *ctx, int32_t common_node, float lambda_rec, float lambda_sim,
                                 float *loss_out);
 

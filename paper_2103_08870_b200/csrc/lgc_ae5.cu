@@ -655,7 +655,7 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         a.dw_hi[l] = take(n);
         a.dw_lo[l] = take(n);
     }
-    if (!ps) {      // training is built for the ring-allreduce form
+    {
         // training: the two outputs inference never stores, the gradients at every layer's pre-activation,
         // the products of the backward GEMMs and the per-chunk partial sums of the parameter gradients
         a.act4_hi = take((size_t)K * a.len[4] * 64);
@@ -675,7 +675,8 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         a.pbuf = take(pmax);
         a.wt = take((size_t)256 * 384);
         a.loss_blocks = (int)((mu + 255) / 256);
-        a.loss_part = reinterpret_cast<double *>(take((size_t)a.loss_blocks * 2));
+        // partial sums of the loss: per decoder the reconstruction term's, then the similarity term's (parameter server)
+        a.loss_part = reinterpret_cast<double *>(take((size_t)(a.decoders + 1) * a.loss_blocks * 2));
     }
     *used = at;
     // offsets of the layers' parameters inside the flat vector (encoder, then decoder)
@@ -690,7 +691,7 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         a.off_dw[i] = pos; pos += (int64_t)kAe5DecCh[i] * kAe5DecCh[i + 1] * 3;
         a.off_db[i] = pos; pos += kAe5DecCh[i + 1];
     }
-    a.off_dw[5] = pos; pos += 32;
+    a.off_dw[5] = pos; pos += ps ? 33 : 32;      // parameter server: one more tap, on the innovation channel
     a.off_db[5] = pos;
     // parameter tensors in order, with the rows their gradient sums run over and the chunks these are cut into
     int64_t part = 0;
@@ -716,9 +717,8 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         tensor(10 + 2 * i, a.off_dw[i], (int64_t)kAe5DecCh[i] * kAe5DecCh[i + 1] * 3, a.len[5 - i], 2, kAe5DecCh[i], kAe5DecCh[i + 1]);
         tensor(11 + 2 * i, a.off_db[i], kAe5DecCh[i + 1], a.len[4 - i], 0, 0, 0);
     }
-    tensor(20, a.off_dw[5], 32, mu, 0, 0, 0);
+    tensor(20, a.off_dw[5], ps ? 33 : 32, mu, 0, 0, 0);
     tensor(21, a.off_db[5], 1, mu, 0, 0, 0);
-    if (ps) return;
     if (base) a.partial = reinterpret_cast<float *>(base + (*used + 1023) / 1024 * 1024);
     *used = (*used + 1023) / 1024 * 1024 + (size_t)part * sizeof(float);
 }
@@ -823,9 +823,10 @@ __global__ void ae5_conv5_kernel(const float *__restrict__ a_hi, const float *__
 }
 
 // Forward pass of a training step: the same kernels as inference, but conv4 and deconv5 store
-// their outputs (the backward pass needs them) and conv5 and the mean run as launches of their own.
-// Leaves the codes in c.code, their mean in c.combined and deconv5's output in dact5.
-cudaError_t launch_ae5_train_forward(Ctx &c)
+// their outputs (the backward pass needs them) and conv5, the combination of the codes and the last
+// convolution run as launches of their own.
+// Encoder: leaves every node's code in c.code (and the kept values in c.val).
+cudaError_t launch_ae5_train_encode(Ctx &c)
 {
     Ae5 &a = *c.ae5;
     const float *P = c.params;
@@ -849,26 +850,42 @@ cudaError_t launch_ae5_train_forward(Ctx &c)
     const int64_t rows = (int64_t)c.K * a.len[4];
     ae5_conv5_kernel<<<blocks(rows, 128), 128, 0, c.stream>>>(a.act4_hi, a.act4_lo, rows, P + a.off_w[4], P + a.off_b[4], c.code),
         ++g_kernel_launches;
-    c.mean_valid = false;
-    e = launch_combine_mean(c);
-    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
+// Decoder d on the code in c.combined, up to deconv5, whose output stays in dact5.
+cudaError_t launch_ae5_train_decode(Ctx &c, int d)
+{
+    Ae5 &a = *c.ae5;
+    const float *P = c.params + d * a.dec_stride;
     ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0),
         ++g_kernel_launches;
     constexpr int kTp = 64, kSmem2 = (3 * 4 * 32 + (kTp + 1) * 4) * 4;
     ae5_deconv_kernel<4, 32, kTp><<<blocks(a.len[4] + 1, kTp), 256, kSmem2, c.stream>>>(a.d0, a.len[4], a.len[3], P + a.off_dw[1],
                                                                                         P + a.off_db[1], a.dact_hi[0], a.dact_lo[0]),
         ++g_kernel_launches;
-    e = cudaGetLastError();
+    cudaError_t e = cudaGetLastError();
+    const CUtensorMap *whi = &a.map_dw_hi[d * 3], *wlo = &a.map_dw_lo[d * 3];
     if (e == cudaSuccess)
-        e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], a.map_dw_hi[0], a.map_dw_lo[0], P + a.off_db[2],
+        e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], whi[0], wlo[0], P + a.off_db[2],
                                          a.len[3] + 1, 1, a.len[2], 0, a.dact_hi[1], a.dact_lo[1], nullptr, nullptr, nullptr);
     if (e == cudaSuccess)
-        e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], a.map_dw_hi[1], a.map_dw_lo[1], P + a.off_db[3],
+        e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], whi[1], wlo[1], P + a.off_db[3],
                                           a.len[2] + 1, 1, a.len[1], 0, a.dact_hi[2], a.dact_lo[2], nullptr, nullptr, nullptr);
     if (e == cudaSuccess)
-        e = launch_gemm<kDeconv, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], a.map_dw_hi[2], a.map_dw_lo[2], P + a.off_db[4],
+        e = launch_gemm<kDeconv, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], whi[2], wlo[2], P + a.off_db[4],
                                           a.len[1] + 1, 1, a.len[0], 0, a.dact5_hi, a.dact5_lo, nullptr, nullptr, nullptr);
     return e;
+}
+
+// Ring-allreduce: encoder, mean of the codes, the one decoder.
+cudaError_t launch_ae5_train_forward(Ctx &c)
+{
+    cudaError_t e = launch_ae5_train_encode(c);
+    if (e != cudaSuccess) return e;
+    c.mean_valid = false;
+    e = launch_combine_mean(c);
+    return e != cudaSuccess ? e : launch_ae5_train_decode(c, 0);
 }
 
 // Stage 5 up to the reconstruction.  Ring-allreduce: the decoder on the mean code; c.recon gets the mu
@@ -902,7 +919,7 @@ cudaError_t launch_ae5_decode(Ctx &c)
         if (e == cudaSuccess)
             e = launch_gemm<kDeconvFinal, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], whi[2], wlo[2], P + a.off_db[4],
                                                    a.len[1] + 1, 1, a.len[0], 0, nullptr, nullptr, P + a.off_dw[5],
-                                                   P + a.off_db[5] + (ps ? 1 : 0), c.recon + (int64_t)d * c.mu,
+                                                   P + a.off_db[5], c.recon + (int64_t)d * c.mu,
                                                    ps ? c.inn + (int64_t)d * c.mu : nullptr);
     }
     return e;

@@ -292,17 +292,21 @@ __device__ __forceinline__ double block_sum256(double x, double *warp_part)
     return tot;                                                   // valid in thread 0
 }
 
-// The last convolution (1x1, 32 -> 1) on deconv5's stored output, the loss, and the way back through
-// it: recon[p], dr[p] = 2 (recon[p] - target[p]) / mu with target = (1/K) sum_k val_k (node order),
-// this CTA's part of sum (recon - target)^2, and g5[p][c] = dr[p] w6[c] leaky'(d5[p][c]).
+// The last convolution (1x1) on deconv5's stored output, the loss, and the way back through it:
+// recon[p] = b6 + sum_c w6[c] d5[p][c] (+ w6[32] extra[p]: the parameter server's innovation channel),
+// dr[p] = scale * 2 (recon[p] - target[p]) / mu with target = (1/Kt) sum_k rows_k[p] (node order; the
+// parameter server compares with the node's own vector: Kt = 1), this CTA's part of
+// sum (recon - target)^2, and g5[p][c] = dr[p] w6[c] leaky'(d5[p][c]).
 __global__ void __launch_bounds__(256)
-final_loss_kernel(const float *__restrict__ d5_hi, const float *__restrict__ d5_lo, const float *__restrict__ val, int K,
-                  int64_t mu, const float *__restrict__ w6, const float *__restrict__ b6, float *__restrict__ recon,
-                  float *__restrict__ dr, float *__restrict__ g5, double *__restrict__ loss_part)
+final_loss_kernel(const float *__restrict__ d5_hi, const float *__restrict__ d5_lo, const float *__restrict__ rows, int Kt,
+                  int64_t mu, const float *__restrict__ w6, const float *__restrict__ b6, const float *__restrict__ extra,
+                  float scale, float *__restrict__ recon, float *__restrict__ dr, float *__restrict__ g5,
+                  double *__restrict__ loss_part)
 {
-    __shared__ float w[32];
+    __shared__ float w[33];
     __shared__ double warp_part[8];
     if (threadIdx.x < 32) w[threadIdx.x] = w6[threadIdx.x];
+    if (threadIdx.x == 32) w[32] = extra ? w6[32] : 0.0f;
     __syncthreads();
     const int64_t p = (int64_t)blockIdx.x * 256 + threadIdx.x;
     double sq = 0.0;
@@ -318,12 +322,13 @@ final_loss_kernel(const float *__restrict__ d5_hi, const float *__restrict__ d5_
             r = __fmaf_rn(w[4 * q + 2], __fadd_rn(h.z, l.z), r);
             r = __fmaf_rn(w[4 * q + 3], __fadd_rn(h.w, l.w), r);
         }
+        if (extra) r = __fmaf_rn(w[32], extra[p], r);
         float target = 0.f;
-        for (int k = 0; k < K; ++k) target = __fadd_rn(target, val[(int64_t)k * mu + p]);
-        target = __fdiv_rn(target, (float)K);
+        for (int k = 0; k < Kt; ++k) target = __fadd_rn(target, rows[(int64_t)k * mu + p]);
+        target = __fdiv_rn(target, (float)Kt);
         const double diff = (double)r - (double)target;
         sq = diff * diff;
-        const float g = (float)(2.0 * diff / (double)mu);
+        const float g = (float)((double)scale * 2.0 * diff / (double)mu);
         recon[p] = r;
         dr[p] = g;
 #pragma unroll
@@ -392,8 +397,9 @@ dec1_grad_kernel(const float *__restrict__ zbar, const float *__restrict__ g1, i
     if (threadIdx.x == 0) (id < 48 ? gw[id] : gb[id - 48]) = (float)tot;
 }
 
-// Way back through the mean and conv5 (1x1, 64 -> 4): every node's code gets dzbar / K, and
-//   g4[k][t][c] = leaky'(a4[k][t][c]) * sum_o w5[o][c] dzk[k][t][o].   Thread per (node, position).
+// Way back through conv5 (1x1, 64 -> 4):  g4[k][t][c] = leaky'(a4[k][t][c]) * sum_o w5[o][c] dzk[k][t][o].
+// Ring-allreduce (dzbar given): every node's code gets dzbar / K (the mean), written to dzk.
+// Parameter server (dzbar == nullptr): dzk already holds every node's own gradient.  Thread per (node, position).
 __global__ void code_bwd_kernel(const float *__restrict__ dzbar, int K, int64_t L4, const float *__restrict__ w5,
                                 const float *__restrict__ a4_hi, float *__restrict__ dzk, float *__restrict__ g4)
 {
@@ -402,10 +408,16 @@ __global__ void code_bwd_kernel(const float *__restrict__ dzbar, int K, int64_t 
     __syncthreads();
     const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= (int64_t)K * L4) return;
-    const float4 z = reinterpret_cast<const float4 *>(dzbar)[r % L4];
-    const float fk = (float)K;
-    const float dz[4] = {__fdiv_rn(z.x, fk), __fdiv_rn(z.y, fk), __fdiv_rn(z.z, fk), __fdiv_rn(z.w, fk)};
-    reinterpret_cast<float4 *>(dzk)[r] = make_float4(dz[0], dz[1], dz[2], dz[3]);
+    float dz[4];
+    if (dzbar) {
+        const float4 z = reinterpret_cast<const float4 *>(dzbar)[r % L4];
+        const float fk = (float)K;
+        dz[0] = __fdiv_rn(z.x, fk); dz[1] = __fdiv_rn(z.y, fk); dz[2] = __fdiv_rn(z.z, fk); dz[3] = __fdiv_rn(z.w, fk);
+        reinterpret_cast<float4 *>(dzk)[r] = make_float4(dz[0], dz[1], dz[2], dz[3]);
+    } else {
+        const float4 z = reinterpret_cast<const float4 *>(dzk)[r];
+        dz[0] = z.x; dz[1] = z.y; dz[2] = z.z; dz[3] = z.w;
+    }
     for (int q = 0; q < 16; ++q) {
         const float4 a = reinterpret_cast<const float4 *>(a4_hi + r * 64)[q];
         const float as[4] = {a.x, a.y, a.z, a.w};
@@ -419,6 +431,53 @@ __global__ void code_bwd_kernel(const float *__restrict__ dzbar, int K, int64_t 
         }
         reinterpret_cast<float4 *>(g4 + r * 64)[q] = make_float4(o[0], o[1], o[2], o[3]);
     }
+}
+
+// Parameter server, similarity loss of Section IV-A over the codes z[K][n]: for every entry e this thread's
+// part of sum over ordered pairs k != m of (z_k[e] - z_m[e])^2 = 2 K sum_k z_k^2 - 2 (sum_k z_k)^2, and the
+// gradient it sends to every node's code, dzk[k][e] = lam_sim * 4 (K z_k[e] - sum_m z_m[e]) / n.
+__global__ void __launch_bounds__(256)
+ps_code_grad_kernel(const float *__restrict__ z, int K, int64_t n, float lam_sim, float *__restrict__ dzk,
+                    double *__restrict__ sim_part)
+{
+    __shared__ double warp_part[8];
+    const int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    double part = 0.0;
+    if (e < n) {
+        double sum = 0.0, sq = 0.0;
+        for (int k = 0; k < K; ++k) {
+            const double x = (double)z[(int64_t)k * n + e];
+            sum += x;
+            sq += x * x;
+        }
+        part = 2.0 * (double)K * sq - 2.0 * sum * sum;
+        for (int k = 0; k < K; ++k)
+            dzk[(int64_t)k * n + e] = (float)((double)lam_sim * 4.0 * ((double)K * (double)z[(int64_t)k * n + e] - sum) / (double)n);
+    }
+    const double tot = block_sum256(part, warp_part);
+    if (threadIdx.x == 0) sim_part[blockIdx.x] = tot;
+}
+
+__global__ void add_kernel(float *__restrict__ dst, const float *__restrict__ src, int64_t n)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) dst[i] = __fadd_rn(dst[i], src[i]);
+}
+
+// loss = lam_rec * (sum of the decoders' squared errors) / mu + lam_sim * (pair sum) / n
+__global__ void __launch_bounds__(256)
+ps_loss_sum_kernel(const double *__restrict__ rec_part, int n_rec, const double *__restrict__ sim_part, int n_sim, int64_t mu,
+                   int64_t n, float lam_rec, float lam_sim, float *__restrict__ out)
+{
+    __shared__ double warp_part[8];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n_rec; i += 256) acc += rec_part[i];
+    const double rec = block_sum256(acc, warp_part);
+    __syncthreads();
+    acc = 0.0;
+    for (int i = threadIdx.x; i < n_sim; i += 256) acc += sim_part[i];
+    const double sim = block_sum256(acc, warp_part);
+    if (threadIdx.x == 0) *out = (float)((double)lam_rec * rec / (double)mu + (double)lam_sim * sim / (double)n);
 }
 
 // Gradient of every parameter from its tensor's per-chunk partial sums (fp64, chunk order), then Adam.
@@ -503,28 +562,26 @@ struct Launcher {
 
 }  // namespace
 
-cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out)
-{
-    Ae5 &a = *c.ae5;
-    const float *P = c.params;
-    const int K = c.K;
-    const int64_t mu = c.mu;
-    const int64_t *len = a.len;                   // mu, L1, L2, L3, L4
-    cudaError_t e = launch_ae5_train_forward(c);
-    if (e != cudaSuccess) return e;
-    Launcher L{c, a};
-    cudaStream_t s = c.stream;
+namespace {
 
-    // ---- the last convolution and the loss ----
-    final_loss_kernel<<<a.loss_blocks, 256, 0, s>>>(a.dact5_hi, a.dact5_lo, c.val, K, mu, P + a.off_dw[5], P + a.off_db[5], c.recon,
-                                                    a.dr, a.g_dec[4], a.loss_part),
-        ++g_kernel_launches;
-    if (loss_out) loss_sum_kernel<<<1, 256, 0, s>>>(a.loss_part, a.loss_blocks, mu, loss_out), ++g_kernel_launches;
+// Backward pass of decoder d from g_dec[4] (gradient at deconv5's pre-activation) and dr (gradient at the
+// reconstruction) down to the code it read from c.combined: fills the partial sums of tensors 10..21 and
+// leaves the gradient at that code in dzbar.  `extra`: the innovation row of the parameter server's decoder.
+void decoder_backward(Launcher &L, int d, const float *extra)
+{
+    Ctx &c = L.c;
+    Ae5 &a = L.a;
+    const float *P = c.params + d * a.dec_stride;
+    const int64_t *len = a.len, mu = c.mu;
     const Rows dr_rows = rows_of(a.dr, nullptr, 0, 1, mu, 1);
     L.tn_narrow(20, rows_of(a.dact5_hi, a.dact5_lo, 0, 32, mu, 32), dr_rows, 1);     // dW6[c] = sum_p d5[p][c] dr[p]
+    if (extra && L.ok()) {                                                           // dW6[32] = sum_p innovation[p] dr[p]
+        const Ae5::Tensor &T = a.tensors[20];
+        tn_narrow_kernel<<<dim3(T.chunks, 1), 256, 0, c.stream>>>(rows_of(extra, nullptr, 0, 1, mu, 1), dr_rows, 1, T.rows, T.chunk,
+                                                                  L.partial_of(20) + 32, L.pstride_of(20));
+        ++g_kernel_launches;
+    }
     L.colsum(21, dr_rows);
-
-    // ---- deconv5 .. deconv2: input of deconv i+1 is the output of deconv i ----
     // inputs: deconv5 <- dact[2] [L1][128], deconv4 <- dact[1] [L2][64], deconv3 <- dact[0] [L3][32], deconv2 <- d0 [L4][4]
     for (int i = 4; i >= 1; --i) {
         const int cin = kAe5DecCh[i], cout = kAe5DecCh[i + 1];
@@ -538,19 +595,29 @@ cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out)
         L.arrange(P + a.off_dw[i], cin, cout, 1);
         L.nn(g_slices, lin, a.wt, cin, a.g_dec[i - 1], &x);
     }
-    // ---- deconv1, the mean, conv5 ----
     if (L.ok()) {
-        dec1_grad_kernel<<<52, 256, 0, s>>>(c.combined, a.g_dec[0], len[4], L.partial_of(10), L.partial_of(11)), ++g_kernel_launches;
-        dec1_bwd_kernel<<<blocks(len[4], 128), 128, 0, s>>>(a.g_dec[0], len[4], P + a.off_dw[0], a.dzbar), ++g_kernel_launches;
-        code_bwd_kernel<<<blocks((int64_t)K * len[4], 128), 128, 0, s>>>(a.dzbar, K, len[4], P + a.off_w[4], a.act4_hi, a.dzk,
-                                                                       a.g_enc[3]),
+        dec1_grad_kernel<<<52, 256, 0, c.stream>>>(c.combined, a.g_dec[0], len[4], L.partial_of(10), L.partial_of(11)), ++g_kernel_launches;
+        dec1_bwd_kernel<<<blocks(len[4], 128), 128, 0, c.stream>>>(a.g_dec[0], len[4], P + a.off_dw[0], a.dzbar), ++g_kernel_launches;
+    }
+}
+
+// Backward pass of the encoder from the gradients at the codes.  dzbar != nullptr: every node's code gets
+// dzbar / K (ring-allreduce); nullptr: dzk holds them already.  Fills the partial sums of tensors 0..9.
+void encoder_backward(Launcher &L, const float *dzbar)
+{
+    Ctx &c = L.c;
+    Ae5 &a = L.a;
+    const float *P = c.params;
+    const int K = c.K;
+    const int64_t *len = a.len, mu = c.mu;
+    if (L.ok()) {
+        code_bwd_kernel<<<blocks((int64_t)K * len[4], 128), 128, 0, c.stream>>>(dzbar, K, len[4], P + a.off_w[4], a.act4_hi, a.dzk,
+                                                                              a.g_enc[3]),
             ++g_kernel_launches;
     }
     const Rows dzk_rows = rows_of(a.dzk, nullptr, len[4] * 4, 4, len[4], 4);
     L.tn(8, dzk_rows, rows_of(a.act4_hi, a.act4_lo, len[4] * 64, 64, len[4], 64));
     L.colsum(9, dzk_rows);
-
-    // ---- conv4 .. conv1 ----
     for (int i = 3; i >= 0; --i) {
         const int cin = kAe5EncCh[i], cout = kAe5EncCh[i + 1];
         const int64_t lin = len[i], lout = len[i + 1];
@@ -565,25 +632,89 @@ cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out)
         L.arrange(P + a.off_w[i], cin, cout, 0);
         L.nn(g, (int64_t)K * lout, a.wt, 3 * cin, a.pbuf, nullptr);
         if (L.ok()) {
-            fold_kernel<<<blocks((int64_t)K * lin * (cin / 4), 256), 256, 0, s>>>(a.pbuf, K, lout, lin, cin, a.act_hi[i - 1], x_node,
-                                                                                 a.g_enc[i - 1]),
+            fold_kernel<<<blocks((int64_t)K * lin * (cin / 4), 256), 256, 0, c.stream>>>(a.pbuf, K, lout, lin, cin, a.act_hi[i - 1],
+                                                                                        x_node, a.g_enc[i - 1]),
                 ++g_kernel_launches;
         }
     }
-    if (!L.ok()) return L.err;
+}
 
-    // ---- Adam on every tensor ----
-    const AdamArgs ad = next_adam(c);
+// Adam on the tensors t0 .. t1 - 1, whose parameters sit `shift` floats behind their place in decoder 0's layout.
+void adam_on(Launcher &L, const AdamArgs &ad, int t0, int t1, int64_t shift)
+{
+    if (!L.ok()) return;
     TensorTable tt;
     tt.first[0] = 0;
     for (int t = 0; t < 22; ++t) {
-        const Ae5::Tensor &T = a.tensors[t];
-        tt.first[t + 1] = tt.first[t] + T.count;
-        tt.param_off[t] = T.param_off; tt.partial_off[t] = T.partial_off; tt.pstride[t] = L.pstride_of(t);
+        const Ae5::Tensor &T = L.a.tensors[t];
+        tt.first[t + 1] = tt.first[t] + (t >= t0 && t < t1 ? T.count : 0);
+        tt.param_off[t] = T.param_off + shift; tt.partial_off[t] = T.partial_off; tt.pstride[t] = L.pstride_of(t);
         tt.chunks[t] = T.chunks; tt.kind[t] = T.kind; tt.cin[t] = T.cin; tt.cout[t] = T.cout;
     }
-    reduce_adam_kernel<<<blocks(tt.first[22], 256), 256, 0, s>>>(a.partial, tt, ad), ++g_kernel_launches;
+    reduce_adam_kernel<<<blocks(tt.first[22], 256), 256, 0, L.c.stream>>>(L.a.partial, tt, ad), ++g_kernel_launches;
+}
+
+}  // namespace
+
+cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out)
+{
+    Ae5 &a = *c.ae5;
+    const float *P = c.params;
+    cudaError_t e = launch_ae5_train_forward(c);
+    if (e != cudaSuccess) return e;
+    Launcher L{c, a};
+    cudaStream_t s = c.stream;
+    // the last convolution and the loss against the mean of the nodes' vectors
+    final_loss_kernel<<<a.loss_blocks, 256, 0, s>>>(a.dact5_hi, a.dact5_lo, c.val, c.K, c.mu, P + a.off_dw[5], P + a.off_db[5], nullptr,
+                                                    1.0f, c.recon, a.dr, a.g_dec[4], a.loss_part),
+        ++g_kernel_launches;
+    if (loss_out) loss_sum_kernel<<<1, 256, 0, s>>>(a.loss_part, a.loss_blocks, c.mu, loss_out), ++g_kernel_launches;
+    decoder_backward(L, 0, nullptr);
+    encoder_backward(L, a.dzbar);
+    if (!L.ok()) return L.err;
+    adam_on(L, next_adam(c), 0, 22, 0);
     a.weights_ready = false;                       // the GEMM forms of the weights follow the new parameters
+    return cudaGetLastError();
+}
+
+// Parameter server (Section IV-A): every node's vector is encoded; the similarity term couples the codes;
+// the common node's code goes through every node's decoder (one after the other, each followed by its
+// backward pass and its Adam update, since they share the activation buffers); the gradients the decoders
+// send back add up, in node order, at the common node's code; then the encoder's backward pass.
+cudaError_t launch_ae5_train_step_ps(Ctx &c, int common, float lam_rec, float lam_sim, float *loss_out)
+{
+    Ae5 &a = *c.ae5;
+    cudaStream_t s = c.stream;
+    const int64_t n = 4 * a.len[4];                                   // entries of one code
+    cudaError_t e = launch_ae5_train_encode(c);
+    if (e == cudaSuccess) e = launch_combine_ps(c, common);           // the common code and every node's innovation
+    if (e != cudaSuccess) return e;
+    Launcher L{c, a};
+    const AdamArgs ad = next_adam(c);
+    double *sim_part = a.loss_part + (size_t)a.decoders * a.loss_blocks;
+    const int sim_blocks = (int)blocks(n, 256);
+    ps_code_grad_kernel<<<sim_blocks, 256, 0, s>>>(c.code, c.K, n, lam_sim, a.dzk, sim_part), ++g_kernel_launches;
+    for (int d = 0; d < a.decoders && L.ok(); ++d) {
+        const float *P = c.params + d * a.dec_stride;
+        L.err = launch_ae5_train_decode(c, d);
+        if (!L.ok()) break;
+        const float *inn = c.inn + (int64_t)d * c.mu;
+        final_loss_kernel<<<a.loss_blocks, 256, 0, s>>>(a.dact5_hi, a.dact5_lo, c.val + (int64_t)d * c.mu, 1, c.mu, P + a.off_dw[5],
+                                                        P + a.off_db[5], inn, lam_rec, c.recon + (int64_t)d * c.mu, a.dr, a.g_dec[4],
+                                                        a.loss_part + (size_t)d * a.loss_blocks),
+            ++g_kernel_launches;
+        decoder_backward(L, d, inn);
+        if (L.ok()) add_kernel<<<blocks(n, 256), 256, 0, s>>>(a.dzk + (int64_t)common * n, a.dzbar, n), ++g_kernel_launches;
+        adam_on(L, ad, 10, 22, d * a.dec_stride);
+    }
+    if (loss_out && L.ok())
+        ps_loss_sum_kernel<<<1, 256, 0, s>>>(a.loss_part, a.decoders * a.loss_blocks, sim_part, sim_blocks, c.mu, n, lam_rec, lam_sim,
+                                             loss_out),
+            ++g_kernel_launches;
+    encoder_backward(L, nullptr);
+    if (!L.ok()) return L.err;
+    adam_on(L, ad, 0, 10, 0);
+    a.weights_ready = false;
     return cudaGetLastError();
 }
 

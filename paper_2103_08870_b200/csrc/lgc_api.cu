@@ -577,13 +577,15 @@ lgc_status lgc_ae_train_step(lgc_ctx *c, float *loss_out)
 lgc_status lgc_ae_train_step_ps(lgc_ctx *c, int32_t common_node, float lambda_rec, float lambda_sim, float *loss_out)
 {
     if (!c) return LGC_ERR_INVALID_ARG;
-    if (c->cfg.variant != LGC_VARIANT_PS || c->cfg.ae_kind != LGC_AE_CONV2)
-        return fail(c, LGC_ERR_UNSUPPORTED, "lgc_ae_train_step_ps needs the parameter-server variant with the two-layer autoencoder");
+    if (c->cfg.variant != LGC_VARIANT_PS || c->cfg.ae_kind == LGC_AE_IDENTITY)
+        return fail(c, LGC_ERR_UNSUPPORTED, "lgc_ae_train_step_ps needs the parameter-server variant with a convolutional autoencoder");
     if (common_node < 0 || common_node >= c->K) return fail(c, LGC_ERR_INVALID_ARG, "common_node out of range");
     if (!(lambda_rec >= 0.0f) || !(lambda_sim >= 0.0f)) return fail(c, LGC_ERR_INVALID_ARG, "the loss weights must not be negative");
     if (c->stage != Ctx::kSelected) return fail(c, LGC_ERR_BAD_STATE, "lgc_ae_train_step_ps must follow lgc_topk");
     cudaError_t e = launch_gather(*c);
-    if (e == cudaSuccess) e = launch_train_step_ps(*c, common_node, lambda_rec, lambda_sim, loss_out);
+    if (e == cudaSuccess)
+        e = c->cfg.ae_kind == LGC_AE_CONV5 ? launch_ae5_train_step_ps(*c, common_node, lambda_rec, lambda_sim, loss_out)
+                                           : launch_train_step_ps(*c, common_node, lambda_rec, lambda_sim, loss_out);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_ae_train_step_ps");
     return LGC_OK;
 }

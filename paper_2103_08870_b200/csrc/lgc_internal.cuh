@@ -237,8 +237,11 @@ cudaError_t ae5_make_maps(Ctx &c);
 cudaError_t launch_ae5_encode(Ctx &c);
 cudaError_t launch_ae5_decode(Ctx &c);
 // training: the forward pass that keeps every layer's output (lgc_ae5.cu), then the backward pass and Adam
-cudaError_t launch_ae5_train_forward(Ctx &c);
+cudaError_t launch_ae5_train_encode(Ctx &c);           // every node's code into c.code
+cudaError_t launch_ae5_train_decode(Ctx &c, int d);    // decoder d on c.combined, up to deconv5 (kept in dact5)
+cudaError_t launch_ae5_train_forward(Ctx &c);          // ring-allreduce: encoder, mean, the decoder
 cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out);
+cudaError_t launch_ae5_train_step_ps(Ctx &c, int common, float lam_rec, float lam_sim, float *loss_out);
 struct AdamArgs {
     float *params, *m, *v;
     double lr, beta1, beta2, eps, corr1, corr2;

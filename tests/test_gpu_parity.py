@@ -478,13 +478,43 @@ def test_full_size_autoencoder_parameter_server(numel, K):
     for t in range(3):
         g = src.step(t) * 300.0
         compare_step(ora, gpu, g, g.cuda(), (2 * t + 1) % K, upd)
-    # training of this form is not built: the call says so and leaves the step usable
+    gpu.check()
+
+
+@pytest.mark.parametrize("numel, K", [([300_000, 5000, 120_000], 2), ([2_000_000, 700_000, 300_001], 3)])
+def test_full_size_autoencoder_parameter_server_training(numel, K):
+    # Section IV-A's loss on Section IV-C's layers: reconstruction through the K decoders (each with its
+    # node's innovation as 33rd channel) + similarity of the codes.  After the first step Adam's first
+    # moment is (1 - beta1) times the gradient: every tensor's gradient (encoder and all decoders) against
+    # the oracle's, the loss, the parameters after that step; then the losses of two more steps on the
+    # same kept values with other common nodes, and the sparse update of the second training phase.
+    from oracle import full_ae as A5
+    ora, gpu = make_pair(numel, K, variant="ps", ae_kind="conv5")
+    src = toy_source(numel, K, seed=53)
+    g = src.step(0) * 300.0
     ora.accumulate(g.numpy())
     gpu.accumulate(g.cuda())
     ora.topk()
     gpu.topk(0)
-    with pytest.raises(lgc.LGCError):
-        gpu.ae_train_step_ps(0)
+    loss_dev = torch.zeros(1, device="cuda")
+    _, _, _, grads_ref = ora.ae_loss_and_grads_ps(1, 0.7, 0.3)
+    losses_ref, losses = [ora.ae_train_step_ps(1, 0.7, 0.3)], []
+    gpu.ae_train_step_ps(1, 0.7, 0.3, loss_dev)
+    losses.append(loss_dev.item())
+    m = adam_moments(gpu)[0].cpu().numpy().astype(np.float64)
+    # The similarity term's gradient at a code, 4 lam_sim (K z_k - sum_m z_m) / n, is a difference of codes that
+    # agree in their leading digits (the nodes share most of their signal), so the codes' own error (1e-6 of
+    # their scale, fp32 against fp64) shows up several times larger in it and in what the encoder makes of it.
+    for name, got in per_tensor(m / 0.1, A5.param_shapes_ps(K)):
+        assert_close(got, grads_ref[name], f"gradient of {name}", rel=1e-4)
+    # Adam's first step is lr g / (|g| + eps): where |g| is near eps = 1e-8 a gradient error of 1e-10 moves it by 1e-5 lr / eps
+    assert_close(gpu.get_ae_params().numpy(), ora.get_params(), "parameters after the first step", rel=1e-4)
+    for common in (0, K - 1):
+        losses_ref.append(ora.ae_train_step_ps(common, 0.7, 0.3))
+        gpu.ae_train_step_ps(common, 0.7, 0.3, loss_dev)
+        losses.append(loss_dev.item())
+    assert_close(np.array(losses), np.array(losses_ref), "training losses")
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
     assert_close(upd_of(gpu, upd), ora.topk_scatter(), "sparse update")
     gpu.check()
 
