@@ -56,15 +56,16 @@ def test_three_phases_against_the_oracle(variant, K):
     gpu.check()
 
 
-def test_three_phases_with_the_full_size_autoencoder():
+@pytest.mark.parametrize("variant", ["rar", "ps"])
+def test_three_phases_with_the_full_size_autoencoder(variant):
     # the same schedule with Section IV-C's autoencoder on the middle layers (mu = 96 kept values there).
     # eps = 1e-2 keeps Adam's step well conditioned, so that the two sides' parameters stay together
     # through the training phase (see test_full_size_autoencoder_training_phase in test_gpu_parity.py).
     K = 2
-    params = W.ae5_init_params(5)
-    gpu = PhasedLGC(NUMEL, MODES, K, ae_kind="conv5", eps=1e-2)
+    params = W.ae5_init_params(5, variant, K)
+    gpu = PhasedLGC(NUMEL, MODES, K, variant=variant, ae_kind="conv5", eps=1e-2)
     gpu.ae_runs()[0].ctx.set_ae_params(params)
-    ora = OraclePhased(NUMEL, MODES, K, {1: params.numpy()}, ae_kind="conv5", eps=1e-2)
+    ora = OraclePhased(NUMEL, MODES, K, {1: params.numpy()}, variant=variant, ae_kind="conv5", eps=1e-2)
     src = W.GradientSource(W.LayerTable("ph", NUMEL, [1, 2, 3, 1, 2, 3, 1]), K, seed=29)
     upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
     loss = torch.zeros(1, device="cuda")
@@ -77,7 +78,10 @@ def test_three_phases_with_the_full_size_autoencoder():
         assert_close(upd.cpu().numpy(), ref, f"step {t} ({phase}): update")
         if losses:
             assert_close(np.array([loss.item()]), np.array(losses), f"step {t}: training loss")
-    assert_close(gpu.ae_runs()[0].ctx.get_ae_params().numpy(), ora.groups[1]["o"].get_params(), "trained parameters")
+    # parameter server: the similarity gradient is a difference of nearly equal codes, known to ~1e-4 of its
+    # scale in fp32 (test_full_size_autoencoder_parameter_server_training), and three Adam steps carry that on
+    assert_close(gpu.ae_runs()[0].ctx.get_ae_params().numpy(), ora.groups[1]["o"].get_params(), "trained parameters",
+                 rel=1e-5 if variant == "rar" else 2e-4)
     gpu.check()
 
 
