@@ -227,6 +227,8 @@ def run_ours(args, w: W.Workload):
     gpu.check()
     elapsed_ms = start.elapsed_time(stop)
     acc_ms = [a.elapsed_time(b) for a, b in ev]
+    # every step's own time: from its first event to the next step's (the last one: to the closing event)
+    step_ms = [ev[t][0].elapsed_time(ev[t + 1][0] if t + 1 < args.steps else stop) for t in range(args.steps)]
 
     # end to end through host buffers: pinned gradients in, dense update out, every step
     e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 20))
@@ -269,6 +271,7 @@ def run_ours(args, w: W.Workload):
                          "frac_of_measured_peak": step_gbs / peak, "frac_of_nominal_8TBps": step_gbs / NOMINAL_HBM_GBS},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": K * N * 4, "d2h_bytes_per_step": N * 4,
                     "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps if e2e_steps else None},
+            "step_ms": {"min": min(step_ms), "median": statistics.median(step_ms), "max": max(step_ms)},   # this rank's steps
             "gpu_launches": gpu_launches,
             "clocks": clocks,
         }
