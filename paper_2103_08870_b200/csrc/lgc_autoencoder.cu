@@ -238,6 +238,81 @@ decode_kernel(const float *__restrict__ z, int64_t mu, int64_t L1, int64_t L2,
     recon[(int64_t)s * mu + p] = y;
 }
 
+// The same reconstructions, organised by the first transposed convolution's output positions: a thread
+// computes the activations d[.][i] of ONE position i once (decode_kernel recomputes them for each of the
+// two or three outputs they feed) and from them the three sums e_tau = sum_ci w2[ci][tau] d[ci][i] that
+// position i adds to outputs 2i, 2i + 1 and 2i + 2.  Thread i then writes
+//     y[2i] = b2 + e_0(i) + e_2(i - 1),    y[2i + 1] = b2 + e_1(i)
+// with e_2(i - 1) handed over through shared memory (the CTA's first slot is the halo i0 - 1 and writes
+// nothing).  Slot i = L1 (no activations) finishes the tail: y[2 L1] = b2 + e_2(L1 - 1), y[2 L1 + 1] = b2.
+// Even and odd positions use different taps of the first layer, so the CTA's first half takes the even
+// slots and the second half the odd ones: warps do not diverge.  Weights sit in shared memory with the
+// hidden channel innermost (16-byte reads).  Grid (ceil((L1 + 1) / 255), decoders), 256 threads.
+template <int C1, int C2, bool PS>
+__global__ void __launch_bounds__(256)
+decode_rows_kernel(const float *__restrict__ z, int64_t mu, int64_t L1, int64_t L2, const float *__restrict__ dec_params,
+                   int dec_stride, const float *__restrict__ inn, float *__restrict__ recon)
+{
+    static_assert(C1 % 4 == 0, "hidden channels are read four at a time");
+    __shared__ __align__(16) float w1s[3][C2][C1];      // [tap][code channel][hidden channel]
+    __shared__ __align__(16) float b1s[C1];
+    __shared__ float w2s[3][C1], e2s[256], tail[4];     // tail: b2, then the fusion scalars w0, w1, b
+    const int s = blockIdx.y;
+    const float *P = dec_params + (int64_t)s * dec_stride;
+    for (int i = threadIdx.x; i < C2 * C1 * 3; i += 256) {
+        const int c2 = i / (C1 * 3), ci = i / 3 % C1, tq = i % 3;
+        w1s[tq][c2][ci] = P[i];
+    }
+    if (threadIdx.x < C1) b1s[threadIdx.x] = P[C2 * C1 * 3 + threadIdx.x];
+    for (int i = threadIdx.x; i < C1 * 3; i += 256) w2s[i % 3][i / 3] = P[C2 * C1 * 3 + C1 + i];
+    if (threadIdx.x < (PS ? 4 : 1)) tail[threadIdx.x] = P[C2 * C1 * 3 + C1 + C1 * 3 + threadIdx.x];
+    __syncthreads();
+    const int slot = threadIdx.x < 128 ? 2 * (int)threadIdx.x : 2 * ((int)threadIdx.x - 128) + 1;
+    const int64_t i = (int64_t)blockIdx.x * 255 - 1 + slot;
+    float e0 = 0.f, e1 = 0.f, e2 = 0.f;
+    if (i >= 0 && i < L1) {
+        float d[C1];
+#pragma unroll
+        for (int ci = 0; ci < C1; ++ci) d[ci] = b1s[ci];
+        for (int tq = (int)(i & 1); tq < 3; tq += 2) {           // the taps that reach position i: i = 2j + tq
+            const int64_t j = (i - tq) >> 1;
+            if (i < tq || j >= L2) continue;
+#pragma unroll
+            for (int c2 = 0; c2 < C2; ++c2) {
+                const float zz = z[(int64_t)c2 * L2 + j];
+#pragma unroll
+                for (int q = 0; q < C1 / 4; ++q) {
+                    const float4 w = *reinterpret_cast<const float4 *>(&w1s[tq][c2][4 * q]);
+                    d[4 * q] = __fmaf_rn(w.x, zz, d[4 * q]);
+                    d[4 * q + 1] = __fmaf_rn(w.y, zz, d[4 * q + 1]);
+                    d[4 * q + 2] = __fmaf_rn(w.z, zz, d[4 * q + 2]);
+                    d[4 * q + 3] = __fmaf_rn(w.w, zz, d[4 * q + 3]);
+                }
+            }
+        }
+#pragma unroll
+        for (int ci = 0; ci < C1; ++ci) {
+            const float r = fmaxf(d[ci], 0.0f);
+            e0 = __fmaf_rn(w2s[0][ci], r, e0);
+            e1 = __fmaf_rn(w2s[1][ci], r, e1);
+            e2 = __fmaf_rn(w2s[2][ci], r, e2);
+        }
+    }
+    e2s[slot] = e2;
+    __syncthreads();
+    if (slot == 0 || i > L1) return;
+    const float b2 = tail[0];
+    float y[2] = {__fadd_rn(b2, __fadd_rn(e0, e2s[slot - 1])), __fadd_rn(b2, e1)};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int64_t p = 2 * i + h;
+        if (p >= mu) break;
+        float out = y[h];
+        if (PS) out = __fmaf_rn(tail[2], inn[(int64_t)s * mu + p], __fmaf_rn(tail[1], out, tail[3]));
+        recon[(int64_t)s * mu + p] = out;
+    }
+}
+
 // identity autoencoder, parameter server: recon_k = code + innovation_k
 __global__ void identity_ps_kernel(const float *__restrict__ z, const float *__restrict__ inn, int64_t mu,
                                    float *__restrict__ recon)
@@ -565,12 +640,25 @@ cudaError_t launch_decode_scatter(Ctx &c, float *update)
     if (c.cfg.ae_kind == LGC_AE_IDENTITY) {
         identity_ps_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.combined, c.inn, c.mu, c.recon), ++g_kernel_launches;
     } else {
-        const dim3 grid(blocks_for(c.mu, kAeThreads), c.S);
         const float *dec = c.params + c.Penc;
+        if (c.cfg.ae_c1 % 4 == 0) {        // one thread per position of the hidden layer
+            const dim3 grid(blocks_for(c.L1 + 1, 255), c.S);
+            if (c.cfg.ae_c1 == 8 && c.cfg.ae_c2 == 4)
+                decode_rows_kernel<8, 4, true><<<grid, 256, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec, (int)c.Pdec, c.inn, c.recon);
+            else if (c.cfg.ae_c1 == 16 && c.cfg.ae_c2 == 8)
+                decode_rows_kernel<16, 8, true><<<grid, 256, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec, (int)c.Pdec, c.inn, c.recon);
+            else if (c.cfg.ae_c1 == 4 && c.cfg.ae_c2 == 2)
+                decode_rows_kernel<4, 2, true><<<grid, 256, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec, (int)c.Pdec, c.inn, c.recon);
+            else
+                return cudaErrorInvalidValue;
+            ++g_kernel_launches;
+        } else {
+            const dim3 grid(blocks_for(c.mu, kAeThreads), c.S);
 #define CALL(A, B) decode_kernel<A, B, true><<<grid, kAeThreads, 0, c.stream>>>(c.combined, c.mu, c.L1, c.L2, dec,     \
                                                                                (int)c.Pdec, c.inn, c.recon)
-        LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
+            LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
 #undef CALL
+        }
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
