@@ -429,6 +429,9 @@ lgc_status lgc_destroy(lgc_ctx *ctx)
         for (cudaEvent_t e : ctx->row_uploaded) cudaEventDestroy(e);
         if (ctx->tail_done) cudaEventDestroy(ctx->tail_done);
         if (ctx->upload_stream) cudaStreamDestroy(ctx->upload_stream);
+        if (ctx->side_fork) cudaEventDestroy(ctx->side_fork);
+        if (ctx->side_join) cudaEventDestroy(ctx->side_join);
+        if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
     }
     delete ctx;
     return LGC_OK;
@@ -494,8 +497,15 @@ lgc_status lgc_topk(lgc_ctx *c, int32_t leader, float *update_hint)
     if (!ps && (leader < 0 || leader >= c->K)) return fail(c, LGC_ERR_INVALID_ARG, "leader out of range");
     // candidates collected during the accumulation count only if they are this leader's
     const bool served = ps ? c->fused_leader == -1 : c->fused_leader == leader;
-    cudaError_t e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, served, c->epoch,
-                                  update_hint, c->N, c->errword, c->stream);
+    cudaError_t e = cudaSuccess;
+    if (ps && !c->side_stream && c->sel_v.num_small && c->sel_v.num_large) {     // many small layers: a stream for them
+        e = cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->side_fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->side_join, cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_fail(c, e, "lgc_topk (side stream)");
+    }
+    e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, served, c->epoch, update_hint, c->N,
+                      c->errword, c->stream, c->side_stream, c->side_fork, c->side_join);
     c->cleared_update = c->sel_v.num_large ? update_hint : nullptr;
     if (c->selections < 2) ++c->selections;
     c->val_valid = false;

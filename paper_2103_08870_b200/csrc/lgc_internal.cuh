@@ -185,6 +185,10 @@ struct Ctx {
     bool mean_valid = false;       // combined holds the mean code of the current selection
     // lgc_step_host: the upload runs row by row on a stream of the library's own, so that rows are
     // accumulated while later rows are still on the bus (created at the first call, released by lgc_destroy)
+    // lgc_topk, many small layers (parameter server): they are selected on a side stream while the large
+    // layers are finished on the context's stream (created at the first such call, released by lgc_destroy)
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t side_fork = nullptr, side_join = nullptr;
     cudaStream_t upload_stream = nullptr;
     std::vector<cudaEvent_t> row_uploaded;   // [K]
     cudaEvent_t tail_done = nullptr;         // the previous lgc_step_host has finished with dev_grads (before its download)
@@ -205,9 +209,12 @@ cudaError_t launch_dense_mean(const float *g, int64_t g_stride, int K, int64_t n
 // served: the accumulation of step `epoch` collected the candidates of exactly these rows.
 // clear/clear_floats: optional 16-byte aligned buffer that spare CTAs of the finishing launch set to zero
 // (only when the tables have large segments).
+// side / fork / join (all or none): a stream and two events of the caller's; when the small segments get a launch
+// of their own it runs on `side`, beside the finishing of the large ones, and `s` continues once both are done.
 cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0,
                           int rows, int32_t *out, int64_t out_stride, bool served, int32_t epoch, float *clear,
-                          int64_t clear_floats, int32_t *errword, cudaStream_t s);
+                          int64_t clear_floats, int32_t *errword, cudaStream_t s, cudaStream_t side = nullptr,
+                          cudaEvent_t fork = nullptr, cudaEvent_t join = nullptr);
 // Accumulation that also collects the selection candidates of the selecting rows (sel_row0 .. +sel_rows
 // of the K rows) against the predicted buckets; needs N % 4 == 0 and g_stride % 4 == 0 (rows of g are
 // g_stride elements apart).

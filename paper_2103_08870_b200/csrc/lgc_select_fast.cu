@@ -1008,7 +1008,7 @@ __global__ void __launch_bounds__(kSelThreads) select_small_only_kernel(FastArgs
 // floats that spare CTAs of the finishing launch set to zero; used only when there are large segments.
 cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_stride, int row0, int rows,
                           int32_t *out, int64_t out_stride, bool served, int32_t epoch, float *clear, int64_t clear_floats,
-                          int32_t *errword, cudaStream_t st)
+                          int32_t *errword, cudaStream_t st, cudaStream_t side, cudaEvent_t fork, cudaEvent_t join)
 {
     if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
     FastArgs f;
@@ -1026,8 +1026,23 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
     }
     // a few small segments ride along in the finishing launch; many get CTAs of their own size
     f.fin_small = (int64_t)rows * t.num_small <= 512 && t.num_large ? t.num_small : 0;
-    if (t.num_small && !f.fin_small)
-        select_small_only_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
+    bool forked = false;
+    if (t.num_small && !f.fin_small) {
+        // both launches are latency bound and write disjoint slots: side by side when the caller lent a stream
+        forked = side && fork && join && t.num_large;
+        cudaStream_t where = st;
+        if (forked) {
+            cudaError_t e = cudaEventRecord(fork, st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(side, fork, 0);
+            if (e != cudaSuccess) return e;
+            where = side;
+        }
+        select_small_only_kernel<<<dim3(t.num_small, rows), kSelThreads, 0, where>>>(f), ++g_kernel_launches;
+        if (forked) {
+            const cudaError_t e = cudaEventRecord(join, side);
+            if (e != cudaSuccess) return e;
+        }
+    }
     if (t.num_group_jobs) {
         const dim3 grid(t.num_group_jobs, rows);
         compact_groups_kernel<<<grid, kFinThreads, 0, st>>>(f), ++g_kernel_launches;
@@ -1045,6 +1060,10 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
     }
     if (t.num_large + f.fin_small)
         finish_kernel<<<dim3(t.num_large + f.fin_small + spare, rows), kFinThreads, kFinDyn, st>>>(f), ++g_kernel_launches;
+    if (forked) {
+        const cudaError_t e = cudaStreamWaitEvent(st, join, 0);
+        if (e != cudaSuccess) return e;
+    }
     return cudaGetLastError();
 }
 
