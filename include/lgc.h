@@ -12,9 +12,14 @@
  *  - Memory.  The caller owns every device byte: `state`, `scratch`, `params`, the gradients and
  *    the update.  The library allocates no device memory and frees none; `lgc_ctx` is its only
  *    host allocation (released by lgc_destroy).  Device pointers must be 16-byte aligned.
- *  - Streams.  All work is enqueued on the stream given in lgc_config.stream (a cudaStream_t,
- *    NULL = the legacy default stream).  Stage calls never synchronise; lgc_init, lgc_check and
- *    the host-pointer forms of the parameter accessors do.
+ *  - Streams.  All work is ordered by the stream given in lgc_config.stream (a cudaStream_t,
+ *    NULL = the legacy default stream): when that stream has drained, everything a call
+ *    enqueued has run.  Two calls fork onto streams of the library's own and join back before
+ *    they return control of the ordering to that stream: lgc_topk of the parameter-server
+ *    variant (small layers beside the large ones) and lgc_step_host (the upload).  Those streams
+ *    and their events are created at the first such call and released by lgc_destroy.  Stage
+ *    calls never synchronise; lgc_init, lgc_check and the host-pointer forms of the parameter
+ *    accessors do.
  *  - Errors.  Every call returns an lgc_status; nothing aborts, throws or traps.  Argument and
  *    call-order errors are detected on the host before anything is enqueued.  Inconsistencies a
  *    kernel detects are recorded in a device word that lgc_check reads.
