@@ -232,7 +232,11 @@ __global__ void ae5_prep_deconv_weights_kernel(const float *__restrict__ w, int 
 // Every wait has a limit; a CTA whose wait runs out records it and leaves without touching the
 // output (tensor memory is released on every path).
 // ------------------------------------------------------------------------------------------
-enum GemmMode { kConv = 0, kConvCode = 1, kDeconv = 2, kDeconvFinal = 3 };
+// kGradDeconv: the gradient at the input of a convolution, which is a transposed convolution of the gradient at
+//   its output with the same weights (w[co][ci][tau] read as [c_in' = co][c_out' = ci][tau]).  As kDeconv, for every
+//   node, but the epilogue adds no bias: it multiplies by the leaky ReLU's derivative at the convolution's input
+//   (sign of the stored activation `extra`, laid out like the output) and writes the two tf32 parts.
+enum GemmMode { kConv = 0, kConvCode = 1, kDeconv = 2, kDeconvFinal = 3, kGradDeconv = 4 };
 
 template <int MODE, int CIN, int COUT>
 struct GemmShape {
@@ -272,7 +276,8 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
     const int t0 = blockIdx.x * kTileM;
     const uint32_t tiles = (smem_u32(dyn_smem) + 1023u) & ~1023u;
 
-    for (int i = threadIdx.x; i < COUT; i += 128) s_bias[i] = bias[i];
+    if (MODE != kGradDeconv)
+        for (int i = threadIdx.x; i < COUT; i += 128) s_bias[i] = bias[i];
     if (MODE == kConvCode) {
         for (int i = threadIdx.x; i < 4 * 64; i += 128) s_wl[i] = w_last[i];
         if (threadIdx.x < 4) s_bl[threadIdx.x] = b_last[threadIdx.x];
@@ -384,8 +389,23 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
             float x[32];
             tmem_load32(trow + (uint32_t)c0, x);
             const int cb = S::kIsConv ? c0 : c0 % COUT;         // channel of column c0
+            if (MODE == kGradDeconv) {
+                const int64_t pos = 2 * t + (c0 >= COUT ? 1 : 0);
+                if (pos < L_out) {
+                    const float4 *m4 = reinterpret_cast<const float4 *>(extra + ((int64_t)node * Lpad_out + pos) * COUT + cb);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) x[j] = leaky(__fadd_rn(x[j], s_bias[cb + j]));
+                    for (int q = 0; q < 8; ++q) {
+                        const float4 m = m4[q];
+                        x[4 * q] = m.x > 0.0f ? x[4 * q] : __fmul_rn(kSlope, x[4 * q]);
+                        x[4 * q + 1] = m.y > 0.0f ? x[4 * q + 1] : __fmul_rn(kSlope, x[4 * q + 1]);
+                        x[4 * q + 2] = m.z > 0.0f ? x[4 * q + 2] : __fmul_rn(kSlope, x[4 * q + 2]);
+                        x[4 * q + 3] = m.w > 0.0f ? x[4 * q + 3] : __fmul_rn(kSlope, x[4 * q + 3]);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) x[j] = leaky(__fadd_rn(x[j], s_bias[cb + j]));
+            }
             if (MODE == kConvCode) {
 #pragma unroll
                 for (int o = 0; o < 4; ++o)
@@ -417,7 +437,8 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
                     // conv: row tr is position tr; deconv: columns below COUT are position 2 tr, the others 2 tr + 1
                     const int64_t pos = S::kIsConv ? tr : 2 * tr + (c0 >= COUT ? 1 : 0);
                     if (pos < L_out) {
-                        const int64_t at = (S::kIsConv ? ((int64_t)node * Lpad_out + tr) * COUT : 2 * tr * COUT) + c0 + 4 * cq;
+                        const int64_t at = (S::kIsConv ? ((int64_t)node * Lpad_out + tr) * COUT
+                                                       : ((int64_t)node * Lpad_out + 2 * tr) * COUT) + c0 + 4 * cq;
                         *reinterpret_cast<float4 *>(out_hi + at) = *reinterpret_cast<const float4 *>(sh_hi + rr * kStagePitch + 4 * cq);
                         *reinterpret_cast<float4 *>(out_lo + at) = *reinterpret_cast<const float4 *>(sh_lo + rr * kStagePitch + 4 * cq);
                     }
@@ -663,9 +684,15 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         a.dact5_hi = take((size_t)mu * 32);
         a.dact5_lo = take((size_t)mu * 32);
         size_t pmax = 0;
-        for (int l = 0; l < 4; ++l) {
-            a.g_enc[l] = take((size_t)K * a.len[l + 1] * kAe5EncCh[l + 1]);
-            if (l > 0) pmax = std::max(pmax, (size_t)K * a.len[l + 1] * 3 * kAe5EncCh[l]);
+        for (int l = 0; l < 3; ++l) {                       // laid out like the outputs of conv1..conv3
+            a.g_enc[l] = take((size_t)K * a.lpad[l] * kAe5EncCh[l + 1]);
+            a.g_enc_lo[l] = take((size_t)K * a.lpad[l] * kAe5EncCh[l + 1]);
+        }
+        a.g_enc[3] = take((size_t)K * a.len[4] * 64);
+        pmax = (size_t)K * a.len[4] * 3 * kAe5EncCh[3];     // only conv4's input gradient goes through the products
+        for (int j = 0; j < 2; ++j) {
+            a.gw_hi[j] = take((size_t)4 * kAe5EncCh[j + 1] * kAe5EncCh[j + 2]);
+            a.gw_lo[j] = take((size_t)4 * kAe5EncCh[j + 1] * kAe5EncCh[j + 2]);
         }
         a.g_dec[0] = take((size_t)a.len[4] * 4);
         for (int l = 1; l < 5; ++l) a.g_dec[l] = take((size_t)a.len[4 - l] * kAe5DecCh[l + 1]);
@@ -739,6 +766,19 @@ cudaError_t ae5_make_maps(Ctx &c)
         const int dcin = kAe5DecCh[l + 2];
         ok = ok && make_dact_map(enc, &a.map_dact_hi[l], a.dact_hi[l], dcin, a.len[3 - l]);
         ok = ok && make_dact_map(enc, &a.map_dact_lo[l], a.dact_lo[l], dcin, a.len[3 - l]);
+    }
+    for (int j = 0; j < 2; ++j) {            // input-gradient GEMMs of conv2 and conv3: A = the gradient at the layer's output
+        const int C = kAe5EncCh[j + 2], cin = kAe5EncCh[j + 1];
+        const cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)a.len[j + 2], (cuuint64_t)c.K};
+        const cuuint64_t strides[2] = {(cuuint64_t)C * 4, (cuuint64_t)a.lpad[j + 1] * C * 4};
+        const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileM, 1};
+        const cuuint32_t es[3] = {1, 1, 1};
+        for (int h = 0; h < 2; ++h)
+            ok = ok && enc(h ? &a.map_g_lo[j] : &a.map_g_hi[j], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
+                           h ? a.g_enc_lo[j + 1] : a.g_enc[j + 1], dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+        ok = ok && make_matrix_map(enc, &a.map_gw_hi[j], a.gw_hi[j], 2 * C, 2 * cin);
+        ok = ok && make_matrix_map(enc, &a.map_gw_lo[j], a.gw_lo[j], 2 * C, 2 * cin);
     }
     a.map_dw_hi.resize((size_t)a.decoders * 3);
     a.map_dw_lo.resize((size_t)a.decoders * 3);
@@ -886,6 +926,25 @@ cudaError_t launch_ae5_train_forward(Ctx &c)
     c.mean_valid = false;
     e = launch_combine_mean(c);
     return e != cudaSuccess ? e : launch_ae5_train_decode(c, 0);
+}
+
+cudaError_t launch_ae5_input_gradient(Ctx &c, int layer)
+{
+    Ae5 &a = *c.ae5;
+    const int j = layer - 1;                                   // 0: conv2, 1: conv3
+    const int cin = kAe5EncCh[layer], cout = kAe5EncCh[layer + 1];
+    // the convolution's weights w[co][ci][tau] are a transposed convolution's with c_in' = co, c_out' = ci
+    ae5_prep_deconv_weights_kernel<<<blocks((int64_t)4 * cin * cout, 256), 256, 0, c.stream>>>(c.params + a.off_w[layer], cout, cin,
+                                                                                             a.gw_hi[j], a.gw_lo[j]),
+        ++g_kernel_launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int64_t rows = a.len[layer + 1] + 1;                 // one more than the output positions: the last makes the tail
+    if (layer == 1)
+        return launch_gemm<kGradDeconv, 128, 64>(c, a.map_g_hi[0], a.map_g_lo[0], a.map_gw_hi[0], a.map_gw_lo[0], nullptr, rows, c.K,
+                                                 a.len[1], a.lpad[0], a.g_enc[0], a.g_enc_lo[0], nullptr, nullptr, nullptr, a.act_hi[0]);
+    return launch_gemm<kGradDeconv, 256, 128>(c, a.map_g_hi[1], a.map_g_lo[1], a.map_gw_hi[1], a.map_gw_lo[1], nullptr, rows, c.K,
+                                              a.len[2], a.lpad[1], a.g_enc[1], a.g_enc_lo[1], nullptr, nullptr, nullptr, a.act_hi[1]);
 }
 
 // Stage 5 up to the reconstruction.  Ring-allreduce: the decoder on the mean code; c.recon gets the mu

@@ -237,11 +237,23 @@ tn_narrow_kernel(Rows A, Rows B, int Q, int64_t M, int64_t chunk, float *__restr
     }
 }
 
+// x = hi + lo with both parts representable in tf32 (what the tensor-core GEMMs take)
+__device__ __forceinline__ void split_tf32(float x, float &hi, float &lo)
+{
+    uint32_t h;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(x));
+    hi = __uint_as_float(h);
+    const float r = __fsub_rn(x, hi);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(r));
+    lo = __uint_as_float(h);
+}
+
 // Gradient at a convolution's input from the products prod[k][t][tau C_in + ci] = (G W)[t]:
-//   g_in[k][pos][ci] = leaky'(x[k][pos][ci]) * sum over (t, tau) with 2t + tau = pos of prod[k][t][tau C_in + ci].
-// Thread per (node, position, four channels).
+//   g_in[k][pos][ci] = leaky'(x[k][pos][ci]) * sum over (t, tau) with 2t + tau = pos of prod[k][t][tau C_in + ci],
+// written as two tf32 parts in the layout of x (node stride x_node_stride).  Thread per (node, position, four channels).
 __global__ void fold_kernel(const float *__restrict__ prod, int K, int64_t L_out, int64_t L_in, int cin,
-                            const float *__restrict__ x_hi, int64_t x_node_stride, float *__restrict__ g_in)
+                            const float *__restrict__ x_hi, int64_t x_node_stride, float *__restrict__ g_hi,
+                            float *__restrict__ g_lo)
 {
     const int quads = cin >> 2;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -256,12 +268,16 @@ __global__ void fold_kernel(const float *__restrict__ prod, int K, int64_t L_out
         const float4 p = *reinterpret_cast<const float4 *>(prod + ((k * L_out + (d >> 1)) * 3 + tau) * cin + 4 * cq);
         acc.x = __fadd_rn(acc.x, p.x); acc.y = __fadd_rn(acc.y, p.y); acc.z = __fadd_rn(acc.z, p.z); acc.w = __fadd_rn(acc.w, p.w);
     }
-    const float4 x = *reinterpret_cast<const float4 *>(x_hi + k * x_node_stride + pos * cin + 4 * cq);
+    const int64_t at = k * x_node_stride + pos * cin + 4 * cq;
+    const float4 x = *reinterpret_cast<const float4 *>(x_hi + at);
     acc.x = x.x > 0.f ? acc.x : __fmul_rn(kSlope, acc.x);
     acc.y = x.y > 0.f ? acc.y : __fmul_rn(kSlope, acc.y);
     acc.z = x.z > 0.f ? acc.z : __fmul_rn(kSlope, acc.z);
     acc.w = x.w > 0.f ? acc.w : __fmul_rn(kSlope, acc.w);
-    *reinterpret_cast<float4 *>(g_in + (k * L_in + pos) * cin + 4 * cq) = acc;
+    float4 hi, lo;
+    split_tf32(acc.x, hi.x, lo.x); split_tf32(acc.y, hi.y, lo.y); split_tf32(acc.z, hi.z, lo.z); split_tf32(acc.w, hi.w, lo.w);
+    *reinterpret_cast<float4 *>(g_hi + at) = hi;
+    *reinterpret_cast<float4 *>(g_lo + at) = lo;
 }
 
 // One layer's weights arranged as the dense [Kd][N] operand of nn_gemm_kernel.
@@ -621,7 +637,9 @@ void encoder_backward(Launcher &L, const float *dzbar)
     for (int i = 3; i >= 0; --i) {
         const int cin = kAe5EncCh[i], cout = kAe5EncCh[i + 1];
         const int64_t lin = len[i], lout = len[i + 1];
-        const Rows g = rows_of(a.g_enc[i], nullptr, lout * cout, cout, lout, cout);  // [K][lout][cout]
+        // gradient at conv(i+1)'s output: conv4's is fp32, the others are two tf32 parts laid out like the output
+        const Rows g = i == 3 ? rows_of(a.g_enc[3], nullptr, lout * cout, cout, lout, cout)
+                              : rows_of(a.g_enc[i], a.g_enc_lo[i], a.lpad[i] * cout, cout, lout, cout);
         L.colsum(2 * i + 1, g);
         if (i == 0) {        // conv1 reads the kept values themselves: rows of three floats, two apart
             L.tn_narrow(0, g, rows_of(c.val, nullptr, mu, 2, lout, 3), 3);
@@ -629,12 +647,16 @@ void encoder_backward(Launcher &L, const float *dzbar)
         }
         const int64_t x_node = a.lpad[i - 1] * cin;
         L.tn(2 * i, g, rows_of(a.act_hi[i - 1], a.act_lo[i - 1], x_node, 2 * cin, lout, 3 * cin));
-        L.arrange(P + a.off_w[i], cin, cout, 0);
-        L.nn(g, (int64_t)K * lout, a.wt, 3 * cin, a.pbuf, nullptr);
-        if (L.ok()) {
-            fold_kernel<<<blocks((int64_t)K * lin * (cin / 4), 256), 256, 0, c.stream>>>(a.pbuf, K, lout, lin, cin, a.act_hi[i - 1],
-                                                                                        x_node, a.g_enc[i - 1]),
-                ++g_kernel_launches;
+        if (i == 3) {        // conv4 (768 output columns: too wide for one accumulator): products on the fp32 pipes, then the fold
+            L.arrange(P + a.off_w[i], cin, cout, 0);
+            L.nn(g, (int64_t)K * lout, a.wt, 3 * cin, a.pbuf, nullptr);
+            if (L.ok()) {
+                fold_kernel<<<blocks((int64_t)K * lin * (cin / 4), 256), 256, 0, c.stream>>>(a.pbuf, K, lout, lin, cin, a.act_hi[i - 1],
+                                                                                            x_node, a.g_enc[i - 1], a.g_enc_lo[i - 1]),
+                    ++g_kernel_launches;
+            }
+        } else if (L.ok()) {  // conv3, conv2: a transposed convolution of g with the same weights, on the tensor cores
+            L.err = launch_ae5_input_gradient(c, i);
         }
     }
 }

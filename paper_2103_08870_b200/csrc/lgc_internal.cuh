@@ -107,7 +107,10 @@ struct Ae5 {
     // ---- training step (lgc_ae_train_step) ----
     float *act4_hi = nullptr, *act4_lo = nullptr;    // [K][L4][64] output of conv4 (inference folds it into conv5)
     float *dact5_hi = nullptr, *dact5_lo = nullptr;  // [mu][32] output of deconv5 (inference folds it into the last conv)
-    float *g_enc[4] = {};               // dLoss/d(pre-activation) of conv1..conv4: [K][L_i][C_i]
+    float *g_enc[4] = {};               // dLoss/d(pre-activation) of conv1..conv4.  conv4's: fp32 [K][L4][64].  conv1..conv3's:
+    float *g_enc_lo[3] = {};            // two tf32 parts laid out like the layer's output, [K][lpad][C] (they feed tensor-core GEMMs)
+    float *gw_hi[2] = {}, *gw_lo[2] = {};   // weights of conv2 / conv3 arranged for the GEMM that makes the gradient at their input
+    CUtensorMap map_g_hi[2], map_g_lo[2], map_gw_hi[2], map_gw_lo[2];
     float *g_dec[5] = {};               // the same for deconv1..deconv5: [L][C], g_dec[4] is [mu][32]
     float *dzk = nullptr;               // [K][L4][4] gradient at every node's code
     float *dzbar = nullptr;             // [L4][4]    gradient at the mean code
@@ -248,6 +251,8 @@ cudaError_t launch_ae5_train_encode(Ctx &c);           // every node's code into
 cudaError_t launch_ae5_train_decode(Ctx &c, int d);    // decoder d on c.combined, up to deconv5 (kept in dact5)
 cudaError_t launch_ae5_train_forward(Ctx &c);          // ring-allreduce: encoder, mean, the decoder
 cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out);
+// gradient at the input of conv2 (layer = 1) or conv3 (layer = 2) from g_enc[layer] into g_enc[layer - 1], on the tensor cores
+cudaError_t launch_ae5_input_gradient(Ctx &c, int layer);
 cudaError_t launch_ae5_train_step_ps(Ctx &c, int common, float lam_rec, float lam_sim, float *loss_out);
 struct AdamArgs {
     float *params, *m, *v;
