@@ -210,20 +210,32 @@ tn_narrow_kernel(Rows A, Rows B, int Q, int64_t M, int64_t chunk, float *__restr
     const int p = blockIdx.y * 32 + lane;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     RowCursor ca(A, first + warp), cb(B, first + warp);
-    for (int64_t m = first + warp; m < last; m += 8, ca.advance(A, 8), cb.advance(B, 8)) {
-        float b[4] = {1.f, 0.f, 0.f, 0.f};
-        if (B.hi) {
-            const int64_t bb = cb.at(B);
+    // four of the warp's rows per trip: their loads are in flight together, the sums are added in row order
+    for (int64_t m = first + warp; m < last; m += 32) {
+        float a[4], b[4][4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (q < Q) b[q] = B.lo ? __fadd_rn(B.hi[bb + q], B.lo[bb + q]) : B.hi[bb + q];
-        }
-        if (p < A.len) {
-            const int64_t ab = ca.at(A) + p;
-            const float a = A.lo ? __fadd_rn(A.hi[ab], A.lo[ab]) : A.hi[ab];
+        for (int r = 0; r < 4; ++r) {
+            a[r] = 0.f;
+            b[r][0] = 1.f; b[r][1] = b[r][2] = b[r][3] = 0.f;
+            if (m + 8 * r < last) {
+                if (B.hi) {
+                    const int64_t bb = cb.at(B);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) acc[q] = __fmaf_rn(a, b[q], acc[q]);
+                    for (int q = 0; q < 4; ++q)
+                        if (q < Q) b[r][q] = B.lo ? __fadd_rn(B.hi[bb + q], B.lo[bb + q]) : B.hi[bb + q];
+                }
+                if (p < A.len) {
+                    const int64_t ab = ca.at(A) + p;
+                    a[r] = A.lo ? __fadd_rn(A.hi[ab], A.lo[ab]) : A.hi[ab];
+                }
+            }
+            ca.advance(A, 8);
+            cb.advance(B, 8);
         }
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[q] = __fmaf_rn(a[r], b[r][q], acc[q]);
     }
 #pragma unroll
     for (int q = 0; q < 4; ++q) part[warp][lane][q] = acc[q];
