@@ -103,13 +103,18 @@ nn_gemm_kernel(Rows A, int64_t M, const float *__restrict__ B, int N, float *__r
     const int64_t am = m0 + ar;
     const int64_t abase = am < M ? A.at(am) : 0;
     const int bk = threadIdx.x >> 4, bnq = threadIdx.x & 15;         // B tile: 16 rows x 64 columns
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    const bool bcol = n0 + 4 * bnq < N;
+    float4 a = am < M ? load4(A, abase, 4 * akq) : zero;
+    float4 b = bcol ? *reinterpret_cast<const float4 *>(B + (int64_t)bk * N + n0 + 4 * bnq) : zero;
     for (int k0 = 0; k0 < A.len; k0 += kStep) {
-        const float4 a = am < M ? load4(A, abase, k0 + 4 * akq) : make_float4(0.f, 0.f, 0.f, 0.f);
         As[4 * akq + 0][ar] = a.x; As[4 * akq + 1][ar] = a.y; As[4 * akq + 2][ar] = a.z; As[4 * akq + 3][ar] = a.w;
-        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (n0 + 4 * bnq < N) b = *reinterpret_cast<const float4 *>(B + (int64_t)(k0 + bk) * N + n0 + 4 * bnq);
         *reinterpret_cast<float4 *>(&Bs[bk][4 * bnq]) = b;
         __syncthreads();
+        if (k0 + kStep < A.len) {               // the next entries travel while these are multiplied
+            a = am < M ? load4(A, abase, k0 + kStep + 4 * akq) : zero;
+            b = bcol ? *reinterpret_cast<const float4 *>(B + (int64_t)(k0 + kStep + bk) * N + n0 + 4 * bnq) : zero;
+        }
 #pragma unroll
         for (int k = 0; k < kStep; ++k) {
             const float4 av = *reinterpret_cast<const float4 *>(&As[k][4 * ty]);
@@ -157,16 +162,24 @@ tn_gemm_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ par
     float2 acc[4][2] = {};
     const int lr = threadIdx.x >> 4, lc = threadIdx.x & 15;          // 16 rows x 64 columns of each operand per trip
     RowCursor ca(A, first + lr), cb(B, first + lr);
-    for (int64_t r0 = first; r0 < last; r0 += kStep, ca.advance(A, kStep), cb.advance(B, kStep)) {
-        const int64_t m = r0 + lr;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-        if (m < last) {
-            a = load4(A, ca.at(A), p0 + 4 * lc);
-            b = load4(B, cb.at(B), q0 + 4 * lc);
-        }
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 a = zero, b = zero;
+    if (first + lr < last) {
+        a = load4(A, ca.at(A), p0 + 4 * lc);
+        b = load4(B, cb.at(B), q0 + 4 * lc);
+    }
+    for (int64_t r0 = first; r0 < last; r0 += kStep) {
         *reinterpret_cast<float4 *>(&As[lr][4 * lc]) = a;
         *reinterpret_cast<float4 *>(&Bs[lr][4 * lc]) = b;
         __syncthreads();
+        // the next trip's rows travel while this one is multiplied
+        ca.advance(A, kStep);
+        cb.advance(B, kStep);
+        a = b = zero;
+        if (r0 + kStep + lr < last) {
+            a = load4(A, ca.at(A), p0 + 4 * lc);
+            b = load4(B, cb.at(B), q0 + 4 * lc);
+        }
 #pragma unroll
         for (int k = 0; k < kStep; ++k) {
             const float4 av = *reinterpret_cast<const float4 *>(&As[k][4 * ty]);
