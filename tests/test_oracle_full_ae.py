@@ -364,3 +364,31 @@ def test_ps_training_gradients_against_finite_differences():
         fd = (A.ps_loss_and_grads(val, inn, unpack_ps(hi, K), 0, 1.0, 0.5)[0]
               - A.ps_loss_and_grads(val, inn, unpack_ps(lo, K), 0, 1.0, 0.5)[0]) / (2 * eps)
         assert abs(fd - gf[i]) <= 1e-5 * max(1e-3, abs(gf[i])) + 1e-8, (i, fd, gf[i])
+
+
+def test_layer_shapes_follow_the_tables_of_the_paper():
+    # tests/golden/full_ae_layers.txt restates the two tables of Section IV-C; every tensor of the oracle, and of
+    # the seeded initialiser the tests and the benchmark use, must have the filters and taps printed there, each
+    # layer taking as many input channels as the layer before it has filters (1 for conv1, 4 = the code for deconv1)
+    import os
+    from paper_2103_08870_b200 import workloads as W
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", "full_ae_layers.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                side, layer, filters, taps, stride = line.split()
+                rows.append((side, layer, int(filters), int(taps), int(stride)))
+    assert len(rows) == 11
+    shapes = dict(A.param_shapes())
+    init_shapes = {n: s for n, s, _ in W.ae5_param_shapes()}
+    prev = {"enc": 1, "dec": 4}
+    for i, (side, layer, filters, taps, stride) in enumerate(rows):
+        n = i + 1 if side == "enc" else i - 4
+        w = shapes[f"{side}.w{n}"]
+        transposed = layer.startswith("deconv")
+        want = (prev[side], filters, taps) if transposed else (filters, prev[side], taps)
+        assert w == want and shapes[f"{side}.b{n}"] == (filters,), (layer, w, want)
+        assert init_shapes[f"{side}.w{n}"] == want
+        prev[side] = filters
+    assert rows[4][2] == 4                                   # the code the decoder starts from has conv5's 4 channels
+    assert [r[4] for r in rows if r[3] == 3] == [2] * 9      # as printed; deconv1's stride is the documented reading
