@@ -553,3 +553,24 @@ def test_full_size_autoencoder_at_its_shortest_inputs(variant, numel):
         for name, got in per_tensor(m / 0.1, A5.param_shapes()):
             assert_close(got, grads_ref[name], f"gradient of {name}", rel=2e-5)
     gpu.check()
+
+
+def test_parameter_server_with_five_nodes():
+    # five index sets that overlap in part: the node-ordered average looks an index up in the other nodes' lists
+    # eight nodes at a time (one batch here, with idle slots), with and without the update buffer announced
+    numel = [70001, 9000, 20000, 4097, 127, 300_000]
+    K = 5
+    ora, gpu = make_pair(numel, K, variant="ps", c1=16, c2=8)
+    src = toy_source(numel, K, seed=59)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    for t in range(4):
+        g = src.step(t)
+        compare_step(ora, gpu, g, g.cuda(), (3 * t + 1) % K, upd, announce_update=(t % 2 == 0))
+    g = src.step(4)                                   # and the second training phase's sparse mean
+    ora.accumulate(g.numpy())
+    gpu.accumulate(g.cuda())
+    ora.topk()
+    gpu.topk(0)
+    assert_close(upd_of(gpu, upd), ora.topk_scatter(), "sparse update")
+    assert_bitwise(gpu.v.cpu().numpy(), ora.v, "v")
+    gpu.check()
