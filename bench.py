@@ -99,6 +99,54 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+class NvmlClockSampler:
+    """The same through NVML (read-only queries), polled from a thread every few milliseconds: a timed
+    region of a fraction of a second still gets tens of samples."""
+
+    def __init__(self, index: int):
+        import pynvml
+        self.nv = pynvml
+        self.REASONS = (("hw_slowdown", pynvml.nvmlClocksThrottleReasonHwSlowdown),
+                        ("hw_thermal_slowdown", pynvml.nvmlClocksThrottleReasonHwThermalSlowdown),
+                        ("sw_thermal_slowdown", pynvml.nvmlClocksThrottleReasonSwThermalSlowdown),
+                        ("sw_power_cap", pynvml.nvmlClocksThrottleReasonSwPowerCap))
+        pynvml.nvmlInit()
+        self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+        self.sm, self.bits, self.stop_flag = [], 0, False
+
+    def start(self):
+        self.thread = threading.Thread(target=self._poll, daemon=True)
+        self.thread.start()
+
+    def _poll(self):
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                self.bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            except Exception:
+                pass
+            time.sleep(0.003)
+
+    def stop(self):
+        self.stop_flag = True
+        self.thread.join(timeout=2)
+        mx = None
+        try:
+            mx = float(self.nv.nvmlDeviceGetMaxClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+        except Exception:
+            pass
+        return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": mx, "samples": len(self.sm),
+                "reasons": sorted(name for name, bit in self.REASONS if self.bits & bit), "source": "nvml"}
+
+
+def clock_sampler(index: int):
+    try:
+        return NvmlClockSampler(index)
+    except Exception:
+        return ClockSampler(index)
+
+
 def visible_gpu_index(local: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -204,7 +252,7 @@ def run_ours(args, w: W.Workload):
     gpu.check()
     barrier()
 
-    sampler = ClockSampler(visible_gpu_index(local))
+    sampler = clock_sampler(visible_gpu_index(local))
     sampler.start()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
