@@ -166,8 +166,9 @@ lgc_status lgc_topk_scatter(lgc_ctx *ctx, float *update);
  * reconstruction loss of Section IV-B scaled by 1/mu,
  *     loss = (1/mu) || D_c((1/K) sum_k E_c(g~_k)) - (1/K) sum_k g~_k ||^2,
  * analytic backward pass, Adam with bias correction.  Ring-allreduce variant, LGC_AE_CONV2 or
- * LGC_AE_CONV5 (whose forward pass runs on the tensor cores as in lgc_encode, the backward pass
- * on the fp32 pipes; gradient sums in fp64 over per-chunk fp32 partial sums).
+ * LGC_AE_CONV5 (whose forward pass and the two largest input-gradient products run on the tensor
+ * cores as in lgc_encode, the rest of the backward pass on the fp32 pipes; gradient sums in fp64
+ * over per-chunk fp32 partial sums).
  * loss_out: device fp32 scalar or NULL.  May be called several times after one lgc_topk. */
 lgc_status lgc_ae_train_step(lgc_ctx *ctx, float *loss_out);
 
