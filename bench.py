@@ -278,6 +278,25 @@ def run_ours(args, w: W.Workload):
     # every step's own time: from its first event to the next step's (the last one: to the closing event)
     step_ms = [ev[t][0].elapsed_time(ev[t + 1][0] if t + 1 < args.steps else stop) for t in range(args.steps)]
 
+    # optional: the five stages' own times, on steps of their own after the timed region (an event between the
+    # stage calls costs about a microsecond each, so they stay out of the reported step time)
+    stages_us = None
+    if args.stage_times:
+        names = ("accumulate", "topk", "encode", "combine", "decode_scatter")
+        marks = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(min(args.steps, 50))]
+        for t, m in enumerate(marks):
+            i = args.warmup + args.steps + t
+            ch = W.choice_for_step(w.seed, i, K)
+            m[0].record(); gpu.accumulate(grads[i % GRAD_SETS], ch)
+            m[1].record(); gpu.topk(ch, update)
+            m[2].record(); gpu.encode()
+            m[3].record(); gpu.combine(ch)
+            m[4].record(); gpu.decode_scatter(update)
+            m[5].record()
+        barrier()
+        gpu.check()
+        stages_us = {n: 1e3 * statistics.median(m[j].elapsed_time(m[j + 1]) for m in marks) for j, n in enumerate(names)}
+
     # end to end through host buffers: pinned gradients in, dense update out, every step
     e2e_steps = 0 if args.no_e2e else max(2, min(args.steps, 20))
     e2e_ms = 0.0
@@ -323,6 +342,8 @@ def run_ours(args, w: W.Workload):
             "gpu_launches": gpu_launches,
             "clocks": clocks,
         }
+        if stages_us is not None:
+            out["stages_us"] = stages_us        # medians, this rank
         if world == 1 and not args.no_cpu_baseline:
             gbs, times = oracle_throughput(w, args.cpu_sample_steps, [g.cpu().numpy() for g in grads])
             out["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
@@ -345,6 +366,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--nodes", type=int, default=0, help="override K (profiling aid: a smaller device footprint)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling aid)")
+    ap.add_argument("--stage-times", action="store_true", help="also report the median time of each of the five stages")
     args = ap.parse_args()
     w = W.workload(args.workload)
     if args.nodes > 0:
