@@ -473,22 +473,31 @@ __device__ __forceinline__ int compact_group(const FastArgs &f, int row, int li,
     // one candidate per thread and trip, eight trips in flight: its chunk by binary search in
     // shared memory, then its record from the chunk's list (neighbouring ranks read
     // neighbouring records)
+    int top = 1;                                           // largest power of two below gn (1 when gn <= 2)
+    while (top * 2 < gn) top *= 2;
     for (int base = 0; base < (int)total; base += kFinThreads * 8) {
         const uint2 *rec[8];
         int tile0[8];
+        // the last chunk whose offset is <= rank, for the eight ranks side by side: the halving steps run in
+        // lock step, so that the eight shared-memory reads of a step are in flight together
+        int lo[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) lo[t] = 0;
+        for (int step = top; step > 0; step >>= 1) {
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const int at = lo[t] + step;
+                if (at < gn && group_off[at] <= base + t * kFinThreads + (int)threadIdx.x) lo[t] = at;
+            }
+        }
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
             const int r = base + t * kFinThreads + (int)threadIdx.x;
             rec[t] = nullptr;
             tile0[t] = 0;
             if (r < (int)total) {
-                int lo = 0, hi = gn;                       // last chunk whose offset is <= rank
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (group_off[mid] <= r) lo = mid; else hi = mid;
-                }
-                rec[t] = f.cand + ((int64_t)row * f.num_tchunks + gb + lo) * kCandCap + (r - group_off[lo]);
-                tile0[t] = (q0 + (gb + lo - c0)) * kSelChunk;                 // N < 2^31
+                rec[t] = f.cand + ((int64_t)row * f.num_tchunks + gb + lo[t]) * kCandCap + (r - group_off[lo[t]]);
+                tile0[t] = (q0 + (gb + lo[t] - c0)) * kSelChunk;              // N < 2^31
             }
         }
         uint2 kp[8];
