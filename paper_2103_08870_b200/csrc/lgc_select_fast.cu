@@ -42,6 +42,7 @@ struct FastArgs {
     uint4 *zero_ptr;               // buffer the spare CTAs of the finishing launch clear (row 0 only), or nullptr
     uint64_t zero_vecs;            // its length in whole 16-byte units
     int zero_tail;                 // floats beyond them (0..3)
+    int zero_ctas, zero_threads;   // spare CTAs that share the clearing, and how many of their threads store
     int32_t epoch;                 // step whose fused accumulation may have filled the lists (-1: none)
     const int64_t *seg_off;
     const int32_t *seg_len, *seg_k, *seg_out, *small_ids, *large_ids, *seg_large, *large_q0, *tchunk0, *tchunk_large;
@@ -64,7 +65,16 @@ constexpr int kFinSmemCap = 20480;    // candidate keys a finishing CTA keeps in
 constexpr int kFinGroup = kSelGroup;  // chunks whose candidate counts are scanned together during the compaction
 constexpr int kFinPerThread = 16;     // consecutive entries per thread in the ordered passes
 constexpr int kCandCap = kSelCandCap;  // entries a chunk's list can hold; a chunk with more sends its segment to the data
-constexpr int kZeroPerThread = 8;     // 16-byte stores per thread of a CTA that clears a slice of the update
+// Spare CTAs that clear the update: at least about one per SM, each thread up to kZeroPerThread stores.  Up to
+// kZeroGentleBytes only a quarter of a CTA's threads store: CTAs of 512 storing threads on every SM made the selecting
+// CTAs beside them wait on the load/store path (their shared-memory searches took ~100 cycles a read), and a buffer of
+// that size is cleared long before the selection is done anyway.  Larger buffers need every thread to reach the
+// memory's write rate.
+constexpr int kZeroCtasMin = 148;
+constexpr int kZeroPerThread = 512;     // stores per thread, gentle form
+constexpr int kZeroPerThreadFast = 8;   // large buffers: many short CTAs of 512 storing threads (4 GiB in 0.66 ms)
+constexpr int kZeroGentleThreads = 128;
+constexpr uint64_t kZeroGentleBytes = 512ull << 20;
 constexpr int kAccThreads = 1024;     // accumulation: one 128-bit g/u/v triple per thread, 4096 elements per CTA
 
 // The key from which the next step collects candidates, given this step's k-th key T.  Error
@@ -738,12 +748,11 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
     const int row = blockIdx.y;
     if ((int)blockIdx.x >= f.num_large + f.fin_small) {      // spare CTAs: clear the dense update meanwhile
         if (row != 0) return;
-        const uint64_t first = (uint64_t)(blockIdx.x - f.num_large - f.fin_small) * (kFinThreads * kZeroPerThread);
-#pragma unroll
-        for (int i = 0; i < kZeroPerThread; ++i) {
-            const uint64_t e = first + (uint64_t)i * kFinThreads + threadIdx.x;
+        if ((int)threadIdx.x >= f.zero_threads) return;
+        const uint64_t stride = (uint64_t)f.zero_ctas * f.zero_threads;
+        for (uint64_t e = (uint64_t)(blockIdx.x - f.num_large - f.fin_small) * f.zero_threads + threadIdx.x; e <= f.zero_vecs; e += stride) {
             if (e < f.zero_vecs) __stcs(f.zero_ptr + e, make_uint4(0u, 0u, 0u, 0u));
-            else if (e == f.zero_vecs)
+            else
                 for (int j = 0; j < f.zero_tail; ++j) reinterpret_cast<float *>(f.zero_ptr + e)[j] = 0.0f;
         }
         return;
@@ -993,7 +1002,7 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
     f.num_large = t.num_large; f.num_small = t.num_small; f.num_tchunks = t.num_tchunks; f.epoch = epoch;
     f.fin_small = 0;
     f.large_order = t.large_order; f.group_job = t.group_job; f.num_group_jobs = t.num_group_jobs;
-    f.job_range = t.job_range; f.job_cnt = t.job_cnt; f.seg_wide = t.seg_wide; f.zero_ptr = nullptr; f.zero_vecs = 0; f.zero_tail = 0;
+    f.job_range = t.job_range; f.job_cnt = t.job_cnt; f.seg_wide = t.seg_wide; f.zero_ptr = nullptr; f.zero_vecs = 0; f.zero_tail = 0; f.zero_ctas = 0; f.zero_threads = 0;
     f.seg_off = t.seg_off; f.seg_len = t.seg_len; f.seg_k = t.seg_k; f.seg_out = t.seg_out;
     f.small_ids = t.small_ids; f.large_ids = t.large_ids; f.seg_large = t.seg_large; f.large_q0 = t.large_q0;
     f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_desc = t.tile_desc;
@@ -1065,7 +1074,13 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
         f.zero_ptr = reinterpret_cast<uint4 *>(clear);
         f.zero_vecs = (uint64_t)clear_floats >> 2;
         f.zero_tail = (int)(clear_floats & 3);
-        spare = (unsigned)((f.zero_vecs + 1 + kFinThreads * kZeroPerThread - 1) / (kFinThreads * kZeroPerThread));
+        f.zero_threads = f.zero_vecs * 16 <= kZeroGentleBytes ? kZeroGentleThreads : kFinThreads;
+        const uint64_t per_cta = (uint64_t)f.zero_threads * (f.zero_threads == kFinThreads ? kZeroPerThreadFast : kZeroPerThread);
+        uint64_t ctas = (f.zero_vecs + 1 + per_cta - 1) / per_cta;
+        if (ctas < (uint64_t)kZeroCtasMin) ctas = (f.zero_vecs + 1 + f.zero_threads - 1) / f.zero_threads < (uint64_t)kZeroCtasMin
+                                                      ? (f.zero_vecs + 1 + f.zero_threads - 1) / f.zero_threads : (uint64_t)kZeroCtasMin;
+        spare = (unsigned)ctas;
+        f.zero_ctas = (int)spare;
     }
     if (t.num_large + f.fin_small)
         finish_kernel<<<dim3(t.num_large + f.fin_small + spare, rows), kFinThreads, kFinDyn, st>>>(f), ++g_kernel_launches;
