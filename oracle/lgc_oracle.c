@@ -15,9 +15,11 @@
  * "sent + kept == accumulated" identity for the accumulation, torch's CPU conv1d /
  * conv_transpose1d and autograd for the convolutions and their gradients, adjointness,
  * finite differences for the training step, special weights for the parameter-server decoder.
- * PARITY UNPINNED: the placement of the innovation inside the two-layer parameter-server
- * decoder (lgc_oracle_ps_fuse) is a reading of Section IV-C / Fig. 3(a), pinned only through
- * special cases.
+ * PARITY UNPINNED: where the innovation joins a TWO-layer parameter-server decoder is a reading of
+ * Section IV-C / Fig. 3(a), which define it for the six-layer decoder only.  What the reading
+ * states -- decoder output and innovation concatenated, then a one-tap Conv1d(2 -> 1) -- is pinned:
+ * lgc_oracle_ps_fuse against torch.cat + torch's conv1d with random per-node weights, and the
+ * special weights that reduce it to either channel.  The reading itself no test can pin.
  */
 #include <math.h>
 #include <stdint.h>

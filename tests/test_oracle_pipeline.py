@@ -166,6 +166,38 @@ def test_ps_special_weights():
         assert not o.v[k, o.idx[k]].any() and not o.u[k, o.idx[k]].any()
 
 
+def test_ps_two_layer_decoder_fusion_is_a_concatenation_and_a_one_tap_convolution():
+    # Section IV-C: the innovation is "concatenated ... before the final convolutional layer".  For the
+    # two-layer decoders that reading is: decoder stack -> 1 channel, torch.cat with the innovation -> 2
+    # channels -> Conv1d(2 -> 1, one tap) whose weights are the node's (w0, w1) and whose bias is b.
+    # Built here from torch's own modules with random per-node scalars, none of the oracle's formula.
+    K = 3
+    g = grads(TOY, K, 1)[0] * 1e3
+    o = OracleLGC(TOY, K, variant="ps", params=params(8, 4, "ps", K))
+    rng = np.random.default_rng(17)
+    for k in range(K):
+        o.p[f"dec{k}.fuse"][:] = rng.uniform(-2.0, 2.0, 3)
+    o.accumulate(g)
+    o.topk()
+    o.encode()
+    o.combine(common_node=2)
+    idx = o.idx.copy()
+    upd = o.decode_scatter()
+    tp = {k: torch.from_numpy(v.copy()) for k, v in o.p.items()}
+    zc = torch.from_numpy(o.z[2])[None]
+    ref = np.zeros(o.N)
+    for k in range(K):
+        d = F.relu(F.conv_transpose1d(zc, tp[f"dec{k}.w1"], tp[f"dec{k}.b1"], stride=2, output_padding=o.op1))
+        y = F.conv_transpose1d(d, tp[f"dec{k}.w2"], tp[f"dec{k}.b2"], stride=2, output_padding=o.op2)     # [1][1][mu]
+        two = torch.cat([y, torch.from_numpy(o.inn[k].astype(np.float64))[None, None]], dim=1)            # [1][2][mu]
+        f = tp[f"dec{k}.fuse"]
+        r = F.conv1d(two, f[:2].reshape(1, 2, 1), f[2:3])[0, 0].numpy()
+        assert np.abs(o.r[k] - r).max() <= 1e-12 * np.abs(r).max(), k
+        np.add.at(ref, idx[k], r / K)
+    assert np.count_nonzero(o.inn) == K * sum(o.ki_l)                  # the second channel is not empty
+    assert np.allclose(upd, ref.astype(np.float32), rtol=1e-6, atol=1e-12)
+
+
 def test_training_gradients_by_finite_differences():
     K = 2
     g = grads(TOY, K, 1)[0] * 1e3                    # O(1) values: well-scaled differences
