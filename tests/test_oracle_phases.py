@@ -58,3 +58,44 @@ def test_topk_only_layer_sends_the_mean_of_the_kept_values_and_keeps_the_rest():
     assert len(losses) == 1 and losses[0] > 0
     ae = o.groups[1]["o"]
     assert np.count_nonzero(upd2[9408:a]) == ae.mu
+
+
+def test_one_group_per_mode_equals_runs_when_the_modes_come_in_runs():
+    # Section VI-A's table (first layer dense, last layer top-k only): every mode is one run, so grouping by
+    # mode and grouping by run are the same pipelines: identical bits, both variants
+    K = 3
+    modes = ["dense", "ae", "ae", "ae", "topk"]
+    for variant in ("rar", "ps"):
+        params = W.ae_init_params(8, 4, variant, K, 3).numpy()
+        runs = OraclePhased(NUMEL, modes, K, {1: params.copy()}, variant=variant)
+        whole = OraclePhased(NUMEL, modes, K, {0: params.copy()}, grouping="modes", variant=variant)
+        for t, phase in enumerate(["raw", "topk_train", "compressed", "compressed"]):
+            g = grads(K, t, 300.0)
+            a, la = runs.step(g, phase, t % K)
+            b, lb = whole.step(g, phase, t % K)
+            assert np.array_equal(a, b) and la == lb, (variant, t)
+        assert np.array_equal(runs.groups[1]["o"].get_params(), whole.groups[1]["o"].get_params())
+
+
+def test_layers_of_a_mode_that_are_apart_share_one_pipeline():
+    # modes (ae, topk, ae, dense, ae): the three "ae" layers feed ONE autoencoder in layer order.  Moving the
+    # layers so that each mode is a run (a permutation of the gradient's columns) gives the pinned case
+    # above; the update must be the same numbers at the moved places, and the indices the same entries.
+    K = 2
+    modes = ["ae", "topk", "ae", "dense", "ae"]
+    order = [0, 2, 4, 1, 3]                                   # ae, ae, ae, topk, dense
+    off = np.concatenate([[0], np.cumsum(NUMEL)])
+    cols = np.concatenate([np.arange(off[l], off[l + 1]) for l in order])
+    params = W.ae_init_params(8, 4, "rar", K, 3).numpy()
+    apart = OraclePhased(NUMEL, modes, K, {0: params.copy()}, grouping="modes")
+    moved = OraclePhased([NUMEL[l] for l in order], [modes[l] for l in order], K, {0: params.copy()})
+    assert [gr["mode"] for gr in apart.groups] == ["ae", "topk", "dense"] and apart.groups[0]["layers"] == [0, 2, 4]
+    for t, phase in enumerate(["topk_train", "compressed", "compressed"]):
+        g = grads(K, t, 300.0)
+        a, la = apart.step(g, phase, t % K)
+        b, lb = moved.step(np.ascontiguousarray(g[:, cols]), phase, t % K)
+        assert np.array_equal(a[cols], b) and la == lb, t
+        full = apart.full_row_indices(apart.groups[0])            # offsets inside the whole row
+        assert np.array_equal(full[0], cols[moved.groups[0]["o"].idx[0]])
+    ae = apart.groups[0]["o"]
+    assert ae.mu == sum(ae.k_l) and len(ae.k_l) == 3
