@@ -33,10 +33,31 @@ UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 GRAD_SETS = 3            # distinct gradient batches cycled through (each far larger than L2)
-# DRAM bytes (read + write) per element that ncu measured for accumulate_select_kernel on the small
-# capture case (profiles/accumulate_select_kernel_resnet50_k2.md); traffic grows in proportion to K * N.
-# Set to None whenever that kernel changes until the counters are taken again.
-NCU_DRAM_BYTES_PER_ELEMENT = 19.00
+CLOCK_WINDOW_MS = 500.0  # the clock sampler watches at least this long a run of steps (see run_ours)
+# DRAM bytes (read + write) per element that one ncu capture measured for the dominant kernel on a small
+# case (K = 2 nodes of the same layer table; traffic grows in proportion to K * N), with the SHA-256 of the
+# kernel's source file as it was when the counters were taken.  While the file differs from that, the
+# figure is not reported ("traffic": null): the kernel has changed since.
+NCU_CAPTURE = {
+    "kernel": "accumulate_select_kernel",
+    "source": os.path.join("paper_2103_08870_b200", "csrc", "lgc_select_fast.cu"),
+    "source_sha256": None,
+    "dram_bytes_per_element": None,
+}
+
+
+def ncu_traffic_bytes(elements: int):
+    """DRAM traffic of one launch over `elements` elements from the stored capture, or None when the
+    kernel's source is no longer the one that was measured."""
+    import hashlib
+    if not NCU_CAPTURE["source_sha256"] or NCU_CAPTURE["dram_bytes_per_element"] is None:
+        return None
+    try:
+        with open(os.path.join(ROOT, NCU_CAPTURE["source"]), "rb") as f:
+            now = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    return NCU_CAPTURE["dram_bytes_per_element"] * elements if now == NCU_CAPTURE["source_sha256"] else None
 
 
 def measured_peak():
@@ -157,25 +178,112 @@ def visible_gpu_index(local: int) -> int:
     return local
 
 
-def oracle_throughput(w: W.Workload, sample_steps: int, host_grads=None):
+def host_description():
+    """Core count, CPU model and memory of the machine the oracle is timed on."""
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    ram = None
+    try:
+        import psutil
+        ram = round(psutil.virtual_memory().total / 2**30, 1)
+    except Exception:
+        pass
+    try:
+        usable = len(os.sched_getaffinity(0))
+    except Exception:
+        usable = os.cpu_count()
+    return {"nproc": os.cpu_count(), "usable_cores": usable, "cpu_model": model, "ram_gib": ram}
+
+
+def make_oracle(w: W.Workload, threads: int):
+    """The oracle of the workload.  threads > 1: the same object with its two loops over independent units --
+    nodes in the accumulation, (node, layer) pairs in the selection -- handed to a thread pool.  Every unit
+    calls the same oracle function on the same slices as the sequential loop does (ctypes releases the
+    interpreter lock during the call); no arithmetic changes, results are identical."""
+    from oracle import OracleLGC
+    import oracle as O
+    import numpy as np
+    params = w.init_params().numpy()
+    kw = dict(density_ppm=w.density_ppm, momentum=w.momentum, variant=w.variant, ae_kind=w.ae_kind, c1=w.ae_c1,
+              c2=w.ae_c2, params=params, innovation_permille=w.innovation_permille)
+    if threads <= 1:
+        return OracleLGC(w.table.numel, w.num_nodes, **kw), None
+    from concurrent.futures import ThreadPoolExecutor
+    pool = ThreadPoolExecutor(max_workers=threads)
+
+    class PooledOracle(OracleLGC):
+        def accumulate(self, g):
+            assert g.shape == (self.K, self.N) and g.dtype == np.float32
+            # a node's row is cut into pieces so that all cores have work when K is small
+            pieces = max(1, (threads + self.K - 1) // self.K)
+            edges = np.linspace(0, self.N, pieces + 1).astype(np.int64)
+            jobs = [(k, int(a), int(b)) for k in range(self.K) for a, b in zip(edges[:-1], edges[1:]) if b > a]
+            list(pool.map(lambda j: O.accumulate(self.u[j[0], j[1]:j[2]], self.v[j[0], j[1]:j[2]],
+                                                 np.ascontiguousarray(g[j[0], j[1]:j[2]]), float(self.m)), jobs))
+
+        def _select(self, k):
+            out = np.empty(self.mu, dtype=np.int32)
+
+            def one(l):
+                a, b = int(self.off[l]), int(self.off[l + 1])
+                out[self.koff[l]:self.koff[l + 1]] = O.topk(self.v[k, a:b], self.k_l[l], base=a, method=self.topk_method)
+            list(pool.map(one, range(self.L)))
+            return out
+
+        def topk(self, leader=0):
+            if self.variant == "rar":
+                self.idx = np.broadcast_to(self._select(leader), (self.K, self.mu)).copy()
+            else:
+                self.idx = np.stack(list(pool.map(self._select_serial, range(self.K))))
+            self.val = np.stack([O.gather(self.v[k], self.idx[k]) for k in range(self.K)])
+
+        def _select_serial(self, k):
+            return OracleLGC._select(self, k)
+
+    return PooledOracle(w.table.numel, w.num_nodes, **kw), pool
+
+
+def oracle_throughput(w: W.Workload, sample_steps: int, host_grads=None, threads: int = 1):
     """The oracle, as it stands, on `sample_steps` whole steps of the workload (host cores).
     `host_grads`: gradient batches (numpy [K][N]) to cycle through; generated on the CPU if absent."""
-    from oracle import OracleLGC
-    params = w.init_params().numpy()
     if host_grads is None:
         src = W.GradientSource(w.table, w.num_nodes, seed=w.seed)
         host_grads = [src.step(t).numpy() for t in range(min(GRAD_SETS, sample_steps))]
-    ora = OracleLGC(w.table.numel, w.num_nodes, density_ppm=w.density_ppm, momentum=w.momentum, variant=w.variant,
-                    ae_kind=w.ae_kind, c1=w.ae_c1, c2=w.ae_c2, params=params,
-                    innovation_permille=w.innovation_permille)
+    ora, pool = make_oracle(w, threads)
     times = []
     for t in range(sample_steps):
         g = host_grads[t % len(host_grads)]
         t0 = time.perf_counter()
         ora.step(g, W.choice_for_step(w.seed, t, w.num_nodes))
         times.append(time.perf_counter() - t0)
+    if pool is not None:
+        pool.shutdown()
     bytes_per_step = w.num_nodes * w.table.total * 4
     return bytes_per_step / 1e9 / statistics.mean(times), times
+
+
+def cpu_baseline_record(w: W.Workload, sample_steps: int, host_grads=None):
+    """The reported CPU baseline: the oracle single-threaded (the figure `value` carries) and once more with
+    its independent units on all usable cores."""
+    host = host_description()
+    gbs1, t1 = oracle_throughput(w, sample_steps, host_grads, threads=1)
+    cores = int(host["usable_cores"] or 1)
+    rec = {"value": gbs1, "unit": UNIT, "cores": 1, "kind": "oracle",
+           "sample": f"{len(t1)} whole steps of {w.name} (K={w.num_nodes}, N={w.table.total}), single thread",
+           "s_per_step": statistics.mean(t1), "host": host}
+    if cores > 1:
+        gbsn, tn = oracle_throughput(w, sample_steps, host_grads, threads=cores)
+        rec["all_cores"] = {"value": gbsn, "unit": UNIT, "cores": cores, "s_per_step": statistics.mean(tn),
+                            "sample": f"{len(tn)} whole steps; nodes (accumulation) and (node, layer) pairs "
+                                      f"(selection) on a pool of {cores} threads, same oracle functions"}
+    return rec
 
 
 def run_reference(args, w: W.Workload):
@@ -187,7 +295,8 @@ def run_reference(args, w: W.Workload):
     timed = times[args.warmup:] or times
     value = w.num_nodes * w.table.total * 4 / 1e9 / statistics.mean(timed)
     base = {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"{len(timed)} whole steps of {w.name} (K={w.num_nodes}, N={w.table.total}), single thread"}
+            "sample": f"{len(timed)} whole steps of {w.name} (K={w.num_nodes}, N={w.table.total}), single thread",
+            "host": host_description()}
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": len(timed),
         "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(timed), "higher_is_better": True,
@@ -271,9 +380,25 @@ def run_ours(args, w: W.Workload):
     stop.record()
     gpu_launches = lgc.kernel_launches() - launches_before
     barrier()
-    clocks = sampler.stop()
-    gpu.check()
     elapsed_ms = start.elapsed_time(stop)
+    # A timed region of a few milliseconds is over before the sampler has read the clocks twice.  The same
+    # steps therefore keep running, untimed, under the sampler until it has watched CLOCK_WINDOW_MS of this
+    # load in all: the clocks reported are those of the timed steps and of their continuation.
+    clock_window_ms = elapsed_ms
+    t = args.steps
+    while clock_window_ms < CLOCK_WINDOW_MS:
+        n = max(1, int((CLOCK_WINDOW_MS - clock_window_ms) / max(elapsed_ms / args.steps, 1e-3)) + 1)
+        for _ in range(n):
+            i = args.warmup + t
+            ch = W.choice_for_step(w.seed, i, K)
+            gpu.step(grads[i % GRAD_SETS], update, ch)
+            t += 1
+        torch.cuda.synchronize(dev)
+        clock_window_ms += n * elapsed_ms / args.steps
+    extra_steps = t - args.steps
+    clocks = sampler.stop()
+    clocks["window"] = f"{args.steps} timed steps + {extra_steps} more of the same steps, about {clock_window_ms:.0f} ms under load"
+    gpu.check()
     acc_ms = [a.elapsed_time(b) for a, b in ev]
     # every step's own time: from its first event to the next step's (the last one: to the closing event)
     step_ms = [ev[t][0].elapsed_time(ev[t + 1][0] if t + 1 < args.steps else stop) for t in range(args.steps)]
@@ -285,7 +410,7 @@ def run_ours(args, w: W.Workload):
         names = ("accumulate", "topk", "encode", "combine", "decode_scatter")
         marks = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(min(args.steps, 50))]
         for t, m in enumerate(marks):
-            i = args.warmup + args.steps + t
+            i = args.warmup + args.steps + extra_steps + t
             ch = W.choice_for_step(w.seed, i, K)
             m[0].record(); gpu.accumulate(grads[i % GRAD_SETS], ch)
             m[1].record(); gpu.topk(ch, update)
@@ -331,7 +456,7 @@ def run_ours(args, w: W.Workload):
             "dtype": "f32", "data": "synthetic", "config": workload_config(w),
             "roofline": {"bound": "hbm", "kernel": "accumulate_select_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                         "traffic": None if NCU_DRAM_BYTES_PER_ELEMENT is None else NCU_DRAM_BYTES_PER_ELEMENT * K * N,
+                         "traffic": ncu_traffic_bytes(K * N),
                          "algorithmic_bytes_per_launch": acc_bytes,
                          "kernel_ms": acc_mean_ms},
             "step_hbm": {"algorithmic_bytes": step_bytes, "achieved_GBps": step_gbs,
@@ -345,11 +470,7 @@ def run_ours(args, w: W.Workload):
         if stages_us is not None:
             out["stages_us"] = stages_us        # medians, this rank
         if world == 1 and not args.no_cpu_baseline:
-            gbs, times = oracle_throughput(w, args.cpu_sample_steps, [g.cpu().numpy() for g in grads])
-            out["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                   "sample": f"{len(times)} whole steps of the same workload, single thread "
-                                             f"({os.cpu_count()} host cores present)",
-                                   "s_per_step": statistics.mean(times)}
+            out["cpu_baseline"] = cpu_baseline_record(w, args.cpu_sample_steps, [g.cpu().numpy() for g in grads])
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -362,7 +483,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=list(W.WORKLOAD_NAMES))
-    ap.add_argument("--cpu-sample-steps", type=int, default=16)
+    ap.add_argument("--cpu-sample-steps", type=int, default=12)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--nodes", type=int, default=0, help="override K (profiling aid: a smaller device footprint)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling aid)")

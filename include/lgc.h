@@ -69,6 +69,18 @@ typedef enum { LGC_VARIANT_RAR = 0, LGC_VARIANT_PS = 1 } lgc_variant;
  * code[K][L4][4].  Training: lgc_ae_train_step (ring-allreduce), lgc_ae_train_step_ps (parameter server). */
 typedef enum { LGC_AE_CONV2 = 0, LGC_AE_IDENTITY = 1, LGC_AE_CONV5 = 2 } lgc_ae_kind;
 
+/* Treatment of a layer (Section VI-A, "Experimental Setup": the first layer's gradient is sent as it is, the
+ * last layer's top-magnitude values are sent without the autoencoder, the layers in between go through
+ * top-k selection and the autoencoder).
+ *   TOPK_AE   : accumulated, selected, and the kept values are part of the autoencoder's input.  The kept
+ *               values of ALL such layers, in layer order, form the one vector g~_k in R^mu that is encoded.
+ *   TOPK_ONLY : accumulated and selected like the others; the kept values bypass the autoencoder: the update
+ *               gets their mean over the nodes at the leader's indices (ring-allreduce), or, parameter server,
+ *               the node-ordered sum over the nodes that kept an index of value / K.  Sent entries leave u and v.
+ *   DENSE     : no state and no selection: update = (((g_0 + g_1) + ...) + g_{K-1}) / K for every element of
+ *               the layer, taken from the gradients of this step's lgc_accumulate when the scatter call runs. */
+typedef enum { LGC_LAYER_TOPK_AE = 0, LGC_LAYER_TOPK_ONLY = 1, LGC_LAYER_DENSE = 2 } lgc_layer_mode;
+
 /*
  * Problem description (Section V: K nodes, L layers, layer l has n_l elements).
  */
@@ -92,6 +104,11 @@ typedef struct {
                                      work on a run of layers inside a longer flat gradient (Section VI-A: the first
                                      layer is sent dense and the last one without the autoencoder, so a model is
                                      served by one context per run of layers that are treated alike) */
+    const uint8_t *layer_mode;    /* host array [L] of lgc_layer_mode, or NULL = every layer TOPK_AE; copied by
+                                     lgc_init.  At least one layer must be TOPK_AE.  With DENSE layers the
+                                     `grads` buffer of lgc_accumulate must stay valid and unchanged until this
+                                     step's lgc_decode_scatter / lgc_topk_scatter has run on the stream (their
+                                     elements are read then); k_l of a DENSE layer is 0 */
 } lgc_config;
 
 /* Sizes the caller must provide, in bytes.
@@ -192,6 +209,14 @@ lgc_status lgc_ae_train_step_ps(lgc_ctx *ctx, int32_t common_node, float lambda_
 lgc_status lgc_dense_mean(const float *grads, int64_t row_stride, int32_t num_nodes, int64_t n, float *update,
                           void *stream);
 
+/* Gives the current step up: whatever stage the context is in, the next call may be lgc_accumulate (or
+ * lgc_step_host) again.  Nothing is enqueued and nothing is undone: if lgc_accumulate has run, u and v
+ * hold this step's gradient and no entry of it has been sent or cleared, which is the state
+ * Algorithm 1/2 has after a step that transmitted nothing (the gradient stays in the residual).
+ * For callers that must drop a step after a failed stage or a change of plan.  lgc_step_host does the
+ * same by itself when one of its stages fails. */
+lgc_status lgc_abort_step(lgc_ctx *ctx);
+
 /* Entropy coding of an index list (Section V-A: the transferred indices are DEFLATE-coded and
  * their rate counts in the compression ratio).  The ascending offsets of every layer become gaps
  * (the first counted from the layer's start, the others from the previous offset + 1), each gap
@@ -215,7 +240,9 @@ lgc_status lgc_encode_innovation_positions(lgc_ctx *ctx, int32_t node, void *str
 /* A whole compression step from host memory: uploads `host_grads` ([K][N], ideally pinned) to
  * `dev_grads`, runs the five stages, downloads the dense update to `host_update` ([N]).
  * The call returns without waiting; when the context's stream has drained, `host_update` is
- * complete.  `choice` is the leader (ring-allreduce) or the common node (parameter server).
+ * complete.  `choice` is the leader (ring-allreduce) or the common node (parameter server), 0 .. K-1
+ * for both variants.  All arguments are checked before anything is copied or enqueued: a refused call
+ * leaves u, v and the context as they were.
  * The upload goes node by node over a stream of the library's own (created at the first call,
  * released by lgc_destroy), and each node's row is accumulated as soon as it has arrived, so
  * stage 1 hides under the transfer; the download stays on the context's stream.  The upload of
@@ -254,6 +281,13 @@ lgc_status lgc_step_host(lgc_ctx *ctx, const float *host_grads, float *dev_grads
 #define LGC_NOALLOC_MAX_N 16777216
 lgc_status lgc_topk_noalloc(const float *v, int64_t n, int64_t k, int32_t *idx_out, void *stream);
 
+/* The consistency checks of lgc_topk_noalloc's kernels (counts that must add up to k) are recorded
+ * in a word of the built-in array, not in a context: lgc_check never reports them, this call does.
+ * It waits for `stream`, reads the word of the current device (a four-byte copy to the host, no
+ * allocation), returns LGC_OK or LGC_ERR_DEVICE_CHECK (text through lgc_last_error(NULL)) and clears
+ * the record.  (No counterpart in the paper either.) */
+lgc_status lgc_topk_noalloc_check(void *stream);
+
 /* ---- inspection --------------------------------------------------------------------------- */
 
 /* N, mu, encoder lengths L1 (after the first convolution) and L2 (code length per channel), and
@@ -261,11 +295,19 @@ lgc_status lgc_topk_noalloc(const float *v, int64_t n, int64_t k, int32_t *idx_o
 lgc_status lgc_get_layout(const lgc_ctx *ctx, int64_t *N, int64_t *mu, int64_t *L1, int64_t *L2,
                           int64_t *param_count);
 
-/* Host array [L] of k_l, owned by the context. */
+/* Host array [L] of k_l, owned by the context (0 for DENSE layers). */
 const int64_t *lgc_keep_counts(const lgc_ctx *ctx);
 
+/* Where the kept entries of each layer sit inside a row of `idx`.  A row has mu_all slots: first the mu
+ * slots of the TOPK_AE layers, in layer order (these are the autoencoder's input, and what lgc_get_layout
+ * reports as mu), then the slots of the TOPK_ONLY layers, in layer order.  Without a layer_mode array
+ * mu_all = mu and the slots follow the layers.  first_slot: host array [L] owned by the context, -1 for DENSE
+ * layers.  val_topk_only: device, fp32 [K][mu_all - mu], the kept values of the TOPK_ONLY layers (filled by
+ * lgc_topk for the parameter server and by lgc_topk_scatter; NULL when there are none).  Any pointer may be NULL. */
+lgc_status lgc_get_slots(const lgc_ctx *ctx, int64_t *mu_all, const int64_t **first_slot, float **val_topk_only);
+
 /* Device pointers into the caller's buffers (any may be NULL):
- *   u, v    [K][N]                     idx   [S][mu] int32, S = 1 (ring-allreduce) or K
+ *   u, v    [K][N]                     idx   [S][mu_all] int32 (see lgc_get_slots), S = 1 (ring-allreduce) or K
  *   val     [K][mu] (filled by lgc_topk for the parameter server and the identity autoencoder,
  *           else by lgc_encode / lgc_ae_train_step / lgc_topk_scatter)
  *   code    [K][c2][L2] (identity: [K][mu])

@@ -49,16 +49,31 @@ accumulate_kernel(const float4 *__restrict__ g4, float4 *__restrict__ u4, float4
 
 // The same for gradient rows that are not back to back (row k of g starts at g + k * g_stride):
 // grid (tiles of 4096 elements, K); 128-bit accesses where the addresses allow, scalars otherwise.
+__device__ __forceinline__ bool in_dense_run(const int64_t *__restrict__ rng, int n, int64_t pos)
+{
+    int lo = 0, hi = n;                         // first run whose end lies beyond pos
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (rng[2 * mid + 1] <= pos) lo = mid + 1;
+        else hi = mid;
+    }
+    return lo < n && rng[2 * lo] <= pos;
+}
+
 __global__ void __launch_bounds__(kAccThreads)
 accumulate_rows_kernel(const float *__restrict__ g, int64_t g_stride, float *__restrict__ u, float *__restrict__ v,
-                       int64_t N, float m)
+                       int64_t N, float m, const int64_t *__restrict__ dense_rng, int num_dense)
 {
     const int row = blockIdx.y;
     const int64_t p0 = ((int64_t)blockIdx.x * kAccThreads + threadIdx.x) * 4;
     if (p0 >= N) return;
     const float *gp = g + (int64_t)row * g_stride + p0;
     float *up = u + (int64_t)row * N + p0, *vp = v + (int64_t)row * N + p0;
-    if (p0 + 4 <= N && ((reinterpret_cast<uintptr_t>(gp) | reinterpret_cast<uintptr_t>(up) | reinterpret_cast<uintptr_t>(vp)) & 15) == 0) {
+    bool any_dense = false;
+    if (num_dense)
+        for (int i = 0; i < 4; ++i) any_dense = any_dense || in_dense_run(dense_rng, num_dense, p0 + i);
+    if (!any_dense && p0 + 4 <= N &&
+        ((reinterpret_cast<uintptr_t>(gp) | reinterpret_cast<uintptr_t>(up) | reinterpret_cast<uintptr_t>(vp)) & 15) == 0) {
         const float4 gg = __ldcs(reinterpret_cast<const float4 *>(gp));
         float4 uu = __ldcs(reinterpret_cast<float4 *>(up)), vv = __ldcs(reinterpret_cast<float4 *>(vp));
         acc4(uu, vv, gg, m);
@@ -66,6 +81,7 @@ accumulate_rows_kernel(const float *__restrict__ g, int64_t g_stride, float *__r
         __stcs(reinterpret_cast<float4 *>(vp), vv);
     } else {
         for (int i = 0; i < 4 && p0 + i < N; ++i) {
+            if (any_dense && in_dense_run(dense_rng, num_dense, p0 + i)) continue;   // dense layers keep no state (u, v stay 0)
             const float x = __fmaf_rn(m, up[i], gp[i]);
             up[i] = x;
             vp[i] = __fadd_rn(vp[i], x);
@@ -109,26 +125,28 @@ __global__ void zero_tail_kernel(unsigned char *p, unsigned n)
     if (threadIdx.x < n) p[threadIdx.x] = 0;
 }
 
-int sm_count()
-{
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-            sms = 148;
-    }
-    return sms;
-}
-
 }  // namespace
 
+int sm_count()
+{
+    static std::mutex mu;
+    static int sms[kMaxDevices] = {};
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    const bool cached = dev >= 0 && dev < kMaxDevices;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached && sms[dev] > 0) return sms[dev];
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    if (cached) sms[dev] = n;
+    return n;
+}
+
 cudaError_t launch_accumulate_rows(const float *g, int64_t g_stride, float *u, float *v, int K, int64_t N, float m,
-                                   cudaStream_t s)
+                                   const int64_t *dense_rng, int num_dense, cudaStream_t s)
 {
     if (K <= 0 || N <= 0) return cudaSuccess;
     const unsigned tiles = (unsigned)((N + 4 * kAccThreads - 1) / (4 * kAccThreads));
-    accumulate_rows_kernel<<<dim3(tiles, K), kAccThreads, 0, s>>>(g, g_stride, u, v, N, m), ++g_kernel_launches;
+    accumulate_rows_kernel<<<dim3(tiles, K), kAccThreads, 0, s>>>(g, g_stride, u, v, N, m, dense_rng, num_dense), ++g_kernel_launches;
     return cudaGetLastError();
 }
 

@@ -599,11 +599,11 @@ cudaError_t launch_gemm(Ctx &c, const CUtensorMap &a_hi, const CUtensorMap &a_lo
 {
     using S = GemmShape<MODE, CIN, COUT>;
     auto kern = ae5_gemm_kernel<MODE, CIN, COUT>;
-    static bool configured = false;
-    if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kSmemBytes);
+    static OncePerDevice configured;            // one per instantiation of this template
+    {
+        const cudaError_t e = configured.run(
+            [&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kSmemBytes); });
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     kern<<<dim3(blocks(rows, kTileM), nodes), 128, S::kSmemBytes, c.stream>>>(a_hi, a_lo, b_hi, b_lo, bias, L_out, Lpad_out, out_hi,
                                                                               out_lo, w_last, b_last, out_last, extra, c.errword),
@@ -821,7 +821,7 @@ cudaError_t launch_ae5_encode(Ctx &c)
     Ae5 &a = *c.ae5;
     const float *P = c.params;
     prepare_weights(c);
-    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu, c.mu, a.len[1], a.lpad[0],
+    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu_all, c.mu, a.len[1], a.lpad[0],
                                                                             P + a.off_w[0], P + a.off_b[0], c.val, a.act_hi[0],
                                                                             a.act_lo[0]),
         ++g_kernel_launches;
@@ -871,7 +871,7 @@ cudaError_t launch_ae5_train_encode(Ctx &c)
     Ae5 &a = *c.ae5;
     const float *P = c.params;
     prepare_weights(c);
-    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu, c.mu, a.len[1], a.lpad[0],
+    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu_all, c.mu, a.len[1], a.lpad[0],
                                                                             P + a.off_w[0], P + a.off_b[0], c.val, a.act_hi[0],
                                                                             a.act_lo[0]),
         ++g_kernel_launches;

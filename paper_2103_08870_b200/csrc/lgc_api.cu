@@ -35,11 +35,23 @@ struct Carver {
     }
 };
 
+// Layers are treated per mode (Section VI-A).  Kept entries live in SLOTS: a row of `idx` holds the
+// slots of the layers that go through the autoencoder first (layer order), then those of the top-k-only
+// layers (layer order), so that the autoencoder's input is one contiguous vector of mu values.
+// "Slot order" below means this order of the selecting layers.
 struct Plan {
     int K, L, S;
-    int64_t N, mu, muI, L1, L2, P, Penc, Pdec, code_len;
+    int L_ae, L_sel;                       // layers through the autoencoder / layers that select at all
+    int64_t N, mu, mu_t, mu_all, muI, L1, L2, P, Penc, Pdec, code_len;   // mu: autoencoder layers' slots, mu_t: top-k-only
     int op1, op2;
-    std::vector<int64_t> numel, off, k_l, koff, ki_l, kioff;
+    bool mixed;                            // some layer is not LGC_LAYER_TOPK_AE
+    std::vector<uint8_t> mode;             // [L]
+    std::vector<int> slot_layers;          // [L_sel] layers in slot order
+    std::vector<int64_t> numel, off;       // [L], [L + 1]
+    std::vector<int64_t> k_l, kslot;       // [L] kept entries (0: dense) and first slot (-1: dense) of every layer
+    std::vector<int64_t> koff;             // [L_sel + 1] first slot of each selecting layer, slot order
+    std::vector<int64_t> ki_l, kioff;      // [L_ae], [L_ae + 1] innovation counts / slots of the autoencoder layers
+    std::vector<int64_t> dense_rng;        // (begin, end) of every maximal run of dense elements, ascending
 };
 
 int64_t pad4(int64_t n) { return (n + 3) / 4 * 4; }   // keeps consecutive fp32 vectors 16-byte aligned
@@ -68,29 +80,59 @@ lgc_status make_plan(const lgc_config *cfg, Plan &p, std::string *why)
     p.L = cfg->num_layers;
     p.S = cfg->variant == LGC_VARIANT_PS ? p.K : 1;
     p.numel.assign(cfg->layer_numel, cfg->layer_numel + p.L);
+    p.mode.assign((size_t)p.L, (uint8_t)LGC_LAYER_TOPK_AE);
+    p.mixed = false;
+    if (cfg->layer_mode)
+        for (int l = 0; l < p.L; ++l) {
+            if (cfg->layer_mode[l] > LGC_LAYER_DENSE) return fail(LGC_ERR_INVALID_ARG, "unknown layer_mode");
+            p.mode[l] = cfg->layer_mode[l];
+            p.mixed = p.mixed || p.mode[l] != LGC_LAYER_TOPK_AE;
+        }
     p.off.assign(p.L + 1, 0);
-    p.koff.assign(p.L + 1, 0);
-    p.kioff.assign(p.L + 1, 0);
-    p.k_l.resize(p.L);
-    p.ki_l.resize(p.L);
+    p.k_l.assign(p.L, 0);
+    p.kslot.assign(p.L, -1);
+    p.dense_rng.clear();
     for (int l = 0; l < p.L; ++l) {
         const int64_t n = p.numel[l];
         if (n < 1) return fail(LGC_ERR_INVALID_ARG, "a layer has fewer than 1 element");
         p.off[l + 1] = p.off[l] + n;
         if (p.off[l + 1] > 2147483647LL) return fail(LGC_ERR_INVALID_ARG, "N exceeds 2^31 - 1");
+        if (p.mode[l] == LGC_LAYER_DENSE) {
+            if (!p.dense_rng.empty() && p.dense_rng.back() == p.off[l]) p.dense_rng.back() = p.off[l + 1];
+            else { p.dense_rng.push_back(p.off[l]); p.dense_rng.push_back(p.off[l + 1]); }
+            continue;
+        }
         int64_t k = (n * (int64_t)cfg->density_ppm + 500000) / 1000000;
-        k = k < 1 ? 1 : (k > n ? n : k);
-        int64_t ki = (k * (int64_t)cfg->innovation_permille + 500) / 1000;
-        ki = ki < 1 ? 1 : (ki > k ? k : ki);
-        p.k_l[l] = k;
-        p.ki_l[l] = ki;
-        p.koff[l + 1] = p.koff[l] + k;
-        p.kioff[l + 1] = p.kioff[l] + ki;
+        p.k_l[l] = k < 1 ? 1 : (k > n ? n : k);
+    }
+    // slot order: the autoencoder's layers, then the top-k-only ones
+    p.slot_layers.clear();
+    for (int l = 0; l < p.L; ++l) if (p.mode[l] == LGC_LAYER_TOPK_AE) p.slot_layers.push_back(l);
+    p.L_ae = (int)p.slot_layers.size();
+    for (int l = 0; l < p.L; ++l) if (p.mode[l] == LGC_LAYER_TOPK_ONLY) p.slot_layers.push_back(l);
+    p.L_sel = (int)p.slot_layers.size();
+    if (p.L_ae == 0)
+        return fail(LGC_ERR_INVALID_ARG, "no layer has LGC_LAYER_TOPK_AE: at least one layer must feed the autoencoder");
+    p.koff.assign(p.L_sel + 1, 0);
+    p.ki_l.assign(p.L_ae, 0);
+    p.kioff.assign(p.L_ae + 1, 0);
+    for (int j = 0; j < p.L_sel; ++j) {
+        const int l = p.slot_layers[j];
+        p.kslot[l] = p.koff[j];
+        p.koff[j + 1] = p.koff[j] + p.k_l[l];
+        if (j < p.L_ae) {
+            int64_t ki = (p.k_l[l] * (int64_t)cfg->innovation_permille + 500) / 1000;
+            ki = ki < 1 ? 1 : (ki > p.k_l[l] ? p.k_l[l] : ki);
+            p.ki_l[j] = ki;
+            p.kioff[j + 1] = p.kioff[j] + ki;
+        }
     }
     p.N = p.off[p.L];
     if (cfg->grad_row_stride != 0 && cfg->grad_row_stride < p.N) return fail(LGC_ERR_INVALID_ARG, "grad_row_stride is smaller than N");
-    p.mu = p.koff[p.L];
-    p.muI = p.kioff[p.L];
+    p.mu = p.koff[p.L_ae];
+    p.mu_all = p.koff[p.L_sel];
+    p.mu_t = p.mu_all - p.mu;
+    p.muI = p.kioff[p.L_ae];
     p.L1 = conv_len(p.mu);
     p.L2 = conv_len(p.L1);
     p.op1 = p.L1 >= 3 ? (int)((p.L1 - 3) % 2) : 0;
@@ -129,8 +171,10 @@ struct SelectPlan {
     int64_t comp_total = 0;
 };
 
+// Segments ascend by offset and may leave gaps (layers that do not select).  row_len: length of a row;
+// dense: (begin, end) pairs of the row's dense runs, ascending (they lie in the gaps).
 SelectPlan plan_select(const std::vector<int64_t> &off, const std::vector<int64_t> &len, const std::vector<int64_t> &k,
-                       const std::vector<int64_t> &out_off)
+                       const std::vector<int64_t> &out_off, int64_t row_len, const std::vector<int64_t> &dense)
 {
     SelectPlan sp;
     const int n = (int)len.size();
@@ -164,23 +208,44 @@ SelectPlan plan_select(const std::vector<int64_t> &off, const std::vector<int64_
     std::stable_sort(sp.large_order.begin(), sp.large_order.end(), [&](int32_t a, int32_t b) {
         return len[sp.large_ids[a]] > len[sp.large_ids[b]];
     });
-    const int64_t row_len = off[n - 1] + len[n - 1];
     sp.tiles_per_row = (int)((row_len + kSelChunk - 1) / kSelChunk);
     int s = 0;
+    size_t d0 = 0;                                                  // first dense run that ends after the tile's start
     for (int q = 0; q < sp.tiles_per_row; ++q) {
         const int64_t t0 = (int64_t)q * kSelChunk, t1 = t0 + kSelChunk < row_len ? t0 + kSelChunk : row_len;
-        while (off[s] + len[s] <= t0) ++s;                          // first segment that reaches into tile q
+        while (s < n && off[s] + len[s] <= t0) ++s;                 // first segment that reaches into tile q or lies behind it
         int4 d = make_int4(s, -2, 0, 0);
-        if (off[s] <= t0 && off[s] + len[s] >= t1 && sp.seg_large[s] >= 0) {
+        if (s < n && off[s] <= t0 && off[s] + len[s] >= t1 && sp.seg_large[s] >= 0) {
             d.y = sp.seg_large[s];                                  // one large segment covers the tile
             d.z = sp.tchunk0[d.y] + (q - sp.large_q0[d.y]);
         } else {
             for (int r = s; r < n && off[r] < t1; ++r)
                 if (sp.seg_large[r] >= 0) d.y = -1;                 // several segments, at least one large
         }
+        while (d0 < dense.size() && dense[d0 + 1] <= t0) d0 += 2;
+        if (d0 < dense.size() && dense[d0] < t1)                    // w: 0 no dense element in the tile, -1 all dense,
+            d.w = dense[d0] <= t0 && dense[d0 + 1] >= t1 ? -1 : (int)(d0 / 2) + 1;   // else 1 + its first dense run
         sp.tile_desc.push_back(d);
     }
     return sp;
+}
+
+// The two selection families of a context: the residual v over the selecting layers (layer order; slots
+// as the plan assigns them), and -- parameter server -- the kept values of the autoencoder layers.
+SelectPlan plan_select_v(const Plan &p)
+{
+    std::vector<int64_t> off, len, k, out;
+    for (int l = 0; l < p.L; ++l)
+        if (p.mode[l] != LGC_LAYER_DENSE) {
+            off.push_back(p.off[l]); len.push_back(p.numel[l]); k.push_back(p.k_l[l]); out.push_back(p.kslot[l]);
+        }
+    return plan_select(off, len, k, out, p.N, p.dense_rng);
+}
+SelectPlan plan_select_inn(const Plan &p)
+{
+    std::vector<int64_t> off(p.koff.begin(), p.koff.begin() + p.L_ae), len, out(p.kioff.begin(), p.kioff.begin() + p.L_ae);
+    for (int j = 0; j < p.L_ae; ++j) len.push_back(p.k_l[p.slot_layers[j]]);
+    return plan_select(off, len, p.ki_l, out, p.mu, {});
 }
 
 void carve_select(Carver &cv, SelectTables &t, const SelectPlan &sp, int rows)
@@ -230,24 +295,33 @@ void carve(Carver &cv, Ctx &c, const Plan &p, const lgc_config &cfg)
     const bool conv = cfg.ae_kind == LGC_AE_CONV2;
     const bool conv5 = cfg.ae_kind == LGC_AE_CONV5;
     c.errword = cv.take<int32_t>(4);
-    c.idx = cv.take<int32_t>((size_t)p.S * p.mu);
+    c.idx = cv.take<int32_t>((size_t)p.S * p.mu_all);
     c.val = cv.take<float>((size_t)p.K * p.mu);
+    c.val_t = p.mu_t ? cv.take<float>((size_t)p.K * p.mu_t) : nullptr;
+    c.num_dense = (int)(p.dense_rng.size() / 2);
+    c.num_dense_chunks = 0;
+    for (size_t r = 0; r < p.dense_rng.size(); r += 2)
+        c.num_dense_chunks += (p.dense_rng[r + 1] - p.dense_rng[r] + kDenseChunk - 1) / kDenseChunk;
+    c.dense_rng = c.num_dense ? cv.take<int64_t>(p.dense_rng.size()) : nullptr;
+    c.dense_chunks = c.num_dense ? cv.take<int64_t>((size_t)2 * c.num_dense_chunks) : nullptr;
     c.code = conv || conv5 ? cv.take<float>((size_t)p.K * p.code_len) : nullptr;
     c.combined = cv.take<float>((size_t)p.code_len);
     c.recon = cv.take<float>((size_t)p.S * p.mu);
-    c.slot_layer = cv.take<int32_t>((size_t)p.mu);
+    c.slot_layer = cv.take<int32_t>((size_t)p.mu_all);
     c.koff_dev = cv.take<int32_t>((size_t)p.L + 1);
     c.layer_off_dev = cv.take<int64_t>((size_t)p.L);
-    c.ic_bytes = cv.take<unsigned char>((size_t)5 * p.mu);
+    c.ic_bytes = cv.take<unsigned char>((size_t)5 * p.mu_all);
     c.tile_lo = cv.take<int32_t>((size_t)((p.N + 4095) / 4096) + 1);
-    carve_select(cv, c.sel_v, plan_select(p.off, p.numel, p.k_l, p.koff), p.S);
+    carve_select(cv, c.sel_v, plan_select_v(p), p.S);
+    c.sel_v.dense_rng = c.dense_rng;
+    c.sel_v.num_dense = c.num_dense;
     if (ps) {
         c.inn = cv.take<float>((size_t)p.K * p.mu);
         c.inn_pos = cv.take<int32_t>((size_t)p.K * p.muI);
         c.inn_slot_layer = cv.take<int32_t>((size_t)p.muI);
         c.kioff_dev = cv.take<int32_t>((size_t)p.L + 1);
         c.koff64_dev = cv.take<int64_t>((size_t)p.L);
-        carve_select(cv, c.sel_inn, plan_select(p.koff, p.k_l, p.ki_l, p.kioff), p.K);
+        carve_select(cv, c.sel_inn, plan_select_inn(p), p.K);
     }
     if (conv && ps) {                       // training work space, one slice per node
         const size_t c1 = cfg.ae_c1, c2 = cfg.ae_c2, K = p.K;
@@ -361,10 +435,12 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     if (!c) return LGC_ERR_NO_MEMORY;
     c->cfg = *cfg;
     c->cfg.layer_numel = nullptr;
+    c->cfg.layer_mode = nullptr;
     c->stream = static_cast<cudaStream_t>(cfg->stream);
     c->K = p.K; c->L = p.L; c->S = p.S; c->N = p.N; c->mu = p.mu; c->muI = p.muI; c->L1 = p.L1; c->L2 = p.L2;
+    c->mu_t = p.mu_t; c->mu_all = p.mu_all; c->mixed = p.mixed; c->L_ae = p.L_ae; c->L_sel = p.L_sel;
     c->P = p.P; c->Penc = p.Penc; c->Pdec = p.Pdec; c->op1 = p.op1; c->op2 = p.op2; c->code_len = p.code_len;
-    c->numel = p.numel; c->off = p.off; c->k_l = p.k_l; c->koff = p.koff; c->ki_l = p.ki_l; c->kioff = p.kioff;
+    c->numel = p.numel; c->off = p.off; c->k_l = p.k_l; c->kslot = p.kslot; c->koff = p.koff; c->ki_l = p.ki_l; c->kioff = p.kioff;
     c->lr = cfg->adam_lr != 0.0f ? (double)cfg->adam_lr : 1e-3;
     c->beta1 = cfg->adam_beta1 != 0.0f ? (double)cfg->adam_beta1 : 0.9;
     c->beta2 = cfg->adam_beta2 != 0.0f ? (double)cfg->adam_beta2 : 0.999;
@@ -384,30 +460,40 @@ lgc_status lgc_init(const lgc_config *cfg, void *state, size_t state_bytes, void
     if (e == cudaSuccess && p.P > 0) e = launch_zero(c->adam_m, (size_t)2 * pad4(p.P) * sizeof(float), s);
     std::vector<SelectPlan> hold;
     hold.reserve(2);
-    if (e == cudaSuccess) e = upload_select(c->sel_v, plan_select(p.off, p.numel, p.k_l, p.koff), s, hold);
+    if (e == cudaSuccess) e = upload_select(c->sel_v, plan_select_v(p), s, hold);
     if (e == cudaSuccess && cfg->variant == LGC_VARIANT_PS)
-        e = upload_select(c->sel_inn, plan_select(p.koff, p.k_l, p.ki_l, p.kioff), s, hold);
-    std::vector<int32_t> slot_layer((size_t)p.mu), koff32((size_t)p.L + 1);
-    for (int l = 0; l < p.L; ++l) {
-        koff32[l] = (int32_t)p.koff[l];
-        for (int64_t q = p.koff[l]; q < p.koff[l + 1]; ++q) slot_layer[(size_t)q] = l;
+        e = upload_select(c->sel_inn, plan_select_inn(p), s, hold);
+    // tables in slot order (the autoencoder's layers first): layer of every slot, first slot and first element of every layer
+    std::vector<int32_t> slot_layer((size_t)p.mu_all), koff32((size_t)p.L_sel + 1);
+    std::vector<int64_t> layer_off((size_t)p.L_sel);
+    for (int j = 0; j < p.L_sel; ++j) {
+        koff32[j] = (int32_t)p.koff[j];
+        layer_off[j] = p.off[p.slot_layers[j]];
+        for (int64_t q = p.koff[j]; q < p.koff[j + 1]; ++q) slot_layer[(size_t)q] = j;
     }
-    koff32[p.L] = (int32_t)p.mu;
+    koff32[p.L_sel] = (int32_t)p.mu_all;
     if (e == cudaSuccess) e = upload(c->slot_layer, slot_layer, s);
     if (e == cudaSuccess) e = upload(c->koff_dev, koff32, s);
-    std::vector<int64_t> layer_off(p.off.begin(), p.off.begin() + p.L);
     if (e == cudaSuccess) e = upload(c->layer_off_dev, layer_off, s);
+    std::vector<int64_t> dense_chunks;
+    for (size_t r = 0; r < p.dense_rng.size(); r += 2)
+        for (int64_t a = p.dense_rng[r]; a < p.dense_rng[r + 1]; a += kDenseChunk) {
+            dense_chunks.push_back(a);
+            dense_chunks.push_back(std::min<int64_t>(a + kDenseChunk, p.dense_rng[r + 1]));
+        }
+    if (e == cudaSuccess) e = upload(c->dense_rng, p.dense_rng, s);
+    if (e == cudaSuccess) e = upload(c->dense_chunks, dense_chunks, s);
     std::vector<int32_t> inn_slot_layer, kioff32;
     std::vector<int64_t> koff64;
     if (cfg->variant == LGC_VARIANT_PS) {
         inn_slot_layer.resize((size_t)p.muI);
-        kioff32.resize((size_t)p.L + 1);
-        koff64.assign(p.koff.begin(), p.koff.begin() + p.L);
-        for (int l = 0; l < p.L; ++l) {
-            kioff32[l] = (int32_t)p.kioff[l];
-            for (int64_t q = p.kioff[l]; q < p.kioff[l + 1]; ++q) inn_slot_layer[(size_t)q] = l;
+        kioff32.resize((size_t)p.L_ae + 1);
+        koff64.assign(p.koff.begin(), p.koff.begin() + p.L_ae);
+        for (int j = 0; j < p.L_ae; ++j) {
+            kioff32[j] = (int32_t)p.kioff[j];
+            for (int64_t q = p.kioff[j]; q < p.kioff[j + 1]; ++q) inn_slot_layer[(size_t)q] = j;
         }
-        kioff32[p.L] = (int32_t)p.muI;
+        kioff32[p.L_ae] = (int32_t)p.muI;
         if (e == cudaSuccess) e = upload(c->inn_slot_layer, inn_slot_layer, s);
         if (e == cudaSuccess) e = upload(c->kioff_dev, kioff32, s);
         if (e == cudaSuccess) e = upload(c->koff64_dev, koff64, s);
@@ -468,9 +554,12 @@ cudaError_t accumulate_nodes(lgc_ctx *c, const float *grads, int32_t leader_hint
     if (fused)   // the kernel's row y is node r0 + y; node n selects into table row n (parameter server) or 0 (the leader)
         return launch_accumulate_select(c->sel_v, g, gs, u, v, r1 - r0, c->N, c->cfg.momentum, (ps ? 0 : leader_hint) - r0,
                                         ps ? c->K : 1, c->epoch, c->errword, c->stream);
-    if (gs == c->N && r0 == 0 && r1 == c->K)
+    if (c->num_dense && c->N % 4 == 0 && gs % 4 == 0)      // the tile kernel, nobody selecting: it skips the dense layers
+        return launch_accumulate_select(c->sel_v, g, gs, u, v, r1 - r0, c->N, c->cfg.momentum, 0, 0, c->epoch, c->errword,
+                                        c->stream);
+    if (gs == c->N && r0 == 0 && r1 == c->K && !c->num_dense)
         return launch_accumulate(g, u, v, (uint64_t)c->K * (uint64_t)c->N, c->cfg.momentum, c->stream);
-    return launch_accumulate_rows(g, gs, u, v, r1 - r0, c->N, c->cfg.momentum, c->stream);
+    return launch_accumulate_rows(g, gs, u, v, r1 - r0, c->N, c->cfg.momentum, c->dense_rng, c->num_dense, c->stream);
 }
 
 }  // namespace
@@ -483,6 +572,7 @@ lgc_status lgc_accumulate(lgc_ctx *c, const float *grads, int32_t leader_hint)
     if (st != LGC_OK) return st;
     const cudaError_t e = accumulate_nodes(c, grads, leader_hint, fused, 0, c->K);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_accumulate");
+    c->step_grads = grads;
     c->tail_recorded = false;      // a later lgc_step_host orders its upload behind this step
     c->stage = Ctx::kAccumulated;
     return LGC_OK;
@@ -504,7 +594,7 @@ lgc_status lgc_topk(lgc_ctx *c, int32_t leader, float *update_hint)
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->side_join, cudaEventDisableTiming);
         if (e != cudaSuccess) return cuda_fail(c, e, "lgc_topk (side stream)");
     }
-    e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu, served, c->epoch, update_hint, c->N,
+    e = launch_select(c->sel_v, c->v, c->N, ps ? 0 : leader, c->S, c->idx, c->mu_all, served, c->epoch, update_hint, c->N,
                       c->errword, c->stream, c->side_stream, c->side_fork, c->side_join);
     c->cleared_update = c->sel_v.num_large ? update_hint : nullptr;
     if (c->selections < 2) ++c->selections;
@@ -564,6 +654,16 @@ lgc_status lgc_topk_scatter(lgc_ctx *c, float *update)
     const cudaError_t e = launch_topk_scatter(*c, update);
     if (e != cudaSuccess) return cuda_fail(c, e, "lgc_topk_scatter");
     c->stage = Ctx::kIdle;
+    return LGC_OK;
+}
+
+lgc_status lgc_abort_step(lgc_ctx *c)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    c->stage = Ctx::kIdle;
+    c->cleared_update = nullptr;
+    c->fused_leader = -2;
+    c->val_valid = c->mean_valid = c->tile_lo_valid = false;
     return LGC_OK;
 }
 
@@ -648,6 +748,9 @@ lgc_status lgc_step_host(lgc_ctx *c, const float *host_grads, float *dev_grads, 
 {
     if (!c) return LGC_ERR_INVALID_ARG;
     if (!host_grads || !dev_grads || !dev_update || !host_update) return fail(c, LGC_ERR_INVALID_ARG, "NULL buffer");
+    if (!aligned16(dev_grads) || !aligned16(dev_update))
+        return fail(c, LGC_ERR_INVALID_ARG, "dev_grads and dev_update must be 16-byte aligned");
+    if (choice < 0 || choice >= c->K) return fail(c, LGC_ERR_INVALID_ARG, "choice (leader / common node) out of range");
     if (c->stage != Ctx::kIdle) return fail(c, LGC_ERR_BAD_STATE, "lgc_step_host must open a step");
     if (c->cfg.grad_row_stride != 0 && c->cfg.grad_row_stride != c->N)
         return fail(c, LGC_ERR_UNSUPPORTED, "lgc_step_host copies rows that are back to back: grad_row_stride must be 0 or N");
@@ -682,14 +785,23 @@ lgc_status lgc_step_host(lgc_ctx *c, const float *host_grads, float *dev_grads, 
             if (e == cudaSuccess) e = by_rows ? accumulate_nodes(c, dev_grads, choice, fused, k, k + 1)
                                               : accumulate_nodes(c, dev_grads, choice, fused, 0, c->K);
         }
-        if (e != cudaSuccess) return cuda_fail(c, e, "lgc_step_host (upload)");
+        if (e != cudaSuccess) {
+            c->stage = Ctx::kIdle;
+            return cuda_fail(c, e, "lgc_step_host (upload)");
+        }
     }
     c->stage = Ctx::kAccumulated;
+    c->step_grads = dev_grads;
     st = lgc_topk(c, choice, dev_update);
     if (st == LGC_OK) st = lgc_encode(c);
     if (st == LGC_OK) st = lgc_combine(c, choice);
     if (st == LGC_OK) st = lgc_decode_scatter(c, dev_update);
-    if (st != LGC_OK) return st;
+    if (st != LGC_OK) {
+        // a stage refused or failed (the arguments were checked above, so this is a CUDA error): the
+        // step is given up, so that the context accepts a new one; the message of the stage stays
+        c->stage = Ctx::kIdle;
+        return st;
+    }
     e = cudaEventRecord(c->tail_done, c->stream);
     c->tail_recorded = e == cudaSuccess;
     if (e == cudaSuccess)
@@ -710,6 +822,15 @@ lgc_status lgc_get_layout(const lgc_ctx *c, int64_t *N, int64_t *mu, int64_t *L1
 }
 
 const int64_t *lgc_keep_counts(const lgc_ctx *c) { return c ? c->k_l.data() : nullptr; }
+
+lgc_status lgc_get_slots(const lgc_ctx *c, int64_t *mu_all, const int64_t **first_slot, float **val_topk_only)
+{
+    if (!c) return LGC_ERR_INVALID_ARG;
+    if (mu_all) *mu_all = c->mu_all;
+    if (first_slot) *first_slot = c->kslot.data();
+    if (val_topk_only) *val_topk_only = c->val_t;
+    return LGC_OK;
+}
 
 lgc_status lgc_get_buffers(const lgc_ctx *c, float **u, float **v, int32_t **idx, float **val, float **code,
                            float **combined, float **inn, float **recon)

@@ -15,14 +15,38 @@ namespace {
 
 constexpr int kAeThreads = 128;
 
+// Kept values of every node: slots below mu (the autoencoder's layers) go to val, the others (top-k-only
+// layers) to val_t.  A row of idx holds mu_all slots.
 __global__ void gather_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restrict__ idx,
-                              int S, int64_t mu, float *__restrict__ val)
+                              int S, int64_t mu, int64_t mu_all, float *__restrict__ val, float *__restrict__ val_t)
 {
     const int k = blockIdx.y;
     const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= mu) return;
-    const int32_t i = idx[(S == 1 ? 0 : (int64_t)k * mu) + p];
-    val[(int64_t)k * mu + p] = v[(int64_t)k * N + i];
+    if (p >= mu_all) return;
+    const int32_t i = idx[(S == 1 ? 0 : (int64_t)k * mu_all) + p];
+    const float x = v[(int64_t)k * N + i];
+    if (p < mu) val[(int64_t)k * mu + p] = x;
+    else val_t[(int64_t)k * (mu_all - mu) + (p - mu)] = x;
+}
+
+// Layers sent as they are (Section VI-A: the first layer): update[j] = (((g_0[j] + g_1[j]) + ...) + g_{K-1}[j]) / K
+// for the elements of one piece [begin, end) of a dense run; pieces hold at most kDenseChunk elements.
+__device__ __forceinline__ void dense_piece(const int64_t *__restrict__ pieces, int64_t piece, const float *__restrict__ g,
+                                            int64_t g_stride, int K, float *__restrict__ update)
+{
+    const int64_t a = pieces[2 * piece], b = pieces[2 * piece + 1];
+    const float fk = (float)K;
+    for (int64_t j = a + threadIdx.x; j < b; j += blockDim.x) {
+        float acc = __ldcs(g + j);
+        for (int k = 1; k < K; ++k) acc = __fadd_rn(acc, __ldcs(g + (int64_t)k * g_stride + j));
+        update[j] = __fdiv_rn(acc, fk);
+    }
+}
+
+__global__ void dense_pieces_kernel(const int64_t *__restrict__ pieces, const float *__restrict__ g, int64_t g_stride, int K,
+                                    float *__restrict__ update)
+{
+    dense_piece(pieces, blockIdx.x, g, g_stride, K, update);
 }
 
 // code[k][co][t] = b2[co] + sum_{ci,tau} w2[co][ci][tau] * relu(b1[ci] + sum_tau' w1[ci][tau'] x[2(2t+tau)+tau'])
@@ -122,7 +146,7 @@ gather_encode_mean_kernel(const float *__restrict__ v, int64_t N, const int32_t 
             for (int i = 4; i < 7; ++i) vo[i] = xin[i];
             for (int64_t p = 4 * t + 7; p < mu; ++p) val[(int64_t)k * mu + p] = vk[idx[p]];
         }
-        if (k == 0) {
+        if (k == 0 && tile_lo) {
             for (int64_t p = 4 * t; p < (last ? mu : 4 * t + 4); ++p) write_tile_lo(idx, p, mu, N, tile_lo);
         }
         float h[3][C1];
@@ -397,25 +421,36 @@ dense_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val,
 
 // Ring-allreduce stage 5 when the update buffer has been cleared already: decode (MODE 0), take the
 // mean code (1) or average the kept values (2) for slot p, write it at its index, and remove the
-// entry from every node's u and v.  One thread per kept slot.
+// entry from every node's u and v.  One thread per kept slot.  Slots from mu on belong to top-k-only
+// layers (Section VI-A: the last layer): their value is the mean over the nodes of the kept entries
+// themselves, read from v.  CTAs beyond the slots average the pieces of the dense layers.
 template <int C1, int C2, int MODE>
 __global__ void __launch_bounds__(kAeThreads)
 sparse_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val, const int32_t *__restrict__ idx,
-                      int64_t mu, int64_t L1, int64_t L2, const float *__restrict__ dec, int K, int64_t N,
+                      int64_t mu, int64_t mu_all, int64_t L1, int64_t L2, const float *__restrict__ dec, int K, int64_t N,
                       float *__restrict__ recon, float *__restrict__ update, float *__restrict__ u,
-                      float *__restrict__ v)
+                      float *__restrict__ v, unsigned slot_ctas, const int64_t *__restrict__ pieces,
+                      const float *__restrict__ g, int64_t g_stride)
 {
     constexpr int kDec = C2 * C1 * 3 + C1 + C1 * 3 + 1;
     __shared__ float w[kDec];
+    if (blockIdx.x >= slot_ctas) {
+        dense_piece(pieces, blockIdx.x - slot_ctas, g, g_stride, K, update);
+        return;
+    }
     if (MODE == 0) {
         for (int i = threadIdx.x; i < kDec; i += kAeThreads) w[i] = dec[i];
         __syncthreads();
     }
     const int64_t p = (int64_t)blockIdx.x * kAeThreads + threadIdx.x;
-    if (p >= mu) return;
+    if (p >= mu_all) return;
     const int32_t i = idx[p];
     float y;
-    if (MODE == 0) {
+    if (p >= mu) {
+        y = v[i];
+        for (int k = 1; k < K; ++k) y = __fadd_rn(y, v[(int64_t)k * N + i]);
+        y = __fdiv_rn(y, (float)K);
+    } else if (MODE == 0) {
         const float *w1 = w, *b1 = w + C2 * C1 * 3, *w2 = b1 + C1;
         y = decode_at<C1, C2>(p, z, L1, L2, w1, b1, w2, w2[C1 * 3]);
     } else if (MODE == 1) {
@@ -426,7 +461,7 @@ sparse_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val
         y = __fdiv_rn(y, (float)K);
     }
     update[i] = y;
-    recon[p] = y;
+    if (p < mu) recon[p] = y;
     for (int k = 0; k < K; ++k) {
         u[(int64_t)k * N + i] = 0.0f;
         v[(int64_t)k * N + i] = 0.0f;
@@ -439,15 +474,19 @@ sparse_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val
 // The index is looked up in the other nodes' lists of the same layer eight nodes at a time: the
 // searches halve the same range in lock step, so their loads are in flight together.
 constexpr int kOwnBatch = 8;
-__global__ void scatter_own_kernel(const float *__restrict__ values, const int32_t *__restrict__ idx,
+// Serves the slots [slot0, slot0 + nslots) of every node's index row (rows are idx_stride apart); the
+// values of node k's slot p are values[k * val_stride + (p - slot0)].
+__global__ void scatter_own_kernel(const float *__restrict__ values, int64_t val_stride, const int32_t *__restrict__ idx,
+                                   int64_t idx_stride, int64_t slot0, int64_t nslots,
                                    const int32_t *__restrict__ slot_layer, const int32_t *__restrict__ koff,
-                                   int64_t mu, int K, int64_t N, float *__restrict__ update,
+                                   int K, int64_t N, float *__restrict__ update,
                                    float *__restrict__ u, float *__restrict__ v)
 {
     const int k = blockIdx.y;
-    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (p >= mu) return;
-    const int32_t i = idx[(int64_t)k * mu + p];
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= nslots) return;
+    const int64_t p = slot0 + q;
+    const int32_t i = idx[(int64_t)k * idx_stride + p];
     u[(int64_t)k * N + i] = 0.0f;
     v[(int64_t)k * N + i] = 0.0f;
     const int l = slot_layer[p];
@@ -459,7 +498,7 @@ __global__ void scatter_own_kernel(const float *__restrict__ values, const int32
         // lower bound of i in the layer's slice of nodes k0 .. k0 + 7 (the own node and nodes >= K idle)
         const int32_t *base[kOwnBatch];
 #pragma unroll
-        for (int j = 0; j < kOwnBatch; ++j) base[j] = idx + (int64_t)(k0 + j < K ? k0 + j : k) * mu + lo;
+        for (int j = 0; j < kOwnBatch; ++j) base[j] = idx + (int64_t)(k0 + j < K ? k0 + j : k) * idx_stride + lo;
         for (int n = len; n > 1;) {
             const int half = n >> 1;
             int32_t probe[kOwnBatch];
@@ -479,17 +518,17 @@ __global__ void scatter_own_kernel(const float *__restrict__ values, const int32
             const int kk = k0 + j;
             if (kk >= K) break;
             if (kk == k) {
-                acc = __fadd_rn(acc, __fdiv_rn(values[(int64_t)k * mu + p], fk));
+                acc = __fadd_rn(acc, __fdiv_rn(values[(int64_t)k * val_stride + q], fk));
                 own_added = true;
                 continue;
             }
-            const int32_t *row = idx + (int64_t)kk * mu;
+            const int32_t *row = idx + (int64_t)kk * idx_stride;
             const int32_t *hit = nullptr;
             if (at[j] == i) hit = base[j];
             else if (at[j] < i && base[j] + 1 < row + lo + len && __ldg(base[j] + 1) == i) hit = base[j] + 1;
             if (!hit) continue;
             if (!own_added) return;                               // a lower node owns this index
-            acc = __fadd_rn(acc, __fdiv_rn(values[(int64_t)kk * mu + (hit - row)], fk));
+            acc = __fadd_rn(acc, __fdiv_rn(values[(int64_t)kk * val_stride + ((hit - row) - slot0)], fk));
         }
     }
     update[i] = acc;
@@ -509,7 +548,8 @@ inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)((n + thre
 cudaError_t launch_gather(Ctx &c)
 {
     if (c.val_valid) return cudaSuccess;
-    gather_kernel<<<dim3(blocks_for(c.mu, 256), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S, c.mu, c.val), ++g_kernel_launches;
+    gather_kernel<<<dim3(blocks_for(c.mu_all, 256), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S, c.mu, c.mu_all, c.val, c.val_t),
+        ++g_kernel_launches;
     c.val_valid = true;
     return cudaGetLastError();
 }
@@ -523,12 +563,12 @@ cudaError_t launch_encode(Ctx &c)
         if (tt > 64) tt = 64;
         const unsigned grid = blocks_for(c.L2, tt);
 #define CALL(A, B) gather_encode_mean_kernel<A, B><<<grid, tt * c.K, 0, c.stream>>>(                                 \
-        c.v, c.N, c.idx, c.K, tt, c.mu, c.L2, c.params, c.val, c.code, c.combined, c.tile_lo)
+        c.v, c.N, c.idx, c.K, tt, c.mu, c.L2, c.params, c.val, c.code, c.combined, c.mixed ? nullptr : c.tile_lo)
         LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
 #undef CALL
-        c.val_valid = true;
+        c.val_valid = c.mu_t == 0;              // the values of top-k-only layers are not gathered here
         c.mean_valid = true;
-        c.tile_lo_valid = true;
+        c.tile_lo_valid = !c.mixed;
         return cudaGetLastError();
     }
     if (c.S == 1) {
@@ -562,18 +602,34 @@ cudaError_t launch_combine_ps(Ctx &c, int common_node)
     return cudaGetLastError();
 }
 
+// Averages the dense layers of the step's gradient into their places of the update (a launch of its own).
+static cudaError_t launch_dense_layers(Ctx &c, float *update)
+{
+    if (!c.num_dense_chunks) return cudaSuccess;
+    const int64_t gs = c.cfg.grad_row_stride ? c.cfg.grad_row_stride : c.N;
+    dense_pieces_kernel<<<(unsigned)c.num_dense_chunks, kAeThreads, 0, c.stream>>>(c.dense_chunks, c.step_grads, gs, c.K, update),
+        ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+// values: [S][mu] of the autoencoder layers' slots; the top-k-only layers' slots send their kept values.
 static cudaError_t launch_scatter(Ctx &c, const float *values, float *update)
 {
     if (update != c.cleared_update) {       // otherwise lgc_topk's finishing launch has cleared it already
         const cudaError_t e = launch_zero(update, (size_t)c.N * sizeof(float), c.stream);
         if (e != cudaSuccess) return e;
     }
-    if (c.S == 1)
+    if (c.S == 1 && !c.mixed) {
         scatter_shared_kernel<<<blocks_for(c.mu, 256), 256, 0, c.stream>>>(values, c.idx, c.mu, c.K, c.N, update, c.u, c.v), ++g_kernel_launches;
-    else
+    } else {
         scatter_own_kernel<<<dim3(blocks_for(c.mu, 128), c.K), 128, 0, c.stream>>>(
-            values, c.idx, c.slot_layer, c.koff_dev, c.mu, c.K, c.N, update, c.u, c.v), ++g_kernel_launches;
-    return cudaGetLastError();
+            values, c.mu, c.idx, c.mu_all, 0, c.mu, c.slot_layer, c.koff_dev, c.K, c.N, update, c.u, c.v), ++g_kernel_launches;
+        if (c.mu_t)
+            scatter_own_kernel<<<dim3(blocks_for(c.mu_t, 128), c.K), 128, 0, c.stream>>>(
+                c.val_t, c.mu_t, c.idx, c.mu_all, c.mu, c.mu_t, c.slot_layer, c.koff_dev, c.K, c.N, update, c.u, c.v), ++g_kernel_launches;
+    }
+    const cudaError_t e = cudaGetLastError();
+    return e != cudaSuccess ? e : launch_dense_layers(c, update);
 }
 
 // Ring-allreduce: the whole of stage 5 (or the phase-two sparse mean) in one pass over the update.
@@ -583,21 +639,29 @@ static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update, const f
 {
     const float *dec = c.params + c.Penc;
     const float *z1 = src ? src : c.combined;
+    if (c.mixed && update != c.cleared_update) {
+        // per-layer modes are served by the slot-wise kernel only: clear the buffer here
+        const cudaError_t e = launch_zero(update, (size_t)c.N * sizeof(float), c.stream);
+        if (e != cudaSuccess) return e;
+        c.cleared_update = update;
+    }
     if (update == c.cleared_update) {
-        // lgc_topk's finishing launch has cleared the buffer: only the kept entries are written
-        const unsigned sgrid = blocks_for(c.mu, kAeThreads);
+        // the buffer has been cleared (by lgc_topk's finishing launch, as a rule): only the kept entries and
+        // the dense layers are written
+        const unsigned slots = blocks_for(c.mu_all, kAeThreads), sgrid = slots + (unsigned)c.num_dense_chunks;
+        const int64_t gs = c.cfg.grad_row_stride ? c.cfg.grad_row_stride : c.N;
+#define SCATTER_ARGS(Z) Z, c.val, c.idx, c.mu, c.mu_all, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v, slots, c.dense_chunks, \
+                        c.step_grads, gs
         if (mode == 1) {
-            sparse_scatter_kernel<3, 2, 1><<<sgrid, kAeThreads, 0, c.stream>>>(
-                z1, c.val, c.idx, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
+            sparse_scatter_kernel<3, 2, 1><<<sgrid, kAeThreads, 0, c.stream>>>(SCATTER_ARGS(z1)), ++g_kernel_launches;
         } else if (mode == 2) {
-            sparse_scatter_kernel<3, 2, 2><<<sgrid, kAeThreads, 0, c.stream>>>(
-                c.combined, c.val, c.idx, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v), ++g_kernel_launches;
+            sparse_scatter_kernel<3, 2, 2><<<sgrid, kAeThreads, 0, c.stream>>>(SCATTER_ARGS(c.combined)), ++g_kernel_launches;
         } else {
-#define CALL(A, B) sparse_scatter_kernel<A, B, 0><<<sgrid, kAeThreads, 0, c.stream>>>(                                \
-        c.combined, c.val, c.idx, c.mu, c.L1, c.L2, dec, c.K, c.N, c.recon, update, c.u, c.v)
+#define CALL(A, B) sparse_scatter_kernel<A, B, 0><<<sgrid, kAeThreads, 0, c.stream>>>(SCATTER_ARGS(c.combined))
             LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
 #undef CALL
         }
+#undef SCATTER_ARGS
         return cudaGetLastError();
     }
     if (!c.tile_lo_valid) {

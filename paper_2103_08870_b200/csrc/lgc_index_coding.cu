@@ -262,8 +262,9 @@ deflate_indices_kernel(const int32_t *__restrict__ idx, const int32_t *__restric
 
 cudaError_t launch_encode_indices(Ctx &c, int node, unsigned char *out, int64_t capacity, unsigned long long *result)
 {
-    const int32_t *idx = c.idx + (c.S == 1 ? 0 : (int64_t)node * c.mu);
-    deflate_indices_kernel<<<1, kIcThreads, 0, c.stream>>>(idx, c.slot_layer, c.koff_dev, c.layer_off_dev, c.mu, c.ic_bytes,
+    // the whole row of slots: the autoencoder's layers, then the top-k-only ones, each layer's gaps from its own start
+    const int32_t *idx = c.idx + (c.S == 1 ? 0 : (int64_t)node * c.mu_all);
+    deflate_indices_kernel<<<1, kIcThreads, 0, c.stream>>>(idx, c.slot_layer, c.koff_dev, c.layer_off_dev, c.mu_all, c.ic_bytes,
                                                           reinterpret_cast<uint32_t *>(out), capacity, result),
         ++g_kernel_launches;
     return cudaGetLastError();

@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include <memory>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -19,6 +20,7 @@ constexpr int kSelThreads = 256;
 constexpr int kSelPerThread = 16;
 constexpr int kSelCandCap = 1024;  // candidates a chunk's list holds; more than that and the segment is finished from the data
 constexpr int kHistBins = 2048;    // first radix digit: 11 bits; the next two: 10 bits each
+constexpr int kDenseChunk = 1024;  // elements of a dense (uncompressed) layer that one CTA averages over the nodes
 constexpr int kSelGroup = 2048;    // chunks whose candidate lists one CTA compacts at a time; a segment of more chunks
                                    // than this has its groups compacted by CTAs of their own before it is finished
 
@@ -61,7 +63,10 @@ struct SelectTables {
     int32_t *tchunk0 = nullptr;      // [num_large + 1] first tile-chunk of each large segment
     int32_t *tchunk_large = nullptr; // [num_tchunks] index into large_ids
     int4 *tile_desc = nullptr;       // [tiles_per_row] x: first segment the tile overlaps; y: the large segment that
-                                     // covers the whole tile (-1: several segments, -2: no large one); z: its chunk
+                                     // covers the whole tile (-1: several segments, -2: no large one); z: its chunk;
+                                     // w: 0 no dense element in the tile, -1 all dense, else 1 + its first dense run
+    const int64_t *dense_rng = nullptr;  // [num_dense] (begin, end) of the row's runs of dense elements
+    int num_dense = 0;
     int32_t *cand_cnt = nullptr;     // [rows][num_tchunks] candidates found in the chunk
     uint2 *cand = nullptr;           // [rows][num_tchunks][kSelCandCap] (key, position inside the tile), ascending position
     int32_t *seg_m = nullptr;        // [rows][num_large] candidates of the segment
@@ -131,18 +136,29 @@ struct Ctx {
     lgc_config cfg{};
     cudaStream_t stream = nullptr;
     int K = 0, L = 0, S = 0;       // S: index sets (1 ring-allreduce, K parameter server)
+    // Per-layer treatment (Section VI-A).  A row of idx holds mu_all slots: first the mu slots of the layers
+    // that go through the autoencoder (layer order), then the mu_t slots of the top-k-only layers.
+    int L_ae = 0, L_sel = 0;       // layers through the autoencoder, layers that select at all
+    int64_t mu_t = 0, mu_all = 0;
+    bool mixed = false;            // some layer is top-k only or dense
     int64_t N = 0, mu = 0, muI = 0, L1 = 0, L2 = 0, P = 0, Penc = 0, Pdec = 0;
     int op1 = 0, op2 = 0;          // output paddings of the two transposed convolutions
     int64_t code_len = 0;          // floats per node code: c2 * L2 (identity: mu)
-    std::vector<int64_t> numel, off, k_l, koff, ki_l, kioff;
+    std::vector<int64_t> numel, off, k_l, kslot, koff, ki_l, kioff;   // k_l, kslot per layer; koff, ki_l, kioff in slot order
     double lr = 0, beta1 = 0, beta2 = 0, eps = 0;
     int64_t adam_t = 0;
     // caller buffers
     float *u = nullptr, *v = nullptr;
     float *params = nullptr, *adam_m = nullptr, *adam_v = nullptr;
     // scratch carve-up
-    int32_t *idx = nullptr;        // [S][mu]
-    float *val = nullptr;          // [K][mu]
+    int32_t *idx = nullptr;        // [S][mu_all]
+    float *val = nullptr;          // [K][mu]   kept values of the autoencoder's layers
+    float *val_t = nullptr;        // [K][mu_t] kept values of the top-k-only layers
+    int64_t *dense_rng = nullptr;  // [num_dense] (begin, end) of the runs of dense elements inside a row
+    int num_dense = 0;
+    int64_t *dense_chunks = nullptr;   // [num_dense_chunks] (begin, end): the dense runs cut into pieces of kDenseChunk
+    int64_t num_dense_chunks = 0;
+    const float *step_grads = nullptr; // gradients of the step in flight: the dense layers are read at the scatter
     float *code = nullptr;         // [K][code_len]
     float *combined = nullptr;     // [code_len]
     float *inn = nullptr;          // [K][mu]
@@ -151,9 +167,9 @@ struct Ctx {
     int32_t *kioff_dev = nullptr;  // [L + 1] first innovation slot of each layer
     int64_t *koff64_dev = nullptr; // [L] first kept slot of each layer: where a layer's innovation positions count from
     float *recon = nullptr;        // [S][mu]
-    int32_t *slot_layer = nullptr; // [mu] layer of each kept slot
-    int32_t *koff_dev = nullptr;   // [L + 1]
-    int64_t *layer_off_dev = nullptr; // [L] first element of each layer inside a row
+    int32_t *slot_layer = nullptr; // [mu_all] layer (its number in slot order) of each kept slot
+    int32_t *koff_dev = nullptr;   // [L_sel + 1] first slot of each selecting layer, slot order
+    int64_t *layer_off_dev = nullptr; // [L_sel] first element of each selecting layer inside a row, slot order
     unsigned char *ic_bytes = nullptr; // [5 mu] varint form of an index list (index coding)
     int32_t *tile_lo = nullptr;    // [ceil(N / 4096) + 1] first kept slot at or after each 4096-entry tile (ring-allreduce)
     int32_t *errword = nullptr;    // device check record
@@ -199,6 +215,28 @@ struct Ctx {
     std::string err;
 };
 
+// A setting that belongs to a device, not to the process (a kernel's opt-in to more dynamic shared
+// memory, the SM count): made once for every device ordinal that becomes current.
+constexpr int kMaxDevices = 64;
+struct OncePerDevice {
+    std::mutex mu;
+    bool done[kMaxDevices] = {};
+    template <typename F>
+    cudaError_t run(F &&f)
+    {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= kMaxDevices) return f();          // beyond the table: every time
+        std::lock_guard<std::mutex> lock(mu);
+        if (done[dev]) return cudaSuccess;
+        e = f();
+        if (e == cudaSuccess) done[dev] = true;
+        return e;
+    }
+};
+int sm_count();                                   // of the current device
+
 extern thread_local uint64_t g_kernel_launches;   // kernels this thread has enqueued (lgc_kernel_launches)
 extern thread_local std::string g_last_error;   // failures without a context (see lgc_last_error)
 
@@ -206,8 +244,9 @@ extern thread_local std::string g_last_error;   // failures without a context (s
 cudaError_t launch_zero(void *p, size_t bytes, cudaStream_t s);
 cudaError_t launch_accumulate(const float *g, float *u, float *v, uint64_t count, float m, cudaStream_t s);
 // rows of g are g_stride elements apart (u and v stay back to back)
+// dense_rng / num_dense: runs of elements that keep no state (their u and v are left alone)
 cudaError_t launch_accumulate_rows(const float *g, int64_t g_stride, float *u, float *v, int K, int64_t N, float m,
-                                   cudaStream_t s);
+                                   const int64_t *dense_rng, int num_dense, cudaStream_t s);
 cudaError_t launch_dense_mean(const float *g, int64_t g_stride, int K, int64_t n, float *update, cudaStream_t s);
 // served: the accumulation of step `epoch` collected the candidates of exactly these rows.
 // clear/clear_floats: optional 16-byte aligned buffer that spare CTAs of the finishing launch set to zero

@@ -123,3 +123,23 @@ extern "C" lgc_status lgc_topk_noalloc(const float *v, int64_t n, int64_t k, int
     if (e != cudaSuccess) return fail(LGC_ERR_CUDA, std::string("lgc_topk_noalloc: ") + cudaGetErrorString(e));
     return LGC_OK;
 }
+
+// What the kernels of the calls so far recorded in the array's check word on the current device
+// (the context-based lgc_check does not see it).  Waits for `stream`, copies four bytes to the
+// host, allocates nothing, and clears the word when it was set.
+extern "C" lgc_status lgc_topk_noalloc_check(void *stream)
+{
+    auto fail = [](lgc_status s, const std::string &msg) { g_last_error = msg; return s; };
+    unsigned char *base = nullptr;
+    cudaError_t e = scratch_address(&base);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t word = 0;
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&word, base + kOffErr, sizeof word, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail(LGC_ERR_CUDA, std::string("lgc_topk_noalloc_check: ") + cudaGetErrorString(e));
+    if (word == 0) return LGC_OK;
+    e = cudaMemsetAsync(base + kOffErr, 0, sizeof word, s);
+    char buf[112];
+    snprintf(buf, sizeof buf, "lgc_topk_noalloc: device check 0x%X: a selection kernel found inconsistent counts", (unsigned)word);
+    return fail(LGC_ERR_DEVICE_CHECK, buf);
+}

@@ -47,6 +47,8 @@ struct FastArgs {
     const int64_t *seg_off;
     const int32_t *seg_len, *seg_k, *seg_out, *small_ids, *large_ids, *seg_large, *large_q0, *tchunk0, *tchunk_large;
     const int4 *tile_desc;
+    const int64_t *dense_rng;      // (begin, end) of the runs of dense elements inside a row (layers kept out of u and v)
+    int num_dense;
     uint32_t *hist, *prefix, *lbkey, *last_key;
     int32_t *k_rem, *cand_cnt, *seg_m, *seg_ticket, *seg_epoch, *seg_path;
     uint2 *cand;                   // [rows][num_tchunks][kCandCap] candidates of a chunk: (key, position in tile), ascending position
@@ -941,6 +943,9 @@ __device__ __forceinline__ void acc4(float4 &u, float4 &v, const float4 &g, floa
     u.w = __fmaf_rn(m, u.w, g.w); v.w = __fadd_rn(v.w, u.w);
 }
 
+// DENSE: the model has layers that are sent as they are (Section VI-A) and keep no state; the instantiation
+// without them is the plain kernel, free of every test this needs.
+template <bool DENSE>
 __global__ void __launch_bounds__(kAccThreads, 2)
 accumulate_select_kernel(FastArgs f, const float *__restrict__ g, int64_t g_stride, float *__restrict__ u,
                          float *__restrict__ v, int64_t N, float m, int sel_row0, int sel_rows)
@@ -952,22 +957,34 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, int64_t g_stri
     const int p0 = (int)threadIdx.x * 4;
     const bool live = p0 < in_tile;
     // a selecting row fetches its tile's description and predicted key before the stream, so that
-    // they are at hand when the stores have been issued
+    // they are at hand when the stores have been issued; so does every row of a model with dense layers
     const int sel = row - sel_row0;
     const bool selecting = sel >= 0 && sel < sel_rows;
     int4 desc = make_int4(0, -2, 0, 0);         // x: first segment, y: the one large segment covering the tile
-                                                // (-1: several segments, -2: no large segment), z: its chunk
+                                                // (-1: several segments, -2: no large segment), z: its chunk,
+                                                // w: 0 no dense element, -1 all dense, else 1 + first dense run
     uint32_t lbkey1 = 0;
-    if (selecting) {
-        desc = __ldg(f.tile_desc + q);
-        if (desc.y >= 0) lbkey1 = f.lbkey[(int64_t)sel * f.num_large + desc.y];
-    }
+    if (selecting || DENSE) desc = __ldg(f.tile_desc + q);
+    if (DENSE && desc.w < 0) return;            // a tile of dense layers only: they keep no state
+    if (selecting && desc.y >= 0) lbkey1 = f.lbkey[(int64_t)sel * f.num_large + desc.y];
     float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
     if (live) {
         const int64_t e = ((int64_t)row * N + tile_base + p0) >> 2;
-        const float4 gg = __ldcs(reinterpret_cast<const float4 *>(g) + (((int64_t)row * g_stride + tile_base + p0) >> 2));
+        float4 gg = __ldcs(reinterpret_cast<const float4 *>(g) + (((int64_t)row * g_stride + tile_base + p0) >> 2));
         float4 uu = __ldcs(reinterpret_cast<float4 *>(u) + e);
         vv = __ldcs(reinterpret_cast<float4 *>(v) + e);
+        if (DENSE && desc.w > 0) {
+            // Dense elements among these four take no gradient: their u and v are zero from lgc_init on and
+            // stay exactly zero (m * 0 + 0 = 0, 0 + 0 = 0), which is "no state" for the layers sent as they are.
+            const int64_t pos = tile_base + p0, tile_end = tile_base + in_tile;
+            for (int r = desc.w - 1; r < f.num_dense && f.dense_rng[2 * r] < tile_end; ++r) {
+                const int64_t a = f.dense_rng[2 * r], b = f.dense_rng[2 * r + 1];
+                if (pos >= a && pos < b) gg.x = 0.0f;
+                if (pos + 1 >= a && pos + 1 < b) gg.y = 0.0f;
+                if (pos + 2 >= a && pos + 2 < b) gg.z = 0.0f;
+                if (pos + 3 >= a && pos + 3 < b) gg.w = 0.0f;
+            }
+        }
         acc4(uu, vv, gg, m);
         __stcs(reinterpret_cast<float4 *>(u) + e, uu);
         __stcs(reinterpret_cast<float4 *>(v) + e, vv);
@@ -1006,6 +1023,7 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
     f.seg_off = t.seg_off; f.seg_len = t.seg_len; f.seg_k = t.seg_k; f.seg_out = t.seg_out;
     f.small_ids = t.small_ids; f.large_ids = t.large_ids; f.seg_large = t.seg_large; f.large_q0 = t.large_q0;
     f.tchunk0 = t.tchunk0; f.tchunk_large = t.tchunk_large; f.tile_desc = t.tile_desc;
+    f.dense_rng = t.dense_rng; f.num_dense = t.num_dense;
     f.hist = t.hist; f.prefix = t.prefix; f.k_rem = t.k_rem; f.cand_cnt = t.cand_cnt; f.seg_m = t.seg_m;
     f.seg_ticket = t.seg_ticket; f.seg_epoch = t.seg_epoch; f.seg_path = t.seg_path; f.lbkey = t.lbkey; f.last_key = t.last_key; f.cand = t.cand;
     f.comp_off = t.comp_off; f.comp_total = t.comp_total; f.comp_key = t.comp_key; f.comp_idx = t.comp_idx;
@@ -1032,11 +1050,11 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
     FastArgs f;
     fill_args(f, t, data, row_stride, row0, out, out_stride, epoch, errword);
     constexpr int kFinDyn = kFinSmemCap * (int)sizeof(uint32_t);
-    static bool configured = false;
-    if (!configured) {
-        const cudaError_t e = cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinDyn);
+    static OncePerDevice configured;
+    {
+        const cudaError_t e = configured.run(
+            [] { return cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinDyn); });
         if (e != cudaSuccess) return e;
-        configured = true;
     }
     if (t.num_large && !served) {
         hist0_fast_kernel<<<dim3(t.num_tchunks, rows), kSelThreads, 0, st>>>(f), ++g_kernel_launches;
@@ -1097,8 +1115,11 @@ cudaError_t launch_accumulate_select(const SelectTables &t, const float *g, int6
 {
     FastArgs f;
     fill_args(f, t, v, N, 0, nullptr, 0, epoch, errword);
-    accumulate_select_kernel<<<dim3(t.tiles_per_row, K), kAccThreads, 0, st>>>(f, g, g_stride, u, v, N, m, sel_row0, sel_rows),
-        ++g_kernel_launches;
+    if (t.num_dense)
+        accumulate_select_kernel<true><<<dim3(t.tiles_per_row, K), kAccThreads, 0, st>>>(f, g, g_stride, u, v, N, m, sel_row0, sel_rows);
+    else
+        accumulate_select_kernel<false><<<dim3(t.tiles_per_row, K), kAccThreads, 0, st>>>(f, g, g_stride, u, v, N, m, sel_row0, sel_rows);
+    ++g_kernel_launches;
     return cudaGetLastError();
 }
 

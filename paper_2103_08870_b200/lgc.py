@@ -18,13 +18,16 @@ LIB_PATH = os.path.join(_HERE, "liblgc.so")
 LGC_OK = 0
 VARIANT_RAR, VARIANT_PS = 0, 1
 AE_CONV2, AE_IDENTITY, AE_CONV5 = 0, 1, 2
+LAYER_TOPK_AE, LAYER_TOPK_ONLY, LAYER_DENSE = 0, 1, 2
+LAYER_MODES = {"ae": LAYER_TOPK_AE, "topk": LAYER_TOPK_ONLY, "dense": LAYER_DENSE}
 
 EXPORTS = (
     "lgc_workspace_bytes", "lgc_init", "lgc_destroy", "lgc_accumulate", "lgc_topk", "lgc_encode",
-    "lgc_combine", "lgc_decode_scatter", "lgc_topk_scatter", "lgc_ae_train_step", "lgc_ae_train_step_ps",
+    "lgc_combine", "lgc_decode_scatter", "lgc_topk_scatter", "lgc_abort_step", "lgc_ae_train_step", "lgc_ae_train_step_ps",
     "lgc_encode_indices", "lgc_encode_innovation_positions", "lgc_dense_mean", "lgc_step_host",
-    "lgc_get_layout", "lgc_keep_counts", "lgc_get_buffers", "lgc_set_ae_params", "lgc_get_ae_params",
-    "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc", "lgc_kernel_launches", "lgc_selection_stats",
+    "lgc_get_layout", "lgc_keep_counts", "lgc_get_slots", "lgc_get_buffers", "lgc_set_ae_params", "lgc_get_ae_params",
+    "lgc_check", "lgc_status_string", "lgc_last_error", "lgc_topk_noalloc", "lgc_topk_noalloc_check", "lgc_kernel_launches",
+    "lgc_selection_stats",
 )
 NOALLOC_MAX_N = 16777216
 
@@ -35,7 +38,7 @@ class lgc_config(C.Structure):
         ("density_ppm", C.c_uint32), ("innovation_permille", C.c_uint32), ("momentum", C.c_float),
         ("variant", C.c_int32), ("ae_kind", C.c_int32), ("ae_c1", C.c_int32), ("ae_c2", C.c_int32),
         ("adam_lr", C.c_float), ("adam_beta1", C.c_float), ("adam_beta2", C.c_float), ("adam_eps", C.c_float),
-        ("stream", C.c_void_p), ("grad_row_stride", C.c_int64),
+        ("stream", C.c_void_p), ("grad_row_stride", C.c_int64), ("layer_mode", C.POINTER(C.c_uint8)),
     ]
 
 
@@ -59,6 +62,7 @@ def lib() -> C.CDLL:
         l.lgc_combine.argtypes = [vp, C.c_int32]
         l.lgc_decode_scatter.argtypes = [vp, vp]
         l.lgc_topk_scatter.argtypes = [vp, vp]
+        l.lgc_abort_step.argtypes = [vp]
         l.lgc_ae_train_step.argtypes = [vp, vp]
         l.lgc_ae_train_step_ps.argtypes = [vp, C.c_int32, C.c_float, C.c_float, vp]
         l.lgc_encode_indices.argtypes = [vp, C.c_int32, vp, C.c_size_t, vp]
@@ -69,6 +73,7 @@ def lib() -> C.CDLL:
         l.lgc_keep_counts.argtypes = [vp]
         l.lgc_keep_counts.restype = C.POINTER(C.c_int64)
         l.lgc_get_buffers.argtypes = [vp] + [C.POINTER(vp)] * 8
+        l.lgc_get_slots.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.POINTER(C.c_int64)), C.POINTER(vp)]
         l.lgc_set_ae_params.argtypes = [vp, vp, sz]
         l.lgc_get_ae_params.argtypes = [vp, vp, sz]
         l.lgc_check.argtypes = [vp]
@@ -77,6 +82,7 @@ def lib() -> C.CDLL:
         l.lgc_last_error.argtypes = [vp]
         l.lgc_last_error.restype = C.c_char_p
         l.lgc_topk_noalloc.argtypes = [vp, C.c_int64, C.c_int64, vp, vp]
+        l.lgc_topk_noalloc_check.argtypes = [vp]
         l.lgc_selection_stats.argtypes = [vp] + [C.POINTER(C.c_int64)] * 5
         l.lgc_kernel_launches.argtypes = []
         l.lgc_kernel_launches.restype = C.c_uint64
@@ -121,6 +127,14 @@ def topk_noalloc(v: torch.Tensor, k: int, idx_out: torch.Tensor, stream: Optiona
         raise LGCError(st, "lgc_topk_noalloc", lib().lgc_last_error(None).decode())
 
 
+def topk_noalloc_check(stream: Optional[torch.cuda.Stream] = None) -> None:
+    """lgc_topk_noalloc_check: waits for the stream and raises if a kernel of lgc_topk_noalloc recorded an inconsistency."""
+    s = stream if stream is not None else torch.cuda.current_stream()
+    st = lib().lgc_topk_noalloc_check(C.c_void_p(s.cuda_stream))
+    if st != LGC_OK:
+        raise LGCError(st, "lgc_topk_noalloc_check", lib().lgc_last_error(None).decode())
+
+
 def kernel_launches() -> int:
     """Kernels the library has enqueued from this thread so far."""
     return int(lib().lgc_kernel_launches())
@@ -141,7 +155,9 @@ class LGC:
                  momentum: float = 0.9, variant: str = "rar", ae_kind: str = "conv2", c1: int = 8,
                  c2: int = 4, innovation_permille: int = 100, lr: float = 0.0, beta1: float = 0.0,
                  beta2: float = 0.0, eps: float = 0.0, device: Optional[torch.device] = None,
-                 stream: Optional[torch.cuda.Stream] = None, grad_row_stride: int = 0):
+                 stream: Optional[torch.cuda.Stream] = None, grad_row_stride: int = 0,
+                 layer_mode: Optional[Sequence] = None):
+        """layer_mode: per layer "ae" / "topk" / "dense" (or the lgc_layer_mode numbers); None = every layer "ae"."""
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2103_08870_b200.lgc needs a CUDA device; there is no CPU path")
         self._l = lib()
@@ -149,13 +165,19 @@ class LGC:
         torch.cuda.set_device(self.device)
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
         self._numel = (C.c_int64 * len(layer_numel))(*[int(n) for n in layer_numel])
+        self._modes = None
+        if layer_mode is not None:
+            if len(layer_mode) != len(layer_numel):
+                raise ValueError("layer_mode: one entry per layer")
+            self._modes = (C.c_uint8 * len(layer_numel))(*[LAYER_MODES.get(m, m) for m in layer_mode])
         self.cfg = lgc_config(
             num_nodes=num_nodes, num_layers=len(layer_numel), layer_numel=self._numel,
             density_ppm=density_ppm, innovation_permille=innovation_permille, momentum=momentum,
             variant={"rar": VARIANT_RAR, "ps": VARIANT_PS}[variant],
             ae_kind={"conv2": AE_CONV2, "identity": AE_IDENTITY, "conv5": AE_CONV5}[ae_kind], ae_c1=c1, ae_c2=c2,
             adam_lr=lr, adam_beta1=beta1, adam_beta2=beta2, adam_eps=eps,
-            stream=C.c_void_p(self.stream.cuda_stream), grad_row_stride=grad_row_stride)
+            stream=C.c_void_p(self.stream.cuda_stream), grad_row_stride=grad_row_stride,
+            layer_mode=self._modes if self._modes is not None else C.POINTER(C.c_uint8)())
         self.grad_row_stride = grad_row_stride
         self.variant, self.ae_kind, self.K, self.c1, self.c2 = variant, ae_kind, num_nodes, c1, c2
         sb, wb, pb = C.c_size_t(), C.c_size_t(), C.c_size_t()
@@ -174,6 +196,11 @@ class LGC:
         self.L = len(layer_numel)
         kc = self._l.lgc_keep_counts(self._ctx)
         self.k_l = [kc[i] for i in range(self.L)]
+        mu_all, slots, vt = C.c_int64(), C.POINTER(C.c_int64)(), C.c_void_p()
+        self._ok(self._l.lgc_get_slots(self._ctx, C.byref(mu_all), C.byref(slots), C.byref(vt)), "lgc_get_slots")
+        self.mu_all, self.mu_t = mu_all.value, mu_all.value - self.mu
+        self.first_slot = [slots[i] for i in range(self.L)]      # of each layer's kept entries in a row of idx; -1: dense
+        self._val_t_ptr = vt.value
         self.S = self.K if variant == "ps" else 1
         self.code_len = self.mu if ae_kind == "identity" else c2 * self.L2
         if ae_kind == "conv5":          # four stride-2 convolutions, four code channels, stored [L4][4]
@@ -232,6 +259,9 @@ class LGC:
 
     def topk_scatter(self, update: torch.Tensor) -> None:
         self._ok(self._l.lgc_topk_scatter(self._ctx, self._dev_f32(update, self.N, "update")), "lgc_topk_scatter")
+
+    def abort_step(self) -> None:
+        self._ok(self._l.lgc_abort_step(self._ctx), "lgc_abort_step")
 
     def ae_train_step(self, loss_out: Optional[torch.Tensor] = None) -> None:
         ptr = self._dev_f32(loss_out, 1, "loss_out") if loss_out is not None else None
@@ -327,11 +357,15 @@ class LGC:
 
     @property
     def idx(self) -> torch.Tensor:
-        return self._view(self.scratch, self._buffers()[2], (self.S, self.mu), torch.int32)
+        return self._view(self.scratch, self._buffers()[2], (self.S, self.mu_all), torch.int32)
 
     @property
     def val(self) -> torch.Tensor:
         return self._view(self.scratch, self._buffers()[3], (self.K, self.mu), torch.float32)
+
+    @property
+    def val_topk_only(self) -> Optional[torch.Tensor]:
+        return self._view(self.scratch, self._val_t_ptr, (self.K, self.mu_t), torch.float32)
 
     @property
     def code(self) -> torch.Tensor:

@@ -7,12 +7,12 @@ the compressed path runs.  Section VI-A: the first layer's gradient is sent as i
 layer's top-magnitude values are sent without the autoencoder, every layer in between goes
 through top-k selection and the autoencoder.
 
-A model is therefore cut into runs of consecutive layers that are treated alike.  A "dense" run
-needs no state: its update is the mean over the nodes (lgc_dense_mean).  A "topk" run and an
-"ae" run each get a context of their own that works on its slice of the flat gradient
-(lgc_config.grad_row_stride = length of a whole row); the "topk" run never calls the autoencoder
-stages (accumulate, top-k, dense mean of the kept values).  This module only sequences calls and
-passes pointers: every step of the path runs in the library's kernels.
+One context serves the whole model: lgc_config.layer_mode gives every layer its treatment
+("dense": the mean of the nodes' gradients, no state; "topk": accumulated and selected, the kept
+values sent without the autoencoder; "ae": top-k selection and the autoencoder, whose input is the
+concatenation of the kept values of all such layers).  The first phase is lgc_dense_mean over the
+whole gradient.  This module only sequences calls and passes pointers: every step of the path runs
+in the library's kernels.
 """
 from __future__ import annotations
 
@@ -54,23 +54,16 @@ class PhasedLGC:
         """`adam`: lr, beta1, beta2, eps of the autoencoder's training steps (defaults 1e-3, 0.9, 0.999, 1e-8)."""
         self.numel = [int(n) for n in layer_numel]
         self.N, self.K, self.variant = sum(self.numel), int(num_nodes), variant
-        self.runs = layer_runs(self.numel, layer_mode)
-        for r in self.runs:
-            if r.begin % 4:
-                raise ValueError("every run of layers must start at a multiple of 4 elements (16-byte aligned slices)")
-            if r.mode == "dense":
-                continue
-            r.ctx = lgc.LGC(self.numel[r.first:r.last], num_nodes, density_ppm=density_ppm, momentum=momentum,
-                            variant=variant, ae_kind=ae_kind if r.mode == "ae" else "identity", c1=c1, c2=c2,
-                            innovation_permille=innovation_permille, device=device, grad_row_stride=self.N, **adam)
-
-    def ae_runs(self) -> List[Run]:
-        return [r for r in self.runs if r.mode == "ae"]
+        self.runs = layer_runs(self.numel, layer_mode)          # for callers that want the element ranges
+        self.ctx = lgc.LGC(self.numel, num_nodes, density_ppm=density_ppm, momentum=momentum, variant=variant,
+                           ae_kind=ae_kind, c1=c1, c2=c2, innovation_permille=innovation_permille, device=device,
+                           layer_mode=list(layer_mode), **adam)
 
     def step(self, grads: torch.Tensor, update: torch.Tensor, phase: str, choice: int = 0,
              loss_out: Optional[torch.Tensor] = None) -> None:
         """One iteration: grads [K][N] fp32 CUDA (contiguous), update [N] fully written.
-        choice: the ring-allreduce leader / the parameter server's common node of this iteration."""
+        choice: the ring-allreduce leader / the parameter server's common node of this iteration.
+        `grads` must stay as it is until the step has run on the stream (the dense layers are read last)."""
         if phase not in PHASES:
             raise ValueError(phase)
         if tuple(grads.shape) != (self.K, self.N) or not grads.is_contiguous() or update.numel() != self.N:
@@ -78,27 +71,20 @@ class PhasedLGC:
         if phase == "raw":
             lgc.dense_mean(grads, update)
             return
-        for r in self.runs:
-            g, u = grads[:, r.begin:r.end], update[r.begin:r.end]
-            if r.mode == "dense":
-                lgc.dense_mean(g, u)
-                continue
-            c = r.ctx
-            c.accumulate(g, choice)
-            c.topk(choice, u)
-            if r.mode == "topk" or phase == "topk_train":
-                if r.mode == "ae" and c.ae_kind != "identity":
-                    if self.variant == "rar":
-                        c.ae_train_step(loss_out)
-                    else:
-                        c.ae_train_step_ps(choice, 1.0, 1.0, loss_out)
-                c.topk_scatter(u)
-            else:
-                c.encode()
-                c.combine(choice)
-                c.decode_scatter(u)
+        c = self.ctx
+        c.accumulate(grads, choice)
+        c.topk(choice, update)
+        if phase == "topk_train":
+            if c.ae_kind != "identity":
+                if self.variant == "rar":
+                    c.ae_train_step(loss_out)
+                else:
+                    c.ae_train_step_ps(choice, 1.0, 1.0, loss_out)
+            c.topk_scatter(update)
+        else:
+            c.encode()
+            c.combine(choice)
+            c.decode_scatter(update)
 
     def check(self) -> None:
-        for r in self.runs:
-            if r.ctx is not None:
-                r.ctx.check()
+        self.ctx.check()

@@ -32,6 +32,20 @@ def assert_close(got, ref, what, rel=REL_TOL):
     assert err <= rel * scale, f"{what}: max error {err:.3e} > {rel:.0e} * {scale:.3e}"
 
 
+def assert_close_elementwise(got, ref, what, rel=REL_TOL, floor=2e-6):
+    """Entry by entry: |a - b| <= rel * |ref| + floor * max|ref|.  The floor is the rounding of the fp32
+    sums themselves (up to 49 terms at the vector's scale); above it every entry is held to `rel` of its
+    own magnitude, so small entries are not covered by the largest one."""
+    got = np.asarray(got, dtype=np.float64).reshape(-1)
+    ref = np.asarray(ref, dtype=np.float64).reshape(-1)
+    assert got.shape == ref.shape, f"{what}: shape {got.shape} vs {ref.shape}"
+    scale = max(np.abs(ref).max(), 1e-30)
+    excess = np.abs(got - ref) - (rel * np.abs(ref) + floor * scale)
+    worst = int(np.argmax(excess))
+    assert excess[worst] <= 0, (f"{what}: entry {worst}: {got[worst]!r} vs {ref[worst]!r} "
+                                f"(allowed {rel:.0e} of the entry + {floor:.0e} of {scale:.3e})")
+
+
 def make_pair(numel, K, variant="rar", ae_kind="conv2", c1=8, c2=4, density_ppm=1000, momentum=0.9,
               innovation_permille=100, seed=W.DEFAULT_SEED, topk_method="auto", **adam):
     """`adam`: lr, beta1, beta2, eps for both sides (defaults 1e-3, 0.9, 0.999, 1e-8)."""
@@ -77,6 +91,8 @@ def compare_step(ora, gpu, g_cpu: torch.Tensor, g_dev: torch.Tensor, choice: int
         assert_close(gpu.code.cpu().numpy(), ora.z.transpose(0, 2, 1).reshape(K, -1), "codes", rel=rel)
     else:
         assert_close(gpu.code.cpu().numpy(), ora.z.reshape(K, -1), "codes")
+        if ora.ae_kind == "conv2":
+            assert_close_elementwise(gpu.code.cpu().numpy(), ora.z.reshape(K, -1), "codes, entry by entry")
     ora.combine(choice)
     gpu.combine(choice)
     if ora.variant == "rar":
@@ -89,6 +105,8 @@ def compare_step(ora, gpu, g_cpu: torch.Tensor, g_dev: torch.Tensor, choice: int
     gpu.decode_scatter(update_dev)
     if not (ora.variant == "rar" and ora.ae_kind == "identity"):
         assert_close(gpu.recon.cpu().numpy(), ora.r, "reconstruction", rel=rel)
+        if ora.ae_kind == "conv2":
+            assert_close_elementwise(gpu.recon.cpu().numpy(), ora.r, "reconstruction, entry by entry")
     upd = update_dev.cpu().numpy()
     assert_close(upd, upd_ref, "dense update", rel=rel)
     touched = np.zeros(ora.N, bool)

@@ -84,6 +84,8 @@ def test_status_strings_and_null_context(lib):
     assert lib.lgc_status_string(99) == b"LGC_ERR_UNKNOWN"
     assert lib.lgc_accumulate(None, None, 0) == 1
     assert lib.lgc_destroy(None) == 0
+    assert lib.lgc_abort_step(None) == 1
+    assert lib.lgc_step_host(None, None, None, None, None, 0) == 1
     assert isinstance(lib.lgc_last_error(None), bytes)
 
 

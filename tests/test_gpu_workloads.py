@@ -1,9 +1,9 @@
 """The five workload configurations at full size, in the launch configuration bench.py times.
 
 Configs 1-3 run the whole oracle beside the CUDA path (they fit in host memory and finish in
-tens of seconds per step); the stress config (2^30 elements per node) compares the elementwise
-stages on sampled positions, the selection against the oracle on the leader's full row, and the
-autoencoder stages in full (they work on mu values only).
+tens of seconds per step); the stress config (2^30 elements per node) does too when the host has
+the memory for the oracle's state (32 GiB), and otherwise compares the elementwise stages on sampled
+positions, the selection on the leader's full row, and the autoencoder stages in full.
 """
 import numpy as np
 import pytest
@@ -145,40 +145,89 @@ def test_segnet_config_with_autoencoder_training():
         compare_step(ora, gpu, g.cpu(), g, W.choice_for_step(w.seed, t, K), upd, check_state=(t == w.ae_train_steps + 2))
 
 
-def test_stress_config_sampled():
+def rows_equal_bitwise(dev_row: torch.Tensor, host_row: np.ndarray, what: str, piece: int = 1 << 28):
+    """Whole-row bitwise comparison of a device row with the oracle's host row, a GiB at a time."""
+    n = dev_row.numel()
+    assert host_row.size == n
+    for a in range(0, n, piece):
+        b = min(n, a + piece)
+        ref = torch.from_numpy(host_row[a:b]).cuda().view(torch.int32)
+        got = dev_row[a:b].view(torch.int32)
+        if not torch.equal(got, ref):
+            bad = torch.nonzero(got != ref).flatten()
+            raise AssertionError(f"{what}: {bad.numel()} entries of [{a}, {b}) differ bitwise; first at {a + int(bad[0])}")
+        del ref
+
+
+def host_memory_available() -> int:
+    import psutil
+    return int(psutil.virtual_memory().available)
+
+
+def test_stress_config():
+    # 2^30 elements per node, K = 4.  With enough host memory the oracle carries the WHOLE state (u, v of all
+    # four nodes, 32 GiB): every step its accumulation is compared with the device rows bit for bit over
+    # the full length, the selection is the oracle's on the leader's full row, and the rows are compared
+    # again in full after the sent entries have been cleared.  The autoencoder stages work on mu values
+    # and are compared in full in either mode.  With less host memory the elementwise stages are compared
+    # on two million sampled positions plus the row edges instead.
     w = W.workload("stress")
     K, N = w.num_nodes, w.table.total
     free, _ = torch.cuda.mem_get_info()
     if free < 70 * 2**30:
         pytest.skip("needs about 70 GiB of free device memory")
+    whole = host_memory_available() >= 56 * 2**30
+    print(f"stress config: host memory available {host_memory_available() / 2**30:.0f} GiB -> "
+          + ("whole-row comparison" if whole else "sampled comparison"))
     gpu = lgc.LGC(w.table.numel, K, density_ppm=w.density_ppm, momentum=w.momentum, c1=w.ae_c1, c2=w.ae_c2)
     params = W.ae_init_params(w.ae_c1, w.ae_c2, "rar", K, w.seed)
     gpu.set_ae_params(params)
     assert gpu.mu == 107_374 and (gpu.L1, gpu.L2) == (53_686, 26_842)
-    # the oracle works on mu-sized vectors in full and on a sample of the 2^30 positions
+    # the oracle of the autoencoder stages works on mu-sized vectors in full
     ora = OracleLGC([gpu.mu * 1000], K, density_ppm=1000, c1=w.ae_c1, c2=w.ae_c2, params=params.numpy())
     assert ora.mu == gpu.mu
+    m = float(np.float32(w.momentum))
     rng = np.random.default_rng(7)
     pos = np.unique(np.concatenate([rng.integers(0, N, 2_000_000), np.arange(0, 4096), np.arange(N - 4099, N)]))
     pos_dev = torch.from_numpy(pos).cuda()
-    u_s = np.zeros((K, pos.size), np.float32)
-    v_s = np.zeros((K, pos.size), np.float32)
+    if whole:
+        u_o = np.zeros((K, N), np.float32)
+        v_o = np.zeros((K, N), np.float32)
+    else:
+        u_s = np.zeros((K, pos.size), np.float32)
+        v_s = np.zeros((K, pos.size), np.float32)
     src = W.GradientSource(w.table, K, seed=w.seed, device="cuda", chunk=1 << 26)
     g = torch.empty((K, N), dtype=torch.float32, device="cuda")
     upd = torch.empty(N, dtype=torch.float32, device="cuda")
     for t in range(w.steps):
         src.step_into(t, g)
         leader = W.choice_for_step(w.seed, t, K)
-        g_s = g[:, pos_dev].cpu().numpy()
+        edge = t in (0, w.steps - 1)
+        if not whole:
+            g_s = g[:, pos_dev].cpu().numpy()
         gpu.accumulate(g, leader)
         for k in range(K):
-            O.accumulate(u_s[k], v_s[k], np.ascontiguousarray(g_s[k]), float(np.float32(w.momentum)))
-        assert_bitwise(gpu.u[:, pos_dev].cpu().numpy(), u_s, f"sampled u, step {t}")
-        assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_s, f"sampled v, step {t}")
+            if whole:
+                g_k = g[k].cpu().numpy()
+                O.accumulate(u_o[k], v_o[k], g_k, m)
+                del g_k
+                if edge or k == leader:
+                    rows_equal_bitwise(gpu.v[k], v_o[k], f"v of node {k} after the accumulation of step {t}")
+                if edge:
+                    rows_equal_bitwise(gpu.u[k], u_o[k], f"u of node {k} after the accumulation of step {t}")
+            else:
+                O.accumulate(u_s[k], v_s[k], np.ascontiguousarray(g_s[k]), m)
+        if whole:
+            assert_bitwise(gpu.u[:, pos_dev].cpu().numpy(), u_o[:, pos], f"sampled u, step {t}")
+            assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_o[:, pos], f"sampled v, step {t}")
+        else:
+            assert_bitwise(gpu.u[:, pos_dev].cpu().numpy(), u_s, f"sampled u, step {t}")
+            assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_s, f"sampled v, step {t}")
         gpu.topk(leader, upd)
         idx = gpu.idx.cpu().numpy()[0]
-        if t in (0, w.steps - 1):                          # the selection against the oracle, whole row
-            v_leader = gpu.v[leader].cpu().numpy()
+        ref_idx = leader_vals = None
+        if whole or edge:                                  # the selection against the oracle, whole row
+            v_leader = v_o[leader] if whole else gpu.v[leader].cpu().numpy()
             ref_idx = O.topk(v_leader, gpu.mu, method="select")
             assert_bitwise(idx, ref_idx, f"selected indices, step {t}")
             leader_vals = O.gather(v_leader, ref_idx)
@@ -187,9 +236,12 @@ def test_stress_config_sampled():
         idx_dev = gpu.idx[0].long()
         gpu.encode()
         val = gpu.val.cpu().numpy()
-        assert_bitwise(val, gpu.v[:, idx_dev].cpu().numpy(), "gathered values")      # same bits as v at idx
-        if t in (0, w.steps - 1):
-            assert_bitwise(val[leader], leader_vals, "leader values against the oracle's gather")
+        if whole:                                          # the oracle's gather on its own rows
+            assert_bitwise(val, np.stack([O.gather(v_o[k], ref_idx) for k in range(K)]), "gathered values")
+        else:
+            assert_bitwise(val, gpu.v[:, idx_dev].cpu().numpy(), "gathered values")  # same bits as v at idx
+            if leader_vals is not None:
+                assert_bitwise(val[leader], leader_vals, "leader values against the oracle's gather")
         ora.idx = np.broadcast_to(idx, (K, gpu.mu)).copy()
         ora.val = val.copy()
         ora.encode()
@@ -203,10 +255,18 @@ def test_stress_config_sampled():
         assert_close(upd[idx_dev].cpu().numpy(), ora.r[0], "update at the scatter positions")
         assert int(torch.count_nonzero(upd).item()) <= gpu.mu
         assert float(upd.abs().sum().item()) == pytest.approx(float(np.abs(ora.r[0].astype(np.float32)).sum()), rel=1e-4)
-        sent = np.isin(pos, idx)
-        u_s[:, sent] = 0
-        v_s[:, sent] = 0
-        assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_s, f"sampled v after clearing, step {t}")
+        if whole:
+            for k in range(K):
+                O.clear(u_o[k], v_o[k], ref_idx)
+                if edge:
+                    rows_equal_bitwise(gpu.u[k], u_o[k], f"u of node {k} after the clearing of step {t}")
+                    rows_equal_bitwise(gpu.v[k], v_o[k], f"v of node {k} after the clearing of step {t}")
+            assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_o[:, pos], f"sampled v after clearing, step {t}")
+        else:
+            sent = np.isin(pos, idx)
+            u_s[:, sent] = 0
+            v_s[:, sent] = 0
+            assert_bitwise(gpu.v[:, pos_dev].cpu().numpy(), v_s, f"sampled v after clearing, step {t}")
         assert not gpu.v[:, idx_dev].any().item() and not gpu.u[:, idx_dev].any().item()
         gpu.check()
 
@@ -221,7 +281,7 @@ def test_resnet50_config_with_the_layer_treatment_of_the_paper():
     modes = ["dense"] + ["ae"] * (len(numel) - 3) + ["topk", "topk"]
     params = W.ae_init_params(w.ae_c1, w.ae_c2, "rar", K, w.seed)
     gpu = PhasedLGC(numel, modes, K, density_ppm=w.density_ppm, momentum=w.momentum)
-    gpu.ae_runs()[0].ctx.set_ae_params(params)
+    gpu.ctx.set_ae_params(params)
     ora = OraclePhased(numel, modes, K, {1: params.numpy()}, density_ppm=w.density_ppm, momentum=w.momentum)
     src = W.GradientSource(w.table, K, seed=w.seed, device="cuda")
     upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
@@ -232,7 +292,12 @@ def test_resnet50_config_with_the_layer_treatment_of_the_paper():
         gpu.step(g, upd, phase, choice)
         ref, _ = ora.step(g.cpu().numpy(), phase, choice)
         assert_close(upd.cpu().numpy(), ref, f"step {t} ({phase}): update")
-    for r, gr in zip(gpu.runs, ora.groups):
-        if r.ctx is not None:
-            assert_bitwise(r.ctx.v.cpu().numpy(), gr["o"].v, f"residual of the {r.mode} run")
+    v = gpu.ctx.v.cpu().numpy()
+    for gr in ora.groups:
+        if gr["mode"] == "dense":
+            assert not v[:, gr["a"]:gr["b"]].any(), "the dense layer holds state"
+        else:
+            assert_bitwise(v[:, gr["a"]:gr["b"]], gr["o"].v, f"residual of the {gr['mode']} layers")
+    large, served, _, _, _ = gpu.ctx.selection_stats()
+    assert served > 0, "the accumulation collected no candidates for the one context"
     gpu.check()
