@@ -199,7 +199,7 @@ SelectPlan plan_select(const std::vector<int64_t> &off, const std::vector<int64_
             if (c1 - c0 > kSelGroup)
                 for (int32_t gb = c0; gb < c1; gb += kSelGroup) sp.group_job.push_back(make_int2(li, gb));
             sp.tchunk0.push_back(c1);
-            sp.comp_off.push_back(sp.comp_off.back() + select_compact_capacity(len[i]));
+            sp.comp_off.push_back(sp.comp_off.back() + select_compact_capacity(len[i], k[i]));
         }
     }
     sp.comp_total = sp.comp_off.back();
@@ -279,6 +279,7 @@ void carve_select(Carver &cv, SelectTables &t, const SelectPlan &sp, int rows)
     t.seg_epoch = cv.take<int32_t>((size_t)rows * nl);
     t.lbkey = cv.take<uint32_t>((size_t)rows * nl);
     t.last_key = cv.take<uint32_t>((size_t)rows * nl);
+    t.key_trend = cv.take<float2>((size_t)rows * nl);
     t.seg_path = cv.take<int32_t>((size_t)rows * nl);
     t.cand_cnt = cv.take<int32_t>((size_t)rows * nc);
     t.cand = cv.take<uint2>((size_t)rows * nc * kSelCandCap);

@@ -18,7 +18,7 @@ namespace lgc {
 constexpr int kSelChunk = 4096;    // elements per selection chunk: 256 threads x 16
 constexpr int kSelThreads = 256;
 constexpr int kSelPerThread = 16;
-constexpr int kSelCandCap = 1024;  // candidates a chunk's list holds; more than that and the segment is finished from the data
+constexpr int kSelCandCap = 256;   // candidates a chunk's list holds; more than that and the segment is finished from the data
 constexpr int kHistBins = 2048;    // first radix digit: 11 bits; the next two: 10 bits each
 constexpr int kDenseChunk = 1024;  // elements of a dense (uncompressed) layer that one CTA averages over the nodes
 constexpr int kSelGroup = 2048;    // chunks whose candidate lists one CTA compacts at a time; a segment of more chunks
@@ -75,17 +75,20 @@ struct SelectTables {
     int32_t *seg_path = nullptr;     // [rows][num_large] how the last selection got its entries (see lgc_selection_stats)
     uint32_t *last_key = nullptr;    // [rows][num_large] k-th key of the previous selection (0: none)
     uint32_t *lbkey = nullptr;       // [rows][num_large] key from which the next accumulation collects candidates (0: none)
+    float2 *key_trend = nullptr;     // [rows][num_large] x: ln of the last ratio of consecutive k-th keys; y: how much that
+                                     // ratio has jumped from step to step lately (decaying maximum)
     int64_t *comp_off = nullptr;     // [num_large + 1] first compact slot of each large segment
     int64_t comp_total = 0;          // compact slots per row
     uint32_t *comp_key = nullptr;    // [rows][comp_total] keys of the candidates, index order
     int32_t *comp_idx = nullptr;     // [rows][comp_total] their offsets inside the row
 };
 
-// Compact-array capacity of a large segment of n elements: above it the segment is finished by
-// streaming over the data itself.
-inline int64_t select_compact_capacity(int64_t n)
+// Compact-array capacity of a large segment of n elements of which k are kept: above it the segment is
+// finished by streaming over the data itself.  Candidates are the entries from a little below the k-th
+// key upwards, a few times k in practice; ties can make them many more.
+inline int64_t select_compact_capacity(int64_t n, int64_t k)
 {
-    const int64_t c = n / 8 > 32768 ? n / 8 : 32768;
+    const int64_t c = 64 * k > 8192 ? 64 * k : 8192;
     return c < n ? c : n;
 }
 

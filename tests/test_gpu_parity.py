@@ -117,11 +117,12 @@ def test_layer_spanning_several_compaction_groups():
     assert gpu.selection_stats()[1] == 2          # both layers served from the accumulation by now
 
 
-@pytest.mark.parametrize("levels, first_from_data", [(50, 0), (3, 1)])
+@pytest.mark.parametrize("levels, first_from_data", [(200, 0), (3, 2)])
 def test_layer_of_several_groups_with_ties(levels, first_from_data):
     # integer-valued gradients: the k-th magnitude is shared by many entries of the 9 M layer, which
-    # is finished group by group (51 levels: ~178 k entries tie for 9000 places in the first step)
-    # or, when the tied entries exceed the layer's compact capacity (4 levels: 2.6 M), from the data
+    # is finished group by group (401 levels: ~45 k entries tie for 9000 places in the first step, and
+    # the candidates, nine levels, are 4.5 % of the layer) or, when the tied entries exceed the layer's
+    # compact capacity or a chunk's list (7 levels: 2.6 M of the large layer, 1400 of the small one), from the data
     numel = [9_000_000, 5000]
     K = 2
     ora, gpu = make_pair(numel, K, momentum=0.0, topk_method="select")
