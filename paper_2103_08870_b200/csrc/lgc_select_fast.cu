@@ -33,6 +33,7 @@ struct FastArgs {
     int row0;
     int num_large, num_small, num_tchunks;
     int fin_small;                 // small segments served by CTAs of finish_kernel (0 or num_small)
+    int smem_keys;                 // candidate keys a finishing CTA can keep in its dynamic shared memory
     const int32_t *large_order;    // large segments, longest first: the order the finishing CTAs take them in
     const int2 *group_job;         // (large segment, first chunk) of every group that the wide kernels serve
     int num_group_jobs;
@@ -62,9 +63,15 @@ struct FastArgs {
     int32_t *errword;
 };
 
-constexpr int kFinThreads = 512;      // two finishing CTAs fit on an SM, so every segment of a ResNet starts at once
+// A finishing CTA has 512 threads and keeps up to 20480 candidate keys in shared memory (80 KB: two CTAs per SM).
+// Two other shapes of the same kernel serve the extremes: when every segment can have an SM of its own (one
+// selecting row of a ResNet: 53 segments), 1024 threads halve everything that is done per candidate; when there
+// are many times more segments than SMs (every row selecting: 16 x 104), 256 threads and 6144 keys let four
+// CTAs share an SM, and these latency-bound CTAs overlap twice as well.
+constexpr int kFinThreads = 512;      // also the CTA size of the kernels that serve segments of several groups
 constexpr int kFinWarps = kFinThreads / 32;
-constexpr int kFinSmemCap = 20480;    // candidate keys a finishing CTA keeps in shared memory (80 KB; two CTAs per SM)
+constexpr int kFinSmemCap = 20480;    // candidate keys in shared memory, 512- and 1024-thread shapes
+constexpr int kFinSmemCapSmall = 6144;   // 256-thread shape
 constexpr int kFinGroup = kSelGroup;  // chunks whose candidate counts are scanned together during the compaction
 constexpr int kFinPerThread = 16;     // consecutive entries per thread in the ordered passes
 constexpr int kCandCap = kSelCandCap;  // entries a chunk's list can hold; a chunk with more sends its segment to the data
@@ -325,19 +332,19 @@ struct DataSource {
 
 struct FinishShared {
     int hist[1024];
-    int warp_i[kFinWarps];
-    unsigned warp_u[kFinWarps];
+    int warp_i[32];
+    unsigned warp_u[32];
     int found[2];
 };
 
 // Ordered emission by counting: an entry of `src` is selected iff its key is above T, or equals T
 // and fewer than r equal keys precede it in the whole segment; its output slot is the number of
 // selected entries before it.  gt_done / eq_done: entries with key > T / == T that precede src.
-template <typename Source>
+template <int THREADS, typename Source>
 __device__ void emit_ordered(const Source &src, uint32_t T, int r, int gt_done, int eq_done, int k,
                              int32_t *__restrict__ out, FinishShared &sh, int32_t *errword)
 {
-    const int tile = kFinThreads * kFinPerThread;
+    const int tile = THREADS * kFinPerThread;
     for (int base = 0; base < src.n; base += tile) {
         uint32_t key[kFinPerThread];
         const int first = base + (int)threadIdx.x * kFinPerThread;
@@ -371,22 +378,22 @@ __device__ void emit_ordered(const Source &src, uint32_t T, int r, int gt_done, 
 // Completes the radix search below the 11-bit bucket d0 (k_rem entries still to find inside it)
 // and emits the k selected offsets in order; returns the k-th key.  Entries below the bucket, if
 // the source has any, are ignored.
-template <typename Source>
+template <int THREADS, typename Source>
 __device__ uint32_t finish_from(const Source &src, uint32_t d0, int k_rem, int k, int32_t *__restrict__ out,
                                 FinishShared &sh, int32_t *errword)
 {
     // the 20 bits below the bucket, ten at a time
     uint32_t prefix = d0 << 20, decided = 0x7ff00000u;
-    constexpr int kBinsPer = 1024 / kFinThreads;
+    constexpr int kBinsPer = 1024 / THREADS;
 #pragma unroll 1
     for (int shift = 10; shift >= 0; shift -= 10) {
-        for (int b = threadIdx.x; b < 1024; b += kFinThreads) sh.hist[b] = 0;
+        for (int b = threadIdx.x; b < 1024; b += THREADS) sh.hist[b] = 0;
         __syncthreads();
-        for (int base = 0; base < src.n; base += kFinThreads * 8) {      // eight independent loads per thread
+        for (int base = 0; base < src.n; base += THREADS * 8) {      // eight independent loads per thread
             uint32_t x[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const int i = base + j * kFinThreads + (int)threadIdx.x;
+                const int i = base + j * THREADS + (int)threadIdx.x;
                 x[j] = i < src.n ? src.key_at(i) : 0xffffffffu;          // never matches the prefix
             }
 #pragma unroll
@@ -417,7 +424,7 @@ __device__ uint32_t finish_from(const Source &src, uint32_t d0, int k_rem, int k
         k_rem = sh.found[1];
         __syncthreads();
     }
-    emit_ordered(src, prefix, k_rem, 0, 0, k, out, sh, errword);
+    emit_ordered<THREADS>(src, prefix, k_rem, 0, 0, k, out, sh, errword);
     const uint32_t T = prefix;
     return T;
 }
@@ -425,9 +432,10 @@ __device__ uint32_t finish_from(const Source &src, uint32_t d0, int k_rem, int k
 // Bucket of the k-th largest key from a complete leading-digit histogram in shared memory (which
 // holds at least k entries): leaves the bucket in sh.found[0] and the rank still to find inside
 // it in sh.found[1].  Run by every thread of the CTA; ends with a barrier.
+template <int THREADS>
 __device__ __forceinline__ void digit_scan(const unsigned *hist, int k, FinishShared &sh)
 {
-    constexpr int kPer = kHistBins / kFinThreads;
+    constexpr int kPer = kHistBins / THREADS;
     int part = 0;
 #pragma unroll
     for (int i = 0; i < kPer; ++i) part += (int)hist[threadIdx.x * kPer + i];
@@ -493,11 +501,12 @@ __device__ __forceinline__ ListVerdict list_verdict(const FastArgs &f, int row, 
 
 // Compacts the candidates of the gn chunks from chunk gb on (large segment li of `row`) in index
 // order into ckey/cidx, which already hold `done` entries; returns how many it added.
-// group_off: kFinGroup ints of shared memory.  All kFinThreads threads take part.
+// group_off: kFinGroup ints of shared memory.  All THREADS threads of the CTA take part.
+template <int THREADS>
 __device__ __forceinline__ int compact_group(const FastArgs &f, int row, int li, int gb, int gn, int done,
                                              uint32_t *ckey, int32_t *cidx, int *group_off, unsigned *warp_u)
 {
-    constexpr int kPerT = kFinGroup / kFinThreads;
+    constexpr int kPerT = kFinGroup / THREADS;
     const int c0 = f.tchunk0[li], q0 = f.large_q0[li];
     const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
     // exclusive prefix of the chunk counts of this group, in shared memory
@@ -522,7 +531,7 @@ __device__ __forceinline__ int compact_group(const FastArgs &f, int row, int li,
     // neighbouring records)
     int top = 1;                                           // largest power of two below gn (1 when gn <= 2)
     while (top * 2 < gn) top *= 2;
-    for (int base = 0; base < (int)total; base += kFinThreads * 8) {
+    for (int base = 0; base < (int)total; base += THREADS * 8) {
         const uint2 *rec[8];
         int tile0[8];
         // the last chunk whose offset is <= rank, for the eight ranks side by side: the halving steps run in
@@ -534,12 +543,12 @@ __device__ __forceinline__ int compact_group(const FastArgs &f, int row, int li,
 #pragma unroll
             for (int t = 0; t < 8; ++t) {
                 const int at = lo[t] + step;
-                if (at < gn && group_off[at] <= base + t * kFinThreads + (int)threadIdx.x) lo[t] = at;
+                if (at < gn && group_off[at] <= base + t * THREADS + (int)threadIdx.x) lo[t] = at;
             }
         }
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
-            const int r = base + t * kFinThreads + (int)threadIdx.x;
+            const int r = base + t * THREADS + (int)threadIdx.x;
             rec[t] = nullptr;
             tile0[t] = 0;
             if (r < (int)total) {
@@ -552,7 +561,7 @@ __device__ __forceinline__ int compact_group(const FastArgs &f, int row, int li,
         for (int t = 0; t < 8; ++t) kp[t] = rec[t] ? __ldg(rec[t]) : make_uint2(0u, 0u);
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
-            const int r = base + t * kFinThreads + (int)threadIdx.x;
+            const int r = base + t * THREADS + (int)threadIdx.x;
             if (rec[t]) {
                 ckey[done + r] = kp[t].x;
                 cidx[done + r] = tile0[t] + (int)kp[t].y;
@@ -622,7 +631,7 @@ __global__ void __launch_bounds__(kFinThreads) compact_groups_kernel(FastArgs f)
     const int gn = c1 - g.gb < kFinGroup ? c1 - g.gb : kFinGroup;
     uint32_t *ckey = f.comp_key + (int64_t)row * f.comp_total + f.comp_off[g.li];
     int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[g.li];
-    const int added = compact_group(f, row, g.li, g.gb, gn, (int)before, ckey, cidx, group_off, warp_u);
+    const int added = compact_group<kFinThreads>(f, row, g.li, g.gb, gn, (int)before, ckey, cidx, group_off, warp_u);
     if (threadIdx.x == 0) {
         f.job_range[g.rec] = make_int2((int)before, added);
         if ((int64_t)before + added > (int64_t)v.m) atomicExch(f.errword, 0x5E71);
@@ -754,7 +763,7 @@ __global__ void __launch_bounds__(kFinThreads) wide_emit_kernel(FastArgs f)
     if (gt0 + (eq0 < r ? eq0 : r) < k) {
         const int64_t base = (int64_t)row * f.comp_total + f.comp_off[g.li] + range.x;
         CompactSource src{f.comp_key + base, f.comp_idx + base, range.y};
-        emit_ordered(src, T, r, gt0, eq0, k, f.out + (int64_t)row * f.out_stride + f.seg_out[s], sh, f.errword);
+        emit_ordered<kFinThreads>(src, T, r, gt0, eq0, k, f.out + (int64_t)row * f.out_stride + f.seg_out[s], sh, f.errword);
     }
     if (g.job == 0 && threadIdx.x == 0) {
         f.seg_m[g.slot] = (int)m;
@@ -774,13 +783,14 @@ __global__ void __launch_bounds__(kFinThreads) wide_emit_kernel(FastArgs f)
 //  3. stores the key from which the next step should collect candidates.
 // CTA order: large segments longest first, then the small ones, then spare CTAs that clear the
 // dense update buffer (if the caller announced it) while the rest of the launch is busy.
-__global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS) finish_kernel(FastArgs f)
 {
     __shared__ FinishShared sh;
     __shared__ SmallShared small_sh;
     __shared__ unsigned full_hist[kHistBins];
     __shared__ int group_off[kFinGroup];
-    extern __shared__ __align__(16) uint32_t fin_dyn[];     // kFinSmemCap candidate keys
+    extern __shared__ __align__(16) uint32_t fin_dyn[];     // f.smem_keys candidate keys
     const int row = blockIdx.y;
     if ((int)blockIdx.x >= f.num_large + f.fin_small) {      // spare CTAs: clear the dense update meanwhile
         if (row != 0) return;
@@ -828,9 +838,9 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
     if (lists) {
         path = settled ? 1 : 0;
         // 2. compaction.  Keys stay in shared memory when they fit; offsets are needed only for the winners.
-        uint32_t *ckey = m <= kFinSmemCap ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
+        uint32_t *ckey = m <= f.smem_keys ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
         int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
-        const int done = compact_group(f, row, li, c0, c1 - c0, 0, ckey, cidx, group_off, sh.warp_u);
+        const int done = compact_group<THREADS>(f, row, li, c0, c1 - c0, 0, ckey, cidx, group_off, sh.warp_u);
         if (threadIdx.x == 0 && done != m) atomicExch(f.errword, 0x5E70);
         // 3. the bucket of the k-th key: from path (b), or from the candidates' own leading digits
         // (every entry at or above the predicted key is a candidate, and there are at least k)
@@ -838,17 +848,17 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
             d0 = f.prefix[slot];
             k_rem = f.k_rem[slot];
         } else {
-            for (int b = threadIdx.x; b < kHistBins; b += kFinThreads) full_hist[b] = 0;
+            for (int b = threadIdx.x; b < kHistBins; b += THREADS) full_hist[b] = 0;
             __syncthreads();
-            for (int i = threadIdx.x; i < m; i += kFinThreads) atomicAdd(&full_hist[ckey[i] >> 20], 1u);
+            for (int i = threadIdx.x; i < m; i += THREADS) atomicAdd(&full_hist[ckey[i] >> 20], 1u);
             __syncthreads();
-            digit_scan(full_hist, k, sh);
+            digit_scan<THREADS>(full_hist, k, sh);
             d0 = (uint32_t)sh.found[0];
             k_rem = sh.found[1];
         }
         __syncthreads();
         CompactSource src{ckey, cidx, m};
-        T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
+        T = finish_from<THREADS>(src, d0, k_rem, k, out, sh, f.errword);
     } else {
         // no lists for this step, a chunk list overflowed, too many candidates, or a prediction
         // that turned out too high: work on the data
@@ -859,9 +869,9 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
         } else {
             path = 2;
             // first read of the segment: its complete leading-digit histogram
-            for (int b = threadIdx.x; b < kHistBins; b += kFinThreads) full_hist[b] = 0;
+            for (int b = threadIdx.x; b < kHistBins; b += THREADS) full_hist[b] = 0;
             __syncthreads();
-            constexpr int kTile = kFinThreads * kSelPerThread;
+            constexpr int kTile = THREADS * kSelPerThread;
             for (int base = 0; base < len; base += kTile) {
                 uint32_t key[kSelPerThread];
                 const int valid = load_keys16(rowp + off, base, len, key);
@@ -870,7 +880,7 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
                     if (i < valid) atomicAdd(&full_hist[key[i] >> 20], 1u);
             }
             __syncthreads();
-            digit_scan(full_hist, k, sh);
+            digit_scan<THREADS>(full_hist, k, sh);
             d0 = (uint32_t)sh.found[0];
             k_rem = sh.found[1];
             const int64_t at_or_above = (int64_t)(k - k_rem) + (int64_t)full_hist[d0];
@@ -878,7 +888,7 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
             if (at_or_above <= cap) {
                 // second read: the entries from the bucket upwards, compacted in index order
                 const int mm = (int)at_or_above;
-                uint32_t *ckey = mm <= kFinSmemCap ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
+                uint32_t *ckey = mm <= f.smem_keys ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
                 int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
                 int done = 0;
                 for (int base = 0; base < len; base += kTile) {
@@ -904,13 +914,13 @@ __global__ void __launch_bounds__(kFinThreads) finish_kernel(FastArgs f)
                 if (threadIdx.x == 0 && done != mm) atomicExch(f.errword, 0x5E80);
                 __syncthreads();
                 CompactSource src{ckey, cidx, mm};
-                T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
+                T = finish_from<THREADS>(src, d0, k_rem, k, out, sh, f.errword);
                 goto finished;
             }
         }
         {
             DataSource src{rowp + off, off, len};
-            T = finish_from(src, d0, k_rem, k, out, sh, f.errword);
+            T = finish_from<THREADS>(src, d0, k_rem, k, out, sh, f.errword);
         }
     }
 finished:
@@ -1051,6 +1061,7 @@ void fill_args(FastArgs &f, const SelectTables &t, const float *data, int64_t ro
     f.data = data; f.row_stride = row_stride; f.row0 = row0;
     f.num_large = t.num_large; f.num_small = t.num_small; f.num_tchunks = t.num_tchunks; f.epoch = epoch;
     f.fin_small = 0;
+    f.smem_keys = 0;
     f.large_order = t.large_order; f.group_job = t.group_job; f.num_group_jobs = t.num_group_jobs;
     f.job_range = t.job_range; f.job_cnt = t.job_cnt; f.seg_wide = t.seg_wide; f.zero_ptr = nullptr; f.zero_vecs = 0; f.zero_tail = 0; f.zero_ctas = 0; f.zero_threads = 0;
     f.seg_off = t.seg_off; f.seg_len = t.seg_len; f.seg_k = t.seg_k; f.seg_out = t.seg_out;
@@ -1082,11 +1093,19 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
     if (rows <= 0 || t.num_segments == 0) return cudaSuccess;
     FastArgs f;
     fill_args(f, t, data, row_stride, row0, out, out_stride, epoch, errword);
-    constexpr int kFinDyn = kFinSmemCap * (int)sizeof(uint32_t);
+    // the finishing launch's shape (see kFinThreads above)
+    const int64_t large_jobs = (int64_t)rows * t.num_large;
+    const int fin_threads = large_jobs <= sm_count() ? 1024 : large_jobs > 4 * (int64_t)sm_count() ? 256 : kFinThreads;
+    f.smem_keys = fin_threads == 256 ? kFinSmemCapSmall : kFinSmemCap;
+    const int fin_dyn = f.smem_keys * (int)sizeof(uint32_t);
     static OncePerDevice configured;
     {
-        const cudaError_t e = configured.run(
-            [] { return cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinDyn); });
+        const cudaError_t e = configured.run([] {
+            cudaError_t x = cudaFuncSetAttribute(finish_kernel<1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinSmemCap * 4);
+            if (x == cudaSuccess) x = cudaFuncSetAttribute(finish_kernel<kFinThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinSmemCap * 4);
+            if (x == cudaSuccess) x = cudaFuncSetAttribute(finish_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinSmemCapSmall * 4);
+            return x;
+        });
         if (e != cudaSuccess) return e;
     }
     if (t.num_large && !served) {
@@ -1125,16 +1144,24 @@ cudaError_t launch_select(const SelectTables &t, const float *data, int64_t row_
         f.zero_ptr = reinterpret_cast<uint4 *>(clear);
         f.zero_vecs = (uint64_t)clear_floats >> 2;
         f.zero_tail = (int)(clear_floats & 3);
-        f.zero_threads = f.zero_vecs * 16 <= kZeroGentleBytes ? kZeroGentleThreads : kFinThreads;
-        const uint64_t per_cta = (uint64_t)f.zero_threads * (f.zero_threads == kFinThreads ? kZeroPerThreadFast : kZeroPerThread);
+        // (a 1024-thread finishing CTA has its SM to itself, registers and all: the clearing CTAs run on other SMs
+        // and need not be gentle)
+        const bool gentle = f.zero_vecs * 16 <= kZeroGentleBytes && fin_threads != 1024;
+        f.zero_threads = gentle ? kZeroGentleThreads : fin_threads;
+        const uint64_t per_cta = (uint64_t)f.zero_threads * (gentle ? kZeroPerThread : kZeroPerThreadFast);
         uint64_t ctas = (f.zero_vecs + 1 + per_cta - 1) / per_cta;
         if (ctas < (uint64_t)kZeroCtasMin) ctas = (f.zero_vecs + 1 + f.zero_threads - 1) / f.zero_threads < (uint64_t)kZeroCtasMin
                                                       ? (f.zero_vecs + 1 + f.zero_threads - 1) / f.zero_threads : (uint64_t)kZeroCtasMin;
         spare = (unsigned)ctas;
         f.zero_ctas = (int)spare;
     }
-    if (t.num_large + f.fin_small)
-        finish_kernel<<<dim3(t.num_large + f.fin_small + spare, rows), kFinThreads, kFinDyn, st>>>(f), ++g_kernel_launches;
+    if (t.num_large + f.fin_small) {
+        const dim3 grid(t.num_large + f.fin_small + spare, rows);
+        if (fin_threads == 1024) finish_kernel<1024><<<grid, 1024, fin_dyn, st>>>(f);
+        else if (fin_threads == 256) finish_kernel<256><<<grid, 256, fin_dyn, st>>>(f);
+        else finish_kernel<kFinThreads><<<grid, kFinThreads, fin_dyn, st>>>(f);
+        ++g_kernel_launches;
+    }
     if (forked) {
         const cudaError_t e = cudaStreamWaitEvent(st, join, 0);
         if (e != cudaSuccess) return e;
