@@ -74,14 +74,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-
 // Shared-memory matrix descriptor of a K-major tile of 128-byte rows, 128-byte swizzle: rows of
 // one 8-row group are 128 bytes apart, groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr)
@@ -260,7 +252,8 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
                 const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
                 const float *__restrict__ bias, int64_t L_out, int64_t Lpad_out, float *__restrict__ out_hi,
                 float *__restrict__ out_lo, const float *__restrict__ w_last, const float *__restrict__ b_last,
-                float *__restrict__ out_last, const float *__restrict__ extra, int32_t *errword)
+                float *__restrict__ out_last, const float *__restrict__ extra, int32_t *errword, int wz0, int wz_step,
+                int64_t param_stride)
 {
     using S = GemmShape<MODE, CIN, COUT>;
     constexpr int N = S::kN;
@@ -275,6 +268,14 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
     const int node = blockIdx.y;
     const int t0 = blockIdx.x * kTileM;
     const uint32_t tiles = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+    // blockIdx.y is the node (encoder: one set of weights, wz_step = 0) or the decoder (parameter server: decoder
+    // y has its own weights, slice wz0 + y of the weight maps, and its own biases param_stride floats further on)
+    const int wz = wz0 + node * wz_step;
+    bias += (int64_t)node * param_stride;
+    if (MODE == kConvCode || MODE == kDeconvFinal) {
+        w_last += (int64_t)node * param_stride;
+        b_last += (int64_t)node * param_stride;
+    }
 
     if (MODE != kGradDeconv)
         for (int i = threadIdx.x; i < COUT; i += 128) s_bias[i] = bias[i];
@@ -331,8 +332,8 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
             }
             tma_load_3d(st, &map_a_hi, bar, col, row, node);
             tma_load_3d(st + S::kABytes, &map_a_lo, bar, col, row, node);
-            tma_load_2d(st + 2 * S::kABytes, &map_b_hi, bar, c, 0);
-            tma_load_2d(st + 2 * S::kABytes + S::kBBytes, &map_b_lo, bar, c, 0);
+            tma_load_3d(st + 2 * S::kABytes, &map_b_hi, bar, c, 0, wz);
+            tma_load_3d(st + 2 * S::kABytes + S::kBBytes, &map_b_lo, bar, c, 0, wz);
         }
     } else if (threadIdx.x == 32) {
         // instruction descriptor: fp32 accumulator, tf32 x tf32, both operands K-major, N columns, M = 128
@@ -450,13 +451,14 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
                 make_float4(__fadd_rn(last[0], s_bl[0]), __fadd_rn(last[1], s_bl[1]), __fadd_rn(last[2], s_bl[2]),
                             __fadd_rn(last[3], s_bl[3]));
         if (MODE == kDeconvFinal) {
+            const int64_t row0 = (int64_t)node * L_out;              // decoder `node` reconstructs row `node`
             if (2 * t < L_out) {
                 const float y = __fadd_rn(last[0], s_bl[0]);
-                out_last[2 * t] = extra ? __fmaf_rn(s_bl[1], extra[2 * t], y) : y;
+                out_last[row0 + 2 * t] = extra ? __fmaf_rn(s_bl[1], extra[row0 + 2 * t], y) : y;
             }
             if (2 * t + 1 < L_out) {
                 const float y = __fadd_rn(last[1], s_bl[0]);
-                out_last[2 * t + 1] = extra ? __fmaf_rn(s_bl[1], extra[2 * t + 1], y) : y;
+                out_last[row0 + 2 * t + 1] = extra ? __fmaf_rn(s_bl[1], extra[row0 + 2 * t + 1], y) : y;
             }
         }
     } else if (threadIdx.x == 0) {
@@ -472,11 +474,15 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
 // Decoder (one pass, fp32 pipes), channels-last.
 // ------------------------------------------------------------------------------------------
 // deconv1: ConvTranspose1d(4 -> 4, k3, stride 1, padding 1) + leaky ReLU on the mean code.
+// blockIdx.y: the decoder (its parameters lie param_stride floats after the previous one's, its output L4 rows on).
 __global__ void ae5_deconv1_kernel(const float *__restrict__ z, int64_t L4, const float *__restrict__ w,
-                                   const float *__restrict__ b, float *__restrict__ out)
+                                   const float *__restrict__ b, float *__restrict__ out, int64_t param_stride)
 {
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= L4) return;
+    w += (int64_t)blockIdx.y * param_stride;
+    b += (int64_t)blockIdx.y * param_stride;
+    out += (int64_t)blockIdx.y * L4 * 4;
     float acc[4] = {b[0], b[1], b[2], b[3]};
 #pragma unroll
     for (int tau = 0; tau < 3; ++tau) {
@@ -500,9 +506,14 @@ __global__ void ae5_deconv1_kernel(const float *__restrict__ z, int64_t L4, cons
 template <int CIN, int COUT, int TP>
 __global__ void __launch_bounds__(256)
 ae5_deconv_kernel(const float *__restrict__ x, int64_t L_in, int64_t L_out, const float *__restrict__ w,
-                  const float *__restrict__ b, float *__restrict__ y, float *__restrict__ y_lo)
+                  const float *__restrict__ b, float *__restrict__ y, float *__restrict__ y_lo, int64_t param_stride)
 {
     extern __shared__ float dsm[];
+    x += (int64_t)blockIdx.y * L_in * CIN;                  // blockIdx.y: the decoder
+    w += (int64_t)blockIdx.y * param_stride;
+    b += (int64_t)blockIdx.y * param_stride;
+    y += (int64_t)blockIdx.y * L_out * COUT;
+    y_lo += (int64_t)blockIdx.y * L_out * COUT;
     float *sw = dsm;                          // [tau][ci][co]
     float *sx = dsm + 3 * CIN * COUT;         // [TP + 1][CIN]: rows j0 - 1 .. j0 + TP - 1
     const int64_t j0 = (int64_t)blockIdx.x * TP;
@@ -570,24 +581,24 @@ bool make_act_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int C, int64_t
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-// Decoder activation [L][C] seen as [1][L][C]; box: 32 floats x 128 rows.
-bool make_dact_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int C, int64_t L)
+// Decoder activations [decoders][L][C]; box: 32 floats x 128 rows of one decoder.
+bool make_dact_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int C, int64_t L, int decoders)
 {
-    const cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)L, 1};
+    const cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)L, (cuuint64_t)decoders};
     const cuuint64_t strides[2] = {(cuuint64_t)C * 4, (cuuint64_t)L * C * 4};
     const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileM, 1};
     const cuuint32_t es[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-// GEMM weights [rows][k]; box: 32 floats x all rows.
-bool make_matrix_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int k, int rows)
+// GEMM weights [count][rows][k] (count sets of weights back to back); box: 32 floats x all rows of one set.
+bool make_matrix_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int k, int rows, int count = 1)
 {
-    const cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)k * 4};
-    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)rows};
-    const cuuint32_t es[2] = {1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    const cuuint64_t dims[3] = {(cuuint64_t)k, (cuuint64_t)rows, (cuuint64_t)count};
+    const cuuint64_t strides[2] = {(cuuint64_t)k * 4, (cuuint64_t)k * rows * 4};
+    const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)rows, 1};
+    const cuuint32_t es[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -595,7 +606,7 @@ template <int MODE, int CIN, int COUT>
 cudaError_t launch_gemm(Ctx &c, const CUtensorMap &a_hi, const CUtensorMap &a_lo, const CUtensorMap &b_hi,
                         const CUtensorMap &b_lo, const float *bias, int64_t rows, int nodes, int64_t L_out, int64_t Lpad_out,
                         float *out_hi, float *out_lo, const float *w_last, const float *b_last, float *out_last,
-                        const float *extra = nullptr)
+                        const float *extra = nullptr, int wz0 = 0, int wz_step = 0, int64_t param_stride = 0)
 {
     using S = GemmShape<MODE, CIN, COUT>;
     auto kern = ae5_gemm_kernel<MODE, CIN, COUT>;
@@ -606,7 +617,8 @@ cudaError_t launch_gemm(Ctx &c, const CUtensorMap &a_hi, const CUtensorMap &a_lo
         if (e != cudaSuccess) return e;
     }
     kern<<<dim3(blocks(rows, kTileM), nodes), 128, S::kSmemBytes, c.stream>>>(a_hi, a_lo, b_hi, b_lo, bias, L_out, Lpad_out, out_hi,
-                                                                              out_lo, w_last, b_last, out_last, extra, c.errword),
+                                                                              out_lo, w_last, b_last, out_last, extra, c.errword, wz0,
+                                                                              wz_step, param_stride),
         ++g_kernel_launches;
     return cudaGetLastError();
 }
@@ -665,9 +677,9 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         a.w_hi[l] = take(n);
         a.w_lo[l] = take(n);
     }
-    a.d0 = take((size_t)a.len[4] * 4);
-    for (int l = 0; l < 3; ++l) {                           // outputs of deconv2..deconv4: lengths L3, L2, L1
-        const size_t n = (size_t)a.len[3 - l] * kAe5DecCh[l + 2];
+    a.d0 = take((size_t)a.decoders * a.len[4] * 4);
+    for (int l = 0; l < 3; ++l) {                           // outputs of deconv2..deconv4 of every decoder: lengths L3, L2, L1
+        const size_t n = (size_t)a.decoders * a.len[3 - l] * kAe5DecCh[l + 2];
         a.dact_hi[l] = take(n);
         a.dact_lo[l] = take(n);
     }
@@ -764,8 +776,8 @@ cudaError_t ae5_make_maps(Ctx &c)
         ok = ok && make_matrix_map(enc, &a.map_w_hi[l], a.w_hi[l], 3 * cin, cout);
         ok = ok && make_matrix_map(enc, &a.map_w_lo[l], a.w_lo[l], 3 * cin, cout);
         const int dcin = kAe5DecCh[l + 2];
-        ok = ok && make_dact_map(enc, &a.map_dact_hi[l], a.dact_hi[l], dcin, a.len[3 - l]);
-        ok = ok && make_dact_map(enc, &a.map_dact_lo[l], a.dact_lo[l], dcin, a.len[3 - l]);
+        ok = ok && make_dact_map(enc, &a.map_dact_hi[l], a.dact_hi[l], dcin, a.len[3 - l], a.decoders);
+        ok = ok && make_dact_map(enc, &a.map_dact_lo[l], a.dact_lo[l], dcin, a.len[3 - l], a.decoders);
     }
     for (int j = 0; j < 2; ++j) {            // input-gradient GEMMs of conv2 and conv3: A = the gradient at the layer's output
         const int C = kAe5EncCh[j + 2], cin = kAe5EncCh[j + 1];
@@ -780,15 +792,13 @@ cudaError_t ae5_make_maps(Ctx &c)
         ok = ok && make_matrix_map(enc, &a.map_gw_hi[j], a.gw_hi[j], 2 * C, 2 * cin);
         ok = ok && make_matrix_map(enc, &a.map_gw_lo[j], a.gw_lo[j], 2 * C, 2 * cin);
     }
-    a.map_dw_hi.resize((size_t)a.decoders * 3);
-    a.map_dw_lo.resize((size_t)a.decoders * 3);
-    for (int d = 0; d < a.decoders; ++d)
-        for (int l = 0; l < 3; ++l) {
-            const int dcin = kAe5DecCh[l + 2], dcout = kAe5DecCh[l + 3];
-            const size_t at = (size_t)d * 4 * dcin * dcout;
-            ok = ok && make_matrix_map(enc, &a.map_dw_hi[d * 3 + l], a.dw_hi[l] + at, 2 * dcin, 2 * dcout);
-            ok = ok && make_matrix_map(enc, &a.map_dw_lo[d * 3 + l], a.dw_lo[l] + at, 2 * dcin, 2 * dcout);
-        }
+    a.map_dw_hi.resize(3);                   // one map per layer: slice d holds decoder d's weights
+    a.map_dw_lo.resize(3);
+    for (int l = 0; l < 3; ++l) {
+        const int dcin = kAe5DecCh[l + 2], dcout = kAe5DecCh[l + 3];
+        ok = ok && make_matrix_map(enc, &a.map_dw_hi[l], a.dw_hi[l], 2 * dcin, 2 * dcout, a.decoders);
+        ok = ok && make_matrix_map(enc, &a.map_dw_lo[l], a.dw_lo[l], 2 * dcin, 2 * dcout, a.decoders);
+    }
     return ok ? cudaSuccess : cudaErrorInvalidValue;
 }
 
@@ -898,23 +908,23 @@ cudaError_t launch_ae5_train_decode(Ctx &c, int d)
 {
     Ae5 &a = *c.ae5;
     const float *P = c.params + d * a.dec_stride;
-    ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0),
+    ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0, 0),
         ++g_kernel_launches;
     constexpr int kTp = 64, kSmem2 = (3 * 4 * 32 + (kTp + 1) * 4) * 4;
     ae5_deconv_kernel<4, 32, kTp><<<blocks(a.len[4] + 1, kTp), 256, kSmem2, c.stream>>>(a.d0, a.len[4], a.len[3], P + a.off_dw[1],
-                                                                                        P + a.off_db[1], a.dact_hi[0], a.dact_lo[0]),
+                                                                                        P + a.off_db[1], a.dact_hi[0], a.dact_lo[0], 0),
         ++g_kernel_launches;
     cudaError_t e = cudaGetLastError();
-    const CUtensorMap *whi = &a.map_dw_hi[d * 3], *wlo = &a.map_dw_lo[d * 3];
+    // the first slice of the activation buffers, slice d of the weights
     if (e == cudaSuccess)
-        e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], whi[0], wlo[0], P + a.off_db[2],
-                                         a.len[3] + 1, 1, a.len[2], 0, a.dact_hi[1], a.dact_lo[1], nullptr, nullptr, nullptr);
+        e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], a.map_dw_hi[0], a.map_dw_lo[0], P + a.off_db[2],
+                                         a.len[3] + 1, 1, a.len[2], 0, a.dact_hi[1], a.dact_lo[1], nullptr, nullptr, nullptr, nullptr, d);
     if (e == cudaSuccess)
-        e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], whi[1], wlo[1], P + a.off_db[3],
-                                          a.len[2] + 1, 1, a.len[1], 0, a.dact_hi[2], a.dact_lo[2], nullptr, nullptr, nullptr);
+        e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], a.map_dw_hi[1], a.map_dw_lo[1], P + a.off_db[3],
+                                          a.len[2] + 1, 1, a.len[1], 0, a.dact_hi[2], a.dact_lo[2], nullptr, nullptr, nullptr, nullptr, d);
     if (e == cudaSuccess)
-        e = launch_gemm<kDeconv, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], whi[2], wlo[2], P + a.off_db[4],
-                                          a.len[1] + 1, 1, a.len[0], 0, a.dact5_hi, a.dact5_lo, nullptr, nullptr, nullptr);
+        e = launch_gemm<kDeconv, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], a.map_dw_hi[2], a.map_dw_lo[2], P + a.off_db[4],
+                                          a.len[1] + 1, 1, a.len[0], 0, a.dact5_hi, a.dact5_lo, nullptr, nullptr, nullptr, nullptr, d);
     return e;
 }
 
@@ -949,38 +959,39 @@ cudaError_t launch_ae5_input_gradient(Ctx &c, int layer)
 
 // Stage 5 up to the reconstruction.  Ring-allreduce: the decoder on the mean code; c.recon gets the mu
 // values.  Parameter server (Section IV-A): node k's decoder on the common code, its innovation as the 33rd
-// input of the last convolution; c.recon gets [K][mu].  The decoders run one after the other through the
-// same activation buffers (each pass fills the device at the benchmark sizes).
+// input of the last convolution; c.recon gets [K][mu].  Every layer is ONE launch over all decoders
+// (blockIdx.y = decoder: its own weights, its own slice of the activation buffers), so that the K decoders'
+// tiles fill the device together.
 cudaError_t launch_ae5_decode(Ctx &c)
 {
     Ae5 &a = *c.ae5;
     prepare_weights(c);
     const bool ps = c.cfg.variant == LGC_VARIANT_PS;
-    cudaError_t e = cudaSuccess;
-    for (int d = 0; d < a.decoders && e == cudaSuccess; ++d) {
-        const float *P = c.params + d * a.dec_stride;          // decoder d's tensors sit at the offsets of decoder 0 from here
-        ae5_deconv1_kernel<<<blocks(a.len[4], 128), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0),
-            ++g_kernel_launches;
-        // deconv2 (4 -> 32): too narrow for the tensor cores
-        constexpr int kTp = 64, kSmem2 = (3 * 4 * 32 + (kTp + 1) * 4) * 4;
-        ae5_deconv_kernel<4, 32, kTp><<<blocks(a.len[4] + 1, kTp), 256, kSmem2, c.stream>>>(a.d0, a.len[4], a.len[3], P + a.off_dw[1],
-                                                                                            P + a.off_db[1], a.dact_hi[0], a.dact_lo[0]),
-            ++g_kernel_launches;
-        e = cudaGetLastError();
-        const CUtensorMap *whi = &a.map_dw_hi[d * 3], *wlo = &a.map_dw_lo[d * 3];
-        // deconv3..5: rows j = 0 .. L_in (one more than the input positions: the last makes the tail)
-        if (e == cudaSuccess)
-            e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], whi[0], wlo[0], P + a.off_db[2],
-                                             a.len[3] + 1, 1, a.len[2], 0, a.dact_hi[1], a.dact_lo[1], nullptr, nullptr, nullptr);
-        if (e == cudaSuccess)
-            e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], whi[1], wlo[1], P + a.off_db[3],
-                                              a.len[2] + 1, 1, a.len[1], 0, a.dact_hi[2], a.dact_lo[2], nullptr, nullptr, nullptr);
-        if (e == cudaSuccess)
-            e = launch_gemm<kDeconvFinal, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], whi[2], wlo[2], P + a.off_db[4],
-                                                   a.len[1] + 1, 1, a.len[0], 0, nullptr, nullptr, P + a.off_dw[5],
-                                                   P + a.off_db[5], c.recon + (int64_t)d * c.mu,
-                                                   ps ? c.inn + (int64_t)d * c.mu : nullptr);
-    }
+    const float *P = c.params;                                 // decoder d's tensors: dec_stride floats per decoder further on
+    const int D = a.decoders;
+    const int64_t ps_stride = a.dec_stride;
+    ae5_deconv1_kernel<<<dim3(blocks(a.len[4], 128), D), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0,
+                                                                             ps_stride),
+        ++g_kernel_launches;
+    // deconv2 (4 -> 32): too narrow for the tensor cores
+    constexpr int kTp = 64, kSmem2 = (3 * 4 * 32 + (kTp + 1) * 4) * 4;
+    ae5_deconv_kernel<4, 32, kTp><<<dim3(blocks(a.len[4] + 1, kTp), D), 256, kSmem2, c.stream>>>(
+        a.d0, a.len[4], a.len[3], P + a.off_dw[1], P + a.off_db[1], a.dact_hi[0], a.dact_lo[0], ps_stride),
+        ++g_kernel_launches;
+    cudaError_t e = cudaGetLastError();
+    // deconv3..5: rows j = 0 .. L_in (one more than the input positions: the last makes the tail)
+    if (e == cudaSuccess)
+        e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], a.map_dw_hi[0], a.map_dw_lo[0], P + a.off_db[2],
+                                         a.len[3] + 1, D, a.len[2], a.len[2], a.dact_hi[1], a.dact_lo[1], nullptr, nullptr, nullptr,
+                                         nullptr, 0, 1, ps_stride);
+    if (e == cudaSuccess)
+        e = launch_gemm<kDeconv, 64, 128>(c, a.map_dact_hi[1], a.map_dact_lo[1], a.map_dw_hi[1], a.map_dw_lo[1], P + a.off_db[3],
+                                          a.len[2] + 1, D, a.len[1], a.len[1], a.dact_hi[2], a.dact_lo[2], nullptr, nullptr, nullptr,
+                                          nullptr, 0, 1, ps_stride);
+    if (e == cudaSuccess)
+        e = launch_gemm<kDeconvFinal, 128, 32>(c, a.map_dact_hi[2], a.map_dact_lo[2], a.map_dw_hi[2], a.map_dw_lo[2], P + a.off_db[4],
+                                               a.len[1] + 1, D, a.len[0], 0, nullptr, nullptr, P + a.off_dw[5], P + a.off_db[5],
+                                               c.recon, ps ? c.inn : nullptr, 0, 1, ps_stride);
     return e;
 }
 
