@@ -50,23 +50,6 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Waits for the phase of the given parity to complete; false if it did not within the limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    for (int i = 0; i < kSpinLimit; ++i) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-    }
-    return false;
-}
-
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2)
 {
     asm volatile(
@@ -234,74 +217,88 @@ template <int MODE, int CIN, int COUT>
 struct GemmShape {
     static constexpr bool kIsConv = MODE == kConv || MODE == kConvCode;
     static constexpr int kK = kIsConv ? 3 * CIN : 2 * CIN;      // operands per row
-    static constexpr int kN = kIsConv ? COUT : 2 * COUT;        // accumulator columns
+    static constexpr int kN = kIsConv ? COUT : 2 * COUT;        // columns of the layer's GEMM
+    static constexpr int kNT = kN > 128 ? 128 : kN;             // columns of one tile: wider layers are cut in two along N
+    static constexpr int kNSplit = kN / kNT;
     static constexpr int kBlocks = kK / kBlockK;
     static constexpr int kABytes = kTileM * kBlockK * 4;        // one (hi or lo) activation tile of a k-block
-    static constexpr int kBBytes = kN * kBlockK * 4;
+    static constexpr int kBBytes = kNT * kBlockK * 4;
     static constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;
-    // as many stages as fit (one CTA per SM; two CTAs of half the stages each measured slower)
-    static constexpr int kStages = (200 * 1024) / kStageBytes < kBlocks ? (200 * 1024) / kStageBytes : kBlocks;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024;   // + slack to align the tiles to 1024 bytes
-    static_assert(kStages * kStageBytes >= 4 * 2 * 32 * kStagePitch * 4, "the epilogue stages its blocks in the operand area");
-    static_assert(kN >= 32 && kN <= 256 && (kN & (kN - 1)) == 0, "accumulator columns: a power of two in [32, 256]");
+    static constexpr int kEpiBytes = 4 * 32 * kStagePitch * 4;  // one 32 x 32 staging block per epilogue warp
+    // as many stages as fit beside the staging blocks (one CTA per SM)
+    static constexpr int kFit = (218 * 1024 - kEpiBytes) / kStageBytes;
+    static constexpr int kStages = kFit < kBlocks ? kFit : kBlocks;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024;   // + slack to align the tiles to 1024 bytes
+    static constexpr int kTmemCols = 2 * kNT;                   // two accumulators: one is drained while the other fills
+    static_assert(kNT >= 32 && kNT <= 128 && (kNT & (kNT - 1)) == 0 && kN % kNT == 0, "tile columns: a power of two in [32, 128]");
+    static_assert(kStages >= 1, "a stage must fit");
 };
 
+constexpr int kGemmThreads = 192;     // warp 0: TMA loads, warp 1: tensor memory + MMA issue, warps 2..5: epilogue
+
+// Polls the barrier; gives up when the limit is reached or another role has given up (then *failed is set).
+__device__ __forceinline__ bool mbar_wait_shared(uint32_t bar, uint32_t parity, volatile int *failed)
+{
+    for (int i = 0; i < kSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if ((i & 255) == 255 && *failed) return false;
+    }
+    *failed = 1;
+    return false;
+}
+
+// The kernel is persistent: a CTA takes tiles blockIdx.x, blockIdx.x + gridDim.x, ... of the layer's
+// nodes x row tiles x column halves.  One thread keeps the TMA loads going through a ring of stages, one
+// thread issues the MMAs of a tile into one of two accumulators in tensor memory, and four epilogue warps
+// drain the other accumulator meanwhile (warp w reads the 32 lanes of tensor memory its number lets it
+// reach: quarter w % 4).  Every wait is bounded; a role that gives up tells the others through `failed`,
+// everybody leaves through the common exit, and tensor memory is released.
 template <int MODE, int CIN, int COUT>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kGemmThreads)
 ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                 const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
-                const float *__restrict__ bias, int64_t L_out, int64_t Lpad_out, float *__restrict__ out_hi,
-                float *__restrict__ out_lo, const float *__restrict__ w_last, const float *__restrict__ b_last,
-                float *__restrict__ out_last, const float *__restrict__ extra, int32_t *errword, int wz0, int wz_step,
-                int64_t param_stride)
+                const float *__restrict__ bias, int tiles_x, int nodes, int64_t L_out, int64_t Lpad_out,
+                float *__restrict__ out_hi, float *__restrict__ out_lo, const float *__restrict__ w_last,
+                const float *__restrict__ b_last, float *__restrict__ out_last, const float *__restrict__ extra,
+                int32_t *errword, int wz0, int wz_step, int64_t param_stride)
 {
     using S = GemmShape<MODE, CIN, COUT>;
-    constexpr int N = S::kN;
+    constexpr int NT = S::kNT;
     extern __shared__ uint8_t dyn_smem[];
-    __shared__ __align__(8) uint64_t full_bar[S::kStages], empty_bar[S::kStages], accum_bar;
+    __shared__ __align__(8) uint64_t full_bar[S::kStages], empty_bar[S::kStages], tfull_bar[2], tempty_bar[2];
     __shared__ uint32_t tmem_base_smem;
-    __shared__ int failed;
-    __shared__ float s_bias[COUT];
-    __shared__ float s_wl[MODE == kConvCode ? 4 * 64 : 32], s_bl[4];
+    __shared__ volatile int failed;
+    // every epilogue warp keeps its own copy of the node's small tensors: no barrier between the warps
+    __shared__ float s_bias[4][COUT];
+    __shared__ float s_wl[4][MODE == kConvCode ? 4 * 64 : 32], s_bl[4][4];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int node = blockIdx.y;
-    const int t0 = blockIdx.x * kTileM;
     const uint32_t tiles = (smem_u32(dyn_smem) + 1023u) & ~1023u;
-    // blockIdx.y is the node (encoder: one set of weights, wz_step = 0) or the decoder (parameter server: decoder
-    // y has its own weights, slice wz0 + y of the weight maps, and its own biases param_stride floats further on)
-    const int wz = wz0 + node * wz_step;
-    bias += (int64_t)node * param_stride;
-    if (MODE == kConvCode || MODE == kDeconvFinal) {
-        w_last += (int64_t)node * param_stride;
-        b_last += (int64_t)node * param_stride;
-    }
+    const int total = tiles_x * nodes * S::kNSplit;
 
-    if (MODE != kGradDeconv)
-        for (int i = threadIdx.x; i < COUT; i += 128) s_bias[i] = bias[i];
-    if (MODE == kConvCode) {
-        for (int i = threadIdx.x; i < 4 * 64; i += 128) s_wl[i] = w_last[i];
-        if (threadIdx.x < 4) s_bl[threadIdx.x] = b_last[threadIdx.x];
-    }
-    if (MODE == kDeconvFinal) {
-        if (threadIdx.x < 32) s_wl[threadIdx.x] = w_last[threadIdx.x];
-        if (threadIdx.x == 0) {
-            s_bl[0] = b_last[0];
-            s_bl[1] = extra ? w_last[32] : 0.0f;          // parameter server: the filter's tap on the innovation channel
-        }
-    }
     if (threadIdx.x == 0) {
         failed = 0;
         for (int s = 0; s < S::kStages; ++s) {
             mbar_init(smem_u32(&full_bar[s]), 1);
             mbar_init(smem_u32(&empty_bar[s]), 1);
         }
-        mbar_init(smem_u32(&accum_bar), 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&tfull_bar[b]), 1);
+            mbar_init(smem_u32(&tempty_bar[b]), 4);               // one arrival per epilogue warp
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {                      // one warp allocates N columns of tensor memory
+    if (warp == 1) {                      // one warp allocates the two accumulators
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)),
-                     "r"((uint32_t)N)
+                     "r"((uint32_t)S::kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -312,162 +309,186 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
 
     if (threadIdx.x == 0) {
         // producer: one k-block (32 floats of the operand row) of both operands, hi and lo, per stage
-        for (int kb = 0; kb < S::kBlocks; ++kb) {
-            const int s = kb % S::kStages;
-            if (kb >= S::kStages && !mbar_wait(smem_u32(&empty_bar[s]), ((kb / S::kStages) & 1) ^ 1)) {
-                atomicExch(&failed, 1);
-                break;
+        int it = 0;                                               // k-blocks loaded so far, over all tiles
+        for (int tile = blockIdx.x; tile < total && !failed; tile += gridDim.x) {
+            const int nt = tile % S::kNSplit, tx = tile / S::kNSplit % tiles_x, node = tile / (S::kNSplit * tiles_x);
+            const int t0 = tx * kTileM, wz = wz0 + node * wz_step;
+            for (int kb = 0; kb < S::kBlocks; ++kb, ++it) {
+                const int s = it % S::kStages;
+                if (it >= S::kStages && !mbar_wait_shared(smem_u32(&empty_bar[s]), ((it / S::kStages) & 1) ^ 1, &failed)) break;
+                const uint32_t bar = smem_u32(&full_bar[s]);
+                const uint32_t st = tiles + (uint32_t)s * S::kStageBytes;
+                mbar_expect_tx(bar, S::kStageBytes);
+                const int c = kb * kBlockK;                       // column inside the operand row
+                int col, row;
+                if (S::kIsConv) {                                 // activation rows hold a pair of positions
+                    col = c < 2 * CIN ? c : c - 2 * CIN;
+                    row = c < 2 * CIN ? t0 : t0 + 1;
+                } else {                                          // activation rows hold one position: j - 1, then j
+                    col = c < CIN ? c : c - CIN;
+                    row = c < CIN ? t0 - 1 : t0;
+                }
+                tma_load_3d(st, &map_a_hi, bar, col, row, node);
+                tma_load_3d(st + S::kABytes, &map_a_lo, bar, col, row, node);
+                tma_load_3d(st + 2 * S::kABytes, &map_b_hi, bar, c, nt * NT, wz);
+                tma_load_3d(st + 2 * S::kABytes + S::kBBytes, &map_b_lo, bar, c, nt * NT, wz);
             }
-            const uint32_t bar = smem_u32(&full_bar[s]);
-            const uint32_t st = tiles + (uint32_t)s * S::kStageBytes;
-            mbar_expect_tx(bar, S::kStageBytes);
-            const int c = kb * kBlockK;                       // column inside the operand row
-            int col, row;
-            if (S::kIsConv) {                                 // activation rows hold a pair of positions
-                col = c < 2 * CIN ? c : c - 2 * CIN;
-                row = c < 2 * CIN ? t0 : t0 + 1;
-            } else {                                          // activation rows hold one position: j - 1, then j
-                col = c < CIN ? c : c - CIN;
-                row = c < CIN ? t0 - 1 : t0;
-            }
-            tma_load_3d(st, &map_a_hi, bar, col, row, node);
-            tma_load_3d(st + S::kABytes, &map_a_lo, bar, col, row, node);
-            tma_load_3d(st + 2 * S::kABytes, &map_b_hi, bar, c, 0, wz);
-            tma_load_3d(st + 2 * S::kABytes + S::kBBytes, &map_b_lo, bar, c, 0, wz);
         }
     } else if (threadIdx.x == 32) {
-        // instruction descriptor: fp32 accumulator, tf32 x tf32, both operands K-major, N columns, M = 128
-        constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-        bool ok = true;
-        for (int kb = 0; kb < S::kBlocks && ok; ++kb) {
-            const int s = kb % S::kStages;
-            if (!mbar_wait(smem_u32(&full_bar[s]), (kb / S::kStages) & 1)) {
-                atomicExch(&failed, 1);
-                ok = false;
-                break;
-            }
+        // instruction descriptor: fp32 accumulator, tf32 x tf32, both operands K-major, NT columns, M = 128
+        constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+        int it = 0, acc = 0;                                      // k-blocks consumed, tiles issued
+        for (int tile = blockIdx.x; tile < total && !failed; tile += gridDim.x, ++acc) {
+            const int buf = acc & 1;
+            // the epilogue must have drained this accumulator's previous tile
+            if (acc >= 2 && !mbar_wait_shared(smem_u32(&tempty_bar[buf]), ((acc >> 1) & 1) ^ 1, &failed)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t st = tiles + (uint32_t)s * S::kStageBytes;
-            const uint64_t a_hi = umma_desc(st), a_lo = umma_desc(st + S::kABytes);
-            const uint64_t b_hi = umma_desc(st + 2 * S::kABytes), b_lo = umma_desc(st + 2 * S::kABytes + S::kBBytes);
+            const uint32_t d = tmem + (uint32_t)(buf * NT);
+            bool ok = true;
+            for (int kb = 0; kb < S::kBlocks; ++kb, ++it) {
+                const int s = it % S::kStages;
+                if (!mbar_wait_shared(smem_u32(&full_bar[s]), (it / S::kStages) & 1, &failed)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t st = tiles + (uint32_t)s * S::kStageBytes;
+                const uint64_t a_hi = umma_desc(st), a_lo = umma_desc(st + S::kABytes);
+                const uint64_t b_hi = umma_desc(st + 2 * S::kABytes), b_lo = umma_desc(st + 2 * S::kABytes + S::kBBytes);
 #pragma unroll
-            for (int ks = 0; ks < kBlockK / 8; ++ks) {        // 8 tf32 = 32 bytes per step along K
-                const uint64_t adv = (uint64_t)(ks * 32 >> 4);
-                umma_tf32(tmem, a_hi + adv, b_hi + adv, idesc, kb > 0 || ks > 0);
-                umma_tf32(tmem, a_hi + adv, b_lo + adv, idesc, true);
-                umma_tf32(tmem, a_lo + adv, b_hi + adv, idesc, true);
-            }
-            umma_commit(smem_u32(&empty_bar[s]));             // the stage may be refilled once these have run
-        }
-        if (ok) umma_commit(smem_u32(&accum_bar));
-    }
-    __syncwarp();
-    // everyone: wait for the accumulator (or for the verdict that it will not come)
-    bool have = false;
-    if (lane == 0) {
-        for (int i = 0; i < kSpinLimit && !have; ++i) {
-            uint32_t done;
-            asm volatile(
-                "{\n\t.reg .pred p;\n\t"
-                "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
-                "selp.u32 %0, 1, 0, p;\n\t}"
-                : "=r"(done)
-                : "r"(smem_u32(&accum_bar))
-                : "memory");
-            have = done != 0;
-            if (!have && *(volatile int *)&failed) break;
-        }
-    }
-    have = __shfl_sync(0xffffffffu, have ? 1 : 0, 0) != 0;
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (have) {
-        const int64_t t = (int64_t)t0 + warp * 32 + lane;       // this thread's row
-        const uint32_t trow = tmem + ((uint32_t)(warp * 32) << 16);
-        float *stage = reinterpret_cast<float *>(dyn_smem + (tiles - smem_u32(dyn_smem)));
-        float last[4] = {0.f, 0.f, 0.f, 0.f};                   // kConvCode: the 4 code channels; kDeconvFinal: 2 positions
-#pragma unroll 1
-        for (int c0 = 0; c0 < N; c0 += 32) {
-            float x[32];
-            tmem_load32(trow + (uint32_t)c0, x);
-            const int cb = S::kIsConv ? c0 : c0 % COUT;         // channel of column c0
-            if (MODE == kGradDeconv) {
-                const int64_t pos = 2 * t + (c0 >= COUT ? 1 : 0);
-                if (pos < L_out) {
-                    const float4 *m4 = reinterpret_cast<const float4 *>(extra + ((int64_t)node * Lpad_out + pos) * COUT + cb);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const float4 m = m4[q];
-                        x[4 * q] = m.x > 0.0f ? x[4 * q] : __fmul_rn(kSlope, x[4 * q]);
-                        x[4 * q + 1] = m.y > 0.0f ? x[4 * q + 1] : __fmul_rn(kSlope, x[4 * q + 1]);
-                        x[4 * q + 2] = m.z > 0.0f ? x[4 * q + 2] : __fmul_rn(kSlope, x[4 * q + 2]);
-                        x[4 * q + 3] = m.w > 0.0f ? x[4 * q + 3] : __fmul_rn(kSlope, x[4 * q + 3]);
-                    }
+                for (int ks = 0; ks < kBlockK / 8; ++ks) {        // 8 tf32 = 32 bytes per step along K
+                    const uint64_t adv = (uint64_t)(ks * 32 >> 4);
+                    umma_tf32(d, a_hi + adv, b_hi + adv, idesc, kb > 0 || ks > 0);
+                    umma_tf32(d, a_hi + adv, b_lo + adv, idesc, true);
+                    umma_tf32(d, a_lo + adv, b_hi + adv, idesc, true);
                 }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) x[j] = leaky(__fadd_rn(x[j], s_bias[cb + j]));
+                umma_commit(smem_u32(&empty_bar[s]));             // the stage may be refilled once these have run
             }
-            if (MODE == kConvCode) {
-#pragma unroll
-                for (int o = 0; o < 4; ++o)
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) last[o] = __fmaf_rn(s_wl[o * 64 + c0 + j], x[j], last[o]);
-            } else if (MODE == kDeconvFinal) {                   // COUT = 32: columns 0..31 position 2t, 32..63 position 2t + 1
-                float acc = 0.f;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) acc = __fmaf_rn(s_wl[j], x[j], acc);
-                last[c0 / 32] = acc;
-            } else {
-                // The 32 x 32 block of this warp (row = lane) goes through shared memory so that the global
-                // stores are whole 128-byte rows: the operand stages are free once the accumulator is complete.
-                float *sh_hi = stage + warp * (2 * 32 * kStagePitch), *sh_lo = sh_hi + 32 * kStagePitch;
-                __syncwarp();                                    // the previous block has been read out
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    float hi[4], lo[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) split_tf32(x[4 * q + j], hi[j], lo[j]);
-                    *reinterpret_cast<float4 *>(sh_hi + lane * kStagePitch + 4 * q) = make_float4(hi[0], hi[1], hi[2], hi[3]);
-                    *reinterpret_cast<float4 *>(sh_lo + lane * kStagePitch + 4 * q) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+            if (!ok) break;
+            umma_commit(smem_u32(&tfull_bar[buf]));               // the accumulator is complete once these have run
+        }
+    } else if (warp >= 2) {
+        const int q = warp & 3;                                   // the quarter of tensor memory this warp reaches
+        float *stage = reinterpret_cast<float *>(dyn_smem + (tiles - smem_u32(dyn_smem)) + S::kStages * S::kStageBytes) +
+                       q * (32 * kStagePitch);
+        int acc = 0, cur_node = -1;
+        for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++acc) {
+            const int nt = tile % S::kNSplit, tx = tile / S::kNSplit % tiles_x, node = tile / (S::kNSplit * tiles_x);
+            const int t0 = tx * kTileM, buf = acc & 1;
+            if (node != cur_node) {                               // this node's (decoder's) small tensors
+                __syncwarp();
+                const float *nb = bias + (int64_t)node * param_stride;
+                if (MODE != kGradDeconv)
+                    for (int i = lane; i < COUT; i += 32) s_bias[q][i] = nb[i];
+                if (MODE == kConvCode) {
+                    for (int i = lane; i < 4 * 64; i += 32) s_wl[q][i] = w_last[(int64_t)node * param_stride + i];
+                    if (lane < 4) s_bl[q][lane] = b_last[(int64_t)node * param_stride + lane];
+                }
+                if (MODE == kDeconvFinal) {
+                    s_wl[q][lane] = w_last[(int64_t)node * param_stride + lane];
+                    if (lane == 0) {
+                        s_bl[q][0] = b_last[(int64_t)node * param_stride];
+                        s_bl[q][1] = extra ? w_last[(int64_t)node * param_stride + 32] : 0.0f;   // parameter server: the tap on the innovation
+                    }
                 }
                 __syncwarp();
-#pragma unroll
-                for (int it = 0; it < 8; ++it) {
-                    const int rr = it * 4 + (lane >> 3), cq = lane & 7;      // four rows per pass, eight lanes per row
-                    const int64_t tr = (int64_t)t0 + warp * 32 + rr;
-                    // conv: row tr is position tr; deconv: columns below COUT are position 2 tr, the others 2 tr + 1
-                    const int64_t pos = S::kIsConv ? tr : 2 * tr + (c0 >= COUT ? 1 : 0);
+                cur_node = node;
+            }
+            int have = 0;
+            if (lane == 0) have = mbar_wait_shared(smem_u32(&tfull_bar[buf]), (acc >> 1) & 1, &failed) ? 1 : 0;
+            have = __shfl_sync(0xffffffffu, have, 0);
+            if (!have) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int64_t t = (int64_t)t0 + q * 32 + lane;          // this thread's row
+            const uint32_t trow = tmem + (uint32_t)(buf * NT) + ((uint32_t)(q * 32) << 16);
+            float last[4] = {0.f, 0.f, 0.f, 0.f};                   // kConvCode: the 4 code channels; kDeconvFinal: 2 positions
+#pragma unroll 1
+            for (int cl = 0; cl < NT; cl += 32) {
+                float x[32];
+                tmem_load32(trow + (uint32_t)cl, x);
+                const int c0 = nt * NT + cl;                        // column of the layer's GEMM
+                const int cb = S::kIsConv ? c0 : c0 % COUT;         // channel of column c0
+                if (MODE == kGradDeconv) {
+                    const int64_t pos = 2 * t + (c0 >= COUT ? 1 : 0);
                     if (pos < L_out) {
-                        const int64_t at = (S::kIsConv ? ((int64_t)node * Lpad_out + tr) * COUT
-                                                       : ((int64_t)node * Lpad_out + 2 * tr) * COUT) + c0 + 4 * cq;
-                        *reinterpret_cast<float4 *>(out_hi + at) = *reinterpret_cast<const float4 *>(sh_hi + rr * kStagePitch + 4 * cq);
-                        *reinterpret_cast<float4 *>(out_lo + at) = *reinterpret_cast<const float4 *>(sh_lo + rr * kStagePitch + 4 * cq);
+                        const float4 *m4 = reinterpret_cast<const float4 *>(extra + ((int64_t)node * Lpad_out + pos) * COUT + cb);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            const float4 m = m4[v];
+                            x[4 * v] = m.x > 0.0f ? x[4 * v] : __fmul_rn(kSlope, x[4 * v]);
+                            x[4 * v + 1] = m.y > 0.0f ? x[4 * v + 1] : __fmul_rn(kSlope, x[4 * v + 1]);
+                            x[4 * v + 2] = m.z > 0.0f ? x[4 * v + 2] : __fmul_rn(kSlope, x[4 * v + 2]);
+                            x[4 * v + 3] = m.w > 0.0f ? x[4 * v + 3] : __fmul_rn(kSlope, x[4 * v + 3]);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) x[j] = leaky(__fadd_rn(x[j], s_bias[q][cb + j]));
+                }
+                if (MODE == kConvCode) {
+#pragma unroll
+                    for (int o = 0; o < 4; ++o)
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) last[o] = __fmaf_rn(s_wl[q][o * 64 + c0 + j], x[j], last[o]);
+                } else if (MODE == kDeconvFinal) {                   // COUT = 32: columns 0..31 position 2t, 32..63 position 2t + 1
+                    float a = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) a = __fmaf_rn(s_wl[q][j], x[j], a);
+                    last[c0 / 32] = a;
+                } else {
+                    // The 32 x 32 block of this warp (row = lane) goes through shared memory, first its hi parts, then
+                    // its lo parts, so that the global stores are whole 128-byte rows.
+#pragma unroll 1
+                    for (int part = 0; part < 2; ++part) {
+                        __syncwarp();                                // the previous block has been read out
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            float hi[4], lo[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) split_tf32(x[4 * v + j], hi[j], lo[j]);
+                            *reinterpret_cast<float4 *>(stage + lane * kStagePitch + 4 * v) =
+                                part == 0 ? make_float4(hi[0], hi[1], hi[2], hi[3]) : make_float4(lo[0], lo[1], lo[2], lo[3]);
+                        }
+                        __syncwarp();
+                        float *out = part == 0 ? out_hi : out_lo;
+#pragma unroll
+                        for (int itr = 0; itr < 8; ++itr) {
+                            const int rr = itr * 4 + (lane >> 3), cq = lane & 7;      // four rows per pass, eight lanes per row
+                            const int64_t tr = (int64_t)t0 + q * 32 + rr;
+                            // conv: row tr is position tr; deconv: columns below COUT are position 2 tr, the others 2 tr + 1
+                            const int64_t pos = S::kIsConv ? tr : 2 * tr + (c0 >= COUT ? 1 : 0);
+                            if (pos < L_out) {
+                                const int64_t at = (S::kIsConv ? ((int64_t)node * Lpad_out + tr) * COUT
+                                                               : ((int64_t)node * Lpad_out + 2 * tr) * COUT) + c0 + 4 * cq;
+                                *reinterpret_cast<float4 *>(out + at) = *reinterpret_cast<const float4 *>(stage + rr * kStagePitch + 4 * cq);
+                            }
+                        }
                     }
                 }
             }
-        }
-        if (MODE == kConvCode && t < L_out)
-            reinterpret_cast<float4 *>(out_last)[(int64_t)node * L_out + t] =
-                make_float4(__fadd_rn(last[0], s_bl[0]), __fadd_rn(last[1], s_bl[1]), __fadd_rn(last[2], s_bl[2]),
-                            __fadd_rn(last[3], s_bl[3]));
-        if (MODE == kDeconvFinal) {
-            const int64_t row0 = (int64_t)node * L_out;              // decoder `node` reconstructs row `node`
-            if (2 * t < L_out) {
-                const float y = __fadd_rn(last[0], s_bl[0]);
-                out_last[row0 + 2 * t] = extra ? __fmaf_rn(s_bl[1], extra[row0 + 2 * t], y) : y;
+            if (MODE == kConvCode && t < L_out)
+                reinterpret_cast<float4 *>(out_last)[(int64_t)node * L_out + t] =
+                    make_float4(__fadd_rn(last[0], s_bl[q][0]), __fadd_rn(last[1], s_bl[q][1]), __fadd_rn(last[2], s_bl[q][2]),
+                                __fadd_rn(last[3], s_bl[q][3]));
+            if (MODE == kDeconvFinal) {
+                const int64_t row0 = (int64_t)node * L_out;              // decoder `node` reconstructs row `node`
+                if (2 * t < L_out) {
+                    const float y = __fadd_rn(last[0], s_bl[q][0]);
+                    out_last[row0 + 2 * t] = extra ? __fmaf_rn(s_bl[q][1], extra[row0 + 2 * t], y) : y;
+                }
+                if (2 * t + 1 < L_out) {
+                    const float y = __fadd_rn(last[1], s_bl[q][0]);
+                    out_last[row0 + 2 * t + 1] = extra ? __fmaf_rn(s_bl[q][1], extra[row0 + 2 * t + 1], y) : y;
+                }
             }
-            if (2 * t + 1 < L_out) {
-                const float y = __fadd_rn(last[1], s_bl[0]);
-                out_last[row0 + 2 * t + 1] = extra ? __fmaf_rn(s_bl[1], extra[row0 + 2 * t + 1], y) : y;
-            }
+            // the accumulator may be overwritten
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&tempty_bar[buf])) : "memory");
         }
-    } else if (threadIdx.x == 0) {
-        atomicExch(errword, 0x5EA5);                              // a wait ran out
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (threadIdx.x == 0 && failed) atomicExch(errword, 0x5EA5);          // a wait ran out
     if (warp == 1)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)N) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)S::kTmemCols) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------
@@ -596,7 +617,7 @@ bool make_matrix_map(EncodeTiledFn enc, CUtensorMap *m, float *base, int k, int 
 {
     const cuuint64_t dims[3] = {(cuuint64_t)k, (cuuint64_t)rows, (cuuint64_t)count};
     const cuuint64_t strides[2] = {(cuuint64_t)k * 4, (cuuint64_t)k * rows * 4};
-    const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)rows, 1};
+    const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)(rows > 128 ? 128 : rows), 1};   // the columns of one tile
     const cuuint32_t es[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -616,9 +637,11 @@ cudaError_t launch_gemm(Ctx &c, const CUtensorMap &a_hi, const CUtensorMap &a_lo
             [&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kSmemBytes); });
         if (e != cudaSuccess) return e;
     }
-    kern<<<dim3(blocks(rows, kTileM), nodes), 128, S::kSmemBytes, c.stream>>>(a_hi, a_lo, b_hi, b_lo, bias, L_out, Lpad_out, out_hi,
-                                                                              out_lo, w_last, b_last, out_last, extra, c.errword, wz0,
-                                                                              wz_step, param_stride),
+    const int tiles_x = (int)blocks(rows, kTileM);
+    const int64_t total = (int64_t)tiles_x * nodes * S::kNSplit;
+    const unsigned grid = (unsigned)(total < sm_count() ? total : sm_count());     // persistent: one CTA per SM at most
+    kern<<<grid, kGemmThreads, S::kSmemBytes, c.stream>>>(a_hi, a_lo, b_hi, b_lo, bias, tiles_x, nodes, L_out, Lpad_out, out_hi, out_lo,
+                                                          w_last, b_last, out_last, extra, c.errword, wz0, wz_step, param_stride),
         ++g_kernel_launches;
     return cudaGetLastError();
 }
