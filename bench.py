@@ -41,8 +41,8 @@ CLOCK_WINDOW_MS = 500.0  # the clock sampler watches at least this long a run of
 NCU_CAPTURE = {
     "kernel": "accumulate_select_kernel",
     "source": os.path.join("paper_2103_08870_b200", "csrc", "lgc_select_fast.cu"),
-    "source_sha256": None,
-    "dram_bytes_per_element": None,
+    "source_sha256": "6303eff12c0425c86a94c5868d2e2f811e15077852f56494ab77aa368a12adac",
+    "dram_bytes_per_element": 19.02,
 }
 
 
@@ -386,8 +386,8 @@ def run_ours(args, w: W.Workload):
     # load in all: the clocks reported are those of the timed steps and of their continuation.
     clock_window_ms = elapsed_ms
     t = args.steps
-    while clock_window_ms < CLOCK_WINDOW_MS:
-        n = max(1, int((CLOCK_WINDOW_MS - clock_window_ms) / max(elapsed_ms / args.steps, 1e-3)) + 1)
+    while clock_window_ms < args.clock_window_ms:
+        n = max(1, int((args.clock_window_ms - clock_window_ms) / max(elapsed_ms / args.steps, 1e-3)) + 1)
         for _ in range(n):
             i = args.warmup + t
             ch = W.choice_for_step(w.seed, i, K)
@@ -487,6 +487,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--nodes", type=int, default=0, help="override K (profiling aid: a smaller device footprint)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling aid)")
+    ap.add_argument("--clock-window-ms", type=float, default=CLOCK_WINDOW_MS,
+                    help="how long a run of steps the clock sampler watches (profiling aid: 0 = the timed steps only)")
     ap.add_argument("--stage-times", action="store_true", help="also report the median time of each of the five stages")
     args = ap.parse_args()
     w = W.workload(args.workload)
