@@ -223,8 +223,16 @@ SelectPlan plan_select(const std::vector<int64_t> &off, const std::vector<int64_
                 if (sp.seg_large[r] >= 0) d.y = -1;                 // several segments, at least one large
         }
         while (d0 < dense.size() && dense[d0 + 1] <= t0) d0 += 2;
-        if (d0 < dense.size() && dense[d0] < t1)                    // w: 0 no dense element in the tile, -1 all dense,
-            d.w = dense[d0] <= t0 && dense[d0 + 1] >= t1 ? -1 : (int)(d0 / 2) + 1;   // else 1 + its first dense run
+        if (d0 < dense.size() && dense[d0] < t1) {
+            // w: 0 no dense element in the tile; one dense run [lo, hi) (positions inside the tile): 1 + lo + (hi << 13);
+            // several runs: -(1 + the first one's number)
+            if (d0 + 2 < dense.size() && dense[d0 + 2] < t1) {
+                d.w = -((int)(d0 / 2) + 1);
+            } else {
+                const int lo = (int)(std::max<int64_t>(dense[d0], t0) - t0), hi = (int)(std::min<int64_t>(dense[d0 + 1], t1) - t0);
+                d.w = 1 + lo + (hi << 13);
+            }
+        }
         sp.tile_desc.push_back(d);
     }
     return sp;

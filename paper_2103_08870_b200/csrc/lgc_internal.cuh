@@ -64,7 +64,8 @@ struct SelectTables {
     int32_t *tchunk_large = nullptr; // [num_tchunks] index into large_ids
     int4 *tile_desc = nullptr;       // [tiles_per_row] x: first segment the tile overlaps; y: the large segment that
                                      // covers the whole tile (-1: several segments, -2: no large one); z: its chunk;
-                                     // w: 0 no dense element in the tile, -1 all dense, else 1 + its first dense run
+                                     // w: 0 no dense element in the tile; one dense run [lo, hi) inside it: 1 + lo + (hi << 13);
+                                     // several runs: -(1 + the first run's number)
     const int64_t *dense_rng = nullptr;  // [num_dense] (begin, end) of the row's runs of dense elements
     int num_dense = 0;
     int32_t *cand_cnt = nullptr;     // [rows][num_tchunks] candidates found in the chunk

@@ -1005,10 +1005,9 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, int64_t g_stri
     const bool selecting = sel >= 0 && sel < sel_rows;
     int4 desc = make_int4(0, -2, 0, 0);         // x: first segment, y: the one large segment covering the tile
                                                 // (-1: several segments, -2: no large segment), z: its chunk,
-                                                // w: 0 no dense element, -1 all dense, else 1 + first dense run
+                                                // w: 0 no dense element, > 0 one dense run (packed), < 0 several
     uint32_t lbkey1 = 0;
-    if (selecting || DENSE) desc = __ldg(f.tile_desc + q);
-    if (DENSE && desc.w < 0) return;            // a tile of dense layers only: they keep no state
+    if (selecting || DENSE) desc = __ldg(f.tile_desc + q);      // consumed after the stream's loads are on their way
     if (selecting && desc.y >= 0) lbkey1 = f.lbkey[(int64_t)sel * f.num_large + desc.y];
     float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
     if (live) {
@@ -1016,11 +1015,17 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, int64_t g_stri
         float4 gg = __ldcs(reinterpret_cast<const float4 *>(g) + (((int64_t)row * g_stride + tile_base + p0) >> 2));
         float4 uu = __ldcs(reinterpret_cast<float4 *>(u) + e);
         vv = __ldcs(reinterpret_cast<float4 *>(v) + e);
-        if (DENSE && desc.w > 0) {
-            // Dense elements among these four take no gradient: their u and v are zero from lgc_init on and
-            // stay exactly zero (m * 0 + 0 = 0, 0 + 0 = 0), which is "no state" for the layers sent as they are.
+        // Dense elements among these four take no gradient: their u and v are zero from lgc_init on and stay
+        // exactly zero (m * 0 + 0 = 0, 0 + 0 = 0), which is "no state" for the layers sent as they are.
+        if (DENSE && desc.w > 0) {                  // one dense run [lo, hi) inside the tile
+            const int lo = (desc.w - 1) & 8191, hi = (desc.w - 1) >> 13;
+            if (p0 >= lo && p0 < hi) gg.x = 0.0f;
+            if (p0 + 1 >= lo && p0 + 1 < hi) gg.y = 0.0f;
+            if (p0 + 2 >= lo && p0 + 2 < hi) gg.z = 0.0f;
+            if (p0 + 3 >= lo && p0 + 3 < hi) gg.w = 0.0f;
+        } else if (DENSE && desc.w < 0) {           // several runs (tiny dense layers side by side)
             const int64_t pos = tile_base + p0, tile_end = tile_base + in_tile;
-            for (int r = desc.w - 1; r < f.num_dense && f.dense_rng[2 * r] < tile_end; ++r) {
+            for (int r = -desc.w - 1; r < f.num_dense && f.dense_rng[2 * r] < tile_end; ++r) {
                 const int64_t a = f.dense_rng[2 * r], b = f.dense_rng[2 * r + 1];
                 if (pos >= a && pos < b) gg.x = 0.0f;
                 if (pos + 1 >= a && pos + 1 < b) gg.y = 0.0f;
