@@ -161,6 +161,55 @@ def test_layer_modes_inside_one_context(variant, K, extra):
         assert gpu.val_topk_only.shape == (K, gpu.mu_t) and top.mu == gpu.mu_t
 
 
+@pytest.mark.parametrize("variant", ["rar", "ps"])
+def test_index_stream_and_host_step_with_layer_modes(variant):
+    # the DEFLATE stream of an index row covers the autoencoder's layers and then the top-k-only ones (slot order),
+    # each layer's gaps counted from the layer's own start; and lgc_step_host serves a context with modes (the dense
+    # layers are read from the device copy of the gradients at the scatter)
+    from oracle import index_coding as IC
+    K = 3
+    numel, modes = APART, APART_MODES
+    params = W.ae_init_params(8, 4, variant, K, 5)
+    gpu = lgc.LGC(numel, K, variant=variant, layer_mode=modes)
+    gpu.set_ae_params(params)
+    ora = OraclePhased(numel, modes, K, {0: params.numpy()}, grouping="modes", variant=variant)
+    src = W.GradientSource(W.LayerTable("apart", numel, [1 + (i % 3) for i in range(len(numel))]), K, seed=71)
+    hu = torch.empty(gpu.N, dtype=torch.float32).pin_memory()
+    dg = torch.empty(K, gpu.N, device="cuda")
+    du = torch.empty(gpu.N, device="cuda")
+    for t in range(4):
+        g = src.step(t) * 300.0
+        choice = W.choice_for_step(11, t, K)
+        gpu.step_host(g.clone().pin_memory(), dg, du, hu, choice)
+        torch.cuda.synchronize()
+        ref, _ = ora.step(g.numpy(), "compressed", choice)
+        assert_close(hu.numpy(), ref, f"step {t}: update through host buffers")
+        compare_state_and_slots(gpu, ora, f"step {t}")
+    # the stream of the last selection: slot-ordered layer starts and slot offsets
+    g = src.step(4) * 300.0
+    choice = W.choice_for_step(11, 4, K)
+    gpu.accumulate(g.cuda(), choice)
+    gpu.topk(choice, None)
+    order = [l for l, m in enumerate(modes) if m == "ae"] + [l for l, m in enumerate(modes) if m == "topk"]
+    off = np.concatenate([[0], np.cumsum(numel)])
+    layer_off = [int(off[l]) for l in order]
+    koff = np.concatenate([[0], np.cumsum([gpu.k_l[l] for l in order])])
+    assert [gpu.first_slot[l] for l in order] == [int(x) for x in koff[:-1]] and koff[-1] == gpu.mu_all
+    for node in range(K if variant == "ps" else 1):
+        row = gpu.idx[node].cpu().numpy()
+        ref_bytes = IC.varint_bytes(row, layer_off, koff)
+        out = torch.full((8 * gpu.mu_all + 1024,), 0xEE, dtype=torch.uint8, device="cuda")
+        sizes = torch.zeros(2, dtype=torch.int64, device="cuda")
+        gpu.encode_indices(node, out, sizes)
+        torch.cuda.synchronize()
+        n_stream, n_bytes = (int(x) for x in sizes.cpu())
+        assert n_bytes == len(ref_bytes)
+        assert IC.inflate(out[:n_stream].cpu().numpy().tobytes()) == ref_bytes
+        assert np.array_equal(IC.indices_from_varint(ref_bytes, layer_off, koff), row)
+    gpu.abort_step()
+    gpu.check()
+
+
 def test_a_context_needs_a_layer_for_the_autoencoder_and_known_modes():
     with pytest.raises(lgc.LGCError, match="INVALID_ARG"):
         lgc.LGC([5000, 6000], 2, layer_mode=["dense", "topk"])
