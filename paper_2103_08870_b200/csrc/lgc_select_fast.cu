@@ -316,6 +316,7 @@ __global__ void __launch_bounds__(kSelThreads) collect_kernel(FastArgs f)
 
 // Where a finishing CTA reads its entries from: the compacted candidates or the segment itself.
 struct CompactSource {
+    static constexpr bool kIndirect = true;       // offsets come from an array in global memory
     const uint32_t *key;
     const int32_t *idx;
     int n;
@@ -323,6 +324,7 @@ struct CompactSource {
     __device__ __forceinline__ int32_t idx_at(int i) const { return idx[i]; }
 };
 struct DataSource {
+    static constexpr bool kIndirect = false;
     const float *seg;
     int64_t off;
     int n;
@@ -340,38 +342,61 @@ struct FinishShared {
 // Ordered emission by counting: an entry of `src` is selected iff its key is above T, or equals T
 // and fewer than r equal keys precede it in the whole segment; its output slot is the number of
 // selected entries before it.  gt_done / eq_done: entries with key > T / == T that precede src.
-template <int THREADS, typename Source>
+// A warp takes 32 * kFinPerThread consecutive entries, 32 consecutive ones per round (lane = entry:
+// shared-memory reads without bank conflicts, coalesced global ones); inside a round the entries before a
+// lane's own are counted with ballots.
+// TRANSLATE (the CTA emits all k entries of the segment, and the source's offsets sit in global memory): the
+// rounds write an entry's NUMBER into its slot and a last pass replaces the numbers by the offsets, k
+// independent loads at once; fetched inside the rounds, every round waited for its winners' offsets.
+template <int THREADS, bool TRANSLATE, typename Source>
 __device__ void emit_ordered(const Source &src, uint32_t T, int r, int gt_done, int eq_done, int k,
                              int32_t *__restrict__ out, FinishShared &sh, int32_t *errword)
 {
     const int tile = THREADS * kFinPerThread;
+    const int lane = (int)threadIdx.x & 31, warp = (int)threadIdx.x >> 5;
+    const unsigned below = (1u << lane) - 1u;
     for (int base = 0; base < src.n; base += tile) {
         uint32_t key[kFinPerThread];
-        const int first = base + (int)threadIdx.x * kFinPerThread;
+        const int first = base + warp * (32 * kFinPerThread) + lane;
         unsigned gt = 0, eq = 0;
 #pragma unroll
         for (int i = 0; i < kFinPerThread; ++i) {
-            key[i] = first + i < src.n ? src.key_at(first + i) : 0u;
-            if (first + i < src.n) { gt += key[i] > T; eq += key[i] == T; }
+            const int at = first + 32 * i;
+            key[i] = at < src.n ? src.key_at(at) : 0u;
+            if (at < src.n) { gt += key[i] > T; eq += key[i] == T; }
         }
         unsigned total;
-        const unsigned before = block_prefix_excl<unsigned>(gt | (eq << 16), sh.warp_u, &total);
+        unsigned before = block_prefix_excl<unsigned>(gt | (eq << 16), sh.warp_u, &total);
+        before = __shfl_sync(kFull, before, 0);                   // what the warps in front of this one hold
         int g = gt_done + (int)(before & 0xffff), e = eq_done + (int)(before >> 16);
 #pragma unroll
         for (int i = 0; i < kFinPerThread; ++i) {
-            if (first + i < src.n) {
+            const int at = first + 32 * i;
+            const bool is_gt = at < src.n && key[i] > T, is_eq = at < src.n && key[i] == T;
+            const unsigned G = __ballot_sync(kFull, is_gt), E = __ballot_sync(kFull, is_eq);
+            if (G | E) {
+                const int gi = g + __popc(G & below), ei = e + __popc(E & below);
                 int pos = -1;
-                if (key[i] > T) { pos = g + (e < r ? e : r); ++g; }
-                else if (key[i] == T) { if (e < r) pos = g + e; ++e; }
+                if (is_gt) pos = gi + (ei < r ? ei : r);
+                else if (is_eq && ei < r) pos = gi + ei;
                 if (pos >= 0) {
-                    if (pos < k) out[pos] = src.idx_at(first + i);
+                    if (pos < k) out[pos] = TRANSLATE ? at : src.idx_at(at);
                     else atomicExch(errword, 0x5E60);
                 }
+                g += __popc(G);
+                e += __popc(E);
             }
         }
         gt_done += (int)(total & 0xffff);
         eq_done += (int)(total >> 16);
         if (gt_done + (eq_done < r ? eq_done : r) >= k) break;     // everything is emitted
+    }
+    if (TRANSLATE) {
+        __syncthreads();                                           // the CTA's own stores to out are visible to it
+        for (int j = threadIdx.x; j < k; j += THREADS) {
+            const int at = out[j];
+            if (at >= 0 && at < src.n) out[j] = src.idx_at(at);
+        }
     }
 }
 
@@ -424,7 +449,7 @@ __device__ uint32_t finish_from(const Source &src, uint32_t d0, int k_rem, int k
         k_rem = sh.found[1];
         __syncthreads();
     }
-    emit_ordered<THREADS>(src, prefix, k_rem, 0, 0, k, out, sh, errword);
+    emit_ordered<THREADS, Source::kIndirect>(src, prefix, k_rem, 0, 0, k, out, sh, errword);
     const uint32_t T = prefix;
     return T;
 }
@@ -501,12 +526,17 @@ __device__ __forceinline__ ListVerdict list_verdict(const FastArgs &f, int row, 
 
 // Compacts the candidates of the gn chunks from chunk gb on (large segment li of `row`) in index
 // order into ckey/cidx, which already hold `done` entries; returns how many it added.
-// group_off: kFinGroup ints of shared memory.  All THREADS threads of the CTA take part.
+// group_off: kFinGroup + 1 ints of shared memory.  All THREADS threads of the CTA take part.
+// A warp copies a chunk's list at a time (its records lie side by side: one coalesced read of up to 32 records,
+// further reads for longer lists), four chunks in flight; where a chunk's records go follows from the prefix
+// of the counts.  (One candidate per thread with a binary search for its chunk spent more issue slots on the
+// searches than the copies take: 12 k cycles per 8192 candidates with 1024 threads.)
 template <int THREADS>
 __device__ __forceinline__ int compact_group(const FastArgs &f, int row, int li, int gb, int gn, int done,
                                              uint32_t *ckey, int32_t *cidx, int *group_off, unsigned *warp_u)
 {
     constexpr int kPerT = kFinGroup / THREADS;
+    constexpr int kWarps = THREADS / 32, kTrip = 4;
     const int c0 = f.tchunk0[li], q0 = f.large_q0[li];
     const int32_t *cnt = f.cand_cnt + (int64_t)row * f.num_tchunks;
     // exclusive prefix of the chunk counts of this group, in shared memory
@@ -525,46 +555,35 @@ __device__ __forceinline__ int compact_group(const FastArgs &f, int row, int li,
         group_off[threadIdx.x * kPerT + j] = (int)at;
         at += (unsigned)mine[j];
     }
+    if (threadIdx.x == THREADS - 1) group_off[kFinGroup] = (int)total;
     __syncthreads();
-    // one candidate per thread and trip, eight trips in flight: its chunk by binary search in
-    // shared memory, then its record from the chunk's list (neighbouring ranks read
-    // neighbouring records)
-    int top = 1;                                           // largest power of two below gn (1 when gn <= 2)
-    while (top * 2 < gn) top *= 2;
-    for (int base = 0; base < (int)total; base += THREADS * 8) {
-        const uint2 *rec[8];
-        int tile0[8];
-        // the last chunk whose offset is <= rank, for the eight ranks side by side: the halving steps run in
-        // lock step, so that the eight shared-memory reads of a step are in flight together
-        int lo[8];
+    const int lane = (int)threadIdx.x & 31, warp = (int)threadIdx.x >> 5;
+    const uint2 *lists = f.cand + ((int64_t)row * f.num_tchunks + gb) * kCandCap;
+    for (int base = warp * kTrip; base < gn; base += kWarps * kTrip) {
+        int first[kTrip], n[kTrip];
+        uint2 kp[kTrip];
 #pragma unroll
-        for (int t = 0; t < 8; ++t) lo[t] = 0;
-        for (int step = top; step > 0; step >>= 1) {
-#pragma unroll
-            for (int t = 0; t < 8; ++t) {
-                const int at = lo[t] + step;
-                if (at < gn && group_off[at] <= base + t * THREADS + (int)threadIdx.x) lo[t] = at;
+        for (int t = 0; t < kTrip; ++t) {
+            const int ch = base + t;
+            first[t] = n[t] = 0;
+            if (ch < gn) {
+                first[t] = group_off[ch];
+                n[t] = group_off[ch + 1] - first[t];
             }
+            kp[t] = lane < n[t] ? __ldg(lists + (int64_t)ch * kCandCap + lane) : make_uint2(0u, 0u);
         }
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const int r = base + t * THREADS + (int)threadIdx.x;
-            rec[t] = nullptr;
-            tile0[t] = 0;
-            if (r < (int)total) {
-                rec[t] = f.cand + ((int64_t)row * f.num_tchunks + gb + lo[t]) * kCandCap + (r - group_off[lo[t]]);
-                tile0[t] = (q0 + (gb + lo[t] - c0)) * kSelChunk;              // N < 2^31
+        for (int t = 0; t < kTrip; ++t) {
+            const int ch = base + t;
+            const int tile0 = (q0 + (gb + ch - c0)) * kSelChunk;               // N < 2^31
+            if (lane < n[t]) {
+                ckey[done + first[t] + lane] = kp[t].x;
+                cidx[done + first[t] + lane] = tile0 + (int)kp[t].y;
             }
-        }
-        uint2 kp[8];
-#pragma unroll
-        for (int t = 0; t < 8; ++t) kp[t] = rec[t] ? __ldg(rec[t]) : make_uint2(0u, 0u);
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const int r = base + t * THREADS + (int)threadIdx.x;
-            if (rec[t]) {
-                ckey[done + r] = kp[t].x;
-                cidx[done + r] = tile0[t] + (int)kp[t].y;
+            for (int j = lane + 32; j < n[t]; j += 32) {                       // a list of more than 32 records
+                const uint2 more = __ldg(lists + (int64_t)ch * kCandCap + j);
+                ckey[done + first[t] + j] = more.x;
+                cidx[done + first[t] + j] = tile0 + (int)more.y;
             }
         }
     }
@@ -617,7 +636,7 @@ __device__ __forceinline__ bool arrives_last(int32_t *ticket, int n, int *flag)
 __global__ void __launch_bounds__(kFinThreads) compact_groups_kernel(FastArgs f)
 {
     __shared__ unsigned h[kHistBins];
-    __shared__ int group_off[kFinGroup];
+    __shared__ int group_off[kFinGroup + 1];
     __shared__ unsigned warp_u[kFinWarps];
     __shared__ int warp_i[kFinWarps];
     __shared__ int is_last, scan_flag;
@@ -763,7 +782,7 @@ __global__ void __launch_bounds__(kFinThreads) wide_emit_kernel(FastArgs f)
     if (gt0 + (eq0 < r ? eq0 : r) < k) {
         const int64_t base = (int64_t)row * f.comp_total + f.comp_off[g.li] + range.x;
         CompactSource src{f.comp_key + base, f.comp_idx + base, range.y};
-        emit_ordered<kFinThreads>(src, T, r, gt0, eq0, k, f.out + (int64_t)row * f.out_stride + f.seg_out[s], sh, f.errword);
+        emit_ordered<kFinThreads, false>(src, T, r, gt0, eq0, k, f.out + (int64_t)row * f.out_stride + f.seg_out[s], sh, f.errword);
     }
     if (g.job == 0 && threadIdx.x == 0) {
         f.seg_m[g.slot] = (int)m;
@@ -789,7 +808,7 @@ __global__ void __launch_bounds__(THREADS) finish_kernel(FastArgs f)
     __shared__ FinishShared sh;
     __shared__ SmallShared small_sh;
     __shared__ unsigned full_hist[kHistBins];
-    __shared__ int group_off[kFinGroup];
+    __shared__ int group_off[kFinGroup + 1];
     extern __shared__ __align__(16) uint32_t fin_dyn[];     // f.smem_keys candidate keys
     const int row = blockIdx.y;
     if ((int)blockIdx.x >= f.num_large + f.fin_small) {      // spare CTAs: clear the dense update meanwhile
