@@ -124,8 +124,10 @@ gather_encode_mean_kernel(const float *__restrict__ v, int64_t N, const int32_t 
     constexpr int kEnc = C1 * 3 + C1 + C2 * C1 * 3 + C2;
     __shared__ float w[kEnc];
     __shared__ float zs[256 * C2];          // [node][channel][position in CTA]
+    grid_release_dependents();              // a single wave: the next kernel's CTAs may come in beside this one's
     for (int i = threadIdx.x; i < kEnc; i += blockDim.x) w[i] = params[i];
     __syncthreads();
+    grid_wait();                            // the selection's indices are complete from here on
     const float *w1 = w, *b1 = w + C1 * 3, *w2 = b1 + C1, *b2 = w2 + C2 * C1 * 3;
     const int k = threadIdx.x / TT, tt = threadIdx.x % TT;
     const int64_t t = (int64_t)blockIdx.x * TT + tt;
@@ -434,7 +436,9 @@ sparse_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val
 {
     constexpr int kDec = C2 * C1 * 3 + C1 + C1 * 3 + 1;
     __shared__ float w[kDec];
+    grid_release_dependents();
     if (blockIdx.x >= slot_ctas) {
+        grid_wait();                                // the update buffer has been cleared by then
         dense_piece(pieces, blockIdx.x - slot_ctas, g, g_stride, K, update);
         return;
     }
@@ -442,6 +446,7 @@ sparse_scatter_kernel(const float *__restrict__ z, const float *__restrict__ val
         for (int i = threadIdx.x; i < kDec; i += kAeThreads) w[i] = dec[i];
         __syncthreads();
     }
+    grid_wait();                                    // codes, indices and the cleared update are complete from here on
     const int64_t p = (int64_t)blockIdx.x * kAeThreads + threadIdx.x;
     if (p >= mu_all) return;
     const int32_t i = idx[p];
@@ -562,10 +567,12 @@ cudaError_t launch_encode(Ctx &c)
         int tt = 256 / c.K;
         if (tt > 64) tt = 64;
         const unsigned grid = blocks_for(c.L2, tt);
-#define CALL(A, B) gather_encode_mean_kernel<A, B><<<grid, tt * c.K, 0, c.stream>>>(                                 \
+        cudaError_t le = cudaSuccess;
+#define CALL(A, B) le = launch_dependent(gather_encode_mean_kernel<A, B>, dim3(grid), dim3(tt * c.K), c.stream,        \
         c.v, c.N, c.idx, c.K, tt, c.mu, c.L2, c.params, c.val, c.code, c.combined, c.mixed ? nullptr : c.tile_lo)
         LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
 #undef CALL
+        if (le != cudaSuccess) return le;
         c.val_valid = c.mu_t == 0;              // the values of top-k-only layers are not gathered here
         c.mean_valid = true;
         c.tile_lo_valid = !c.mixed;
@@ -657,9 +664,11 @@ static cudaError_t launch_dense_scatter(Ctx &c, int mode, float *update, const f
         } else if (mode == 2) {
             sparse_scatter_kernel<3, 2, 2><<<sgrid, kAeThreads, 0, c.stream>>>(SCATTER_ARGS(c.combined)), ++g_kernel_launches;
         } else {
-#define CALL(A, B) sparse_scatter_kernel<A, B, 0><<<sgrid, kAeThreads, 0, c.stream>>>(SCATTER_ARGS(c.combined))
+            cudaError_t le = cudaSuccess;
+#define CALL(A, B) le = launch_dependent(sparse_scatter_kernel<A, B, 0>, dim3(sgrid), dim3(kAeThreads), c.stream, SCATTER_ARGS(c.combined))
             LGC_DISPATCH_AE(c.cfg.ae_c1, c.cfg.ae_c2, CALL)
 #undef CALL
+            if (le != cudaSuccess) return le;
         }
 #undef SCATTER_ARGS
         return cudaGetLastError();

@@ -241,6 +241,34 @@ struct OncePerDevice {
 };
 int sm_count();                                   // of the current device
 
+// Programmatic dependent launch: a kernel launched this way may start while its predecessor in the stream is
+// still draining; it runs its own prologue (weights into shared memory) and then waits, with grid_wait(), for
+// the predecessor to have completed and its memory to be visible.  Nothing it reads or writes before that wait
+// may be touched by the predecessor.  Launched the ordinary way the same kernels' waits return at once.
+__device__ __forceinline__ void grid_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... Params, typename... Args>
+cudaError_t launch_dependent_smem(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+template <typename... Params, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(Params...), dim3 grid, dim3 block, cudaStream_t stream, Args... args)
+{
+    return launch_dependent_smem(kernel, grid, block, 0, stream, args...);
+}
+
 extern thread_local uint64_t g_kernel_launches;   // kernels this thread has enqueued (lgc_kernel_launches)
 extern thread_local std::string g_last_error;   // failures without a context (see lgc_last_error)
 
