@@ -29,17 +29,6 @@ constexpr int kStagePitch = 36;       // floats per row of the epilogue's stagin
 
 __device__ __forceinline__ float leaky(float x) { return x > 0.0f ? x : kSlope * x; }
 
-// x = hi + lo with both parts representable in tf32 (10 explicit mantissa bits)
-__device__ __forceinline__ void split_tf32(float x, float &hi, float &lo)
-{
-    uint32_t h;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(x));
-    hi = __uint_as_float(h);
-    const float r = __fsub_rn(x, hi);
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(r));
-    lo = __uint_as_float(h);
-}
-
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
@@ -492,6 +481,174 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------
+// Weight gradients of the wide convolutions as GEMMs that sum over rows (the backward pass's
+//     dW[co][tau C_in + ci] = sum over (node, t) of G[t][co] X[2t + tau][ci]):
+// the reduction runs along the ROWS of both operands, so both are read "MN-major": a k-block is 32 rows
+// (positions t) of 128-byte pieces of the operand's columns, and one tcgen05.mma consumes 8 rows.
+// Shared-memory layout of an operand tile of C columns: C / 32 pieces, each 32 rows x 128 bytes as the TMA
+// writes a box of 32 floats x 32 rows with the 128-byte swizzle of 32-byte atoms (the one layout the tensor
+// cores read 32-bit operands from in this orientation); the matrix descriptor's leading offset is the
+// piece (4096 bytes), its stride offset the group of 4 rows (512 bytes), and the instruction descriptor marks
+// both operands as transposed.  The M operand is 128 columns of one matrix, the N operand NT columns of the
+// other; each is either the gradient G (one map) or the input slices X (two maps: columns below `split` are
+// taps 0 and 1 of pair-row t, the others tap 2 = the first C_in floats of pair-row t + 1).  Rows beyond the
+// layer's length are outside the maps and arrive as zeros.
+// One CTA = (M tile, N tile, node, part of the node's rows); its 128 x NT sums go to partial[chunk], chunk =
+// node * splits + part, as [M][N] or (TRANS) as [N][M]; the kernel that applies Adam adds the chunks up.
+// Same roles and bounded waits as ae5_gemm_kernel: TMA thread, MMA thread, four warps that read the accumulator.
+// ------------------------------------------------------------------------------------------
+struct alignas(64) WgradMaps {
+    CUtensorMap m[2][2], n[2][2];      // [hi, lo][columns below the split, columns from the split on]
+};
+
+template <int NT>
+struct WgradShape {
+    static constexpr int kABytes = 128 * kBlockK * 4;          // one part (hi or lo) of the M operand's k-block
+    static constexpr int kBBytes = NT * kBlockK * 4;
+    static constexpr int kStageBytes = 2 * kABytes + 2 * kBBytes;
+    static constexpr int kFit = 218 * 1024 / kStageBytes;
+    static constexpr int kStages = kFit < 4 ? kFit : 4;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024;
+    static constexpr int kTmemCols = NT <= 32 ? 32 : NT <= 64 ? 64 : NT <= 128 ? 128 : 256;
+    static_assert(NT % 32 == 0 && NT >= 32 && NT <= 256, "N tile: whole 128-byte pieces, one accumulator");
+    static_assert(kStages >= 2, "two stages must fit");
+};
+
+// Matrix descriptor of an MN-major operand tile as laid out above.  32-bit operands read along their rows have
+// one layout: the 128-byte swizzle in units of 32 bytes, whose pattern repeats every 4 rows (512 bytes).
+__device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);         // start address, 16-byte units
+    d |= (uint64_t)(4096 >> 4) << 16;                     // leading byte offset: from one 128-byte piece of columns to the next
+    d |= (uint64_t)(512 >> 4) << 32;                      // stride byte offset: from one group of 4 rows to the next
+    d |= (uint64_t)1 << 46;                               // descriptor version of this architecture
+    d |= (uint64_t)1 << 61;                               // 128-byte swizzle with 32-byte atoms
+    return d;
+}
+
+template <int NT, bool TRANS>
+__global__ void __launch_bounds__(kGemmThreads)
+ae5_wgrad_kernel(const __grid_constant__ WgradMaps maps, int m_split, int n_split, int tiles_m, int tiles_n, int splits,
+                 int kb_per_node, int kbps, int m_total, int n_total, float *__restrict__ partial, int64_t pstride,
+                 int32_t *errword)
+{
+    using S = WgradShape<NT>;
+    extern __shared__ uint8_t dyn_smem[];
+    __shared__ __align__(8) uint64_t full_bar[S::kStages], empty_bar[S::kStages], tfull_bar;
+    __shared__ uint32_t tmem_base_smem;
+    __shared__ volatile int failed;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t tiles = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+    // this CTA's work
+    int w = blockIdx.x;
+    const int tm = w % tiles_m; w /= tiles_m;
+    const int tn = w % tiles_n; w /= tiles_n;
+    const int part = w % splits, node = w / splits;
+    const int kb0 = part * kbps, kb1 = kb0 + kbps < kb_per_node ? kb0 + kbps : kb_per_node;   // (never empty: see the host)
+    const int m0 = tm * 128, n0 = tn * NT;
+
+    if (threadIdx.x == 0) {
+        failed = 0;
+        for (int s = 0; s < S::kStages; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), 1);
+            mbar_init(smem_u32(&empty_bar[s]), 1);
+        }
+        mbar_init(smem_u32(&tfull_bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)),
+                     "r"((uint32_t)S::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = tmem_base_smem;
+
+    if (threadIdx.x == 0) {
+        for (int kb = kb0, it = 0; kb < kb1; ++kb, ++it) {
+            const int s = it % S::kStages;
+            if (it >= S::kStages && !mbar_wait_shared(smem_u32(&empty_bar[s]), ((it / S::kStages) & 1) ^ 1, &failed)) break;
+            const uint32_t bar = smem_u32(&full_bar[s]);
+            const uint32_t st = tiles + (uint32_t)s * S::kStageBytes;
+            mbar_expect_tx(bar, S::kStageBytes);
+            const int row = kb * kBlockK;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {                 // the M operand: four pieces of 32 columns
+                    const int col = m0 + 32 * j;
+                    const uint32_t dst = st + (uint32_t)(h * S::kABytes + j * 4096);
+                    if (col < m_split) tma_load_3d(dst, &maps.m[h][0], bar, col, row, node);
+                    else tma_load_3d(dst, &maps.m[h][1], bar, col - m_split, row + 1, node);
+                }
+#pragma unroll
+                for (int j = 0; j < NT / 32; ++j) {
+                    const int col = n0 + 32 * j;
+                    const uint32_t dst = st + (uint32_t)(2 * S::kABytes + h * S::kBBytes + j * 4096);
+                    if (col < n_split) tma_load_3d(dst, &maps.n[h][0], bar, col, row, node);
+                    else tma_load_3d(dst, &maps.n[h][1], bar, col - n_split, row + 1, node);
+                }
+            }
+        }
+    } else if (threadIdx.x == 32) {
+        // instruction descriptor: fp32 accumulator, tf32 x tf32, both operands MN-major (bits 15 and 16), N = NT, M = 128
+        constexpr uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(NT >> 3) << 17) |
+                                   ((uint32_t)(128 >> 4) << 24);
+        bool ok = true;
+        for (int kb = kb0, it = 0; kb < kb1; ++kb, ++it) {
+            const int s = it % S::kStages;
+            if (!mbar_wait_shared(smem_u32(&full_bar[s]), (it / S::kStages) & 1, &failed)) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t st = tiles + (uint32_t)s * S::kStageBytes;
+#pragma unroll
+            for (int ks = 0; ks < kBlockK / 8; ++ks) {            // 8 rows per step: two groups of the layout
+                const uint64_t a_hi = umma_desc_mn(st + ks * 1024), a_lo = umma_desc_mn(st + S::kABytes + ks * 1024);
+                const uint64_t b_hi = umma_desc_mn(st + 2 * S::kABytes + ks * 1024);
+                const uint64_t b_lo = umma_desc_mn(st + 2 * S::kABytes + S::kBBytes + ks * 1024);
+                umma_tf32(tmem, a_hi, b_hi, idesc, it > 0 || ks > 0);
+                umma_tf32(tmem, a_hi, b_lo, idesc, true);
+                umma_tf32(tmem, a_lo, b_hi, idesc, true);
+            }
+            umma_commit(smem_u32(&empty_bar[s]));
+        }
+        if (ok) umma_commit(smem_u32(&tfull_bar));
+    } else if (warp >= 2) {
+        const int q = warp & 3;
+        int have = 0;
+        if (lane == 0) have = mbar_wait_shared(smem_u32(&tfull_bar), 0, &failed) ? 1 : 0;
+        have = __shfl_sync(0xffffffffu, have, 0);
+        if (have) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            float *out = partial + (int64_t)(node * splits + part) * pstride;
+            const int m = m0 + q * 32 + lane;                     // this thread's row of the accumulator
+            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int cl = 0; cl < NT; cl += 32) {
+                float x[32];
+                tmem_load32(trow + (uint32_t)cl, x);
+                if (TRANS) {                                      // out[n][m]: a warp writes 32 consecutive floats per column
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) out[(int64_t)(n0 + cl + j) * m_total + m] = x[j];
+                } else {                                          // out[m][n]: 128 bytes per thread
+                    float4 *o4 = reinterpret_cast<float4 *>(out + (int64_t)m * n_total + n0 + cl);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) o4[v] = make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]);
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && failed) atomicExch(errword, 0x5EA6);          // a wait ran out
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)S::kTmemCols) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------
 // Decoder (one pass, fp32 pipes), channels-last.
 // ------------------------------------------------------------------------------------------
 // deconv1: ConvTranspose1d(4 -> 4, k3, stride 1, padding 1) + leaky ReLU on the mean code.
@@ -677,6 +834,20 @@ bool ae5_lengths(int64_t mu, int64_t (&len)[5])
     return true;
 }
 
+// How the rows of a wide convolution's weight gradient are cut: every node's l_out rows (k-blocks of 32) into
+// `splits` parts of `kbps` k-blocks, so that tiles x nodes x parts comes to at most two CTAs per SM (two rounds
+// of one CTA per SM), a part has at least four k-blocks where the layer is long enough, and none is empty.
+void ae5_weight_gradient_chunks(int K, int64_t l_out, int cin, int cout, int *splits, int *kbps)
+{
+    const int kb = (int)((l_out + kBlockK - 1) / kBlockK);
+    // tiles of the launch (launch_ae5_weight_gradient): 128 output channels x 192 or 128 slice columns; 64 channels: 128 slice columns x 64
+    const int tiles = cout >= 128 ? (cout / 128) * (3 * cin % 128 == 0 ? 3 * cin / 128 : 1) : 3 * cin / 128;
+    int want = 2 * 148 / (tiles * K);                 // (a tuning figure: the SM count of the B200; any device computes the same sums)
+    want = std::max(1, std::min(want, std::max(1, kb / 4)));
+    *kbps = (kb + want - 1) / want;
+    *splits = (kb + *kbps - 1) / *kbps;
+}
+
 void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
 {
     ae5_lengths(mu, a.len);
@@ -724,6 +895,8 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
             a.g_enc_lo[l] = take((size_t)K * a.lpad[l] * kAe5EncCh[l + 1]);
         }
         a.g_enc[3] = take((size_t)K * a.len[4] * 64);
+        a.g4_hi = take((size_t)K * a.len[4] * 64);
+        a.g4_lo = take((size_t)K * a.len[4] * 64);
         pmax = (size_t)K * a.len[4] * 3 * kAe5EncCh[3];     // only conv4's input gradient goes through the products
         for (int j = 0; j < 2; ++j) {
             a.gw_hi[j] = take((size_t)4 * kAe5EncCh[j + 1] * kAe5EncCh[j + 2]);
@@ -764,6 +937,11 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         // convolutions) are summed by few CTAs per chunk, so they get up to 192 shorter chunks
         t.chunk = count > 256 ? std::max<int64_t>(256, (rows + 47) / 48) : std::max<int64_t>(128, (rows + 191) / 192);
         t.chunks = kind == 3 ? 1 : (int)((rows + t.chunk - 1) / t.chunk);
+        if (kind == 1 && cin >= 64) {        // conv2..conv4: summed on the tensor cores, node by node
+            const int l = i / 2;
+            ae5_weight_gradient_chunks(K, a.len[l + 1], cin, cout, &a.wg_splits[l - 1], &a.wg_kbps[l - 1]);
+            t.chunks = K * a.wg_splits[l - 1];
+        }
         t.partial_off = part;
         part += t.chunks * ((count + 3) / 4 * 4);
     };
@@ -814,6 +992,31 @@ cudaError_t ae5_make_maps(Ctx &c)
                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
         ok = ok && make_matrix_map(enc, &a.map_gw_hi[j], a.gw_hi[j], 2 * C, 2 * cin);
         ok = ok && make_matrix_map(enc, &a.map_gw_lo[j], a.gw_lo[j], 2 * C, 2 * cin);
+    }
+    for (int l = 1; l <= 3; ++l) {           // weight gradients of conv2..conv4: boxes of 32 floats x 32 rows, zeros beyond the length
+        const int cin = kAe5EncCh[l], cout = kAe5EncCh[l + 1];
+        const int64_t lout = a.len[l + 1];
+        const cuuint32_t box[3] = {32, 32, 1};
+        const cuuint32_t es[3] = {1, 1, 1};
+        for (int h = 0; h < 2; ++h) {
+            float *g = l == 3 ? (h ? a.g4_lo : a.g4_hi) : (h ? a.g_enc_lo[l] : a.g_enc[l]);
+            const cuuint64_t gdims[3] = {(cuuint64_t)cout, (cuuint64_t)lout, (cuuint64_t)c.K};
+            const cuuint64_t gstr[2] = {(cuuint64_t)cout * 4, (cuuint64_t)(l == 3 ? lout : a.lpad[l]) * cout * 4};
+            ok = ok && enc(&a.map_wg_g[l - 1][h], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, g, gdims, gstr, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            float *x = h ? a.act_lo[l - 1] : a.act_hi[l - 1];
+            const cuuint64_t xstr[2] = {(cuuint64_t)(2 * cin) * 4, (cuuint64_t)a.lpad[l - 1] * cin * 4};
+            // taps 0 and 1: pair-rows 0 .. lout - 1 in full; tap 2: the first half of pair-rows 1 .. lout
+            const cuuint64_t xdims0[3] = {(cuuint64_t)(2 * cin), (cuuint64_t)lout, (cuuint64_t)c.K};
+            const cuuint64_t xdims1[3] = {(cuuint64_t)cin, (cuuint64_t)(lout + 1), (cuuint64_t)c.K};
+            ok = ok && enc(&a.map_wg_x[l - 1][h][0], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, x, xdims0, xstr, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            ok = ok && enc(&a.map_wg_x[l - 1][h][1], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, x, xdims1, xstr, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+        }
     }
     a.map_dw_hi.resize(3);                   // one map per layer: slice d holds decoder d's weights
     a.map_dw_lo.resize(3);
@@ -978,6 +1181,51 @@ cudaError_t launch_ae5_input_gradient(Ctx &c, int layer)
                                                  a.len[1], a.lpad[0], a.g_enc[0], a.g_enc_lo[0], nullptr, nullptr, nullptr, a.act_hi[0]);
     return launch_gemm<kGradDeconv, 256, 128>(c, a.map_g_hi[1], a.map_g_lo[1], a.map_gw_hi[1], a.map_gw_lo[1], nullptr, rows, c.K,
                                               a.len[2], a.lpad[1], a.g_enc[1], a.g_enc_lo[1], nullptr, nullptr, nullptr, a.act_hi[1]);
+}
+
+template <int NT, bool TRANS>
+static cudaError_t launch_wgrad(Ctx &c, const WgradMaps &maps, int m_split, int n_split, int m_total, int n_total, int layer)
+{
+    using S = WgradShape<NT>;
+    Ae5 &a = *c.ae5;
+    auto kern = ae5_wgrad_kernel<NT, TRANS>;
+    static OncePerDevice configured;
+    {
+        const cudaError_t e = configured.run(
+            [&] { return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kSmemBytes); });
+        if (e != cudaSuccess) return e;
+    }
+    const Ae5::Tensor &T = a.tensors[2 * layer];
+    const int splits = a.wg_splits[layer - 1], kbps = a.wg_kbps[layer - 1];
+    const int kb_per_node = (int)((a.len[layer + 1] + kBlockK - 1) / kBlockK);
+    const int tiles_m = m_total / 128, tiles_n = n_total / NT;
+    const unsigned grid = (unsigned)(tiles_m * tiles_n * splits * c.K);
+    kern<<<grid, kGemmThreads, S::kSmemBytes, c.stream>>>(maps, m_split, n_split, tiles_m, tiles_n, splits, kb_per_node, kbps, m_total,
+                                                          n_total, a.partial + T.partial_off, (T.count + 3) / 4 * 4, c.errword),
+        ++g_kernel_launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_ae5_weight_gradient(Ctx &c, int layer)
+{
+    Ae5 &a = *c.ae5;
+    const int cin = kAe5EncCh[layer], cout = kAe5EncCh[layer + 1];
+    const int l = layer - 1;
+    constexpr int kNoSplit = 1 << 30;
+    WgradMaps maps;
+    if (layer == 3) {                         // 64 output channels: the slices make the rows of the accumulator, dW comes out transposed
+        for (int h = 0; h < 2; ++h) {
+            maps.m[h][0] = a.map_wg_x[l][h][0]; maps.m[h][1] = a.map_wg_x[l][h][1];
+            maps.n[h][0] = a.map_wg_g[l][h];    maps.n[h][1] = a.map_wg_g[l][h];
+        }
+        return launch_wgrad<64, true>(c, maps, 2 * cin, kNoSplit, 3 * cin, cout, layer);
+    }
+    for (int h = 0; h < 2; ++h) {
+        maps.m[h][0] = a.map_wg_g[l][h];    maps.m[h][1] = a.map_wg_g[l][h];
+        maps.n[h][0] = a.map_wg_x[l][h][0]; maps.n[h][1] = a.map_wg_x[l][h][1];
+    }
+    if (layer == 1) return launch_wgrad<192, false>(c, maps, kNoSplit, 2 * cin, cout, 3 * cin, layer);
+    return launch_wgrad<128, false>(c, maps, kNoSplit, 2 * cin, cout, 3 * cin, layer);
 }
 
 // Stage 5 up to the reconstruction.  Ring-allreduce: the decoder on the mean code; c.recon gets the mu

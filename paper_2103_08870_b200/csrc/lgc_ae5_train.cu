@@ -442,7 +442,8 @@ dec1_grad_kernel(const float *__restrict__ zbar, const float *__restrict__ g1, i
 // Ring-allreduce (dzbar given): every node's code gets dzbar / K (the mean), written to dzk.
 // Parameter server (dzbar == nullptr): dzk already holds every node's own gradient.  Thread per (node, position).
 __global__ void code_bwd_kernel(const float *__restrict__ dzbar, int K, int64_t L4, const float *__restrict__ w5,
-                                const float *__restrict__ a4_hi, float *__restrict__ dzk, float *__restrict__ g4)
+                                const float *__restrict__ a4_hi, float *__restrict__ dzk, float *__restrict__ g4,
+                                float *__restrict__ g4_hi, float *__restrict__ g4_lo)
 {
     __shared__ float w[4 * 64];
     for (int i = threadIdx.x; i < 4 * 64; i += blockDim.x) w[i] = w5[i];
@@ -471,6 +472,11 @@ __global__ void code_bwd_kernel(const float *__restrict__ dzbar, int K, int64_t 
             o[j] = as[j] > 0.f ? acc : __fmul_rn(kSlope, acc);
         }
         reinterpret_cast<float4 *>(g4 + r * 64)[q] = make_float4(o[0], o[1], o[2], o[3]);
+        float hi[4], lo[4];                       // and as two tf32 parts, for the weight gradient on the tensor cores
+#pragma unroll
+        for (int j = 0; j < 4; ++j) split_tf32(o[j], hi[j], lo[j]);
+        reinterpret_cast<float4 *>(g4_hi + r * 64)[q] = make_float4(hi[0], hi[1], hi[2], hi[3]);
+        reinterpret_cast<float4 *>(g4_lo + r * 64)[q] = make_float4(lo[0], lo[1], lo[2], lo[3]);
     }
 }
 
@@ -653,7 +659,7 @@ void encoder_backward(Launcher &L, const float *dzbar)
     const int64_t *len = a.len, mu = c.mu;
     if (L.ok()) {
         code_bwd_kernel<<<blocks((int64_t)K * len[4], 128), 128, 0, c.stream>>>(dzbar, K, len[4], P + a.off_w[4], a.act4_hi, a.dzk,
-                                                                              a.g_enc[3]),
+                                                                              a.g_enc[3], a.g4_hi, a.g4_lo),
             ++g_kernel_launches;
     }
     const Rows dzk_rows = rows_of(a.dzk, nullptr, len[4] * 4, 4, len[4], 4);
@@ -671,7 +677,7 @@ void encoder_backward(Launcher &L, const float *dzbar)
             break;
         }
         const int64_t x_node = a.lpad[i - 1] * cin;
-        L.tn(2 * i, g, rows_of(a.act_hi[i - 1], a.act_lo[i - 1], x_node, 2 * cin, lout, 3 * cin));
+        if (L.ok()) L.err = launch_ae5_weight_gradient(c, i);       // dW = sum over rows of G^T X, on the tensor cores
         if (i == 3) {        // conv4 (768 output columns: too wide for one accumulator): products on the fp32 pipes, then the fold
             L.arrange(P + a.off_w[i], cin, cout, 0);
             L.nn(g, (int64_t)K * lout, a.wt, 3 * cin, a.pbuf, nullptr);

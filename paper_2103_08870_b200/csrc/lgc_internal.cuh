@@ -118,6 +118,12 @@ struct Ae5 {
     float *dact5_hi = nullptr, *dact5_lo = nullptr;  // [mu][32] output of deconv5 (inference folds it into the last conv)
     float *g_enc[4] = {};               // dLoss/d(pre-activation) of conv1..conv4.  conv4's: fp32 [K][L4][64].  conv1..conv3's:
     float *g_enc_lo[3] = {};            // two tf32 parts laid out like the layer's output, [K][lpad][C] (they feed tensor-core GEMMs)
+    float *g4_hi = nullptr, *g4_lo = nullptr;   // conv4's gradient once more as two tf32 parts, [K][L4][64] (operand of its weight gradient)
+    // Weight gradients of conv2..conv4 (index 0..2) on the tensor cores: maps over the gradient at the layer's output (G) and
+    // over the layer's input seen as rows of a pair of positions (X: taps 0 and 1, and tap 2 one pair further), hi and lo
+    // parts; positions beyond the layer's length read as zeros.  wg_splits: parts a node's rows are cut into.
+    CUtensorMap map_wg_g[3][2], map_wg_x[3][2][2];
+    int wg_splits[3] = {1, 1, 1}, wg_kbps[3] = {1, 1, 1};
     float *gw_hi[2] = {}, *gw_lo[2] = {};   // weights of conv2 / conv3 arranged for the GEMM that makes the gradient at their input
     CUtensorMap map_g_hi[2], map_g_lo[2], map_gw_hi[2], map_gw_lo[2];
     float *g_dec[5] = {};               // the same for deconv1..deconv5: [L][C], g_dec[4] is [mu][32]
@@ -269,6 +275,17 @@ cudaError_t launch_dependent(void (*kernel)(Params...), dim3 grid, dim3 block, c
     return launch_dependent_smem(kernel, grid, block, 0, stream, args...);
 }
 
+// x = hi + lo with both parts representable in tf32 (10 explicit mantissa bits)
+__device__ __forceinline__ void split_tf32(float x, float &hi, float &lo)
+{
+    uint32_t h;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(x));
+    hi = __uint_as_float(h);
+    const float r = __fsub_rn(x, hi);
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(r));
+    lo = __uint_as_float(h);
+}
+
 extern thread_local uint64_t g_kernel_launches;   // kernels this thread has enqueued (lgc_kernel_launches)
 extern thread_local std::string g_last_error;   // failures without a context (see lgc_last_error)
 
@@ -324,6 +341,9 @@ cudaError_t launch_ae5_train_forward(Ctx &c);          // ring-allreduce: encode
 cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out);
 // gradient at the input of conv2 (layer = 1) or conv3 (layer = 2) from g_enc[layer] into g_enc[layer - 1], on the tensor cores
 cudaError_t launch_ae5_input_gradient(Ctx &c, int layer);
+// weight gradient of conv2, conv3 or conv4 (layer = 1, 2, 3) into the partial sums of tensor 2 * layer, on the tensor cores
+cudaError_t launch_ae5_weight_gradient(Ctx &c, int layer);
+void ae5_weight_gradient_chunks(int K, int64_t l_out, int cin, int cout, int *splits, int *kbps);   // how the rows are cut
 cudaError_t launch_ae5_train_step_ps(Ctx &c, int common, float lam_rec, float lam_sim, float *loss_out);
 struct AdamArgs {
     float *params, *m, *v;
