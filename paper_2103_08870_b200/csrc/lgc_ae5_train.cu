@@ -209,6 +209,79 @@ tn_gemm_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ par
     }
 }
 
+// Column sums of a wide A (a bias gradient) in one streaming pass:  psum[s][p] = sum over the rows m of chunk s of
+// A(m, p), and with Q > 0 also the sums weighted by the Q entries of B's row (conv1's weight gradient, whose rows are the
+// three kept values a position reads):  pw[s][p][q] = sum_m A(m, p) B(m, q).
+// A.len is 4 times a power of two, at most 1024, rows 16-byte aligned.  A thread holds four columns; 256 / (A.len / 4) rows
+// are in flight per pass and four passes per trip, so that a CTA keeps 32 KB (64 KB with two tf32 parts) in flight;
+// the rows' sums are then added across the threads of a column in thread order.  Grid: the chunks.
+template <int Q>
+__global__ void __launch_bounds__(256)
+colsum_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ psum, int64_t psum_stride, float *__restrict__ pw,
+              int64_t pw_stride)
+{
+    __shared__ float4 red[1 + Q][256];
+    const int tpr = A.len >> 2, rpp = 256 / tpr;             // threads per row, rows per pass
+    const int c4 = threadIdx.x % tpr, rr = threadIdx.x / tpr;
+    const int64_t first = (int64_t)blockIdx.x * chunk;
+    const int64_t last = first + chunk < M ? first + chunk : M;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), accw[Q > 0 ? Q : 1];
+#pragma unroll
+    for (int q = 0; q < Q; ++q) accw[q] = acc;
+    RowCursor ca(A, first + rr), cb(B, first + rr);
+    for (int64_t m = first + rr; m < last; m += 4 * rpp) {
+        float4 a[4];
+        float b[4][Q > 0 ? Q : 1];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {                        // the four rows' loads are issued before any is used
+            a[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+            const bool in = m + (int64_t)r * rpp < last;
+            const int64_t ab = ca.at(A) + 4 * c4;
+            if (in) a[r] = *reinterpret_cast<const float4 *>(A.hi + ab);
+            if (in && A.lo) {
+                const float4 l = *reinterpret_cast<const float4 *>(A.lo + ab);
+                a[r].x = __fadd_rn(a[r].x, l.x); a[r].y = __fadd_rn(a[r].y, l.y);
+                a[r].z = __fadd_rn(a[r].z, l.z); a[r].w = __fadd_rn(a[r].w, l.w);
+            }
+            if (Q > 0) {
+                const int64_t bb = cb.at(B);
+#pragma unroll
+                for (int q = 0; q < Q; ++q) b[r][q] = in ? B.hi[bb + q] : 0.f;
+                cb.advance(B, rpp);
+            }
+            ca.advance(A, rpp);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            acc.x = __fadd_rn(acc.x, a[r].x); acc.y = __fadd_rn(acc.y, a[r].y);
+            acc.z = __fadd_rn(acc.z, a[r].z); acc.w = __fadd_rn(acc.w, a[r].w);
+#pragma unroll
+            for (int q = 0; q < Q; ++q) {
+                accw[q].x = __fmaf_rn(a[r].x, b[r][q], accw[q].x); accw[q].y = __fmaf_rn(a[r].y, b[r][q], accw[q].y);
+                accw[q].z = __fmaf_rn(a[r].z, b[r][q], accw[q].z); accw[q].w = __fmaf_rn(a[r].w, b[r][q], accw[q].w);
+            }
+        }
+    }
+    red[0][threadIdx.x] = acc;
+#pragma unroll
+    for (int q = 0; q < Q; ++q) red[1 + q][threadIdx.x] = accw[q];
+    __syncthreads();
+    if (rr != 0) return;
+    for (int j = 0; j <= Q; ++j) {
+        float4 tot = red[j][c4];
+        for (int g = 1; g < rpp; ++g) {
+            const float4 x = red[j][g * tpr + c4];
+            tot.x = __fadd_rn(tot.x, x.x); tot.y = __fadd_rn(tot.y, x.y); tot.z = __fadd_rn(tot.z, x.z); tot.w = __fadd_rn(tot.w, x.w);
+        }
+        if (j == 0) {
+            *reinterpret_cast<float4 *>(psum + (int64_t)blockIdx.x * psum_stride + 4 * c4) = tot;
+        } else {
+            float *o = pw + (int64_t)blockIdx.x * pw_stride + (int64_t)(4 * c4) * Q + (j - 1);
+            o[0] = tot.x; o[Q] = tot.y; o[2 * Q] = tot.z; o[3 * Q] = tot.w;
+        }
+    }
+}
+
 // The same for a narrow right-hand side (at most four columns; B.hi == nullptr: one column of ones,
 // which makes the column sums of A, i.e. a bias gradient): partial[s][p][q] = sum_m A(m, p) B(m, q).
 // Grid (chunks, ceil(P / 32)), 256 threads: lane = column p, the eight warps stride over the rows and are
@@ -260,17 +333,6 @@ tn_narrow_kernel(Rows A, Rows B, int Q, int64_t M, int64_t chunk, float *__restr
             partial[(int64_t)blockIdx.x * pstride + (int64_t)p * Q + q] = tot;
         }
     }
-}
-
-// x = hi + lo with both parts representable in tf32 (what the tensor-core GEMMs take)
-__device__ __forceinline__ void split_tf32(float x, float &hi, float &lo)
-{
-    uint32_t h;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(x));
-    hi = __uint_as_float(h);
-    const float r = __fsub_rn(x, hi);
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(r));
-    lo = __uint_as_float(h);
 }
 
 // Gradient at a convolution's input from the products prod[k][t][tau C_in + ci] = (G W)[t]:
@@ -598,7 +660,29 @@ struct Launcher {
                                                                                   pstride_of(t));
         ++g_kernel_launches;
     }
-    void colsum(int t, const Rows &A) { tn_narrow(t, A, rows_of(nullptr, nullptr, 0, 0, 1, 1), 1); }
+    static bool streams(const Rows &A) { return A.vec && A.len >= 4 && A.len <= 1024 && (A.len & (A.len - 1)) == 0; }
+    void colsum(int t, const Rows &A)
+    {
+        if (!streams(A)) return tn_narrow(t, A, rows_of(nullptr, nullptr, 0, 0, 1, 1), 1);
+        if (!ok()) return;
+        const Ae5::Tensor &T = a.tensors[t];
+        colsum_kernel<0><<<T.chunks, 256, 0, c.stream>>>(A, A, T.rows, T.chunk, partial_of(t), pstride_of(t), nullptr, 0);
+        ++g_kernel_launches;
+    }
+    // conv1: the bias gradient (tensor tb, column sums of A) and the weight gradient (tensor tw, A^T B with B's three columns)
+    // from one pass over A
+    void colsum_and_narrow3(int tb, int tw, const Rows &A, const Rows &B)
+    {
+        const Ae5::Tensor &Tb = a.tensors[tb], &Tw = a.tensors[tw];
+        if (!streams(A) || Tb.chunks != Tw.chunks || Tb.chunk != Tw.chunk || B.lo) {
+            colsum(tb, A);
+            return tn_narrow(tw, A, B, 3);
+        }
+        if (!ok()) return;
+        colsum_kernel<3><<<Tb.chunks, 256, 0, c.stream>>>(A, B, Tb.rows, Tb.chunk, partial_of(tb), pstride_of(tb), partial_of(tw),
+                                                          pstride_of(tw));
+        ++g_kernel_launches;
+    }
     void arrange(const float *w, int cin, int cout, int mode)
     {
         if (!ok()) return;
@@ -671,11 +755,11 @@ void encoder_backward(Launcher &L, const float *dzbar)
         // gradient at conv(i+1)'s output: conv4's is fp32, the others are two tf32 parts laid out like the output
         const Rows g = i == 3 ? rows_of(a.g_enc[3], nullptr, lout * cout, cout, lout, cout)
                               : rows_of(a.g_enc[i], a.g_enc_lo[i], a.lpad[i] * cout, cout, lout, cout);
-        L.colsum(2 * i + 1, g);
         if (i == 0) {        // conv1 reads the kept values themselves: rows of three floats, two apart
-            L.tn_narrow(0, g, rows_of(c.val, nullptr, mu, 2, lout, 3), 3);
+            L.colsum_and_narrow3(1, 0, g, rows_of(c.val, nullptr, mu, 2, lout, 3));
             break;
         }
+        L.colsum(2 * i + 1, g);
         const int64_t x_node = a.lpad[i - 1] * cin;
         if (L.ok()) L.err = launch_ae5_weight_gradient(c, i);       // dW = sum over rows of G^T X, on the tensor cores
         if (i == 3) {        // conv4 (768 output columns: too wide for one accumulator): products on the fp32 pipes, then the fold
