@@ -889,7 +889,6 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         a.act4_lo = take((size_t)K * a.len[4] * 64);
         a.dact5_hi = take((size_t)mu * 32);
         a.dact5_lo = take((size_t)mu * 32);
-        size_t pmax = 0;
         for (int l = 0; l < 3; ++l) {                       // laid out like the outputs of conv1..conv3
             a.g_enc[l] = take((size_t)K * a.lpad[l] * kAe5EncCh[l + 1]);
             a.g_enc_lo[l] = take((size_t)K * a.lpad[l] * kAe5EncCh[l + 1]);
@@ -897,8 +896,7 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         a.g_enc[3] = take((size_t)K * a.len[4] * 64);
         a.g4_hi = take((size_t)K * a.len[4] * 64);
         a.g4_lo = take((size_t)K * a.len[4] * 64);
-        pmax = (size_t)K * a.len[4] * 3 * kAe5EncCh[3];     // only conv4's input gradient goes through the products
-        for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < 3; ++j) {
             a.gw_hi[j] = take((size_t)4 * kAe5EncCh[j + 1] * kAe5EncCh[j + 2]);
             a.gw_lo[j] = take((size_t)4 * kAe5EncCh[j + 1] * kAe5EncCh[j + 2]);
         }
@@ -907,7 +905,6 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
         a.dzk = take((size_t)K * a.len[4] * 4);
         a.dzbar = take((size_t)a.len[4] * 4);
         a.dr = take((size_t)mu);
-        a.pbuf = take(pmax);
         a.wt = take((size_t)256 * 384);
         a.loss_blocks = (int)((mu + 255) / 256);
         // partial sums of the loss: per decoder the reconstruction term's, then the similarity term's (parameter server)
@@ -980,16 +977,18 @@ cudaError_t ae5_make_maps(Ctx &c)
         ok = ok && make_dact_map(enc, &a.map_dact_hi[l], a.dact_hi[l], dcin, a.len[3 - l], a.decoders);
         ok = ok && make_dact_map(enc, &a.map_dact_lo[l], a.dact_lo[l], dcin, a.len[3 - l], a.decoders);
     }
-    for (int j = 0; j < 2; ++j) {            // input-gradient GEMMs of conv2 and conv3: A = the gradient at the layer's output
+    for (int j = 0; j < 3; ++j) {            // input-gradient GEMMs of conv2..conv4: A = the gradient at the layer's output
         const int C = kAe5EncCh[j + 2], cin = kAe5EncCh[j + 1];
         const cuuint64_t dims[3] = {(cuuint64_t)C, (cuuint64_t)a.len[j + 2], (cuuint64_t)c.K};
-        const cuuint64_t strides[2] = {(cuuint64_t)C * 4, (cuuint64_t)a.lpad[j + 1] * C * 4};
+        const cuuint64_t strides[2] = {(cuuint64_t)C * 4, (cuuint64_t)(j == 2 ? a.len[4] : a.lpad[j + 1]) * C * 4};
         const cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileM, 1};
         const cuuint32_t es[3] = {1, 1, 1};
-        for (int h = 0; h < 2; ++h)
-            ok = ok && enc(h ? &a.map_g_lo[j] : &a.map_g_hi[j], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3,
-                           h ? a.g_enc_lo[j + 1] : a.g_enc[j + 1], dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+        for (int h = 0; h < 2; ++h) {
+            float *g = j == 2 ? (h ? a.g4_lo : a.g4_hi) : (h ? a.g_enc_lo[j + 1] : a.g_enc[j + 1]);
+            ok = ok && enc(h ? &a.map_g_lo[j] : &a.map_g_hi[j], CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, g, dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+        }
         ok = ok && make_matrix_map(enc, &a.map_gw_hi[j], a.gw_hi[j], 2 * C, 2 * cin);
         ok = ok && make_matrix_map(enc, &a.map_gw_lo[j], a.gw_lo[j], 2 * C, 2 * cin);
     }
@@ -1179,8 +1178,12 @@ cudaError_t launch_ae5_input_gradient(Ctx &c, int layer)
     if (layer == 1)
         return launch_gemm<kGradDeconv, 128, 64>(c, a.map_g_hi[0], a.map_g_lo[0], a.map_gw_hi[0], a.map_gw_lo[0], nullptr, rows, c.K,
                                                  a.len[1], a.lpad[0], a.g_enc[0], a.g_enc_lo[0], nullptr, nullptr, nullptr, a.act_hi[0]);
-    return launch_gemm<kGradDeconv, 256, 128>(c, a.map_g_hi[1], a.map_g_lo[1], a.map_gw_hi[1], a.map_gw_lo[1], nullptr, rows, c.K,
-                                              a.len[2], a.lpad[1], a.g_enc[1], a.g_enc_lo[1], nullptr, nullptr, nullptr, a.act_hi[1]);
+    if (layer == 2)
+        return launch_gemm<kGradDeconv, 256, 128>(c, a.map_g_hi[1], a.map_g_lo[1], a.map_gw_hi[1], a.map_gw_lo[1], nullptr, rows, c.K,
+                                                  a.len[2], a.lpad[1], a.g_enc[1], a.g_enc_lo[1], nullptr, nullptr, nullptr, a.act_hi[1]);
+    // conv4: 64 channels in, 2 x 256 columns out, cut into four column tiles
+    return launch_gemm<kGradDeconv, 64, 256>(c, a.map_g_hi[2], a.map_g_lo[2], a.map_gw_hi[2], a.map_gw_lo[2], nullptr, rows, c.K,
+                                             a.len[3], a.lpad[2], a.g_enc[2], a.g_enc_lo[2], nullptr, nullptr, nullptr, a.act_hi[2]);
 }
 
 template <int NT, bool TRANS>

@@ -12,9 +12,10 @@
 //   transposed convolution  y[2j+tau][co] += w[ci][co][tau] x[j][ci]
 //     dW[ci][tau C_out + co] = sum_j X[j][ci] G[2j+tau][co]      (rows of G seen as slices of 3 C_out floats)
 //     dX[j][ci]              = sum G[2j+tau][co] w[ci][co][tau]
-// so every layer is one GEMM over rows (dX) and one GEMM that sums over rows (dW), here on the fp32
-// pipes; the sums over rows are cut into chunks whose partial results are added up in fp64, in
-// chunk order, by the kernel that applies Adam.  Leaky-ReLU derivatives are taken from the sign of
+// so every layer is one GEMM over rows (dX) and one GEMM that sums over rows (dW): for the encoder's wide
+// convolutions both run on the tensor cores (lgc_ae5.cu), for the decoder (one pass, not one per node) and the
+// narrow layers on the fp32 pipes here; the sums over rows are cut into chunks whose partial results are added
+// up in fp64, in chunk order, by the kernel that applies Adam.  Leaky-ReLU derivatives are taken from the sign of
 // the stored outputs (the slope is positive, so output and pre-activation have the same sign).
 #include <algorithm>
 
@@ -333,38 +334,6 @@ tn_narrow_kernel(Rows A, Rows B, int Q, int64_t M, int64_t chunk, float *__restr
             partial[(int64_t)blockIdx.x * pstride + (int64_t)p * Q + q] = tot;
         }
     }
-}
-
-// Gradient at a convolution's input from the products prod[k][t][tau C_in + ci] = (G W)[t]:
-//   g_in[k][pos][ci] = leaky'(x[k][pos][ci]) * sum over (t, tau) with 2t + tau = pos of prod[k][t][tau C_in + ci],
-// written as two tf32 parts in the layout of x (node stride x_node_stride).  Thread per (node, position, four channels).
-__global__ void fold_kernel(const float *__restrict__ prod, int K, int64_t L_out, int64_t L_in, int cin,
-                            const float *__restrict__ x_hi, int64_t x_node_stride, float *__restrict__ g_hi,
-                            float *__restrict__ g_lo)
-{
-    const int quads = cin >> 2;
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= (int64_t)K * L_in * quads) return;
-    const int cq = (int)(i % quads);
-    const int64_t pos = (i / quads) % L_in, k = i / quads / L_in;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int tau = 0; tau < 3; ++tau) {
-        const int64_t d = pos - tau;
-        if (d < 0 || (d & 1) || (d >> 1) >= L_out) continue;
-        const float4 p = *reinterpret_cast<const float4 *>(prod + ((k * L_out + (d >> 1)) * 3 + tau) * cin + 4 * cq);
-        acc.x = __fadd_rn(acc.x, p.x); acc.y = __fadd_rn(acc.y, p.y); acc.z = __fadd_rn(acc.z, p.z); acc.w = __fadd_rn(acc.w, p.w);
-    }
-    const int64_t at = k * x_node_stride + pos * cin + 4 * cq;
-    const float4 x = *reinterpret_cast<const float4 *>(x_hi + at);
-    acc.x = x.x > 0.f ? acc.x : __fmul_rn(kSlope, acc.x);
-    acc.y = x.y > 0.f ? acc.y : __fmul_rn(kSlope, acc.y);
-    acc.z = x.z > 0.f ? acc.z : __fmul_rn(kSlope, acc.z);
-    acc.w = x.w > 0.f ? acc.w : __fmul_rn(kSlope, acc.w);
-    float4 hi, lo;
-    split_tf32(acc.x, hi.x, lo.x); split_tf32(acc.y, hi.y, lo.y); split_tf32(acc.z, hi.z, lo.z); split_tf32(acc.w, hi.w, lo.w);
-    *reinterpret_cast<float4 *>(g_hi + at) = hi;
-    *reinterpret_cast<float4 *>(g_lo + at) = lo;
 }
 
 // One layer's weights arranged as the dense [Kd][N] operand of nn_gemm_kernel.
@@ -750,8 +719,8 @@ void encoder_backward(Launcher &L, const float *dzbar)
     L.tn(8, dzk_rows, rows_of(a.act4_hi, a.act4_lo, len[4] * 64, 64, len[4], 64));
     L.colsum(9, dzk_rows);
     for (int i = 3; i >= 0; --i) {
-        const int cin = kAe5EncCh[i], cout = kAe5EncCh[i + 1];
-        const int64_t lin = len[i], lout = len[i + 1];
+        const int cout = kAe5EncCh[i + 1];
+        const int64_t lout = len[i + 1];
         // gradient at conv(i+1)'s output: conv4's is fp32, the others are two tf32 parts laid out like the output
         const Rows g = i == 3 ? rows_of(a.g_enc[3], nullptr, lout * cout, cout, lout, cout)
                               : rows_of(a.g_enc[i], a.g_enc_lo[i], a.lpad[i] * cout, cout, lout, cout);
@@ -760,19 +729,9 @@ void encoder_backward(Launcher &L, const float *dzbar)
             break;
         }
         L.colsum(2 * i + 1, g);
-        const int64_t x_node = a.lpad[i - 1] * cin;
         if (L.ok()) L.err = launch_ae5_weight_gradient(c, i);       // dW = sum over rows of G^T X, on the tensor cores
-        if (i == 3) {        // conv4 (768 output columns: too wide for one accumulator): products on the fp32 pipes, then the fold
-            L.arrange(P + a.off_w[i], cin, cout, 0);
-            L.nn(g, (int64_t)K * lout, a.wt, 3 * cin, a.pbuf, nullptr);
-            if (L.ok()) {
-                fold_kernel<<<blocks((int64_t)K * lin * (cin / 4), 256), 256, 0, c.stream>>>(a.pbuf, K, lout, lin, cin, a.act_hi[i - 1],
-                                                                                            x_node, a.g_enc[i - 1], a.g_enc_lo[i - 1]),
-                    ++g_kernel_launches;
-            }
-        } else if (L.ok()) {  // conv3, conv2: a transposed convolution of g with the same weights, on the tensor cores
-            L.err = launch_ae5_input_gradient(c, i);
-        }
+        // the gradient at the layer's input: a transposed convolution of g with the same weights, on the tensor cores
+        if (L.ok()) L.err = launch_ae5_input_gradient(c, i);
     }
 }
 

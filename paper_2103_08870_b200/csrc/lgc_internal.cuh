@@ -124,13 +124,12 @@ struct Ae5 {
     // parts; positions beyond the layer's length read as zeros.  wg_splits: parts a node's rows are cut into.
     CUtensorMap map_wg_g[3][2], map_wg_x[3][2][2];
     int wg_splits[3] = {1, 1, 1}, wg_kbps[3] = {1, 1, 1};
-    float *gw_hi[2] = {}, *gw_lo[2] = {};   // weights of conv2 / conv3 arranged for the GEMM that makes the gradient at their input
-    CUtensorMap map_g_hi[2], map_g_lo[2], map_gw_hi[2], map_gw_lo[2];
+    float *gw_hi[3] = {}, *gw_lo[3] = {};   // weights of conv2..conv4 arranged for the GEMM that makes the gradient at their input
+    CUtensorMap map_g_hi[3], map_g_lo[3], map_gw_hi[3], map_gw_lo[3];
     float *g_dec[5] = {};               // the same for deconv1..deconv5: [L][C], g_dec[4] is [mu][32]
     float *dzk = nullptr;               // [K][L4][4] gradient at every node's code
     float *dzbar = nullptr;             // [L4][4]    gradient at the mean code
     float *dr = nullptr;                // [mu]       gradient at the reconstruction
-    float *pbuf = nullptr;              // products dY W of a convolution, before they are folded onto the input positions
     float *wt = nullptr;                // one layer's weights arranged for the backward GEMM
     float *partial = nullptr;           // per-chunk partial sums of every parameter tensor's gradient
     double *loss_part = nullptr;        // [loss_blocks]
@@ -339,7 +338,7 @@ cudaError_t launch_ae5_train_encode(Ctx &c);           // every node's code into
 cudaError_t launch_ae5_train_decode(Ctx &c, int d);    // decoder d on c.combined, up to deconv5 (kept in dact5)
 cudaError_t launch_ae5_train_forward(Ctx &c);          // ring-allreduce: encoder, mean, the decoder
 cudaError_t launch_ae5_train_step(Ctx &c, float *loss_out);
-// gradient at the input of conv2 (layer = 1) or conv3 (layer = 2) from g_enc[layer] into g_enc[layer - 1], on the tensor cores
+// gradient at the input of conv2, conv3 or conv4 (layer = 1, 2, 3) from g_enc[layer] into g_enc[layer - 1], on the tensor cores
 cudaError_t launch_ae5_input_gradient(Ctx &c, int layer);
 // weight gradient of conv2, conv3 or conv4 (layer = 1, 2, 3) into the partial sums of tensor 2 * layer, on the tensor cores
 cudaError_t launch_ae5_weight_gradient(Ctx &c, int layer);
