@@ -105,6 +105,7 @@ ae5_conv1_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restri
 {
     __shared__ float x[2 * 64 + 2];
     __shared__ float w[64 * 3], b[64];
+    grid_release_dependents();            // conv2's CTAs may set themselves up meanwhile (they wait for this launch before they load)
     const int k = blockIdx.y;
     const int64_t t0 = (int64_t)blockIdx.x * 64;
     for (int i = threadIdx.x; i < 64 * 3; i += 256) w[i] = w1[i];
@@ -261,6 +262,7 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
 {
     using S = GemmShape<MODE, CIN, COUT>;
     constexpr int NT = S::kNT;
+    grid_release_dependents();            // the next launch may set itself up while this one runs
     extern __shared__ uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t full_bar[S::kStages], empty_bar[S::kStages], tfull_bar[2], tempty_bar[2];
     __shared__ uint32_t tmem_base_smem;
@@ -295,6 +297,7 @@ ae5_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_const
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = tmem_base_smem;
+    grid_wait();                          // barriers and tensor memory are set up: now the predecessor's results are needed
 
     if (threadIdx.x == 0) {
         // producer: one k-block (32 floats of the operand row) of both operands, hi and lo, per stage
@@ -656,6 +659,7 @@ ae5_wgrad_kernel(const __grid_constant__ WgradMaps maps, int m_split, int n_spli
 __global__ void ae5_deconv1_kernel(const float *__restrict__ z, int64_t L4, const float *__restrict__ w,
                                    const float *__restrict__ b, float *__restrict__ out, int64_t param_stride)
 {
+    grid_release_dependents();
     const int64_t s = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= L4) return;
     w += (int64_t)blockIdx.y * param_stride;
@@ -687,6 +691,7 @@ ae5_deconv_kernel(const float *__restrict__ x, int64_t L_in, int64_t L_out, cons
                   const float *__restrict__ b, float *__restrict__ y, float *__restrict__ y_lo, int64_t param_stride)
 {
     extern __shared__ float dsm[];
+    grid_release_dependents();
     x += (int64_t)blockIdx.y * L_in * CIN;                  // blockIdx.y: the decoder
     w += (int64_t)blockIdx.y * param_stride;
     b += (int64_t)blockIdx.y * param_stride;
@@ -797,9 +802,11 @@ cudaError_t launch_gemm(Ctx &c, const CUtensorMap &a_hi, const CUtensorMap &a_lo
     const int tiles_x = (int)blocks(rows, kTileM);
     const int64_t total = (int64_t)tiles_x * nodes * S::kNSplit;
     const unsigned grid = (unsigned)(total < sm_count() ? total : sm_count());     // persistent: one CTA per SM at most
-    kern<<<grid, kGemmThreads, S::kSmemBytes, c.stream>>>(a_hi, a_lo, b_hi, b_lo, bias, tiles_x, nodes, L_out, Lpad_out, out_hi, out_lo,
-                                                          w_last, b_last, out_last, extra, c.errword, wz0, wz_step, param_stride),
-        ++g_kernel_launches;
+    const cudaError_t e = launch_dependent_smem(kern, dim3(grid), dim3(kGemmThreads), S::kSmemBytes, c.stream, a_hi, a_lo, b_hi, b_lo, bias,
+                                                tiles_x, nodes, L_out, Lpad_out, out_hi, out_lo, w_last, b_last, out_last, extra,
+                                                c.errword, wz0, wz_step, param_stride);
+    if (e != cudaSuccess) return e;
+    ++g_kernel_launches;
     return cudaGetLastError();
 }
 
