@@ -25,6 +25,7 @@ constexpr float kSlope = 0.01f;       // leaky-ReLU slope (the paper names the a
 constexpr int kTileM = 128;           // output positions per CTA of the GEMM: the M of one tcgen05.mma
 constexpr int kBlockK = 32;           // fp32 per 128-byte swizzled row
 constexpr int kSpinLimit = 4000000;   // mbarrier polls before a wait gives up
+constexpr int kConv1Pos = 128;        // output positions per CTA of conv1
 constexpr int kStagePitch = 36;       // floats per row of the epilogue's staging blocks (16-byte aligned, spreads the banks)
 
 __device__ __forceinline__ float leaky(float x) { return x > 0.0f ? x : kSlope * x; }
@@ -96,21 +97,21 @@ __device__ __forceinline__ void tmem_load32(uint32_t taddr, float (&x)[32])
 
 // ------------------------------------------------------------------------------------------
 // conv1: gather of the kept values + Conv1d(1 -> 64, k3, s2) + leaky ReLU, written channels-last
-// as (hi, lo).  Grid (ceil(L1 / 64), K), 256 threads: thread = (position, group of 16 channels).
+// as (hi, lo).  Grid (ceil(L1 / 128), K), 256 threads: thread = (position of a pass of 16, four channels).
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 ae5_conv1_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restrict__ idx, int64_t idx_node_stride, int64_t mu,
                  int64_t L1, int64_t Lpad1, const float *__restrict__ w1, const float *__restrict__ b1, float *__restrict__ val,
                  float *__restrict__ a_hi, float *__restrict__ a_lo)
 {
-    __shared__ float x[2 * 64 + 2];
+    __shared__ float x[2 * kConv1Pos + 2];
     __shared__ float w[64 * 3], b[64];
     grid_release_dependents();            // conv2's CTAs may set themselves up meanwhile (they wait for this launch before they load)
     const int k = blockIdx.y;
-    const int64_t t0 = (int64_t)blockIdx.x * 64;
+    const int64_t t0 = (int64_t)blockIdx.x * kConv1Pos;
     for (int i = threadIdx.x; i < 64 * 3; i += 256) w[i] = w1[i];
     if (threadIdx.x < 64) b[threadIdx.x] = b1[threadIdx.x];
-    for (int i = threadIdx.x; i < 2 * 64 + 2; i += 256) {
+    for (int i = threadIdx.x; i < 2 * kConv1Pos + 2; i += 256) {
         const int64_t p = 2 * t0 + i;
         float xv = 0.0f;
         if (p < mu) {
@@ -120,26 +121,32 @@ ae5_conv1_kernel(const float *__restrict__ v, int64_t N, const int32_t *__restri
         x[i] = xv;
     }
     __syncthreads();
-    const int tl = threadIdx.x >> 2, cg = threadIdx.x & 3;
-    const int64_t t = t0 + tl;
-    if (t >= L1) return;
-    const float x0 = x[2 * tl], x1 = x[2 * tl + 1], x2 = x[2 * tl + 2];
-    float *oh = a_hi + ((int64_t)k * Lpad1 + t) * 64 + cg * 16;
-    float *ol = a_lo + ((int64_t)k * Lpad1 + t) * 64 + cg * 16;
+    // sixteen threads per position, four channels each: a warp's store is 512 consecutive bytes
+    const int c4 = threadIdx.x & 15;
+    float wr[4][3], br[4];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int j = 0; j < 4; ++j) {
+        br[j] = b[4 * c4 + j];
+#pragma unroll
+        for (int tau = 0; tau < 3; ++tau) wr[j][tau] = w[(4 * c4 + j) * 3 + tau];
+    }
+#pragma unroll 2
+    for (int tl = threadIdx.x >> 4; tl < kConv1Pos; tl += 16) {
+        const int64_t t = t0 + tl;
+        if (t >= L1) break;
+        const float x0 = x[2 * tl], x1 = x[2 * tl + 1], x2 = x[2 * tl + 2];
         float hi[4], lo[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int co = cg * 16 + q * 4 + j;
-            float acc = b[co];
-            acc = __fmaf_rn(w[co * 3 + 0], x0, acc);
-            acc = __fmaf_rn(w[co * 3 + 1], x1, acc);
-            acc = __fmaf_rn(w[co * 3 + 2], x2, acc);
+            float acc = br[j];
+            acc = __fmaf_rn(wr[j][0], x0, acc);
+            acc = __fmaf_rn(wr[j][1], x1, acc);
+            acc = __fmaf_rn(wr[j][2], x2, acc);
             split_tf32(leaky(acc), hi[j], lo[j]);
         }
-        reinterpret_cast<float4 *>(oh)[q] = make_float4(hi[0], hi[1], hi[2], hi[3]);
-        reinterpret_cast<float4 *>(ol)[q] = make_float4(lo[0], lo[1], lo[2], lo[3]);
+        const int64_t at = ((int64_t)k * Lpad1 + t) * 64 + 4 * c4;
+        *reinterpret_cast<float4 *>(a_hi + at) = make_float4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<float4 *>(a_lo + at) = make_float4(lo[0], lo[1], lo[2], lo[3]);
     }
 }
 
@@ -1063,7 +1070,7 @@ cudaError_t launch_ae5_encode(Ctx &c)
     Ae5 &a = *c.ae5;
     const float *P = c.params;
     prepare_weights(c);
-    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu_all, c.mu, a.len[1], a.lpad[0],
+    ae5_conv1_kernel<<<dim3(blocks(a.len[1], kConv1Pos), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu_all, c.mu, a.len[1], a.lpad[0],
                                                                             P + a.off_w[0], P + a.off_b[0], c.val, a.act_hi[0],
                                                                             a.act_lo[0]),
         ++g_kernel_launches;
@@ -1113,7 +1120,7 @@ cudaError_t launch_ae5_train_encode(Ctx &c)
     Ae5 &a = *c.ae5;
     const float *P = c.params;
     prepare_weights(c);
-    ae5_conv1_kernel<<<dim3(blocks(a.len[1], 64), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu_all, c.mu, a.len[1], a.lpad[0],
+    ae5_conv1_kernel<<<dim3(blocks(a.len[1], kConv1Pos), c.K), 256, 0, c.stream>>>(c.v, c.N, c.idx, c.S == 1 ? 0 : c.mu_all, c.mu, a.len[1], a.lpad[0],
                                                                             P + a.off_w[0], P + a.off_b[0], c.val, a.act_hi[0],
                                                                             a.act_lo[0]),
         ++g_kernel_launches;
