@@ -673,6 +673,7 @@ __global__ void ae5_deconv1_kernel(const float *__restrict__ z, int64_t L4, cons
     b += (int64_t)blockIdx.y * param_stride;
     out += (int64_t)blockIdx.y * L4 * 4;
     float acc[4] = {b[0], b[1], b[2], b[3]};
+    grid_wait();                          // the code comes from the launch in front
 #pragma unroll
     for (int tau = 0; tau < 3; ++tau) {
         const int64_t j = s + 1 - tau;                            // y[s] += w[ci][co][tau] x[ci][j], s = j + tau - 1
@@ -711,6 +712,7 @@ ae5_deconv_kernel(const float *__restrict__ x, int64_t L_in, int64_t L_out, cons
         const int tau = i / (CIN * COUT), rem = i % (CIN * COUT), ci = rem / COUT, co = rem % COUT;
         sw[i] = w[(ci * COUT + co) * 3 + tau];
     }
+    grid_wait();                          // the weights are in place: now the input rows of the launch in front
     for (int i = threadIdx.x; i < (TP + 1) * CIN; i += 256) {
         const int64_t j = j0 - 1 + i / CIN;
         sx[i] = j >= 0 && j < L_in ? x[j * CIN + i % CIN] : 0.0f;
@@ -1258,15 +1260,17 @@ cudaError_t launch_ae5_decode(Ctx &c)
     const float *P = c.params;                                 // decoder d's tensors: dec_stride floats per decoder further on
     const int D = a.decoders;
     const int64_t ps_stride = a.dec_stride;
-    ae5_deconv1_kernel<<<dim3(blocks(a.len[4], 128), D), 128, 0, c.stream>>>(c.combined, a.len[4], P + a.off_dw[0], P + a.off_db[0], a.d0,
-                                                                             ps_stride),
-        ++g_kernel_launches;
+    cudaError_t e = launch_dependent(ae5_deconv1_kernel, dim3(blocks(a.len[4], 128), D), dim3(128), c.stream, c.combined, a.len[4],
+                                     P + a.off_dw[0], P + a.off_db[0], a.d0, ps_stride);
+    if (e != cudaSuccess) return e;
+    ++g_kernel_launches;
     // deconv2 (4 -> 32): too narrow for the tensor cores
     constexpr int kTp = 64, kSmem2 = (3 * 4 * 32 + (kTp + 1) * 4) * 4;
-    ae5_deconv_kernel<4, 32, kTp><<<dim3(blocks(a.len[4] + 1, kTp), D), 256, kSmem2, c.stream>>>(
-        a.d0, a.len[4], a.len[3], P + a.off_dw[1], P + a.off_db[1], a.dact_hi[0], a.dact_lo[0], ps_stride),
-        ++g_kernel_launches;
-    cudaError_t e = cudaGetLastError();
+    e = launch_dependent_smem(ae5_deconv_kernel<4, 32, kTp>, dim3(blocks(a.len[4] + 1, kTp), D), dim3(256), kSmem2, c.stream, a.d0,
+                              a.len[4], a.len[3], P + a.off_dw[1], P + a.off_db[1], a.dact_hi[0], a.dact_lo[0], ps_stride);
+    if (e != cudaSuccess) return e;
+    ++g_kernel_launches;
+    e = cudaGetLastError();
     // deconv3..5: rows j = 0 .. L_in (one more than the input positions: the last makes the tail)
     if (e == cudaSuccess)
         e = launch_gemm<kDeconv, 32, 64>(c, a.map_dact_hi[0], a.map_dact_lo[0], a.map_dw_hi[0], a.map_dw_lo[0], P + a.off_db[2],

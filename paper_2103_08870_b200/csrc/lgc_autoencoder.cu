@@ -186,6 +186,8 @@ gather_encode_mean_kernel(const float *__restrict__ v, int64_t N, const int32_t 
 // out[i] = (rows[0][i] + rows[1][i] + ... + rows[K-1][i]) / K, summed in node order
 __global__ void mean_rows_kernel(const float *__restrict__ rows, int K, int64_t len, float *__restrict__ out)
 {
+    grid_release_dependents();
+    grid_wait();                          // (launched as a dependent of the kernel that writes the rows)
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= len) return;
     float a = rows[i];
@@ -592,7 +594,10 @@ cudaError_t launch_encode(Ctx &c)
 cudaError_t launch_combine_mean(Ctx &c)
 {
     if (c.mean_valid) return cudaSuccess;   // the encoder launch already averaged the codes
-    mean_rows_kernel<<<blocks_for(c.code_len, 256), 256, 0, c.stream>>>(c.code, c.K, c.code_len, c.combined), ++g_kernel_launches;
+    const cudaError_t e = launch_dependent(mean_rows_kernel, dim3(blocks_for(c.code_len, 256)), dim3(256), c.stream, c.code, c.K,
+                                           c.code_len, c.combined);
+    if (e != cudaSuccess) return e;
+    ++g_kernel_launches;
     return cudaGetLastError();
 }
 
