@@ -946,9 +946,10 @@ void ae5_carve(Ae5 &a, int K, int64_t mu, bool ps, char *base, size_t *used)
     auto tensor = [&](int i, int64_t off, int64_t count, int64_t rows, int kind, int cin, int cout) {
         Ae5::Tensor &t = a.tensors[i];
         t.param_off = off; t.count = count; t.rows = rows; t.kind = kind; t.cin = cin; t.cout = cout;
-        // wide tensors: up to 48 chunks (their partial sums are large); narrow ones (biases, conv1, the 1x1
-        // convolutions) are summed by few CTAs per chunk, so they get up to 192 shorter chunks
-        t.chunk = count > 256 ? std::max<int64_t>(256, (rows + 47) / 48) : std::max<int64_t>(128, (rows + 191) / 192);
+        // up to 192 chunks: the decoder's weight gradients (64 x 64 tiles of a few thousand rows of ONE node) are a
+        // handful of tiles, and a CTA's walk over its rows is a chain of load-multiply trips; biases, conv1 and the 1x1
+        // convolutions are summed by few CTAs per chunk
+        t.chunk = count > 256 ? std::max<int64_t>(64, (rows + 191) / 192) : std::max<int64_t>(128, (rows + 191) / 192);
         t.chunks = kind == 3 ? 1 : (int)((rows + t.chunk - 1) / t.chunk);
         if (kind == 1 && cin >= 64) {        // conv2..conv4: summed on the tensor cores, node by node
             const int l = i / 2;
