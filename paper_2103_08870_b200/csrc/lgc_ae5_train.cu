@@ -230,30 +230,31 @@ colsum_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ psum
 #pragma unroll
     for (int q = 0; q < Q; ++q) accw[q] = acc;
     RowCursor ca(A, first + rr), cb(B, first + rr);
-    for (int64_t m = first + rr; m < last; m += 4 * rpp) {
-        float4 a[4];
+    int64_t m = first + rr;
+    // whole trips of four rows: the eight loads are issued back to back, without a branch between them (a thread that
+    // waits for each load before the next keeps a quarter of the bytes in flight)
+    for (; m + 3 * (int64_t)rpp < last; m += 4 * rpp) {
+        float4 a[4], l[4];
         float b[4][Q > 0 ? Q : 1];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {                        // the four rows' loads are issued before any is used
-            a[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-            const bool in = m + (int64_t)r * rpp < last;
+        for (int r = 0; r < 4; ++r) {
             const int64_t ab = ca.at(A) + 4 * c4;
-            if (in) a[r] = *reinterpret_cast<const float4 *>(A.hi + ab);
-            if (in && A.lo) {
-                const float4 l = *reinterpret_cast<const float4 *>(A.lo + ab);
-                a[r].x = __fadd_rn(a[r].x, l.x); a[r].y = __fadd_rn(a[r].y, l.y);
-                a[r].z = __fadd_rn(a[r].z, l.z); a[r].w = __fadd_rn(a[r].w, l.w);
-            }
+            a[r] = *reinterpret_cast<const float4 *>(A.hi + ab);
+            l[r] = A.lo ? *reinterpret_cast<const float4 *>(A.lo + ab) : make_float4(0.f, 0.f, 0.f, 0.f);
             if (Q > 0) {
                 const int64_t bb = cb.at(B);
 #pragma unroll
-                for (int q = 0; q < Q; ++q) b[r][q] = in ? B.hi[bb + q] : 0.f;
+                for (int q = 0; q < Q; ++q) b[r][q] = B.hi[bb + q];
                 cb.advance(B, rpp);
             }
             ca.advance(A, rpp);
         }
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
+            if (A.lo) {
+                a[r].x = __fadd_rn(a[r].x, l[r].x); a[r].y = __fadd_rn(a[r].y, l[r].y);
+                a[r].z = __fadd_rn(a[r].z, l[r].z); a[r].w = __fadd_rn(a[r].w, l[r].w);
+            }
             acc.x = __fadd_rn(acc.x, a[r].x); acc.y = __fadd_rn(acc.y, a[r].y);
             acc.z = __fadd_rn(acc.z, a[r].z); acc.w = __fadd_rn(acc.w, a[r].w);
 #pragma unroll
@@ -262,6 +263,22 @@ colsum_kernel(Rows A, Rows B, int64_t M, int64_t chunk, float *__restrict__ psum
                 accw[q].z = __fmaf_rn(a[r].z, b[r][q], accw[q].z); accw[q].w = __fmaf_rn(a[r].w, b[r][q], accw[q].w);
             }
         }
+    }
+    for (; m < last; m += rpp) {                              // the rows that are left, one at a time
+        float4 x = load4(A, ca.at(A), 4 * c4);
+        acc.x = __fadd_rn(acc.x, x.x); acc.y = __fadd_rn(acc.y, x.y);
+        acc.z = __fadd_rn(acc.z, x.z); acc.w = __fadd_rn(acc.w, x.w);
+        if (Q > 0) {
+            const int64_t bb = cb.at(B);
+#pragma unroll
+            for (int q = 0; q < Q; ++q) {
+                const float bq = B.hi[bb + q];
+                accw[q].x = __fmaf_rn(x.x, bq, accw[q].x); accw[q].y = __fmaf_rn(x.y, bq, accw[q].y);
+                accw[q].z = __fmaf_rn(x.z, bq, accw[q].z); accw[q].w = __fmaf_rn(x.w, bq, accw[q].w);
+            }
+            cb.advance(B, rpp);
+        }
+        ca.advance(A, rpp);
     }
     red[0][threadIdx.x] = acc;
 #pragma unroll
