@@ -55,7 +55,9 @@ __device__ __forceinline__ int block_suffix_incl(int x, int *warp_tot)
     return x + add;
 }
 
-// Sum of x over threads with index < own (exclusive prefix sum); *total gets the CTA sum.
+// Sum of x over threads with index < own (exclusive prefix sum); *total gets the CTA sum.  warp_tot: one slot per
+// warp.  Every warp scans the warps' totals itself with shuffles: with each thread adding the totals up one by one
+// (32 of them in a CTA of 1024 threads) this function was most of what a finishing CTA executed per tile of data.
 template <typename T>
 __device__ __forceinline__ T block_prefix_excl(T x, T *warp_tot, T *total)
 {
@@ -68,15 +70,18 @@ __device__ __forceinline__ T block_prefix_excl(T x, T *warp_tot, T *total)
     }
     if (lane == 31) warp_tot[warp] = incl;
     __syncthreads();
-    T add = 0, tot = 0;
-    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
-        const T t = warp_tot[w];
-        if (w < warp) add += t;
-        tot += t;
+    const T t = lane < (int)(blockDim.x >> 5) ? warp_tot[lane] : T(0);
+    T s = t;                                      // inclusive scan of the warps' totals; lanes beyond them keep the CTA's sum
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const T y = __shfl_up_sync(kFull, s, d);
+        if (lane >= d) s += y;
     }
-    __syncthreads();
+    const T before = __shfl_sync(kFull, s - t, warp);
+    const T tot = __shfl_sync(kFull, s, 31);
+    __syncthreads();                              // warp_tot may be written again
     if (total) *total = tot;
-    return add + incl - x;
+    return before + incl - x;
 }
 
 // Ordered emission of one thread's selected entries.  gt_before / eq_before: entries of the

@@ -489,6 +489,7 @@ __device__ __forceinline__ void digit_scan(const unsigned *hist, int k, FinishSh
 struct ListVerdict {
     bool settled;    // the two-pass path found the bucket of the k-th key in this step
     bool lists;
+    bool too_high;   // the lists are complete but hold fewer than k entries: the predicted key was too high
     int m;           // candidates of the segment (valid when lists)
 };
 __device__ __forceinline__ ListVerdict list_verdict(const FastArgs &f, int row, int li, int upto, unsigned *before,
@@ -502,6 +503,7 @@ __device__ __forceinline__ ListVerdict list_verdict(const FastArgs &f, int row, 
     ListVerdict v;
     v.settled = f.seg_epoch[slot] == f.epoch;
     v.lists = v.settled ? (int64_t)f.seg_m[slot] <= cap : f.lbkey[slot] != 0;
+    v.too_high = false;
     v.m = 0;
     if (before) *before = 0;
     if (!v.lists) return v;
@@ -519,7 +521,8 @@ __device__ __forceinline__ ListVerdict list_verdict(const FastArgs &f, int row, 
         *before = total_front;
     }
     const int64_t m64 = total;
-    if (__syncthreads_or((int)over) || m64 > cap || (!v.settled && m64 < k)) v.lists = false;
+    if (__syncthreads_or((int)over) || m64 > cap) v.lists = false;
+    else if (!v.settled && m64 < k) v.lists = false, v.too_high = true;
     v.m = (int)m64;
     return v;
 }
@@ -791,6 +794,48 @@ __global__ void __launch_bounds__(kFinThreads) wide_emit_kernel(FastArgs f)
     }
 }
 
+// One read of a segment (len entries at seg, offset `off` in the row): the entries whose key is at least
+// `from`, compacted in index order into ckey/cidx, of which only the first `cap` are stored; returns how many
+// there are.  All THREADS threads of the CTA take part; ends with a barrier.  The next tile's loads are issued
+// before this tile's scan (two barriers) so that they overlap it.
+template <int THREADS>
+__device__ __forceinline__ int collect_from_data(const float *__restrict__ seg, int64_t off, int len, uint32_t from,
+                                                 int64_t cap, uint32_t *ckey, int32_t *cidx, unsigned *warp_u)
+{
+    constexpr int kTile = THREADS * kSelPerThread;
+    int done = 0;                                  // (a segment has fewer than 2^31 entries)
+    uint32_t next[kSelPerThread];
+    int next_valid = load_keys16(seg, 0, len, next);
+    for (int base = 0; base < len; base += kTile) {
+        uint32_t key[kSelPerThread];
+        const int valid = next_valid;
+#pragma unroll
+        for (int i = 0; i < kSelPerThread; ++i) key[i] = next[i];
+        if (base + kTile < len) next_valid = load_keys16(seg, base + kTile, len, next);
+        unsigned flags = 0;
+#pragma unroll
+        for (int i = 0; i < kSelPerThread; ++i)
+            if (i < valid && key[i] >= from) flags |= 1u << i;
+        unsigned total;
+        int at = done + (int)block_prefix_excl<unsigned>((unsigned)__popc(flags), warp_u, &total);
+        // a thread holds a candidate in one tile of three: a loop over the set bits instead of sixteen predicated stores
+        // (the read is bound by the instructions a lone CTA can issue, not by memory)
+        const int32_t first = (int32_t)off + base + (int)threadIdx.x * kSelPerThread;
+        while (flags) {
+            const int i = __ffs((int)flags) - 1;
+            flags &= flags - 1u;
+            if (at < cap) {           // (the key once more from the line this thread has just read: registers cannot be indexed)
+                ckey[at] = mag_key(__ldg(seg + base + (int)threadIdx.x * kSelPerThread + i));
+                cidx[at] = first + i;
+            }
+            ++at;
+        }
+        done += (int)total;
+    }
+    __syncthreads();
+    return done;
+}
+
 // The selection of one (segment, row) is completed by one CTA.  The first num_small CTAs of a
 // row each do one small segment outright.  For a large segment the CTA
 //  1. settles the bucket of the k-th key from the histogram the accumulation left, unless path
@@ -803,7 +848,7 @@ __global__ void __launch_bounds__(kFinThreads) wide_emit_kernel(FastArgs f)
 // CTA order: large segments longest first, then the small ones, then spare CTAs that clear the
 // dense update buffer (if the caller announced it) while the rest of the launch is busy.
 template <int THREADS>
-__global__ void __launch_bounds__(THREADS) finish_kernel(FastArgs f)
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) finish_kernel(FastArgs f)
 {
     __shared__ FinishShared sh;
     __shared__ SmallShared small_sh;
@@ -845,13 +890,14 @@ __global__ void __launch_bounds__(THREADS) finish_kernel(FastArgs f)
     if (grouped) {
         verdict.settled = f.seg_epoch[slot] == f.epoch;
         verdict.lists = false;
+        verdict.too_high = false;
         verdict.m = 0;
     } else {
         verdict = list_verdict(f, row, li, c0, nullptr, sh.warp_u);
     }
     const bool settled = verdict.settled, lists = verdict.lists;
     const int m = verdict.m;
-    int path;
+    int path, retried = 0;
     uint32_t d0 = 0, T;
     int k_rem = 0;
     if (lists) {
@@ -886,6 +932,31 @@ __global__ void __launch_bounds__(THREADS) finish_kernel(FastArgs f)
             d0 = f.prefix[slot];
             k_rem = f.k_rem[slot];
         } else {
+            if (verdict.too_high) {
+                // The predicted key was a little too high (the usual miss is a few per cent): one read of the
+                // segment with the key lowered by 12 % (a quarter lower already collects more than the compact
+                // arrays hold, so thickly do the residuals lie below the k-th key), then on as with lists.  Only
+                // if that still brings fewer than k entries, or more than the arrays hold, the full search below runs.
+                const uint32_t from = __float_as_uint(__uint_as_float(f.lbkey[slot]) * 0.88f);
+                uint32_t *ckey = f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
+                int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
+                const int got = collect_from_data<THREADS>(rowp + off, off, len, from, cap, ckey, cidx, sh.warp_u);
+                if (got >= k && got <= cap) {
+                    path = 4;
+                    retried = got;
+                    for (int b = threadIdx.x; b < kHistBins; b += THREADS) full_hist[b] = 0;
+                    __syncthreads();
+                    for (int i = threadIdx.x; i < retried; i += THREADS) atomicAdd(&full_hist[ckey[i] >> 20], 1u);
+                    __syncthreads();
+                    digit_scan<THREADS>(full_hist, k, sh);
+                    d0 = (uint32_t)sh.found[0];
+                    k_rem = sh.found[1];
+                    __syncthreads();
+                    CompactSource src{ckey, cidx, retried};
+                    T = finish_from<THREADS>(src, d0, k_rem, k, out, sh, f.errword);
+                    goto finished;
+                }
+            }
             path = 2;
             // first read of the segment: its complete leading-digit histogram
             for (int b = threadIdx.x; b < kHistBins; b += THREADS) full_hist[b] = 0;
@@ -909,29 +980,8 @@ __global__ void __launch_bounds__(THREADS) finish_kernel(FastArgs f)
                 const int mm = (int)at_or_above;
                 uint32_t *ckey = mm <= f.smem_keys ? s_key : f.comp_key + (int64_t)row * f.comp_total + f.comp_off[li];
                 int32_t *cidx = f.comp_idx + (int64_t)row * f.comp_total + f.comp_off[li];
-                int done = 0;
-                for (int base = 0; base < len; base += kTile) {
-                    uint32_t key[kSelPerThread];
-                    const int valid = load_keys16(rowp + off, base, len, key);
-                    unsigned flags = 0;
-#pragma unroll
-                    for (int i = 0; i < kSelPerThread; ++i)
-                        if (i < valid && (key[i] >> 20) >= d0) flags |= 1u << i;
-                    unsigned total;
-                    unsigned at = (unsigned)done + block_prefix_excl<unsigned>((unsigned)__popc(flags), sh.warp_u, &total);
-                    if (flags) {
-                        const int first = base + (int)threadIdx.x * kSelPerThread;
-#pragma unroll
-                        for (int i = 0; i < kSelPerThread; ++i)
-                            if (flags >> i & 1u) {
-                                ckey[at] = key[i];
-                                cidx[at++] = (int32_t)(off + first + i);
-                            }
-                    }
-                    done += (int)total;
-                }
+                const int done = collect_from_data<THREADS>(rowp + off, off, len, d0 << 20, cap, ckey, cidx, sh.warp_u);
                 if (threadIdx.x == 0 && done != mm) atomicExch(f.errword, 0x5E80);
-                __syncthreads();
                 CompactSource src{ckey, cidx, mm};
                 T = finish_from<THREADS>(src, d0, k_rem, k, out, sh, f.errword);
                 goto finished;
@@ -943,9 +993,9 @@ __global__ void __launch_bounds__(THREADS) finish_kernel(FastArgs f)
         }
     }
 finished:
-    if (threadIdx.x == 0) f.seg_m[slot] = lists ? m : len;
+    if (threadIdx.x == 0) f.seg_m[slot] = lists ? m : path == 4 ? retried : len;
     if (threadIdx.x == 0) {
-        store_prediction(f, slot, T, k, path == 2 && f.lbkey[slot] != 0);
+        store_prediction(f, slot, T, k, (path == 2 || path == 4) && f.lbkey[slot] != 0);
         f.seg_path[slot] = path;
     }
 }

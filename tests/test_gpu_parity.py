@@ -77,6 +77,29 @@ def test_prediction_survives_a_collapse_of_the_gradient_scale():
         compare_step(ora, gpu, g, g.cuda(), t % K, upd)
 
 
+def test_prediction_a_little_too_high():
+    # the k-th key drops by a tenth from one step to the next (the residual is wiped and the gradient
+    # scaled by 0.9): fewer than k entries pass the predicted key, and the layers are finished from one read
+    # of the data with a lowered key; a drop by a third (last but one step) is beyond that and takes the full search
+    numel = [300000, 3000, 70000]
+    K = 2
+    ora, gpu = make_pair(numel, K, momentum=0.0, density_ppm=5000)
+    src = toy_source(numel, K)
+    upd = torch.empty(gpu.N, dtype=torch.float32, device="cuda")
+    from_data = []
+    for t, scale in enumerate([1.0, 1.0, 0.9, 0.9, 0.8, 0.8, 0.55, 1.0]):
+        g = src.step(t % 2) * scale
+        gpu.v.zero_(); gpu.u.zero_(); ora.v[:] = 0; ora.u[:] = 0
+        compare_step(ora, gpu, g, g.cuda(), t % K, upd)
+        stats = gpu.selection_stats()
+        from_data.append(stats[4])
+        if t in (2, 4):
+            assert stats[3] < numel[0], stats         # a handful of candidates, not the whole layer
+        if t == 6:
+            assert stats[3] == numel[0], stats
+    assert from_data[2] == 2 and from_data[4] == 2 and from_data[6] == 2, from_data
+
+
 def test_ragged_layers_parameter_server():
     ora, gpu = run_steps(TOY, 3, 3, variant="ps")
     assert gpu.idx.shape == (3, gpu.mu)
