@@ -40,24 +40,28 @@ CLOCK_WINDOW_MS = 500.0  # the clock sampler watches at least this long a run of
 # figure is not reported ("traffic": null): the kernel has changed since.
 NCU_CAPTURE = {
     "kernel": "accumulate_select_kernel",
-    "source": os.path.join("paper_2103_08870_b200", "csrc", "lgc_select_fast.cu"),
-    "source_sha256": "fbc1bc687e794e8d50c58a020ac1e2804137ac502545f5062a5e97dc3e2d808c",
-    "dram_bytes_per_element": 19.01,
+    # the kernel's source and the headers it is built from; the digest is over their bytes, in this order
+    "sources": [os.path.join("paper_2103_08870_b200", "csrc", n)
+                for n in ("lgc_select_fast.cu", "lgc_select_common.cuh", "lgc_internal.cuh")],
+    "sources_sha256": "b69902d76f2fd6131a0db8f10cc71c72a701966ef12c153c45160918cc96aeb6",
+    "dram_bytes_per_element": 19.00,
 }
 
 
 def ncu_traffic_bytes(elements: int):
     """DRAM traffic of one launch over `elements` elements from the stored capture, or None when the
-    kernel's source is no longer the one that was measured."""
+    kernel's sources are no longer the ones that were measured."""
     import hashlib
-    if not NCU_CAPTURE["source_sha256"] or NCU_CAPTURE["dram_bytes_per_element"] is None:
+    if not NCU_CAPTURE["sources_sha256"] or NCU_CAPTURE["dram_bytes_per_element"] is None:
         return None
+    h = hashlib.sha256()
     try:
-        with open(os.path.join(ROOT, NCU_CAPTURE["source"]), "rb") as f:
-            now = hashlib.sha256(f.read()).hexdigest()
+        for name in NCU_CAPTURE["sources"]:
+            with open(os.path.join(ROOT, name), "rb") as f:
+                h.update(f.read())
     except OSError:
         return None
-    return NCU_CAPTURE["dram_bytes_per_element"] * elements if now == NCU_CAPTURE["source_sha256"] else None
+    return NCU_CAPTURE["dram_bytes_per_element"] * elements if h.hexdigest() == NCU_CAPTURE["sources_sha256"] else None
 
 
 def measured_peak():

@@ -1077,13 +1077,17 @@ accumulate_select_kernel(FastArgs f, const float *__restrict__ g, int64_t g_stri
                                                 // w: 0 no dense element, > 0 one dense run (packed), < 0 several
     uint32_t lbkey1 = 0;
     if (selecting || DENSE) desc = __ldg(f.tile_desc + q);      // consumed after the stream's loads are on their way
-    if (selecting && desc.y >= 0) lbkey1 = f.lbkey[(int64_t)sel * f.num_large + desc.y];
-    float4 vv = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 vv = make_float4(0.f, 0.f, 0.f, 0.f), gg = vv, uu = vv;
+    const int64_t e = ((int64_t)row * N + tile_base + p0) >> 2;
     if (live) {
-        const int64_t e = ((int64_t)row * N + tile_base + p0) >> 2;
-        float4 gg = __ldcs(reinterpret_cast<const float4 *>(g) + (((int64_t)row * g_stride + tile_base + p0) >> 2));
-        float4 uu = __ldcs(reinterpret_cast<float4 *>(u) + e);
+        gg = __ldcs(reinterpret_cast<const float4 *>(g) + (((int64_t)row * g_stride + tile_base + p0) >> 2));
+        uu = __ldcs(reinterpret_cast<float4 *>(u) + e);
         vv = __ldcs(reinterpret_cast<float4 *>(v) + e);
+    }
+    // (only now the description is looked at: the predicted key's address depends on it, and a warp that waits for the
+    // description before it has issued its three loads starts its stream a memory latency late)
+    if (selecting && desc.y >= 0) lbkey1 = f.lbkey[(int64_t)sel * f.num_large + desc.y];
+    if (live) {
         // Dense elements among these four take no gradient: their u and v are zero from lgc_init on and stay
         // exactly zero (m * 0 + 0 = 0, 0 + 0 = 0), which is "no state" for the layers sent as they are.
         if (DENSE && desc.w > 0) {                  // one dense run [lo, hi) inside the tile
