@@ -43,8 +43,8 @@ NCU_CAPTURE = {
     # the kernel's source and the headers it is built from; the digest is over their bytes, in this order
     "sources": [os.path.join("paper_2103_08870_b200", "csrc", n)
                 for n in ("lgc_select_fast.cu", "lgc_select_common.cuh", "lgc_internal.cuh")],
-    "sources_sha256": "b69902d76f2fd6131a0db8f10cc71c72a701966ef12c153c45160918cc96aeb6",
-    "dram_bytes_per_element": 19.00,
+    "sources_sha256": "0e3a7186a36d74f3181d4f637b6ea77c44f9669739b802759f19065fc33650a3",
+    "dram_bytes_per_element": 19.02,
 }
 
 
