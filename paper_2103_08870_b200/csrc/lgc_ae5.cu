@@ -11,8 +11,11 @@
 // run on the tensor cores (tcgen05.mma kind::tf32, operands staged by TMA into 128-byte-swizzled
 // shared memory, accumulator in tensor memory).  fp32 accuracy is kept by splitting every
 // operand into two tf32 numbers, x = hi + lo, and accumulating hi*hi + hi*lo + lo*hi.
-// The first convolution (one input channel), the 1x1 convolutions and the decoder (which runs
-// once, not once per node) use the ordinary fp32 pipes.
+// The first convolution (one input channel), the 1x1 convolutions and the two narrow decoder layers use the
+// ordinary fp32 pipes; the decoder's three wide transposed convolutions are GEMMs of the same kernel.
+// For training, the same kernel makes the gradients at the inputs of conv2..conv4 (a transposed convolution of
+// the output's gradient), and ae5_wgrad_kernel their weight gradients (a GEMM that sums over rows, both operands
+// read along their rows).
 #include <algorithm>
 
 #include "lgc_internal.cuh"
